@@ -1,0 +1,175 @@
+/*
+ * dynakv.h -- C ABI of libdynakv: cluster-based KV-cache retrieval with migration-free
+ * cluster adaptation (arXiv 2511.07427, "DynaKV"), with the whole index and KV store
+ * resident in the HBM of one sm_100a GPU.
+ *
+ * Vocabulary (paper, Section 4.1).  A *unit* is one KV head of one layer of one
+ * sequence: the cache K_t that the paper partitions into M_t disjoint clusters
+ * (Eq. 1-3), each with a representative r_j = mean of its members (Eq. 4).  Every call
+ * below works on all U units of a context at once; units never interact.
+ * G = query heads sharing one KV head, d = head dimension, n = tokens in a unit.
+ *
+ * Pointers.  Unless a parameter says "host", data pointers are DEVICE pointers owned by
+ * the caller; the library reads or writes them on the context's stream and never frees
+ * them.  Everything else (cluster arenas, tables, scratch) is owned by the context and
+ * released by dynakv_destroy().  Calls enqueue work on the context's stream and return
+ * without synchronising unless stated.
+ *
+ * Errors.  Host-detectable problems (NULL pointer, size mismatch, wrong call order)
+ * return a negative code and enqueue nothing.  Conditions only the device can see
+ * (budget smaller than the best cluster, cluster-id or token capacity reached, page pool
+ * exhausted) never trap: the kernel skips the step it cannot do, sets a sticky bit in a
+ * device status word, and dynakv_get_status() reports it.
+ */
+#ifndef DYNAKV_H_
+#define DYNAKV_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define DYNAKV_F32 0
+#define DYNAKV_BF16 1
+
+#define DYNAKV_INIT_KMEANSPP 0
+#define DYNAKV_INIT_RANDOM 1
+
+#define DYNAKV_OK 0
+#define DYNAKV_ERR_ARG (-1)     /* NULL pointer or value out of range            */
+#define DYNAKV_ERR_STATE (-2)   /* call order: e.g. decode before build_index    */
+#define DYNAKV_ERR_CUDA (-3)    /* a CUDA runtime call failed                    */
+#define DYNAKV_ERR_NOMEM (-4)   /* device allocation failed                      */
+
+/* sticky device status bits */
+#define DYNAKV_ST_BUDGET_EXCEEDED 1u  /* best cluster alone larger than the budget; taken whole */
+#define DYNAKV_ST_MAX_CLUSTERS 2u     /* a split was skipped: max_clusters ids in use            */
+#define DYNAKV_ST_MAX_TOKENS 4u       /* an append was dropped: unit holds max_tokens            */
+#define DYNAKV_ST_PAGE_POOL 8u        /* a split or append was skipped: no free page             */
+#define DYNAKV_ST_INTERNAL 16u        /* an internal bound was hit (bounded wait ran out, ...)   */
+
+typedef struct dynakv_ctx dynakv_ctx;
+
+typedef struct dynakv_config {
+    int32_t n_units;           /* U = sequences x layers x KV heads                              */
+    int32_t gqa_group;         /* G, 1..8                                                        */
+    int32_t head_dim;          /* d: 64 or 128                                                   */
+    int32_t kv_dtype;          /* DYNAKV_F32 or DYNAKV_BF16 for K, V; q, out, centroids are fp32 */
+    int32_t max_tokens;        /* capacity per unit (prefill + decode)                           */
+    int32_t max_clusters;      /* cluster ids per unit, <= 4096                                  */
+    int32_t kmeans_iters;      /* T: Lloyd rounds at build time (all are run, no early exit)     */
+    int32_t init_mode;         /* DYNAKV_INIT_KMEANSPP or DYNAKV_INIT_RANDOM                     */
+    float split_size_factor;   /* gamma: split when n_j * M_live > gamma * N; <= 0 disables      */
+    float split_var_factor;    /* alpha: tau = alpha * mean live sigma_j^2 at build; <= 0 disables */
+    int32_t split_min_size;    /* clusters smaller than this are never split                     */
+    int32_t split_iters;       /* cap on 2-means rounds in a split                               */
+    int32_t trace;             /* 1: keep every Lloyd round's assignment for dynakv_get_build_trace */
+    int32_t assign_mode;       /* 0: auto (tensor-core distance GEMM for bf16, d=128), 1: force fp32 path */
+} dynakv_config;
+
+typedef struct dynakv_status {
+    uint32_t error_bits;       /* OR of DYNAKV_ST_*                                              */
+    int32_t reserved;
+    int64_t n_appended;        /* appends stored, summed over units                              */
+    int64_t n_splits;          /* splits performed, summed over units                            */
+    int64_t tokens_selected;   /* tokens attended in the last decode step, summed over units     */
+    int64_t clusters_selected; /* clusters selected in the last decode step, summed over units   */
+    int64_t pages_in_use;      /* 32-token pages holding data, summed over units                 */
+    int64_t assign_rechecked;  /* keys whose tensor-core argmin was re-decided in fp32 (build)   */
+} dynakv_status;
+
+/* Create a context on the current CUDA device; all later work runs on `cuda_stream`
+ * (a cudaStream_t passed as void*, NULL = the legacy default stream).  Allocates the
+ * arenas: about max_tokens * 4 * d * sizeof(kv) bytes per unit plus tables. */
+int dynakv_create(const dynakv_config* cfg, void* cuda_stream, dynakv_ctx** out);
+
+/* Prefill: NewCluster of Algorithm 1 / the k-means partition of Section 4.1 (Eq. 3) with
+ * centroid representatives (Eq. 4).  K, V: [U][n][d] row-major in cfg.kv_dtype.
+ * Seeded init (k-means++ by exponential race, or the n_clusters keys with the smallest
+ * counter-based uniforms), then cfg.kmeans_iters rounds of nearest-centre assignment
+ * (squared Euclidean, ties to the lowest id) and mean update (an empty cluster keeps its
+ * centre).  Then the members of each cluster are stored contiguously in 32-token pages
+ * (Section 5.1, intra-cluster placement), n_j, r_j and M2_j = sum ||k - r_j||^2 are
+ * initialised (Algorithm 1, "Initialize cluster size, centroid, variance") and the unit's
+ * variance threshold tau is set.  Token id = row index.  Requires
+ * n_clusters <= n <= max_tokens, n_clusters <= max_clusters, d == head_dim.
+ * May be called once per context. */
+int dynakv_build_index(dynakv_ctx* ctx, const void* K, const void* V, int64_t n, int32_t d,
+                       int32_t n_clusters, uint64_t seed);
+
+/* Algorithm 1, "Assign new KV entry to its nearest cluster", UpdateVar, AddEntry,
+ * UpdateStats: for every unit, the new key k [U][d] joins the live cluster with the
+ * nearest representative; n_j, r_j, M2_j are updated incrementally and the (k, v) row is
+ * written into the tail page of that cluster (no existing entry moves).  The new token id
+ * is the unit's token count before the call. */
+int dynakv_append(dynakv_ctx* ctx, const void* k, const void* v);
+
+/* Section 4.1 / Algorithm 1 "Load top-k clusters by query-centroid similarity", then
+ * attention over the retrieved entries only (Section 2.1).  q: [U][G][d] fp32.
+ * score_j = mean over the G heads of q_g . r_j; clusters are taken in (score descending,
+ * id ascending) order while their sizes sum to <= token_budget (the best cluster is taken
+ * whole if it alone is larger, with DYNAKV_ST_BUDGET_EXCEEDED).  out: [U][G][d] fp32 =
+ * softmax(q_g . k_i / sqrt(d)) v_i over the members of the selected clusters; zeros when
+ * nothing is selected.  selected_ids: [U][max_clusters] int32, selection in score order,
+ * -1 padded; may be NULL. */
+int dynakv_decode_step(dynakv_ctx* ctx, const float* q, int32_t token_budget, float* out,
+                       int32_t* selected_ids);
+
+/* Algorithm 1's split decision and SplitCluster (Section 4.2, 5.2).  A live cluster with
+ * n_j >= split_min_size splits when sigma_j^2 = M2_j / n_j > tau (variance rule) or
+ * n_j * M_live > gamma * N (size rule), triggers evaluated on the state at entry, each
+ * triggered cluster once, in ascending id.  2-means over its members: centre A = member
+ * farthest from r_j, B = member farthest from A, up to split_iters rounds, ties to A.
+ * The child holding the smallest token id keeps the id and its pages, compacted in place;
+ * the other child moves to fresh pages under the next free id.  A split that leaves a
+ * side empty is abandoned and not retried until the cluster's next append. */
+int dynakv_split_check(dynakv_ctx* ctx);
+
+/* n_steps iterations of { decode_step(q_t); append(k_t, v_t); split_check() } (the order
+ * of Algorithm 1's loop body), replayed from one captured CUDA graph whose kernels read
+ * the step index from device memory.  q_steps: [n_steps][U][G][d] fp32, k_steps,
+ * v_steps: [n_steps][U][d] kv_dtype, out_steps: [n_steps][U][G][d] fp32, all device. */
+int dynakv_decode_loop(dynakv_ctx* ctx, const float* q_steps, const void* k_steps,
+                       const void* v_steps, int64_t n_steps, int32_t token_budget,
+                       float* out_steps);
+
+/* One loop iteration as above with HOST buffers (pinned memory recommended): copies
+ * q, k, v to the device, runs the three calls, copies out back and synchronises the
+ * stream.  q_host [U][G][d] fp32, k_host, v_host [U][d] kv_dtype, out_host [U][G][d]. */
+int dynakv_step_host(dynakv_ctx* ctx, const float* q_host, const void* k_host,
+                     const void* v_host, int32_t token_budget, float* out_host);
+
+/* Synchronises the stream and fills *host_out (host memory). */
+int dynakv_get_status(dynakv_ctx* ctx, dynakv_status* host_out);
+
+/* Synchronises and copies the index state to HOST arrays; any pointer may be NULL.
+ *   tok_cluster [U][max_tokens] int32  cluster id of each token id (-1 beyond n)
+ *   centroids   [U][max_clusters][d] fp32
+ *   counts      [U][max_clusters] int32 (0 = dead or unused id)
+ *   M2          [U][max_clusters] fp32
+ *   n_tokens    [U] int32,  n_ids [U] int32 (ids handed out),  tau [U] fp32 */
+int dynakv_export_state(dynakv_ctx* ctx, int32_t* tok_cluster, float* centroids, int32_t* counts,
+                        float* M2, int32_t* n_tokens, int32_t* n_ids, float* tau);
+
+/* Synchronises and copies the last decode step's selection sizes to HOST arrays:
+ * n_selected [U], tokens_selected [U]; either may be NULL. */
+int dynakv_get_selection(dynakv_ctx* ctx, int32_t* n_selected, int32_t* tokens_selected);
+
+/* With cfg.trace = 1: HOST arrays picks [U][n_clusters] (token ids chosen as initial
+ * centres, in centre order) and assign [T][U][n] (assignment of every Lloyd round);
+ * either may be NULL.  Returns DYNAKV_ERR_STATE if tracing was off. */
+int dynakv_get_build_trace(dynakv_ctx* ctx, int32_t* picks, int32_t* assign);
+
+/* Number of kernels this context has launched so far (graph replays count their nodes). */
+int64_t dynakv_launch_count(dynakv_ctx* ctx);
+
+/* Text of the last CUDA error seen by this library on the calling thread ("" if none). */
+const char* dynakv_last_error(void);
+
+void dynakv_destroy(dynakv_ctx* ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DYNAKV_H_ */

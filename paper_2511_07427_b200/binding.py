@@ -1,0 +1,247 @@
+"""ctypes binding of libdynakv.so: argument marshalling only, same names as the C ABI."""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from dataclasses import dataclass
+from typing import Optional
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_LIB_PATH = os.path.join(_HERE, "libdynakv.so")
+
+F32, BF16 = 0, 1
+INIT_KMEANSPP, INIT_RANDOM = 0, 1
+ST_BUDGET_EXCEEDED, ST_MAX_CLUSTERS, ST_MAX_TOKENS, ST_PAGE_POOL, ST_INTERNAL = 1, 2, 4, 8, 16
+
+EXPORTED_SYMBOLS = [
+    "dynakv_create", "dynakv_build_index", "dynakv_append", "dynakv_decode_step", "dynakv_split_check",
+    "dynakv_decode_loop", "dynakv_step_host", "dynakv_get_status", "dynakv_export_state", "dynakv_get_selection",
+    "dynakv_get_build_trace", "dynakv_launch_count", "dynakv_last_error", "dynakv_destroy",
+]
+
+
+class DynaKVError(RuntimeError):
+    pass
+
+
+class _Config(C.Structure):
+    _fields_ = [("n_units", C.c_int32), ("gqa_group", C.c_int32), ("head_dim", C.c_int32), ("kv_dtype", C.c_int32),
+                ("max_tokens", C.c_int32), ("max_clusters", C.c_int32), ("kmeans_iters", C.c_int32),
+                ("init_mode", C.c_int32), ("split_size_factor", C.c_float), ("split_var_factor", C.c_float),
+                ("split_min_size", C.c_int32), ("split_iters", C.c_int32), ("trace", C.c_int32),
+                ("assign_mode", C.c_int32)]
+
+
+class _Status(C.Structure):
+    _fields_ = [("error_bits", C.c_uint32), ("reserved", C.c_int32), ("n_appended", C.c_int64),
+                ("n_splits", C.c_int64), ("tokens_selected", C.c_int64), ("clusters_selected", C.c_int64),
+                ("pages_in_use", C.c_int64), ("assign_rechecked", C.c_int64)]
+
+
+@dataclass
+class DynaKVConfig:
+    n_units: int
+    gqa_group: int
+    head_dim: int
+    kv_dtype: int
+    max_tokens: int
+    max_clusters: int
+    kmeans_iters: int = 10
+    init_mode: int = INIT_KMEANSPP
+    split_size_factor: float = 2.0
+    split_var_factor: float = 2.0
+    split_min_size: int = 8
+    split_iters: int = 8
+    trace: int = 0
+    assign_mode: int = 0
+
+
+_lib = None
+
+
+def load_library() -> C.CDLL:
+    """Load libdynakv.so from the package directory; raise if it has not been built."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(_LIB_PATH):
+        raise DynaKVError(f"{_LIB_PATH} is missing: build it with `python -m paper_2511_07427_b200.build` "
+                          "(there is no CPU fallback)")
+    L = C.CDLL(_LIB_PATH)
+    vp, i32, i64, u64 = C.c_void_p, C.c_int32, C.c_int64, C.c_uint64
+    L.dynakv_create.restype = C.c_int
+    L.dynakv_create.argtypes = [C.POINTER(_Config), vp, C.POINTER(vp)]
+    L.dynakv_build_index.restype = C.c_int
+    L.dynakv_build_index.argtypes = [vp, vp, vp, i64, i32, i32, u64]
+    L.dynakv_append.restype = C.c_int
+    L.dynakv_append.argtypes = [vp, vp, vp]
+    L.dynakv_decode_step.restype = C.c_int
+    L.dynakv_decode_step.argtypes = [vp, vp, i32, vp, vp]
+    L.dynakv_split_check.restype = C.c_int
+    L.dynakv_split_check.argtypes = [vp]
+    L.dynakv_decode_loop.restype = C.c_int
+    L.dynakv_decode_loop.argtypes = [vp, vp, vp, vp, i64, i32, vp]
+    L.dynakv_step_host.restype = C.c_int
+    L.dynakv_step_host.argtypes = [vp, vp, vp, vp, i32, vp]
+    L.dynakv_get_status.restype = C.c_int
+    L.dynakv_get_status.argtypes = [vp, C.POINTER(_Status)]
+    L.dynakv_export_state.restype = C.c_int
+    L.dynakv_export_state.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp]
+    L.dynakv_get_selection.restype = C.c_int
+    L.dynakv_get_selection.argtypes = [vp, vp, vp]
+    L.dynakv_get_build_trace.restype = C.c_int
+    L.dynakv_get_build_trace.argtypes = [vp, vp, vp]
+    L.dynakv_launch_count.restype = C.c_int64
+    L.dynakv_launch_count.argtypes = [vp]
+    L.dynakv_last_error.restype = C.c_char_p
+    L.dynakv_last_error.argtypes = []
+    L.dynakv_destroy.restype = None
+    L.dynakv_destroy.argtypes = [vp]
+    _lib = L
+    return L
+
+
+def _np_ptr(a: Optional[np.ndarray]):
+    return a.ctypes.data_as(C.c_void_p) if a is not None else None
+
+
+class DynaKV:
+    """One context: U independent KV heads with their cluster index and paged KV store in HBM.
+
+    Methods mirror the C entry points (``build_index``, ``append``, ``decode_step``,
+    ``split_check``, ``decode_loop``, ``step_host``) and take ``torch`` CUDA tensors (or
+    pinned host tensors for ``step_host``).  Work is enqueued on the stream that was current
+    when the context was created."""
+
+    def __init__(self, cfg: DynaKVConfig, stream=None):
+        import torch
+        if not torch.cuda.is_available():
+            raise DynaKVError("no CUDA device: libdynakv has no CPU fallback")
+        self._L = load_library()
+        self.cfg = cfg
+        self._torch = torch
+        self._stream = stream if stream is not None else torch.cuda.current_stream()
+        c = _Config(cfg.n_units, cfg.gqa_group, cfg.head_dim, cfg.kv_dtype, cfg.max_tokens, cfg.max_clusters,
+                    cfg.kmeans_iters, cfg.init_mode, cfg.split_size_factor, cfg.split_var_factor,
+                    cfg.split_min_size, cfg.split_iters, cfg.trace, cfg.assign_mode)
+        h = C.c_void_p()
+        self._check(self._L.dynakv_create(C.byref(c), C.c_void_p(self._stream.cuda_stream), C.byref(h)), "dynakv_create")
+        self._h = h
+        self.n_prefill = 0
+        self.n_clusters0 = 0
+        self._keep = []
+
+    # ---- helpers
+    def _check(self, rc: int, what: str) -> None:
+        if rc != 0:
+            msg = self._L.dynakv_last_error().decode()
+            raise DynaKVError(f"{what} returned {rc} {msg}")
+
+    def _kv(self, t, shape):
+        torch = self._torch
+        want = torch.float32 if self.cfg.kv_dtype == F32 else torch.bfloat16
+        if t.dtype != want or not t.is_contiguous() or tuple(t.shape) != tuple(shape):
+            raise DynaKVError(f"expected contiguous {want} tensor of shape {tuple(shape)}, got {t.dtype} {tuple(t.shape)}")
+        return C.c_void_p(t.data_ptr())
+
+    def _f32(self, t, shape):
+        torch = self._torch
+        if t.dtype != torch.float32 or not t.is_contiguous() or tuple(t.shape) != tuple(shape):
+            raise DynaKVError(f"expected contiguous float32 tensor of shape {tuple(shape)}, got {t.dtype} {tuple(t.shape)}")
+        return C.c_void_p(t.data_ptr())
+
+    # ---- the C ABI, one method per entry point
+    def build_index(self, K, V, n_clusters: int, seed: int) -> None:
+        U, d = self.cfg.n_units, self.cfg.head_dim
+        n = K.shape[1]
+        assert K.is_cuda and V.is_cuda
+        self._check(self._L.dynakv_build_index(self._h, self._kv(K, (U, n, d)), self._kv(V, (U, n, d)), n, d,
+                                               n_clusters, seed), "dynakv_build_index")
+        self.n_prefill, self.n_clusters0 = n, n_clusters
+
+    def append(self, k, v) -> None:
+        U, d = self.cfg.n_units, self.cfg.head_dim
+        assert k.is_cuda and v.is_cuda
+        self._check(self._L.dynakv_append(self._h, self._kv(k, (U, d)), self._kv(v, (U, d))), "dynakv_append")
+
+    def decode_step(self, q, token_budget: int, out=None, selected_ids=None):
+        torch = self._torch
+        U, G, d = self.cfg.n_units, self.cfg.gqa_group, self.cfg.head_dim
+        assert q.is_cuda
+        if out is None:
+            out = torch.empty((U, G, d), dtype=torch.float32, device=q.device)
+        sp = None
+        if selected_ids is not None:
+            assert selected_ids.dtype == torch.int32 and selected_ids.is_contiguous() and \
+                tuple(selected_ids.shape) == (U, self.cfg.max_clusters)
+            sp = C.c_void_p(selected_ids.data_ptr())
+        self._check(self._L.dynakv_decode_step(self._h, self._f32(q, (U, G, d)), token_budget,
+                                               self._f32(out, (U, G, d)), sp), "dynakv_decode_step")
+        return out
+
+    def split_check(self) -> None:
+        self._check(self._L.dynakv_split_check(self._h), "dynakv_split_check")
+
+    def decode_loop(self, q_steps, k_steps, v_steps, token_budget: int, out_steps=None):
+        torch = self._torch
+        U, G, d = self.cfg.n_units, self.cfg.gqa_group, self.cfg.head_dim
+        n = q_steps.shape[0]
+        if out_steps is None:
+            out_steps = torch.empty((n, U, G, d), dtype=torch.float32, device=q_steps.device)
+        self._check(self._L.dynakv_decode_loop(self._h, self._f32(q_steps, (n, U, G, d)), self._kv(k_steps, (n, U, d)),
+                                               self._kv(v_steps, (n, U, d)), n, token_budget,
+                                               self._f32(out_steps, (n, U, G, d))), "dynakv_decode_loop")
+        self._keep = [q_steps, k_steps, v_steps, out_steps]
+        return out_steps
+
+    def step_host(self, q_host, k_host, v_host, token_budget: int, out_host) -> None:
+        U, G, d = self.cfg.n_units, self.cfg.gqa_group, self.cfg.head_dim
+        assert not q_host.is_cuda and not out_host.is_cuda
+        self._check(self._L.dynakv_step_host(self._h, self._f32(q_host, (U, G, d)), self._kv(k_host, (U, d)),
+                                             self._kv(v_host, (U, d)), token_budget, self._f32(out_host, (U, G, d))),
+                    "dynakv_step_host")
+
+    def get_status(self) -> dict:
+        s = _Status()
+        self._check(self._L.dynakv_get_status(self._h, C.byref(s)), "dynakv_get_status")
+        return {k: getattr(s, k) for k, _ in _Status._fields_ if k != "reserved"}
+
+    def export_state(self) -> dict:
+        U, Mx, d, nt = self.cfg.n_units, self.cfg.max_clusters, self.cfg.head_dim, self.cfg.max_tokens
+        out = {
+            "tok_cluster": np.empty((U, nt), np.int32), "centroids": np.empty((U, Mx, d), np.float32),
+            "counts": np.empty((U, Mx), np.int32), "M2": np.empty((U, Mx), np.float32),
+            "n_tokens": np.empty(U, np.int32), "n_ids": np.empty(U, np.int32), "tau": np.empty(U, np.float32),
+        }
+        self._check(self._L.dynakv_export_state(self._h, *[_np_ptr(out[k]) for k in
+                    ("tok_cluster", "centroids", "counts", "M2", "n_tokens", "n_ids", "tau")]), "dynakv_export_state")
+        return out
+
+    def get_selection(self):
+        U = self.cfg.n_units
+        a, b = np.empty(U, np.int32), np.empty(U, np.int32)
+        self._check(self._L.dynakv_get_selection(self._h, _np_ptr(a), _np_ptr(b)), "dynakv_get_selection")
+        return a, b
+
+    def get_build_trace(self):
+        U, T = self.cfg.n_units, self.cfg.kmeans_iters
+        picks = np.empty((U, self.n_clusters0), np.int32)
+        assign = np.empty((T, U, self.n_prefill), np.int32)
+        self._check(self._L.dynakv_get_build_trace(self._h, _np_ptr(picks), _np_ptr(assign)), "dynakv_get_build_trace")
+        return picks, assign
+
+    def launch_count(self) -> int:
+        return int(self._L.dynakv_launch_count(self._h))
+
+    def destroy(self) -> None:
+        if getattr(self, "_h", None):
+            self._L.dynakv_destroy(self._h)
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.destroy()
+        except Exception:
+            pass

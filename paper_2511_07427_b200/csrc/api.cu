@@ -1,0 +1,363 @@
+// C ABI of libdynakv: context management, argument checks, and the call sequences that
+// string the kernels together.  No arithmetic of the method lives here.
+#include <stdio.h>
+#include <string.h>
+
+#include <new>
+#include <vector>
+
+#include "common.cuh"
+
+using namespace dkv;
+
+namespace dkv {
+// tensor-core distance GEMM path (assign_tc.cu)
+bool tc_assign_supported(const Tables& t, long long n, int M);
+size_t tc_assign_scratch_bytes(const Tables& t, long long n, int M);
+void launch_assign_tc(const Tables& t, const void* K, long long n, int M, const float* C, int* assign, void* scratch,
+                      cudaStream_t s, long long* launches);
+}  // namespace dkv
+
+static thread_local char g_err[256] = "";
+
+struct dynakv_ctx {
+    dynakv_config cfg;
+    cudaStream_t stream;
+    Tables t;
+    std::vector<void*> allocs;
+    bool built = false;
+    long long n_prefill = 0;
+    int M0 = 0;
+    long long launches = 0;
+    // build trace
+    int* trace_assign = nullptr;   // [T][U][n]
+    int* trace_picks = nullptr;    // [U][M0]
+    // graph loop
+    int* step_ctr = nullptr;
+    cudaGraphExec_t graph_exec = nullptr;
+    const void* g_q = nullptr; const void* g_k = nullptr; const void* g_v = nullptr; void* g_out = nullptr;
+    int g_budget = -1;
+    long long graph_nodes = 0;
+    // staging for dynakv_step_host
+    float* st_q = nullptr; void* st_k = nullptr; void* st_v = nullptr; float* st_out = nullptr;
+};
+
+#define CK(call)                                                                                   \
+    do {                                                                                           \
+        cudaError_t e_ = (call);                                                                   \
+        if (e_ != cudaSuccess) {                                                                   \
+            snprintf(g_err, sizeof(g_err), "%s failed: %s (%s:%d)", #call, cudaGetErrorString(e_), __FILE__, __LINE__); \
+            return DYNAKV_ERR_CUDA;                                                                \
+        }                                                                                          \
+    } while (0)
+
+template <typename T>
+static int dev_alloc(dynakv_ctx* c, T** p, size_t count, bool zero = false) {
+    void* q = nullptr;
+    size_t bytes = sizeof(T) * (count ? count : 1);
+    cudaError_t e = cudaMalloc(&q, bytes);
+    if (e != cudaSuccess) {
+        snprintf(g_err, sizeof(g_err), "cudaMalloc of %zu bytes failed: %s", bytes, cudaGetErrorString(e));
+        cudaGetLastError();
+        return DYNAKV_ERR_NOMEM;
+    }
+    c->allocs.push_back(q);
+    if (zero) cudaMemsetAsync(q, 0, bytes, c->stream);
+    *p = reinterpret_cast<T*>(q);
+    return DYNAKV_OK;
+}
+
+#define ALLOC(ptr, count, zero)                                    \
+    do {                                                           \
+        int rc_ = dev_alloc(c, &(ptr), (size_t)(count), zero);     \
+        if (rc_ != DYNAKV_OK) { dynakv_destroy(c); return rc_; }   \
+    } while (0)
+
+// inside build_index a failed allocation must not tear the caller's context down
+#define ALLOC_B(ptr, count, zero)                                  \
+    do {                                                           \
+        int rc_ = dev_alloc(c, &(ptr), (size_t)(count), zero);     \
+        if (rc_ != DYNAKV_OK) return rc_;                          \
+    } while (0)
+
+static size_t kv_bytes(const dynakv_config& cfg) { return cfg.kv_dtype == DYNAKV_F32 ? 4 : 2; }
+
+extern "C" const char* dynakv_last_error(void) { return g_err; }
+
+extern "C" int dynakv_create(const dynakv_config* cfg, void* cuda_stream, dynakv_ctx** out) {
+    if (!cfg || !out) return DYNAKV_ERR_ARG;
+    *out = nullptr;
+    if (cfg->n_units < 1 || cfg->gqa_group < 1 || cfg->gqa_group > MAX_G) return DYNAKV_ERR_ARG;
+    if (cfg->head_dim != 64 && cfg->head_dim != 128) return DYNAKV_ERR_ARG;
+    if (cfg->kv_dtype != DYNAKV_F32 && cfg->kv_dtype != DYNAKV_BF16) return DYNAKV_ERR_ARG;
+    if (cfg->max_tokens < 1 || cfg->max_clusters < 1 || cfg->max_clusters > 4096) return DYNAKV_ERR_ARG;
+    if (cfg->kmeans_iters < 1 || cfg->split_iters < 1) return DYNAKV_ERR_ARG;
+    if (cfg->init_mode != DYNAKV_INIT_KMEANSPP && cfg->init_mode != DYNAKV_INIT_RANDOM) return DYNAKV_ERR_ARG;
+    dynakv_ctx* c = new (std::nothrow) dynakv_ctx();
+    if (!c) return DYNAKV_ERR_NOMEM;
+    c->cfg = *cfg;
+    c->stream = reinterpret_cast<cudaStream_t>(cuda_stream);
+    Tables& t = c->t;
+    memset(&t, 0, sizeof(t));
+    t.U = cfg->n_units; t.G = cfg->gqa_group; t.d = cfg->head_dim; t.kv_dtype = cfg->kv_dtype;
+    t.max_tokens = cfg->max_tokens; t.max_clusters = cfg->max_clusters;
+    const int full_pages = (cfg->max_tokens + PAGE - 1) / PAGE;
+    int slack = full_pages / 8; if (slack < 64) slack = 64;
+    t.P = full_pages + cfg->max_clusters + slack;
+    t.W = t.P;
+    t.n_splits_attn = 8;
+    const size_t U = t.U, P = t.P, Mx = t.max_clusters, d = t.d;
+    const size_t page_elems = U * P * PAGE * d;
+    if (cfg->kv_dtype == DYNAKV_F32) {
+        float *a, *b; ALLOC(a, page_elems, false); ALLOC(b, page_elems, false); t.kpages = a; t.vpages = b;
+    } else {
+        __nv_bfloat16 *a, *b; ALLOC(a, page_elems, false); ALLOC(b, page_elems, false); t.kpages = a; t.vpages = b;
+    }
+    ALLOC(t.page_tok, U * P * PAGE, false);
+    ALLOC(t.page_next, U * P, false);
+    ALLOC(t.free_stack, U * P, false);
+    ALLOC(t.cl_r, U * Mx * d, true);
+    ALLOC(t.cl_M2, U * Mx, true);
+    ALLOC(t.cl_n, U * Mx, true);
+    ALLOC(t.cl_head, U * Mx, true);
+    ALLOC(t.cl_tail, U * Mx, true);
+    ALLOC(t.cl_flags, U * Mx, true);
+    ALLOC(t.u_N, U, true); ALLOC(t.u_M, U, true); ALLOC(t.u_Mlive, U, true); ALLOC(t.u_tau, U, true);
+    ALLOC(t.u_page_top, U, true); ALLOC(t.u_free_cnt, U, true);
+    ALLOC(t.tok_cluster, U * (size_t)t.max_tokens, false);
+    ALLOC(t.scores, U * Mx, true);
+    ALLOC(t.sel_ids, U * Mx, true);
+    ALLOC(t.sel_n, U, true); ALLOC(t.sel_tokens, U, true);
+    ALLOC(t.work, U * (size_t)t.W, false);
+    ALLOC(t.n_work, U, true);
+    ALLOC(t.part, U * (size_t)t.n_splits_attn * t.G * (d + 2), false);
+    ALLOC(t.sp_label, U * (size_t)t.max_tokens, false);
+    ALLOC(t.sp_pos, U * 2 * (size_t)t.max_tokens, false);
+    ALLOC(t.status, 1, true);
+    ALLOC(t.counters, 8, true);
+    ALLOC(c->step_ctr, 1, true);
+    ALLOC(c->st_q, U * t.G * d, false);
+    ALLOC(c->st_out, U * t.G * d, false);
+    {
+        char *a, *b; ALLOC(a, U * d * kv_bytes(*cfg), false); ALLOC(b, U * d * kv_bytes(*cfg), false);
+        c->st_k = a; c->st_v = b;
+    }
+    CK(cudaStreamSynchronize(c->stream));
+    *out = c;
+    return DYNAKV_OK;
+}
+
+extern "C" void dynakv_destroy(dynakv_ctx* c) {
+    if (!c) return;
+    cudaStreamSynchronize(c->stream);
+    if (c->graph_exec) cudaGraphExecDestroy(c->graph_exec);
+    for (void* p : c->allocs) cudaFree(p);
+    delete c;
+}
+
+extern "C" int dynakv_build_index(dynakv_ctx* c, const void* K, const void* V, int64_t n, int32_t d,
+                                  int32_t n_clusters, uint64_t seed) {
+    if (!c || !K || !V) return DYNAKV_ERR_ARG;
+    if (c->built) return DYNAKV_ERR_STATE;
+    Tables& t = c->t;
+    if (d != t.d || n_clusters < 1 || n_clusters > t.max_clusters || n < n_clusters || n > t.max_tokens) return DYNAKV_ERR_ARG;
+    const int M = n_clusters, T = c->cfg.kmeans_iters;
+    const size_t U = t.U;
+    BuildScratch b;
+    memset(&b, 0, sizeof(b));
+    const size_t mark = c->allocs.size();
+    ALLOC_B(b.C, U * M * d, false);
+    ALLOC_B(b.sums, U * M * d, false);
+    ALLOC_B(b.counts, U * M, false);
+    ALLOC_B(b.cursor, U * M, false);
+    ALLOC_B(b.picks, U * M, false);
+    if (c->cfg.init_mode == DYNAKV_INIT_KMEANSPP) ALLOC_B(b.D2, U * (size_t)n, false);
+    int* assign_buf = nullptr;
+    if (c->cfg.trace) { ALLOC_B(c->trace_assign, (size_t)T * U * n, false); }
+    else ALLOC_B(assign_buf, U * (size_t)n, false);
+    const bool use_tc = c->cfg.assign_mode == 0 && tc_assign_supported(t, n, M);
+    void* tc_scratch = nullptr;
+    if (use_tc) { char* p; ALLOC_B(p, tc_assign_scratch_bytes(t, n, M), false); tc_scratch = p; }
+
+    launch_init_centres(t, K, n, M, seed, c->cfg.init_mode, b, c->stream, &c->launches);
+    for (int it = 0; it < T; it++) {
+        b.assign = c->cfg.trace ? c->trace_assign + (size_t)it * U * n : assign_buf;
+        if (use_tc) launch_assign_tc(t, K, n, M, b.C, b.assign, tc_scratch, c->stream, &c->launches);
+        else launch_assign_f32(t, K, n, M, b.C, b.assign, c->stream, &c->launches);
+        launch_update(t, K, n, M, b.assign, b, c->stream, &c->launches);
+    }
+    launch_finalize(t, K, V, n, M, b, c->cfg.split_var_factor, c->stream, &c->launches);
+    CK(cudaGetLastError());
+    CK(cudaStreamSynchronize(c->stream));
+    // keep the picks for the trace; free the rest of the build scratch
+    if (c->cfg.trace) c->trace_picks = b.picks;
+    std::vector<void*> keep;
+    for (size_t i = mark; i < c->allocs.size(); i++) {
+        void* p = c->allocs[i];
+        if (c->cfg.trace && (p == (void*)c->trace_assign || p == (void*)b.picks)) keep.push_back(p);
+        else cudaFree(p);
+    }
+    c->allocs.resize(mark);
+    for (void* p : keep) c->allocs.push_back(p);
+    c->built = true; c->n_prefill = n; c->M0 = M;
+    return DYNAKV_OK;
+}
+
+static int enqueue_decode(dynakv_ctx* c, StepPtr q, int budget, StepPtrW out, int* sel_ids) {
+    launch_score_select(c->t, q, budget, sel_ids, c->stream, &c->launches);
+    launch_gather_attn(c->t, q, out, c->stream, &c->launches);
+    return DYNAKV_OK;
+}
+
+extern "C" int dynakv_decode_step(dynakv_ctx* c, const float* q, int32_t token_budget, float* out, int32_t* selected_ids) {
+    if (!c || !q || !out || token_budget < 0) return DYNAKV_ERR_ARG;
+    if (!c->built) return DYNAKV_ERR_STATE;
+    enqueue_decode(c, StepPtr{q, 0, nullptr}, token_budget, StepPtrW{out, 0, nullptr}, selected_ids);
+    CK(cudaGetLastError());
+    return DYNAKV_OK;
+}
+
+extern "C" int dynakv_append(dynakv_ctx* c, const void* k, const void* v) {
+    if (!c || !k || !v) return DYNAKV_ERR_ARG;
+    if (!c->built) return DYNAKV_ERR_STATE;
+    launch_append(c->t, StepPtr{k, 0, nullptr}, StepPtr{v, 0, nullptr}, c->stream, &c->launches);
+    CK(cudaGetLastError());
+    return DYNAKV_OK;
+}
+
+static void enqueue_split(dynakv_ctx* c) {
+    launch_split_check(c->t, c->cfg.split_size_factor, c->cfg.split_var_factor > 0.f ? 1 : 0, c->cfg.split_min_size,
+                       c->cfg.split_iters, c->stream, &c->launches);
+}
+
+extern "C" int dynakv_split_check(dynakv_ctx* c) {
+    if (!c) return DYNAKV_ERR_ARG;
+    if (!c->built) return DYNAKV_ERR_STATE;
+    enqueue_split(c);
+    CK(cudaGetLastError());
+    return DYNAKV_OK;
+}
+
+extern "C" int dynakv_decode_loop(dynakv_ctx* c, const float* q_steps, const void* k_steps, const void* v_steps,
+                                  int64_t n_steps, int32_t token_budget, float* out_steps) {
+    if (!c || !q_steps || !k_steps || !v_steps || !out_steps || n_steps < 0 || token_budget < 0) return DYNAKV_ERR_ARG;
+    if (!c->built) return DYNAKV_ERR_STATE;
+    const Tables& t = c->t;
+    if (!c->graph_exec || c->g_q != q_steps || c->g_k != k_steps || c->g_v != v_steps || c->g_out != out_steps ||
+        c->g_budget != token_budget) {
+        if (c->graph_exec) { cudaGraphExecDestroy(c->graph_exec); c->graph_exec = nullptr; }
+        const long long qs = (long long)t.U * t.G * t.d * 4, ks = (long long)t.U * t.d * (long long)kv_bytes(c->cfg);
+        cudaGraph_t graph = nullptr;
+        long long before = c->launches;
+        CK(cudaStreamBeginCapture(c->stream, cudaStreamCaptureModeThreadLocal));
+        enqueue_decode(c, StepPtr{q_steps, qs, c->step_ctr}, token_budget, StepPtrW{out_steps, qs, c->step_ctr}, nullptr);
+        launch_append(t, StepPtr{k_steps, ks, c->step_ctr}, StepPtr{v_steps, ks, c->step_ctr}, c->stream, &c->launches);
+        enqueue_split(c);
+        launch_step_inc(c->step_ctr, c->stream, &c->launches);
+        cudaError_t e = cudaStreamEndCapture(c->stream, &graph);
+        c->graph_nodes = c->launches - before;
+        c->launches = before;
+        if (e != cudaSuccess || !graph) {
+            snprintf(g_err, sizeof(g_err), "graph capture failed: %s", cudaGetErrorString(e));
+            return DYNAKV_ERR_CUDA;
+        }
+        e = cudaGraphInstantiate(&c->graph_exec, graph, 0);
+        cudaGraphDestroy(graph);
+        if (e != cudaSuccess) {
+            c->graph_exec = nullptr;
+            snprintf(g_err, sizeof(g_err), "graph instantiate failed: %s", cudaGetErrorString(e));
+            return DYNAKV_ERR_CUDA;
+        }
+        c->g_q = q_steps; c->g_k = k_steps; c->g_v = v_steps; c->g_out = out_steps; c->g_budget = token_budget;
+    }
+    CK(cudaMemsetAsync(c->step_ctr, 0, sizeof(int), c->stream));
+    for (int64_t s = 0; s < n_steps; s++) CK(cudaGraphLaunch(c->graph_exec, c->stream));
+    c->launches += c->graph_nodes * n_steps;
+    return DYNAKV_OK;
+}
+
+extern "C" int dynakv_step_host(dynakv_ctx* c, const float* q_host, const void* k_host, const void* v_host,
+                                int32_t token_budget, float* out_host) {
+    if (!c || !q_host || !k_host || !v_host || !out_host || token_budget < 0) return DYNAKV_ERR_ARG;
+    if (!c->built) return DYNAKV_ERR_STATE;
+    const Tables& t = c->t;
+    const size_t qb = (size_t)t.U * t.G * t.d * 4, kb = (size_t)t.U * t.d * kv_bytes(c->cfg);
+    CK(cudaMemcpyAsync(c->st_q, q_host, qb, cudaMemcpyHostToDevice, c->stream));
+    CK(cudaMemcpyAsync(c->st_k, k_host, kb, cudaMemcpyHostToDevice, c->stream));
+    CK(cudaMemcpyAsync(c->st_v, v_host, kb, cudaMemcpyHostToDevice, c->stream));
+    enqueue_decode(c, StepPtr{c->st_q, 0, nullptr}, token_budget, StepPtrW{c->st_out, 0, nullptr}, nullptr);
+    launch_append(t, StepPtr{c->st_k, 0, nullptr}, StepPtr{c->st_v, 0, nullptr}, c->stream, &c->launches);
+    enqueue_split(c);
+    CK(cudaMemcpyAsync(out_host, c->st_out, qb, cudaMemcpyDeviceToHost, c->stream));
+    CK(cudaStreamSynchronize(c->stream));
+    return DYNAKV_OK;
+}
+
+__global__ void k_sum_status(Tables t, long long* out) {
+    // out[0] tokens selected, out[1] clusters selected, out[2] pages in use
+    long long a = 0, b = 0, p = 0;
+    for (int u = threadIdx.x; u < t.U; u += blockDim.x) {
+        a += t.sel_tokens[u]; b += t.sel_n[u]; p += t.u_page_top[u] - t.u_free_cnt[u];
+    }
+    atomicAdd((unsigned long long*)&out[0], (unsigned long long)a);
+    atomicAdd((unsigned long long*)&out[1], (unsigned long long)b);
+    atomicAdd((unsigned long long*)&out[2], (unsigned long long)p);
+}
+
+extern "C" int dynakv_get_status(dynakv_ctx* c, dynakv_status* host_out) {
+    if (!c || !host_out) return DYNAKV_ERR_ARG;
+    memset(host_out, 0, sizeof(*host_out));
+    unsigned long long cnt[8];
+    CK(cudaMemsetAsync(c->t.counters + 4, 0, 3 * sizeof(unsigned long long), c->stream));
+    if (c->built) { k_sum_status<<<1, 256, 0, c->stream>>>(c->t, (long long*)(c->t.counters + 4)); c->launches++; }
+    CK(cudaMemcpyAsync(&host_out->error_bits, c->t.status, sizeof(unsigned int), cudaMemcpyDeviceToHost, c->stream));
+    CK(cudaMemcpyAsync(cnt, c->t.counters, sizeof(cnt), cudaMemcpyDeviceToHost, c->stream));
+    CK(cudaStreamSynchronize(c->stream));
+    host_out->n_appended = (int64_t)cnt[CNT_APPENDED];
+    host_out->n_splits = (int64_t)cnt[CNT_SPLITS];
+    host_out->assign_rechecked = (int64_t)cnt[CNT_RECHECKED];
+    host_out->tokens_selected = (int64_t)cnt[4];
+    host_out->clusters_selected = (int64_t)cnt[5];
+    host_out->pages_in_use = (int64_t)cnt[6];
+    return DYNAKV_OK;
+}
+
+extern "C" int dynakv_export_state(dynakv_ctx* c, int32_t* tok_cluster, float* centroids, int32_t* counts, float* M2,
+                                   int32_t* n_tokens, int32_t* n_ids, float* tau) {
+    if (!c) return DYNAKV_ERR_ARG;
+    if (!c->built) return DYNAKV_ERR_STATE;
+    const Tables& t = c->t;
+    const size_t U = t.U, Mx = t.max_clusters;
+    cudaStream_t s = c->stream;
+    if (tok_cluster) CK(cudaMemcpyAsync(tok_cluster, t.tok_cluster, sizeof(int) * U * t.max_tokens, cudaMemcpyDeviceToHost, s));
+    if (centroids) CK(cudaMemcpyAsync(centroids, t.cl_r, sizeof(float) * U * Mx * t.d, cudaMemcpyDeviceToHost, s));
+    if (counts) CK(cudaMemcpyAsync(counts, t.cl_n, sizeof(int) * U * Mx, cudaMemcpyDeviceToHost, s));
+    if (M2) CK(cudaMemcpyAsync(M2, t.cl_M2, sizeof(float) * U * Mx, cudaMemcpyDeviceToHost, s));
+    if (n_tokens) CK(cudaMemcpyAsync(n_tokens, t.u_N, sizeof(int) * U, cudaMemcpyDeviceToHost, s));
+    if (n_ids) CK(cudaMemcpyAsync(n_ids, t.u_M, sizeof(int) * U, cudaMemcpyDeviceToHost, s));
+    if (tau) CK(cudaMemcpyAsync(tau, t.u_tau, sizeof(float) * U, cudaMemcpyDeviceToHost, s));
+    CK(cudaStreamSynchronize(s));
+    return DYNAKV_OK;
+}
+
+extern "C" int dynakv_get_selection(dynakv_ctx* c, int32_t* n_selected, int32_t* tokens_selected) {
+    if (!c) return DYNAKV_ERR_ARG;
+    if (!c->built) return DYNAKV_ERR_STATE;
+    if (n_selected) CK(cudaMemcpyAsync(n_selected, c->t.sel_n, sizeof(int) * c->t.U, cudaMemcpyDeviceToHost, c->stream));
+    if (tokens_selected) CK(cudaMemcpyAsync(tokens_selected, c->t.sel_tokens, sizeof(int) * c->t.U, cudaMemcpyDeviceToHost, c->stream));
+    CK(cudaStreamSynchronize(c->stream));
+    return DYNAKV_OK;
+}
+
+extern "C" int dynakv_get_build_trace(dynakv_ctx* c, int32_t* picks, int32_t* assign) {
+    if (!c) return DYNAKV_ERR_ARG;
+    if (!c->built || !c->cfg.trace) return DYNAKV_ERR_STATE;
+    const size_t U = c->t.U;
+    if (picks) CK(cudaMemcpyAsync(picks, c->trace_picks, sizeof(int) * U * c->M0, cudaMemcpyDeviceToHost, c->stream));
+    if (assign) CK(cudaMemcpyAsync(assign, c->trace_assign, sizeof(int) * (size_t)c->cfg.kmeans_iters * U * c->n_prefill,
+                                   cudaMemcpyDeviceToHost, c->stream));
+    CK(cudaStreamSynchronize(c->stream));
+    return DYNAKV_OK;
+}
+
+extern "C" int64_t dynakv_launch_count(dynakv_ctx* c) { return c ? c->launches : 0; }

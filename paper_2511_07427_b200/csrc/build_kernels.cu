@@ -1,0 +1,449 @@
+// Prefill kernels: seeded initial centres, fp32 nearest-centre assignment, centroid
+// reduction, and the layout step that stores each cluster's members contiguously in pages
+// (arXiv 2511.07427: NewCluster of Algorithm 1, Eq. 3-4, Section 5.1 placement).
+#include <float.h>
+
+#include "common.cuh"
+
+namespace dkv {
+
+// ------------------------------------------------------------------ init: k-means++
+
+// One block per unit.  Exponential-race form of D^2 sampling: round 0 picks
+// argmin_i E_i, round r picks argmax_i D2_i / E_i with E_i = -ln u(seed, unit, r, i);
+// ties go to the lowest index.
+template <typename KV, int HD>
+__global__ void __launch_bounds__(1024) k_init_kmeanspp(const KV* __restrict__ K, int n, int M,
+                                                        unsigned long long seed, float* __restrict__ C,
+                                                        float* __restrict__ D2, int* __restrict__ picks) {
+    const int u = blockIdx.x, tid = threadIdx.x;
+    const KV* Ku = K + (size_t)u * n * HD;
+    float* D2u = D2 + (size_t)u * n;
+    __shared__ float cen[HD];
+    __shared__ float red_v[32];
+    __shared__ int red_i[32];
+    __shared__ int s_pick;
+    for (int r = 0; r < M; r++) {
+        float bv = -FLT_MAX; int bi = 0x7fffffff;
+        for (int i = tid; i < n; i += blockDim.x) {
+            float uu = ((float)hash23(seed, u, r, i) + 0.5f) * (1.0f / 8388608.0f);
+            float E = -logf(uu);
+            float v;
+            if (r == 0) v = -E;
+            else {
+                const KV* k = Ku + (size_t)i * HD;
+                float dist = 0.f;
+#pragma unroll 4
+                for (int e = 0; e < HD; e += 4) {
+                    float4 kk = ld4(k, e);
+                    float a = kk.x - cen[e], b = kk.y - cen[e + 1], c = kk.z - cen[e + 2], dd = kk.w - cen[e + 3];
+                    dist = fmaf(a, a, dist); dist = fmaf(b, b, dist); dist = fmaf(c, c, dist); dist = fmaf(dd, dd, dist);
+                }
+                float d2 = (r == 1) ? dist : fminf(D2u[i], dist);
+                D2u[i] = d2;
+                v = d2 / E;
+            }
+            if (v > bv || (v == bv && i < bi)) { bv = v; bi = i; }
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            float ov = __shfl_xor_sync(0xffffffffu, bv, o); int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+            if (ov > bv || (ov == bv && oi < bi)) { bv = ov; bi = oi; }
+        }
+        if ((tid & 31) == 0) { red_v[tid >> 5] = bv; red_i[tid >> 5] = bi; }
+        __syncthreads();
+        if (tid < 32) {
+            int nw = blockDim.x >> 5;
+            bv = tid < nw ? red_v[tid] : -FLT_MAX; bi = tid < nw ? red_i[tid] : 0x7fffffff;
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) {
+                float ov = __shfl_xor_sync(0xffffffffu, bv, o); int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+                if (ov > bv || (ov == bv && oi < bi)) { bv = ov; bi = oi; }
+            }
+            if (tid == 0) { s_pick = bi; picks[(size_t)u * M + r] = bi; }
+        }
+        __syncthreads();
+        for (int e = tid; e < HD; e += blockDim.x) {
+            float x = to_f(Ku[(size_t)s_pick * HD + e]);
+            cen[e] = x;
+            C[((size_t)u * M + r) * HD + e] = x;
+        }
+        __syncthreads();
+    }
+}
+
+// ------------------------------------------------------------------ init: random distinct
+
+// One block per unit.  Selects the M keys with the smallest (hash23, index) and lists
+// them in index order: two histogram passes find the boundary hash value, a chunked
+// ordered compaction writes the picks.
+template <typename KV, int HD>
+__global__ void __launch_bounds__(1024) k_init_random(const KV* __restrict__ K, int n, int M,
+                                                      unsigned long long seed, float* __restrict__ C,
+                                                      int* __restrict__ picks) {
+    const int u = blockIdx.x, tid = threadIdx.x;
+    __shared__ int hist[4096];
+    __shared__ int sh[33];
+    __shared__ int s_bin, s_before;
+    // pass 1: top 12 bits
+    for (int b = tid; b < 4096; b += blockDim.x) hist[b] = 0;
+    __syncthreads();
+    for (int i = tid; i < n; i += blockDim.x) atomicAdd(&hist[hash23(seed, u, 0, i) >> 11], 1);
+    __syncthreads();
+    if (tid == 0) {
+        int cum = 0, b = 0;
+        for (; b < 4096; b++) { if (cum + hist[b] >= M) break; cum += hist[b]; }
+        s_bin = b; s_before = cum;
+    }
+    __syncthreads();
+    const int bin1 = s_bin; const int need1 = M - s_before;
+    __syncthreads();
+    // pass 2: low 11 bits inside the boundary bin
+    for (int b = tid; b < 2048; b += blockDim.x) hist[b] = 0;
+    __syncthreads();
+    for (int i = tid; i < n; i += blockDim.x) {
+        unsigned int h = hash23(seed, u, 0, i);
+        if ((int)(h >> 11) == bin1) atomicAdd(&hist[h & 2047], 1);
+    }
+    __syncthreads();
+    if (tid == 0) {
+        int cum = 0, b = 0;
+        for (; b < 2048; b++) { if (cum + hist[b] >= need1) break; cum += hist[b]; }
+        s_bin = b; s_before = cum;
+    }
+    __syncthreads();
+    const unsigned int hstar = ((unsigned int)bin1 << 11) | (unsigned int)s_bin;
+    const int need_eq = need1 - s_before;   // how many keys with hash == hstar are taken (lowest indices first)
+    int eq_seen = 0, out_pos = 0;
+    for (int base = 0; base < n; base += blockDim.x) {
+        int i = base + tid;
+        unsigned int h = i < n ? hash23(seed, u, 0, i) : 0xffffffffu;
+        int is_eq = (i < n && h == hstar) ? 1 : 0;
+        int tot_eq, tot_sel;
+        int eq_rank = eq_seen + block_scan_excl(is_eq, sh, &tot_eq);
+        int sel = (i < n && (h < hstar || (is_eq && eq_rank < need_eq))) ? 1 : 0;
+        int pos = out_pos + block_scan_excl(sel, sh, &tot_sel);
+        if (sel && pos < M) picks[(size_t)u * M + pos] = i;
+        eq_seen += tot_eq; out_pos += tot_sel;
+    }
+    __syncthreads();
+    const KV* Ku = K + (size_t)u * n * HD;
+    for (int idx = tid; idx < M * HD; idx += blockDim.x) {
+        int j = idx / HD, e = idx % HD;
+        C[((size_t)u * M + j) * HD + e] = to_f(Ku[(size_t)picks[(size_t)u * M + j] * HD + e]);
+    }
+}
+
+// ------------------------------------------------------------------ assign (fp32, direct form)
+
+// a_i = argmin_j sum_t (k_it - c_jt)^2, ties to the lowest j.  Block tile: 128 keys x 64
+// centres, whole head dimension staged in shared memory (transposed, so the inner loop
+// reads 3 vectors per t); thread tile 8 keys x 4 centres.
+constexpr int AS_BK = 128, AS_BC = 64, AS_THREADS = 256;
+template <int HD> struct AssignSmem {
+    static constexpr int KS = AS_BK + 4, CS = AS_BC + 4;
+    static constexpr size_t bytes = sizeof(float) * ((size_t)HD * KS + (size_t)HD * CS);
+};
+
+template <typename KV, int HD>
+__global__ void __launch_bounds__(AS_THREADS) k_assign_f32(const KV* __restrict__ K, int n, int M,
+                                                           const float* __restrict__ C, int* __restrict__ assign) {
+    extern __shared__ __align__(16) float smem[];
+    constexpr int KS = AssignSmem<HD>::KS, CS = AssignSmem<HD>::CS;
+    float* keysT = smem;                 // [HD][KS]
+    float* centT = smem + (size_t)HD * KS;  // [HD][CS]
+    const int u = blockIdx.y, tid = threadIdx.x;
+    const int key0 = blockIdx.x * AS_BK;
+    const KV* Ku = K + (size_t)u * n * HD;
+    const float* Cu = C + (size_t)u * M * HD;
+    const int ty = tid >> 4, tx = tid & 15;
+
+    for (int idx = tid; idx < AS_BK * (HD / 4); idx += AS_THREADS) {
+        int key = idx % AS_BK, t4 = idx / AS_BK;
+        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (key0 + key < n) v = ld4(Ku + (size_t)(key0 + key) * HD, t4 * 4);
+        keysT[(t4 * 4 + 0) * KS + key] = v.x; keysT[(t4 * 4 + 1) * KS + key] = v.y;
+        keysT[(t4 * 4 + 2) * KS + key] = v.z; keysT[(t4 * 4 + 3) * KS + key] = v.w;
+    }
+    float best[8]; int bj[8];
+#pragma unroll
+    for (int i = 0; i < 8; i++) { best[i] = FLT_MAX; bj[i] = 0x7fffffff; }
+
+    for (int c0 = 0; c0 < M; c0 += AS_BC) {
+        __syncthreads();
+        for (int idx = tid; idx < AS_BC * (HD / 4); idx += AS_THREADS) {
+            int c = idx % AS_BC, t4 = idx / AS_BC;
+            float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (c0 + c < M) v = ld4(Cu + (size_t)(c0 + c) * HD, t4 * 4);
+            centT[(t4 * 4 + 0) * CS + c] = v.x; centT[(t4 * 4 + 1) * CS + c] = v.y;
+            centT[(t4 * 4 + 2) * CS + c] = v.z; centT[(t4 * 4 + 3) * CS + c] = v.w;
+        }
+        __syncthreads();
+        float acc[8][4];
+#pragma unroll
+        for (int i = 0; i < 8; i++)
+#pragma unroll
+            for (int j = 0; j < 4; j++) acc[i][j] = 0.f;
+#pragma unroll 4
+        for (int t = 0; t < HD; t++) {
+            float4 k0 = *reinterpret_cast<const float4*>(keysT + t * KS + ty * 8);
+            float4 k1 = *reinterpret_cast<const float4*>(keysT + t * KS + ty * 8 + 4);
+            float4 cc = *reinterpret_cast<const float4*>(centT + t * CS + tx * 4);
+            float kk[8] = {k0.x, k0.y, k0.z, k0.w, k1.x, k1.y, k1.z, k1.w};
+            float cv[4] = {cc.x, cc.y, cc.z, cc.w};
+#pragma unroll
+            for (int i = 0; i < 8; i++)
+#pragma unroll
+                for (int j = 0; j < 4; j++) { float df = kk[i] - cv[j]; acc[i][j] = fmaf(df, df, acc[i][j]); }
+        }
+#pragma unroll
+        for (int i = 0; i < 8; i++)
+#pragma unroll
+            for (int j = 0; j < 4; j++) {
+                int cj = c0 + tx * 4 + j;
+                if (cj < M && (acc[i][j] < best[i] || (acc[i][j] == best[i] && cj < bj[i]))) { best[i] = acc[i][j]; bj[i] = cj; }
+            }
+    }
+#pragma unroll
+    for (int i = 0; i < 8; i++) {
+#pragma unroll
+        for (int o = 8; o > 0; o >>= 1) {
+            float ov = __shfl_xor_sync(0xffffffffu, best[i], o); int oj = __shfl_xor_sync(0xffffffffu, bj[i], o);
+            if (ov < best[i] || (ov == best[i] && oj < bj[i])) { best[i] = ov; bj[i] = oj; }
+        }
+        int key = key0 + ty * 8 + i;
+        if (tx == 0 && key < n) assign[(size_t)u * n + key] = bj[i];
+    }
+}
+
+// ------------------------------------------------------------------ update (centroid reduction)
+
+// One warp per key: add the key into its cluster's fp32 sum with vector atomics, count it.
+template <typename KV, int HD>
+__global__ void __launch_bounds__(256) k_update_sums(const KV* __restrict__ K, long long n_total, int n, int M,
+                                                      const int* __restrict__ assign, float* __restrict__ sums,
+                                                      int* __restrict__ counts) {
+    const int lane = threadIdx.x & 31;
+    long long w = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const long long nwarps = ((long long)gridDim.x * blockDim.x) >> 5;
+    for (; w < n_total; w += nwarps) {
+        int u = (int)(w / n);
+        int j = assign[w];
+        const KV* k = K + (size_t)w * HD;
+        float* dst = sums + ((size_t)u * M + j) * HD;
+        if (lane * 4 < HD) {
+            float4 v = ld4(k, lane * 4);
+            atomicAdd(reinterpret_cast<float4*>(dst + lane * 4), v);
+        }
+        if (lane == 0) atomicAdd(&counts[(size_t)u * M + j], 1);
+    }
+}
+
+// c_j = sum_j / count_j; an empty cluster keeps its previous centre.
+__global__ void k_centroid_div(float* __restrict__ C, const float* __restrict__ sums, const int* __restrict__ counts,
+                               long long total, int d) {
+    long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= total) return;
+    int c = counts[i / d];
+    if (c > 0) C[i] = sums[i] / (float)c;
+}
+
+// ------------------------------------------------------------------ finalize: layout
+
+// One block per unit: page chains for every non-empty cluster (consecutive pages at build
+// time), per-unit counters, cursors zeroed.
+__global__ void __launch_bounds__(1024) k_fin_layout(Tables t, int n, int M, const int* __restrict__ counts,
+                                                     int* __restrict__ cursor) {
+    const int u = blockIdx.x, tid = threadIdx.x;
+    __shared__ int sh[33];
+    __shared__ int s_live;
+    if (tid == 0) s_live = 0;
+    __syncthreads();
+    int page_base = 0, live = 0;
+    for (int base = 0; base < t.max_clusters; base += blockDim.x) {
+        int j = base + tid;
+        int c = (j < M) ? counts[(size_t)u * M + j] : 0;
+        int np = (c + PAGE - 1) / PAGE;
+        int tot;
+        int first = page_base + block_scan_excl(np, sh, &tot);
+        if (j < t.max_clusters) {
+            size_t cj = (size_t)u * t.max_clusters + j;
+            t.cl_n[cj] = c;
+            t.cl_flags[cj] = 0;
+            t.cl_M2[cj] = 0.f;
+            t.cl_head[cj] = c > 0 ? first : -1;
+            t.cl_tail[cj] = c > 0 ? first + np - 1 : -1;
+            if (j < M) cursor[(size_t)u * M + j] = 0;
+            for (int p = 0; p < np; p++) t.page_next[(size_t)u * t.P + first + p] = (p + 1 < np) ? first + p + 1 : -1;
+            if (c > 0) live++;
+        }
+        page_base += tot;
+    }
+    atomicAdd(&s_live, live);
+    __syncthreads();
+    if (tid == 0) {
+        t.u_N[u] = n; t.u_M[u] = M; t.u_Mlive[u] = s_live; t.u_page_top[u] = page_base; t.u_free_cnt[u] = 0;
+    }
+    for (int i = n + tid; i < t.max_tokens; i += blockDim.x) t.tok_cluster[(size_t)u * t.max_tokens + i] = -1;
+}
+
+// One warp per token: claim the next slot of the token's cluster and copy its K, V rows.
+template <typename KV, int HD>
+__global__ void __launch_bounds__(256) k_fin_scatter(Tables t, const KV* __restrict__ K, const KV* __restrict__ V,
+                                                      long long n_total, int n, int M, const int* __restrict__ assign,
+                                                      int* __restrict__ cursor) {
+    const int lane = threadIdx.x & 31;
+    long long w = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const long long nwarps = ((long long)gridDim.x * blockDim.x) >> 5;
+    KV* kp = reinterpret_cast<KV*>(t.kpages);
+    KV* vp = reinterpret_cast<KV*>(t.vpages);
+    for (; w < n_total; w += nwarps) {
+        int u = (int)(w / n), i = (int)(w % n);
+        int j = assign[w];
+        int slot = 0;
+        if (lane == 0) slot = atomicAdd(&cursor[(size_t)u * M + j], 1);
+        slot = __shfl_sync(0xffffffffu, slot, 0);
+        int page = t.cl_head[(size_t)u * t.max_clusters + j] + slot / PAGE, row = slot % PAGE;
+        size_t dst = (((size_t)u * t.P + page) * PAGE + row) * HD;
+        constexpr int EPL = HD / 32;   // elements per lane
+        const KV* ks = K + (size_t)w * HD + lane * EPL;
+        const KV* vs = V + (size_t)w * HD + lane * EPL;
+#pragma unroll
+        for (int e = 0; e < EPL; e++) { kp[dst + lane * EPL + e] = ks[e]; vp[dst + lane * EPL + e] = vs[e]; }
+        if (lane == 0) {
+            t.page_tok[((size_t)u * t.P + page) * PAGE + row] = i;
+            t.tok_cluster[(size_t)u * t.max_tokens + i] = j;
+        }
+    }
+}
+
+// One warp per cluster: r_j = the final centre, M2_j = sum over members ||k - r_j||^2.
+template <typename KV, int HD>
+__global__ void __launch_bounds__(256) k_fin_stats(Tables t, int M, const float* __restrict__ C) {
+    const int lane = threadIdx.x & 31;
+    long long w = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    if (w >= (long long)t.U * M) return;
+    int u = (int)(w / M), j = (int)(w % M);
+    size_t cj = (size_t)u * t.max_clusters + j;
+    constexpr int EPL = HD / 32;
+    float r[EPL];
+#pragma unroll
+    for (int e = 0; e < EPL; e++) {
+        r[e] = C[((size_t)u * M + j) * HD + lane * EPL + e];
+        t.cl_r[cj * HD + lane * EPL + e] = r[e];
+    }
+    int c = t.cl_n[cj];
+    const KV* kp = reinterpret_cast<const KV*>(t.kpages);
+    float m2 = 0.f;
+    int page = t.cl_head[cj];
+    for (int s = 0; s < c; s++) {
+        int row = s % PAGE;
+        if (s > 0 && row == 0) page = t.page_next[(size_t)u * t.P + page];
+        const KV* k = kp + (((size_t)u * t.P + page) * PAGE + row) * HD + lane * EPL;
+        float part = 0.f;
+#pragma unroll
+        for (int e = 0; e < EPL; e++) { float df = to_f(k[e]) - r[e]; part = fmaf(df, df, part); }
+        m2 += warp_sum(part);
+    }
+    if (lane == 0) t.cl_M2[cj] = m2;
+}
+
+// One block per unit: tau = alpha * mean over live clusters of M2_j / n_j.
+__global__ void __launch_bounds__(256) k_fin_tau(Tables t, int M, float alpha) {
+    const int u = blockIdx.x;
+    __shared__ float red[256];
+    float s = 0.f;
+    for (int j = threadIdx.x; j < M; j += blockDim.x) {
+        size_t cj = (size_t)u * t.max_clusters + j;
+        int c = t.cl_n[cj];
+        if (c > 0) s += t.cl_M2[cj] / (float)c;
+    }
+    red[threadIdx.x] = s;
+    __syncthreads();
+    for (int o = 128; o > 0; o >>= 1) { if (threadIdx.x < o) red[threadIdx.x] += red[threadIdx.x + o]; __syncthreads(); }
+    if (threadIdx.x == 0) t.u_tau[u] = alpha * red[0] / (float)max(t.u_Mlive[u], 1);
+}
+
+// ------------------------------------------------------------------ launchers
+
+template <typename KV, int HD>
+static void init_centres_t(const Tables& t, const void* K, long long n, int M, unsigned long long seed, int mode,
+                           const BuildScratch& b, cudaStream_t s, long long* launches) {
+    if (mode == DYNAKV_INIT_KMEANSPP)
+        k_init_kmeanspp<KV, HD><<<t.U, 1024, 0, s>>>((const KV*)K, (int)n, M, seed, b.C, b.D2, b.picks);
+    else
+        k_init_random<KV, HD><<<t.U, 1024, 0, s>>>((const KV*)K, (int)n, M, seed, b.C, b.picks);
+    (*launches)++;
+}
+
+#define DKV_DISPATCH(FN, ...)                                                             \
+    do {                                                                                  \
+        if (t.kv_dtype == DYNAKV_F32) {                                                   \
+            if (t.d == 64) FN<float, 64>(__VA_ARGS__); else FN<float, 128>(__VA_ARGS__);  \
+        } else {                                                                          \
+            if (t.d == 64) FN<__nv_bfloat16, 64>(__VA_ARGS__); else FN<__nv_bfloat16, 128>(__VA_ARGS__); \
+        }                                                                                 \
+    } while (0)
+
+void launch_init_centres(const Tables& t, const void* K, long long n, int M, unsigned long long seed,
+                         int init_mode, const BuildScratch& b, cudaStream_t s, long long* launches) {
+    DKV_DISPATCH(init_centres_t, t, K, n, M, seed, init_mode, b, s, launches);
+}
+
+template <typename KV, int HD>
+static void assign_f32_t(const Tables& t, const void* K, long long n, int M, const float* C, int* assign,
+                         cudaStream_t s, long long* launches) {
+    static bool attr_set = false;
+    if (!attr_set) {
+        cudaFuncSetAttribute(k_assign_f32<KV, HD>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)AssignSmem<HD>::bytes);
+        attr_set = true;
+    }
+    dim3 grid((unsigned)((n + AS_BK - 1) / AS_BK), t.U);
+    k_assign_f32<KV, HD><<<grid, AS_THREADS, AssignSmem<HD>::bytes, s>>>((const KV*)K, (int)n, M, C, assign);
+    (*launches)++;
+}
+
+void launch_assign_f32(const Tables& t, const void* K, long long n, int M, const float* C, int* assign,
+                       cudaStream_t s, long long* launches) {
+    DKV_DISPATCH(assign_f32_t, t, K, n, M, C, assign, s, launches);
+}
+
+template <typename KV, int HD>
+static void update_t(const Tables& t, const void* K, long long n, int M, const int* assign, const BuildScratch& b,
+                     cudaStream_t s, long long* launches) {
+    long long total = (long long)t.U * n;
+    cudaMemsetAsync(b.sums, 0, sizeof(float) * (size_t)t.U * M * HD, s);
+    cudaMemsetAsync(b.counts, 0, sizeof(int) * (size_t)t.U * M, s);
+    long long blocks = (total + 7) / 8;
+    if (blocks > 148LL * 64) blocks = 148LL * 64;
+    k_update_sums<KV, HD><<<(unsigned)blocks, 256, 0, s>>>((const KV*)K, total, (int)n, M, assign, b.sums, b.counts);
+    long long cd = (long long)t.U * M * HD;
+    k_centroid_div<<<(unsigned)((cd + 255) / 256), 256, 0, s>>>(b.C, b.sums, b.counts, cd, HD);
+    (*launches) += 2;
+}
+
+void launch_update(const Tables& t, const void* K, long long n, int M, const int* assign, const BuildScratch& b,
+                   cudaStream_t s, long long* launches) {
+    DKV_DISPATCH(update_t, t, K, n, M, assign, b, s, launches);
+}
+
+template <typename KV, int HD>
+static void finalize_t(const Tables& t, const void* K, const void* V, long long n, int M, const BuildScratch& b,
+                       float alpha, cudaStream_t s, long long* launches) {
+    k_fin_layout<<<t.U, 1024, 0, s>>>(t, (int)n, M, b.counts, b.cursor);
+    long long total = (long long)t.U * n;
+    long long blocks = (total + 7) / 8;
+    if (blocks > 148LL * 64) blocks = 148LL * 64;
+    k_fin_scatter<KV, HD><<<(unsigned)blocks, 256, 0, s>>>(t, (const KV*)K, (const KV*)V, total, (int)n, M, b.assign, b.cursor);
+    long long nw = (long long)t.U * M;
+    k_fin_stats<KV, HD><<<(unsigned)((nw + 7) / 8), 256, 0, s>>>(t, M, b.C);
+    k_fin_tau<<<t.U, 256, 0, s>>>(t, M, alpha);
+    (*launches) += 4;
+}
+
+void launch_finalize(const Tables& t, const void* K, const void* V, long long n, int M, const BuildScratch& b,
+                     float alpha, cudaStream_t s, long long* launches) {
+    DKV_DISPATCH(finalize_t, t, K, V, n, M, b, alpha, s, launches);
+}
+
+}  // namespace dkv

@@ -1,0 +1,157 @@
+// Shared declarations of libdynakv's kernels: the table of device arrays that holds one
+// context's index and KV store, small device helpers, and the host launchers each .cu
+// file exports to api.cu.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/dynakv.h"
+
+namespace dkv {
+
+constexpr int PAGE = 32;            // tokens per page
+constexpr int MAX_G = 8;
+constexpr int FLAG_HOLD = 1;        // split abandoned; not retried until the next append
+
+// Device-resident state of a context.  All arrays are unit-major.
+//   KV store: kpages/vpages [U][P][PAGE][d] in kv dtype; every cluster owns a chain of
+//   pages (cl_head -> page_next -> ... -> cl_tail) in which all pages but the tail are
+//   full, so cluster members are contiguous page by page (intra-cluster placement).
+struct Tables {
+    int U, G, d, kv_dtype, max_tokens, max_clusters, P, n_splits_attn;
+    int W;                           // work-list capacity per unit (page entries)
+    void* kpages; void* vpages;
+    int* page_tok;                   // [U][P][PAGE] token id per slot
+    int* page_next;                  // [U][P]
+    int* free_stack;                 // [U][P]
+    float* cl_r;                     // [U][Mmax][d] representatives (fp32)
+    float* cl_M2;                    // [U][Mmax]
+    int* cl_n;                       // [U][Mmax]   0 = dead / unused
+    int* cl_head; int* cl_tail;      // [U][Mmax]
+    unsigned char* cl_flags;         // [U][Mmax]
+    int* u_N; int* u_M; int* u_Mlive; float* u_tau; int* u_page_top; int* u_free_cnt;   // [U]
+    int* tok_cluster;                // [U][max_tokens]
+    // decode scratch
+    float* scores;                   // [U][Mmax]
+    int* sel_ids;                    // [U][Mmax]
+    int* sel_n; int* sel_tokens;     // [U]
+    int2* work;                      // [U][W] (page, count)
+    int* n_work;                     // [U]
+    float* part;                     // [U][S][G][d + 2]  partial (acc, m, l)
+    // split scratch
+    unsigned char* sp_label;         // [U][max_tokens]
+    int* sp_pos;                     // [U][2 * max_tokens]: rank per position, then hole list
+    // status / counters
+    unsigned int* status;            // [1]
+    unsigned long long* counters;    // [8]: 0 appended, 1 splits, 2 rechecked
+};
+
+enum { CNT_APPENDED = 0, CNT_SPLITS = 1, CNT_RECHECKED = 2 };
+
+// A per-step operand: base pointer plus a stride applied with the device-side step index,
+// so the same kernel serves a direct call (ctr == nullptr) and a captured graph replay.
+struct StepPtr {
+    const void* base;
+    long long stride_bytes;
+    const int* ctr;
+    __device__ __forceinline__ const void* get() const {
+        long long t = ctr ? (long long)(*ctr) : 0;
+        return (const char*)base + t * stride_bytes;
+    }
+};
+struct StepPtrW {
+    void* base;
+    long long stride_bytes;
+    const int* ctr;
+    __device__ __forceinline__ void* get() const {
+        long long t = ctr ? (long long)(*ctr) : 0;
+        return (char*)base + t * stride_bytes;
+    }
+};
+
+// ---- element load helpers -------------------------------------------------------------
+__device__ __forceinline__ float to_f(float x) { return x; }
+__device__ __forceinline__ float to_f(__nv_bfloat16 x) { return __bfloat162float(x); }
+
+// Load 4 consecutive elements starting at element index e (e % 4 == 0) as floats.
+__device__ __forceinline__ float4 ld4(const float* p, int e) {
+    return *reinterpret_cast<const float4*>(p + e);
+}
+__device__ __forceinline__ float4 ld4(const __nv_bfloat16* p, int e) {
+    uint2 r = *reinterpret_cast<const uint2*>(p + e);
+    float4 o;
+    o.x = __uint_as_float(r.x << 16); o.y = __uint_as_float(r.x & 0xffff0000u);
+    o.z = __uint_as_float(r.y << 16); o.w = __uint_as_float(r.y & 0xffff0000u);
+    return o;
+}
+__device__ __forceinline__ void st4(float* p, int e, float4 v) { *reinterpret_cast<float4*>(p + e) = v; }
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+
+// Exclusive prefix sum of one int per thread over the block; *total gets the block sum.
+// `sh` must hold 33 ints.  Contains __syncthreads; every thread of the block must call it.
+__device__ __forceinline__ int block_scan_excl(int v, int* sh, int* total) {
+    int lane = threadIdx.x & 31, w = threadIdx.x >> 5, nw = (blockDim.x + 31) >> 5;
+    int x = v;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) { int y = __shfl_up_sync(0xffffffffu, x, o); if (lane >= o) x += y; }
+    __syncthreads();
+    if (lane == 31) sh[w] = x;
+    __syncthreads();
+    if (w == 0) {
+        int s = lane < nw ? sh[lane] : 0;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) { int y = __shfl_up_sync(0xffffffffu, s, o); if (lane >= o) s += y; }
+        sh[lane] = s;
+        if (lane == 31) sh[32] = s;
+    }
+    __syncthreads();
+    int base = w > 0 ? sh[w - 1] : 0;
+    *total = sh[32];
+    return base + x - v;
+}
+
+// Counter-based uniform with 23 random bits, u = (bits + 1/2) / 2^23: the 64-bit counter
+// built from (seed, unit, round, i) goes through the splitmix64 finaliser.
+__device__ __forceinline__ unsigned int hash23(unsigned long long seed, int unit, int round, long long i) {
+    unsigned long long x = seed ^ ((unsigned long long)(unit + 1) * 0x9E3779B97F4A7C15ULL);
+    x += (unsigned long long)round * 0xBF58476D1CE4E5B9ULL + (unsigned long long)i * 0x94D049BB133111EBULL;
+    x ^= x >> 30; x *= 0xBF58476D1CE4E5B9ULL;
+    x ^= x >> 27; x *= 0x94D049BB133111EBULL;
+    x ^= x >> 31;
+    return (unsigned int)(x >> 41);
+}
+
+// ---- host launchers (defined in the kernel files) ---------------------------------------
+struct BuildScratch {
+    float* C;            // [U][M][d] current centres
+    float* sums;         // [U][M][d]
+    int* counts;         // [U][M]
+    int* assign;         // [U][n] (or a slice of the trace)
+    float* D2;           // [U][n] k-means++ distances
+    int* picks;          // [U][M]
+    int* cursor;         // [U][M]
+};
+
+void launch_init_centres(const Tables& t, const void* K, long long n, int M, unsigned long long seed,
+                         int init_mode, const BuildScratch& b, cudaStream_t s, long long* launches);
+void launch_assign_f32(const Tables& t, const void* K, long long n, int M, const float* C, int* assign,
+                       cudaStream_t s, long long* launches);
+void launch_update(const Tables& t, const void* K, long long n, int M, const int* assign, const BuildScratch& b,
+                   cudaStream_t s, long long* launches);
+void launch_finalize(const Tables& t, const void* K, const void* V, long long n, int M, const BuildScratch& b,
+                     float alpha, cudaStream_t s, long long* launches);
+void launch_score_select(const Tables& t, StepPtr q, int budget, int* user_sel_ids, cudaStream_t s, long long* launches);
+void launch_gather_attn(const Tables& t, StepPtr q, StepPtrW out, cudaStream_t s, long long* launches);
+void launch_append(const Tables& t, StepPtr k, StepPtr v, cudaStream_t s, long long* launches);
+void launch_split_check(const Tables& t, float gamma, int var_enabled, int min_size, int iters, cudaStream_t s,
+                        long long* launches);
+void launch_step_inc(int* ctr, cudaStream_t s, long long* launches);
+
+}  // namespace dkv

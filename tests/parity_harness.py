@@ -1,0 +1,172 @@
+"""Lock-step parity driver: runs the CUDA library and the fp64 oracle on the same seeded
+inputs, call by call, and compares them under the tie-follow protocol.
+
+Protocol.  Every discrete decision the GPU takes (initial centres, every Lloyd round's
+assignment, the selected cluster list, the append target, the split partition) is read
+back and offered to the oracle as a *hint*.  The oracle computes its own answer first;
+it follows the hint only if its own fp64 numbers put the two candidates within 1e-5
+relative of each other (a logged tie), otherwise it keeps its answer, counts a violation,
+and the comparison that follows fails.  Compared after each call: cluster membership and
+ids (exact), selected lists (exact), centroids (<= 1e-4 relative per vector), attention
+output (max abs <= 2e-3, relative L2 <= 1e-3).
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass, field
+from typing import List, Optional, Sequence
+
+import numpy as np
+import torch
+
+import oracle as O
+import paper_2511_07427_b200 as P
+from gen import UnitStream, WorkloadConfig, make_decode_chunk, make_prefill
+
+TOL_TIE = 1e-5
+TOL_CENTROID = 1e-4
+TOL_OUT_ABS = 2e-3
+TOL_OUT_L2 = 1e-3
+
+
+@dataclass
+class ParityReport:
+    ties: int = 0
+    violations: int = 0
+    steps: int = 0
+    splits: int = 0
+    max_out_abs: float = 0.0
+    max_out_l2: float = 0.0
+    max_centroid_rel: float = 0.0
+    tokens_selected: List[int] = field(default_factory=list)
+    status_bits: int = 0
+    rechecked: int = 0
+
+
+def make_ctx(cfg: WorkloadConfig, n_units: int, trace: int = 1, assign_mode: int = 0) -> P.DynaKV:
+    return P.DynaKV(P.DynaKVConfig(
+        n_units=n_units, gqa_group=cfg.G, head_dim=cfg.d,
+        kv_dtype=P.F32 if cfg.kv_dtype == "f32" else P.BF16,
+        max_tokens=cfg.max_tokens, max_clusters=cfg.max_clusters, kmeans_iters=cfg.T,
+        init_mode=P.INIT_KMEANSPP if cfg.init_mode == "kmeanspp" else P.INIT_RANDOM,
+        split_size_factor=cfg.split_size_factor, split_var_factor=cfg.split_var_factor,
+        split_min_size=cfg.split_min_size, split_iters=cfg.split_iters, trace=trace, assign_mode=assign_mode))
+
+
+def make_oracle(cfg: WorkloadConfig) -> O.OracleUnit:
+    return O.OracleUnit(cfg.d, cfg.G, cfg.max_tokens, cfg.max_clusters,
+                        gamma=float(np.float32(cfg.split_size_factor)), alpha=float(np.float32(cfg.split_var_factor)),
+                        split_min_size=cfg.split_min_size, split_iters=cfg.split_iters, tol=TOL_TIE)
+
+
+def rel_l2(a: np.ndarray, b: np.ndarray) -> float:
+    den = float(np.linalg.norm(b))
+    return float(np.linalg.norm(a - b)) / den if den > 0 else float(np.linalg.norm(a))
+
+
+def check_state(o: O.OracleUnit, st: dict, ui: int, rep: ParityReport, where: str) -> None:
+    n, M = o.n, o.M
+    assert int(st["n_tokens"][ui]) == n, f"{where}: token count {st['n_tokens'][ui]} vs oracle {n}"
+    assert int(st["n_ids"][ui]) == M, f"{where}: ids in use {st['n_ids'][ui]} vs oracle {M}"
+    a_gpu = st["tok_cluster"][ui, :n]
+    a_or = o.assign()
+    bad = np.nonzero(a_gpu != a_or)[0]
+    assert bad.size == 0, f"{where}: membership differs at tokens {bad[:8]} gpu {a_gpu[bad[:8]]} oracle {a_or[bad[:8]]}"
+    cnt = o.counts()
+    assert np.array_equal(st["counts"][ui, :M], cnt), f"{where}: cluster sizes differ"
+    Cg, Co = st["centroids"][ui, :M].astype(np.float64), o.centroids()
+    live = cnt > 0
+    if live.any():
+        num = np.linalg.norm(Cg[live] - Co[live], axis=1)
+        den = np.maximum(np.linalg.norm(Co[live], axis=1), 1e-30)
+        r = float((num / den).max())
+        rep.max_centroid_rel = max(rep.max_centroid_rel, r)
+        assert r <= TOL_CENTROID, f"{where}: centroid relative error {r:.3e}"
+        m2g, m2o = st["M2"][ui, :M].astype(np.float64)[live], o.M2()[live]
+        scale = np.maximum(m2o, 1e-3 * max(float(m2o.max()), 1e-30))
+        assert float((np.abs(m2g - m2o) / scale).max()) <= 1e-3, f"{where}: M2 differs"
+
+
+def run_parity(cfg: WorkloadConfig, units: Sequence[int], steps: int, *, assign_mode: int = 0,
+               state_every: int = 1, budget: Optional[int] = None, ctx_units: Optional[Sequence[int]] = None,
+               seed: int = 1234, device: str = "cuda") -> ParityReport:
+    """Run `steps` decode iterations of `cfg`.  The GPU context holds `ctx_units` (default:
+    `units`); the oracle follows the units listed in `units` (a subset of ctx_units)."""
+    rep = ParityReport()
+    ctx_units = list(ctx_units) if ctx_units is not None else list(units)
+    pos = {u: i for i, u in enumerate(ctx_units)}
+    watch = [pos[u] for u in units]
+    budget = cfg.budget if budget is None else budget
+    streams = [UnitStream(cfg, u) for u in ctx_units]
+    K, V = make_prefill(streams)
+    ctx = make_ctx(cfg, len(ctx_units), trace=1, assign_mode=assign_mode)
+    ctx.build_index(K.to(device), V.to(device), cfg.M0, seed)
+    picks, trace = ctx.get_build_trace()
+    st = ctx.export_state()
+    oracles = {}
+    for ui in watch:
+        o = make_oracle(cfg)
+        o.build(K[ui].double().numpy(), V[ui].double().numpy(), cfg.M0, cfg.T, seed, unit_index=ui,
+                init_mode=O.INIT_KMEANSPP if cfg.init_mode == "kmeanspp" else O.INIT_RANDOM,
+                hint_picks=picks[ui] if cfg.init_mode == "kmeanspp" else None, hint_assign=trace[:, ui, :])
+        assert o.violations == 0, f"build unit {ui}: {o.violations} decisions differ beyond the tie tolerance"
+        check_state(o, st, ui, rep, f"build unit {ui}")
+        tau_g, tau_o = float(st["tau"][ui]), o.tau
+        assert abs(tau_g - tau_o) <= 1e-4 * abs(tau_o) + 1e-30, f"tau {tau_g} vs {tau_o}"
+        oracles[ui] = o
+    sel = torch.full((len(ctx_units), cfg.max_clusters), -1, dtype=torch.int32, device=device)
+    done = 0
+    while done < steps:
+        nb = min(64, steps - done)
+        q, k, v = make_decode_chunk(streams, nb)
+        qd, kd, vd = q.to(device), k.to(device), v.to(device)
+        for t in range(nb):
+            out = ctx.decode_step(qd[t], budget, selected_ids=sel)
+            out_np = out.cpu().numpy().astype(np.float64)
+            sel_np = sel.cpu().numpy()
+            nsel, ntok = ctx.get_selection()
+            for ui in watch:
+                o = oracles[ui]
+                ids_gpu = sel_np[ui][: nsel[ui]]
+                assert np.all(sel_np[ui][nsel[ui]:] == -1)
+                v0 = o.violations
+                out_o, ids_o, tok_o = o.decode_step(q[t, ui].double().numpy(), budget, hint_ids=ids_gpu)
+                assert o.violations == v0 and list(ids_o) == list(ids_gpu), \
+                    f"step {done + t} unit {ui}: selection differs: gpu {ids_gpu[:12]} oracle {ids_o[:12]}"
+                assert tok_o == int(ntok[ui])
+                rep.tokens_selected.append(tok_o)
+                ea = float(np.abs(out_np[ui] - out_o).max()); el = rel_l2(out_np[ui], out_o)
+                rep.max_out_abs = max(rep.max_out_abs, ea); rep.max_out_l2 = max(rep.max_out_l2, el)
+                assert ea <= TOL_OUT_ABS and el <= TOL_OUT_L2, \
+                    f"step {done + t} unit {ui}: attention error abs {ea:.3e} relL2 {el:.3e}"
+            ctx.append(kd[t], vd[t])
+            st = ctx.export_state()
+            for ui in watch:
+                o = oracles[ui]
+                n0 = o.n
+                v0 = o.violations
+                j = o.append(k[t, ui].double().numpy(), v[t, ui].double().numpy(),
+                             hint_cluster=int(st["tok_cluster"][ui, n0]))
+                assert o.violations == v0 and j == int(st["tok_cluster"][ui, n0]), \
+                    f"step {done + t} unit {ui}: append target gpu {st['tok_cluster'][ui, n0]} oracle {j}"
+            ctx.split_check()
+            st = ctx.export_state()
+            for ui in watch:
+                o = oracles[ui]
+                v0 = o.violations
+                o.split_check(hint_assign_after=st["tok_cluster"][ui, : o.n])
+                assert o.violations == v0, f"step {done + t} unit {ui}: split decisions differ beyond the tie tolerance"
+                if (done + t) % state_every == 0 or done + t == steps - 1:
+                    check_state(o, st, ui, rep, f"step {done + t} unit {ui}")
+                else:
+                    assert np.array_equal(st["tok_cluster"][ui, : o.n], o.assign()), f"step {done + t} unit {ui}: membership"
+        done += nb
+    status = ctx.get_status()
+    rep.steps = steps
+    rep.status_bits = status["error_bits"]
+    rep.rechecked = status["assign_rechecked"]
+    for ui in watch:
+        o = oracles[ui]
+        rep.ties += o.ties; rep.violations += o.violations; rep.splits += o.n_splits
+    rep.gpu_splits = status["n_splits"]
+    ctx.destroy()
+    return rep

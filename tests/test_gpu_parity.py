@@ -1,0 +1,33 @@
+"""GPU parity tests: the CUDA library against the fp64 oracle through the C ABI."""
+import numpy as np
+import pytest
+import torch
+
+from gen import CONFIGS
+
+pytestmark = pytest.mark.gpu
+
+
+def _run(cfg, units, steps, **kw):
+    from parity_harness import run_parity
+    rep = run_parity(cfg, units, steps, **kw)
+    print(f"\n[{cfg.name}] steps={rep.steps} ties={rep.ties} splits={rep.splits} max_abs={rep.max_out_abs:.2e} "
+          f"max_relL2={rep.max_out_l2:.2e} centroid_rel={rep.max_centroid_rel:.2e} "
+          f"tokens/step={np.mean(rep.tokens_selected):.0f} status={rep.status_bits} rechecked={rep.rechecked}")
+    assert rep.violations == 0
+    return rep
+
+
+def test_config1_full():
+    """Config 1 in full: 2048-key prefill, 64 clusters, 10 rounds from k-means++, 512 decode steps."""
+    rep = _run(CONFIGS[1], [0], CONFIGS[1].steps)
+    assert rep.splits > 0
+
+
+@pytest.mark.parametrize("cid", [2, 3, 4, 5])
+def test_scaled_bf16_configs(cid):
+    """Configs 2-5 at reduced size (several tiles plus a ragged tail), 3 units, fp32 assign path."""
+    base = CONFIGS[cid]
+    cfg = base.scaled(n_prefill=1111 if cid != 3 else 333, steps=96, M0=37 if cid != 3 else 13,
+                      max_clusters=160, budget=300, T=6, new_every=32 if base.new_every else 0)
+    _run(cfg, [0, 1, 2], cfg.steps, assign_mode=1)
