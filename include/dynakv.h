@@ -77,6 +77,8 @@ typedef struct dynakv_status {
     int64_t clusters_selected; /* clusters selected in the last decode step, summed over units   */
     int64_t pages_in_use;      /* 32-token pages holding data, summed over units                 */
     int64_t assign_rechecked;  /* keys whose tensor-core argmin was re-decided in fp32 (build)   */
+    int64_t tokens_attended_total;   /* tokens attended, summed over units and all decode steps  */
+    int64_t clusters_selected_total; /* clusters selected, summed over units and all decode steps */
 } dynakv_status;
 
 /* Create a context on the current CUDA device; all later work runs on `cuda_stream`
@@ -129,7 +131,9 @@ int dynakv_split_check(dynakv_ctx* ctx);
 /* n_steps iterations of { decode_step(q_t); append(k_t, v_t); split_check() } (the order
  * of Algorithm 1's loop body), replayed from one captured CUDA graph whose kernels read
  * the step index from device memory.  q_steps: [n_steps][U][G][d] fp32, k_steps,
- * v_steps: [n_steps][U][d] kv_dtype, out_steps: [n_steps][U][G][d] fp32, all device. */
+ * v_steps: [n_steps][U][d] kv_dtype, out_steps: [n_steps][U][G][d] fp32, all device.
+ * The context must have been created on a non-default stream (stream capture), else
+ * DYNAKV_ERR_STATE. */
 int dynakv_decode_loop(dynakv_ctx* ctx, const float* q_steps, const void* k_steps,
                        const void* v_steps, int64_t n_steps, int32_t token_budget,
                        float* out_steps);
@@ -160,6 +164,24 @@ int dynakv_get_selection(dynakv_ctx* ctx, int32_t* n_selected, int32_t* tokens_s
  * centres, in centre order) and assign [T][U][n] (assignment of every Lloyd round);
  * either may be NULL.  Returns DYNAKV_ERR_STATE if tracing was off. */
 int dynakv_get_build_trace(dynakv_ctx* ctx, int32_t* picks, int32_t* assign);
+
+/* Measurement aid (no counterpart in the paper).  With timing on, every kernel launched
+ * by a direct call (not by dynakv_decode_loop's graph replay) is bracketed by CUDA events on
+ * the context's stream.  dynakv_get_kernel_times synchronises and returns, per kernel class,
+ * the summed event time in ms and the number of launches since the last reset, into HOST
+ * arrays of DYNAKV_KC_COUNT entries. */
+#define DYNAKV_KC_INIT 0
+#define DYNAKV_KC_ASSIGN 1
+#define DYNAKV_KC_UPDATE 2
+#define DYNAKV_KC_FINALIZE 3
+#define DYNAKV_KC_SELECT 4
+#define DYNAKV_KC_ATTN 5
+#define DYNAKV_KC_COMBINE 6
+#define DYNAKV_KC_APPEND 7
+#define DYNAKV_KC_SPLIT 8
+#define DYNAKV_KC_COUNT 9
+int dynakv_set_timing(dynakv_ctx* ctx, int32_t on);
+int dynakv_get_kernel_times(dynakv_ctx* ctx, double* ms_total, int64_t* launches, int32_t reset);
 
 /* Number of kernels this context has launched so far (graph replays count their nodes). */
 int64_t dynakv_launch_count(dynakv_ctx* ctx);

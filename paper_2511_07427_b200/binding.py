@@ -18,7 +18,7 @@ ST_BUDGET_EXCEEDED, ST_MAX_CLUSTERS, ST_MAX_TOKENS, ST_PAGE_POOL, ST_INTERNAL = 
 EXPORTED_SYMBOLS = [
     "dynakv_create", "dynakv_build_index", "dynakv_append", "dynakv_decode_step", "dynakv_split_check",
     "dynakv_decode_loop", "dynakv_step_host", "dynakv_get_status", "dynakv_export_state", "dynakv_get_selection",
-    "dynakv_get_build_trace", "dynakv_launch_count", "dynakv_last_error", "dynakv_destroy",
+    "dynakv_get_build_trace", "dynakv_set_timing", "dynakv_get_kernel_times", "dynakv_launch_count", "dynakv_last_error", "dynakv_destroy",
 ]
 
 
@@ -37,7 +37,10 @@ class _Config(C.Structure):
 class _Status(C.Structure):
     _fields_ = [("error_bits", C.c_uint32), ("reserved", C.c_int32), ("n_appended", C.c_int64),
                 ("n_splits", C.c_int64), ("tokens_selected", C.c_int64), ("clusters_selected", C.c_int64),
-                ("pages_in_use", C.c_int64), ("assign_rechecked", C.c_int64)]
+                ("pages_in_use", C.c_int64), ("assign_rechecked", C.c_int64), ("tokens_attended_total", C.c_int64),
+                ("clusters_selected_total", C.c_int64)]
+
+KERNEL_CLASSES = ["init", "assign", "update", "finalize", "select", "attn", "combine", "append", "split"]
 
 
 @dataclass
@@ -93,6 +96,10 @@ def load_library() -> C.CDLL:
     L.dynakv_get_selection.argtypes = [vp, vp, vp]
     L.dynakv_get_build_trace.restype = C.c_int
     L.dynakv_get_build_trace.argtypes = [vp, vp, vp]
+    L.dynakv_set_timing.restype = C.c_int
+    L.dynakv_set_timing.argtypes = [vp, i32]
+    L.dynakv_get_kernel_times.restype = C.c_int
+    L.dynakv_get_kernel_times.argtypes = [vp, vp, vp, i32]
     L.dynakv_launch_count.restype = C.c_int64
     L.dynakv_launch_count.argtypes = [vp]
     L.dynakv_last_error.restype = C.c_char_p
@@ -231,6 +238,15 @@ class DynaKV:
         assign = np.empty((T, U, self.n_prefill), np.int32)
         self._check(self._L.dynakv_get_build_trace(self._h, _np_ptr(picks), _np_ptr(assign)), "dynakv_get_build_trace")
         return picks, assign
+
+    def set_timing(self, on: bool) -> None:
+        self._check(self._L.dynakv_set_timing(self._h, 1 if on else 0), "dynakv_set_timing")
+
+    def get_kernel_times(self, reset: bool = True) -> dict:
+        ms = np.zeros(len(KERNEL_CLASSES), np.float64); n = np.zeros(len(KERNEL_CLASSES), np.int64)
+        self._check(self._L.dynakv_get_kernel_times(self._h, _np_ptr(ms), _np_ptr(n), 1 if reset else 0),
+                    "dynakv_get_kernel_times")
+        return {k: {"ms": float(ms[i]), "launches": int(n[i])} for i, k in enumerate(KERNEL_CLASSES)}
 
     def launch_count(self) -> int:
         return int(self._L.dynakv_launch_count(self._h))

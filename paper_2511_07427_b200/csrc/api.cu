@@ -40,6 +40,32 @@ struct dynakv_ctx {
     long long graph_nodes = 0;
     // staging for dynakv_step_host
     float* st_q = nullptr; void* st_k = nullptr; void* st_v = nullptr; float* st_out = nullptr;
+    // optional per-kernel event timing (off inside graph capture)
+    bool timing = false;
+    struct Span { int kc; cudaEvent_t e0, e1; };
+    std::vector<Span> spans;
+    std::vector<cudaEvent_t> event_pool;
+    double kc_ms[KC_COUNT] = {0};
+    long long kc_n[KC_COUNT] = {0};
+};
+
+// Scope that brackets one kernel launch with events when timing is on.
+struct TimeScope {
+    dynakv_ctx* c; bool on; dynakv_ctx::Span sp;
+    TimeScope(dynakv_ctx* c_, int kc, bool allowed = true) : c(c_), on(c_->timing && allowed) {
+        if (!on) return;
+        sp.kc = kc;
+        for (cudaEvent_t* e : {&sp.e0, &sp.e1}) {
+            if (!c->event_pool.empty()) { *e = c->event_pool.back(); c->event_pool.pop_back(); }
+            else cudaEventCreate(e);
+        }
+        cudaEventRecord(sp.e0, c->stream);
+    }
+    ~TimeScope() {
+        if (!on) return;
+        cudaEventRecord(sp.e1, c->stream);
+        c->spans.push_back(sp);
+    }
 };
 
 #define CK(call)                                                                                   \
@@ -151,6 +177,8 @@ extern "C" void dynakv_destroy(dynakv_ctx* c) {
     if (!c) return;
     cudaStreamSynchronize(c->stream);
     if (c->graph_exec) cudaGraphExecDestroy(c->graph_exec);
+    for (auto& sp : c->spans) { cudaEventDestroy(sp.e0); cudaEventDestroy(sp.e1); }
+    for (cudaEvent_t e : c->event_pool) cudaEventDestroy(e);
     for (void* p : c->allocs) cudaFree(p);
     delete c;
 }
@@ -179,14 +207,17 @@ extern "C" int dynakv_build_index(dynakv_ctx* c, const void* K, const void* V, i
     void* tc_scratch = nullptr;
     if (use_tc) { char* p; ALLOC_B(p, tc_assign_scratch_bytes(t, n, M), false); tc_scratch = p; }
 
-    launch_init_centres(t, K, n, M, seed, c->cfg.init_mode, b, c->stream, &c->launches);
+    { TimeScope ts(c, KC_INIT); launch_init_centres(t, K, n, M, seed, c->cfg.init_mode, b, c->stream, &c->launches); }
     for (int it = 0; it < T; it++) {
         b.assign = c->cfg.trace ? c->trace_assign + (size_t)it * U * n : assign_buf;
-        if (use_tc) launch_assign_tc(t, K, n, M, b.C, b.assign, tc_scratch, c->stream, &c->launches);
-        else launch_assign_f32(t, K, n, M, b.C, b.assign, c->stream, &c->launches);
-        launch_update(t, K, n, M, b.assign, b, c->stream, &c->launches);
+        {
+            TimeScope ts(c, KC_ASSIGN);
+            if (use_tc) launch_assign_tc(t, K, n, M, b.C, b.assign, tc_scratch, c->stream, &c->launches);
+            else launch_assign_f32(t, K, n, M, b.C, b.assign, c->stream, &c->launches);
+        }
+        { TimeScope ts(c, KC_UPDATE); launch_update(t, K, n, M, b.assign, b, c->stream, &c->launches); }
     }
-    launch_finalize(t, K, V, n, M, b, c->cfg.split_var_factor, c->stream, &c->launches);
+    { TimeScope ts(c, KC_FINALIZE); launch_finalize(t, K, V, n, M, b, c->cfg.split_var_factor, c->stream, &c->launches); }
     CK(cudaGetLastError());
     CK(cudaStreamSynchronize(c->stream));
     // keep the picks for the trace; free the rest of the build scratch
@@ -203,10 +234,16 @@ extern "C" int dynakv_build_index(dynakv_ctx* c, const void* K, const void* V, i
     return DYNAKV_OK;
 }
 
-static int enqueue_decode(dynakv_ctx* c, StepPtr q, int budget, StepPtrW out, int* sel_ids) {
-    launch_score_select(c->t, q, budget, sel_ids, c->stream, &c->launches);
-    launch_gather_attn(c->t, q, out, c->stream, &c->launches);
+static int enqueue_decode(dynakv_ctx* c, StepPtr q, int budget, StepPtrW out, int* sel_ids, bool timed = true) {
+    { TimeScope ts(c, KC_SELECT, timed); launch_score_select(c->t, q, budget, sel_ids, c->stream, &c->launches); }
+    { TimeScope ts(c, KC_ATTN, timed); launch_gather_attn_v1(c->t, q, c->stream, &c->launches); }
+    { TimeScope ts(c, KC_COMBINE, timed); launch_attn_combine(c->t, out, c->stream, &c->launches); }
     return DYNAKV_OK;
+}
+
+static void enqueue_append(dynakv_ctx* c, StepPtr k, StepPtr v, bool timed = true) {
+    TimeScope ts(c, KC_APPEND, timed);
+    launch_append(c->t, k, v, c->stream, &c->launches);
 }
 
 extern "C" int dynakv_decode_step(dynakv_ctx* c, const float* q, int32_t token_budget, float* out, int32_t* selected_ids) {
@@ -220,12 +257,13 @@ extern "C" int dynakv_decode_step(dynakv_ctx* c, const float* q, int32_t token_b
 extern "C" int dynakv_append(dynakv_ctx* c, const void* k, const void* v) {
     if (!c || !k || !v) return DYNAKV_ERR_ARG;
     if (!c->built) return DYNAKV_ERR_STATE;
-    launch_append(c->t, StepPtr{k, 0, nullptr}, StepPtr{v, 0, nullptr}, c->stream, &c->launches);
+    enqueue_append(c, StepPtr{k, 0, nullptr}, StepPtr{v, 0, nullptr});
     CK(cudaGetLastError());
     return DYNAKV_OK;
 }
 
-static void enqueue_split(dynakv_ctx* c) {
+static void enqueue_split(dynakv_ctx* c, bool timed = true) {
+    TimeScope ts(c, KC_SPLIT, timed);
     launch_split_check(c->t, c->cfg.split_size_factor, c->cfg.split_var_factor > 0.f ? 1 : 0, c->cfg.split_min_size,
                        c->cfg.split_iters, c->stream, &c->launches);
 }
@@ -242,6 +280,10 @@ extern "C" int dynakv_decode_loop(dynakv_ctx* c, const float* q_steps, const voi
                                   int64_t n_steps, int32_t token_budget, float* out_steps) {
     if (!c || !q_steps || !k_steps || !v_steps || !out_steps || n_steps < 0 || token_budget < 0) return DYNAKV_ERR_ARG;
     if (!c->built) return DYNAKV_ERR_STATE;
+    if (c->stream == nullptr || c->stream == cudaStreamLegacy) {
+        snprintf(g_err, sizeof(g_err), "dynakv_decode_loop captures a CUDA graph and needs a context created on a non-default stream");
+        return DYNAKV_ERR_STATE;
+    }
     const Tables& t = c->t;
     if (!c->graph_exec || c->g_q != q_steps || c->g_k != k_steps || c->g_v != v_steps || c->g_out != out_steps ||
         c->g_budget != token_budget) {
@@ -250,9 +292,9 @@ extern "C" int dynakv_decode_loop(dynakv_ctx* c, const float* q_steps, const voi
         cudaGraph_t graph = nullptr;
         long long before = c->launches;
         CK(cudaStreamBeginCapture(c->stream, cudaStreamCaptureModeThreadLocal));
-        enqueue_decode(c, StepPtr{q_steps, qs, c->step_ctr}, token_budget, StepPtrW{out_steps, qs, c->step_ctr}, nullptr);
-        launch_append(t, StepPtr{k_steps, ks, c->step_ctr}, StepPtr{v_steps, ks, c->step_ctr}, c->stream, &c->launches);
-        enqueue_split(c);
+        enqueue_decode(c, StepPtr{q_steps, qs, c->step_ctr}, token_budget, StepPtrW{out_steps, qs, c->step_ctr}, nullptr, false);
+        enqueue_append(c, StepPtr{k_steps, ks, c->step_ctr}, StepPtr{v_steps, ks, c->step_ctr}, false);
+        enqueue_split(c, false);
         launch_step_inc(c->step_ctr, c->stream, &c->launches);
         cudaError_t e = cudaStreamEndCapture(c->stream, &graph);
         c->graph_nodes = c->launches - before;
@@ -286,7 +328,7 @@ extern "C" int dynakv_step_host(dynakv_ctx* c, const float* q_host, const void* 
     CK(cudaMemcpyAsync(c->st_k, k_host, kb, cudaMemcpyHostToDevice, c->stream));
     CK(cudaMemcpyAsync(c->st_v, v_host, kb, cudaMemcpyHostToDevice, c->stream));
     enqueue_decode(c, StepPtr{c->st_q, 0, nullptr}, token_budget, StepPtrW{c->st_out, 0, nullptr}, nullptr);
-    launch_append(t, StepPtr{c->st_k, 0, nullptr}, StepPtr{c->st_v, 0, nullptr}, c->stream, &c->launches);
+    enqueue_append(c, StepPtr{c->st_k, 0, nullptr}, StepPtr{c->st_v, 0, nullptr});
     enqueue_split(c);
     CK(cudaMemcpyAsync(out_host, c->st_out, qb, cudaMemcpyDeviceToHost, c->stream));
     CK(cudaStreamSynchronize(c->stream));
@@ -316,6 +358,8 @@ extern "C" int dynakv_get_status(dynakv_ctx* c, dynakv_status* host_out) {
     host_out->n_appended = (int64_t)cnt[CNT_APPENDED];
     host_out->n_splits = (int64_t)cnt[CNT_SPLITS];
     host_out->assign_rechecked = (int64_t)cnt[CNT_RECHECKED];
+    host_out->tokens_attended_total = (int64_t)cnt[CNT_TOKENS_ATTENDED];
+    host_out->clusters_selected_total = (int64_t)cnt[CNT_CLUSTERS_SELECTED];
     host_out->tokens_selected = (int64_t)cnt[4];
     host_out->clusters_selected = (int64_t)cnt[5];
     host_out->pages_in_use = (int64_t)cnt[6];
@@ -357,6 +401,28 @@ extern "C" int dynakv_get_build_trace(dynakv_ctx* c, int32_t* picks, int32_t* as
     if (assign) CK(cudaMemcpyAsync(assign, c->trace_assign, sizeof(int) * (size_t)c->cfg.kmeans_iters * U * c->n_prefill,
                                    cudaMemcpyDeviceToHost, c->stream));
     CK(cudaStreamSynchronize(c->stream));
+    return DYNAKV_OK;
+}
+
+extern "C" int dynakv_set_timing(dynakv_ctx* c, int32_t on) {
+    if (!c) return DYNAKV_ERR_ARG;
+    c->timing = on != 0;
+    return DYNAKV_OK;
+}
+
+extern "C" int dynakv_get_kernel_times(dynakv_ctx* c, double* ms_total, int64_t* launches, int32_t reset) {
+    if (!c || !ms_total || !launches) return DYNAKV_ERR_ARG;
+    CK(cudaStreamSynchronize(c->stream));
+    for (auto& sp : c->spans) {
+        float ms = 0.f;
+        if (cudaEventElapsedTime(&ms, sp.e0, sp.e1) == cudaSuccess) { c->kc_ms[sp.kc] += ms; c->kc_n[sp.kc]++; }
+        c->event_pool.push_back(sp.e0); c->event_pool.push_back(sp.e1);
+    }
+    c->spans.clear();
+    for (int k = 0; k < KC_COUNT; k++) {
+        ms_total[k] = c->kc_ms[k]; launches[k] = c->kc_n[k];
+        if (reset) { c->kc_ms[k] = 0; c->kc_n[k] = 0; }
+    }
     return DYNAKV_OK;
 }
 

@@ -45,10 +45,10 @@ struct Tables {
     int* sp_pos;                     // [U][2 * max_tokens]: rank per position, then hole list
     // status / counters
     unsigned int* status;            // [1]
-    unsigned long long* counters;    // [8]: 0 appended, 1 splits, 2 rechecked
+    unsigned long long* counters;    // [8]: see CNT_*; 4..6 are scratch of get_status
 };
 
-enum { CNT_APPENDED = 0, CNT_SPLITS = 1, CNT_RECHECKED = 2 };
+enum { CNT_APPENDED = 0, CNT_SPLITS = 1, CNT_RECHECKED = 2, CNT_TOKENS_ATTENDED = 3, CNT_CLUSTERS_SELECTED = 7 };
 
 // A per-step operand: base pointer plus a stride applied with the device-side step index,
 // so the same kernel serves a direct call (ctr == nullptr) and a captured graph replay.
@@ -128,6 +128,10 @@ __device__ __forceinline__ unsigned int hash23(unsigned long long seed, int unit
     return (unsigned int)(x >> 41);
 }
 
+// Kernel classes for the optional per-kernel event timing.
+enum { KC_INIT = 0, KC_ASSIGN = 1, KC_UPDATE = 2, KC_FINALIZE = 3, KC_SELECT = 4, KC_ATTN = 5, KC_COMBINE = 6,
+       KC_APPEND = 7, KC_SPLIT = 8, KC_COUNT = 9 };
+
 // ---- host launchers (defined in the kernel files) ---------------------------------------
 struct BuildScratch {
     float* C;            // [U][M][d] current centres
@@ -148,7 +152,8 @@ void launch_update(const Tables& t, const void* K, long long n, int M, const int
 void launch_finalize(const Tables& t, const void* K, const void* V, long long n, int M, const BuildScratch& b,
                      float alpha, cudaStream_t s, long long* launches);
 void launch_score_select(const Tables& t, StepPtr q, int budget, int* user_sel_ids, cudaStream_t s, long long* launches);
-void launch_gather_attn(const Tables& t, StepPtr q, StepPtrW out, cudaStream_t s, long long* launches);
+void launch_gather_attn_v1(const Tables& t, StepPtr q, cudaStream_t s, long long* launches);
+void launch_attn_combine(const Tables& t, StepPtrW out, cudaStream_t s, long long* launches);
 void launch_append(const Tables& t, StepPtr k, StepPtr v, cudaStream_t s, long long* launches);
 void launch_split_check(const Tables& t, float gamma, int var_enabled, int min_size, int iters, cudaStream_t s,
                         long long* launches);

@@ -124,6 +124,8 @@ __global__ void __launch_bounds__(SS_THREADS) k_score_select(Tables t, StepPtr q
         t.sel_n[u] = L;
         t.sel_tokens[u] = tokens;
         t.n_work[u] = min(wbase, t.W);
+        atomicAdd(&t.counters[CNT_TOKENS_ATTENDED], (unsigned long long)tokens);
+        atomicAdd(&t.counters[CNT_CLUSTERS_SELECTED], (unsigned long long)L);
     }
     if (user_ids) {
         int* uo = user_ids + (size_t)u * t.max_clusters;
@@ -331,7 +333,7 @@ void launch_score_select(const Tables& t, StepPtr q, int budget, int* user_sel_i
 }
 
 template <typename KV, int HD>
-static void gather_attn_t(const Tables& t, StepPtr q, StepPtrW out, cudaStream_t s, long long* launches) {
+static void gather_attn_t(const Tables& t, StepPtr q, cudaStream_t s, long long* launches) {
     dim3 grid(t.n_splits_attn, t.U);
     switch (t.G) {
         case 1: k_gather_attn_v1<KV, HD, 1><<<grid, 128, 0, s>>>(t, q); break;
@@ -343,16 +345,21 @@ static void gather_attn_t(const Tables& t, StepPtr q, StepPtrW out, cudaStream_t
         case 7: k_gather_attn_v1<KV, HD, 7><<<grid, 128, 0, s>>>(t, q); break;
         default: k_gather_attn_v1<KV, HD, 8><<<grid, 128, 0, s>>>(t, q); break;
     }
-    k_attn_combine<HD><<<t.U, 256, 0, s>>>(t, out, t.n_splits_attn);
-    (*launches) += 2;
+    (*launches)++;
 }
 
-void launch_gather_attn(const Tables& t, StepPtr q, StepPtrW out, cudaStream_t s, long long* launches) {
+void launch_gather_attn_v1(const Tables& t, StepPtr q, cudaStream_t s, long long* launches) {
     if (t.kv_dtype == DYNAKV_F32) {
-        if (t.d == 64) gather_attn_t<float, 64>(t, q, out, s, launches); else gather_attn_t<float, 128>(t, q, out, s, launches);
+        if (t.d == 64) gather_attn_t<float, 64>(t, q, s, launches); else gather_attn_t<float, 128>(t, q, s, launches);
     } else {
-        if (t.d == 64) gather_attn_t<__nv_bfloat16, 64>(t, q, out, s, launches); else gather_attn_t<__nv_bfloat16, 128>(t, q, out, s, launches);
+        if (t.d == 64) gather_attn_t<__nv_bfloat16, 64>(t, q, s, launches); else gather_attn_t<__nv_bfloat16, 128>(t, q, s, launches);
     }
+}
+
+void launch_attn_combine(const Tables& t, StepPtrW out, cudaStream_t s, long long* launches) {
+    if (t.d == 64) k_attn_combine<64><<<t.U, 256, 0, s>>>(t, out, t.n_splits_attn);
+    else k_attn_combine<128><<<t.U, 256, 0, s>>>(t, out, t.n_splits_attn);
+    (*launches)++;
 }
 
 void launch_append(const Tables& t, StepPtr k, StepPtr v, cudaStream_t s, long long* launches) {
