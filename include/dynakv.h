@@ -66,6 +66,7 @@ typedef struct dynakv_config {
     int32_t split_iters;       /* cap on 2-means rounds in a split                               */
     int32_t trace;             /* 1: keep every Lloyd round's assignment for dynakv_get_build_trace */
     int32_t assign_mode;       /* 0: auto (tensor-core distance GEMM for bf16, d=128), 1: force fp32 path */
+    int32_t attn_mode;         /* 0: auto (tensor-core gather-attention for bf16 K/V), 1: force the plain fp32 kernel */
 } dynakv_config;
 
 typedef struct dynakv_status {
@@ -179,7 +180,8 @@ int dynakv_get_build_trace(dynakv_ctx* ctx, int32_t* picks, int32_t* assign);
 #define DYNAKV_KC_COMBINE 6
 #define DYNAKV_KC_APPEND 7
 #define DYNAKV_KC_SPLIT 8
-#define DYNAKV_KC_COUNT 9
+#define DYNAKV_KC_FRONT 9
+#define DYNAKV_KC_COUNT 10
 int dynakv_set_timing(dynakv_ctx* ctx, int32_t on);
 int dynakv_get_kernel_times(dynakv_ctx* ctx, double* ms_total, int64_t* launches, int32_t reset);
 

@@ -152,6 +152,8 @@ extern "C" int dynakv_create(const dynakv_config* cfg, void* cuda_stream, dynakv
     ALLOC(t.u_page_top, U, true); ALLOC(t.u_free_cnt, U, true);
     ALLOC(t.tok_cluster, U * (size_t)t.max_tokens, false);
     ALLOC(t.scores, U * Mx, true);
+    ALLOC(t.dists, U * Mx, true);
+    ALLOC(t.u_scan, U, true); ALLOC(t.u_last, U, true);
     ALLOC(t.sel_ids, U * Mx, true);
     ALLOC(t.sel_n, U, true); ALLOC(t.sel_tokens, U, true);
     ALLOC(t.work, U * (size_t)t.W, false);
@@ -234,22 +236,39 @@ extern "C" int dynakv_build_index(dynakv_ctx* c, const void* K, const void* V, i
     return DYNAKV_OK;
 }
 
-static int enqueue_decode(dynakv_ctx* c, StepPtr q, int budget, StepPtrW out, int* sel_ids, bool timed = true) {
-    { TimeScope ts(c, KC_SELECT, timed); launch_score_select(c->t, q, budget, sel_ids, c->stream, &c->launches); }
-    { TimeScope ts(c, KC_ATTN, timed); launch_gather_attn_v1(c->t, q, c->stream, &c->launches); }
-    { TimeScope ts(c, KC_COMBINE, timed); launch_attn_combine(c->t, out, c->stream, &c->launches); }
-    return DYNAKV_OK;
+static void enqueue_front(dynakv_ctx* c, StepPtr q, StepPtr k, int has_q, int has_k, bool timed) {
+    TimeScope ts(c, KC_FRONT, timed);
+    launch_front(c->t, q, k, has_q, has_k, c->stream, &c->launches);
 }
 
-static void enqueue_append(dynakv_ctx* c, StepPtr k, StepPtr v, bool timed = true) {
+// select -> gather attention -> combine, on scores already written by the front pass
+static void enqueue_retrieve(dynakv_ctx* c, StepPtr q, int budget, StepPtrW out, int* sel_ids, bool timed) {
+    { TimeScope ts(c, KC_SELECT, timed); launch_select(c->t, budget, sel_ids, c->stream, &c->launches); }
+    {
+        TimeScope ts(c, KC_ATTN, timed);
+        if (c->t.kv_dtype == DYNAKV_BF16 && c->cfg.attn_mode == 0) launch_gather_attn_mma(c->t, q, c->stream, &c->launches);
+        else launch_gather_attn_v1(c->t, q, c->stream, &c->launches);
+    }
+    { TimeScope ts(c, KC_COMBINE, timed); launch_attn_combine(c->t, out, c->stream, &c->launches); }
+}
+
+static void enqueue_append_apply(dynakv_ctx* c, StepPtr k, StepPtr v, bool timed) {
     TimeScope ts(c, KC_APPEND, timed);
-    launch_append(c->t, k, v, c->stream, &c->launches);
+    launch_append_apply(c->t, k, v, c->stream, &c->launches);
+}
+
+// one whole loop iteration: a single centroid pass serves both the query scores and the new key's distances
+static void enqueue_step(dynakv_ctx* c, StepPtr q, StepPtr k, StepPtr v, int budget, StepPtrW out, bool timed) {
+    enqueue_front(c, q, k, 1, 1, timed);
+    enqueue_retrieve(c, q, budget, out, nullptr, timed);
+    enqueue_append_apply(c, k, v, timed);
 }
 
 extern "C" int dynakv_decode_step(dynakv_ctx* c, const float* q, int32_t token_budget, float* out, int32_t* selected_ids) {
     if (!c || !q || !out || token_budget < 0) return DYNAKV_ERR_ARG;
     if (!c->built) return DYNAKV_ERR_STATE;
-    enqueue_decode(c, StepPtr{q, 0, nullptr}, token_budget, StepPtrW{out, 0, nullptr}, selected_ids);
+    enqueue_front(c, StepPtr{q, 0, nullptr}, StepPtr{nullptr, 0, nullptr}, 1, 0, true);
+    enqueue_retrieve(c, StepPtr{q, 0, nullptr}, token_budget, StepPtrW{out, 0, nullptr}, selected_ids, true);
     CK(cudaGetLastError());
     return DYNAKV_OK;
 }
@@ -257,7 +276,8 @@ extern "C" int dynakv_decode_step(dynakv_ctx* c, const float* q, int32_t token_b
 extern "C" int dynakv_append(dynakv_ctx* c, const void* k, const void* v) {
     if (!c || !k || !v) return DYNAKV_ERR_ARG;
     if (!c->built) return DYNAKV_ERR_STATE;
-    enqueue_append(c, StepPtr{k, 0, nullptr}, StepPtr{v, 0, nullptr});
+    enqueue_front(c, StepPtr{nullptr, 0, nullptr}, StepPtr{k, 0, nullptr}, 0, 1, true);
+    enqueue_append_apply(c, StepPtr{k, 0, nullptr}, StepPtr{v, 0, nullptr}, true);
     CK(cudaGetLastError());
     return DYNAKV_OK;
 }
@@ -292,8 +312,8 @@ extern "C" int dynakv_decode_loop(dynakv_ctx* c, const float* q_steps, const voi
         cudaGraph_t graph = nullptr;
         long long before = c->launches;
         CK(cudaStreamBeginCapture(c->stream, cudaStreamCaptureModeThreadLocal));
-        enqueue_decode(c, StepPtr{q_steps, qs, c->step_ctr}, token_budget, StepPtrW{out_steps, qs, c->step_ctr}, nullptr, false);
-        enqueue_append(c, StepPtr{k_steps, ks, c->step_ctr}, StepPtr{v_steps, ks, c->step_ctr}, false);
+        enqueue_step(c, StepPtr{q_steps, qs, c->step_ctr}, StepPtr{k_steps, ks, c->step_ctr},
+                     StepPtr{v_steps, ks, c->step_ctr}, token_budget, StepPtrW{out_steps, qs, c->step_ctr}, false);
         enqueue_split(c, false);
         launch_step_inc(c->step_ctr, c->stream, &c->launches);
         cudaError_t e = cudaStreamEndCapture(c->stream, &graph);
@@ -327,8 +347,8 @@ extern "C" int dynakv_step_host(dynakv_ctx* c, const float* q_host, const void* 
     CK(cudaMemcpyAsync(c->st_q, q_host, qb, cudaMemcpyHostToDevice, c->stream));
     CK(cudaMemcpyAsync(c->st_k, k_host, kb, cudaMemcpyHostToDevice, c->stream));
     CK(cudaMemcpyAsync(c->st_v, v_host, kb, cudaMemcpyHostToDevice, c->stream));
-    enqueue_decode(c, StepPtr{c->st_q, 0, nullptr}, token_budget, StepPtrW{c->st_out, 0, nullptr}, nullptr);
-    enqueue_append(c, StepPtr{c->st_k, 0, nullptr}, StepPtr{c->st_v, 0, nullptr});
+    enqueue_step(c, StepPtr{c->st_q, 0, nullptr}, StepPtr{c->st_k, 0, nullptr}, StepPtr{c->st_v, 0, nullptr},
+                 token_budget, StepPtrW{c->st_out, 0, nullptr}, true);
     enqueue_split(c);
     CK(cudaMemcpyAsync(out_host, c->st_out, qb, cudaMemcpyDeviceToHost, c->stream));
     CK(cudaStreamSynchronize(c->stream));

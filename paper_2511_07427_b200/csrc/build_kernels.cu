@@ -283,6 +283,7 @@ __global__ void __launch_bounds__(1024) k_fin_layout(Tables t, int n, int M, con
     __syncthreads();
     if (tid == 0) {
         t.u_N[u] = n; t.u_M[u] = M; t.u_Mlive[u] = s_live; t.u_page_top[u] = page_base; t.u_free_cnt[u] = 0;
+        t.u_scan[u] = 1; t.u_last[u] = -1;
     }
     for (int i = n + tid; i < t.max_tokens; i += blockDim.x) t.tok_cluster[(size_t)u * t.max_tokens + i] = -1;
 }

@@ -32,9 +32,11 @@ struct Tables {
     int* cl_head; int* cl_tail;      // [U][Mmax]
     unsigned char* cl_flags;         // [U][Mmax]
     int* u_N; int* u_M; int* u_Mlive; float* u_tau; int* u_page_top; int* u_free_cnt;   // [U]
+    int* u_scan; int* u_last;        // [U] split check: full scan needed; cluster of the last append (-1 none)
     int* tok_cluster;                // [U][max_tokens]
     // decode scratch
     float* scores;                   // [U][Mmax]
+    float* dists;                    // [U][Mmax] squared distance of the step's new key to every representative
     int* sel_ids;                    // [U][Mmax]
     int* sel_n; int* sel_tokens;     // [U]
     int2* work;                      // [U][W] (page, count)
@@ -130,7 +132,7 @@ __device__ __forceinline__ unsigned int hash23(unsigned long long seed, int unit
 
 // Kernel classes for the optional per-kernel event timing.
 enum { KC_INIT = 0, KC_ASSIGN = 1, KC_UPDATE = 2, KC_FINALIZE = 3, KC_SELECT = 4, KC_ATTN = 5, KC_COMBINE = 6,
-       KC_APPEND = 7, KC_SPLIT = 8, KC_COUNT = 9 };
+       KC_APPEND = 7, KC_SPLIT = 8, KC_FRONT = 9, KC_COUNT = 10 };
 
 // ---- host launchers (defined in the kernel files) ---------------------------------------
 struct BuildScratch {
@@ -151,10 +153,12 @@ void launch_update(const Tables& t, const void* K, long long n, int M, const int
                    cudaStream_t s, long long* launches);
 void launch_finalize(const Tables& t, const void* K, const void* V, long long n, int M, const BuildScratch& b,
                      float alpha, cudaStream_t s, long long* launches);
-void launch_score_select(const Tables& t, StepPtr q, int budget, int* user_sel_ids, cudaStream_t s, long long* launches);
+void launch_front(const Tables& t, StepPtr q, StepPtr k, int has_q, int has_k, cudaStream_t s, long long* launches);
+void launch_select(const Tables& t, int budget, int* user_sel_ids, cudaStream_t s, long long* launches);
+void launch_append_apply(const Tables& t, StepPtr k, StepPtr v, cudaStream_t s, long long* launches);
+void launch_gather_attn_mma(const Tables& t, StepPtr q, cudaStream_t s, long long* launches);
 void launch_gather_attn_v1(const Tables& t, StepPtr q, cudaStream_t s, long long* launches);
 void launch_attn_combine(const Tables& t, StepPtrW out, cudaStream_t s, long long* launches);
-void launch_append(const Tables& t, StepPtr k, StepPtr v, cudaStream_t s, long long* launches);
 void launch_split_check(const Tables& t, float gamma, int var_enabled, int min_size, int iters, cudaStream_t s,
                         long long* launches);
 void launch_step_inc(int* ctr, cudaStream_t s, long long* launches);

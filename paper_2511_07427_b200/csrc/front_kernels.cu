@@ -1,0 +1,371 @@
+// Front half of a decode step (arXiv 2511.07427, Section 4.1 and Algorithm 1):
+//   k_front          one streaming pass over the fp32 representatives that produces both
+//                    the query scores ("similarity scores between q and all
+//                    representatives") and the new key's squared distances ("assign new KV
+//                    entry to its nearest cluster"), so the centroid table is read once;
+//   k_select         budgeted top-cluster selection by weighted radix select on the scores,
+//                    then the flat (page, rows) work list of the selected clusters;
+//   k_append_apply   argmin of the distances, incremental statistics, slot claim.
+#include <float.h>
+
+#include "common.cuh"
+
+namespace dkv {
+
+__device__ __forceinline__ unsigned int ord_key(float f) {
+    unsigned int b = __float_as_uint(f);
+    return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
+}
+
+// ------------------------------------------------------------------ k_front
+
+constexpr int FR_THREADS = 256;
+constexpr int FR_ROWS = 128;      // representatives per block
+
+// Grid (ceil(max_clusters / FR_ROWS), U).  Eight lanes share one representative row (each
+// lane reads HD/8 floats as float4s), four rows per warp instruction.
+template <typename KV, int HD>
+__global__ void __launch_bounds__(FR_THREADS) k_front(Tables t, StepPtr qp, StepPtr kp, int has_q, int has_k) {
+    constexpr int V4 = HD / 32;   // float4 loads per lane per row
+    const int u = blockIdx.y;
+    const int Mcur = t.u_M[u];
+    const int j0 = blockIdx.x * FR_ROWS;
+    if (j0 >= Mcur) return;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int sub = lane >> 3, l8 = lane & 7;
+    float qs[V4][4], kk[V4][4];
+#pragma unroll
+    for (int i = 0; i < V4; i++)
+#pragma unroll
+        for (int e = 0; e < 4; e++) { qs[i][e] = 0.f; kk[i][e] = 0.f; }
+    if (has_q) {
+        const float* q = reinterpret_cast<const float*>(qp.get()) + (size_t)u * t.G * HD;
+        for (int g = 0; g < t.G; g++)
+#pragma unroll
+            for (int i = 0; i < V4; i++) {
+                const float4 v = *reinterpret_cast<const float4*>(q + g * HD + l8 * 4 + 32 * i);
+                qs[i][0] += v.x; qs[i][1] += v.y; qs[i][2] += v.z; qs[i][3] += v.w;
+            }
+    }
+    if (has_k) {
+        const KV* k = reinterpret_cast<const KV*>(kp.get()) + (size_t)u * HD;
+#pragma unroll
+        for (int i = 0; i < V4; i++) {
+            const float4 v = ld4(k, l8 * 4 + 32 * i);
+            kk[i][0] = v.x; kk[i][1] = v.y; kk[i][2] = v.z; kk[i][3] = v.w;
+        }
+    }
+    const float invG = 1.0f / (float)t.G;
+    const float* R = t.cl_r + (size_t)u * t.max_clusters * HD;
+    const int* CN = t.cl_n + (size_t)u * t.max_clusters;
+    float* SC = t.scores + (size_t)u * t.max_clusters;
+    float* DS = t.dists + (size_t)u * t.max_clusters;
+    const int jend = min(Mcur, j0 + FR_ROWS);
+    for (int j = j0 + warp * 4 + sub; j < j0 + FR_ROWS; j += (FR_THREADS / 32) * 4) {
+        const bool in = j < jend;
+        const bool live = in && CN[j] > 0;
+        float s = 0.f, dd = 0.f;
+        if (live) {
+#pragma unroll
+            for (int i = 0; i < V4; i++) {
+                const float4 rv = *reinterpret_cast<const float4*>(R + (size_t)j * HD + l8 * 4 + 32 * i);
+                s = fmaf(qs[i][0], rv.x, s); s = fmaf(qs[i][1], rv.y, s); s = fmaf(qs[i][2], rv.z, s); s = fmaf(qs[i][3], rv.w, s);
+                float a = kk[i][0] - rv.x, b = kk[i][1] - rv.y, c = kk[i][2] - rv.z, e = kk[i][3] - rv.w;
+                dd = fmaf(a, a, dd); dd = fmaf(b, b, dd); dd = fmaf(c, c, dd); dd = fmaf(e, e, dd);
+            }
+        }
+#pragma unroll
+        for (int o = 4; o > 0; o >>= 1) { s += __shfl_xor_sync(0xffffffffu, s, o); dd += __shfl_xor_sync(0xffffffffu, dd, o); }
+        if (in && l8 == 0) {
+            if (has_q) SC[j] = live ? s * invG : -INFINITY;
+            if (has_k) DS[j] = live ? dd : INFINITY;
+        }
+    }
+}
+
+// ------------------------------------------------------------------ k_select
+
+constexpr int SL_THREADS = 1024;
+constexpr int SL_MAXM = 4096;
+constexpr int SL_EPT = SL_MAXM / SL_THREADS;   // entries per thread
+
+// One block per unit.  Finds, in (score descending, id ascending) order, the longest
+// prefix of live clusters whose sizes sum to <= budget, by a three-level radix select on
+// the orderable score key with the cluster sizes as weights; if not even the best cluster
+// fits it is taken alone.  Writes the selection (id order) and its page work list; when
+// `user_ids` is given it also writes the selection in score order, -1 padded.
+__global__ void __launch_bounds__(SL_THREADS) k_select(Tables t, int budget, int* __restrict__ user_ids) {
+    const int u = blockIdx.x, tid = threadIdx.x;
+    __shared__ unsigned int keys[SL_MAXM];
+    __shared__ int hist[2048];
+    __shared__ int sh[33];
+    __shared__ int s_bin, s_rem, s_done, s_eqtake, s_eqcnt, s_L, s_tok;
+    __shared__ unsigned long long s_best;
+    const int Mcur = t.u_M[u];
+    const float* SC = t.scores + (size_t)u * t.max_clusters;
+    const int* CN = t.cl_n + (size_t)u * t.max_clusters;
+    unsigned int key[SL_EPT]; int sz[SL_EPT];
+    unsigned long long best = 0ull;
+#pragma unroll
+    for (int e = 0; e < SL_EPT; e++) {
+        const int j = tid + e * SL_THREADS;
+        key[e] = 0u; sz[e] = 0;
+        if (j < Mcur) { sz[e] = CN[j]; if (sz[e] > 0) key[e] = ord_key(SC[j]); }
+        keys[j] = key[e];
+        if (sz[e] > 0) {
+            unsigned long long kk = ((unsigned long long)key[e] << 32) | (unsigned long long)(0xffffffffu - (unsigned)j);
+            best = kk > best ? kk : best;
+        }
+    }
+    if (tid == 0) { s_rem = budget; s_done = 0; s_eqtake = 0; s_eqcnt = 0; s_L = 0; s_tok = 0; s_best = 0ull; }
+    __syncthreads();
+    // ---- radix select: digits [31:21], [20:10], [9:0]
+    unsigned int prefix = 0u, pmask = 0u;
+    const int shifts[3] = {21, 10, 0};
+    const int nbins[3] = {2048, 2048, 1024};
+    for (int lvl = 0; lvl < 3; lvl++) {
+        for (int b = tid; b < 2048; b += SL_THREADS) hist[b] = 0;
+        __syncthreads();
+        if (s_done) break;
+#pragma unroll
+        for (int e = 0; e < SL_EPT; e++)
+            if (sz[e] > 0 && (key[e] & pmask) == prefix) atomicAdd(&hist[(key[e] >> shifts[lvl]) & (nbins[lvl] - 1)], sz[e]);
+        __syncthreads();
+        // suffix sums over the bins, descending: thread i owns bins (nb-1-2i, nb-2-2i)
+        const int nb = nbins[lvl];
+        int b_hi = nb - 1 - 2 * tid, b_lo = nb - 2 - 2 * tid;
+        int h_hi = b_hi >= 0 ? hist[b_hi] : 0, h_lo = b_lo >= 0 ? hist[b_lo] : 0;
+        int tot;
+        int before = block_scan_excl(h_hi + h_lo, sh, &tot);   // weight of all bins above b_hi
+        const int rem = s_rem;
+        __syncthreads();
+        if (tid == 0 && tot <= rem) s_done = 1;                 // everything under this prefix fits
+        // the boundary bin is the first (from the top) whose inclusive suffix sum exceeds rem
+        if (b_hi >= 0 && before <= rem && before + h_hi > rem) { s_bin = b_hi; s_rem = rem - before; }
+        else if (b_lo >= 0 && before + h_hi <= rem && before + h_hi + h_lo > rem) { s_bin = b_lo; s_rem = rem - before - h_hi; }
+        __syncthreads();
+        if (s_done) break;
+        prefix |= (unsigned int)s_bin << shifts[lvl];
+        pmask |= (unsigned int)(nb - 1) << shifts[lvl];
+    }
+    __syncthreads();
+    // Selected: key above the boundary key; among clusters exactly at the boundary key, the
+    // lowest ids while they still fit.  With s_done every key >= the current prefix range is in.
+    const bool all_in = s_done != 0;
+    const unsigned int kb = prefix;
+    if (!all_in) {
+        // a single cluster at the boundary key cannot fit (its bin overflowed the remaining budget);
+        // only with several equal scores does the id-order walk matter
+        int ne = 0;
+#pragma unroll
+        for (int e = 0; e < SL_EPT; e++) ne += (sz[e] > 0 && key[e] == kb) ? 1 : 0;
+        if (ne) atomicAdd(&s_eqcnt, ne);
+        __syncthreads();
+        if (tid == 0 && s_eqcnt > 1) {
+            int rem = s_rem, take = 0;
+            for (int j = 0; j < Mcur; j++)
+                if (keys[j] == kb && CN[j] > 0) { if (CN[j] <= rem) { rem -= CN[j]; take++; } else break; }
+            s_eqtake = take;
+        }
+    }
+    __syncthreads();
+    // When all_in, pmask covers the levels already fixed: keys matching the prefix there, or larger, are selected.
+    int selc = 0, tokc = 0;
+    bool selected[SL_EPT];
+#pragma unroll
+    for (int e = 0; e < SL_EPT; e++) {
+        bool in = false;
+        if (sz[e] > 0) {
+            if (all_in) in = (key[e] & pmask) >= prefix;
+            else in = key[e] > kb;
+        }
+        selected[e] = in;
+    }
+    if (!all_in && s_eqtake > 0) {
+        // the first s_eqtake clusters (by id) with key == kb are selected too
+#pragma unroll
+        for (int e = 0; e < SL_EPT; e++) {
+            const int j = tid + e * SL_THREADS;
+            if (sz[e] > 0 && key[e] == kb) {
+                int rank = 0;
+                for (int jj = 0; jj < j; jj++) rank += (keys[jj] == kb) ? 1 : 0;
+                if (rank < s_eqtake) selected[e] = true;
+            }
+        }
+    }
+#pragma unroll
+    for (int e = 0; e < SL_EPT; e++) if (selected[e]) { selc++; tokc += sz[e]; }
+    if (selc) { atomicAdd(&s_L, selc); atomicAdd(&s_tok, tokc); }
+    if (best) atomicMax(&s_best, best);
+    __syncthreads();
+    int L = s_L;
+    if (L == 0 && budget > 0 && s_best != 0ull) {
+        // not even the best cluster fits: take it alone
+        const int jb = (int)(0xffffffffu - (unsigned)(s_best & 0xffffffffull));
+#pragma unroll
+        for (int e = 0; e < SL_EPT; e++) if (tid + e * SL_THREADS == jb) selected[e] = true;
+        L = 1;
+        if (tid == 0) { s_tok = CN[jb]; atomicOr(t.status, DYNAKV_ST_BUDGET_EXCEEDED); }
+    }
+    __syncthreads();
+    // ---- compaction in id order + work list.  Thread-major order (j = tid + e*T) is not id
+    // order, so scan one e-slab at a time.
+    int* sel = t.sel_ids + (size_t)u * t.max_clusters;
+    int2* work = t.work + (size_t)u * t.W;
+    int sbase = 0, wbase = 0;
+#pragma unroll
+    for (int e = 0; e < SL_EPT; e++) {
+        if (e * SL_THREADS >= Mcur) break;
+        const int j = tid + e * SL_THREADS;
+        const int isel = selected[e] ? 1 : 0;
+        const int np = isel ? (sz[e] + PAGE - 1) / PAGE : 0;
+        int ts, tw;
+        const int spos = sbase + block_scan_excl(isel, sh, &ts);
+        const int wpos = wbase + block_scan_excl(np, sh, &tw);
+        if (isel) {
+            sel[spos] = j;
+            int page = t.cl_head[(size_t)u * t.max_clusters + j];
+            for (int i = 0; i < np && wpos + i < t.W; i++) {
+                work[wpos + i] = make_int2(page, (i + 1 < np) ? PAGE : sz[e] - PAGE * (np - 1));
+                page = t.page_next[(size_t)u * t.P + page];
+            }
+        }
+        sbase += ts; wbase += tw;
+    }
+    if (tid == 0) {
+        t.sel_n[u] = L;
+        t.sel_tokens[u] = s_tok;
+        t.n_work[u] = min(wbase, t.W);
+        atomicAdd(&t.counters[CNT_TOKENS_ATTENDED], (unsigned long long)s_tok);
+        atomicAdd(&t.counters[CNT_CLUSTERS_SELECTED], (unsigned long long)L);
+    }
+    if (user_ids) {
+        // score order: rank = number of selected clusters that come first
+        __syncthreads();
+        int* uo = user_ids + (size_t)u * t.max_clusters;
+        for (int a = tid; a < L; a += SL_THREADS) {
+            const int j = sel[a];
+            const unsigned int kj = keys[j];
+            int rank = 0;
+            for (int b = 0; b < L; b++) {
+                const int jb = sel[b];
+                const unsigned int kq = keys[jb];
+                rank += (kq > kj || (kq == kj && jb < j)) ? 1 : 0;
+            }
+            uo[rank] = j;
+        }
+        for (int p = L + tid; p < t.max_clusters; p += SL_THREADS) uo[p] = -1;
+    }
+}
+
+// ------------------------------------------------------------------ k_append_apply
+
+// One block per unit: argmin over the distances written by k_front (ties to the lowest id),
+// then n <- n+1, delta = k - r, r <- r + delta/n, M2 <- M2 + delta.(k - r_new), and the
+// (k, v) row goes to the next slot of the cluster's tail page (a fresh page is linked when
+// the tail is full).  No stored entry moves.
+template <typename KV, int HD>
+__global__ void __launch_bounds__(256) k_append_apply(Tables t, StepPtr kp_, StepPtr vp_) {
+    constexpr int EPL = HD / 32;
+    const int u = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    __shared__ float red_d[8];
+    __shared__ int red_j[8];
+    const int Mcur = t.u_M[u];
+    const int N = t.u_N[u];
+    if (N >= t.max_tokens) { if (tid == 0) atomicOr(t.status, DYNAKV_ST_MAX_TOKENS); return; }
+    const float* DS = t.dists + (size_t)u * t.max_clusters;
+    float bd = INFINITY; int bj = 0x7fffffff;
+    for (int j = tid; j < Mcur; j += 256) {
+        const float dd = DS[j];
+        if (dd < bd) { bd = dd; bj = j; }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        const float od = __shfl_xor_sync(0xffffffffu, bd, o); const int oj = __shfl_xor_sync(0xffffffffu, bj, o);
+        if (od < bd || (od == bd && oj < bj)) { bd = od; bj = oj; }
+    }
+    if (lane == 0) { red_d[warp] = bd; red_j[warp] = bj; }
+    __syncthreads();
+    if (warp != 0) return;
+    bd = red_d[0]; bj = red_j[0];
+#pragma unroll
+    for (int w = 1; w < 8; w++) if (red_d[w] < bd || (red_d[w] == bd && red_j[w] < bj)) { bd = red_d[w]; bj = red_j[w]; }
+    if (bj == 0x7fffffff) return;    // no live cluster
+    const KV* knew = reinterpret_cast<const KV*>(kp_.get()) + (size_t)u * HD;
+    const KV* vnew = reinterpret_cast<const KV*>(vp_.get()) + (size_t)u * HD;
+    const size_t cj = (size_t)u * t.max_clusters + bj;
+    const int n_old = t.cl_n[cj];
+    int page = t.cl_tail[cj];
+    const int row = n_old % PAGE;
+    if (row == 0) {   // tail is full: link a fresh page
+        int np = -1;
+        if (lane == 0) {
+            int fc = t.u_free_cnt[u];
+            if (fc > 0) { np = t.free_stack[(size_t)u * t.P + fc - 1]; t.u_free_cnt[u] = fc - 1; }
+            else { int top = t.u_page_top[u]; if (top < t.P) { np = top; t.u_page_top[u] = top + 1; } }
+            if (np >= 0) { t.page_next[(size_t)u * t.P + page] = np; t.page_next[(size_t)u * t.P + np] = -1; t.cl_tail[cj] = np; }
+            else atomicOr(t.status, DYNAKV_ST_PAGE_POOL);
+        }
+        np = __shfl_sync(0xffffffffu, np, 0);
+        if (np < 0) return;
+        page = np;
+    }
+    const float n_new = (float)(n_old + 1);
+    float* r = t.cl_r + cj * HD;
+    float add = 0.f;
+    float kk[EPL];
+#pragma unroll
+    for (int e = 0; e < EPL; e++) {
+        kk[e] = to_f(knew[lane * EPL + e]);
+        const float ro = r[lane * EPL + e];
+        const float delta = kk[e] - ro;
+        const float rn = ro + delta / n_new;
+        r[lane * EPL + e] = rn;
+        add = fmaf(delta, kk[e] - rn, add);
+    }
+    add = warp_sum(add);
+    KV* kpg = reinterpret_cast<KV*>(t.kpages) + (((size_t)u * t.P + page) * PAGE + row) * HD;
+    KV* vpg = reinterpret_cast<KV*>(t.vpages) + (((size_t)u * t.P + page) * PAGE + row) * HD;
+#pragma unroll
+    for (int e = 0; e < EPL; e++) { kpg[lane * EPL + e] = knew[lane * EPL + e]; vpg[lane * EPL + e] = vnew[lane * EPL + e]; }
+    if (lane == 0) {
+        t.cl_M2[cj] += add;
+        t.cl_n[cj] = n_old + 1;
+        t.cl_flags[cj] &= ~FLAG_HOLD;
+        t.page_tok[((size_t)u * t.P + page) * PAGE + row] = N;
+        t.tok_cluster[(size_t)u * t.max_tokens + N] = bj;
+        t.u_N[u] = N + 1;
+        t.u_last[u] = bj;
+        atomicAdd(&t.counters[CNT_APPENDED], 1ull);
+    }
+}
+
+// ------------------------------------------------------------------ launchers
+
+void launch_front(const Tables& t, StepPtr q, StepPtr k, int has_q, int has_k, cudaStream_t s, long long* launches) {
+    dim3 grid((t.max_clusters + FR_ROWS - 1) / FR_ROWS, t.U);
+    if (t.kv_dtype == DYNAKV_F32) {
+        if (t.d == 64) k_front<float, 64><<<grid, FR_THREADS, 0, s>>>(t, q, k, has_q, has_k);
+        else k_front<float, 128><<<grid, FR_THREADS, 0, s>>>(t, q, k, has_q, has_k);
+    } else {
+        if (t.d == 64) k_front<__nv_bfloat16, 64><<<grid, FR_THREADS, 0, s>>>(t, q, k, has_q, has_k);
+        else k_front<__nv_bfloat16, 128><<<grid, FR_THREADS, 0, s>>>(t, q, k, has_q, has_k);
+    }
+    (*launches)++;
+}
+
+void launch_select(const Tables& t, int budget, int* user_sel_ids, cudaStream_t s, long long* launches) {
+    k_select<<<t.U, SL_THREADS, 0, s>>>(t, budget, user_sel_ids);
+    (*launches)++;
+}
+
+void launch_append_apply(const Tables& t, StepPtr k, StepPtr v, cudaStream_t s, long long* launches) {
+    if (t.kv_dtype == DYNAKV_F32) {
+        if (t.d == 64) k_append_apply<float, 64><<<t.U, 256, 0, s>>>(t, k, v); else k_append_apply<float, 128><<<t.U, 256, 0, s>>>(t, k, v);
+    } else {
+        if (t.d == 64) k_append_apply<__nv_bfloat16, 64><<<t.U, 256, 0, s>>>(t, k, v); else k_append_apply<__nv_bfloat16, 128><<<t.U, 256, 0, s>>>(t, k, v);
+    }
+    (*launches)++;
+}
+
+}  // namespace dkv

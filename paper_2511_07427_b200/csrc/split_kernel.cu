@@ -39,13 +39,44 @@ __global__ void __launch_bounds__(SP_THREADS) k_split_check(Tables t, float gamm
     int* rank_of = t.sp_pos + (size_t)u * 2 * t.max_tokens;     // per position
     int* holes = rank_of + t.max_tokens;                        // hole positions, in order
 
-    for (int j = 0; j < M0; j++) {
+    // ---- triggered clusters, ascending id, evaluated on the state at entry.  A full scan is
+    // needed only after a split changed M_live or created clusters (u_scan); otherwise only the
+    // cluster that received the last append can have become triggered: for every other cluster
+    // n_j and M2_j are unchanged while N only grew.
+    int* trig = dyn + 2 * maxch;
+    __shared__ int s_ntrig, s_nsplit;
+    if (tid == 0) { s_ntrig = 0; s_nsplit = 0; }
+    __syncthreads();
+    {
+        const int full = t.u_scan[u];
+        const int last = t.u_last[u];
+        int base = 0;
+        const int jlim = full ? M0 : (last >= 0 ? 1 : 0);
+        for (int b0 = 0; b0 < jlim; b0 += SP_THREADS) {
+            const int j = full ? b0 + tid : (tid == 0 ? last : -1);
+            int hit = 0;
+            if (j >= 0 && j < M0) {
+                const size_t cj = (size_t)u * t.max_clusters + j;
+                const int c = t.cl_n[cj];
+                if (c > 0 && c >= min_size && !(t.cl_flags[cj] & FLAG_HOLD)) {
+                    const bool by_var = var_enabled && (t.cl_M2[cj] / (float)c > tau);
+                    const bool by_size = gamma > 0.f && ((double)c * (double)Mlive0 > (double)gamma * (double)N);
+                    hit = (by_var || by_size) ? 1 : 0;
+                }
+            }
+            int tot;
+            const int pos = base + block_scan_excl(hit, sh, &tot);
+            if (hit) trig[pos] = j;
+            base += tot;
+        }
+        if (tid == 0) s_ntrig = base;
+        __syncthreads();
+    }
+    const int ntrig = s_ntrig;
+    for (int li = 0; li < ntrig; li++) {
+        const int j = trig[li];
         const size_t cj = (size_t)u * t.max_clusters + j;
         const int c = t.cl_n[cj];
-        if (c <= 0 || c < min_size || (t.cl_flags[cj] & FLAG_HOLD)) continue;
-        const bool by_var = var_enabled && (t.cl_M2[cj] / (float)c > tau);
-        const bool by_size = gamma > 0.f && ((double)c * (double)Mlive0 > (double)gamma * (double)N);
-        if (!by_var && !by_size) continue;
         if (t.u_M[u] >= t.max_clusters) { if (tid == 0) atomicOr(t.status, DYNAKV_ST_MAX_CLUSTERS); continue; }
 
         __syncthreads();    // previous cluster's work is complete
@@ -244,6 +275,7 @@ __global__ void __launch_bounds__(SP_THREADS) k_split_check(Tables t, float gamm
             t.cl_flags[cj] = 0; t.cl_flags[cn] = 0;
             t.u_M[u] = new_id + 1; t.u_Mlive[u] = t.u_Mlive[u] + 1;
             atomicAdd(&t.counters[CNT_SPLITS], 1ull);
+            s_nsplit = s_nsplit + 1;
         }
         __syncthreads();
         // ---- phase 4: exact statistics of both children (mean, then M2 about the mean)
@@ -290,11 +322,13 @@ __global__ void __launch_bounds__(SP_THREADS) k_split_check(Tables t, float gamm
             __syncthreads();
         }
     }
+    __syncthreads();
+    if (tid == 0) { t.u_scan[u] = s_nsplit > 0 ? 1 : 0; t.u_last[u] = -1; }
 }
 
 template <typename KV, int HD>
 static void split_t(const Tables& t, float gamma, int var_enabled, int min_size, int iters, cudaStream_t s) {
-    size_t dyn = sizeof(int) * 2 * (size_t)(t.max_tokens / PAGE + 2);
+    size_t dyn = sizeof(int) * (2 * (size_t)(t.max_tokens / PAGE + 2) + (size_t)t.max_clusters);
     if (dyn > 32 * 1024)
         cudaFuncSetAttribute(k_split_check<KV, HD>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn);
     k_split_check<KV, HD><<<t.U, SP_THREADS, dyn, s>>>(t, gamma, var_enabled, min_size, iters);

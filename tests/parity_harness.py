@@ -82,7 +82,9 @@ def check_state(o: O.OracleUnit, st: dict, ui: int, rep: ParityReport, where: st
         rep.max_centroid_rel = max(rep.max_centroid_rel, r)
         assert r <= TOL_CENTROID, f"{where}: centroid relative error {r:.3e}"
         m2g, m2o = st["M2"][ui, :M].astype(np.float64)[live], o.M2()[live]
-        scale = np.maximum(m2o, 1e-3 * max(float(m2o.max()), 1e-30))
+        # floor: fp32 rounding of the centroid itself leaves about n * |c|^2 * 2^-46 in M2 even when the members coincide
+        floor = 1e-6 * cnt[live] * (np.linalg.norm(Co[live], axis=1) ** 2)
+        scale = np.maximum(np.maximum(m2o, 1e-3 * float(m2o.max())), np.maximum(floor, 1e-30))
         assert float((np.abs(m2g - m2o) / scale).max()) <= 1e-3, f"{where}: M2 differs"
 
 

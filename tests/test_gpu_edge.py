@@ -1,0 +1,205 @@
+"""GPU edge cases through the C ABI, each checked against the fp64 oracle."""
+import numpy as np
+import pytest
+import torch
+
+import oracle as O
+import paper_2511_07427_b200 as P
+from gen import CONFIGS, UnitStream, make_decode_chunk, make_prefill
+
+pytestmark = pytest.mark.gpu
+
+
+def _run(cfg, units, steps, **kw):
+    from parity_harness import run_parity
+    rep = run_parity(cfg, units, steps, **kw)
+    assert rep.violations == 0
+    return rep
+
+
+@pytest.mark.parametrize("budget", [0, 1, 40, 10_000])
+def test_budget_extremes(budget):
+    cfg = CONFIGS[2].scaled(n_prefill=700, steps=12, M0=20, max_clusters=64, T=4)
+    rep = _run(cfg, [0, 1], cfg.steps, budget=budget, assign_mode=1)
+    if budget == 0:
+        assert max(rep.tokens_selected) == 0
+    if budget == 1:
+        assert rep.status_bits & P.ST_BUDGET_EXCEEDED
+    if budget == 10_000:
+        assert min(rep.tokens_selected) >= 700
+
+
+@pytest.mark.parametrize("G,d,dtype", [(1, 128, "bf16"), (2, 64, "bf16"), (7, 128, "bf16"), (8, 128, "bf16"),
+                                       (3, 64, "f32"), (5, 128, "f32"), (8, 64, "bf16")])
+def test_group_sizes_head_dims_dtypes(G, d, dtype):
+    base = CONFIGS[2] if dtype == "bf16" else CONFIGS[1]
+    cfg = base.scaled(Hq=G, Hkv=1, L=1, B=1, d=d, n_prefill=515, steps=24, M0=19, max_clusters=64, budget=150, T=4,
+                      init_mode="kmeanspp" if G % 2 else "random")
+    _run(cfg, [0], cfg.steps, assign_mode=1)
+
+
+def test_plain_attention_kernel_on_bf16():
+    cfg = CONFIGS[5].scaled(B=1, L=1, n_prefill=600, steps=16, M0=24, max_clusters=64, budget=200, T=3)
+    from parity_harness import make_ctx
+    import parity_harness as H
+    orig = H.make_ctx
+
+    def forced(cfg_, n_units, trace=1, assign_mode=0):
+        c = P.DynaKVConfig(n_units=n_units, gqa_group=cfg_.G, head_dim=cfg_.d, kv_dtype=P.BF16, max_tokens=cfg_.max_tokens,
+                           max_clusters=cfg_.max_clusters, kmeans_iters=cfg_.T, init_mode=P.INIT_RANDOM,
+                           split_size_factor=cfg_.split_size_factor, split_var_factor=cfg_.split_var_factor,
+                           split_min_size=cfg_.split_min_size, split_iters=cfg_.split_iters, trace=trace, assign_mode=1,
+                           attn_mode=1)
+        return P.DynaKV(c)
+    H.make_ctx = forced
+    try:
+        _run(cfg, [0, 1, 2, 3], cfg.steps)
+    finally:
+        H.make_ctx = orig
+
+
+def test_every_key_its_own_cluster_and_page_boundaries():
+    # n == M: every cluster has one member after the first round; then 31/32/33-row pages via appends
+    cfg = CONFIGS[2].scaled(n_prefill=48, steps=80, M0=48, max_clusters=64, budget=64, T=2, split_size_factor=0.0,
+                            split_var_factor=0.0)
+    _run(cfg, [0], cfg.steps, assign_mode=1)
+
+
+def test_few_clusters_long_chains_and_capacity_bits():
+    # 3 clusters over 200 keys (multi-page chains), splitting until the id cap, then the token cap
+    cfg = CONFIGS[2].scaled(n_prefill=200, steps=40, M0=3, max_clusters=6, budget=120, T=3, split_min_size=4,
+                            split_size_factor=1.05)
+    rep = _run(cfg, [0, 1], cfg.steps, assign_mode=1)
+    assert rep.status_bits & P.ST_MAX_CLUSTERS
+
+
+def _single_ctx(cfg, K, V, **kw):
+    from parity_harness import make_ctx
+    ctx = make_ctx(cfg, K.shape[0], trace=0, **kw)
+    ctx.build_index(K.cuda(), V.cuda(), cfg.M0, 99)
+    return ctx
+
+
+def test_token_capacity_sets_status_and_drops_append():
+    cfg = CONFIGS[2].scaled(n_prefill=64, steps=4, M0=4, max_clusters=16, budget=64, T=2)
+    s = [UnitStream(cfg, 0)]
+    K, V = make_prefill(s)
+    q, k, v = make_decode_chunk(s, 4)
+    ctx = _single_ctx(cfg, K, V, assign_mode=1)
+    for t in range(4):
+        ctx.append(k[t].cuda(), v[t].cuda())
+    assert ctx.get_status()["error_bits"] & P.ST_MAX_TOKENS == 0
+    ctx.append(k[0].cuda(), v[0].cuda())
+    st = ctx.get_status()
+    assert st["error_bits"] & P.ST_MAX_TOKENS and st["n_appended"] == 4
+    assert ctx.export_state()["n_tokens"][0] == 68
+    ctx.destroy()
+
+
+def test_zero_query_breaks_score_ties_by_id():
+    cfg = CONFIGS[2].scaled(n_prefill=400, steps=4, M0=16, max_clusters=32, budget=100, T=3)
+    s = [UnitStream(cfg, 0)]
+    K, V = make_prefill(s)
+    ctx = _single_ctx(cfg, K, V, assign_mode=1)
+    st = ctx.export_state()
+    q = torch.zeros((1, cfg.G, cfg.d), dtype=torch.float32, device="cuda")
+    sel = torch.full((1, cfg.max_clusters), -1, dtype=torch.int32, device="cuda")
+    out = ctx.decode_step(q, 100, selected_ids=sel)
+    ids = sel[0].cpu().numpy(); ids = ids[ids >= 0]
+    cnt = st["counts"][0]
+    exp, cum = [], 0
+    for j in range(16):
+        if cnt[j] == 0:
+            continue
+        if cum + cnt[j] > 100:
+            break
+        exp.append(j); cum += cnt[j]
+    assert list(ids) == exp
+    # uniform softmax over the selected members
+    a = st["tok_cluster"][0, :400]
+    ref = V[0].double()[np.isin(a, exp)].mean(0).numpy()
+    assert np.abs(out[0].cpu().numpy() - ref[None]).max() < 1e-4
+    ctx.destroy()
+
+
+def test_duplicate_keys_leave_dead_clusters():
+    cfg = CONFIGS[1].scaled(n_prefill=256, steps=16, M0=12, max_clusters=32, budget=80, T=4, init_mode="random")
+    from parity_harness import make_ctx, make_oracle, check_state, ParityReport
+    rng = np.random.default_rng(0)
+    base = rng.normal(size=(6, cfg.d)).astype(np.float32)
+    K = torch.tensor(base[rng.integers(0, 6, size=256)])[None].contiguous()     # only 6 distinct keys, 12 centres
+    V = torch.tensor(rng.normal(size=(1, 256, cfg.d)).astype(np.float32))
+    ctx = make_ctx(cfg, 1, trace=1)
+    ctx.build_index(K.cuda(), V.cuda(), cfg.M0, 5)
+    picks, trace = ctx.get_build_trace()
+    o = make_oracle(cfg)
+    o.build(K[0].double().numpy(), V[0].double().numpy(), cfg.M0, cfg.T, 5, unit_index=0, init_mode=O.INIT_RANDOM,
+            hint_assign=trace[:, 0, :])
+    st = ctx.export_state()
+    assert o.violations == 0 and (o.counts() == 0).sum() >= 6
+    check_state(o, st, 0, ParityReport(), "dup build")
+    q = torch.tensor(rng.normal(size=(1, cfg.G, cfg.d)).astype(np.float32))
+    sel = torch.full((1, cfg.max_clusters), -1, dtype=torch.int32, device="cuda")
+    out = ctx.decode_step(q.cuda(), 80, selected_ids=sel).cpu().numpy()
+    ids = sel[0].cpu().numpy(); ids = ids[ids >= 0]
+    out_o, ids_o, _ = o.decode_step(q[0].double().numpy(), 80, hint_ids=ids)
+    assert list(ids_o) == list(ids) and np.abs(out[0] - out_o).max() < 2e-3
+    ctx.destroy()
+
+
+def test_graph_loop_and_host_step_match_direct_calls():
+    cfg = CONFIGS[2].scaled(n_prefill=900, steps=48, M0=30, max_clusters=96, budget=256, T=4)
+    units = [0, 1, 2, 3, 4]
+    s = [UnitStream(cfg, u) for u in units]
+    K, V = make_prefill(s)
+    q, k, v = make_decode_chunk(s, 48)
+    side = torch.cuda.Stream()
+    outs = {}
+    states = {}
+    for mode in ("direct", "graph", "host"):
+        with torch.cuda.stream(side):
+            from parity_harness import make_ctx
+            ctx = make_ctx(cfg, len(units), trace=0, assign_mode=1)
+            ctx.build_index(K.cuda(), V.cuda(), cfg.M0, 7)
+            qd, kd, vd = q.cuda(), k.cuda(), v.cuda()
+            if mode == "direct":
+                out = torch.empty((48, len(units), cfg.G, cfg.d), device="cuda")
+                for t in range(48):
+                    ctx.decode_step(qd[t], cfg.budget, out=out[t]); ctx.append(kd[t], vd[t]); ctx.split_check()
+            elif mode == "graph":
+                out = ctx.decode_loop(qd[:20], kd[:20], vd[:20], cfg.budget)
+                out2 = ctx.decode_loop(qd[20:], kd[20:], vd[20:], cfg.budget)
+                out = torch.cat([out, out2])
+            else:
+                out = torch.empty((48, len(units), cfg.G, cfg.d))
+                qh, kh, vh = q.pin_memory(), k.pin_memory(), v.pin_memory()
+                oh = torch.empty((len(units), cfg.G, cfg.d)).pin_memory()
+                for t in range(48):
+                    ctx.step_host(qh[t], kh[t], vh[t], cfg.budget, oh); out[t] = oh
+            side.synchronize()
+            outs[mode] = out.cpu().numpy()
+            states[mode] = ctx.export_state()
+            assert ctx.get_status()["n_splits"] > 0
+            ctx.destroy()
+    for mode in ("graph", "host"):
+        assert np.array_equal(states[mode]["tok_cluster"], states["direct"]["tok_cluster"])
+        assert np.abs(outs[mode] - outs["direct"]).max() < 1e-4
+
+
+def test_wrong_call_order_and_shapes():
+    cfg = P.DynaKVConfig(n_units=1, gqa_group=2, head_dim=64, kv_dtype=P.F32, max_tokens=64, max_clusters=8)
+    ctx = P.DynaKV(cfg)
+    q = torch.zeros((1, 2, 64), device="cuda")
+    with pytest.raises(P.DynaKVError):
+        ctx.decode_step(q, 8)                      # before build_index
+    with pytest.raises(P.DynaKVError):
+        ctx.split_check()
+    K = torch.randn((1, 32, 64), device="cuda")
+    with pytest.raises(P.DynaKVError):
+        ctx.build_index(K, K, 33, 0)               # more clusters than keys
+    ctx.build_index(K, K, 4, 0)
+    with pytest.raises(P.DynaKVError):
+        ctx.build_index(K, K, 4, 0)                # twice
+    with pytest.raises(P.DynaKVError):
+        ctx.decode_loop(q[None], K[:, 0][None], K[:, 0][None], 8)   # default stream: no graph capture
+    ctx.destroy()

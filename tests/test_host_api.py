@@ -34,7 +34,7 @@ def test_library_exports_every_declared_symbol():
 def _cfg(**kw):
     base = dict(n_units=1, gqa_group=4, head_dim=64, kv_dtype=0, max_tokens=128, max_clusters=16, kmeans_iters=2,
                 init_mode=0, split_size_factor=2.0, split_var_factor=2.0, split_min_size=8, split_iters=8, trace=0,
-                assign_mode=0)
+                assign_mode=0, attn_mode=0)
     base.update(kw)
     return _Config(**base)
 
