@@ -20,7 +20,6 @@ import os
 import statistics
 import subprocess
 import sys
-import tempfile
 import time
 
 ROOT = os.path.dirname(os.path.abspath(__file__))
@@ -39,113 +38,160 @@ def _peaks():
 
 
 class ClockSampler:
-    """Samples nvidia-smi clocks and throttle reasons in the background."""
-    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
-         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+    """Reads SM clock, power and clock-event reasons from NVML on a background thread
+    (read-only queries, about every 20 ms) between start() and stop()."""
 
-    def __init__(self, gpu_index: int):
-        self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
-        self.p = None
+    def __init__(self, torch_device_index: int):
+        import threading
+        self.samples = []          # (t, sm_mhz, power_w, reasons bitmask)
+        self.sm_max = None
+        self._stop = threading.Event()
+        self._thread = None
+        self._h = None
         try:
-            self.p = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
-                                       "-lms", "100", "-i", str(gpu_index)], stdout=self.f, stderr=subprocess.DEVNULL)
-        except Exception:
-            self.p = None
-
-    def stop(self) -> dict:
-        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
-        if self.p is None:
-            return out
-        self.p.terminate()
-        try:
-            self.p.wait(timeout=5)
-        except Exception:
-            self.p.kill()
-        self.f.flush(); self.f.seek(0)
-        sm, smax, reasons = [], [], set()
-        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for line in self.f.read().splitlines():
-            parts = [x.strip() for x in line.split(",")]
-            if len(parts) < 9:
-                continue
+            import pynvml
+            import torch
+            pynvml.nvmlInit()
+            h = None
             try:
-                sm.append(float(parts[1])); smax.append(float(parts[2]))
-            except ValueError:
-                continue
-            for name, val in zip(names, parts[5:9]):
-                if val.lower().startswith("active"):
-                    reasons.add(name)
-        try:
-            os.unlink(self.f.name)
-        except OSError:
-            pass
-        if sm:
-            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(smax), reasons=sorted(reasons), samples=len(sm))
+                uuid = str(torch.cuda.get_device_properties(torch_device_index).uuid)
+                h = pynvml.nvmlDeviceGetHandleByUUID(("GPU-" + uuid).encode())
+            except Exception:
+                h = pynvml.nvmlDeviceGetHandleByIndex(torch_device_index)
+            self._h, self._nv = h, pynvml
+            self.sm_max = float(pynvml.nvmlDeviceGetMaxClockInfo(h, pynvml.NVML_CLOCK_SM))
+            self._thread = threading.Thread(target=self._run, daemon=True)
+        except Exception:
+            self._h = None
+
+    def _run(self):
+        nv, h = self._nv, self._h
+        while not self._stop.is_set():
+            try:
+                sm = float(nv.nvmlDeviceGetClockInfo(h, nv.NVML_CLOCK_SM))
+                pw = nv.nvmlDeviceGetPowerUsage(h) / 1000.0
+                rs = int(nv.nvmlDeviceGetCurrentClocksEventReasons(h))
+                self.samples.append((time.perf_counter(), sm, pw, rs))
+            except Exception:
+                pass
+            self._stop.wait(0.02)
+
+    def start(self):
+        if self._thread is not None:
+            self._thread.start()
+
+    def stop(self, t0: float = None, t1: float = None) -> dict:
+        out = {"sm_mhz": None, "sm_max_mhz": self.sm_max, "reasons": [], "samples": 0, "power_w_max": None}
+        if self._thread is None:
+            return out
+        self._stop.set(); self._thread.join(timeout=2)
+        nv = self._nv
+        rows = [r for r in self.samples if (t0 is None or r[0] >= t0) and (t1 is None or r[0] <= t1)]
+        if not rows:
+            rows = self.samples
+        if rows:
+            names = [("hw_slowdown", nv.nvmlClocksEventReasonHwSlowdown),
+                     ("hw_thermal_slowdown", nv.nvmlClocksEventReasonHwThermalSlowdown),
+                     ("sw_thermal_slowdown", nv.nvmlClocksEventReasonSwThermalSlowdown),
+                     ("sw_power_cap", nv.nvmlClocksEventReasonSwPowerCap)]
+            mask = 0
+            for r in rows:
+                mask |= r[3]
+            out.update(sm_mhz=statistics.median(r[1] for r in rows), reasons=[n for n, b in names if mask & b],
+                       samples=len(rows), power_w_max=max(r[2] for r in rows))
         return out
 
 
-def _oracle_sample(cfg, n_units: int, steps: int, lloyd_rounds: int):
-    """Time the fp64 oracle, as it stands, on a bounded sample of the workload: `n_units`
-    units of the config (index built by the oracle itself with `lloyd_rounds` rounds, untimed),
-    then `steps` iterations of decode_step + append + split_check, one thread per unit."""
-    from concurrent.futures import ThreadPoolExecutor
+class OracleSample:
+    """The fp64 oracle, as it stands, on a bounded sample of the workload: `n_units` units of
+    the config at full size, one host thread per unit.  The index is built by the oracle
+    itself (one Lloyd round, untimed); run(n) then times n iterations of
+    decode_step + append + split_check on every sampled unit."""
 
-    import numpy as np
+    def __init__(self, cfg, n_units: int, capacity_steps: int):
+        from concurrent.futures import ThreadPoolExecutor
 
-    import oracle as O
-    from gen import UnitStream
+        import oracle as O
+        from gen import UnitStream
 
-    cores = min(n_units, os.cpu_count() or 1)
+        self.cfg, self.n_units = cfg, n_units
+        self.cores = min(n_units, os.cpu_count() or 1)
+        self.ex = ThreadPoolExecutor(max_workers=self.cores)
+        max_tokens = cfg.n_prefill + capacity_steps + 1
 
-    def prep(u):
-        s = UnitStream(cfg, u)
-        K, V = s.prefill()
-        o = O.OracleUnit(cfg.d, cfg.G, cfg.max_tokens, cfg.max_clusters, gamma=cfg.split_size_factor,
-                         alpha=cfg.split_var_factor, split_min_size=cfg.split_min_size, split_iters=cfg.split_iters)
-        o.build(K.double().numpy(), V.double().numpy(), cfg.M0, lloyd_rounds, 1234, unit_index=u,
-                init_mode=O.INIT_RANDOM)
-        q, k, v = s.decode(steps)
-        return o, q.double().numpy(), k.double().numpy(), v.double().numpy()
+        def prep(u):
+            s = UnitStream(cfg.scaled(steps=max(cfg.steps, capacity_steps)), u)
+            K, V = s.prefill()
+            o = O.OracleUnit(cfg.d, cfg.G, max_tokens, cfg.max_clusters, gamma=cfg.split_size_factor,
+                             alpha=cfg.split_var_factor, split_min_size=cfg.split_min_size, split_iters=cfg.split_iters)
+            o.build(K.double().numpy(), V.double().numpy(), cfg.M0, 1, 1234, unit_index=u, init_mode=O.INIT_RANDOM)
+            return [o, s]
 
-    def run(item):
-        o, q, k, v = item
-        for t in range(steps):
-            o.decode_step(q[t], cfg.budget)
-            o.append(k[t], v[t])
-            o.split_check()
+        self.items = list(self.ex.map(prep, range(n_units)))
 
-    with ThreadPoolExecutor(max_workers=cores) as ex:
-        items = list(ex.map(prep, range(n_units)))
+    def run(self, steps: int) -> float:
+        """Seconds taken by `steps` iterations on all sampled units (input generation untimed)."""
+        cfg = self.cfg
+
+        def gen(item):
+            q, k, v = item[1].decode(steps)
+            return item[0], q.double().numpy(), k.double().numpy(), v.double().numpy()
+
+        def work(a):
+            o, q, k, v = a
+            for t in range(steps):
+                o.decode_step(q[t], cfg.budget)
+                o.append(k[t], v[t])
+                o.split_check()
+
+        args = list(self.ex.map(gen, self.items))
         t0 = time.perf_counter()
-        list(ex.map(run, items))
-        dt = time.perf_counter() - t0
-    # one "step" of the metric covers all U units; the sample covered n_units of them
-    per_step_all_units = dt / steps * (cfg.U / n_units)
-    return 1.0 / per_step_all_units, cores, dt
+        list(self.ex.map(work, args))
+        return time.perf_counter() - t0
+
+    def steps_per_s(self, dt: float, steps: int) -> float:
+        # one step of the metric covers all U units; the sample covered n_units of them
+        return 1.0 / (dt / steps * (self.cfg.U / self.n_units))
+
+    def describe(self, steps: int, dt: float) -> str:
+        cfg = self.cfg
+        return (f"{self.n_units} of {cfg.U} units of config {cfg.cfg_id} at full size (index built by the oracle with "
+                f"1 Lloyd round, untimed), {steps} decode steps in {dt:.1f} s on {self.cores} threads, scaled per unit "
+                f"to all {cfg.U} units")
+
+
+def _cpu_baseline(cfg, target_seconds: float = 12.0) -> dict:
+    n_units = min(16, os.cpu_count() or 1)
+    cap = 4096
+    smp = OracleSample(cfg, n_units, cap)
+    probe = 8
+    dt = smp.run(probe)
+    steps = int(max(8, min(cap - probe - 1, target_seconds / max(dt / probe, 1e-6))))
+    dt = smp.run(steps)
+    return {"value": smp.steps_per_s(dt, steps), "unit": "steps/s", "cores": smp.cores, "kind": "oracle",
+            "sample": smp.describe(steps, dt)}
 
 
 def run_reference(args, cfg):
+    """The reference arm: the oracle on the host cores.  Every step is one iteration over the
+    bounded sample of units; W warm-up steps, then exactly K timed steps."""
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    n_units = min(8, os.cpu_count() or 1)
-    per = max(1, min(args.steps, 4))
-    vals = []
-    total_dt = 0.0
-    reps = max(1, min(3, args.steps // per))
-    for _ in range(reps):
-        v, cores, dt = _oracle_sample(cfg, n_units, per, lloyd_rounds=1)
-        vals.append(v); total_dt += dt
-    value = statistics.median(vals)
-    sample = (f"{n_units} of {cfg.U} units of config {cfg.cfg_id} at full size (index built by the oracle with 1 Lloyd "
-              f"round, untimed), {per} decode steps per repeat x {reps} repeats, scaled per unit to all {cfg.U} units")
+    n_units = min(16, os.cpu_count() or 1)
+    smp = OracleSample(cfg, n_units, args.warmup + args.steps)
+    if args.warmup > 0:
+        smp.run(args.warmup)
+    dt = smp.run(args.steps)
+    value = smp.steps_per_s(dt, args.steps)
     line = {
         "impl": "reference", "metric": METRIC, "value": value, "unit": "steps/s", "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1000.0 / value, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
         "config": {"workload": f"config{cfg.cfg_id}:{cfg.name}", "units": cfg.U, "context": cfg.n_prefill,
                    "budget": cfg.budget},
-        "cpu_baseline": {"value": value, "unit": "steps/s", "cores": cores, "kind": "oracle", "sample": sample},
+        "cpu_baseline": {"value": value, "unit": "steps/s", "cores": smp.cores, "kind": "oracle",
+                         "sample": smp.describe(args.steps, dt)},
         "e2e": {"value": value, "unit": "steps/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }
     print(json.dumps(line), flush=True)
@@ -226,17 +272,23 @@ def run_ours(args, cfg):
     if world > 1:
         dist.barrier()
     st0 = ctx.get_status()
+    if st0["error_bits"] & P.ST_INTERNAL:
+        raise RuntimeError("a bounded wait ran out inside a kernel during warm-up (status bit INTERNAL); not timing")
     launches0 = ctx.launch_count()
     sampler = ClockSampler(local) if rank == 0 else None
+    if sampler:
+        sampler.start()
     torch.cuda.synchronize()
+    t_wall0 = time.perf_counter()
     e0.record()
     loop(pos, pos + K_steps)
     e1.record()
     torch.cuda.synchronize()
+    t_wall1 = time.perf_counter()
     if world > 1:
         dist.barrier()
     ms = e0.elapsed_time(e1)
-    clocks = sampler.stop() if sampler else None
+    clocks = sampler.stop(t_wall0, t_wall1) if sampler else None
     pos += K_steps
     st1 = ctx.get_status()
     gpu_launches = ctx.launch_count() - launches0
@@ -263,7 +315,7 @@ def run_ours(args, cfg):
     attn_bytes = tokens_per_launch * 2 * cfg.d * bytes_kv + U * cfg.G * cfg.d * 4
     achieved = attn_bytes / (attn_ms * 1e-3) / 1e9 if attn_ms > 0 else 0.0
     kernels = {k: (v["ms"] / v["launches"] * 1e3 if v["launches"] else None) for k, v in kt.items()
-               if k in ("select", "attn", "combine", "append", "split")}
+               if k in ("front", "select", "attn", "combine", "append", "split")}
     roofline = {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                 "frac": achieved / peaks["hbm_gbs"], "traffic": args.attn_traffic_bytes,
                 "kernel": "gather_attn", "us_per_launch": attn_ms * 1e3, "algorithmic_bytes_per_launch": attn_bytes,
@@ -296,12 +348,7 @@ def run_ours(args, cfg):
     if rank == 0:
         cpu_baseline = None
         if world == 1 and not args.no_cpu_baseline:
-            n_units = min(8, os.cpu_count() or 1)
-            v, cores, dt = _oracle_sample(cfg, n_units, 4, lloyd_rounds=1)
-            cpu_baseline = {"value": v, "unit": "steps/s", "cores": cores, "kind": "oracle",
-                            "sample": f"{n_units} of {cfg.U} units of config {cfg.cfg_id} at full size (index built by the "
-                                      f"oracle with 1 Lloyd round, untimed), 4 decode steps ({dt:.1f} s), scaled per unit "
-                                      f"to all {cfg.U} units"}
+            cpu_baseline = _cpu_baseline(cfg)
         line = {
             "metric": METRIC, "value": value, "unit": "steps/s", "n_gpus": world, "steps": K_steps, "warmup": W,
             "ms_per_step": ms / K_steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
@@ -325,7 +372,7 @@ def run_ours(args, cfg):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=512)
+    ap.add_argument("--steps", type=int, default=1024)
     ap.add_argument("--warmup", type=int, default=16)
     ap.add_argument("--config", type=int, default=4)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
@@ -333,11 +380,16 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=64)
     ap.add_argument("--profile-steps", type=int, default=64)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--units", type=int, default=0,
+                    help="run only the first N units of the config (profiling aid: smaller device footprint); 0 = all")
     ap.add_argument("--attn-traffic-bytes", type=float, default=None,
                     help="ncu dram bytes per launch of the gather-attention kernel (from profiles/), echoed in roofline.traffic")
     args = ap.parse_args()
     from gen import CONFIGS
     cfg = CONFIGS[args.config]
+    if args.units > 0:
+        # keep the per-unit shape; B*L*Hkv collapses to N units of one layer
+        cfg = cfg.scaled(B=1, L=1, Hkv=args.units, Hq=args.units * cfg.G, name=cfg.name + f"[first {args.units} units]")
     if args.impl == "reference":
         run_reference(args, cfg)
     else:

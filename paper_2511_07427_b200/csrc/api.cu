@@ -132,6 +132,16 @@ extern "C" int dynakv_create(const dynakv_config* cfg, void* cuda_stream, dynakv
     t.P = full_pages + cfg->max_clusters + slack;
     t.W = t.P;
     t.n_splits_attn = 8;
+    {
+        int dev = 0, sms = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1) {
+            snprintf(g_err, sizeof(g_err), "no usable CUDA device: %s", cudaGetErrorString(cudaGetLastError()));
+            delete c;
+            return DYNAKV_ERR_CUDA;
+        }
+        t.n_attn_ctas = 2 * sms;
+        t.attn_pf_in_smem = cfg->n_units <= 1024 ? 1 : 0;
+    }
     const size_t U = t.U, P = t.P, Mx = t.max_clusters, d = t.d;
     const size_t page_elems = U * P * PAGE * d;
     if (cfg->kv_dtype == DYNAKV_F32) {
@@ -158,7 +168,19 @@ extern "C" int dynakv_create(const dynakv_config* cfg, void* cuda_stream, dynakv
     ALLOC(t.sel_n, U, true); ALLOC(t.sel_tokens, U, true);
     ALLOC(t.work, U * (size_t)t.W, false);
     ALLOC(t.n_work, U, true);
-    ALLOC(t.part, U * (size_t)t.n_splits_attn * t.G * (d + 2), false);
+    {
+        size_t recs = U * (size_t)t.n_splits_attn;
+        if (recs < 2 * (size_t)t.n_attn_ctas) recs = 2 * (size_t)t.n_attn_ctas;
+        ALLOC(t.part, recs * t.G * (d + 2), false);
+    }
+    ALLOC(t.work_prefix, U + 1, true);
+    ALLOC(t.unit_arrive, U, true);
+    ALLOC(t.plan_counter, 1, true);
+    if (cfg->kv_dtype == DYNAKV_BF16 && attn_tma_prepare(t) != 0) {
+        snprintf(g_err, sizeof(g_err), "cannot reserve shared memory for the gather-attention kernel: %s", cudaGetErrorString(cudaGetLastError()));
+        dynakv_destroy(c);
+        return DYNAKV_ERR_CUDA;
+    }
     ALLOC(t.sp_label, U * (size_t)t.max_tokens, false);
     ALLOC(t.sp_pos, U * 2 * (size_t)t.max_tokens, false);
     ALLOC(t.status, 1, true);
@@ -244,12 +266,14 @@ static void enqueue_front(dynakv_ctx* c, StepPtr q, StepPtr k, int has_q, int ha
 // select -> gather attention -> combine, on scores already written by the front pass
 static void enqueue_retrieve(dynakv_ctx* c, StepPtr q, int budget, StepPtrW out, int* sel_ids, bool timed) {
     { TimeScope ts(c, KC_SELECT, timed); launch_select(c->t, budget, sel_ids, c->stream, &c->launches); }
-    {
+    if (c->t.kv_dtype == DYNAKV_BF16 && c->cfg.attn_mode == 0) {
+        // gather, attend and combine in one persistent kernel
         TimeScope ts(c, KC_ATTN, timed);
-        if (c->t.kv_dtype == DYNAKV_BF16 && c->cfg.attn_mode == 0) launch_gather_attn_mma(c->t, q, c->stream, &c->launches);
-        else launch_gather_attn_v1(c->t, q, c->stream, &c->launches);
+        launch_gather_attn_tma(c->t, q, out, c->stream, &c->launches);
+    } else {
+        { TimeScope ts(c, KC_ATTN, timed); launch_gather_attn_v1(c->t, q, c->stream, &c->launches); }
+        { TimeScope ts(c, KC_COMBINE, timed); launch_attn_combine(c->t, out, c->stream, &c->launches); }
     }
-    { TimeScope ts(c, KC_COMBINE, timed); launch_attn_combine(c->t, out, c->stream, &c->launches); }
 }
 
 static void enqueue_append_apply(dynakv_ctx* c, StepPtr k, StepPtr v, bool timed) {

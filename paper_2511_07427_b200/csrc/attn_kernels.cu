@@ -2,15 +2,27 @@
 // the retrieved entries (arXiv 2511.07427, Section 2.1 / 4.1), G query heads sharing every
 // K/V row that is read.
 //
-// Each warp owns whole pages.  K and V rows go from HBM straight into mma.sync operand
-// registers with 128-bit loads (no shared-memory staging): the contraction index of
+// One persistent CTA per half SM.  The step's pages of ALL units form one flat list
+// (work_prefix[u] .. work_prefix[u+1] are unit u's entries); CTA b owns the contiguous
+// slice [b*per, (b+1)*per).  A producer warp streams the slice's pages -- exactly the
+// valid rows of each, K and V, as two bulk-asynchronous copies (TMA, 1-D) -- into a
+// shared-memory ring guarded by full/empty mbarriers; three consumer warps take the pages
+// round-robin, each keeping an online-softmax state (m, l, acc) for the unit in progress.
+//
+// Consumer arithmetic: mma.sync m16n8k16 bf16 with fp32 accumulation.  K and V rows go
+// from shared memory into operand registers with 128-bit loads: the contraction index of
 // Q.K^T is permuted so that the 16 bytes a thread loads from a K row are exactly its B
 // fragments of two k-steps, and the output columns of P.V are permuted so that the 16
 // bytes a thread loads from each of its four V rows become, after one byte-permute per
 // register, its B fragments of eight n-tiles.  Q (pre-scaled by log2(e)/sqrt(d)) and the
 // softmax weights P are each split into bf16 hi + lo parts that sit in rows r and r+8 of
 // the 16-row MMA tile, which the same thread accumulates, so fp32 queries and weights
-// lose nothing that matters (2^-17 relative) and no cross-lane traffic is needed.
+// lose nothing that matters (2^-17 relative).
+//
+// Split-K combine: a unit whose entries lie inside one CTA's slice is normalised and
+// written by that CTA.  A unit cut by slice boundaries leaves one unnormalised partial per
+// CTA; each such CTA bumps the unit's arrival counter and the last one to arrive merges
+// the partials and writes the output, so no CTA ever waits for another.
 #include <float.h>
 
 #include "common.cuh"
@@ -33,165 +45,384 @@ __device__ __forceinline__ void split2(float x, float y, unsigned& hi, unsigned&
     lo = (unsigned)__bfloat16_as_ushort(xl) | ((unsigned)__bfloat16_as_ushort(yl) << 16);
 }
 
-__device__ __forceinline__ uint4 ldg16(const void* p) {
+__device__ __forceinline__ uint4 lds16(unsigned addr) {
     uint4 v;
-    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];\n"
-                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+    asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];\n" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
     return v;
 }
 
-constexpr int AT_WARPS = 4;
+// ---- mbarrier / bulk-copy primitives (shared::cta addresses as 32-bit values)
+__device__ __forceinline__ unsigned smem_u32(const void* p) { return (unsigned)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(unsigned bar, unsigned count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(unsigned bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];\n" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(unsigned bar, unsigned bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(unsigned bar, unsigned parity) {
+    unsigned ok;
+    asm volatile(
+        "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}\n"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ unsigned long long global_ns() {
+    unsigned long long v;
+    asm volatile("mov.u64 %0, %%globaltimer;\n" : "=l"(v));
+    return v;
+}
+// Bounded wait: gives up after 2^22 polls or about 0.2 s, whichever comes first.
+__device__ __forceinline__ bool mbar_wait(unsigned bar, unsigned parity) {
+    unsigned long long t0 = 0;
+    for (int i = 0; i < (1 << 22); i++) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((i & 63) == 63) {
+            const unsigned long long now = global_ns();
+            if (t0 == 0) t0 = now;
+            else if (now - t0 > 200000000ull) return false;
+        }
+    }
+    return false;
+}
+__device__ __forceinline__ void bulk_g2s(unsigned dst, const void* src, unsigned bytes, unsigned bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];\n"
+                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+constexpr int AT_CONSUMERS = 3;                     // consumer warps
+constexpr int AT_THREADS = (AT_CONSUMERS + 1) * 32; // + one producer warp
+constexpr int AT_STAGES = 6;                        // pages in flight per CTA
+// Item i of a CTA's slice is consumed by warp i % AT_CONSUMERS from ring stage i % AT_STAGES.  A stage
+// must always be consumed by the same warp: a parity wait cannot tell phase p from phase p + 2, so a
+// warp must never be able to run two phases ahead of another warp on a shared stage.
+static_assert(AT_STAGES % AT_CONSUMERS == 0, "each ring stage belongs to one consumer warp");
+
+__device__ __forceinline__ void consumer_sync() { asm volatile("bar.sync 1, %0;\n" ::"n"(AT_CONSUMERS * 32) : "memory"); }
+
+template <int HD> struct AttnSmem {
+    static constexpr int stage_bytes = 2 * PAGE * HD * 2;                 // K page then V page
+    static constexpr int ring_bytes = AT_STAGES * stage_bytes;
+    static constexpr int merge_bytes = AT_CONSUMERS * 8 * (HD + 2) * 4;   // per warp: acc[8][HD], m[8], l[8]
+    static constexpr int fixed_bytes = ring_bytes + merge_bytes + 2 * AT_STAGES * 8 + AT_STAGES * 4 + 64;
+};
+
+// Smallest u with pf[u+1] > k, starting the search at u0 (pf non-decreasing).
+__device__ __forceinline__ int unit_of(const int* pf, int u0, int k) {
+    int u = u0;
+    while (pf[u + 1] <= k) u++;
+    return u;
+}
 
 template <int HD>
-__global__ void __launch_bounds__(AT_WARPS * 32, 2) k_gather_attn_mma(Tables t, StepPtr qp) {
+__global__ void __launch_bounds__(AT_THREADS, 2) k_gather_attn_tma(Tables t, StepPtr qp, StepPtrW outp) {
     constexpr int KS = HD / 16;       // k-steps of Q.K^T
     constexpr int KJ = KS / 2;        // 16-byte chunks a thread loads per K row
     constexpr int NT = HD / 8;        // n-tiles of P.V
     constexpr int VI = HD / 64;       // 16-byte chunks a thread loads per V row
-    const int s = blockIdx.x, u = blockIdx.y, S = gridDim.x;
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int r = lane >> 2, c = lane & 3;
-    const int G = t.G;
-    const float* q = reinterpret_cast<const float*>(qp.get()) + (size_t)u * G * HD;
-    const float scale = rsqrtf((float)HD) * 1.4426950408889634f;
+    constexpr int ROWB = HD * 2;      // bytes per K or V row
+    extern __shared__ __align__(128) unsigned char smem[];
+    unsigned char* ring = smem;
+    float* mrg = reinterpret_cast<float*>(smem + AttnSmem<HD>::ring_bytes);
+    unsigned long long* bars = reinterpret_cast<unsigned long long*>(smem + AttnSmem<HD>::ring_bytes + AttnSmem<HD>::merge_bytes);
+    int* meta = reinterpret_cast<int*>(bars + 2 * AT_STAGES);
+    int* s_flag = meta + AT_STAGES;                  // [0] abort, [1] combine-here, [2] copies issued
+    int* pf_s = s_flag + 16;                         // copy of work_prefix when it fits
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int U = t.U, G = t.G;
+    const int nb = gridDim.x, b = blockIdx.x;
 
-    // Q fragments: rows 0..7 = hi part of head r, rows 8..15 = lo part of head r
-    unsigned qa[KS][4];
-#pragma unroll
-    for (int ks = 0; ks < KS; ks++) {
-        const int base = 8 * (c + 4 * (ks >> 1)) + 4 * (ks & 1);
-        float x0 = 0.f, x1 = 0.f, x2 = 0.f, x3 = 0.f;
-        if (r < G) {
-            const float4 v = *reinterpret_cast<const float4*>(q + r * HD + base);
-            x0 = v.x * scale; x1 = v.y * scale; x2 = v.z * scale; x3 = v.w * scale;
-        }
-        split2(x0, x1, qa[ks][0], qa[ks][1]);
-        split2(x2, x3, qa[ks][2], qa[ks][3]);
+    // ---- prologue: barriers, prefix copy, slice bounds
+    if (tid == 0) {
+        for (int s = 0; s < AT_STAGES; s++) { mbar_init(smem_u32(&bars[s]), 1); mbar_init(smem_u32(&bars[AT_STAGES + s]), 1); }
+        s_flag[0] = 0; s_flag[1] = 0; s_flag[2] = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
     }
-    float o[NT][4];
-#pragma unroll
-    for (int x = 0; x < NT; x++) { o[x][0] = 0.f; o[x][1] = 0.f; o[x][2] = 0.f; o[x][3] = 0.f; }
-    float m = -INFINITY, l = 0.f;
-
-    const int nw = t.n_work[u];
-    const int per = (nw + S - 1) / S;
-    const int w0 = s * per, w1 = min(nw, w0 + per);
-    const int2* work = t.work + (size_t)u * t.W;
-    const __nv_bfloat16* kpg = reinterpret_cast<const __nv_bfloat16*>(t.kpages) + (size_t)u * t.P * PAGE * HD;
-    const __nv_bfloat16* vpg = reinterpret_cast<const __nv_bfloat16*>(t.vpages) + (size_t)u * t.P * PAGE * HD;
-
-    for (int w = w0 + warp; w < w1; w += AT_WARPS) {
-        const int2 ent = work[w];
-        for (int half = 0; half < 2; half++) {
-            const int nvalid = ent.y - half * 16;
-            if (nvalid <= 0) break;
-            const size_t row0 = (size_t)ent.x * PAGE + half * 16;
-            // ---- loads: K rows (tile*8 + r), chunks c + 4j; V rows 2c, 2c+1, 2c+8, 2c+9, chunks r + 8i
-            uint4 kw[2][KJ];
-#pragma unroll
-            for (int tile = 0; tile < 2; tile++) {
-                const bool ok = tile * 8 + r < nvalid;
-                const __nv_bfloat16* kr = kpg + (row0 + tile * 8 + r) * HD;
-#pragma unroll
-                for (int j = 0; j < KJ; j++) kw[tile][j] = ok ? ldg16(kr + 8 * (c + 4 * j)) : make_uint4(0, 0, 0, 0);
-            }
-            uint4 vw[4][VI];
-#pragma unroll
-            for (int rr = 0; rr < 4; rr++) {
-                const int tok = 2 * c + (rr & 1) + 8 * (rr >> 1);
-                const bool ok = tok < nvalid;
-                const __nv_bfloat16* vr = vpg + (row0 + tok) * HD;
-#pragma unroll
-                for (int i = 0; i < VI; i++) vw[rr][i] = ok ? ldg16(vr + 8 * (r + 8 * i)) : make_uint4(0, 0, 0, 0);
-            }
-            // ---- S = Q K^T for the two 8-token tiles
-            float sc[2][4];
-#pragma unroll
-            for (int tile = 0; tile < 2; tile++) {
-                sc[tile][0] = 0.f; sc[tile][1] = 0.f; sc[tile][2] = 0.f; sc[tile][3] = 0.f;
-#pragma unroll
-                for (int j = 0; j < KJ; j++) {
-                    mma_bf16(sc[tile], qa[2 * j][0], qa[2 * j][1], qa[2 * j][2], qa[2 * j][3], kw[tile][j].x, kw[tile][j].y);
-                    mma_bf16(sc[tile], qa[2 * j + 1][0], qa[2 * j + 1][1], qa[2 * j + 1][2], qa[2 * j + 1][3], kw[tile][j].z, kw[tile][j].w);
-                }
-            }
-            // logits of head r for tokens tile*8 + 2c + {0,1}: hi row + lo row
-            float lg[4];
-#pragma unroll
-            for (int tile = 0; tile < 2; tile++) {
-                const int tok = tile * 8 + 2 * c;
-                lg[tile * 2 + 0] = tok < nvalid ? sc[tile][0] + sc[tile][2] : -INFINITY;
-                lg[tile * 2 + 1] = tok + 1 < nvalid ? sc[tile][1] + sc[tile][3] : -INFINITY;
-            }
-            float mx = fmaxf(fmaxf(lg[0], lg[1]), fmaxf(lg[2], lg[3]));
-            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
-            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
-            const float mn = fmaxf(m, mx);                 // finite: token 0 of the half page is valid
-            const float corr = exp2f(m - mn);
-            m = mn;
-            float p[4];
-#pragma unroll
-            for (int e = 0; e < 4; e++) p[e] = exp2f(lg[e] - mn);
-            l = l * corr + (p[0] + p[1]) + (p[2] + p[3]);
-            unsigned pa[4];
-            split2(p[0], p[1], pa[0], pa[1]);   // a0 = hi(tile 0), a1 = lo(tile 0)
-            split2(p[2], p[3], pa[2], pa[3]);   // a2 = hi(tile 1), a3 = lo(tile 1)
-#pragma unroll
-            for (int x = 0; x < NT; x++) { o[x][0] *= corr; o[x][1] *= corr; o[x][2] *= corr; o[x][3] *= corr; }
-            // ---- O += P V : n-tile (i, e) takes element e of chunk i of the thread's four rows
-#pragma unroll
-            for (int i = 0; i < VI; i++) {
-                const unsigned* a0 = reinterpret_cast<const unsigned*>(&vw[0][i]);
-                const unsigned* a1 = reinterpret_cast<const unsigned*>(&vw[1][i]);
-                const unsigned* a2 = reinterpret_cast<const unsigned*>(&vw[2][i]);
-                const unsigned* a3 = reinterpret_cast<const unsigned*>(&vw[3][i]);
-#pragma unroll
-                for (int e = 0; e < 8; e++) {
-                    const unsigned sel = (e & 1) ? 0x7632u : 0x5410u;
-                    const unsigned b0 = __byte_perm(a0[e >> 1], a1[e >> 1], sel);
-                    const unsigned b1 = __byte_perm(a2[e >> 1], a3[e >> 1], sel);
-                    mma_bf16(o[i * 8 + e], pa[0], pa[1], pa[2], pa[3], b0, b1);
-                }
-            }
-        }
-    }
-    l += __shfl_xor_sync(0xffffffffu, l, 1);
-    l += __shfl_xor_sync(0xffffffffu, l, 2);
-
-    // ---- merge the warps of the block, write the partial (acc, m, l) of split s
-    __shared__ float sm_m[AT_WARPS][8], sm_l[AT_WARPS][8];
-    __shared__ float sm_o[AT_WARPS][8][HD];
-    if (c == 0) { sm_m[warp][r] = m; sm_l[warp][r] = l; }
-#pragma unroll
-    for (int x = 0; x < NT; x++) {
-        const int i = x >> 3, e = x & 7;
-        sm_o[warp][r][8 * (2 * c + 8 * i) + e] = o[x][0] + o[x][2];
-        sm_o[warp][r][8 * (2 * c + 1 + 8 * i) + e] = o[x][1] + o[x][3];
+    const int* pf = t.work_prefix;
+    if (t.attn_pf_in_smem) {
+        for (int i = tid; i <= U; i += AT_THREADS) pf_s[i] = pf[i];
+        pf = pf_s;
     }
     __syncthreads();
-    float* part = t.part + (((size_t)u * S + s) * G) * (HD + 2);
-    for (int idx = threadIdx.x; idx < G * HD; idx += AT_WARPS * 32) {
-        const int g = idx / HD, e = idx % HD;
-        float mm = sm_m[0][g];
+    const int Wtot = pf[U];
+    const int per = max((Wtot + nb - 1) / nb, 1);
+    const int lo = min(b * per, Wtot), hi = min(lo + per, Wtot);
+    float* out = reinterpret_cast<float*>(outp.get());
+    // units with nothing selected: zeros
+    if (warp > 0) {
+        for (int u = b; u < U; u += nb)
+            if (pf[u + 1] == pf[u])
+                for (int i = tid - 32; i < G * HD; i += AT_CONSUMERS * 32) out[(size_t)u * G * HD + i] = 0.f;
+    }
+    if (lo >= hi) return;
+    const int n_items = hi - lo;
+
+    if (warp == 0) {
+        // =============================== producer ===============================
+        int u = unit_of(pf, 0, lo);
+        const __nv_bfloat16* kp = reinterpret_cast<const __nv_bfloat16*>(t.kpages);
+        const __nv_bfloat16* vp = reinterpret_cast<const __nv_bfloat16*>(t.vpages);
+        for (int it0 = 0; it0 < n_items; it0 += 32) {
+            // every lane fetches the work entry of one item
+            const int myk = lo + it0 + lane;
+            int2 ent = make_int2(0, 0); int myu = 0;
+            if (myk < hi) {
+                myu = unit_of(pf, u, myk);
+                ent = t.work[(size_t)myu * t.W + (myk - pf[myu])];
+            }
+            const int cnt = min(32, n_items - it0);
+            for (int j = 0; j < cnt; j++) {
+                const int page = __shfl_sync(0xffffffffu, ent.x, j), rows = __shfl_sync(0xffffffffu, ent.y, j);
+                const int uu = __shfl_sync(0xffffffffu, myu, j);
+                const int it = it0 + j, stage = it % AT_STAGES;
+                const unsigned ph = (unsigned)(it / AT_STAGES) & 1u;
+                if (lane == 0) {
+                    bool ok = mbar_wait(smem_u32(&bars[AT_STAGES + stage]), ph ^ 1u);
+                    if (!ok || *(volatile int*)&s_flag[0]) { s_flag[0] = 1; }
+                    else {
+                        const unsigned bytes = (unsigned)rows * ROWB;
+                        const unsigned full = smem_u32(&bars[stage]);
+                        const unsigned dst = smem_u32(ring + (size_t)stage * AttnSmem<HD>::stage_bytes);
+                        const size_t src = (((size_t)uu * t.P + page) * PAGE) * HD;
+                        meta[stage] = rows;
+                        mbar_arrive_expect_tx(full, 2 * bytes);
+                        bulk_g2s(dst, kp + src, bytes, full);
+                        bulk_g2s(dst + PAGE * ROWB, vp + src, bytes, full);
+                        s_flag[2] = it + 1;          // copies issued so far
+                    }
+                }
+                if (__shfl_sync(0xffffffffu, *(volatile int*)&s_flag[0], 0)) break;
+            }
+            if (*(volatile int*)&s_flag[0]) break;
+            u = __shfl_sync(0xffffffffu, myu, cnt - 1);
+        }
+        if (lane == 0 && *(volatile int*)&s_flag[0]) {
+            // a bounded wait ran out: report it, and let every copy already issued land before this
+            // CTA's shared memory can be handed to another CTA
+            atomicOr(t.status, DYNAKV_ST_INTERNAL);
+            const int issued = *(volatile int*)&s_flag[2];
+            for (int s = 0; s < AT_STAGES; s++)
+                if (issued - 1 >= s) {
+                    const int it_s = ((issued - 1 - s) / AT_STAGES) * AT_STAGES + s;
+                    mbar_wait(smem_u32(&bars[s]), (unsigned)(it_s / AT_STAGES) & 1u);
+                }
+        }
+        return;
+    }
+
+    // =============================== consumers ===============================
+    const int cw = warp - 1, ctid = tid - 32;
+    const int r = lane >> 2, c = lane & 3;
+    const float scale = rsqrtf((float)HD) * 1.4426950408889634f;
+    const float* qbase = reinterpret_cast<const float*>(qp.get());
+    float* mrg_o = mrg;                                   // [AT_CONSUMERS][8][HD]
+    float* mrg_m = mrg + AT_CONSUMERS * 8 * HD;           // [AT_CONSUMERS][8]
+    float* mrg_l = mrg_m + AT_CONSUMERS * 8;              // [AT_CONSUMERS][8]
+
+    int u = unit_of(pf, 0, lo);
+    const int u_first = u;
+    int k = lo;
+    while (k < hi) {
+        u = unit_of(pf, u, k);
+        const int seg_end = min(hi, pf[u + 1]);
+        // ---- Q fragments of unit u: rows 0..7 = hi part of head r, rows 8..15 = lo part of head r
+        const float* q = qbase + (size_t)u * G * HD;
+        unsigned qa[KS][4];
 #pragma unroll
-        for (int w = 1; w < AT_WARPS; w++) mm = fmaxf(mm, sm_m[w][g]);
-        float a = 0.f, ll = 0.f;
-        if (mm != -INFINITY) {
+        for (int ks = 0; ks < KS; ks++) {
+            const int base = 8 * (c + 4 * (ks >> 1)) + 4 * (ks & 1);
+            float x0 = 0.f, x1 = 0.f, x2 = 0.f, x3 = 0.f;
+            if (r < G) {
+                const float4 v = *reinterpret_cast<const float4*>(q + r * HD + base);
+                x0 = v.x * scale; x1 = v.y * scale; x2 = v.z * scale; x3 = v.w * scale;
+            }
+            split2(x0, x1, qa[ks][0], qa[ks][1]);
+            split2(x2, x3, qa[ks][2], qa[ks][3]);
+        }
+        float o[NT][4];
 #pragma unroll
-            for (int w = 0; w < AT_WARPS; w++) {
-                const float f = exp2f(sm_m[w][g] - mm);
-                a += sm_o[w][g][e] * f; ll += sm_l[w][g] * f;
+        for (int x = 0; x < NT; x++) { o[x][0] = 0.f; o[x][1] = 0.f; o[x][2] = 0.f; o[x][3] = 0.f; }
+        float m = -INFINITY, l = 0.f;
+
+        // first item of this segment owned by this warp: (kk - lo) % AT_CONSUMERS == cw
+        int kk = k + ((cw - ((k - lo) % AT_CONSUMERS)) + AT_CONSUMERS) % AT_CONSUMERS;
+        bool dead = false;
+        for (; kk < seg_end; kk += AT_CONSUMERS) {
+            const int it = kk - lo, stage = it % AT_STAGES;
+            const unsigned ph = (unsigned)(it / AT_STAGES) & 1u;
+            if (!mbar_wait(smem_u32(&bars[stage]), ph) || *(volatile int*)&s_flag[0]) { s_flag[0] = 1; dead = true; break; }
+            const int rows = meta[stage];
+            const unsigned kbase = smem_u32(ring + (size_t)stage * AttnSmem<HD>::stage_bytes);
+            const unsigned vbase = kbase + PAGE * ROWB;
+#pragma unroll 1
+            for (int half = 0; half < 2; half++) {
+                const int nvalid = rows - half * 16;
+                if (nvalid <= 0) break;
+                const unsigned krow0 = kbase + (unsigned)(half * 16) * ROWB, vrow0 = vbase + (unsigned)(half * 16) * ROWB;
+                // ---- loads: K rows (tile*8 + r), chunks c + 4j; V rows 2c, 2c+1, 2c+8, 2c+9, chunks r + 8i
+                uint4 kw[2][KJ];
+#pragma unroll
+                for (int tile = 0; tile < 2; tile++) {
+                    const bool ok = tile * 8 + r < nvalid;
+#pragma unroll
+                    for (int j = 0; j < KJ; j++)
+                        kw[tile][j] = ok ? lds16(krow0 + (unsigned)(tile * 8 + r) * ROWB + 16u * (c + 4 * j)) : make_uint4(0, 0, 0, 0);
+                }
+                uint4 vw[4][VI];
+#pragma unroll
+                for (int rr = 0; rr < 4; rr++) {
+                    const int tok = 2 * c + (rr & 1) + 8 * (rr >> 1);
+                    const bool ok = tok < nvalid;
+#pragma unroll
+                    for (int i = 0; i < VI; i++)
+                        vw[rr][i] = ok ? lds16(vrow0 + (unsigned)tok * ROWB + 16u * (r + 8 * i)) : make_uint4(0, 0, 0, 0);
+                }
+                // ---- S = Q K^T for the two 8-token tiles
+                float sc[2][4];
+#pragma unroll
+                for (int tile = 0; tile < 2; tile++) {
+                    sc[tile][0] = 0.f; sc[tile][1] = 0.f; sc[tile][2] = 0.f; sc[tile][3] = 0.f;
+#pragma unroll
+                    for (int j = 0; j < KJ; j++) {
+                        mma_bf16(sc[tile], qa[2 * j][0], qa[2 * j][1], qa[2 * j][2], qa[2 * j][3], kw[tile][j].x, kw[tile][j].y);
+                        mma_bf16(sc[tile], qa[2 * j + 1][0], qa[2 * j + 1][1], qa[2 * j + 1][2], qa[2 * j + 1][3], kw[tile][j].z, kw[tile][j].w);
+                    }
+                }
+                // logits of head r for tokens tile*8 + 2c + {0,1}: hi row + lo row
+                float lg[4];
+#pragma unroll
+                for (int tile = 0; tile < 2; tile++) {
+                    const int tok = tile * 8 + 2 * c;
+                    lg[tile * 2 + 0] = tok < nvalid ? sc[tile][0] + sc[tile][2] : -INFINITY;
+                    lg[tile * 2 + 1] = tok + 1 < nvalid ? sc[tile][1] + sc[tile][3] : -INFINITY;
+                }
+                float mx = fmaxf(fmaxf(lg[0], lg[1]), fmaxf(lg[2], lg[3]));
+                mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+                mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+                const float mn = fmaxf(m, mx);                 // finite: token 0 of the half page is valid
+                const float corr = exp2f(m - mn);
+                m = mn;
+                float p[4];
+#pragma unroll
+                for (int e = 0; e < 4; e++) p[e] = exp2f(lg[e] - mn);
+                l = l * corr + (p[0] + p[1]) + (p[2] + p[3]);
+                unsigned pa[4];
+                split2(p[0], p[1], pa[0], pa[1]);   // a0 = hi(tile 0), a1 = lo(tile 0)
+                split2(p[2], p[3], pa[2], pa[3]);   // a2 = hi(tile 1), a3 = lo(tile 1)
+#pragma unroll
+                for (int x = 0; x < NT; x++) { o[x][0] *= corr; o[x][1] *= corr; o[x][2] *= corr; o[x][3] *= corr; }
+                // ---- O += P V : n-tile (i, e) takes element e of chunk i of the thread's four rows
+#pragma unroll
+                for (int i = 0; i < VI; i++) {
+                    const unsigned* a0 = reinterpret_cast<const unsigned*>(&vw[0][i]);
+                    const unsigned* a1 = reinterpret_cast<const unsigned*>(&vw[1][i]);
+                    const unsigned* a2 = reinterpret_cast<const unsigned*>(&vw[2][i]);
+                    const unsigned* a3 = reinterpret_cast<const unsigned*>(&vw[3][i]);
+#pragma unroll
+                    for (int e = 0; e < 8; e++) {
+                        const unsigned sel = (e & 1) ? 0x7632u : 0x5410u;
+                        const unsigned b0 = __byte_perm(a0[e >> 1], a1[e >> 1], sel);
+                        const unsigned b1 = __byte_perm(a2[e >> 1], a3[e >> 1], sel);
+                        mma_bf16(o[i * 8 + e], pa[0], pa[1], pa[2], pa[3], b0, b1);
+                    }
+                }
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&bars[AT_STAGES + stage]));
+        }
+        l += __shfl_xor_sync(0xffffffffu, l, 1);
+        l += __shfl_xor_sync(0xffffffffu, l, 2);
+
+        // ---- merge the consumer warps' states for unit u
+        if (c == 0) { mrg_m[cw * 8 + r] = m; mrg_l[cw * 8 + r] = l; }
+#pragma unroll
+        for (int x = 0; x < NT; x++) {
+            const int i = x >> 3, e = x & 7;
+            mrg_o[(cw * 8 + r) * HD + 8 * (2 * c + 8 * i) + e] = o[x][0] + o[x][2];
+            mrg_o[(cw * 8 + r) * HD + 8 * (2 * c + 1 + 8 * i) + e] = o[x][1] + o[x][3];
+        }
+        consumer_sync();
+        if (*(volatile int*)&s_flag[0] || dead) {
+            if (ctid == 0) atomicOr(t.status, DYNAKV_ST_INTERNAL);
+            return;      // all consumer warps see the flag after the barrier and leave together
+        }
+        const bool whole = pf[u] >= lo && pf[u + 1] <= hi;
+        float* part = t.part + ((size_t)(2 * b + (u == u_first ? 0 : 1)) * G) * (HD + 2);
+        for (int idx = ctid; idx < G * HD; idx += AT_CONSUMERS * 32) {
+            const int g = idx / HD, e = idx % HD;
+            float mm = mrg_m[g];
+#pragma unroll
+            for (int w = 1; w < AT_CONSUMERS; w++) mm = fmaxf(mm, mrg_m[w * 8 + g]);
+            float a = 0.f, ll = 0.f;
+            if (mm != -INFINITY) {
+#pragma unroll
+                for (int w = 0; w < AT_CONSUMERS; w++) {
+                    const float f = exp2f(mrg_m[w * 8 + g] - mm);
+                    a += mrg_o[(w * 8 + g) * HD + e] * f; ll += mrg_l[w * 8 + g] * f;
+                }
+            }
+            if (whole) out[(size_t)u * G * HD + idx] = ll > 0.f ? a / ll : 0.f;
+            else {
+                __stcg(&part[g * (HD + 2) + e], a);
+                if (e == 0) { __stcg(&part[g * (HD + 2) + HD], mm); __stcg(&part[g * (HD + 2) + HD + 1], ll); }
             }
         }
-        part[g * (HD + 2) + e] = a;
-        if (e == 0) { part[g * (HD + 2) + HD] = mm; part[g * (HD + 2) + HD + 1] = ll; }
+        if (!whole) {
+            // ---- arrival: the last CTA holding a piece of unit u merges all pieces
+            const int c_lo = pf[u] / per, c_hi = (pf[u + 1] - 1) / per;
+            __threadfence();
+            consumer_sync();
+            if (ctid == 0) {
+                const int old = atomicAdd(&t.unit_arrive[u], 1);
+                s_flag[1] = (old == c_hi - c_lo) ? 1 : 0;
+                if (old == c_hi - c_lo) t.unit_arrive[u] = 0;
+            }
+            consumer_sync();
+            if (s_flag[1]) {
+                __threadfence();
+                for (int idx = ctid; idx < G * HD; idx += AT_CONSUMERS * 32) {
+                    const int g = idx / HD, e = idx % HD;
+                    float mm = -INFINITY;
+                    for (int cc = c_lo; cc <= c_hi; cc++) {
+                        const int slot = (cc == c_lo && cc * per != pf[u]) ? 1 : 0;
+                        mm = fmaxf(mm, __ldcg(t.part + ((size_t)(2 * cc + slot) * G + g) * (HD + 2) + HD));
+                    }
+                    float a = 0.f, ll = 0.f;
+                    if (mm != -INFINITY) {
+                        for (int cc = c_lo; cc <= c_hi; cc++) {
+                            const int slot = (cc == c_lo && cc * per != pf[u]) ? 1 : 0;
+                            const float* ps = t.part + ((size_t)(2 * cc + slot) * G + g) * (HD + 2);
+                            const float f = exp2f(__ldcg(ps + HD) - mm);
+                            a += __ldcg(ps + e) * f; ll += __ldcg(ps + HD + 1) * f;
+                        }
+                    }
+                    out[(size_t)u * G * HD + idx] = ll > 0.f ? a / ll : 0.f;
+                }
+            }
+        }
+        consumer_sync();     // merge scratch and s_flag[1] are free again
+        k = seg_end;
     }
 }
 
-void launch_gather_attn_mma(const Tables& t, StepPtr q, cudaStream_t s, long long* launches) {
-    dim3 grid(t.n_splits_attn, t.U);
-    if (t.d == 64) k_gather_attn_mma<64><<<grid, AT_WARPS * 32, 0, s>>>(t, q);
-    else k_gather_attn_mma<128><<<grid, AT_WARPS * 32, 0, s>>>(t, q);
+size_t attn_tma_smem_bytes(const Tables& t) {
+    const size_t fixed = t.d == 64 ? AttnSmem<64>::fixed_bytes : AttnSmem<128>::fixed_bytes;
+    return fixed + (t.attn_pf_in_smem ? (size_t)(t.U + 1) * 4 : 0) + 64;
+}
+
+int attn_tma_prepare(const Tables& t) {
+    const int bytes = (int)attn_tma_smem_bytes(t);
+    cudaError_t e = t.d == 64
+        ? cudaFuncSetAttribute(k_gather_attn_tma<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes)
+        : cudaFuncSetAttribute(k_gather_attn_tma<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+    return e == cudaSuccess ? 0 : -1;
+}
+
+void launch_gather_attn_tma(const Tables& t, StepPtr q, StepPtrW out, cudaStream_t s, long long* launches) {
+    const size_t bytes = attn_tma_smem_bytes(t);
+    if (t.d == 64) k_gather_attn_tma<64><<<t.n_attn_ctas, AT_THREADS, bytes, s>>>(t, q, out);
+    else k_gather_attn_tma<128><<<t.n_attn_ctas, AT_THREADS, bytes, s>>>(t, q, out);
     (*launches)++;
 }
 

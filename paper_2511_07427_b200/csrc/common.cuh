@@ -41,7 +41,12 @@ struct Tables {
     int* sel_n; int* sel_tokens;     // [U]
     int2* work;                      // [U][W] (page, count)
     int* n_work;                     // [U]
-    float* part;                     // [U][S][G][d + 2]  partial (acc, m, l)
+    float* part;                     // partial (acc, m, l) records of [G][d + 2] floats: [U][S] (plain kernel) or [2 * n_attn_ctas]
+    int* work_prefix;                // [U + 1] exclusive prefix of n_work over the units (written by the last select block)
+    int* unit_arrive;                // [U] arrival counters of the split-K combine (zero between steps)
+    int* plan_counter;               // [1] select blocks finished in this step
+    int n_attn_ctas;                 // persistent gather-attention CTAs (2 per SM)
+    int attn_pf_in_smem;             // 1: every attention CTA keeps a copy of work_prefix in shared memory
     // split scratch
     unsigned char* sp_label;         // [U][max_tokens]
     int* sp_pos;                     // [U][2 * max_tokens]: rank per position, then hole list
@@ -156,7 +161,8 @@ void launch_finalize(const Tables& t, const void* K, const void* V, long long n,
 void launch_front(const Tables& t, StepPtr q, StepPtr k, int has_q, int has_k, cudaStream_t s, long long* launches);
 void launch_select(const Tables& t, int budget, int* user_sel_ids, cudaStream_t s, long long* launches);
 void launch_append_apply(const Tables& t, StepPtr k, StepPtr v, cudaStream_t s, long long* launches);
-void launch_gather_attn_mma(const Tables& t, StepPtr q, cudaStream_t s, long long* launches);
+void launch_gather_attn_tma(const Tables& t, StepPtr q, StepPtrW out, cudaStream_t s, long long* launches);
+int attn_tma_prepare(const Tables& t);
 void launch_gather_attn_v1(const Tables& t, StepPtr q, cudaStream_t s, long long* launches);
 void launch_attn_combine(const Tables& t, StepPtrW out, cudaStream_t s, long long* launches);
 void launch_split_check(const Tables& t, float gamma, int var_enabled, int min_size, int iters, cudaStream_t s,

@@ -93,7 +93,8 @@ constexpr int SL_EPT = SL_MAXM / SL_THREADS;   // entries per thread
 // prefix of live clusters whose sizes sum to <= budget, by a three-level radix select on
 // the orderable score key with the cluster sizes as weights; if not even the best cluster
 // fits it is taken alone.  Writes the selection (id order) and its page work list; when
-// `user_ids` is given it also writes the selection in score order, -1 padded.
+// `user_ids` is given it also writes the selection in score order, -1 padded.  The last block
+// to finish also writes the exclusive prefix of the units' work-list lengths.
 __global__ void __launch_bounds__(SL_THREADS) k_select(Tables t, int budget, int* __restrict__ user_ids) {
     const int u = blockIdx.x, tid = threadIdx.x;
     __shared__ unsigned int keys[SL_MAXM];
@@ -255,6 +256,25 @@ __global__ void __launch_bounds__(SL_THREADS) k_select(Tables t, int budget, int
             uo[rank] = j;
         }
         for (int p = L + tid; p < t.max_clusters; p += SL_THREADS) uo[p] = -1;
+    }
+    // ---- the last unit block to finish lays the units' work lists end to end: exclusive prefix of n_work
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) {
+        const int old = atomicAdd(t.plan_counter, 1);
+        s_done = (old == t.U - 1) ? 1 : 0;
+    }
+    __syncthreads();
+    if (s_done) {
+        __threadfence();
+        const int per_t = (t.U + SL_THREADS - 1) / SL_THREADS;
+        const int b0 = min(tid * per_t, t.U), b1 = min(b0 + per_t, t.U);
+        int sum = 0;
+        for (int i = b0; i < b1; i++) sum += __ldcg(&t.n_work[i]);
+        int tot;
+        int base = block_scan_excl(sum, sh, &tot);
+        for (int i = b0; i < b1; i++) { t.work_prefix[i] = base; base += __ldcg(&t.n_work[i]); }
+        if (tid == 0) { t.work_prefix[t.U] = tot; *t.plan_counter = 0; }
     }
 }
 

@@ -38,6 +38,14 @@ def test_group_sizes_head_dims_dtypes(G, d, dtype):
     _run(cfg, [0], cfg.steps, assign_mode=1)
 
 
+def test_attention_ring_wraps_and_units_cut_by_slices():
+    # 96 units x ~190 pages: every persistent attention CTA streams a slice of ~60 pages (ten times its
+    # ring depth) and most units are cut by slice boundaries, so the split-K combine runs for them
+    cfg = CONFIGS[4].scaled(n_prefill=6000, steps=6, M0=200, max_clusters=512, budget=4096, T=3)
+    rep = _run(cfg, [0, 17, 95], cfg.steps, ctx_units=list(range(96)), assign_mode=1)
+    assert rep.status_bits & P.ST_INTERNAL == 0 and min(rep.tokens_selected) > 3000
+
+
 def test_plain_attention_kernel_on_bf16():
     cfg = CONFIGS[5].scaled(B=1, L=1, n_prefill=600, steps=16, M0=24, max_clusters=64, budget=200, T=3)
     from parity_harness import make_ctx
