@@ -380,6 +380,7 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=64)
     ap.add_argument("--profile-steps", type=int, default=64)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--budget", type=int, default=0, help="override the config's token budget (tuning aid)")
     ap.add_argument("--units", type=int, default=0,
                     help="run only the first N units of the config (profiling aid: smaller device footprint); 0 = all")
     ap.add_argument("--attn-traffic-bytes", type=float, default=None,
@@ -390,6 +391,8 @@ def main():
     if args.units > 0:
         # keep the per-unit shape; B*L*Hkv collapses to N units of one layer
         cfg = cfg.scaled(B=1, L=1, Hkv=args.units, Hq=args.units * cfg.G, name=cfg.name + f"[first {args.units} units]")
+    if args.budget > 0:
+        cfg = cfg.scaled(budget=args.budget, name=cfg.name + f"[budget {args.budget}]")
     if args.impl == "reference":
         run_reference(args, cfg)
     else:

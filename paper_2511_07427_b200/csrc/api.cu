@@ -130,7 +130,7 @@ extern "C" int dynakv_create(const dynakv_config* cfg, void* cuda_stream, dynakv
     const int full_pages = (cfg->max_tokens + PAGE - 1) / PAGE;
     int slack = full_pages / 8; if (slack < 64) slack = 64;
     t.P = full_pages + cfg->max_clusters + slack;
-    t.W = t.P;
+    t.W = (PAGE / ENTRY_ROWS) * t.P;
     t.n_splits_attn = 8;
     {
         int dev = 0, sms = 0;
@@ -171,7 +171,7 @@ extern "C" int dynakv_create(const dynakv_config* cfg, void* cuda_stream, dynakv
     {
         size_t recs = U * (size_t)t.n_splits_attn;
         if (recs < 2 * (size_t)t.n_attn_ctas) recs = 2 * (size_t)t.n_attn_ctas;
-        ALLOC(t.part, recs * t.G * (d + 2), false);
+        ALLOC(t.part, recs * (t.G * (d + 2) + 16), false);
     }
     ALLOC(t.work_prefix, U + 1, true);
     ALLOC(t.unit_arrive, U, true);

@@ -91,18 +91,24 @@ __device__ __forceinline__ void bulk_g2s(unsigned dst, const void* src, unsigned
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];\n"
                  ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
 }
-constexpr int AT_CONSUMERS = 3;                     // consumer warps
+#ifndef DKV_AT_CONSUMERS
+#define DKV_AT_CONSUMERS 3
+#endif
+#ifndef DKV_AT_STAGES
+#define DKV_AT_STAGES 6
+#endif
+constexpr int AT_CONSUMERS = DKV_AT_CONSUMERS;      // consumer warps
 constexpr int AT_THREADS = (AT_CONSUMERS + 1) * 32; // + one producer warp
-constexpr int AT_STAGES = 6;                        // pages in flight per CTA
+constexpr int AT_STAGES = DKV_AT_STAGES;                      // work entries (runs of <= ENTRY_ROWS rows) in flight per CTA
 // Item i of a CTA's slice is consumed by warp i % AT_CONSUMERS from ring stage i % AT_STAGES.  A stage
 // must always be consumed by the same warp: a parity wait cannot tell phase p from phase p + 2, so a
 // warp must never be able to run two phases ahead of another warp on a shared stage.
-static_assert(AT_STAGES % AT_CONSUMERS == 0, "each ring stage belongs to one consumer warp");
+static_assert(AT_STAGES <= 32 && AT_STAGES % AT_CONSUMERS == 0, "each ring stage belongs to one consumer warp");
 
 __device__ __forceinline__ void consumer_sync() { asm volatile("bar.sync 1, %0;\n" ::"n"(AT_CONSUMERS * 32) : "memory"); }
 
 template <int HD> struct AttnSmem {
-    static constexpr int stage_bytes = 2 * PAGE * HD * 2;                 // K page then V page
+    static constexpr int stage_bytes = 2 * ENTRY_ROWS * HD * 2;                 // K rows then V rows of one entry
     static constexpr int ring_bytes = AT_STAGES * stage_bytes;
     static constexpr int merge_bytes = AT_CONSUMERS * 8 * (HD + 2) * 4;   // per warp: acc[8][HD], m[8], l[8]
     static constexpr int fixed_bytes = ring_bytes + merge_bytes + 2 * AT_STAGES * 8 + AT_STAGES * 4 + 64;
@@ -113,6 +119,16 @@ __device__ __forceinline__ int unit_of(const int* pf, int u0, int k) {
     int u = u0;
     while (pf[u + 1] <= k) u++;
     return u;
+}
+
+// Same by bisection over all U units.
+__device__ __forceinline__ int unit_of_bisect(const int* pf, int U, int k) {
+    int a = 0, b = U - 1;            // invariant: the answer lies in [a, b]
+    while (a < b) {
+        const int mid = (a + b) >> 1;
+        if (pf[mid + 1] > k) b = mid; else a = mid + 1;
+    }
+    return a;
 }
 
 template <int HD>
@@ -127,7 +143,7 @@ __global__ void __launch_bounds__(AT_THREADS, 2) k_gather_attn_tma(Tables t, Ste
     float* mrg = reinterpret_cast<float*>(smem + AttnSmem<HD>::ring_bytes);
     unsigned long long* bars = reinterpret_cast<unsigned long long*>(smem + AttnSmem<HD>::ring_bytes + AttnSmem<HD>::merge_bytes);
     int* meta = reinterpret_cast<int*>(bars + 2 * AT_STAGES);
-    int* s_flag = meta + AT_STAGES;                  // [0] abort, [1] combine-here, [2] copies issued
+    int* s_flag = meta + AT_STAGES;                  // [0] abort, [1] combine-here
     int* pf_s = s_flag + 16;                         // copy of work_prefix when it fits
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int U = t.U, G = t.G;
@@ -136,7 +152,7 @@ __global__ void __launch_bounds__(AT_THREADS, 2) k_gather_attn_tma(Tables t, Ste
     // ---- prologue: barriers, prefix copy, slice bounds
     if (tid == 0) {
         for (int s = 0; s < AT_STAGES; s++) { mbar_init(smem_u32(&bars[s]), 1); mbar_init(smem_u32(&bars[AT_STAGES + s]), 1); }
-        s_flag[0] = 0; s_flag[1] = 0; s_flag[2] = 0;
+        s_flag[0] = 0; s_flag[1] = 0;
         asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
     }
     const int* pf = t.work_prefix;
@@ -160,53 +176,39 @@ __global__ void __launch_bounds__(AT_THREADS, 2) k_gather_attn_tma(Tables t, Ste
 
     if (warp == 0) {
         // =============================== producer ===============================
-        int u = unit_of(pf, 0, lo);
-        const __nv_bfloat16* kp = reinterpret_cast<const __nv_bfloat16*>(t.kpages);
-        const __nv_bfloat16* vp = reinterpret_cast<const __nv_bfloat16*>(t.vpages);
-        for (int it0 = 0; it0 < n_items; it0 += 32) {
-            // every lane fetches the work entry of one item
-            const int myk = lo + it0 + lane;
-            int2 ent = make_int2(0, 0); int myu = 0;
-            if (myk < hi) {
-                myu = unit_of(pf, u, myk);
-                ent = t.work[(size_t)myu * t.W + (myk - pf[myu])];
-            }
-            const int cnt = min(32, n_items - it0);
-            for (int j = 0; j < cnt; j++) {
-                const int page = __shfl_sync(0xffffffffu, ent.x, j), rows = __shfl_sync(0xffffffffu, ent.y, j);
-                const int uu = __shfl_sync(0xffffffffu, myu, j);
-                const int it = it0 + j, stage = it % AT_STAGES;
+        // Lane j owns ring stage j: it fetches the work entries of items j, j + AT_STAGES, ... and issues
+        // their copies as soon as the stage's consumer has released it, independently of the other lanes.
+        if (lane < AT_STAGES && lane < n_items) {
+            const __nv_bfloat16* kp = reinterpret_cast<const __nv_bfloat16*>(t.kpages);
+            const __nv_bfloat16* vp = reinterpret_cast<const __nv_bfloat16*>(t.vpages);
+            const unsigned full = smem_u32(&bars[lane]), empty = smem_u32(&bars[AT_STAGES + lane]);
+            const unsigned dst = smem_u32(ring + (size_t)lane * AttnSmem<HD>::stage_bytes);
+            int u = unit_of_bisect(pf, U, lo + lane);
+            int2 ent = t.work[(size_t)u * t.W + (lo + lane - pf[u])];
+            int last_issued = -1;
+            for (int it = lane; it < n_items; it += AT_STAGES) {
+                const int2 cur = ent;
+                const int cu = u;
+                if (it + AT_STAGES < n_items) {          // next entry: its load is in flight during the wait below
+                    u = unit_of(pf, u, lo + it + AT_STAGES);
+                    ent = t.work[(size_t)u * t.W + (lo + it + AT_STAGES - pf[u])];
+                }
                 const unsigned ph = (unsigned)(it / AT_STAGES) & 1u;
-                if (lane == 0) {
-                    bool ok = mbar_wait(smem_u32(&bars[AT_STAGES + stage]), ph ^ 1u);
-                    if (!ok || *(volatile int*)&s_flag[0]) { s_flag[0] = 1; }
-                    else {
-                        const unsigned bytes = (unsigned)rows * ROWB;
-                        const unsigned full = smem_u32(&bars[stage]);
-                        const unsigned dst = smem_u32(ring + (size_t)stage * AttnSmem<HD>::stage_bytes);
-                        const size_t src = (((size_t)uu * t.P + page) * PAGE) * HD;
-                        meta[stage] = rows;
-                        mbar_arrive_expect_tx(full, 2 * bytes);
-                        bulk_g2s(dst, kp + src, bytes, full);
-                        bulk_g2s(dst + PAGE * ROWB, vp + src, bytes, full);
-                        s_flag[2] = it + 1;          // copies issued so far
-                    }
-                }
-                if (__shfl_sync(0xffffffffu, *(volatile int*)&s_flag[0], 0)) break;
+                if (!mbar_wait(empty, ph ^ 1u)) { s_flag[0] = 1; break; }
+                const unsigned bytes = (unsigned)cur.y * ROWB;
+                const size_t src = ((size_t)cu * t.P * PAGE + cur.x) * HD;
+                meta[lane] = cur.y;
+                mbar_arrive_expect_tx(full, 2 * bytes);
+                bulk_g2s(dst, kp + src, bytes, full);
+                bulk_g2s(dst + ENTRY_ROWS * ROWB, vp + src, bytes, full);
+                last_issued = it;
             }
-            if (*(volatile int*)&s_flag[0]) break;
-            u = __shfl_sync(0xffffffffu, myu, cnt - 1);
-        }
-        if (lane == 0 && *(volatile int*)&s_flag[0]) {
-            // a bounded wait ran out: report it, and let every copy already issued land before this
-            // CTA's shared memory can be handed to another CTA
-            atomicOr(t.status, DYNAKV_ST_INTERNAL);
-            const int issued = *(volatile int*)&s_flag[2];
-            for (int s = 0; s < AT_STAGES; s++)
-                if (issued - 1 >= s) {
-                    const int it_s = ((issued - 1 - s) / AT_STAGES) * AT_STAGES + s;
-                    mbar_wait(smem_u32(&bars[s]), (unsigned)(it_s / AT_STAGES) & 1u);
-                }
+            if (*(volatile int*)&s_flag[0]) {
+                // a bounded wait ran out: report it, and let this lane's last copy land before the CTA's
+                // shared memory can be handed to another CTA
+                atomicOr(t.status, DYNAKV_ST_INTERNAL);
+                if (last_issued >= 0) mbar_wait(full, (unsigned)(last_issued / AT_STAGES) & 1u);
+            }
         }
         return;
     }
@@ -220,7 +222,7 @@ __global__ void __launch_bounds__(AT_THREADS, 2) k_gather_attn_tma(Tables t, Ste
     float* mrg_m = mrg + AT_CONSUMERS * 8 * HD;           // [AT_CONSUMERS][8]
     float* mrg_l = mrg_m + AT_CONSUMERS * 8;              // [AT_CONSUMERS][8]
 
-    int u = unit_of(pf, 0, lo);
+    int u = unit_of_bisect(pf, U, lo);
     const int u_first = u;
     int k = lo;
     while (k < hi) {
@@ -251,15 +253,15 @@ __global__ void __launch_bounds__(AT_THREADS, 2) k_gather_attn_tma(Tables t, Ste
         for (; kk < seg_end; kk += AT_CONSUMERS) {
             const int it = kk - lo, stage = it % AT_STAGES;
             const unsigned ph = (unsigned)(it / AT_STAGES) & 1u;
-            if (!mbar_wait(smem_u32(&bars[stage]), ph) || *(volatile int*)&s_flag[0]) { s_flag[0] = 1; dead = true; break; }
+            if (!mbar_wait(smem_u32(&bars[stage]), ph)) { s_flag[0] = 1; dead = true; break; }
             const int rows = meta[stage];
             const unsigned kbase = smem_u32(ring + (size_t)stage * AttnSmem<HD>::stage_bytes);
-            const unsigned vbase = kbase + PAGE * ROWB;
+            const unsigned vbase = kbase + ENTRY_ROWS * ROWB;
 #pragma unroll 1
-            for (int half = 0; half < 2; half++) {
-                const int nvalid = rows - half * 16;
+            for (int sub = 0; sub < ENTRY_ROWS / 16; sub++) {
+                const int nvalid = rows - sub * 16;
                 if (nvalid <= 0) break;
-                const unsigned krow0 = kbase + (unsigned)(half * 16) * ROWB, vrow0 = vbase + (unsigned)(half * 16) * ROWB;
+                const unsigned krow0 = kbase + (unsigned)(sub * 16) * ROWB, vrow0 = vbase + (unsigned)(sub * 16) * ROWB;
                 // ---- loads: K rows (tile*8 + r), chunks c + 4j; V rows 2c, 2c+1, 2c+8, 2c+9, chunks r + 8i
                 uint4 kw[2][KJ];
 #pragma unroll
@@ -300,7 +302,7 @@ __global__ void __launch_bounds__(AT_THREADS, 2) k_gather_attn_tma(Tables t, Ste
                 float mx = fmaxf(fmaxf(lg[0], lg[1]), fmaxf(lg[2], lg[3]));
                 mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
                 mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
-                const float mn = fmaxf(m, mx);                 // finite: token 0 of the half page is valid
+                const float mn = fmaxf(m, mx);                 // finite: row 0 of the entry is valid
                 const float corr = exp2f(m - mn);
                 m = mn;
                 float p[4];
@@ -310,8 +312,10 @@ __global__ void __launch_bounds__(AT_THREADS, 2) k_gather_attn_tma(Tables t, Ste
                 unsigned pa[4];
                 split2(p[0], p[1], pa[0], pa[1]);   // a0 = hi(tile 0), a1 = lo(tile 0)
                 split2(p[2], p[3], pa[2], pa[3]);   // a2 = hi(tile 1), a3 = lo(tile 1)
+                if (__any_sync(0xffffffffu, corr != 1.f)) {      // the running maximum rarely moves after the first entries
 #pragma unroll
-                for (int x = 0; x < NT; x++) { o[x][0] *= corr; o[x][1] *= corr; o[x][2] *= corr; o[x][3] *= corr; }
+                    for (int x = 0; x < NT; x++) { o[x][0] *= corr; o[x][1] *= corr; o[x][2] *= corr; o[x][3] *= corr; }
+                }
                 // ---- O += P V : n-tile (i, e) takes element e of chunk i of the thread's four rows
 #pragma unroll
                 for (int i = 0; i < VI; i++) {
@@ -348,7 +352,9 @@ __global__ void __launch_bounds__(AT_THREADS, 2) k_gather_attn_tma(Tables t, Ste
             return;      // all consumer warps see the flag after the barrier and leave together
         }
         const bool whole = pf[u] >= lo && pf[u + 1] <= hi;
-        float* part = t.part + ((size_t)(2 * b + (u == u_first ? 0 : 1)) * G) * (HD + 2);
+        // partial record: acc[G][HD], then m[8], then l[8] (floats; every row 16-byte aligned)
+        const size_t rec_floats = (size_t)G * HD + 16;
+        float* part = t.part + (size_t)(2 * b + (u == u_first ? 0 : 1)) * rec_floats;
         for (int idx = ctid; idx < G * HD; idx += AT_CONSUMERS * 32) {
             const int g = idx / HD, e = idx % HD;
             float mm = mrg_m[g];
@@ -364,8 +370,8 @@ __global__ void __launch_bounds__(AT_THREADS, 2) k_gather_attn_tma(Tables t, Ste
             }
             if (whole) out[(size_t)u * G * HD + idx] = ll > 0.f ? a / ll : 0.f;
             else {
-                __stcg(&part[g * (HD + 2) + e], a);
-                if (e == 0) { __stcg(&part[g * (HD + 2) + HD], mm); __stcg(&part[g * (HD + 2) + HD + 1], ll); }
+                __stcg(&part[idx], a);
+                if (e == 0) { __stcg(&part[G * HD + g], mm); __stcg(&part[G * HD + 8 + g], ll); }
             }
         }
         if (!whole) {
@@ -381,23 +387,40 @@ __global__ void __launch_bounds__(AT_THREADS, 2) k_gather_attn_tma(Tables t, Ste
             consumer_sync();
             if (s_flag[1]) {
                 __threadfence();
-                for (int idx = ctid; idx < G * HD; idx += AT_CONSUMERS * 32) {
-                    const int g = idx / HD, e = idx % HD;
-                    float mm = -INFINITY;
-                    for (int cc = c_lo; cc <= c_hi; cc++) {
-                        const int slot = (cc == c_lo && cc * per != pf[u]) ? 1 : 0;
-                        mm = fmaxf(mm, __ldcg(t.part + ((size_t)(2 * cc + slot) * G + g) * (HD + 2) + HD));
-                    }
-                    float a = 0.f, ll = 0.f;
-                    if (mm != -INFINITY) {
-                        for (int cc = c_lo; cc <= c_hi; cc++) {
-                            const int slot = (cc == c_lo && cc * per != pf[u]) ? 1 : 0;
-                            const float* ps = t.part + ((size_t)(2 * cc + slot) * G + g) * (HD + 2);
-                            const float f = exp2f(__ldcg(ps + HD) - mm);
-                            a += __ldcg(ps + e) * f; ll += __ldcg(ps + HD + 1) * f;
+                // every thread merges one float4 column of one head; the pieces are read four at a time
+                // so that their loads are in flight together
+                for (int i4 = ctid; i4 < G * HD / 4; i4 += AT_CONSUMERS * 32) {
+                    const int g = (i4 * 4) / HD;
+                    float mm = -INFINITY, ll = 0.f;
+                    float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
+                    for (int cc0 = c_lo; cc0 <= c_hi; cc0 += 4) {
+                        float mv[4], lv[4]; float4 pv[4];
+#pragma unroll
+                        for (int j = 0; j < 4; j++) {
+                            const int cc = cc0 + j;
+                            mv[j] = -INFINITY; lv[j] = 0.f; pv[j] = make_float4(0.f, 0.f, 0.f, 0.f);
+                            if (cc <= c_hi) {
+                                const int slot = (cc == c_lo && cc * per != pf[u]) ? 1 : 0;
+                                const float* ps = t.part + (size_t)(2 * cc + slot) * rec_floats;
+                                mv[j] = __ldcg(ps + G * HD + g); lv[j] = __ldcg(ps + G * HD + 8 + g);
+                                pv[j] = __ldcg(reinterpret_cast<const float4*>(ps) + i4);
+                            }
+                        }
+                        const float mnew = fmaxf(fmaxf(mm, mv[0]), fmaxf(fmaxf(mv[1], mv[2]), mv[3]));
+                        if (mnew != -INFINITY) {
+                            const float f0 = mm == -INFINITY ? 0.f : exp2f(mm - mnew);
+                            a.x *= f0; a.y *= f0; a.z *= f0; a.w *= f0; ll *= f0;
+#pragma unroll
+                            for (int j = 0; j < 4; j++) {
+                                const float f = mv[j] == -INFINITY ? 0.f : exp2f(mv[j] - mnew);
+                                a.x += pv[j].x * f; a.y += pv[j].y * f; a.z += pv[j].z * f; a.w += pv[j].w * f;
+                                ll += lv[j] * f;
+                            }
+                            mm = mnew;
                         }
                     }
-                    out[(size_t)u * G * HD + idx] = ll > 0.f ? a / ll : 0.f;
+                    const float inv = ll > 0.f ? 1.f / ll : 0.f;
+                    reinterpret_cast<float4*>(out + (size_t)u * G * HD)[i4] = make_float4(a.x * inv, a.y * inv, a.z * inv, a.w * inv);
                 }
             }
         }

@@ -12,6 +12,10 @@
 namespace dkv {
 
 constexpr int PAGE = 32;            // tokens per page
+#ifndef DKV_ENTRY_ROWS
+#define DKV_ENTRY_ROWS 32
+#endif
+constexpr int ENTRY_ROWS = DKV_ENTRY_ROWS;   // rows per gather work entry (16 or 32: a run inside one page)
 constexpr int MAX_G = 8;
 constexpr int FLAG_HOLD = 1;        // split abandoned; not retried until the next append
 
@@ -21,7 +25,7 @@ constexpr int FLAG_HOLD = 1;        // split abandoned; not retried until the ne
 //   full, so cluster members are contiguous page by page (intra-cluster placement).
 struct Tables {
     int U, G, d, kv_dtype, max_tokens, max_clusters, P, n_splits_attn;
-    int W;                           // work-list capacity per unit (page entries)
+    int W;                           // work-list capacity per unit (entries)
     void* kpages; void* vpages;
     int* page_tok;                   // [U][P][PAGE] token id per slot
     int* page_next;                  // [U][P]
@@ -39,7 +43,7 @@ struct Tables {
     float* dists;                    // [U][Mmax] squared distance of the step's new key to every representative
     int* sel_ids;                    // [U][Mmax]
     int* sel_n; int* sel_tokens;     // [U]
-    int2* work;                      // [U][W] (page, count)
+    int2* work;                      // [U][W] (first row = page * PAGE + offset, rows <= ENTRY_ROWS)
     int* n_work;                     // [U]
     float* part;                     // partial (acc, m, l) records of [G][d + 2] floats: [U][S] (plain kernel) or [2 * n_attn_ctas]
     int* work_prefix;                // [U + 1] exclusive prefix of n_work over the units (written by the last select block)

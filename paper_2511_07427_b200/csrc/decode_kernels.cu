@@ -40,7 +40,7 @@ __global__ void __launch_bounds__(128) k_gather_attn_v1(Tables t, StepPtr qp) {
     const KV* vp = reinterpret_cast<const KV*>(t.vpages);
     for (int w = w0 + warp; w < w1; w += 4) {
         int2 ent = work[w];
-        size_t pbase = (((size_t)u * t.P + ent.x) * PAGE) * HD;
+        size_t pbase = ((size_t)u * t.P * PAGE + ent.x) * HD;
         for (int r = 0; r < ent.y; r++) {
             const KV* k = kp + pbase + (size_t)r * HD + lane * EPL;
             const KV* v = vp + pbase + (size_t)r * HD + lane * EPL;

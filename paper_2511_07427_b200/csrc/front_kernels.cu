@@ -92,7 +92,8 @@ constexpr int SL_EPT = SL_MAXM / SL_THREADS;   // entries per thread
 // One block per unit.  Finds, in (score descending, id ascending) order, the longest
 // prefix of live clusters whose sizes sum to <= budget, by a three-level radix select on
 // the orderable score key with the cluster sizes as weights; if not even the best cluster
-// fits it is taken alone.  Writes the selection (id order) and its page work list; when
+// fits it is taken alone.  Writes the selection (id order) and its work list (first row, rows) of
+// runs inside one page; when
 // `user_ids` is given it also writes the selection in score order, -1 padded.  The last block
 // to finish also writes the exclusive prefix of the units' work-list lengths.
 __global__ void __launch_bounds__(SL_THREADS) k_select(Tables t, int budget, int* __restrict__ user_ids) {
@@ -219,7 +220,7 @@ __global__ void __launch_bounds__(SL_THREADS) k_select(Tables t, int budget, int
         if (e * SL_THREADS >= Mcur) break;
         const int j = tid + e * SL_THREADS;
         const int isel = selected[e] ? 1 : 0;
-        const int np = isel ? (sz[e] + PAGE - 1) / PAGE : 0;
+        const int np = isel ? (sz[e] + ENTRY_ROWS - 1) / ENTRY_ROWS : 0;   // work entries: runs of <= ENTRY_ROWS rows inside one page
         int ts, tw;
         const int spos = sbase + block_scan_excl(isel, sh, &ts);
         const int wpos = wbase + block_scan_excl(np, sh, &tw);
@@ -227,8 +228,9 @@ __global__ void __launch_bounds__(SL_THREADS) k_select(Tables t, int budget, int
             sel[spos] = j;
             int page = t.cl_head[(size_t)u * t.max_clusters + j];
             for (int i = 0; i < np && wpos + i < t.W; i++) {
-                work[wpos + i] = make_int2(page, (i + 1 < np) ? PAGE : sz[e] - PAGE * (np - 1));
-                page = t.page_next[(size_t)u * t.P + page];
+                constexpr int EPP = PAGE / ENTRY_ROWS;       // entries per page
+                work[wpos + i] = make_int2(page * PAGE + (i % EPP) * ENTRY_ROWS, min(ENTRY_ROWS, sz[e] - ENTRY_ROWS * i));
+                if (i % EPP == EPP - 1) page = t.page_next[(size_t)u * t.P + page];
             }
         }
         sbase += ts; wbase += tw;
