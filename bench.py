@@ -27,6 +27,12 @@ sys.path.insert(0, ROOT)
 
 METRIC = "decode steps/s at 32-layer 32K ctx; retrieval-attention HBM GB/s vs peak"
 
+# DRAM traffic of the gather-attention kernel from its ncu capture (profiles/gather_attn_config4_96units.txt):
+# dram__bytes_read.sum + dram__bytes_write.sum of one launch, and the tokens that launch attended.  Traffic
+# is proportional to the rows attended, so a launch's traffic is scaled by its own token count.  Set
+# NCU_ATTN_CAPTURE to None whenever the kernel changes after the capture.
+NCU_ATTN_CAPTURE = {"dram_bytes": 100.3072e6 + 2.9903e6, "tokens": 195006.5}
+
 
 def _peaks():
     p = os.path.join(ROOT, "MEASURED_PEAKS.json")
@@ -317,7 +323,10 @@ def run_ours(args, cfg):
     kernels = {k: (v["ms"] / v["launches"] * 1e3 if v["launches"] else None) for k, v in kt.items()
                if k in ("front", "select", "attn", "combine", "append", "split")}
     roofline = {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                "frac": achieved / peaks["hbm_gbs"], "traffic": args.attn_traffic_bytes,
+                "frac": achieved / peaks["hbm_gbs"],
+                "traffic": (args.attn_traffic_bytes if args.attn_traffic_bytes is not None else
+                            (NCU_ATTN_CAPTURE["dram_bytes"] * tokens_per_launch / NCU_ATTN_CAPTURE["tokens"]
+                             if NCU_ATTN_CAPTURE and cfg.kv_dtype == "bf16" and cfg.d == 128 else None)),
                 "kernel": "gather_attn", "us_per_launch": attn_ms * 1e3, "algorithmic_bytes_per_launch": attn_bytes,
                 "tokens_per_launch": tokens_per_launch, "frac_of_8TBs_nominal": achieved / 8000.0,
                 "peak_source": peaks["source"] + " copy bandwidth", "per_kernel_us": kernels}
