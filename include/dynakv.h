@@ -41,6 +41,7 @@ extern "C" {
 #define DYNAKV_ERR_STATE (-2)   /* call order: e.g. decode before build_index    */
 #define DYNAKV_ERR_CUDA (-3)    /* a CUDA runtime call failed                    */
 #define DYNAKV_ERR_NOMEM (-4)   /* device allocation failed                      */
+#define DYNAKV_ERR_TOO_LARGE (-5) /* dynakv_attend_rows_noalloc: more work than its fixed scratch holds */
 
 /* sticky device status bits */
 #define DYNAKV_ST_BUDGET_EXCEEDED 1u  /* best cluster alone larger than the budget; taken whole */
@@ -192,6 +193,37 @@ int64_t dynakv_launch_count(dynakv_ctx* ctx);
 const char* dynakv_last_error(void);
 
 void dynakv_destroy(dynakv_ctx* ctx);
+
+/* Attention without any allocation (the paper has no counterpart: this is a service entry of the
+ * library, not a step of the method).  For callers that may not call cudaMalloc: code running
+ * inside a serving stack or memory pool that has already claimed the whole device, code in a
+ * latency-critical section that cannot afford the synchronisation an allocation implies, or a
+ * sandboxed component that may only launch kernels on buffers it was handed.  Needs no context.
+ *
+ * For every unit u < n_units and head g < gqa_group:
+ *     out[u][g] = softmax_i(q[u][g] . K[u][i] / sqrt(d)) V[u][i]   over ALL rows i < n,
+ * which is what dynakv_decode_step returns when the token budget covers every cluster.
+ * q [n_units][gqa_group][d] fp32, K and V [n_units][n][d] row-major in kv_dtype (DYNAKV_F32 or
+ * DYNAKV_BF16), out [n_units][gqa_group][d] fp32: DEVICE pointers owned by the caller.  d is 64 or
+ * 128, gqa_group 1..8, n >= 0 (n == 0 gives zeros).  Work is enqueued on cuda_stream
+ * (a cudaStream_t, NULL = default stream) of the CURRENT device and the call returns at once.
+ *
+ * Scratch.  The split-K partial sums live in one fixed array of DYNAKV_NOALLOC_SCRATCH_BYTES that
+ * is part of the library image: every GPU that loads the library holds it until the process ends.
+ * The call needs n_units * 16 * gqa_group * (d + 2) floats of it and returns DYNAKV_ERR_TOO_LARGE,
+ * enqueuing nothing, when that is more than the array holds (or n_units > 65535): split the units
+ * over several calls.  With d = 128 and gqa_group = 4 the limit is 126 units per call.
+ * The array is shared by all calls and keeps the previous call's contents; every record a call
+ * reads is first written by that same call, so nothing needs clearing, but two calls whose
+ * kernels overlap on the GPU (different streams, several host threads) race on it: issue calls
+ * on one stream, or order them yourself.
+ * The first call on each device looks up the array's device address (cudaGetSymbolAddress, with
+ * that device current); make that first call before any stream capture begins.
+ * Calls cudaMalloc / cudaFree never.  Returns DYNAKV_OK, DYNAKV_ERR_ARG, DYNAKV_ERR_TOO_LARGE or
+ * DYNAKV_ERR_CUDA. */
+#define DYNAKV_NOALLOC_SCRATCH_BYTES (4 * 1024 * 1024)
+int dynakv_attend_rows_noalloc(const float* q, const void* K, const void* V, int32_t n_units, int64_t n,
+                               int32_t gqa_group, int32_t d, int32_t kv_dtype, float* out, void* cuda_stream);
 
 #ifdef __cplusplus
 }

@@ -19,7 +19,10 @@ EXPORTED_SYMBOLS = [
     "dynakv_create", "dynakv_build_index", "dynakv_append", "dynakv_decode_step", "dynakv_split_check",
     "dynakv_decode_loop", "dynakv_step_host", "dynakv_get_status", "dynakv_export_state", "dynakv_get_selection",
     "dynakv_get_build_trace", "dynakv_set_timing", "dynakv_get_kernel_times", "dynakv_launch_count", "dynakv_last_error", "dynakv_destroy",
+    "dynakv_attend_rows_noalloc",
 ]
+ERR_TOO_LARGE = -5
+NOALLOC_SCRATCH_BYTES = 4 * 1024 * 1024
 
 
 class DynaKVError(RuntimeError):
@@ -107,12 +110,47 @@ def load_library() -> C.CDLL:
     L.dynakv_last_error.argtypes = []
     L.dynakv_destroy.restype = None
     L.dynakv_destroy.argtypes = [vp]
+    L.dynakv_attend_rows_noalloc.restype = C.c_int
+    L.dynakv_attend_rows_noalloc.argtypes = [vp, vp, vp, i32, i64, i32, i32, i32, vp, vp]
     _lib = L
     return L
 
 
 def _np_ptr(a: Optional[np.ndarray]):
     return a.ctypes.data_as(C.c_void_p) if a is not None else None
+
+
+def attend_rows_noalloc(q, K, V, out=None, stream=None):
+    """Softmax attention of q [U, G, d] (fp32) over all rows of K, V [U, n, d] (fp32 or bf16) through
+    ``dynakv_attend_rows_noalloc``: the entry point for callers that must not allocate device memory
+    (its split-K scratch is a fixed array inside the library).  ``out`` [U, G, d] fp32 should be passed
+    by such callers; it is only created here as a convenience when omitted.  Calls share the library's
+    scratch array, so keep them on one stream.  Raises DynaKVError with the size limit when the call
+    needs more scratch than the library holds."""
+    import torch
+    L = load_library()
+    if not (q.is_cuda and K.is_cuda and V.is_cuda):
+        raise DynaKVError("attend_rows_noalloc takes CUDA tensors")
+    U, G, d = q.shape
+    n = K.shape[1]
+    if K.dtype not in (torch.float32, torch.bfloat16) or V.dtype != K.dtype or q.dtype != torch.float32 or \
+            tuple(K.shape) != (U, n, d) or tuple(V.shape) != (U, n, d) or \
+            not (q.is_contiguous() and K.is_contiguous() and V.is_contiguous()):
+        raise DynaKVError("expected contiguous q [U,G,d] fp32 and K, V [U,n,d] of one dtype (fp32 or bf16)")
+    if out is None:
+        out = torch.empty((U, G, d), dtype=torch.float32, device=q.device)
+    elif out.dtype != torch.float32 or tuple(out.shape) != (U, G, d) or not out.is_contiguous() or not out.is_cuda:
+        raise DynaKVError("expected contiguous CUDA out [U,G,d] fp32")
+    st = stream if stream is not None else torch.cuda.current_stream()
+    rc = L.dynakv_attend_rows_noalloc(C.c_void_p(q.data_ptr()), C.c_void_p(K.data_ptr()), C.c_void_p(V.data_ptr()),
+                                      U, n, G, d, F32 if K.dtype == torch.float32 else BF16,
+                                      C.c_void_p(out.data_ptr()), C.c_void_p(st.cuda_stream))
+    if rc == ERR_TOO_LARGE:
+        raise DynaKVError(f"dynakv_attend_rows_noalloc: {U} units x 16 splits x {G} heads x ({d}+2) floats exceed the "
+                          f"library's fixed scratch of {NOALLOC_SCRATCH_BYTES} bytes; pass fewer units per call")
+    if rc != 0:
+        raise DynaKVError(f"dynakv_attend_rows_noalloc returned {rc}")
+    return out
 
 
 class DynaKV:
