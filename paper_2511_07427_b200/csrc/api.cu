@@ -14,6 +14,7 @@ namespace dkv {
 // tensor-core distance GEMM path (assign_tc.cu)
 bool tc_assign_supported(const Tables& t, long long n, int M);
 size_t tc_assign_scratch_bytes(const Tables& t, long long n, int M);
+bool tc_assign_begin(const Tables& t, const void* K, long long n, int M, void* scratch, cudaStream_t s, long long* launches);
 void launch_assign_tc(const Tables& t, const void* K, long long n, int M, const float* C, int* assign, void* scratch,
                       cudaStream_t s, long long* launches);
 }  // namespace dkv
@@ -227,9 +228,11 @@ extern "C" int dynakv_build_index(dynakv_ctx* c, const void* K, const void* V, i
     int* assign_buf = nullptr;
     if (c->cfg.trace) { ALLOC_B(c->trace_assign, (size_t)T * U * n, false); }
     else ALLOC_B(assign_buf, U * (size_t)n, false);
-    const bool use_tc = c->cfg.assign_mode == 0 && tc_assign_supported(t, n, M);
+    bool use_tc = c->cfg.assign_mode == 0 && tc_assign_supported(t, n, M);
     void* tc_scratch = nullptr;
     if (use_tc) { char* p; ALLOC_B(p, tc_assign_scratch_bytes(t, n, M), false); tc_scratch = p; }
+    // fp16 copy of the keys; falls back to the fp32 kernel when a key is out of fp16 range
+    if (use_tc) { TimeScope ts(c, KC_INIT); use_tc = tc_assign_begin(t, K, n, M, tc_scratch, c->stream, &c->launches); }
 
     { TimeScope ts(c, KC_INIT); launch_init_centres(t, K, n, M, seed, c->cfg.init_mode, b, c->stream, &c->launches); }
     for (int it = 0; it < T; it++) {

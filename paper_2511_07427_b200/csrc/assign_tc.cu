@@ -1,8 +1,448 @@
-// Tensor-core (tcgen05) distance GEMM fused with argmin -- placeholder until the kernel lands.
+// Nearest-centre assignment of the k-means rounds as a tensor-core distance GEMM fused with
+// argmin (arXiv 2511.07427, Section 4.1: the k-means partition of Eq. 3; NewCluster of
+// Algorithm 1), for bf16 keys with d = 128.
+//
+//   a_i = argmin_j ||k_i - c_j||^2 = argmin_j ( ||c_j||^2 - 2 k_i . c_j )
+//
+// Filter + exact re-decision.  The [n x M] matrix of k_i . c_j is a dense contraction: it runs
+// on the 5th-generation tensor cores (tcgen05.mma, kind::f16, fp32 accumulators in TMEM) with the
+// keys converted to fp16 (exact for |k| in [2^-14, 65504], which a pre-pass checks) and the fp32
+// centres rounded to fp16.  Rounding the centres perturbs every value by at most
+// E_i = 2 ||k_i|| max_j||c_j|| 2^-11 (plus accumulation and packing slack), so the tensor-core
+// result is used as a FILTER: the epilogue keeps, per key, the best and second-best value; when
+// they are further apart than 2 E_i the best is provably the true argmin.  Otherwise the key is
+// put on a list and re-decided exactly in fp32 with the direct form sum (k - c)^2 over all
+// centres, the same arithmetic as the plain fp32 assignment kernel.  The [n x M] matrix never
+// leaves the chip.
+//
+// Kernel shape.  Persistent CTAs, one per SM, each looping over (unit, 128-key block) items.
+// Warp 0 issues TMA tensor loads (128-byte swizzle, no multicast) of the key block (kept for
+// all centre tiles of the item) and of 256-centre tiles into a two-stage ring; warp 1 issues
+// tcgen05.mma (M=128, N=256, K=16, eight per tile) into one of two 256-column TMEM accumulators
+// and commits to an mbarrier; warps 2-5 drain the other accumulator with tcgen05.ld, one key per
+// thread.  Every wait is bounded; on expiry the kernel sets a status bit, frees its TMEM and
+// returns.
+#include <cuda.h>
+#include <float.h>
+
+#include <cuda_fp16.h>
+
 #include "common.cuh"
 
 namespace dkv {
-bool tc_assign_supported(const Tables&, long long, int) { return false; }
-size_t tc_assign_scratch_bytes(const Tables&, long long, int) { return 0; }
-void launch_assign_tc(const Tables&, const void*, long long, int, const float*, int*, void*, cudaStream_t, long long*) {}
+
+// ------------------------------------------------------------------ small PTX wrappers
+
+__device__ __forceinline__ unsigned tc_smem_u32(const void* p) { return (unsigned)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void tc_mbar_init(unsigned bar, unsigned count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void tc_mbar_arrive(unsigned bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];\n" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_mbar_expect_tx(unsigned bar, unsigned bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool tc_mbar_try_wait(unsigned bar, unsigned parity) {
+    unsigned ok;
+    asm volatile(
+        "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}\n"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ unsigned long long tc_global_ns() {
+    unsigned long long v;
+    asm volatile("mov.u64 %0, %%globaltimer;\n" : "=l"(v));
+    return v;
+}
+// Bounded wait: 2^22 polls or about 0.5 s.
+__device__ __forceinline__ bool tc_mbar_wait(unsigned bar, unsigned parity) {
+    unsigned long long t0 = 0;
+    for (int i = 0; i < (1 << 22); i++) {
+        if (tc_mbar_try_wait(bar, parity)) return true;
+        if ((i & 63) == 63) {
+            const unsigned long long now = tc_global_ns();
+            if (t0 == 0) t0 = now;
+            else if (now - t0 > 500000000ull) return false;
+        }
+    }
+    return false;
+}
+// 2-D tiled TMA load (inner coordinate x in elements, outer coordinate y in rows), no multicast.
+__device__ __forceinline__ void tc_tma_load_2d(unsigned dst, const CUtensorMap* map, int x, int y, unsigned bar) {
+    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];\n"
+                 ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory"); }
+// D[tmem] (+)= A[smem desc] * B[smem desc]; accumulate = 0 overwrites D.
+__device__ __forceinline__ void tc_mma_f16(unsigned d_tmem, unsigned long long a_desc, unsigned long long b_desc,
+                                           unsigned idesc, unsigned accumulate) {
+    asm volatile(
+        "{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}\n"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+// mbarrier arrive once every MMA issued so far by this thread has completed.
+__device__ __forceinline__ void tc_commit(unsigned bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n" ::"r"(bar) : "memory");
+}
+// 32 consecutive fp32 columns of this thread's TMEM lane.
+__device__ __forceinline__ void tc_ld32(unsigned taddr, unsigned (&r)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];\n"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tc_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory"); }
+
+// ------------------------------------------------------------------ tiles, descriptors
+
+constexpr int TC_D = 128;                 // head dimension = contraction length
+constexpr int TC_BM = 128;                // keys per item (one TMEM lane each)
+constexpr int TC_BN = 256;                // centres per accumulator
+constexpr int TC_A_BYTES = TC_BM * TC_D * 2;          // 32 KB: two [128 rows x 128 B] swizzle panels
+constexpr int TC_B_BYTES = TC_BN * TC_D * 2;          // 64 KB: two [256 rows x 128 B] swizzle panels
+constexpr int TC_SMEM_BYTES = 2 * TC_A_BYTES + 2 * TC_B_BYTES + 1024 /* alignment */ + 256 /* barriers */;
+constexpr int TC_THREADS = 192;           // warp 0 loads, warp 1 issues MMAs, warps 2..5 drain accumulators
+constexpr unsigned TC_TMEM_COLS = 512;    // two 256-column fp32 accumulators
+
+// Shared-memory matrix descriptor of a K-major panel with 128-byte rows under the 128-byte swizzle:
+// start address / 16, leading offset unused (1), 1024 B between 8-row groups, descriptor version 1,
+// layout type 2 (128-byte swizzle).
+__device__ __forceinline__ unsigned long long tc_panel_desc(unsigned smem_addr) {
+    return (unsigned long long)((smem_addr & 0x3FFFFu) >> 4) | (1ull << 16) | ((unsigned long long)(1024 >> 4) << 32) |
+           (1ull << 46) | (2ull << 61);
+}
+// Instruction descriptor of kind::f16: fp32 accumulate, fp16 A and B, both K-major, M = 128, N = 256.
+constexpr unsigned TC_IDESC = (1u << 4) | ((unsigned)(TC_BN >> 3) << 17) | ((unsigned)(TC_BM >> 4) << 24);
+
+// ------------------------------------------------------------------ pre-passes
+
+// Keys bf16 -> fp16 (exact unless |k| > 65504, which raises *bad; values below 2^-24 lose bits, which
+// the margin covers) and ||k_i|| in fp32.  One warp per key.
+__global__ void __launch_bounds__(256) k_tc_prep_keys(const __nv_bfloat16* __restrict__ K, long long rows,
+                                                      __half* __restrict__ A16, float* __restrict__ knorm, int* __restrict__ bad) {
+    const int lane = threadIdx.x & 31;
+    long long w = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const long long nw = ((long long)gridDim.x * blockDim.x) >> 5;
+    for (; w < rows; w += nw) {
+        const float4 v = ld4(K + (size_t)w * TC_D, lane * 4);
+        const float m = fmaxf(fmaxf(fabsf(v.x), fabsf(v.y)), fmaxf(fabsf(v.z), fabsf(v.w)));
+        if (!(m <= 65504.f)) atomicOr(bad, 1);
+        __half2 h0 = __floats2half2_rn(v.x, v.y), h1 = __floats2half2_rn(v.z, v.w);
+        uint2 pk;
+        pk.x = *reinterpret_cast<unsigned*>(&h0); pk.y = *reinterpret_cast<unsigned*>(&h1);
+        *reinterpret_cast<uint2*>(A16 + (size_t)w * TC_D + lane * 4) = pk;
+        float s = v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
+        s = warp_sum(s);
+        if (lane == 0) knorm[w] = sqrtf(s);
+    }
+}
+
+// Centres fp32 -> fp16, bias_j = ||c_j||^2 (fp32, of the unrounded centre; 1e38 for the padding
+// columns j >= M), cmax[u] = max_j ||c_j||.  One warp per (unit, padded centre index).
+__global__ void __launch_bounds__(256) k_tc_prep_centres(const float* __restrict__ C, int U, int M, int Mpad,
+                                                         __half* __restrict__ B16, float* __restrict__ bias,
+                                                         unsigned* __restrict__ cmax_bits, int* __restrict__ bad) {
+    const int lane = threadIdx.x & 31;
+    const long long w = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    if (w >= (long long)U * Mpad) return;
+    const int u = (int)(w / Mpad), j = (int)(w % Mpad);
+    if (j >= M) { if (lane == 0) bias[w] = 1.0e38f; return; }     // finite: inf with packed column bits would read as NaN
+    const size_t row = (size_t)u * M + j;
+    const float4 v = *reinterpret_cast<const float4*>(C + row * TC_D + lane * 4);
+    const float m = fmaxf(fmaxf(fabsf(v.x), fabsf(v.y)), fmaxf(fabsf(v.z), fabsf(v.w)));
+    if (!(m <= 65504.f)) atomicOr(bad, 1);
+    __half2 h0 = __floats2half2_rn(v.x, v.y), h1 = __floats2half2_rn(v.z, v.w);
+    uint2 pk;
+    pk.x = *reinterpret_cast<unsigned*>(&h0); pk.y = *reinterpret_cast<unsigned*>(&h1);
+    *reinterpret_cast<uint2*>(B16 + row * TC_D + lane * 4) = pk;
+    float s = v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
+    s = warp_sum(s);
+    if (lane == 0) {
+        bias[w] = s;
+        atomicMax(&cmax_bits[u], __float_as_uint(sqrtf(s)));     // non-negative floats order like their bit patterns
+    }
+}
+
+// ------------------------------------------------------------------ the distance GEMM + top-2 filter
+
+struct TcArgs {
+    int U, n, M, Mpad, KB;               // KB = 128-key blocks per unit
+    const float* bias;                   // [U][Mpad]
+    const float* knorm;                  // [U * n]
+    const unsigned* cmax_bits;           // [U]
+    int* assign;                         // [U * n]
+    int* recheck_list;                   // [U][n] key indices (inside the unit) to re-decide exactly
+    unsigned* recheck_count;             // [U]
+    unsigned int* status;
+};
+
+__global__ void __launch_bounds__(TC_THREADS, 1) k_tc_assign(const __grid_constant__ CUtensorMap mapA,
+                                                             const __grid_constant__ CUtensorMap mapB, TcArgs p) {
+    extern __shared__ unsigned char tc_smem_raw[];
+    const unsigned raw = tc_smem_u32(tc_smem_raw);
+    const unsigned base = (raw + 1023u) & ~1023u;                    // swizzle panels need 1024-byte alignment
+    unsigned char* gen = tc_smem_raw + (base - raw);
+    const unsigned sA = base, sB = base + 2 * TC_A_BYTES;
+    unsigned long long* bars = reinterpret_cast<unsigned long long*>(gen + 2 * TC_A_BYTES + 2 * TC_B_BYTES);
+    // barrier indices: 0,1 a_full; 2,3 a_empty; 4,5 b_full; 6,7 b_empty; 8,9 acc_full; 10,11 acc_empty
+    auto bar = [&](int i) { return tc_smem_u32(&bars[i]); };
+    volatile unsigned* s_tmem = reinterpret_cast<volatile unsigned*>(&bars[12]);
+    volatile int* s_abort = reinterpret_cast<volatile int*>(&bars[13]);
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int NT = p.Mpad / TC_BN;
+    const long long n_items = (long long)p.U * p.KB;
+
+    if (tid == 0) {
+        for (int i = 0; i < 8; i++) tc_mbar_init(bar(i), 1);
+        tc_mbar_init(bar(8), 1); tc_mbar_init(bar(9), 1);
+        tc_mbar_init(bar(10), 4); tc_mbar_init(bar(11), 4);           // one arrival per epilogue warp
+        *s_abort = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;\n"
+                     ::"r"(tc_smem_u32((const void*)s_tmem)), "r"(TC_TMEM_COLS) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;\n" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const unsigned tmem = *s_tmem;
+
+    if (warp == 0) {
+        // =============================== TMA producer ===============================
+        if (lane == 0) {
+            long long ia = 0, tb = 0;
+            long long lastA[2] = {-1, -1}, lastB[2] = {-1, -1};
+            for (long long it = blockIdx.x; it < n_items && !*s_abort; it += gridDim.x, ia++) {
+                const int u = (int)(it / p.KB), kb = (int)(it % p.KB);
+                const int ab = (int)(ia & 1);
+                if (!tc_mbar_wait(bar(2 + ab), (unsigned)((ia >> 1) & 1) ^ 1u)) { *s_abort = 1; break; }
+                tc_mbar_expect_tx(bar(ab), TC_A_BYTES);
+                const int rowA = u * p.n + kb * TC_BM;
+                tc_tma_load_2d(sA + ab * TC_A_BYTES, &mapA, 0, rowA, bar(ab));
+                tc_tma_load_2d(sA + ab * TC_A_BYTES + TC_A_BYTES / 2, &mapA, 64, rowA, bar(ab));
+                lastA[ab] = ia;
+                for (int nt = 0; nt < NT; nt++, tb++) {
+                    const int st = (int)(tb & 1);
+                    if (!tc_mbar_wait(bar(6 + st), (unsigned)((tb >> 1) & 1) ^ 1u)) { *s_abort = 1; break; }
+                    tc_mbar_expect_tx(bar(4 + st), TC_B_BYTES);
+                    const int rowB = u * p.M + nt * TC_BN;
+                    tc_tma_load_2d(sB + st * TC_B_BYTES, &mapB, 0, rowB, bar(4 + st));
+                    tc_tma_load_2d(sB + st * TC_B_BYTES + TC_B_BYTES / 2, &mapB, 64, rowB, bar(4 + st));
+                    lastB[st] = tb;
+                }
+            }
+            if (*s_abort) {
+                // let the copies already issued land before the shared memory can be reused
+                for (int i = 0; i < 2; i++) {
+                    if (lastA[i] >= 0) tc_mbar_wait(bar(i), (unsigned)((lastA[i] >> 1) & 1));
+                    if (lastB[i] >= 0) tc_mbar_wait(bar(4 + i), (unsigned)((lastB[i] >> 1) & 1));
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // =============================== MMA issuer ===============================
+        if (lane == 0) {
+            long long ia = 0, tb = 0;
+            for (long long it = blockIdx.x; it < n_items && !*s_abort; it += gridDim.x, ia++) {
+                const int ab = (int)(ia & 1);
+                if (!tc_mbar_wait(bar(ab), (unsigned)((ia >> 1) & 1))) { *s_abort = 1; break; }
+                for (int nt = 0; nt < NT; nt++, tb++) {
+                    const int st = (int)(tb & 1);
+                    if (!tc_mbar_wait(bar(4 + st), (unsigned)((tb >> 1) & 1)) ||
+                        !tc_mbar_wait(bar(10 + st), (unsigned)((tb >> 1) & 1) ^ 1u)) { *s_abort = 1; break; }
+                    tc_fence_after();
+#pragma unroll
+                    for (int k = 0; k < TC_D / 16; k++) {
+                        const unsigned a_addr = sA + ab * TC_A_BYTES + (k >> 2) * (TC_A_BYTES / 2) + (k & 3) * 32;
+                        const unsigned b_addr = sB + st * TC_B_BYTES + (k >> 2) * (TC_B_BYTES / 2) + (k & 3) * 32;
+                        tc_mma_f16(tmem + st * TC_BN, tc_panel_desc(a_addr), tc_panel_desc(b_addr), TC_IDESC, k > 0 ? 1u : 0u);
+                    }
+                    tc_commit(bar(6 + st));       // centre tile may be overwritten
+                    tc_commit(bar(8 + st));       // accumulator is complete
+                }
+                if (*s_abort) break;
+                tc_commit(bar(2 + ab));           // key block may be overwritten
+            }
+        }
+    } else {
+        // =============================== accumulator drain (warps 2..5) ===============================
+        const int q = warp & 3;                       // TMEM lane quarter this warp may read
+        const int row = q * 32 + lane;                // key of this thread inside the item
+        long long tb = 0;
+        for (long long it = blockIdx.x; it < n_items; it += gridDim.x) {
+            const int u = (int)(it / p.KB), kb = (int)(it % p.KB);
+            const int i = kb * TC_BM + row;
+            float b1 = INFINITY, b2 = INFINITY;       // best and second-best packed values (low 8 bits = column)
+            int best_nt = 0;
+            bool dead = false;
+            for (int nt = 0; nt < NT; nt++, tb++) {
+                const int st = (int)(tb & 1);
+                if (*s_abort || !tc_mbar_wait(bar(8 + st), (unsigned)((tb >> 1) & 1))) { *s_abort = 1; dead = true; break; }
+                tc_fence_after();
+                const unsigned old_bits = __float_as_uint(b1);
+                const float4* bias4 = reinterpret_cast<const float4*>(p.bias + (size_t)u * p.Mpad + (size_t)nt * TC_BN);
+#pragma unroll 1
+                for (int c = 0; c < TC_BN / 32; c++) {
+                    unsigned acc[32];
+                    tc_ld32(tmem + st * TC_BN + c * 32 + ((unsigned)(q * 32) << 16), acc);
+                    float bs[32];
+#pragma unroll
+                    for (int e = 0; e < 8; e++) {
+                        const float4 v = __ldg(bias4 + c * 8 + e);
+                        bs[4 * e] = v.x; bs[4 * e + 1] = v.y; bs[4 * e + 2] = v.z; bs[4 * e + 3] = v.w;
+                    }
+                    tc_ld_wait();
+#pragma unroll
+                    for (int e = 0; e < 32; e++) {
+                        const float x = fmaf(-2.f, __uint_as_float(acc[e]), bs[e]);
+                        const float pk = __uint_as_float((__float_as_uint(x) & 0xFFFFFF00u) | (unsigned)(c * 32 + e));
+                        const float hi = fmaxf(b1, pk);
+                        b1 = fminf(b1, pk);
+                        b2 = fminf(b2, hi);
+                    }
+                }
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) tc_mbar_arrive(bar(10 + st));          // accumulator may be overwritten
+                if (__float_as_uint(b1) != old_bits) best_nt = nt;
+            }
+            if (dead) break;
+            if (i < p.n) {
+                const size_t gi = (size_t)u * p.n + i;
+                const int j = best_nt * TC_BN + (int)(__float_as_uint(b1) & 0xFFu);
+                p.assign[gi] = j < p.M ? j : 0;
+                const float kn = p.knorm[gi], cm = __uint_as_float(p.cmax_bits[u]);
+                // bound on |filter value - true value|: fp16 rounding of the centres (2 kn cm 2^-11, with 3 % slack
+                // for the accumulation), truncation of the 8 packed bits (2^-15 |x|), sub-normal keys
+                const float E = kn * cm * (1.03f / 1024.f) + (cm * cm + 2.f * kn * cm) * (1.f / 32768.f) + cm * 1e-6f;
+                if (!(b2 - b1 > 2.f * E)) {
+                    const unsigned pos = atomicAdd(&p.recheck_count[u], 1u);
+                    p.recheck_list[(size_t)u * p.n + pos] = i;
+                }
+            }
+        }
+    }
+    // ---- everyone meets here, on every path; then the allocating warp frees the tensor memory
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    if (warp == 1) {
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;\n" ::"r"(tmem), "r"(TC_TMEM_COLS) : "memory");
+    }
+    if (tid == 0 && *s_abort) atomicOr(p.status, DYNAKV_ST_INTERNAL);
+}
+
+// ------------------------------------------------------------------ host side
+
+static size_t tc_align(size_t x) { return (x + 255) & ~(size_t)255; }
+
+struct TcLayout {
+    size_t a16, knorm, b16, bias, cmax, bad, list, count, total;
+    int Mpad;
+};
+static TcLayout tc_layout(const Tables& t, long long n, int M) {
+    TcLayout L;
+    const size_t U = t.U;
+    L.Mpad = (M + TC_BN - 1) / TC_BN * TC_BN;
+    size_t off = 0;
+    L.a16 = off; off += tc_align(U * (size_t)n * TC_D * 2);
+    L.knorm = off; off += tc_align(U * (size_t)n * 4);
+    L.b16 = off; off += tc_align(U * (size_t)M * TC_D * 2);
+    L.bias = off; off += tc_align(U * (size_t)L.Mpad * 4);
+    L.cmax = off; off += tc_align(U * 4);
+    L.bad = off; off += 256;
+    L.list = off; off += tc_align(U * (size_t)n * 4);
+    L.count = off; off += tc_align(U * 4);
+    L.total = off;
+    return L;
+}
+
+bool tc_assign_supported(const Tables& t, long long n, int M) {
+    return t.kv_dtype == DYNAKV_BF16 && t.d == TC_D && M >= 1 && n >= 1 && (long long)t.U * n < (1ll << 31) &&
+           (long long)t.U * M < (1ll << 31);
+}
+
+size_t tc_assign_scratch_bytes(const Tables& t, long long n, int M) { return tc_layout(t, n, M).total; }
+
+// Once per build: fp16 copy of the keys and their norms.  Synchronises the stream to read the range flag;
+// returns false (use the fp32 kernel) when a key does not fit fp16 or a CUDA call failed.
+bool tc_assign_begin(const Tables& t, const void* K, long long n, int M, void* scratch, cudaStream_t s, long long* launches) {
+    const TcLayout L = tc_layout(t, n, M);
+    char* base = reinterpret_cast<char*>(scratch);
+    int* bad = reinterpret_cast<int*>(base + L.bad);
+    if (cudaMemsetAsync(bad, 0, 256, s) != cudaSuccess) return false;
+    const long long rows = (long long)t.U * n;
+    long long blocks = (rows + 7) / 8;
+    if (blocks > 148LL * 32) blocks = 148LL * 32;
+    k_tc_prep_keys<<<(unsigned)blocks, 256, 0, s>>>(reinterpret_cast<const __nv_bfloat16*>(K), rows,
+                                                   reinterpret_cast<__half*>(base + L.a16),
+                                                   reinterpret_cast<float*>(base + L.knorm), bad);
+    (*launches)++;
+    int h_bad = 1;
+    if (cudaMemcpyAsync(&h_bad, bad, sizeof(int), cudaMemcpyDeviceToHost, s) != cudaSuccess) return false;
+    if (cudaStreamSynchronize(s) != cudaSuccess) return false;
+    if (h_bad) return false;
+    static bool attr_set = false;
+    if (!attr_set) {
+        if (cudaFuncSetAttribute(k_tc_assign, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_SMEM_BYTES) != cudaSuccess) {
+            cudaGetLastError();
+            return false;
+        }
+        attr_set = true;
+    }
+    return true;
+}
+
+static bool tc_make_map(CUtensorMap* map, void* ptr, unsigned long long rows, unsigned box_rows) {
+    cuuint64_t dims[2] = {(cuuint64_t)TC_D, (cuuint64_t)rows};
+    cuuint64_t strides[1] = {(cuuint64_t)TC_D * 2};
+    cuuint32_t box[2] = {64u, box_rows};
+    cuuint32_t estr[2] = {1u, 1u};
+    return cuTensorMapEncodeTiled(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, ptr, dims, strides, box, estr,
+                                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                                  CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// One Lloyd round's assignment: centre pre-pass, distance GEMM + filter, exact re-decision of the listed keys.
+void launch_assign_tc(const Tables& t, const void* K, long long n, int M, const float* C, int* assign, void* scratch,
+                      cudaStream_t s, long long* launches) {
+    const TcLayout L = tc_layout(t, n, M);
+    char* base = reinterpret_cast<char*>(scratch);
+    __half* A16 = reinterpret_cast<__half*>(base + L.a16);
+    __half* B16 = reinterpret_cast<__half*>(base + L.b16);
+    float* bias = reinterpret_cast<float*>(base + L.bias);
+    unsigned* cmax = reinterpret_cast<unsigned*>(base + L.cmax);
+    int* bad = reinterpret_cast<int*>(base + L.bad);
+    int* list = reinterpret_cast<int*>(base + L.list);
+    unsigned* count = reinterpret_cast<unsigned*>(base + L.count);
+    cudaMemsetAsync(cmax, 0, (size_t)t.U * 4, s);
+    cudaMemsetAsync(count, 0, (size_t)t.U * 4, s);
+    const long long cw = (long long)t.U * L.Mpad;
+    k_tc_prep_centres<<<(unsigned)((cw + 7) / 8), 256, 0, s>>>(C, t.U, M, L.Mpad, B16, bias, cmax, bad);
+    CUtensorMap mapA, mapB;
+    if (!tc_make_map(&mapA, A16, (unsigned long long)t.U * n, TC_BM) || !tc_make_map(&mapB, B16, (unsigned long long)t.U * M, TC_BN)) {
+        // cannot describe the operands to the TMA unit: do the whole round exactly
+        launch_assign_f32(t, K, n, M, C, assign, s, launches);
+        return;
+    }
+    TcArgs a;
+    a.U = t.U; a.n = (int)n; a.M = M; a.Mpad = L.Mpad; a.KB = (int)((n + TC_BM - 1) / TC_BM);
+    a.bias = bias; a.knorm = reinterpret_cast<const float*>(base + L.knorm); a.cmax_bits = cmax;
+    a.assign = assign; a.recheck_list = list; a.recheck_count = count; a.status = t.status;
+    const int grid = t.n_attn_ctas / 2;        // one persistent CTA per SM
+    k_tc_assign<<<grid, TC_THREADS, TC_SMEM_BYTES, s>>>(mapA, mapB, a);
+    (*launches) += 2;
+    launch_assign_f32_listed(t, K, n, M, C, assign, list, count, &t.counters[CNT_RECHECKED], s, launches);
+}
+
 }  // namespace dkv

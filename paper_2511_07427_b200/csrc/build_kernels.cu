@@ -145,9 +145,12 @@ template <int HD> struct AssignSmem {
     static constexpr size_t bytes = sizeof(float) * ((size_t)HD * KS + (size_t)HD * CS);
 };
 
+// With `list` given (per unit: list[u][0 .. counts[u]) are key indices), only the listed keys are assigned.
 template <typename KV, int HD>
 __global__ void __launch_bounds__(AS_THREADS) k_assign_f32(const KV* __restrict__ K, int n, int M,
-                                                           const float* __restrict__ C, int* __restrict__ assign) {
+                                                           const float* __restrict__ C, int* __restrict__ assign,
+                                                           const int* __restrict__ list, const unsigned* __restrict__ counts,
+                                                           unsigned long long* __restrict__ listed_total) {
     extern __shared__ __align__(16) float smem[];
     constexpr int KS = AssignSmem<HD>::KS, CS = AssignSmem<HD>::CS;
     float* keysT = smem;                 // [HD][KS]
@@ -157,11 +160,15 @@ __global__ void __launch_bounds__(AS_THREADS) k_assign_f32(const KV* __restrict_
     const KV* Ku = K + (size_t)u * n * HD;
     const float* Cu = C + (size_t)u * M * HD;
     const int ty = tid >> 4, tx = tid & 15;
+    const int n_here = list ? (int)counts[u] : n;          // keys this unit has to assign
+    if (key0 >= n_here) return;
+    const int* lu = list ? list + (size_t)u * n : nullptr;
+    if (list && blockIdx.x == 0 && tid == 0) atomicAdd(listed_total, (unsigned long long)n_here);
 
     for (int idx = tid; idx < AS_BK * (HD / 4); idx += AS_THREADS) {
         int key = idx % AS_BK, t4 = idx / AS_BK;
         float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (key0 + key < n) v = ld4(Ku + (size_t)(key0 + key) * HD, t4 * 4);
+        if (key0 + key < n_here) v = ld4(Ku + (size_t)(lu ? lu[key0 + key] : key0 + key) * HD, t4 * 4);
         keysT[(t4 * 4 + 0) * KS + key] = v.x; keysT[(t4 * 4 + 1) * KS + key] = v.y;
         keysT[(t4 * 4 + 2) * KS + key] = v.z; keysT[(t4 * 4 + 3) * KS + key] = v.w;
     }
@@ -212,7 +219,7 @@ __global__ void __launch_bounds__(AS_THREADS) k_assign_f32(const KV* __restrict_
             if (ov < best[i] || (ov == best[i] && oj < bj[i])) { best[i] = ov; bj[i] = oj; }
         }
         int key = key0 + ty * 8 + i;
-        if (tx == 0 && key < n) assign[(size_t)u * n + key] = bj[i];
+        if (tx == 0 && key < n_here) assign[(size_t)u * n + (lu ? lu[key] : key)] = bj[i];
     }
 }
 
@@ -393,6 +400,7 @@ void launch_init_centres(const Tables& t, const void* K, long long n, int M, uns
 
 template <typename KV, int HD>
 static void assign_f32_t(const Tables& t, const void* K, long long n, int M, const float* C, int* assign,
+                         const int* list, const unsigned* counts, unsigned long long* listed_total,
                          cudaStream_t s, long long* launches) {
     static bool attr_set = false;
     if (!attr_set) {
@@ -400,13 +408,21 @@ static void assign_f32_t(const Tables& t, const void* K, long long n, int M, con
         attr_set = true;
     }
     dim3 grid((unsigned)((n + AS_BK - 1) / AS_BK), t.U);
-    k_assign_f32<KV, HD><<<grid, AS_THREADS, AssignSmem<HD>::bytes, s>>>((const KV*)K, (int)n, M, C, assign);
+    k_assign_f32<KV, HD><<<grid, AS_THREADS, AssignSmem<HD>::bytes, s>>>((const KV*)K, (int)n, M, C, assign, list, counts,
+                                                                       listed_total);
     (*launches)++;
 }
 
 void launch_assign_f32(const Tables& t, const void* K, long long n, int M, const float* C, int* assign,
                        cudaStream_t s, long long* launches) {
-    DKV_DISPATCH(assign_f32_t, t, K, n, M, C, assign, s, launches);
+    const int* list = nullptr; const unsigned* counts = nullptr; unsigned long long* listed_total = nullptr;
+    DKV_DISPATCH(assign_f32_t, t, K, n, M, C, assign, list, counts, listed_total, s, launches);
+}
+
+void launch_assign_f32_listed(const Tables& t, const void* K, long long n, int M, const float* C, int* assign,
+                              const int* list, const unsigned* counts, unsigned long long* listed_total,
+                              cudaStream_t s, long long* launches) {
+    DKV_DISPATCH(assign_f32_t, t, K, n, M, C, assign, list, counts, listed_total, s, launches);
 }
 
 template <typename KV, int HD>

@@ -158,6 +158,9 @@ void launch_init_centres(const Tables& t, const void* K, long long n, int M, uns
                          int init_mode, const BuildScratch& b, cudaStream_t s, long long* launches);
 void launch_assign_f32(const Tables& t, const void* K, long long n, int M, const float* C, int* assign,
                        cudaStream_t s, long long* launches);
+void launch_assign_f32_listed(const Tables& t, const void* K, long long n, int M, const float* C, int* assign,
+                              const int* list, const unsigned* counts, unsigned long long* listed_total,
+                              cudaStream_t s, long long* launches);
 void launch_update(const Tables& t, const void* K, long long n, int M, const int* assign, const BuildScratch& b,
                    cudaStream_t s, long long* launches);
 void launch_finalize(const Tables& t, const void* K, const void* V, long long n, int M, const BuildScratch& b,

@@ -31,3 +31,24 @@ def test_scaled_bf16_configs(cid):
     cfg = base.scaled(n_prefill=1111 if cid != 3 else 333, steps=96, M0=37 if cid != 3 else 13,
                       max_clusters=160, budget=300, T=6, new_every=32 if base.new_every else 0)
     _run(cfg, [0, 1, 2], cfg.steps, assign_mode=1)
+
+
+@pytest.mark.parametrize("cid", [2, 5])
+def test_tensor_core_assign_ragged(cid):
+    """Distance GEMM on the tensor cores (assign_mode 0): 1111 keys = 8 full 128-key blocks + 87, 37 centres
+    padded to one 256-column accumulator; every Lloyd round's assignment is checked against the oracle."""
+    import paper_2511_07427_b200 as P
+    base = CONFIGS[cid]
+    cfg = base.scaled(B=1, L=1, n_prefill=1111, steps=8, M0=37, max_clusters=160, budget=300, T=6)
+    rep = _run(cfg, [0, 1, 2], cfg.steps, assign_mode=0)
+    assert rep.status_bits & P.ST_INTERNAL == 0
+
+
+def test_tensor_core_assign_several_centre_tiles():
+    """600 centres = 3 accumulator tiles (the two TMEM accumulators and the two centre stages wrap), 4500 keys,
+    5 units in the context so that CTAs take items of different units."""
+    import paper_2511_07427_b200 as P
+    cfg = CONFIGS[4].scaled(n_prefill=4500, steps=4, M0=600, max_clusters=1200, budget=512, T=4)
+    rep = _run(cfg, [0, 4], cfg.steps, ctx_units=list(range(5)), assign_mode=0)
+    assert rep.status_bits & P.ST_INTERNAL == 0
+    assert rep.rechecked < 0.5 * 5 * 4500 * 4      # the filter decides most keys
