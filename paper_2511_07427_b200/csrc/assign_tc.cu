@@ -9,10 +9,11 @@
 // keys converted to fp16 (exact for |k| in [2^-14, 65504], which a pre-pass checks) and the fp32
 // centres rounded to fp16.  Rounding the centres perturbs every value by at most
 // E_i = 2 ||k_i|| max_j||c_j|| 2^-11 (plus accumulation and packing slack), so the tensor-core
-// result is used as a FILTER: the epilogue keeps, per key, the best and second-best value; when
-// they are further apart than 2 E_i the best is provably the true argmin.  Otherwise the key is
-// put on a list and re-decided exactly in fp32 with the direct form sum (k - c)^2 over all
-// centres, the same arithmetic as the plain fp32 assignment kernel.  The [n x M] matrix never
+// result is used as a FILTER: the epilogue keeps, per key, the three smallest values; when the
+// second is further than 2 E_i from the first, the first is provably the true argmin.  Otherwise
+// the key is re-decided exactly in fp32 with the direct form sum (k - c)^2, the same arithmetic
+// as the plain fp32 assignment kernel: between the best two centres when the third value is out
+// of reach, over all centres when it is not.  The [n x M] matrix never
 // leaves the chip.
 //
 // Kernel shape.  Persistent CTAs, one per SM, each looping over (unit, 128-key block) items.
@@ -170,7 +171,30 @@ __global__ void __launch_bounds__(256) k_tc_prep_centres(const float* __restrict
     }
 }
 
-// ------------------------------------------------------------------ the distance GEMM + top-2 filter
+// ------------------------------------------------------------------ the distance GEMM + top-3 filter
+
+__device__ __forceinline__ float tc_min3(float a, float b, float c) {
+    float r;
+    asm("min.f32 %0, %1, %2, %3;\n" : "=f"(r) : "f"(a), "f"(b), "f"(c));
+    return r;
+}
+// Value with its low 8 mantissa bits replaced by a column index (a relative change below 2^-15).
+__device__ __forceinline__ float tc_pack(float x, int col) {
+    return __uint_as_float((__float_as_uint(x) & 0xFFFFFF00u) | (unsigned)col);
+}
+// (t1 <= t2 <= t3) <- the three smallest of {t1, t2, t3, x, y}.
+__device__ __forceinline__ void tc_top3_pair(float& t1, float& t2, float& t3, float x, float y) {
+    const float lo = fminf(x, y), hi = fmaxf(x, y);
+    t3 = tc_min3(t3, fmaxf(t2, lo), fmaxf(t1, hi));
+    t2 = tc_min3(fmaxf(t1, lo), t2, hi);
+    t1 = fminf(t1, lo);
+}
+// Insert (v, j) into the sorted best two (with indices) and third value.
+__device__ __forceinline__ void tc_insert(float& g1, int& j1, float& g2, int& j2, float& g3, float v, int j) {
+    if (v < g1) { g3 = g2; g2 = g1; j2 = j1; g1 = v; j1 = j; }
+    else if (v < g2) { g3 = g2; g2 = v; j2 = j; }
+    else if (v < g3) g3 = v;
+}
 
 struct TcArgs {
     int U, n, M, Mpad, KB;               // KB = 128-key blocks per unit
@@ -180,6 +204,8 @@ struct TcArgs {
     int* assign;                         // [U * n]
     int* recheck_list;                   // [U][n] key indices (inside the unit) to re-decide exactly
     unsigned* recheck_count;             // [U]
+    int2* pair_list;                     // [U * n] (global key row, j1 | j2 << 16): decide exactly between two centres
+    unsigned long long* pair_count;      // [1]
     unsigned int* status;
 };
 
@@ -276,20 +302,22 @@ __global__ void __launch_bounds__(TC_THREADS, 1) k_tc_assign(const __grid_consta
         }
     } else {
         // =============================== accumulator drain (warps 2..5) ===============================
+        // One key per thread.  Per centre tile the thread keeps the three smallest packed values (low 8 bits =
+        // column) in two independent chains, merges them into the item's best two (with indices) and third value.
         const int q = warp & 3;                       // TMEM lane quarter this warp may read
         const int row = q * 32 + lane;                // key of this thread inside the item
         long long tb = 0;
         for (long long it = blockIdx.x; it < n_items; it += gridDim.x) {
             const int u = (int)(it / p.KB), kb = (int)(it % p.KB);
             const int i = kb * TC_BM + row;
-            float b1 = INFINITY, b2 = INFINITY;       // best and second-best packed values (low 8 bits = column)
-            int best_nt = 0;
+            float g1 = INFINITY, g2 = INFINITY, g3 = INFINITY;
+            int j1 = 0, j2 = 0;
             bool dead = false;
             for (int nt = 0; nt < NT; nt++, tb++) {
                 const int st = (int)(tb & 1);
                 if (*s_abort || !tc_mbar_wait(bar(8 + st), (unsigned)((tb >> 1) & 1))) { *s_abort = 1; dead = true; break; }
                 tc_fence_after();
-                const unsigned old_bits = __float_as_uint(b1);
+                float a1 = INFINITY, a2 = INFINITY, a3 = INFINITY, c1 = INFINITY, c2 = INFINITY, c3 = INFINITY;
                 const float4* bias4 = reinterpret_cast<const float4*>(p.bias + (size_t)u * p.Mpad + (size_t)nt * TC_BN);
 #pragma unroll 1
                 for (int c = 0; c < TC_BN / 32; c++) {
@@ -303,31 +331,44 @@ __global__ void __launch_bounds__(TC_THREADS, 1) k_tc_assign(const __grid_consta
                     }
                     tc_ld_wait();
 #pragma unroll
-                    for (int e = 0; e < 32; e++) {
-                        const float x = fmaf(-2.f, __uint_as_float(acc[e]), bs[e]);
-                        const float pk = __uint_as_float((__float_as_uint(x) & 0xFFFFFF00u) | (unsigned)(c * 32 + e));
-                        const float hi = fmaxf(b1, pk);
-                        b1 = fminf(b1, pk);
-                        b2 = fminf(b2, hi);
+                    for (int e = 0; e < 32; e += 4) {
+                        const float x0 = tc_pack(fmaf(-2.f, __uint_as_float(acc[e]), bs[e]), c * 32 + e);
+                        const float x1 = tc_pack(fmaf(-2.f, __uint_as_float(acc[e + 1]), bs[e + 1]), c * 32 + e + 1);
+                        const float x2 = tc_pack(fmaf(-2.f, __uint_as_float(acc[e + 2]), bs[e + 2]), c * 32 + e + 2);
+                        const float x3 = tc_pack(fmaf(-2.f, __uint_as_float(acc[e + 3]), bs[e + 3]), c * 32 + e + 3);
+                        tc_top3_pair(a1, a2, a3, x0, x1);
+                        tc_top3_pair(c1, c2, c3, x2, x3);
                     }
                 }
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) tc_mbar_arrive(bar(10 + st));          // accumulator may be overwritten
-                if (__float_as_uint(b1) != old_bits) best_nt = nt;
+                // the tile's three smallest out of the two chains
+                const float t1 = fminf(a1, c1);
+                const float t2 = tc_min3(fmaxf(a1, c1), a2, c2);
+                const float t3 = fminf(tc_min3(a3, c3, fmaxf(a2, c1)), fmaxf(a1, c2));
+                tc_insert(g1, j1, g2, j2, g3, t1, nt * TC_BN + (int)(__float_as_uint(t1) & 0xFFu));
+                tc_insert(g1, j1, g2, j2, g3, t2, nt * TC_BN + (int)(__float_as_uint(t2) & 0xFFu));
+                tc_insert(g1, j1, g2, j2, g3, t3, nt * TC_BN + (int)(__float_as_uint(t3) & 0xFFu));
             }
             if (dead) break;
             if (i < p.n) {
                 const size_t gi = (size_t)u * p.n + i;
-                const int j = best_nt * TC_BN + (int)(__float_as_uint(b1) & 0xFFu);
-                p.assign[gi] = j < p.M ? j : 0;
+                if (j1 >= p.M) j1 = 0;
+                p.assign[gi] = j1;
                 const float kn = p.knorm[gi], cm = __uint_as_float(p.cmax_bits[u]);
                 // bound on |filter value - true value|: fp16 rounding of the centres (2 kn cm 2^-11, with 3 % slack
                 // for the accumulation), truncation of the 8 packed bits (2^-15 |x|), sub-normal keys
                 const float E = kn * cm * (1.03f / 1024.f) + (cm * cm + 2.f * kn * cm) * (1.f / 32768.f) + cm * 1e-6f;
-                if (!(b2 - b1 > 2.f * E)) {
-                    const unsigned pos = atomicAdd(&p.recheck_count[u], 1u);
-                    p.recheck_list[(size_t)u * p.n + pos] = i;
+                if (!(g2 - g1 > 2.f * E)) {
+                    if (g3 - g1 > 2.f * E && j2 < p.M) {
+                        // only the best two can be the true argmin: decide between them exactly
+                        const unsigned long long pos = atomicAdd(p.pair_count, 1ull);
+                        p.pair_list[pos] = make_int2((int)gi, j1 | (j2 << 16));
+                    } else {
+                        const unsigned pos = atomicAdd(&p.recheck_count[u], 1u);
+                        p.recheck_list[(size_t)u * p.n + pos] = i;
+                    }
                 }
             }
         }
@@ -342,12 +383,43 @@ __global__ void __launch_bounds__(TC_THREADS, 1) k_tc_assign(const __grid_consta
     if (tid == 0 && *s_abort) atomicOr(p.status, DYNAKV_ST_INTERNAL);
 }
 
+// Exact decision between two centres for the keys whose third-best filter value is out of reach: squared
+// distances by the direct form, summed in index order in fp32 like the plain assignment kernel; ties to the
+// lower id.  One thread per listed key.
+__global__ void __launch_bounds__(256) k_tc_pair_decide(const __nv_bfloat16* __restrict__ K, const float* __restrict__ C, int n, int M,
+                                                        const int2* __restrict__ list, const unsigned long long* __restrict__ count,
+                                                        int* __restrict__ assign, unsigned long long* __restrict__ rechecked_total) {
+    const unsigned long long idx = (unsigned long long)blockIdx.x * blockDim.x + threadIdx.x;
+    const unsigned long long cnt = *count;
+    if (idx == 0 && cnt) atomicAdd(rechecked_total, cnt);
+    if (idx >= cnt) return;
+    const int2 ent = list[idx];
+    const int j1 = ent.y & 0xFFFF, j2 = (ent.y >> 16) & 0xFFFF;
+    const int u = ent.x / n;
+    const __nv_bfloat16* k = K + (size_t)ent.x * TC_D;
+    const float* ca = C + ((size_t)u * M + j1) * TC_D;
+    const float* cb = C + ((size_t)u * M + j2) * TC_D;
+    float d1 = 0.f, d2 = 0.f;
+#pragma unroll 4
+    for (int e = 0; e < TC_D; e += 4) {
+        const float4 kk = ld4(k, e);
+        const float4 a = *reinterpret_cast<const float4*>(ca + e);
+        const float4 b = *reinterpret_cast<const float4*>(cb + e);
+        float df;
+        df = kk.x - a.x; d1 = fmaf(df, df, d1); df = kk.y - a.y; d1 = fmaf(df, df, d1);
+        df = kk.z - a.z; d1 = fmaf(df, df, d1); df = kk.w - a.w; d1 = fmaf(df, df, d1);
+        df = kk.x - b.x; d2 = fmaf(df, df, d2); df = kk.y - b.y; d2 = fmaf(df, df, d2);
+        df = kk.z - b.z; d2 = fmaf(df, df, d2); df = kk.w - b.w; d2 = fmaf(df, df, d2);
+    }
+    assign[ent.x] = (d2 < d1 || (d2 == d1 && j2 < j1)) ? j2 : j1;
+}
+
 // ------------------------------------------------------------------ host side
 
 static size_t tc_align(size_t x) { return (x + 255) & ~(size_t)255; }
 
 struct TcLayout {
-    size_t a16, knorm, b16, bias, cmax, bad, list, count, total;
+    size_t a16, knorm, b16, bias, cmax, bad, list, count, pairs, pair_count, total;
     int Mpad;
 };
 static TcLayout tc_layout(const Tables& t, long long n, int M) {
@@ -363,6 +435,8 @@ static TcLayout tc_layout(const Tables& t, long long n, int M) {
     L.bad = off; off += 256;
     L.list = off; off += tc_align(U * (size_t)n * 4);
     L.count = off; off += tc_align(U * 4);
+    L.pairs = off; off += tc_align(U * (size_t)n * 8);
+    L.pair_count = off; off += 256;
     L.total = off;
     return L;
 }
@@ -427,6 +501,9 @@ void launch_assign_tc(const Tables& t, const void* K, long long n, int M, const 
     unsigned* count = reinterpret_cast<unsigned*>(base + L.count);
     cudaMemsetAsync(cmax, 0, (size_t)t.U * 4, s);
     cudaMemsetAsync(count, 0, (size_t)t.U * 4, s);
+    int2* pairs = reinterpret_cast<int2*>(base + L.pairs);
+    unsigned long long* pair_count = reinterpret_cast<unsigned long long*>(base + L.pair_count);
+    cudaMemsetAsync(pair_count, 0, 8, s);
     const long long cw = (long long)t.U * L.Mpad;
     k_tc_prep_centres<<<(unsigned)((cw + 7) / 8), 256, 0, s>>>(C, t.U, M, L.Mpad, B16, bias, cmax, bad);
     CUtensorMap mapA, mapB;
@@ -439,9 +516,13 @@ void launch_assign_tc(const Tables& t, const void* K, long long n, int M, const 
     a.U = t.U; a.n = (int)n; a.M = M; a.Mpad = L.Mpad; a.KB = (int)((n + TC_BM - 1) / TC_BM);
     a.bias = bias; a.knorm = reinterpret_cast<const float*>(base + L.knorm); a.cmax_bits = cmax;
     a.assign = assign; a.recheck_list = list; a.recheck_count = count; a.status = t.status;
+    a.pair_list = pairs; a.pair_count = pair_count;
     const int grid = t.n_attn_ctas / 2;        // one persistent CTA per SM
     k_tc_assign<<<grid, TC_THREADS, TC_SMEM_BYTES, s>>>(mapA, mapB, a);
-    (*launches) += 2;
+    const unsigned long long rows = (unsigned long long)t.U * n;
+    k_tc_pair_decide<<<(unsigned)((rows + 255) / 256), 256, 0, s>>>(reinterpret_cast<const __nv_bfloat16*>(K), C, (int)n, M, pairs,
+                                                                    pair_count, assign, &t.counters[CNT_RECHECKED]);
+    (*launches) += 3;
     launch_assign_f32_listed(t, K, n, M, C, assign, list, count, &t.counters[CNT_RECHECKED], s, launches);
 }
 
