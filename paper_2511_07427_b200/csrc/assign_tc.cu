@@ -20,8 +20,8 @@
 // Warp 0 issues TMA tensor loads (128-byte swizzle, no multicast) of the key block (kept for
 // all centre tiles of the item) and of 256-centre tiles into a two-stage ring; warp 1 issues
 // tcgen05.mma (M=128, N=256, K=16, eight per tile) into one of two 256-column TMEM accumulators
-// and commits to an mbarrier; warps 2-5 drain the other accumulator with tcgen05.ld, one key per
-// thread.  Every wait is bounded; on expiry the kernel sets a status bit, frees its TMEM and
+// and commits to an mbarrier; warps 2-9 drain the accumulators with tcgen05.ld, one key per
+// thread (two groups of four warps, one per accumulator).  Every wait is bounded; on expiry the kernel sets a status bit, frees its TMEM and
 // returns.
 #include <cuda.h>
 #include <float.h>
@@ -108,8 +108,9 @@ constexpr int TC_BM = 128;                // keys per item (one TMEM lane each)
 constexpr int TC_BN = 256;                // centres per accumulator
 constexpr int TC_A_BYTES = TC_BM * TC_D * 2;          // 32 KB: two [128 rows x 128 B] swizzle panels
 constexpr int TC_B_BYTES = TC_BN * TC_D * 2;          // 64 KB: two [256 rows x 128 B] swizzle panels
-constexpr int TC_SMEM_BYTES = 2 * TC_A_BYTES + 2 * TC_B_BYTES + 1024 /* alignment */ + 256 /* barriers */;
-constexpr int TC_THREADS = 192;           // warp 0 loads, warp 1 issues MMAs, warps 2..5 drain accumulators
+constexpr int TC_XCHG_BYTES = 2 * TC_BM * 5 * 4;      // hand-over of (g1, g2, g3, j1, j2) between the drain groups
+constexpr int TC_SMEM_BYTES = 2 * TC_A_BYTES + 2 * TC_B_BYTES + 1024 /* alignment */ + 256 /* barriers */ + TC_XCHG_BYTES;
+constexpr int TC_THREADS = 320;           // warp 0 loads, warp 1 issues MMAs, warps 2..9 drain the accumulators
 constexpr unsigned TC_TMEM_COLS = 512;    // two 256-column fp32 accumulators
 
 // Shared-memory matrix descriptor of a K-major panel with 128-byte rows under the 128-byte swizzle:
@@ -221,6 +222,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) k_tc_assign(const __grid_consta
     auto bar = [&](int i) { return tc_smem_u32(&bars[i]); };
     volatile unsigned* s_tmem = reinterpret_cast<volatile unsigned*>(&bars[12]);
     volatile int* s_abort = reinterpret_cast<volatile int*>(&bars[13]);
+    float* xchg = reinterpret_cast<float*>(gen + 2 * TC_A_BYTES + 2 * TC_B_BYTES + 256);
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int NT = p.Mpad / TC_BN;
@@ -301,13 +303,17 @@ __global__ void __launch_bounds__(TC_THREADS, 1) k_tc_assign(const __grid_consta
             }
         }
     } else {
-        // =============================== accumulator drain (warps 2..5) ===============================
-        // One key per thread.  Per centre tile the thread keeps the three smallest packed values (low 8 bits =
-        // column) in two independent chains, merges them into the item's best two (with indices) and third value.
+        // =============================== accumulator drain (warps 2..9) ===============================
+        // Two groups of four warps; group g drains accumulator g, i.e. the tiles whose running number is g mod 2,
+        // so both accumulators are drained at the same time while the next MMAs run.  One key per thread and
+        // group.  Per tile the thread keeps the three smallest packed values (low 8 bits = column) in two
+        // independent chains and merges them into its best two (with indices) and third value; at the end of an
+        // item group 1 hands its triple to group 0 through shared memory, and group 0 decides.
+        const int grp = (warp - 2) >> 2;              // 0 or 1
         const int q = warp & 3;                       // TMEM lane quarter this warp may read
         const int row = q * 32 + lane;                // key of this thread inside the item
-        long long tb = 0;
-        for (long long it = blockIdx.x; it < n_items; it += gridDim.x) {
+        long long tb = 0, item_no = 0;
+        for (long long it = blockIdx.x; it < n_items; it += gridDim.x, item_no++) {
             const int u = (int)(it / p.KB), kb = (int)(it % p.KB);
             const int i = kb * TC_BM + row;
             float g1 = INFINITY, g2 = INFINITY, g3 = INFINITY;
@@ -315,27 +321,30 @@ __global__ void __launch_bounds__(TC_THREADS, 1) k_tc_assign(const __grid_consta
             bool dead = false;
             for (int nt = 0; nt < NT; nt++, tb++) {
                 const int st = (int)(tb & 1);
+                if (st != grp) continue;
                 if (*s_abort || !tc_mbar_wait(bar(8 + st), (unsigned)((tb >> 1) & 1))) { *s_abort = 1; dead = true; break; }
                 tc_fence_after();
                 float a1 = INFINITY, a2 = INFINITY, a3 = INFINITY, c1 = INFINITY, c2 = INFINITY, c3 = INFINITY;
                 const float4* bias4 = reinterpret_cast<const float4*>(p.bias + (size_t)u * p.Mpad + (size_t)nt * TC_BN);
-#pragma unroll 1
+                const unsigned tbase = tmem + st * TC_BN + ((unsigned)(q * 32) << 16);
+                unsigned acc[2][32];
+                tc_ld32(tbase, acc[0]);
+#pragma unroll
                 for (int c = 0; c < TC_BN / 32; c++) {
-                    unsigned acc[32];
-                    tc_ld32(tmem + st * TC_BN + c * 32 + ((unsigned)(q * 32) << 16), acc);
                     float bs[32];
 #pragma unroll
                     for (int e = 0; e < 8; e++) {
                         const float4 v = __ldg(bias4 + c * 8 + e);
                         bs[4 * e] = v.x; bs[4 * e + 1] = v.y; bs[4 * e + 2] = v.z; bs[4 * e + 3] = v.w;
                     }
-                    tc_ld_wait();
+                    tc_ld_wait();                                           // chunk c has arrived
+                    if (c + 1 < TC_BN / 32) tc_ld32(tbase + (c + 1) * 32, acc[(c + 1) & 1]);   // chunk c + 1 in flight
 #pragma unroll
                     for (int e = 0; e < 32; e += 4) {
-                        const float x0 = tc_pack(fmaf(-2.f, __uint_as_float(acc[e]), bs[e]), c * 32 + e);
-                        const float x1 = tc_pack(fmaf(-2.f, __uint_as_float(acc[e + 1]), bs[e + 1]), c * 32 + e + 1);
-                        const float x2 = tc_pack(fmaf(-2.f, __uint_as_float(acc[e + 2]), bs[e + 2]), c * 32 + e + 2);
-                        const float x3 = tc_pack(fmaf(-2.f, __uint_as_float(acc[e + 3]), bs[e + 3]), c * 32 + e + 3);
+                        const float x0 = tc_pack(fmaf(-2.f, __uint_as_float(acc[c & 1][e]), bs[e]), c * 32 + e);
+                        const float x1 = tc_pack(fmaf(-2.f, __uint_as_float(acc[c & 1][e + 1]), bs[e + 1]), c * 32 + e + 1);
+                        const float x2 = tc_pack(fmaf(-2.f, __uint_as_float(acc[c & 1][e + 2]), bs[e + 2]), c * 32 + e + 2);
+                        const float x3 = tc_pack(fmaf(-2.f, __uint_as_float(acc[c & 1][e + 3]), bs[e + 3]), c * 32 + e + 3);
                         tc_top3_pair(a1, a2, a3, x0, x1);
                         tc_top3_pair(c1, c2, c3, x2, x3);
                     }
@@ -351,8 +360,19 @@ __global__ void __launch_bounds__(TC_THREADS, 1) k_tc_assign(const __grid_consta
                 tc_insert(g1, j1, g2, j2, g3, t2, nt * TC_BN + (int)(__float_as_uint(t2) & 0xFFu));
                 tc_insert(g1, j1, g2, j2, g3, t3, nt * TC_BN + (int)(__float_as_uint(t3) & 0xFFu));
             }
-            if (dead) break;
-            if (i < p.n) {
+            // ---- hand-over: group 1 -> group 0 (slot alternates per item; the barrier orders write, read and reuse)
+            float* slot = xchg + (size_t)(item_no & 1) * TC_BM * 5 + row * 5;
+            if (grp == 1) {
+                slot[0] = g1; slot[1] = g2; slot[2] = g3; slot[3] = __int_as_float(j1); slot[4] = __int_as_float(j2);
+            }
+            asm volatile("bar.sync 2, 256;\n" ::: "memory");
+            if (dead || *s_abort) break;
+            if (grp == 0) {
+                tc_insert(g1, j1, g2, j2, g3, slot[0], __float_as_int(slot[3]));
+                tc_insert(g1, j1, g2, j2, g3, slot[1], __float_as_int(slot[4]));
+                tc_insert(g1, j1, g2, j2, g3, slot[2], 0);
+            }
+            if (grp == 0 && i < p.n) {
                 const size_t gi = (size_t)u * p.n + i;
                 if (j1 >= p.M) j1 = 0;
                 p.assign[gi] = j1;
