@@ -203,6 +203,28 @@ def run_reference(args, cfg):
     print(json.dumps(line), flush=True)
 
 
+def rank_units(cfg, rank: int):
+    """Global unit ids of one rank.  Units are independent, so the job shards with no exchange step: every rank
+    owns one full replica of the configuration's unit grid, seeded by its global unit ids (weak scaling)."""
+    return [rank * cfg.U + u for u in range(cfg.U)]
+
+
+def max_over_ranks(value: float, device=None) -> float:
+    """MAX all-reduce of a scalar over the default process group (NCCL on GPUs, gloo in the CPU tests)."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return float(value)
+    t = torch.tensor([value], dtype=torch.float64, device=device if device is not None else "cpu")
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_steps_per_s(world: int, steps: int, ms_max: float) -> float:
+    """Aggregate over all ranks: every rank advanced its own replica by `steps` in at most `ms_max`."""
+    return world * steps / (ms_max * 1e-3)
+
+
 def run_ours(args, cfg):
     import torch
     import torch.distributed as dist
@@ -229,7 +251,7 @@ def run_ours(args, cfg):
 
     # ---- synthetic inputs, generated on the device (seeded per unit and rank)
     U = cfg.U
-    streams = [UnitStream(cfg, rank * U + u, device=str(dev)) for u in range(U)]
+    streams = [UnitStream(cfg, g, device=str(dev)) for g in rank_units(cfg, rank)]
     Kp, Vp = make_prefill(streams)
     q_all, k_all, v_all = make_decode_chunk(streams, total_steps)
     del streams
@@ -298,11 +320,8 @@ def run_ours(args, cfg):
     pos += K_steps
     st1 = ctx.get_status()
     gpu_launches = ctx.launch_count() - launches0
-    if world > 1:
-        tmax = torch.tensor([ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
-        ms = float(tmax.item())
-    value = world * K_steps / (ms * 1e-3)
+    ms = max_over_ranks(ms, dev)
+    value = whole_job_steps_per_s(world, K_steps, ms)
 
     # ---- per-kernel breakdown with CUDA events around every launch (direct calls, same stream)
     ctx.set_timing(True)
@@ -344,10 +363,7 @@ def run_ours(args, cfg):
             ctx.step_host(qh[t], kh[t], vh[t], cfg.budget, oh)
         torch.cuda.synchronize()
         dt = time.perf_counter() - t0
-        if world > 1:
-            tm = torch.tensor([dt], device=dev, dtype=torch.float64)
-            dist.all_reduce(tm, op=dist.ReduceOp.MAX)
-            dt = float(tm.item())
+        dt = max_over_ranks(dt, dev)
         e2e = {"value": world * (n_e2e - 1) / dt if n_e2e > 1 else None, "unit": "steps/s",
                "h2d_bytes_per_step": int(qh[0].numel() * 4 + 2 * kh[0].numel() * bytes_kv),
                "d2h_bytes_per_step": int(oh.numel() * 4)}

@@ -190,6 +190,13 @@ __device__ __forceinline__ void tc_top3_pair(float& t1, float& t2, float& t3, fl
     t2 = tc_min3(fmaxf(t1, lo), t2, hi);
     t1 = fminf(t1, lo);
 }
+// a <- the three smallest of the sorted triples a and c.
+__device__ __forceinline__ void tc_merge3(float (&a)[3], const float (&c)[3]) {
+    const float t1 = fminf(a[0], c[0]);
+    const float t2 = tc_min3(fmaxf(a[0], c[0]), a[1], c[1]);
+    const float t3 = fminf(tc_min3(a[2], c[2], fmaxf(a[1], c[0])), fmaxf(a[0], c[1]));
+    a[0] = t1; a[1] = t2; a[2] = t3;
+}
 // Insert (v, j) into the sorted best two (with indices) and third value.
 __device__ __forceinline__ void tc_insert(float& g1, int& j1, float& g2, int& j2, float& g3, float v, int j) {
     if (v < g1) { g3 = g2; g2 = g1; j2 = j1; g1 = v; j1 = j; }
@@ -324,7 +331,9 @@ __global__ void __launch_bounds__(TC_THREADS, 1) k_tc_assign(const __grid_consta
                 if (st != grp) continue;
                 if (*s_abort || !tc_mbar_wait(bar(8 + st), (unsigned)((tb >> 1) & 1))) { *s_abort = 1; dead = true; break; }
                 tc_fence_after();
-                float a1 = INFINITY, a2 = INFINITY, a3 = INFINITY, c1 = INFINITY, c2 = INFINITY, c3 = INFINITY;
+                float ch[4][3];                                        // four independent chains of three smallest
+#pragma unroll
+                for (int x = 0; x < 4; x++) { ch[x][0] = INFINITY; ch[x][1] = INFINITY; ch[x][2] = INFINITY; }
                 const float4* bias4 = reinterpret_cast<const float4*>(p.bias + (size_t)u * p.Mpad + (size_t)nt * TC_BN);
                 const unsigned tbase = tmem + st * TC_BN + ((unsigned)(q * 32) << 16);
                 unsigned acc[2][32];
@@ -340,22 +349,24 @@ __global__ void __launch_bounds__(TC_THREADS, 1) k_tc_assign(const __grid_consta
                     tc_ld_wait();                                           // chunk c has arrived
                     if (c + 1 < TC_BN / 32) tc_ld32(tbase + (c + 1) * 32, acc[(c + 1) & 1]);   // chunk c + 1 in flight
 #pragma unroll
-                    for (int e = 0; e < 32; e += 4) {
-                        const float x0 = tc_pack(fmaf(-2.f, __uint_as_float(acc[c & 1][e]), bs[e]), c * 32 + e);
-                        const float x1 = tc_pack(fmaf(-2.f, __uint_as_float(acc[c & 1][e + 1]), bs[e + 1]), c * 32 + e + 1);
-                        const float x2 = tc_pack(fmaf(-2.f, __uint_as_float(acc[c & 1][e + 2]), bs[e + 2]), c * 32 + e + 2);
-                        const float x3 = tc_pack(fmaf(-2.f, __uint_as_float(acc[c & 1][e + 3]), bs[e + 3]), c * 32 + e + 3);
-                        tc_top3_pair(a1, a2, a3, x0, x1);
-                        tc_top3_pair(c1, c2, c3, x2, x3);
+                    for (int e = 0; e < 32; e += 8) {
+#pragma unroll
+                        for (int x = 0; x < 4; x++) {
+                            const int e0 = e + 2 * x;
+                            const float x0 = tc_pack(fmaf(-2.f, __uint_as_float(acc[c & 1][e0]), bs[e0]), c * 32 + e0);
+                            const float x1 = tc_pack(fmaf(-2.f, __uint_as_float(acc[c & 1][e0 + 1]), bs[e0 + 1]), c * 32 + e0 + 1);
+                            tc_top3_pair(ch[x][0], ch[x][1], ch[x][2], x0, x1);
+                        }
                     }
                 }
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) tc_mbar_arrive(bar(10 + st));          // accumulator may be overwritten
-                // the tile's three smallest out of the two chains
-                const float t1 = fminf(a1, c1);
-                const float t2 = tc_min3(fmaxf(a1, c1), a2, c2);
-                const float t3 = fminf(tc_min3(a3, c3, fmaxf(a2, c1)), fmaxf(a1, c2));
+                // the tile's three smallest out of the four chains
+                tc_merge3(ch[0], ch[1]);
+                tc_merge3(ch[2], ch[3]);
+                tc_merge3(ch[0], ch[2]);
+                const float t1 = ch[0][0], t2 = ch[0][1], t3 = ch[0][2];
                 tc_insert(g1, j1, g2, j2, g3, t1, nt * TC_BN + (int)(__float_as_uint(t1) & 0xFFu));
                 tc_insert(g1, j1, g2, j2, g3, t2, nt * TC_BN + (int)(__float_as_uint(t2) & 0xFFu));
                 tc_insert(g1, j1, g2, j2, g3, t3, nt * TC_BN + (int)(__float_as_uint(t3) & 0xFFu));
