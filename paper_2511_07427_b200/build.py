@@ -53,7 +53,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
             list(ex.map(compile_one, jobs))
     if jobs or _stale(LIB, objs):
         subprocess.check_call(["nvcc", "-shared", "-o", LIB, *objs, "-gencode", "arch=compute_100a,code=sm_100a",
-                               "-lcudart", "-lcuda"])
+                               "-lcudart"])
     return LIB
 
 

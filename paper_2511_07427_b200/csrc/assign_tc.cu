@@ -508,14 +508,34 @@ bool tc_assign_begin(const Tables& t, const void* K, long long n, int M, void* s
     return true;
 }
 
+// cuTensorMapEncodeTiled is looked up through the runtime, so the library carries no link-time dependency on
+// the driver library and still loads on a machine without a GPU.
+typedef CUresult (*tc_encode_fn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                 const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                 CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+static tc_encode_fn tc_encode_entry() {
+    static tc_encode_fn fn = nullptr;
+    if (!fn) {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult qr;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qr) == cudaSuccess &&
+            qr == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<tc_encode_fn>(p);
+        else
+            cudaGetLastError();
+    }
+    return fn;
+}
+
 static bool tc_make_map(CUtensorMap* map, void* ptr, unsigned long long rows, unsigned box_rows) {
+    tc_encode_fn enc = tc_encode_entry();
+    if (!enc) return false;
     cuuint64_t dims[2] = {(cuuint64_t)TC_D, (cuuint64_t)rows};
     cuuint64_t strides[1] = {(cuuint64_t)TC_D * 2};
     cuuint32_t box[2] = {64u, box_rows};
     cuuint32_t estr[2] = {1u, 1u};
-    return cuTensorMapEncodeTiled(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, ptr, dims, strides, box, estr,
-                                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
-                                  CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+    return enc(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, ptr, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+               CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
 // One Lloyd round's assignment: centre pre-pass, distance GEMM + filter, exact re-decision of the listed keys.
