@@ -61,18 +61,32 @@ __global__ void __launch_bounds__(FR_THREADS) k_front(Tables t, StepPtr qp, Step
     float* SC = t.scores + (size_t)u * t.max_clusters;
     float* DS = t.dists + (size_t)u * t.max_clusters;
     const int jend = min(Mcur, j0 + FR_ROWS);
-    for (int j = j0 + warp * 4 + sub; j < j0 + FR_ROWS; j += (FR_THREADS / 32) * 4) {
-        const bool in = j < jend;
-        const bool live = in && CN[j] > 0;
-        float s = 0.f, dd = 0.f;
-        if (live) {
+    // all row loads of the thread are issued before any arithmetic (rows of dead clusters are read too and
+    // masked afterwards, so no load waits for the cluster-size load)
+    constexpr int NIT = FR_ROWS / ((FR_THREADS / 32) * 4);
+    float4 rv[NIT][V4];
+    int cn[NIT];
 #pragma unroll
-            for (int i = 0; i < V4; i++) {
-                const float4 rv = *reinterpret_cast<const float4*>(R + (size_t)j * HD + l8 * 4 + 32 * i);
-                s = fmaf(qs[i][0], rv.x, s); s = fmaf(qs[i][1], rv.y, s); s = fmaf(qs[i][2], rv.z, s); s = fmaf(qs[i][3], rv.w, s);
-                float a = kk[i][0] - rv.x, b = kk[i][1] - rv.y, c = kk[i][2] - rv.z, e = kk[i][3] - rv.w;
-                dd = fmaf(a, a, dd); dd = fmaf(b, b, dd); dd = fmaf(c, c, dd); dd = fmaf(e, e, dd);
-            }
+    for (int it = 0; it < NIT; it++) {
+        const int j = j0 + warp * 4 + sub + it * (FR_THREADS / 32) * 4;
+        const bool in = j < jend;
+        cn[it] = in ? CN[j] : 0;
+#pragma unroll
+        for (int i = 0; i < V4; i++)
+            rv[it][i] = in ? __ldcs(reinterpret_cast<const float4*>(R + (size_t)j * HD + l8 * 4 + 32 * i)) : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+#pragma unroll
+    for (int it = 0; it < NIT; it++) {
+        const int j = j0 + warp * 4 + sub + it * (FR_THREADS / 32) * 4;
+        const bool in = j < jend;
+        const bool live = in && cn[it] > 0;
+        float s = 0.f, dd = 0.f;
+#pragma unroll
+        for (int i = 0; i < V4; i++) {
+            const float4 r4 = rv[it][i];
+            s = fmaf(qs[i][0], r4.x, s); s = fmaf(qs[i][1], r4.y, s); s = fmaf(qs[i][2], r4.z, s); s = fmaf(qs[i][3], r4.w, s);
+            float a = kk[i][0] - r4.x, b = kk[i][1] - r4.y, c = kk[i][2] - r4.z, e = kk[i][3] - r4.w;
+            dd = fmaf(a, a, dd); dd = fmaf(b, b, dd); dd = fmaf(c, c, dd); dd = fmaf(e, e, dd);
         }
 #pragma unroll
         for (int o = 4; o > 0; o >>= 1) { s += __shfl_xor_sync(0xffffffffu, s, o); dd += __shfl_xor_sync(0xffffffffu, dd, o); }

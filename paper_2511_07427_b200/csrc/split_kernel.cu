@@ -10,7 +10,8 @@
 
 namespace dkv {
 
-constexpr int SP_THREADS = 256;
+constexpr int SP_THREADS = 512;
+constexpr int SP_CACHE_BYTES = 32 * 1024;      // member keys of the cluster being split are staged here when they fit
 constexpr int SP_WARPS = SP_THREADS / 32;
 
 template <typename KV, int HD>
@@ -35,15 +36,24 @@ __global__ void __launch_bounds__(SP_THREADS) k_split_check(Tables t, float gamm
     KV* vpg = reinterpret_cast<KV*>(t.vpages) + (size_t)u * t.P * PAGE * HD;
     int* ptok = t.page_tok + (size_t)u * t.P * PAGE;
     int* pnext = t.page_next + (size_t)u * t.P;
-    unsigned char* label = t.sp_label + (size_t)u * t.max_tokens;
-    int* rank_of = t.sp_pos + (size_t)u * 2 * t.max_tokens;     // per position
-    int* holes = rank_of + t.max_tokens;                        // hole positions, in order
+    unsigned char* label_g = t.sp_label + (size_t)u * t.max_tokens;
+    int* rank_g = t.sp_pos + (size_t)u * 2 * t.max_tokens;      // per position
+    int* holes_g = rank_g + t.max_tokens;                       // hole positions, in order
+    // the same three arrays in shared memory for a cluster small enough to be staged
+    __shared__ unsigned char label_s[SP_CACHE_BYTES / 128];
+    __shared__ int rank_s[SP_CACHE_BYTES / 128], holes_s[SP_CACHE_BYTES / 128];
 
     // ---- triggered clusters, ascending id, evaluated on the state at entry.  A full scan is
     // needed only after a split changed M_live or created clusters (u_scan); otherwise only the
     // cluster that received the last append can have become triggered: for every other cluster
     // n_j and M2_j are unchanged while N only grew.
     int* trig = dyn + 2 * maxch;
+    // staged copy of the member keys (and their token ids) when the cluster fits: every pass below then
+    // reads shared memory instead of walking the pages again
+    constexpr int CACHE_ROWS = SP_CACHE_BYTES / (HD * (int)sizeof(KV));
+    KV* krows = reinterpret_cast<KV*>(reinterpret_cast<unsigned char*>(dyn) +
+                                      (((size_t)(2 * maxch + t.max_clusters) * sizeof(int) + 15) & ~(size_t)15));
+    int* tok_s = reinterpret_cast<int*>(krows + (size_t)CACHE_ROWS * HD);
     __shared__ int s_ntrig, s_nsplit;
     if (tid == 0) { s_ntrig = 0; s_nsplit = 0; }
     __syncthreads();
@@ -87,6 +97,25 @@ __global__ void __launch_bounds__(SP_THREADS) k_split_check(Tables t, float gamm
         }
         for (int e = tid; e < HD; e += SP_THREADS) cA[e] = t.cl_r[cj * HD + e];
         __syncthreads();
+        const bool cached = c <= CACHE_ROWS;
+        if (cached) {
+            constexpr int V16 = HD * (int)sizeof(KV) / 16;      // 16-byte pieces per row
+            for (int idx = tid; idx < c * V16; idx += SP_THREADS) {
+                const int p = idx / V16, v = idx % V16;
+                const size_t row = (size_t)chain[p >> 5] * PAGE + (p & 31);
+                reinterpret_cast<uint4*>(krows + (size_t)p * HD)[v] = reinterpret_cast<const uint4*>(kpg + row * HD)[v];
+            }
+            for (int p = tid; p < c; p += SP_THREADS) tok_s[p] = ptok[(size_t)chain[p >> 5] * PAGE + (p & 31)];
+            __syncthreads();
+        }
+        unsigned char* label = cached ? label_s : label_g;
+        int* rank_of = cached ? rank_s : rank_g;
+        int* holes = cached ? holes_s : holes_g;
+        // key row and token id of member position p
+        auto key_of = [&](int p) -> const KV* {
+            return cached ? krows + (size_t)p * HD : kpg + ((size_t)chain[p >> 5] * PAGE + (p & 31)) * HD;
+        };
+        auto tok_of = [&](int p) -> int { return cached ? tok_s[p] : ptok[(size_t)chain[p >> 5] * PAGE + (p & 31)]; };
 
         // ---- centre A: member farthest from r_j; centre B: member farthest from A (ties: lowest token id)
         for (int round = 0; round < 2; round++) {
@@ -95,13 +124,12 @@ __global__ void __launch_bounds__(SP_THREADS) k_split_check(Tables t, float gamm
             for (int e = 0; e < EPL; e++) cen[e] = cA[lane * EPL + e];
             float bd = -1.f; int bt = 0x7fffffff, bp = -1;
             for (int p = warp; p < c; p += SP_WARPS) {
-                const size_t row = (size_t)chain[p >> 5] * PAGE + (p & 31);
-                const KV* k = kpg + row * HD + lane * EPL;
+                const KV* k = key_of(p) + lane * EPL;
                 float part = 0.f;
 #pragma unroll
                 for (int e = 0; e < EPL; e++) { float df = to_f(k[e]) - cen[e]; part = fmaf(df, df, part); }
                 part = warp_sum(part);
-                int tok = ptok[row];
+                int tok = tok_of(p);
                 if (part > bd || (part == bd && tok < bt)) { bd = part; bt = tok; bp = p; }
             }
             if (lane == 0) { red_f[warp] = bd; red_i[warp] = bt; red_k[warp] = bp; }
@@ -114,10 +142,10 @@ __global__ void __launch_bounds__(SP_THREADS) k_split_check(Tables t, float gamm
             }
             __syncthreads();
             {
-                const size_t row = (size_t)chain[s_a >> 5] * PAGE + (s_a & 31);
+                const KV* src = key_of(s_a);
                 float* dst = (round == 0) ? cA : cB;
                 __syncthreads();
-                for (int e = tid; e < HD; e += SP_THREADS) dst[e] = to_f(kpg[row * HD + e]);
+                for (int e = tid; e < HD; e += SP_THREADS) dst[e] = to_f(src[e]);
                 __syncthreads();
             }
         }
@@ -136,8 +164,7 @@ __global__ void __launch_bounds__(SP_THREADS) k_split_check(Tables t, float gamm
             for (int e = 0; e < EPL; e++) { a_c[e] = cA[lane * EPL + e]; b_c[e] = cB[lane * EPL + e]; sa[e] = 0.f; sb[e] = 0.f; }
             int chg = 0, ca = 0, cb = 0;
             for (int p = warp; p < c; p += SP_WARPS) {
-                const size_t row = (size_t)chain[p >> 5] * PAGE + (p & 31);
-                const KV* k = kpg + row * HD + lane * EPL;
+                const KV* k = key_of(p) + lane * EPL;
                 float kk[EPL], da = 0.f, db = 0.f;
 #pragma unroll
                 for (int e = 0; e < EPL; e++) {
@@ -173,7 +200,7 @@ __global__ void __launch_bounds__(SP_THREADS) k_split_check(Tables t, float gamm
         {
             int bt = 0x7fffffff, bl = 0;
             for (int p = tid; p < c; p += SP_THREADS) {
-                int tok = ptok[(size_t)chain[p >> 5] * PAGE + (p & 31)];
+                int tok = tok_of(p);
                 if (tok < bt) { bt = tok; bl = label[p]; }
             }
 #pragma unroll
@@ -286,8 +313,11 @@ __global__ void __launch_bounds__(SP_THREADS) k_split_check(Tables t, float gamm
             float sa[EPL];
 #pragma unroll
             for (int e = 0; e < EPL; e++) sa[e] = 0.f;
-            for (int p = warp; p < cc; p += SP_WARPS) {
-                const KV* k = kpg + ((size_t)pages[p >> 5] * PAGE + (p & 31)) * HD + lane * EPL;
+            // staged members of this child (by label) when the cluster was staged, else its rows in their new place
+            const int n_scan = cached ? c : cc;
+            for (int p = warp; p < n_scan; p += SP_WARPS) {
+                if (cached && ((label[p] == stay) != (child == 0))) continue;
+                const KV* k = (cached ? krows + (size_t)p * HD : kpg + ((size_t)pages[p >> 5] * PAGE + (p & 31)) * HD) + lane * EPL;
 #pragma unroll
                 for (int e = 0; e < EPL; e++) sa[e] += to_f(k[e]);
             }
@@ -305,8 +335,9 @@ __global__ void __launch_bounds__(SP_THREADS) k_split_check(Tables t, float gamm
             float mean[EPL], m2 = 0.f;
 #pragma unroll
             for (int e = 0; e < EPL; e++) mean[e] = cA[lane * EPL + e];
-            for (int p = warp; p < cc; p += SP_WARPS) {
-                const KV* k = kpg + ((size_t)pages[p >> 5] * PAGE + (p & 31)) * HD + lane * EPL;
+            for (int p = warp; p < n_scan; p += SP_WARPS) {
+                if (cached && ((label[p] == stay) != (child == 0))) continue;
+                const KV* k = (cached ? krows + (size_t)p * HD : kpg + ((size_t)pages[p >> 5] * PAGE + (p & 31)) * HD) + lane * EPL;
                 float part = 0.f;
 #pragma unroll
                 for (int e = 0; e < EPL; e++) { float df = to_f(k[e]) - mean[e]; part = fmaf(df, df, part); }
@@ -329,6 +360,7 @@ __global__ void __launch_bounds__(SP_THREADS) k_split_check(Tables t, float gamm
 template <typename KV, int HD>
 static void split_t(const Tables& t, float gamma, int var_enabled, int min_size, int iters, cudaStream_t s) {
     size_t dyn = sizeof(int) * (2 * (size_t)(t.max_tokens / PAGE + 2) + (size_t)t.max_clusters);
+    dyn = ((dyn + 15) & ~(size_t)15) + SP_CACHE_BYTES + sizeof(int) * (SP_CACHE_BYTES / (HD * sizeof(KV))) + 16;
     if (dyn > 32 * 1024)
         cudaFuncSetAttribute(k_split_check<KV, HD>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn);
     k_split_check<KV, HD><<<t.U, SP_THREADS, dyn, s>>>(t, gamma, var_enabled, min_size, iters);
