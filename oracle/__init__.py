@@ -58,6 +58,8 @@ def lib() -> C.CDLL:
         L.ork_destroy.argtypes = [C.c_void_p]
         L.ork_build.restype = C.c_int
         L.ork_build.argtypes = [C.c_void_p, dp, dp, C.c_int, C.c_int, C.c_int, C.c_uint64, C.c_int, C.c_int, ip, ip]
+        L.ork_install.restype = C.c_int
+        L.ork_install.argtypes = [C.c_void_p, dp, dp, C.c_int, ip, C.c_int]
         L.ork_score.restype = None
         L.ork_score.argtypes = [C.c_void_p, dp, dp]
         L.ork_select.restype = C.c_int
@@ -170,6 +172,13 @@ class OracleUnit:
                              init_mode, _ip(hp), _ip(ha))
         if rc != 0:
             raise ValueError("oracle build: bad sizes")
+
+    def install(self, K, V, assign, n_ids: int) -> None:
+        """Continue from a given partition: token -> cluster id map with `n_ids` ids in use; statistics are
+        recomputed from the members (Eq. 4)."""
+        K = _d(K); V = _d(V); a = _i(assign)
+        if lib().ork_install(self._h, _dp(K), _dp(V), K.shape[0], _ip(a), n_ids) != 0:
+            raise ValueError("oracle install: bad sizes or ids")
 
     def scores(self, q) -> np.ndarray:
         q = _d(q); s = np.zeros(self.M, np.float64)

@@ -560,6 +560,30 @@ int ork_split_check(ork_unit *u, const int *hint_assign_after) {
     return done;
 }
 
+/* Install a given partition instead of building one: keys and values in token-id order, the cluster id of
+ * every token, and the number of ids in use.  Representatives are recomputed as member means (Eq. 4), M2 as the
+ * sum of squared distances to them, both from the members in token-id order (UpdateStats of Algorithm 1); ids
+ * without members are dead; tau = alpha * mean live variance, as after a build.  Lets a test continue from
+ * another implementation's partition at sizes where running the oracle's own k-means would take minutes. */
+int ork_install(ork_unit *u, const double *K, const double *V, int n, const int *assign, int M) {
+    int d = u->d;
+    if (n > u->max_tokens || M > u->max_clusters || M < 1 || n < 1) return -1;
+    for (int i = 0; i < n; i++) if (assign[i] < 0 || assign[i] >= M) return -1;
+    memcpy(u->K, K, sizeof(double) * (size_t)n * d);
+    memcpy(u->V, V, sizeof(double) * (size_t)n * d);
+    memcpy(u->assign, assign, sizeof(int) * (size_t)n);
+    u->n = n; u->M = M;
+    double vs = 0.0; int nl = 0;
+    for (int j = 0; j < M; j++) {
+        u->hold[j] = 0;
+        recompute_stats(u, j);
+        u->live[j] = u->cnt[j] > 0;
+        if (u->live[j]) { vs += u->M2[j] / u->cnt[j]; nl++; }
+    }
+    u->tau = nl ? u->alpha * (vs / nl) : 0.0;
+    return 0;
+}
+
 /* ---------------------------------------------------------------- getters */
 
 int ork_n(const ork_unit *u) { return u->n; }

@@ -1,0 +1,110 @@
+"""Config 4 at its full size (256 units x 32768 keys, 1024 clusters, budget 2048), in the launch configuration
+that bench.py times (tensor-core build, one launch per kernel for all units, CUDA-graph decode loop), checked on
+sampled units.  The oracle's own k-means would take minutes per unit at this size, so it continues from the
+library's partition (installed, with representatives and M2 recomputed from the members, which checks Eq. 4 and
+the statistics on the way) and then follows every decode call exactly as in the small parity runs."""
+import numpy as np
+import pytest
+import torch
+
+import oracle as O
+import paper_2511_07427_b200 as P
+from gen import CONFIGS, UnitStream, make_decode_chunk, make_prefill
+from parity_harness import (TOL_OUT_ABS, TOL_OUT_L2, ParityReport, check_state, make_ctx, make_oracle, rel_l2)
+
+pytestmark = pytest.mark.gpu
+
+SAMPLED = [0, 101, 255]
+DIRECT_STEPS, GRAPH_STEPS = 3, 3
+
+
+def test_config4_full_size_sampled_units():
+    cfg = CONFIGS[4]
+    U, n = cfg.U, cfg.n_prefill
+    side = torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        streams = [UnitStream(cfg, u, device="cuda") for u in range(U)]
+        K, V = make_prefill(streams)
+        q, k, v = make_decode_chunk(streams, DIRECT_STEPS + GRAPH_STEPS)
+        ctx = make_ctx(cfg, U, trace=0, assign_mode=0)
+        ctx.build_index(K, V, cfg.M0, 1234)
+        st = ctx.export_state()
+        rep = ParityReport()
+        oracles = {}
+        for u in SAMPLED:
+            a = st["tok_cluster"][u, :n]
+            # Eq. 3: every key in exactly one cluster, sizes add up
+            assert a.min() >= 0 and a.max() < cfg.M0 and np.array_equal(np.bincount(a, minlength=cfg.M0), st["counts"][u, :cfg.M0])
+            o = make_oracle(cfg)
+            o.install(K[u].double().cpu().numpy(), V[u].double().cpu().numpy(), a, int(st["n_ids"][u]))
+            check_state(o, st, u, rep, f"full-size build unit {u}")          # Eq. 4 centroids, M2, sizes
+            assert abs(float(st["tau"][u]) - o.tau) <= 1e-4 * o.tau
+            oracles[u] = o
+        sel = torch.full((U, cfg.max_clusters), -1, dtype=torch.int32, device="cuda")
+        for t in range(DIRECT_STEPS):
+            out = ctx.decode_step(q[t], cfg.budget, selected_ids=sel).cpu().numpy().astype(np.float64)
+            sel_np = sel.cpu().numpy()
+            nsel, ntok = ctx.get_selection()
+            for u in SAMPLED:
+                o = oracles[u]
+                ids = sel_np[u][: nsel[u]]
+                out_o, ids_o, tok_o = o.decode_step(q[t, u].double().cpu().numpy(), cfg.budget, hint_ids=ids)
+                assert list(ids_o) == list(ids) and tok_o == int(ntok[u]) and o.violations == 0
+                ea, el = float(np.abs(out[u] - out_o).max()), rel_l2(out[u], out_o)
+                assert ea <= TOL_OUT_ABS and el <= TOL_OUT_L2, f"step {t} unit {u}: abs {ea:.3e} relL2 {el:.3e}"
+            ctx.append(k[t], v[t])
+            ctx.split_check()
+            st = ctx.export_state()
+            for u in SAMPLED:
+                o = oracles[u]
+                n0 = o.n
+                # the append target is read from the map before the split may have moved the token
+                o.append(k[t, u].double().cpu().numpy(), v[t, u].double().cpu().numpy(), hint_cluster=-1)
+                o.split_check(hint_assign_after=st["tok_cluster"][u, : o.n])
+                assert o.violations == 0 and o.n == n0 + 1
+                check_state(o, st, u, rep, f"full-size step {t} unit {u}")
+        # ---- the graph-replayed loop, as timed by the benchmark
+        a, b = DIRECT_STEPS, DIRECT_STEPS + GRAPH_STEPS
+        outs = ctx.decode_loop(q[a:b], k[a:b], v[a:b], cfg.budget)
+        side.synchronize()
+        outs = outs.cpu().numpy().astype(np.float64)
+        st = ctx.export_state()
+        status = ctx.get_status()
+        for t in range(GRAPH_STEPS):
+            for u in SAMPLED:
+                o = oracles[u]
+                out_o, _, _ = o.decode_step(q[a + t, u].double().cpu().numpy(), cfg.budget)
+                ea, el = float(np.abs(outs[t, u] - out_o).max()), rel_l2(outs[t, u], out_o)
+                assert ea <= TOL_OUT_ABS and el <= TOL_OUT_L2, f"graph step {t} unit {u}: abs {ea:.3e} relL2 {el:.3e}"
+                o.append(k[a + t, u].double().cpu().numpy(), v[a + t, u].double().cpu().numpy())
+                o.split_check()
+        for u in SAMPLED:
+            check_state(oracles[u], st, u, rep, f"after the graph loop, unit {u}")
+        assert status["error_bits"] & (P.ST_INTERNAL | P.ST_PAGE_POOL | P.ST_MAX_TOKENS) == 0
+        assert status["assign_rechecked"] < 0.1 * U * n * cfg.T          # the filter decides most keys
+        ctx.destroy()
+
+
+def test_config4_full_size_first_assignment_sampled_keys():
+    """The tensor-core assignment at full size: with one Lloyd round the stored membership is the nearest-centre
+    assignment to the initial centres, which the oracle reproduces from the seed; 1500 sampled keys of each
+    sampled unit are re-decided by brute force in fp64."""
+    cfg = CONFIGS[4].scaled(T=1)
+    U, n, M = cfg.U, cfg.n_prefill, cfg.M0
+    streams = [UnitStream(cfg, u, device="cuda") for u in range(U)]
+    K, V = make_prefill(streams)
+    ctx = make_ctx(cfg, U, trace=0, assign_mode=0)
+    ctx.build_index(K, V, M, 4321)
+    st = ctx.export_state()
+    status = ctx.get_status()
+    rng = np.random.default_rng(9)
+    for u in SAMPLED:
+        Ku = K[u].double().cpu().numpy()
+        picks = O.init_random(n, M, 4321, unit=u)
+        C0 = Ku[picks]
+        sample = np.sort(rng.choice(n, size=1500, replace=False))
+        a_gpu = st["tok_cluster"][u, :n][sample]
+        a_or, ties, viol = O.assign(Ku[sample], C0, hint=a_gpu)
+        assert viol == 0 and np.array_equal(a_or, a_gpu), f"unit {u}: {viol} sampled keys assigned to a farther centre"
+    assert status["error_bits"] & P.ST_INTERNAL == 0 and 0 < status["assign_rechecked"] < 0.2 * U * n
+    ctx.destroy()

@@ -468,3 +468,25 @@ def test_size_trigger_uses_live_cluster_count():
     u, K = _unit_with_dead_cluster(gamma=1.2, alpha=0, split_min_size=2)
     assert sorted(u.counts()) == [0, 5, 5]
     assert u.split_check() == 0
+
+
+# ------------------------------------------------------------------ installing a partition
+
+def test_install_reproduces_the_state_of_a_build():
+    """A partition installed from outside must give exactly the statistics the oracle's own build ends with
+    (same member means, M2, sizes, tau), and decode from there must agree."""
+    rng = np.random.default_rng(5)
+    K = rng.normal(size=(300, 16)); V = rng.normal(size=(300, 16))
+    a = O.OracleUnit(16, 2, 400, 32)
+    a.build(K, V, 9, 4, 77, init_mode=O.INIT_RANDOM)
+    b = O.OracleUnit(16, 2, 400, 32)
+    b.install(K, V, a.assign(), a.M)
+    assert np.array_equal(a.counts(), b.counts()) and np.array_equal(a.live(), b.live())
+    assert np.allclose(a.centroids(), b.centroids(), rtol=0, atol=1e-13)
+    assert np.allclose(a.M2(), b.M2(), rtol=1e-12) and abs(a.tau - b.tau) <= 1e-12 * a.tau
+    q = rng.normal(size=(2, 16))
+    oa, ia, _ = a.decode_step(q, 120); ob, ib, _ = b.decode_step(q, 120)
+    assert list(ia) == list(ib) and np.allclose(oa, ob, atol=1e-13)
+    # centroid of an installed cluster is the plain mean of its members
+    j = int(np.argmax(b.counts()))
+    assert np.allclose(b.centroids()[j], K[a.assign() == j].mean(0), atol=1e-13)
