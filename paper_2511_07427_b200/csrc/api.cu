@@ -176,7 +176,7 @@ extern "C" int dynakv_create(const dynakv_config* cfg, void* cuda_stream, dynakv
     }
     ALLOC(t.work_prefix, U + 1, true);
     ALLOC(t.unit_arrive, U, true);
-    ALLOC(t.plan_counter, 1, true);
+    ALLOC(t.plan_counter, 2, true);
     if (cfg->kv_dtype == DYNAKV_BF16 && attn_tma_prepare(t) != 0) {
         snprintf(g_err, sizeof(g_err), "cannot reserve shared memory for the gather-attention kernel: %s", cudaGetErrorString(cudaGetLastError()));
         dynakv_destroy(c);
@@ -284,11 +284,15 @@ static void enqueue_append_apply(dynakv_ctx* c, StepPtr k, StepPtr v, bool timed
     launch_append_apply(c->t, k, v, c->stream, &c->launches);
 }
 
-// one whole loop iteration: a single centroid pass serves both the query scores and the new key's distances
-static void enqueue_step(dynakv_ctx* c, StepPtr q, StepPtr k, StepPtr v, int budget, StepPtrW out, bool timed) {
+// One whole loop iteration in four launches: a single centroid pass serves both the query scores and the new
+// key's distances; selection; gather-attention with its combine; then append + split check in one kernel
+// (which also advances the device-side step index when the iteration belongs to a captured loop).
+static void enqueue_step(dynakv_ctx* c, StepPtr q, StepPtr k, StepPtr v, int budget, StepPtrW out, int* step_ctr, bool timed) {
     enqueue_front(c, q, k, 1, 1, timed);
     enqueue_retrieve(c, q, budget, out, nullptr, timed);
-    enqueue_append_apply(c, k, v, timed);
+    TimeScope ts(c, KC_SPLIT, timed);
+    launch_append_split(c->t, c->cfg.split_size_factor, c->cfg.split_var_factor > 0.f ? 1 : 0, c->cfg.split_min_size,
+                        c->cfg.split_iters, 1, k, v, step_ctr, c->stream, &c->launches);
 }
 
 extern "C" int dynakv_decode_step(dynakv_ctx* c, const float* q, int32_t token_budget, float* out, int32_t* selected_ids) {
@@ -340,9 +344,7 @@ extern "C" int dynakv_decode_loop(dynakv_ctx* c, const float* q_steps, const voi
         long long before = c->launches;
         CK(cudaStreamBeginCapture(c->stream, cudaStreamCaptureModeThreadLocal));
         enqueue_step(c, StepPtr{q_steps, qs, c->step_ctr}, StepPtr{k_steps, ks, c->step_ctr},
-                     StepPtr{v_steps, ks, c->step_ctr}, token_budget, StepPtrW{out_steps, qs, c->step_ctr}, false);
-        enqueue_split(c, false);
-        launch_step_inc(c->step_ctr, c->stream, &c->launches);
+                     StepPtr{v_steps, ks, c->step_ctr}, token_budget, StepPtrW{out_steps, qs, c->step_ctr}, c->step_ctr, false);
         cudaError_t e = cudaStreamEndCapture(c->stream, &graph);
         c->graph_nodes = c->launches - before;
         c->launches = before;
@@ -375,8 +377,7 @@ extern "C" int dynakv_step_host(dynakv_ctx* c, const float* q_host, const void* 
     CK(cudaMemcpyAsync(c->st_k, k_host, kb, cudaMemcpyHostToDevice, c->stream));
     CK(cudaMemcpyAsync(c->st_v, v_host, kb, cudaMemcpyHostToDevice, c->stream));
     enqueue_step(c, StepPtr{c->st_q, 0, nullptr}, StepPtr{c->st_k, 0, nullptr}, StepPtr{c->st_v, 0, nullptr},
-                 token_budget, StepPtrW{c->st_out, 0, nullptr}, true);
-    enqueue_split(c);
+                 token_budget, StepPtrW{c->st_out, 0, nullptr}, nullptr, true);
     CK(cudaMemcpyAsync(out_host, c->st_out, qb, cudaMemcpyDeviceToHost, c->stream));
     CK(cudaStreamSynchronize(c->stream));
     return DYNAKV_OK;

@@ -1,0 +1,93 @@
+// The append of one decode step for one unit, as a block-level device function shared by the stand-alone
+// append kernel and by the split-check kernel of the fused loop iteration (arXiv 2511.07427, Algorithm 1:
+// "Assign new KV entry to its nearest cluster", UpdateVar, AddEntry, UpdateStats).
+#pragma once
+
+#include "common.cuh"
+
+namespace dkv {
+
+// One block per unit: argmin over the distances written by k_front (ties to the lowest id),
+// then n <- n+1, delta = k - r, r <- r + delta/n, M2 <- M2 + delta.(k - r_new), and the
+// (k, v) row goes to the next slot of the cluster's tail page (a fresh page is linked when
+// the tail is full).  No stored entry moves.
+// Called by every thread of a block (any block size that is a multiple of 32, up to 1024); contains one
+// __syncthreads().  Global writes are made by warp 0; callers that go on reading them synchronise first.
+template <typename KV, int HD>
+__device__ __forceinline__ void append_block(const Tables& t, int u, StepPtr kp_, StepPtr vp_) {
+    constexpr int EPL = HD / 32;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarp = blockDim.x >> 5;
+    __shared__ float red_d[32];
+    __shared__ int red_j[32];
+    const int Mcur = t.u_M[u];
+    const int N = t.u_N[u];
+    if (N >= t.max_tokens) { if (tid == 0) atomicOr(t.status, DYNAKV_ST_MAX_TOKENS); return; }
+    const float* DS = t.dists + (size_t)u * t.max_clusters;
+    float bd = INFINITY; int bj = 0x7fffffff;
+    for (int j = tid; j < Mcur; j += blockDim.x) {
+        const float dd = DS[j];
+        if (dd < bd) { bd = dd; bj = j; }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        const float od = __shfl_xor_sync(0xffffffffu, bd, o); const int oj = __shfl_xor_sync(0xffffffffu, bj, o);
+        if (od < bd || (od == bd && oj < bj)) { bd = od; bj = oj; }
+    }
+    if (lane == 0) { red_d[warp] = bd; red_j[warp] = bj; }
+    __syncthreads();
+    if (warp != 0) return;
+    bd = red_d[0]; bj = red_j[0];
+#pragma unroll
+    for (int w = 1; w < nwarp; w++) if (red_d[w] < bd || (red_d[w] == bd && red_j[w] < bj)) { bd = red_d[w]; bj = red_j[w]; }
+    if (bj == 0x7fffffff) return;    // no live cluster
+    const KV* knew = reinterpret_cast<const KV*>(kp_.get()) + (size_t)u * HD;
+    const KV* vnew = reinterpret_cast<const KV*>(vp_.get()) + (size_t)u * HD;
+    const size_t cj = (size_t)u * t.max_clusters + bj;
+    const int n_old = t.cl_n[cj];
+    int page = t.cl_tail[cj];
+    const int row = n_old % PAGE;
+    if (row == 0) {   // tail is full: link a fresh page
+        int np = -1;
+        if (lane == 0) {
+            int fc = t.u_free_cnt[u];
+            if (fc > 0) { np = t.free_stack[(size_t)u * t.P + fc - 1]; t.u_free_cnt[u] = fc - 1; }
+            else { int top = t.u_page_top[u]; if (top < t.P) { np = top; t.u_page_top[u] = top + 1; } }
+            if (np >= 0) { t.page_next[(size_t)u * t.P + page] = np; t.page_next[(size_t)u * t.P + np] = -1; t.cl_tail[cj] = np; }
+            else atomicOr(t.status, DYNAKV_ST_PAGE_POOL);
+        }
+        np = __shfl_sync(0xffffffffu, np, 0);
+        if (np < 0) return;
+        page = np;
+    }
+    const float n_new = (float)(n_old + 1);
+    float* r = t.cl_r + cj * HD;
+    float add = 0.f;
+    float kk[EPL];
+#pragma unroll
+    for (int e = 0; e < EPL; e++) {
+        kk[e] = to_f(knew[lane * EPL + e]);
+        const float ro = r[lane * EPL + e];
+        const float delta = kk[e] - ro;
+        const float rn = ro + delta / n_new;
+        r[lane * EPL + e] = rn;
+        add = fmaf(delta, kk[e] - rn, add);
+    }
+    add = warp_sum(add);
+    KV* kpg = reinterpret_cast<KV*>(t.kpages) + (((size_t)u * t.P + page) * PAGE + row) * HD;
+    KV* vpg = reinterpret_cast<KV*>(t.vpages) + (((size_t)u * t.P + page) * PAGE + row) * HD;
+#pragma unroll
+    for (int e = 0; e < EPL; e++) { kpg[lane * EPL + e] = knew[lane * EPL + e]; vpg[lane * EPL + e] = vnew[lane * EPL + e]; }
+    if (lane == 0) {
+        t.cl_M2[cj] += add;
+        t.cl_n[cj] = n_old + 1;
+        t.cl_flags[cj] &= ~FLAG_HOLD;
+        t.page_tok[((size_t)u * t.P + page) * PAGE + row] = N;
+        t.tok_cluster[(size_t)u * t.max_tokens + N] = bj;
+        t.u_N[u] = N + 1;
+        t.u_last[u] = bj;
+        atomicAdd(&t.counters[CNT_APPENDED], 1ull);
+    }
+}
+
+
+}  // namespace dkv

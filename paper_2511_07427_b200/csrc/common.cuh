@@ -48,7 +48,7 @@ struct Tables {
     float* part;                     // partial (acc, m, l) records of [G][d + 2] floats: [U][S] (plain kernel) or [2 * n_attn_ctas]
     int* work_prefix;                // [U + 1] exclusive prefix of n_work over the units (written by the last select block)
     int* unit_arrive;                // [U] arrival counters of the split-K combine (zero between steps)
-    int* plan_counter;               // [1] select blocks finished in this step
+    int* plan_counter;               // [2] blocks finished in this step: [0] of the selection, [1] of the append/split kernel
     int n_attn_ctas;                 // persistent gather-attention CTAs (2 per SM)
     int attn_pf_in_smem;             // 1: every attention CTA keeps a copy of work_prefix in shared memory
     // split scratch
@@ -174,6 +174,8 @@ void launch_gather_attn_v1(const Tables& t, StepPtr q, cudaStream_t s, long long
 void launch_attn_combine(const Tables& t, StepPtrW out, cudaStream_t s, long long* launches);
 void launch_split_check(const Tables& t, float gamma, int var_enabled, int min_size, int iters, cudaStream_t s,
                         long long* launches);
+void launch_append_split(const Tables& t, float gamma, int var_enabled, int min_size, int iters, int do_append, StepPtr k,
+                         StepPtr v, int* step_ctr, cudaStream_t s, long long* launches);
 void launch_step_inc(int* ctr, cudaStream_t s, long long* launches);
 
 }  // namespace dkv

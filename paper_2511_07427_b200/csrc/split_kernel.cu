@@ -6,6 +6,7 @@
 // already owns, and the moving child is written to fresh pages under the next free id.
 #include <float.h>
 
+#include "append_block.cuh"
 #include "common.cuh"
 
 namespace dkv {
@@ -15,7 +16,8 @@ constexpr int SP_CACHE_BYTES = 32 * 1024;      // member keys of the cluster bei
 constexpr int SP_WARPS = SP_THREADS / 32;
 
 template <typename KV, int HD>
-__global__ void __launch_bounds__(SP_THREADS) k_split_check(Tables t, float gamma, int var_enabled, int min_size, int iters) {
+__global__ void __launch_bounds__(SP_THREADS) k_split_check(Tables t, float gamma, int var_enabled, int min_size, int iters,
+                                                            int do_append, StepPtr app_k, StepPtr app_v, int* step_ctr) {
     constexpr int EPL = HD / 32;
     extern __shared__ int dyn[];
     const int maxch = t.max_tokens / PAGE + 2;
@@ -30,6 +32,8 @@ __global__ void __launch_bounds__(SP_THREADS) k_split_check(Tables t, float gamm
     __shared__ int s_a, s_ok;
 
     const int u = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    // fused loop iteration: the step's append for this unit comes first (Algorithm 1's order)
+    if (do_append) { append_block<KV, HD>(t, u, app_k, app_v); __syncthreads(); }
     const int N = t.u_N[u], M0 = t.u_M[u], Mlive0 = t.u_Mlive[u];
     const float tau = t.u_tau[u];
     KV* kpg = reinterpret_cast<KV*>(t.kpages) + (size_t)u * t.P * PAGE * HD;
@@ -354,26 +358,42 @@ __global__ void __launch_bounds__(SP_THREADS) k_split_check(Tables t, float gamm
         }
     }
     __syncthreads();
-    if (tid == 0) { t.u_scan[u] = s_nsplit > 0 ? 1 : 0; t.u_last[u] = -1; }
+    if (tid == 0) {
+        t.u_scan[u] = s_nsplit > 0 ? 1 : 0; t.u_last[u] = -1;
+        if (step_ctr) {
+            // the last block of the iteration advances the device-side step index that every kernel of the loop reads
+            __threadfence();
+            if (atomicAdd(t.plan_counter + 1, 1) == (int)gridDim.x - 1) { t.plan_counter[1] = 0; *step_ctr += 1; }
+        }
+    }
 }
 
 template <typename KV, int HD>
-static void split_t(const Tables& t, float gamma, int var_enabled, int min_size, int iters, cudaStream_t s) {
+static void split_t(const Tables& t, float gamma, int var_enabled, int min_size, int iters, int do_append, StepPtr k, StepPtr v,
+                    int* step_ctr, cudaStream_t s) {
     size_t dyn = sizeof(int) * (2 * (size_t)(t.max_tokens / PAGE + 2) + (size_t)t.max_clusters);
     dyn = ((dyn + 15) & ~(size_t)15) + SP_CACHE_BYTES + sizeof(int) * (SP_CACHE_BYTES / (HD * sizeof(KV))) + 16;
     if (dyn > 32 * 1024)
         cudaFuncSetAttribute(k_split_check<KV, HD>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn);
-    k_split_check<KV, HD><<<t.U, SP_THREADS, dyn, s>>>(t, gamma, var_enabled, min_size, iters);
+    k_split_check<KV, HD><<<t.U, SP_THREADS, dyn, s>>>(t, gamma, var_enabled, min_size, iters, do_append, k, v, step_ctr);
 }
 
 void launch_split_check(const Tables& t, float gamma, int var_enabled, int min_size, int iters, cudaStream_t s,
                         long long* launches) {
+    launch_append_split(t, gamma, var_enabled, min_size, iters, 0, StepPtr{nullptr, 0, nullptr}, StepPtr{nullptr, 0, nullptr}, nullptr, s,
+                        launches);
+}
+
+// The tail of a fused loop iteration in one launch: append (when do_append), split check, and, when step_ctr is
+// given, the increment of the device-side step index by the last block to finish.
+void launch_append_split(const Tables& t, float gamma, int var_enabled, int min_size, int iters, int do_append, StepPtr k,
+                         StepPtr v, int* step_ctr, cudaStream_t s, long long* launches) {
     if (t.kv_dtype == DYNAKV_F32) {
-        if (t.d == 64) split_t<float, 64>(t, gamma, var_enabled, min_size, iters, s);
-        else split_t<float, 128>(t, gamma, var_enabled, min_size, iters, s);
+        if (t.d == 64) split_t<float, 64>(t, gamma, var_enabled, min_size, iters, do_append, k, v, step_ctr, s);
+        else split_t<float, 128>(t, gamma, var_enabled, min_size, iters, do_append, k, v, step_ctr, s);
     } else {
-        if (t.d == 64) split_t<__nv_bfloat16, 64>(t, gamma, var_enabled, min_size, iters, s);
-        else split_t<__nv_bfloat16, 128>(t, gamma, var_enabled, min_size, iters, s);
+        if (t.d == 64) split_t<__nv_bfloat16, 64>(t, gamma, var_enabled, min_size, iters, do_append, k, v, step_ctr, s);
+        else split_t<__nv_bfloat16, 128>(t, gamma, var_enabled, min_size, iters, do_append, k, v, step_ctr, s);
     }
     (*launches)++;
 }
