@@ -155,6 +155,8 @@ __global__ void __launch_bounds__(AT_THREADS, 2) k_gather_attn_tma(Tables t, Ste
         s_flag[0] = 0; s_flag[1] = 0;
         asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
     }
+    pdl_trigger();       // the append/split kernel may move in as CTAs of this grid retire; it waits before it moves rows
+    pdl_wait();          // the work lists and their prefix come from the selection kernel
     const int* pf = t.work_prefix;
     if (t.attn_pf_in_smem) {
         for (int i = tid; i <= U; i += AT_THREADS) pf_s[i] = pf[i];
@@ -444,8 +446,8 @@ int attn_tma_prepare(const Tables& t) {
 
 void launch_gather_attn_tma(const Tables& t, StepPtr q, StepPtrW out, cudaStream_t s, long long* launches) {
     const size_t bytes = attn_tma_smem_bytes(t);
-    if (t.d == 64) k_gather_attn_tma<64><<<t.n_attn_ctas, AT_THREADS, bytes, s>>>(t, q, out);
-    else k_gather_attn_tma<128><<<t.n_attn_ctas, AT_THREADS, bytes, s>>>(t, q, out);
+    if (t.d == 64) launch_pdl(k_gather_attn_tma<64>, dim3(t.n_attn_ctas), dim3(AT_THREADS), bytes, s, t, q, out);
+    else launch_pdl(k_gather_attn_tma<128>, dim3(t.n_attn_ctas), dim3(AT_THREADS), bytes, s, t, q, out);
     (*launches)++;
 }
 

@@ -139,6 +139,24 @@ __device__ __forceinline__ unsigned int hash23(unsigned long long seed, int unit
     return (unsigned int)(x >> 41);
 }
 
+// ---- programmatic dependent launch: a kernel launched with launch_pdl may start while its predecessor on the
+// stream is still finishing; it must call pdl_wait() before it touches anything the predecessor writes (or
+// writes anything the predecessor reads).  pdl_trigger() in the predecessor lets the dependents start early;
+// without it they start when the predecessor's blocks have exited.  Both are no-ops in an ordinary launch.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;\n" ::: "memory"); }
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;\n" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s, Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = s;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = at; cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kern, KArgs(args)...);
+}
+
 // Kernel classes for the optional per-kernel event timing.
 enum { KC_INIT = 0, KC_ASSIGN = 1, KC_UPDATE = 2, KC_FINALIZE = 3, KC_SELECT = 4, KC_ATTN = 5, KC_COMBINE = 6,
        KC_APPEND = 7, KC_SPLIT = 8, KC_FRONT = 9, KC_COUNT = 10 };

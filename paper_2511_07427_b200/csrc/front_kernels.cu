@@ -31,7 +31,7 @@ __global__ void __launch_bounds__(FR_THREADS) k_front(Tables t, StepPtr qp, Step
     const int u = blockIdx.y;
     const int Mcur = t.u_M[u];
     const int j0 = blockIdx.x * FR_ROWS;
-    if (j0 >= Mcur) return;
+    if (j0 >= Mcur) { pdl_trigger(); return; }
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int sub = lane >> 3, l8 = lane & 7;
     float qs[V4][4], kk[V4][4];
@@ -96,6 +96,7 @@ __global__ void __launch_bounds__(FR_THREADS) k_front(Tables t, StepPtr qp, Step
             if (has_k) DS[j] = live ? dd : INFINITY;
         }
     }
+    pdl_trigger();
 }
 
 // ------------------------------------------------------------------ k_select
@@ -118,6 +119,7 @@ __global__ void __launch_bounds__(SL_THREADS) k_select(Tables t, int budget, int
     __shared__ int sh[33];
     __shared__ int s_bin, s_rem, s_done, s_eqtake, s_eqcnt, s_L, s_tok;
     __shared__ unsigned long long s_best;
+    pdl_wait();                          // the scores come from the kernel before
     const int Mcur = t.u_M[u];
     const float* SC = t.scores + (size_t)u * t.max_clusters;
     const int* CN = t.cl_n + (size_t)u * t.max_clusters;
@@ -293,6 +295,7 @@ __global__ void __launch_bounds__(SL_THREADS) k_select(Tables t, int budget, int
         for (int i = b0; i < b1; i++) { t.work_prefix[i] = base; base += __ldcg(&t.n_work[i]); }
         if (tid == 0) { t.work_prefix[t.U] = tot; *t.plan_counter = 0; }
     }
+    pdl_trigger();
 }
 
 // ------------------------------------------------------------------ k_append_apply
@@ -318,7 +321,7 @@ void launch_front(const Tables& t, StepPtr q, StepPtr k, int has_q, int has_k, c
 }
 
 void launch_select(const Tables& t, int budget, int* user_sel_ids, cudaStream_t s, long long* launches) {
-    k_select<<<t.U, SL_THREADS, 0, s>>>(t, budget, user_sel_ids);
+    launch_pdl(k_select, dim3(t.U), dim3(SL_THREADS), 0, s, t, budget, user_sel_ids);
     (*launches)++;
 }
 

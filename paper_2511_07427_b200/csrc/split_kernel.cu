@@ -87,6 +87,9 @@ __global__ void __launch_bounds__(SP_THREADS) k_split_check(Tables t, float gamm
         __syncthreads();
     }
     const int ntrig = s_ntrig;
+    // Everything above reads and writes only what the gather-attention kernel before this one never touches
+    // (statistics, the new row beyond every listed row); the splits below move rows, so they wait for it.
+    if (ntrig > 0) pdl_wait();
     for (int li = 0; li < ntrig; li++) {
         const int j = trig[li];
         const size_t cj = (size_t)u * t.max_clusters + j;
@@ -358,6 +361,9 @@ __global__ void __launch_bounds__(SP_THREADS) k_split_check(Tables t, float gamm
         }
     }
     __syncthreads();
+    // No block leaves before the kernel ahead has completed: the next kernel on the stream (the next iteration's
+    // centroid pass and selection, which rewrite the work lists) is ordered behind THIS kernel only.
+    pdl_wait();
     if (tid == 0) {
         t.u_scan[u] = s_nsplit > 0 ? 1 : 0; t.u_last[u] = -1;
         if (step_ctr) {
@@ -375,7 +381,7 @@ static void split_t(const Tables& t, float gamma, int var_enabled, int min_size,
     dyn = ((dyn + 15) & ~(size_t)15) + SP_CACHE_BYTES + sizeof(int) * (SP_CACHE_BYTES / (HD * sizeof(KV))) + 16;
     if (dyn > 32 * 1024)
         cudaFuncSetAttribute(k_split_check<KV, HD>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn);
-    k_split_check<KV, HD><<<t.U, SP_THREADS, dyn, s>>>(t, gamma, var_enabled, min_size, iters, do_append, k, v, step_ctr);
+    launch_pdl(k_split_check<KV, HD>, dim3(t.U), dim3(SP_THREADS), dyn, s, t, gamma, var_enabled, min_size, iters, do_append, k, v, step_ctr);
 }
 
 void launch_split_check(const Tables& t, float gamma, int var_enabled, int min_size, int iters, cudaStream_t s,
