@@ -35,7 +35,7 @@ struct dynakv_ctx {
     int* trace_picks = nullptr;    // [U][M0]
     // graph loop
     int* step_ctr = nullptr;
-    cudaGraphExec_t graph_exec = nullptr;
+    cudaGraphExec_t graph_exec = nullptr, graph_exec_long = nullptr;   // one iteration / eight iterations
     const void* g_q = nullptr; const void* g_k = nullptr; const void* g_v = nullptr; void* g_out = nullptr;
     int g_budget = -1;
     long long graph_nodes = 0;
@@ -202,6 +202,7 @@ extern "C" void dynakv_destroy(dynakv_ctx* c) {
     if (!c) return;
     cudaStreamSynchronize(c->stream);
     if (c->graph_exec) cudaGraphExecDestroy(c->graph_exec);
+    if (c->graph_exec_long) cudaGraphExecDestroy(c->graph_exec_long);
     for (auto& sp : c->spans) { cudaEventDestroy(sp.e0); cudaEventDestroy(sp.e1); }
     for (cudaEvent_t e : c->event_pool) cudaEventDestroy(e);
     for (void* p : c->allocs) cudaFree(p);
@@ -336,33 +337,42 @@ extern "C" int dynakv_decode_loop(dynakv_ctx* c, const float* q_steps, const voi
         return DYNAKV_ERR_STATE;
     }
     const Tables& t = c->t;
+    constexpr int UNROLL = 8;            // iterations in the long graph; the remainder runs the one-iteration graph
     if (!c->graph_exec || c->g_q != q_steps || c->g_k != k_steps || c->g_v != v_steps || c->g_out != out_steps ||
         c->g_budget != token_budget) {
         if (c->graph_exec) { cudaGraphExecDestroy(c->graph_exec); c->graph_exec = nullptr; }
+        if (c->graph_exec_long) { cudaGraphExecDestroy(c->graph_exec_long); c->graph_exec_long = nullptr; }
         const long long qs = (long long)t.U * t.G * t.d * 4, ks = (long long)t.U * t.d * (long long)kv_bytes(c->cfg);
-        cudaGraph_t graph = nullptr;
-        long long before = c->launches;
-        CK(cudaStreamBeginCapture(c->stream, cudaStreamCaptureModeThreadLocal));
-        enqueue_step(c, StepPtr{q_steps, qs, c->step_ctr}, StepPtr{k_steps, ks, c->step_ctr},
-                     StepPtr{v_steps, ks, c->step_ctr}, token_budget, StepPtrW{out_steps, qs, c->step_ctr}, c->step_ctr, false);
-        cudaError_t e = cudaStreamEndCapture(c->stream, &graph);
-        c->graph_nodes = c->launches - before;
-        c->launches = before;
-        if (e != cudaSuccess || !graph) {
-            snprintf(g_err, sizeof(g_err), "graph capture failed: %s", cudaGetErrorString(e));
-            return DYNAKV_ERR_CUDA;
-        }
-        e = cudaGraphInstantiate(&c->graph_exec, graph, 0);
-        cudaGraphDestroy(graph);
-        if (e != cudaSuccess) {
-            c->graph_exec = nullptr;
-            snprintf(g_err, sizeof(g_err), "graph instantiate failed: %s", cudaGetErrorString(e));
-            return DYNAKV_ERR_CUDA;
+        for (int which = 0; which < 2; which++) {
+            const int reps = which == 0 ? 1 : UNROLL;
+            cudaGraph_t graph = nullptr;
+            long long before = c->launches;
+            CK(cudaStreamBeginCapture(c->stream, cudaStreamCaptureModeThreadLocal));
+            for (int r = 0; r < reps; r++)
+                enqueue_step(c, StepPtr{q_steps, qs, c->step_ctr}, StepPtr{k_steps, ks, c->step_ctr},
+                             StepPtr{v_steps, ks, c->step_ctr}, token_budget, StepPtrW{out_steps, qs, c->step_ctr}, c->step_ctr, false);
+            cudaError_t e = cudaStreamEndCapture(c->stream, &graph);
+            if (which == 0) c->graph_nodes = c->launches - before;
+            c->launches = before;
+            if (e != cudaSuccess || !graph) {
+                snprintf(g_err, sizeof(g_err), "graph capture failed: %s", cudaGetErrorString(e));
+                return DYNAKV_ERR_CUDA;
+            }
+            e = cudaGraphInstantiate(which == 0 ? &c->graph_exec : &c->graph_exec_long, graph, 0);
+            cudaGraphDestroy(graph);
+            if (e != cudaSuccess) {
+                if (c->graph_exec) { cudaGraphExecDestroy(c->graph_exec); c->graph_exec = nullptr; }
+                c->graph_exec_long = nullptr;
+                snprintf(g_err, sizeof(g_err), "graph instantiate failed: %s", cudaGetErrorString(e));
+                return DYNAKV_ERR_CUDA;
+            }
         }
         c->g_q = q_steps; c->g_k = k_steps; c->g_v = v_steps; c->g_out = out_steps; c->g_budget = token_budget;
     }
     CK(cudaMemsetAsync(c->step_ctr, 0, sizeof(int), c->stream));
-    for (int64_t s = 0; s < n_steps; s++) CK(cudaGraphLaunch(c->graph_exec, c->stream));
+    int64_t s = 0;
+    for (; s + UNROLL <= n_steps; s += UNROLL) CK(cudaGraphLaunch(c->graph_exec_long, c->stream));
+    for (; s < n_steps; s++) CK(cudaGraphLaunch(c->graph_exec, c->stream));
     c->launches += c->graph_nodes * n_steps;
     return DYNAKV_OK;
 }

@@ -29,6 +29,7 @@ template <typename KV, int HD>
 __global__ void __launch_bounds__(FR_THREADS) k_front(Tables t, StepPtr qp, StepPtr kp, int has_q, int has_k) {
     constexpr int V4 = HD / 32;   // float4 loads per lane per row
     const int u = blockIdx.y;
+    pdl_wait();                          // inside a captured loop the representatives come from the iteration before
     const int Mcur = t.u_M[u];
     const int j0 = blockIdx.x * FR_ROWS;
     if (j0 >= Mcur) { pdl_trigger(); return; }
@@ -311,11 +312,11 @@ __global__ void __launch_bounds__(256) k_append_apply(Tables t, StepPtr kp_, Ste
 void launch_front(const Tables& t, StepPtr q, StepPtr k, int has_q, int has_k, cudaStream_t s, long long* launches) {
     dim3 grid((t.max_clusters + FR_ROWS - 1) / FR_ROWS, t.U);
     if (t.kv_dtype == DYNAKV_F32) {
-        if (t.d == 64) k_front<float, 64><<<grid, FR_THREADS, 0, s>>>(t, q, k, has_q, has_k);
-        else k_front<float, 128><<<grid, FR_THREADS, 0, s>>>(t, q, k, has_q, has_k);
+        if (t.d == 64) launch_pdl(k_front<float, 64>, grid, dim3(FR_THREADS), 0, s, t, q, k, has_q, has_k);
+        else launch_pdl(k_front<float, 128>, grid, dim3(FR_THREADS), 0, s, t, q, k, has_q, has_k);
     } else {
-        if (t.d == 64) k_front<__nv_bfloat16, 64><<<grid, FR_THREADS, 0, s>>>(t, q, k, has_q, has_k);
-        else k_front<__nv_bfloat16, 128><<<grid, FR_THREADS, 0, s>>>(t, q, k, has_q, has_k);
+        if (t.d == 64) launch_pdl(k_front<__nv_bfloat16, 64>, grid, dim3(FR_THREADS), 0, s, t, q, k, has_q, has_k);
+        else launch_pdl(k_front<__nv_bfloat16, 128>, grid, dim3(FR_THREADS), 0, s, t, q, k, has_q, has_k);
     }
     (*launches)++;
 }
