@@ -44,11 +44,14 @@ __device__ __forceinline__ void tc_mbar_arrive(unsigned bar) {
 __device__ __forceinline__ void tc_mbar_expect_tx(unsigned bar, unsigned bytes) {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n" ::"r"(bar), "r"(bytes) : "memory");
 }
+// One poll; the thread is suspended in hardware until the phase completes or about `hint_ns` have passed, so
+// a waiting role does not compete for issue slots with the warps that drain the accumulators.
 __device__ __forceinline__ bool tc_mbar_try_wait(unsigned bar, unsigned parity) {
     unsigned ok;
+    const unsigned hint_ns = 20000u;
     asm volatile(
-        "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}\n"
-        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+        "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n selp.u32 %0, 1, 0, p;\n}\n"
+        : "=r"(ok) : "r"(bar), "r"(parity), "r"(hint_ns) : "memory");
     return ok != 0;
 }
 __device__ __forceinline__ unsigned long long tc_global_ns() {
@@ -181,7 +184,7 @@ __device__ __forceinline__ float tc_min3(float a, float b, float c) {
 }
 // Value with its low 8 mantissa bits replaced by a column index (a relative change below 2^-15).
 __device__ __forceinline__ float tc_pack(float x, int col) {
-    return __uint_as_float((__float_as_uint(x) & 0xFFFFFF00u) | (unsigned)col);
+    return __uint_as_float(__byte_perm(__float_as_uint(x), (unsigned)col, 0x3214));   // one byte-permute: bytes 3..1 of x, byte 0 of col
 }
 // (t1 <= t2 <= t3) <- the three smallest of {t1, t2, t3, x, y}.
 __device__ __forceinline__ void tc_top3_pair(float& t1, float& t2, float& t3, float x, float y) {
