@@ -130,12 +130,16 @@ constexpr unsigned TC_IDESC = (1u << 4) | ((unsigned)(TC_BN >> 3) << 17) | ((uns
 
 // Keys bf16 -> fp16 (exact unless |k| > 65504, which raises *bad; values below 2^-24 lose bits, which
 // the margin covers) and ||k_i|| in fp32.  One warp per key.
-__global__ void __launch_bounds__(256) k_tc_prep_keys(const __nv_bfloat16* __restrict__ K, long long rows,
-                                                      __half* __restrict__ A16, float* __restrict__ knorm, int* __restrict__ bad) {
+__global__ void __launch_bounds__(256) k_tc_prep_keys(const __nv_bfloat16* __restrict__ K, long long rows, int n,
+                                                      __half* __restrict__ A16, float* __restrict__ knorm,
+                                                      unsigned* __restrict__ knmax_bits, int* __restrict__ bad) {
     const int lane = threadIdx.x & 31;
-    long long w = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const long long wid = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const long long nw = ((long long)gridDim.x * blockDim.x) >> 5;
-    for (; w < rows; w += nw) {
+    const long long per = (rows + nw - 1) / nw;          // a contiguous run of keys per warp: few unit changes
+    long long cur_u = -1;
+    float cur_max = 0.f;
+    for (long long w = wid * per; w < min(rows, (wid + 1) * per); w++) {
         const float4 v = ld4(K + (size_t)w * TC_D, lane * 4);
         const float m = fmaxf(fmaxf(fabsf(v.x), fabsf(v.y)), fmaxf(fabsf(v.z), fabsf(v.w)));
         if (!(m <= 65504.f)) atomicOr(bad, 1);
@@ -145,12 +149,21 @@ __global__ void __launch_bounds__(256) k_tc_prep_keys(const __nv_bfloat16* __res
         *reinterpret_cast<uint2*>(A16 + (size_t)w * TC_D + lane * 4) = pk;
         float s = v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
         s = warp_sum(s);
-        if (lane == 0) knorm[w] = sqrtf(s);
+        const float kn = sqrtf(s);
+        if (lane == 0) knorm[w] = kn;
+        const long long uu = w / n;
+        if (uu != cur_u) {
+            if (lane == 0 && cur_u >= 0) atomicMax(&knmax_bits[cur_u], __float_as_uint(cur_max));
+            cur_u = uu; cur_max = 0.f;
+        }
+        cur_max = fmaxf(cur_max, kn);
     }
+    if (lane == 0 && cur_u >= 0) atomicMax(&knmax_bits[cur_u], __float_as_uint(cur_max));   // largest key norm of the unit
 }
 
-// Centres fp32 -> fp16, bias_j = ||c_j||^2 (fp32, of the unrounded centre; 1e38 for the padding
-// columns j >= M), cmax[u] = max_j ||c_j||.  One warp per (unit, padded centre index).
+// Centres fp32 -> fp16 into a copy padded to Mpad rows per unit (padding rows are zero, so their dot products
+// are exactly zero), bias_j = ||c_j||^2 in fp32 of the unrounded centre, cmax[u] = max_j ||c_j||.
+// One warp per (unit, padded centre index).
 __global__ void __launch_bounds__(256) k_tc_prep_centres(const float* __restrict__ C, int U, int M, int Mpad,
                                                          __half* __restrict__ B16, float* __restrict__ bias,
                                                          unsigned* __restrict__ cmax_bits, int* __restrict__ bad) {
@@ -158,7 +171,11 @@ __global__ void __launch_bounds__(256) k_tc_prep_centres(const float* __restrict
     const long long w = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     if (w >= (long long)U * Mpad) return;
     const int u = (int)(w / Mpad), j = (int)(w % Mpad);
-    if (j >= M) { if (lane == 0) bias[w] = 1.0e38f; return; }     // finite: inf with packed column bits would read as NaN
+    if (j >= M) {
+        *reinterpret_cast<uint2*>(B16 + (size_t)w * TC_D + lane * 4) = make_uint2(0u, 0u);
+        if (lane == 0) bias[w] = 0.f;
+        return;
+    }
     const size_t row = (size_t)u * M + j;
     const float4 v = *reinterpret_cast<const float4*>(C + row * TC_D + lane * 4);
     const float m = fmaxf(fmaxf(fabsf(v.x), fabsf(v.y)), fmaxf(fabsf(v.z), fabsf(v.w)));
@@ -166,13 +183,37 @@ __global__ void __launch_bounds__(256) k_tc_prep_centres(const float* __restrict
     __half2 h0 = __floats2half2_rn(v.x, v.y), h1 = __floats2half2_rn(v.z, v.w);
     uint2 pk;
     pk.x = *reinterpret_cast<unsigned*>(&h0); pk.y = *reinterpret_cast<unsigned*>(&h1);
-    *reinterpret_cast<uint2*>(B16 + row * TC_D + lane * 4) = pk;
+    *reinterpret_cast<uint2*>(B16 + (size_t)w * TC_D + lane * 4) = pk;
     float s = v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
     s = warp_sum(s);
     if (lane == 0) {
         bias[w] = s;
         atomicMax(&cmax_bits[u], __float_as_uint(sqrtf(s)));     // non-negative floats order like their bit patterns
     }
+}
+
+// Fixed-point form of the filter values.  With S_u a power of two such that |x| S_u <= 2^29 for every value
+// x = ||c_j||^2 - 2 k.c_j of the unit, the single fma  v = acc * (-2 S_u) + B_j,  B_j = 1.5 * 2^31 + bias_j S_u,
+// lands in [2^31, 2^32), where floats are 256 apart: the 23 mantissa bits of v ARE the value on a grid of
+// g_u = 256 / S_u (offset 2^22), already rounded, and one integer multiply-add  bits(v) * 256 + column  (the
+// exponent falls off the top) makes a word whose low 8 bits are free for the column and which still orders like
+// the value when compared as a positive float.  Padding columns get the largest mantissa in use.
+// scale[u] = (S_u, g_u); one thread per (unit, padded column).
+constexpr float TC_MAGIC = 3221225472.f;                 // 1.5 * 2^31
+constexpr unsigned TC_PAD_MANT = 0x700000u;              // above 2^22 + 2^21, below the NaN patterns after the shift
+__global__ void __launch_bounds__(256) k_tc_fixed_bias(const float* __restrict__ bias, const unsigned* __restrict__ cmax_bits,
+                                                       const unsigned* __restrict__ knmax_bits, int U, int M, int Mpad,
+                                                       float* __restrict__ Bfix, float2* __restrict__ scale) {
+    const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= (long long)U * Mpad) return;
+    const int u = (int)(idx / Mpad), j = (int)(idx % Mpad);
+    const float cm = __uint_as_float(cmax_bits[u]), kn = __uint_as_float(knmax_bits[u]);
+    const float xmax = fmaxf(cm * cm + 2.f * kn * cm, 1e-30f);
+    int e = (int)floorf(log2f(536870912.f / xmax));      // 2^29 / xmax
+    e = max(-100, min(100, e));
+    const float S = exp2f((float)e);
+    if (j == 0) scale[u] = make_float2(S, 256.f / S);
+    Bfix[idx] = j < M ? TC_MAGIC + bias[idx] * S : __uint_as_float(0x4F000000u | TC_PAD_MANT);   // 2^31 * (1 + mant / 2^23)
 }
 
 // ------------------------------------------------------------------ the distance GEMM + top-3 filter
@@ -182,9 +223,13 @@ __device__ __forceinline__ float tc_min3(float a, float b, float c) {
     asm("min.f32 %0, %1, %2, %3;\n" : "=f"(r) : "f"(a), "f"(b), "f"(c));
     return r;
 }
-// Value with its low 8 mantissa bits replaced by a column index (a relative change below 2^-15).
-__device__ __forceinline__ float tc_pack(float x, int col) {
-    return __uint_as_float(__byte_perm(__float_as_uint(x), (unsigned)col, 0x3214));   // one byte-permute: bytes 3..1 of x, byte 0 of col
+// Fixed-point filter word: bits(v) * 256 + column (see k_tc_fixed_bias), as a positive float for min/max.  The
+// multiply-add is written in PTX so that it stays an integer multiply-add (FMA pipe) and does not become
+// shift/logic instructions on the ALU pipe, which the min/max chains keep busy.
+__device__ __forceinline__ float tc_pack(float v, int col) {
+    unsigned r;
+    asm("mad.lo.u32 %0, %1, 256, %2;\n" : "=r"(r) : "r"(__float_as_uint(v)), "r"((unsigned)col));
+    return __uint_as_float(r);
 }
 // (t1 <= t2 <= t3) <- the three smallest of {t1, t2, t3, x, y}.
 __device__ __forceinline__ void tc_top3_pair(float& t1, float& t2, float& t3, float x, float y) {
@@ -209,7 +254,8 @@ __device__ __forceinline__ void tc_insert(float& g1, int& j1, float& g2, int& j2
 
 struct TcArgs {
     int U, n, M, Mpad, KB;               // KB = 128-key blocks per unit
-    const float* bias;                   // [U][Mpad]
+    const float* Bfix;                   // [U][Mpad] fixed-point bias 1.5 * 2^31 + ||c_j||^2 S_u
+    const float2* scale;                 // [U] (S_u, g_u = 256 / S_u)
     const float* knorm;                  // [U * n]
     const unsigned* cmax_bits;           // [U]
     int* assign;                         // [U * n]
@@ -273,7 +319,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) k_tc_assign(const __grid_consta
                     const int st = (int)(tb & 1);
                     if (!tc_mbar_wait(bar(6 + st), (unsigned)((tb >> 1) & 1) ^ 1u)) { *s_abort = 1; break; }
                     tc_mbar_expect_tx(bar(4 + st), TC_B_BYTES);
-                    const int rowB = u * p.M + nt * TC_BN;
+                    const int rowB = u * p.Mpad + nt * TC_BN;
                     tc_tma_load_2d(sB + st * TC_B_BYTES, &mapB, 0, rowB, bar(4 + st));
                     tc_tma_load_2d(sB + st * TC_B_BYTES + TC_B_BYTES / 2, &mapB, 64, rowB, bar(4 + st));
                     lastB[st] = tb;
@@ -329,6 +375,8 @@ __global__ void __launch_bounds__(TC_THREADS, 1) k_tc_assign(const __grid_consta
             float g1 = INFINITY, g2 = INFINITY, g3 = INFINITY;
             int j1 = 0, j2 = 0;
             bool dead = false;
+            const float2 sc = p.scale[u];
+            const float m2S = -2.f * sc.x;
             for (int nt = 0; nt < NT; nt++, tb++) {
                 const int st = (int)(tb & 1);
                 if (st != grp) continue;
@@ -337,27 +385,33 @@ __global__ void __launch_bounds__(TC_THREADS, 1) k_tc_assign(const __grid_consta
                 float ch[4][3];                                        // four independent chains of three smallest
 #pragma unroll
                 for (int x = 0; x < 4; x++) { ch[x][0] = INFINITY; ch[x][1] = INFINITY; ch[x][2] = INFINITY; }
-                const float4* bias4 = reinterpret_cast<const float4*>(p.bias + (size_t)u * p.Mpad + (size_t)nt * TC_BN);
+                const float4* bias4 = reinterpret_cast<const float4*>(p.Bfix + (size_t)u * p.Mpad + (size_t)nt * TC_BN);
                 const unsigned tbase = tmem + st * TC_BN + ((unsigned)(q * 32) << 16);
                 unsigned acc[2][32];
-                tc_ld32(tbase, acc[0]);
-#pragma unroll
-                for (int c = 0; c < TC_BN / 32; c++) {
-                    float bs[32];
+                float bs[2][32];
+                auto load_bias = [&](int c, float (&dst)[32]) {
 #pragma unroll
                     for (int e = 0; e < 8; e++) {
                         const float4 v = __ldg(bias4 + c * 8 + e);
-                        bs[4 * e] = v.x; bs[4 * e + 1] = v.y; bs[4 * e + 2] = v.z; bs[4 * e + 3] = v.w;
+                        dst[4 * e] = v.x; dst[4 * e + 1] = v.y; dst[4 * e + 2] = v.z; dst[4 * e + 3] = v.w;
                     }
+                };
+                tc_ld32(tbase, acc[0]);
+                load_bias(0, bs[0]);
+#pragma unroll
+                for (int c = 0; c < TC_BN / 32; c++) {
                     tc_ld_wait();                                           // chunk c has arrived
-                    if (c + 1 < TC_BN / 32) tc_ld32(tbase + (c + 1) * 32, acc[(c + 1) & 1]);   // chunk c + 1 in flight
+                    if (c + 1 < TC_BN / 32) {                               // chunk c + 1 and its bias in flight
+                        tc_ld32(tbase + (c + 1) * 32, acc[(c + 1) & 1]);
+                        load_bias(c + 1, bs[(c + 1) & 1]);
+                    }
 #pragma unroll
                     for (int e = 0; e < 32; e += 8) {
 #pragma unroll
                         for (int x = 0; x < 4; x++) {
                             const int e0 = e + 2 * x;
-                            const float x0 = tc_pack(fmaf(-2.f, __uint_as_float(acc[c & 1][e0]), bs[e0]), c * 32 + e0);
-                            const float x1 = tc_pack(fmaf(-2.f, __uint_as_float(acc[c & 1][e0 + 1]), bs[e0 + 1]), c * 32 + e0 + 1);
+                            const float x0 = tc_pack(fmaf(__uint_as_float(acc[c & 1][e0]), m2S, bs[c & 1][e0]), c * 32 + e0);
+                            const float x1 = tc_pack(fmaf(__uint_as_float(acc[c & 1][e0 + 1]), m2S, bs[c & 1][e0 + 1]), c * 32 + e0 + 1);
                             tc_top3_pair(ch[x][0], ch[x][1], ch[x][2], x0, x1);
                         }
                     }
@@ -392,10 +446,13 @@ __global__ void __launch_bounds__(TC_THREADS, 1) k_tc_assign(const __grid_consta
                 p.assign[gi] = j1;
                 const float kn = p.knorm[gi], cm = __uint_as_float(p.cmax_bits[u]);
                 // bound on |filter value - true value|: fp16 rounding of the centres (2 kn cm 2^-11, with 3 % slack
-                // for the accumulation), truncation of the 8 packed bits (2^-15 |x|), sub-normal keys
-                const float E = kn * cm * (1.03f / 1024.f) + (cm * cm + 2.f * kn * cm) * (1.f / 32768.f) + cm * 1e-6f;
-                if (!(g2 - g1 > 2.f * E)) {
-                    if (g3 - g1 > 2.f * E && j2 < p.M) {
+                // for the accumulation), the two roundings to the fixed-point grid, sub-normal keys
+                const float E = kn * cm * (1.03f / 1024.f) + 2.f * sc.y + cm * 1e-6f;
+                // gaps in value units: mantissa differences times the grid
+                const unsigned m1 = __float_as_uint(g1) >> 8, m2 = __float_as_uint(g2) >> 8, m3 = __float_as_uint(g3) >> 8;
+                const float gap2 = (float)(m2 - m1) * sc.y, gap3 = (float)(m3 - m1) * sc.y;
+                if (!(gap2 > 2.f * E)) {
+                    if (gap3 > 2.f * E && j2 < p.M) {
                         // only the best two can be the true argmin: decide between them exactly
                         const unsigned long long pos = atomicAdd(p.pair_count, 1ull);
                         p.pair_list[pos] = make_int2((int)gi, j1 | (j2 << 16));
@@ -453,7 +510,7 @@ __global__ void __launch_bounds__(256) k_tc_pair_decide(const __nv_bfloat16* __r
 static size_t tc_align(size_t x) { return (x + 255) & ~(size_t)255; }
 
 struct TcLayout {
-    size_t a16, knorm, b16, bias, cmax, bad, list, count, pairs, pair_count, total;
+    size_t a16, knorm, b16, bias, bfix, scale, cmax, knmax, bad, list, count, pairs, pair_count, total;
     int Mpad;
 };
 static TcLayout tc_layout(const Tables& t, long long n, int M) {
@@ -463,9 +520,12 @@ static TcLayout tc_layout(const Tables& t, long long n, int M) {
     size_t off = 0;
     L.a16 = off; off += tc_align(U * (size_t)n * TC_D * 2);
     L.knorm = off; off += tc_align(U * (size_t)n * 4);
-    L.b16 = off; off += tc_align(U * (size_t)M * TC_D * 2);
+    L.b16 = off; off += tc_align(U * (size_t)L.Mpad * TC_D * 2);
     L.bias = off; off += tc_align(U * (size_t)L.Mpad * 4);
+    L.bfix = off; off += tc_align(U * (size_t)L.Mpad * 4);
+    L.scale = off; off += tc_align(U * 8);
     L.cmax = off; off += tc_align(U * 4);
+    L.knmax = off; off += tc_align(U * 4);
     L.bad = off; off += 256;
     L.list = off; off += tc_align(U * (size_t)n * 4);
     L.count = off; off += tc_align(U * 4);
@@ -477,7 +537,7 @@ static TcLayout tc_layout(const Tables& t, long long n, int M) {
 
 bool tc_assign_supported(const Tables& t, long long n, int M) {
     return t.kv_dtype == DYNAKV_BF16 && t.d == TC_D && M >= 1 && n >= 1 && (long long)t.U * n < (1ll << 31) &&
-           (long long)t.U * M < (1ll << 31);
+           (long long)t.U * (M + TC_BN) < (1ll << 31);
 }
 
 size_t tc_assign_scratch_bytes(const Tables& t, long long n, int M) { return tc_layout(t, n, M).total; }
@@ -492,9 +552,11 @@ bool tc_assign_begin(const Tables& t, const void* K, long long n, int M, void* s
     const long long rows = (long long)t.U * n;
     long long blocks = (rows + 7) / 8;
     if (blocks > 148LL * 32) blocks = 148LL * 32;
-    k_tc_prep_keys<<<(unsigned)blocks, 256, 0, s>>>(reinterpret_cast<const __nv_bfloat16*>(K), rows,
+    if (cudaMemsetAsync(base + L.knmax, 0, (size_t)t.U * 4, s) != cudaSuccess) return false;
+    k_tc_prep_keys<<<(unsigned)blocks, 256, 0, s>>>(reinterpret_cast<const __nv_bfloat16*>(K), rows, (int)n,
                                                    reinterpret_cast<__half*>(base + L.a16),
-                                                   reinterpret_cast<float*>(base + L.knorm), bad);
+                                                   reinterpret_cast<float*>(base + L.knorm),
+                                                   reinterpret_cast<unsigned*>(base + L.knmax), bad);
     (*launches)++;
     int h_bad = 1;
     if (cudaMemcpyAsync(&h_bad, bad, sizeof(int), cudaMemcpyDeviceToHost, s) != cudaSuccess) return false;
@@ -560,15 +622,19 @@ void launch_assign_tc(const Tables& t, const void* K, long long n, int M, const 
     cudaMemsetAsync(pair_count, 0, 8, s);
     const long long cw = (long long)t.U * L.Mpad;
     k_tc_prep_centres<<<(unsigned)((cw + 7) / 8), 256, 0, s>>>(C, t.U, M, L.Mpad, B16, bias, cmax, bad);
+    float* Bfix = reinterpret_cast<float*>(base + L.bfix);
+    float2* scale = reinterpret_cast<float2*>(base + L.scale);
+    k_tc_fixed_bias<<<(unsigned)((cw + 255) / 256), 256, 0, s>>>(bias, cmax, reinterpret_cast<const unsigned*>(base + L.knmax), t.U, M,
+                                                                 L.Mpad, Bfix, scale);
     CUtensorMap mapA, mapB;
-    if (!tc_make_map(&mapA, A16, (unsigned long long)t.U * n, TC_BM) || !tc_make_map(&mapB, B16, (unsigned long long)t.U * M, TC_BN)) {
+    if (!tc_make_map(&mapA, A16, (unsigned long long)t.U * n, TC_BM) || !tc_make_map(&mapB, B16, (unsigned long long)t.U * L.Mpad, TC_BN)) {
         // cannot describe the operands to the TMA unit: do the whole round exactly
         launch_assign_f32(t, K, n, M, C, assign, s, launches);
         return;
     }
     TcArgs a;
     a.U = t.U; a.n = (int)n; a.M = M; a.Mpad = L.Mpad; a.KB = (int)((n + TC_BM - 1) / TC_BM);
-    a.bias = bias; a.knorm = reinterpret_cast<const float*>(base + L.knorm); a.cmax_bits = cmax;
+    a.Bfix = Bfix; a.scale = scale; a.knorm = reinterpret_cast<const float*>(base + L.knorm); a.cmax_bits = cmax;
     a.assign = assign; a.recheck_list = list; a.recheck_count = count; a.status = t.status;
     a.pair_list = pairs; a.pair_count = pair_count;
     const int grid = t.n_attn_ctas / 2;        // one persistent CTA per SM
@@ -576,7 +642,7 @@ void launch_assign_tc(const Tables& t, const void* K, long long n, int M, const 
     const unsigned long long rows = (unsigned long long)t.U * n;
     k_tc_pair_decide<<<(unsigned)((rows + 255) / 256), 256, 0, s>>>(reinterpret_cast<const __nv_bfloat16*>(K), C, (int)n, M, pairs,
                                                                     pair_count, assign, &t.counters[CNT_RECHECKED]);
-    (*launches) += 3;
+    (*launches) += 4;
     launch_assign_f32_listed(t, K, n, M, C, assign, list, count, &t.counters[CNT_RECHECKED], s, launches);
 }
 
