@@ -111,9 +111,13 @@ constexpr int TC_BM = 128;                // keys per item (one TMEM lane each)
 constexpr int TC_BN = 256;                // centres per accumulator
 constexpr int TC_A_BYTES = TC_BM * TC_D * 2;          // 32 KB: two [128 rows x 128 B] swizzle panels
 constexpr int TC_B_BYTES = TC_BN * TC_D * 2;          // 64 KB: two [256 rows x 128 B] swizzle panels
-constexpr int TC_XCHG_BYTES = 2 * TC_BM * 5 * 4;      // hand-over of (g1, g2, g3, j1, j2) between the drain groups
+constexpr int TC_XCHG_BYTES = 2 * 3 * TC_BM * 5 * 4;      // hand-over of (g1, g2, g3, j1, j2) between the drain groups
 constexpr int TC_SMEM_BYTES = 2 * TC_A_BYTES + 2 * TC_B_BYTES + 1024 /* alignment */ + 256 /* barriers */ + TC_XCHG_BYTES;
-constexpr int TC_THREADS = 320;           // warp 0 loads, warp 1 issues MMAs, warps 2..9 drain the accumulators
+#ifndef DKV_TC_GROUPS
+#define DKV_TC_GROUPS 4
+#endif
+constexpr int TC_GROUPS = DKV_TC_GROUPS;  // drain groups of four warps: 2 (one per accumulator) or 4 (two per accumulator, half the columns each)
+constexpr int TC_THREADS = 64 + 128 * TC_GROUPS;   // warp 0 loads, warp 1 issues MMAs, the rest drain the accumulators
 constexpr unsigned TC_TMEM_COLS = 512;    // two 256-column fp32 accumulators
 
 // Shared-memory matrix descriptor of a K-major panel with 128-byte rows under the 128-byte swizzle:
@@ -287,7 +291,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) k_tc_assign(const __grid_consta
     if (tid == 0) {
         for (int i = 0; i < 8; i++) tc_mbar_init(bar(i), 1);
         tc_mbar_init(bar(8), 1); tc_mbar_init(bar(9), 1);
-        tc_mbar_init(bar(10), 4); tc_mbar_init(bar(11), 4);           // one arrival per epilogue warp
+        tc_mbar_init(bar(10), 2 * TC_GROUPS); tc_mbar_init(bar(11), 2 * TC_GROUPS);   // one arrival per draining warp
         *s_abort = 0;
         asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
     }
@@ -365,7 +369,10 @@ __global__ void __launch_bounds__(TC_THREADS, 1) k_tc_assign(const __grid_consta
         // group.  Per tile the thread keeps the three smallest packed values (low 8 bits = column) in two
         // independent chains and merges them into its best two (with indices) and third value; at the end of an
         // item group 1 hands its triple to group 0 through shared memory, and group 0 decides.
-        const int grp = (warp - 2) >> 2;              // 0 or 1
+        const int grp = (warp - 2) >> 2;              // drain group
+        const int my_st = grp & 1;                    // accumulator this group drains
+        constexpr int CPG = (TC_BN / 32) / (TC_GROUPS / 2);   // 32-column chunks per group and tile
+        const int c_first = (grp >> 1) * CPG;         // first chunk of this group's column range
         const int q = warp & 3;                       // TMEM lane quarter this warp may read
         const int row = q * 32 + lane;                // key of this thread inside the item
         long long tb = 0, item_no = 0;
@@ -379,7 +386,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) k_tc_assign(const __grid_consta
             const float m2S = -2.f * sc.x;
             for (int nt = 0; nt < NT; nt++, tb++) {
                 const int st = (int)(tb & 1);
-                if (st != grp) continue;
+                if (st != my_st) continue;
                 if (*s_abort || !tc_mbar_wait(bar(8 + st), (unsigned)((tb >> 1) & 1))) { *s_abort = 1; dead = true; break; }
                 tc_fence_after();
                 float ch[4][3];                                        // four independent chains of three smallest
@@ -396,22 +403,23 @@ __global__ void __launch_bounds__(TC_THREADS, 1) k_tc_assign(const __grid_consta
                         dst[4 * e] = v.x; dst[4 * e + 1] = v.y; dst[4 * e + 2] = v.z; dst[4 * e + 3] = v.w;
                     }
                 };
-                tc_ld32(tbase, acc[0]);
-                load_bias(0, bs[0]);
+                tc_ld32(tbase + c_first * 32, acc[0]);
+                load_bias(c_first, bs[0]);
 #pragma unroll
-                for (int c = 0; c < TC_BN / 32; c++) {
+                for (int cc = 0; cc < CPG; cc++) {
+                    const int c = c_first + cc;
                     tc_ld_wait();                                           // chunk c has arrived
-                    if (c + 1 < TC_BN / 32) {                               // chunk c + 1 and its bias in flight
-                        tc_ld32(tbase + (c + 1) * 32, acc[(c + 1) & 1]);
-                        load_bias(c + 1, bs[(c + 1) & 1]);
+                    if (cc + 1 < CPG) {                                     // chunk c + 1 and its bias in flight
+                        tc_ld32(tbase + (c + 1) * 32, acc[(cc + 1) & 1]);
+                        load_bias(c + 1, bs[(cc + 1) & 1]);
                     }
 #pragma unroll
                     for (int e = 0; e < 32; e += 8) {
 #pragma unroll
                         for (int x = 0; x < 4; x++) {
                             const int e0 = e + 2 * x;
-                            const float x0 = tc_pack(fmaf(__uint_as_float(acc[c & 1][e0]), m2S, bs[c & 1][e0]), c * 32 + e0);
-                            const float x1 = tc_pack(fmaf(__uint_as_float(acc[c & 1][e0 + 1]), m2S, bs[c & 1][e0 + 1]), c * 32 + e0 + 1);
+                            const float x0 = tc_pack(fmaf(__uint_as_float(acc[cc & 1][e0]), m2S, bs[cc & 1][e0]), c * 32 + e0);
+                            const float x1 = tc_pack(fmaf(__uint_as_float(acc[cc & 1][e0 + 1]), m2S, bs[cc & 1][e0 + 1]), c * 32 + e0 + 1);
                             tc_top3_pair(ch[x][0], ch[x][1], ch[x][2], x0, x1);
                         }
                     }
@@ -429,16 +437,21 @@ __global__ void __launch_bounds__(TC_THREADS, 1) k_tc_assign(const __grid_consta
                 tc_insert(g1, j1, g2, j2, g3, t3, nt * TC_BN + (int)(__float_as_uint(t3) & 0xFFu));
             }
             // ---- hand-over: group 1 -> group 0 (slot alternates per item; the barrier orders write, read and reuse)
-            float* slot = xchg + (size_t)(item_no & 1) * TC_BM * 5 + row * 5;
-            if (grp == 1) {
+            float* slots = xchg + (size_t)(item_no & 1) * 3 * TC_BM * 5 + row * 5;     // [3 groups][128 keys][5]
+            if (grp > 0) {
+                float* slot = slots + (size_t)(grp - 1) * TC_BM * 5;
                 slot[0] = g1; slot[1] = g2; slot[2] = g3; slot[3] = __int_as_float(j1); slot[4] = __int_as_float(j2);
             }
-            asm volatile("bar.sync 2, 256;\n" ::: "memory");
+            asm volatile("bar.sync 2, %0;\n" ::"n"(128 * TC_GROUPS) : "memory");
             if (dead || *s_abort) break;
             if (grp == 0) {
-                tc_insert(g1, j1, g2, j2, g3, slot[0], __float_as_int(slot[3]));
-                tc_insert(g1, j1, g2, j2, g3, slot[1], __float_as_int(slot[4]));
-                tc_insert(g1, j1, g2, j2, g3, slot[2], 0);
+#pragma unroll
+                for (int g = 0; g < TC_GROUPS - 1; g++) {
+                    const float* slot = slots + (size_t)g * TC_BM * 5;
+                    tc_insert(g1, j1, g2, j2, g3, slot[0], __float_as_int(slot[3]));
+                    tc_insert(g1, j1, g2, j2, g3, slot[1], __float_as_int(slot[4]));
+                    tc_insert(g1, j1, g2, j2, g3, slot[2], 0);
+                }
             }
             if (grp == 0 && i < p.n) {
                 const size_t gi = (size_t)u * p.n + i;
