@@ -46,6 +46,14 @@ def test_attention_ring_wraps_and_units_cut_by_slices():
     assert rep.status_bits & P.ST_INTERNAL == 0 and min(rep.tokens_selected) > 3000
 
 
+def test_more_than_1024_units_keep_the_work_prefix_in_global_memory():
+    # above 1024 units the attention CTAs read the prefix of the work lists from global memory instead of a
+    # shared-memory copy, and the per-unit kernels run in several waves
+    cfg = CONFIGS[5].scaled(B=1, L=1, n_prefill=96, steps=4, M0=6, max_clusters=16, budget=64, T=2)
+    rep = _run(cfg, [0, 555, 1099], cfg.steps, ctx_units=list(range(1100)), assign_mode=0)
+    assert rep.status_bits & P.ST_INTERNAL == 0
+
+
 def test_plain_attention_kernel_on_bf16():
     cfg = CONFIGS[5].scaled(B=1, L=1, n_prefill=600, steps=16, M0=24, max_clusters=64, budget=200, T=3)
     from parity_harness import make_ctx
