@@ -194,6 +194,5 @@ void launch_split_check(const Tables& t, float gamma, int var_enabled, int min_s
                         long long* launches);
 void launch_append_split(const Tables& t, float gamma, int var_enabled, int min_size, int iters, int do_append, StepPtr k,
                          StepPtr v, int* step_ctr, cudaStream_t s, long long* launches);
-void launch_step_inc(int* ctr, cudaStream_t s, long long* launches);
 
 }  // namespace dkv

@@ -111,8 +111,6 @@ __global__ void __launch_bounds__(256) k_attn_combine(Tables t, StepPtrW outp, i
     }
 }
 
-__global__ void k_step_inc(int* ctr) { *ctr += 1; }
-
 // ------------------------------------------------------------------ launchers
 
 template <typename KV, int HD>
@@ -142,11 +140,6 @@ void launch_gather_attn_v1(const Tables& t, StepPtr q, cudaStream_t s, long long
 void launch_attn_combine(const Tables& t, StepPtrW out, cudaStream_t s, long long* launches) {
     if (t.d == 64) k_attn_combine<64><<<t.U, 256, 0, s>>>(t, out, t.n_splits_attn);
     else k_attn_combine<128><<<t.U, 256, 0, s>>>(t, out, t.n_splits_attn);
-    (*launches)++;
-}
-
-void launch_step_inc(int* ctr, cudaStream_t s, long long* launches) {
-    k_step_inc<<<1, 1, 0, s>>>(ctr);
     (*launches)++;
 }
 
