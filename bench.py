@@ -194,13 +194,19 @@ def run_reference(args, cfg):
         "impl": "reference", "metric": METRIC, "value": value, "unit": "steps/s", "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1000.0 / value, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": f"config{cfg.cfg_id}:{cfg.name}", "units": cfg.U, "context": cfg.n_prefill,
-                   "budget": cfg.budget},
+        "config": config_dict(cfg, args.warmup),
         "cpu_baseline": {"value": value, "unit": "steps/s", "cores": smp.cores, "kind": "oracle",
                          "sample": smp.describe(args.steps, dt)},
         "e2e": {"value": value, "unit": "steps/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }
     print(json.dumps(line), flush=True)
+
+
+def config_dict(cfg, warmup: int) -> dict:
+    """The `config` object of the JSON line, the same for both arms."""
+    return {"workload": f"config{cfg.cfg_id}:{cfg.name}", "units_per_gpu": cfg.U, "layers": cfg.L, "kv_heads": cfg.Hkv,
+            "gqa_group": cfg.G, "head_dim": cfg.d, "context": cfg.n_prefill + warmup, "clusters": cfg.M0, "budget": cfg.budget,
+            "l2": "inputs_larger_than_l2", "loop": "cuda_graph_replay(decode_step,append,split_check)"}
 
 
 def rank_units(cfg, rank: int):
@@ -378,10 +384,7 @@ def run_ours(args, cfg):
             "metric": METRIC, "value": value, "unit": "steps/s", "n_gpus": world, "steps": K_steps, "warmup": W,
             "ms_per_step": ms / K_steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "f32" if cfg.kv_dtype == "f32" else "bf16 KV / f32 math", "data": "synthetic",
-            "config": {"workload": f"config{cfg.cfg_id}:{cfg.name}", "units_per_gpu": U, "layers": cfg.L,
-                       "kv_heads": cfg.Hkv, "gqa_group": cfg.G, "head_dim": cfg.d, "context": cfg.n_prefill + W,
-                       "clusters": cfg.M0, "budget": cfg.budget, "l2": "inputs_larger_than_l2",
-                       "loop": "cuda_graph_replay(decode_step,append,split_check)"},
+            "config": config_dict(cfg, W),
             "e2e": e2e, "gpu_launches": int(gpu_launches), "clocks": clocks, "roofline": roofline,
             "cpu_baseline": cpu_baseline, "build": build,
             "counters": {"splits_in_timed_region": st1["n_splits"] - st0["n_splits"],
