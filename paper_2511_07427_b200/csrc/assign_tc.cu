@@ -8,7 +8,7 @@
 // on the 5th-generation tensor cores (tcgen05.mma, kind::f16, fp32 accumulators in TMEM) with the
 // keys converted to fp16 (exact for |k| in [2^-14, 65504], which a pre-pass checks) and the fp32
 // centres rounded to fp16.  Rounding the centres perturbs every value by at most
-// E_i = 2 ||k_i|| max_j||c_j|| 2^-11 (plus accumulation and packing slack), so the tensor-core
+// E_i = 2 ||k_i|| max_j||c_j|| 2^-11 (plus accumulation and fixed-point slack), so the tensor-core
 // result is used as a FILTER: the epilogue keeps, per key, the three smallest values; when the
 // second is further than 2 E_i from the first, the first is provably the true argmin.  Otherwise
 // the key is re-decided exactly in fp32 with the direct form sum (k - c)^2, the same arithmetic
@@ -458,9 +458,13 @@ __global__ void __launch_bounds__(TC_THREADS, 1) k_tc_assign(const __grid_consta
                 if (j1 >= p.M) j1 = 0;
                 p.assign[gi] = j1;
                 const float kn = p.knorm[gi], cm = __uint_as_float(p.cmax_bits[u]);
-                // bound on |filter value - true value|: fp16 rounding of the centres (2 kn cm 2^-11, with 3 % slack
-                // for the accumulation), the two roundings to the fixed-point grid, sub-normal keys
-                const float E = kn * cm * (1.03f / 1024.f) + 2.f * sc.y + cm * 1e-6f;
+                // Bound on |filter value - true value|, term by term:
+                //   fp16 rounding of the centres: 2 |k.(c - c16)| <= 2 kn cm 2^-11 = kn cm 2^-10;
+                //   fp32 accumulation of 128 exact products in the tensor core, doubled by the factor -2: below
+                //   kn cm 2^-15, covered with margin by the 10 % slack on the first term;
+                //   sub-normal fp16 elements of keys and centres (absolute error 2^-25 each, 128 of them): (kn + cm) 1e-6;
+                //   fp32 rounding of ||c||^2: cm^2 5e-7;  the two roundings to the fixed-point grid: 2 g.
+                const float E = kn * cm * (1.10f / 1024.f) + 2.f * sc.y + (kn + cm) * 1e-6f + cm * cm * 5e-7f;
                 // gaps in value units: mantissa differences times the grid
                 const unsigned m1 = __float_as_uint(g1) >> 8, m2 = __float_as_uint(g2) >> 8, m3 = __float_as_uint(g3) >> 8;
                 const float gap2 = (float)(m2 - m1) * sc.y, gap3 = (float)(m3 - m1) * sc.y;
