@@ -52,3 +52,37 @@ def test_tensor_core_assign_several_centre_tiles():
     rep = _run(cfg, [0, 4], cfg.steps, ctx_units=list(range(5)), assign_mode=0)
     assert rep.status_bits & P.ST_INTERNAL == 0
     assert rep.rechecked < 0.5 * 5 * 4500 * 4      # the filter decides most keys
+
+
+def test_tensor_core_assign_adversarial_keys():
+    """Keys chosen to sit on the filter's weak spots: exact duplicates of other keys (exact ties between the
+    centres initialised from them), midpoints of key pairs, one channel of magnitude ~200, values around the fp16
+    sub-normal range, and all-zero rows.  Every Lloyd round's assignment must still equal the oracle's
+    (ties to the lowest id), i.e. whatever the tensor-core filter cannot prove goes through the exact stage."""
+    import oracle as O
+    import paper_2511_07427_b200 as P
+    from parity_harness import ParityReport, check_state, make_ctx, make_oracle
+    rng = np.random.default_rng(3)
+    n, d, M, T = 1500, 128, 48, 5
+    base = rng.normal(size=(40, d)).astype(np.float32)
+    K = base[rng.integers(0, 40, size=n)] + 0.05 * rng.normal(size=(n, d)).astype(np.float32)
+    K[:200] = K[200:400]                                   # exact duplicates
+    K[400:500] = 0.5 * (K[500:600] + K[600:700])           # midpoints
+    K[:, 7] *= 200.0                                       # one huge channel
+    K[700:800] *= 1e-6                                     # around and below the fp16 sub-normal range
+    K[800:820] = 0.0
+    Kb = torch.tensor(K).to(torch.bfloat16)[None].contiguous()
+    Vb = torch.tensor(rng.normal(size=(1, n, d)).astype(np.float32)).to(torch.bfloat16)
+    cfg = CONFIGS[2].scaled(B=1, L=1, Hkv=1, Hq=4, n_prefill=n, steps=2, M0=M, max_clusters=96, T=T)
+    ctx = make_ctx(cfg, 1, trace=1, assign_mode=0)
+    ctx.build_index(Kb.cuda(), Vb.cuda(), M, 21)
+    picks, trace = ctx.get_build_trace()
+    o = make_oracle(cfg)
+    o.build(Kb[0].double().numpy(), Vb[0].double().numpy(), M, T, 21, unit_index=0, init_mode=O.INIT_RANDOM,
+            hint_assign=trace[:, 0, :])
+    assert o.violations == 0
+    check_state(o, ctx.export_state(), 0, ParityReport(), "adversarial build")
+    st = ctx.get_status()
+    assert st["error_bits"] & P.ST_INTERNAL == 0 and st["assign_rechecked"] > 0
+    print(f"\n[adversarial] ties followed {o.ties}, re-decided exactly {st['assign_rechecked']} of {n * T}")
+    ctx.destroy()
