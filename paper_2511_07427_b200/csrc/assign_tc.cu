@@ -20,9 +20,9 @@
 // Warp 0 issues TMA tensor loads (128-byte swizzle, no multicast) of the key block (kept for
 // all centre tiles of the item) and of 256-centre tiles into a two-stage ring; warp 1 issues
 // tcgen05.mma (M=128, N=256, K=16, eight per tile) into one of two 256-column TMEM accumulators
-// and commits to an mbarrier; warps 2-9 drain the accumulators with tcgen05.ld, one key per
-// thread (two groups of four warps, one per accumulator).  Every wait is bounded; on expiry the kernel sets a status bit, frees its TMEM and
-// returns.
+// and commits to an mbarrier; warps 2-17 drain the accumulators with tcgen05.ld, one key per
+// thread (four groups of four warps: two per accumulator, half of its columns each).  Every wait
+// is bounded; on expiry the kernel sets a status bit, frees its TMEM and returns.
 #include <cuda.h>
 #include <float.h>
 
@@ -363,12 +363,13 @@ __global__ void __launch_bounds__(TC_THREADS, 1) k_tc_assign(const __grid_consta
             }
         }
     } else {
-        // =============================== accumulator drain (warps 2..9) ===============================
-        // Two groups of four warps; group g drains accumulator g, i.e. the tiles whose running number is g mod 2,
-        // so both accumulators are drained at the same time while the next MMAs run.  One key per thread and
-        // group.  Per tile the thread keeps the three smallest packed values (low 8 bits = column) in two
-        // independent chains and merges them into its best two (with indices) and third value; at the end of an
-        // item group 1 hands its triple to group 0 through shared memory, and group 0 decides.
+        // =============================== accumulator drain (warps 2 and up) ===============================
+        // Groups of four warps (one warp per TMEM lane quarter).  Group g drains accumulator g mod 2, i.e. the
+        // tiles whose running number is g mod 2, and of those the column range g / 2, so both accumulators are
+        // drained at the same time while the next MMAs run.  One key per thread and group.  Per tile the thread
+        // keeps the three smallest fixed-point words (low 8 bits = column) in four independent chains and merges
+        // them into its best two (with indices) and third value; at the end of an item the other groups hand
+        // their triples to group 0 through shared memory, and group 0 decides.
         const int grp = (warp - 2) >> 2;              // drain group
         const int my_st = grp & 1;                    // accumulator this group drains
         constexpr int CPG = (TC_BN / 32) / (TC_GROUPS / 2);   // 32-column chunks per group and tile
