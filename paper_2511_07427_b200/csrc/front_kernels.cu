@@ -21,7 +21,10 @@ __device__ __forceinline__ unsigned int ord_key(float f) {
 // ------------------------------------------------------------------ k_front
 
 constexpr int FR_THREADS = 256;
-constexpr int FR_ROWS = 128;      // representatives per block
+#ifndef DKV_FR_ROWS
+#define DKV_FR_ROWS 128
+#endif
+constexpr int FR_ROWS = DKV_FR_ROWS;      // representatives per block (a multiple of 32)
 
 // Grid (ceil(max_clusters / FR_ROWS), U).  Eight lanes share one representative row (each
 // lane reads HD/8 floats as float4s), four rows per warp instruction.
