@@ -259,6 +259,7 @@ extern "C" int dynakv_build_index(dynakv_ctx* c, const void* K, const void* V, i
     c->allocs.resize(mark);
     for (void* p : keep) c->allocs.push_back(p);
     c->built = true; c->n_prefill = n; c->M0 = M;
+    t.M_floor = M;
     return DYNAKV_OK;
 }
 

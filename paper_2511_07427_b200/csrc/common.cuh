@@ -26,6 +26,7 @@ constexpr int FLAG_HOLD = 1;        // split abandoned; not retried until the ne
 struct Tables {
     int U, G, d, kv_dtype, max_tokens, max_clusters, P, n_splits_attn;
     int W;                           // work-list capacity per unit (entries)
+    int M_floor;                     // clusters every unit has had since the build (ids never go away); 0 before it
     void* kpages; void* vpages;
     int* page_tok;                   // [U][P][PAGE] token id per slot
     int* page_next;                  // [U][P]

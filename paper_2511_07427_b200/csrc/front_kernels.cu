@@ -27,48 +27,29 @@ constexpr int FR_THREADS = 256;
 constexpr int FR_ROWS = DKV_FR_ROWS;      // representatives per block (a multiple of 32)
 
 // Grid (ceil(max_clusters / FR_ROWS), U).  Eight lanes share one representative row (each
-// lane reads HD/8 floats as float4s), four rows per warp instruction.
+// lane reads HD/8 floats as float4s), four rows per warp instruction.  Every global load of a
+// thread -- its rows, their cluster sizes, its share of the query heads, the new key -- is issued
+// before the first use of any of them, so a block pays one memory latency, not a chain of them.
 template <typename KV, int HD>
-__global__ void __launch_bounds__(FR_THREADS) k_front(Tables t, StepPtr qp, StepPtr kp, int has_q, int has_k) {
+__global__ void __launch_bounds__(FR_THREADS, 2) k_front(Tables t, StepPtr qp, StepPtr kp, int has_q, int has_k) {
     constexpr int V4 = HD / 32;   // float4 loads per lane per row
+    constexpr int NIT = FR_ROWS / ((FR_THREADS / 32) * 4);
     const int u = blockIdx.y;
-    pdl_wait();                          // inside a captured loop the representatives come from the iteration before
-    const int Mcur = t.u_M[u];
     const int j0 = blockIdx.x * FR_ROWS;
-    if (j0 >= Mcur) { pdl_trigger(); return; }
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int sub = lane >> 3, l8 = lane & 7;
-    float qs[V4][4], kk[V4][4];
-#pragma unroll
-    for (int i = 0; i < V4; i++)
-#pragma unroll
-        for (int e = 0; e < 4; e++) { qs[i][e] = 0.f; kk[i][e] = 0.f; }
-    if (has_q) {
-        const float* q = reinterpret_cast<const float*>(qp.get()) + (size_t)u * t.G * HD;
-        for (int g = 0; g < t.G; g++)
-#pragma unroll
-            for (int i = 0; i < V4; i++) {
-                const float4 v = *reinterpret_cast<const float4*>(q + g * HD + l8 * 4 + 32 * i);
-                qs[i][0] += v.x; qs[i][1] += v.y; qs[i][2] += v.z; qs[i][3] += v.w;
-            }
+    pdl_wait();                          // inside a captured loop the representatives come from the iteration before
+    // A unit never has fewer clusters than the build gave it: blocks wholly below that count need not
+    // wait for the unit's current count before they issue their row loads.
+    int jend = j0 + FR_ROWS;
+    if (jend > t.M_floor) {
+        const int Mcur = t.u_M[u];
+        if (j0 >= Mcur) { pdl_trigger(); return; }
+        jend = min(Mcur, jend);
     }
-    if (has_k) {
-        const KV* k = reinterpret_cast<const KV*>(kp.get()) + (size_t)u * HD;
-#pragma unroll
-        for (int i = 0; i < V4; i++) {
-            const float4 v = ld4(k, l8 * 4 + 32 * i);
-            kk[i][0] = v.x; kk[i][1] = v.y; kk[i][2] = v.z; kk[i][3] = v.w;
-        }
-    }
-    const float invG = 1.0f / (float)t.G;
     const float* R = t.cl_r + (size_t)u * t.max_clusters * HD;
     const int* CN = t.cl_n + (size_t)u * t.max_clusters;
-    float* SC = t.scores + (size_t)u * t.max_clusters;
-    float* DS = t.dists + (size_t)u * t.max_clusters;
-    const int jend = min(Mcur, j0 + FR_ROWS);
-    // all row loads of the thread are issued before any arithmetic (rows of dead clusters are read too and
-    // masked afterwards, so no load waits for the cluster-size load)
-    constexpr int NIT = FR_ROWS / ((FR_THREADS / 32) * 4);
+    // rows of dead clusters are read too and masked afterwards, so no load waits for the cluster-size load
     float4 rv[NIT][V4];
     int cn[NIT];
 #pragma unroll
@@ -80,6 +61,48 @@ __global__ void __launch_bounds__(FR_THREADS) k_front(Tables t, StepPtr qp, Step
         for (int i = 0; i < V4; i++)
             rv[it][i] = in ? __ldcs(reinterpret_cast<const float4*>(R + (size_t)j * HD + l8 * 4 + 32 * i)) : make_float4(0.f, 0.f, 0.f, 0.f);
     }
+    // sum of the unit's query heads: the four row groups of a warp take heads sub and sub + 4 and
+    // exchange their partial sums, so a thread loads G/4 heads instead of G
+    float qs[V4][4], kk[V4][4];
+#pragma unroll
+    for (int i = 0; i < V4; i++)
+#pragma unroll
+        for (int e = 0; e < 4; e++) { qs[i][e] = 0.f; kk[i][e] = 0.f; }
+    if (has_q) {
+        const float* q = reinterpret_cast<const float*>(qp.get()) + (size_t)u * t.G * HD;
+        static_assert(MAX_G <= 8, "two heads per row group");
+#pragma unroll
+        for (int h = 0; h < 2; h++) {
+            const int g = sub + 4 * h;
+            if (g < t.G) {
+#pragma unroll
+                for (int i = 0; i < V4; i++) {
+                    const float4 v = *reinterpret_cast<const float4*>(q + g * HD + l8 * 4 + 32 * i);
+                    qs[i][0] += v.x; qs[i][1] += v.y; qs[i][2] += v.z; qs[i][3] += v.w;
+                }
+            }
+        }
+    }
+    if (has_k) {
+        const KV* k = reinterpret_cast<const KV*>(kp.get()) + (size_t)u * HD;
+#pragma unroll
+        for (int i = 0; i < V4; i++) {
+            const float4 v = ld4(k, l8 * 4 + 32 * i);
+            kk[i][0] = v.x; kk[i][1] = v.y; kk[i][2] = v.z; kk[i][3] = v.w;
+        }
+    }
+    if (has_q) {
+#pragma unroll
+        for (int i = 0; i < V4; i++)
+#pragma unroll
+            for (int e = 0; e < 4; e++) {
+                qs[i][e] += __shfl_xor_sync(0xffffffffu, qs[i][e], 8);
+                qs[i][e] += __shfl_xor_sync(0xffffffffu, qs[i][e], 16);
+            }
+    }
+    const float invG = 1.0f / (float)t.G;
+    float* SC = t.scores + (size_t)u * t.max_clusters;
+    float* DS = t.dists + (size_t)u * t.max_clusters;
 #pragma unroll
     for (int it = 0; it < NIT; it++) {
         const int j = j0 + warp * 4 + sub + it * (FR_THREADS / 32) * 4;
