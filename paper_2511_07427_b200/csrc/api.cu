@@ -34,7 +34,8 @@ struct dynakv_ctx {
     int* trace_assign = nullptr;   // [T][U][n]
     int* trace_picks = nullptr;    // [U][M0]
     // graph loop
-    int* step_ctr = nullptr;
+    int* step_ctr = nullptr;          // device: step index of the captured loop
+    int* step_lim = nullptr;          // device: number of steps of the loop in flight
     cudaGraphExec_t graph_exec = nullptr, graph_exec_long = nullptr;   // one iteration / eight iterations
     const void* g_q = nullptr; const void* g_k = nullptr; const void* g_v = nullptr; void* g_out = nullptr;
     int g_budget = -1;
@@ -187,6 +188,7 @@ extern "C" int dynakv_create(const dynakv_config* cfg, void* cuda_stream, dynakv
     ALLOC(t.status, 1, true);
     ALLOC(t.counters, 8, true);
     ALLOC(c->step_ctr, 1, true);
+    ALLOC(c->step_lim, 1, true);
     ALLOC(c->st_q, U * t.G * d, false);
     ALLOC(c->st_out, U * t.G * d, false);
     {
@@ -286,16 +288,29 @@ static void enqueue_append_apply(dynakv_ctx* c, StepPtr k, StepPtr v, bool timed
     launch_append_apply(c->t, k, v, c->stream, &c->launches);
 }
 
+static const NextFront kNoNextFront = {0, StepPtr{nullptr, 0, nullptr}, StepPtr{nullptr, 0, nullptr}, nullptr};
+
 // One whole loop iteration in four launches: a single centroid pass serves both the query scores and the new
-// key's distances; selection; gather-attention with its combine; then append + split check in one kernel
-// (which also advances the device-side step index when the iteration belongs to a captured loop).
-static void enqueue_step(dynakv_ctx* c, StepPtr q, StepPtr k, StepPtr v, int budget, StepPtrW out, int* step_ctr, bool timed) {
+// key's distances; selection; gather-attention with its combine; then append + split check in one kernel.
+static void enqueue_step(dynakv_ctx* c, StepPtr q, StepPtr k, StepPtr v, int budget, StepPtrW out, bool timed) {
     enqueue_front(c, q, k, 1, 1, timed);
     enqueue_retrieve(c, q, budget, out, nullptr, timed);
     TimeScope ts(c, KC_SPLIT, timed);
     launch_append_split(c->t, c->cfg.split_size_factor, c->cfg.split_var_factor > 0.f ? 1 : 0, c->cfg.split_min_size,
-                        c->cfg.split_iters, 1, k, v, step_ctr, c->stream, &c->launches);
+                        c->cfg.split_iters, 1, k, v, nullptr, kNoNextFront, c->stream, &c->launches);
 }
+
+// One iteration of a captured loop in three launches.  The centroid pass of step t + 1 is part of the tail kernel
+// of step t (every unit's block runs it as soon as the unit's own append is done), so an iteration starts at the
+// selection; the pass of step 0 is launched once ahead of the loop.  The tail kernel's last block advances the
+// device-side step index that all kernels of the loop read.
+static void enqueue_loop_iteration(dynakv_ctx* c, StepPtr q, StepPtr k, StepPtr v, int budget, StepPtrW out) {
+    enqueue_retrieve(c, q, budget, out, nullptr, false);
+    launch_append_split(c->t, c->cfg.split_size_factor, c->cfg.split_var_factor > 0.f ? 1 : 0, c->cfg.split_min_size,
+                        c->cfg.split_iters, 1, k, v, c->step_ctr, NextFront{1, q, k, c->step_lim}, c->stream, &c->launches);
+}
+
+__global__ void k_loop_begin(int* step_ctr, int* step_lim, int n_steps) { *step_ctr = 0; *step_lim = n_steps; }
 
 extern "C" int dynakv_decode_step(dynakv_ctx* c, const float* q, int32_t token_budget, float* out, int32_t* selected_ids) {
     if (!c || !q || !out || token_budget < 0) return DYNAKV_ERR_ARG;
@@ -331,7 +346,7 @@ extern "C" int dynakv_split_check(dynakv_ctx* c) {
 
 extern "C" int dynakv_decode_loop(dynakv_ctx* c, const float* q_steps, const void* k_steps, const void* v_steps,
                                   int64_t n_steps, int32_t token_budget, float* out_steps) {
-    if (!c || !q_steps || !k_steps || !v_steps || !out_steps || n_steps < 0 || token_budget < 0) return DYNAKV_ERR_ARG;
+    if (!c || !q_steps || !k_steps || !v_steps || !out_steps || n_steps < 0 || n_steps > 0x7fffffff || token_budget < 0) return DYNAKV_ERR_ARG;
     if (!c->built) return DYNAKV_ERR_STATE;
     if (c->stream == nullptr || c->stream == cudaStreamLegacy) {
         snprintf(g_err, sizeof(g_err), "dynakv_decode_loop captures a CUDA graph and needs a context created on a non-default stream");
@@ -350,8 +365,8 @@ extern "C" int dynakv_decode_loop(dynakv_ctx* c, const float* q_steps, const voi
             long long before = c->launches;
             CK(cudaStreamBeginCapture(c->stream, cudaStreamCaptureModeThreadLocal));
             for (int r = 0; r < reps; r++)
-                enqueue_step(c, StepPtr{q_steps, qs, c->step_ctr}, StepPtr{k_steps, ks, c->step_ctr},
-                             StepPtr{v_steps, ks, c->step_ctr}, token_budget, StepPtrW{out_steps, qs, c->step_ctr}, c->step_ctr, false);
+                enqueue_loop_iteration(c, StepPtr{q_steps, qs, c->step_ctr}, StepPtr{k_steps, ks, c->step_ctr},
+                                       StepPtr{v_steps, ks, c->step_ctr}, token_budget, StepPtrW{out_steps, qs, c->step_ctr});
             cudaError_t e = cudaStreamEndCapture(c->stream, &graph);
             if (which == 0) c->graph_nodes = c->launches - before;
             c->launches = before;
@@ -370,7 +385,14 @@ extern "C" int dynakv_decode_loop(dynakv_ctx* c, const float* q_steps, const voi
         }
         c->g_q = q_steps; c->g_k = k_steps; c->g_v = v_steps; c->g_out = out_steps; c->g_budget = token_budget;
     }
-    CK(cudaMemsetAsync(c->step_ctr, 0, sizeof(int), c->stream));
+    if (n_steps == 0) return DYNAKV_OK;
+    {
+        const long long qs = (long long)t.U * t.G * t.d * 4, ks = (long long)t.U * t.d * (long long)kv_bytes(c->cfg);
+        k_loop_begin<<<1, 1, 0, c->stream>>>(c->step_ctr, c->step_lim, (int)n_steps);
+        c->launches++;
+        // step 0's centroid pass; every later one rides in the tail kernel of the step before it
+        enqueue_front(c, StepPtr{q_steps, qs, c->step_ctr}, StepPtr{k_steps, ks, c->step_ctr}, 1, 1, false);
+    }
     int64_t s = 0;
     for (; s + UNROLL <= n_steps; s += UNROLL) CK(cudaGraphLaunch(c->graph_exec_long, c->stream));
     for (; s < n_steps; s++) CK(cudaGraphLaunch(c->graph_exec, c->stream));
@@ -388,7 +410,7 @@ extern "C" int dynakv_step_host(dynakv_ctx* c, const float* q_host, const void* 
     CK(cudaMemcpyAsync(c->st_k, k_host, kb, cudaMemcpyHostToDevice, c->stream));
     CK(cudaMemcpyAsync(c->st_v, v_host, kb, cudaMemcpyHostToDevice, c->stream));
     enqueue_step(c, StepPtr{c->st_q, 0, nullptr}, StepPtr{c->st_k, 0, nullptr}, StepPtr{c->st_v, 0, nullptr},
-                 token_budget, StepPtrW{c->st_out, 0, nullptr}, nullptr, true);
+                 token_budget, StepPtrW{c->st_out, 0, nullptr}, true);
     CK(cudaMemcpyAsync(out_host, c->st_out, qb, cudaMemcpyDeviceToHost, c->stream));
     CK(cudaStreamSynchronize(c->stream));
     return DYNAKV_OK;

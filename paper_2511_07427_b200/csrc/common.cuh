@@ -72,6 +72,8 @@ struct StepPtr {
         long long t = ctr ? (long long)(*ctr) : 0;
         return (const char*)base + t * stride_bytes;
     }
+    // the operand of step `step`, whatever the step index says
+    __device__ __forceinline__ const void* at(long long step) const { return (const char*)base + step * stride_bytes; }
 };
 struct StepPtrW {
     void* base;
@@ -193,7 +195,13 @@ void launch_gather_attn_v1(const Tables& t, StepPtr q, cudaStream_t s, long long
 void launch_attn_combine(const Tables& t, StepPtrW out, cudaStream_t s, long long* launches);
 void launch_split_check(const Tables& t, float gamma, int var_enabled, int min_size, int iters, cudaStream_t s,
                         long long* launches);
+// Operands of the next step's centroid pass when it is fused into the tail of a loop iteration.
+struct NextFront {
+    int on;                  // 0: no fused pass
+    StepPtr q, k;            // per-step query and key arrays (indexed with step + 1)
+    const int* step_lim;     // device: number of steps of the loop; the pass is skipped when step + 1 reaches it
+};
 void launch_append_split(const Tables& t, float gamma, int var_enabled, int min_size, int iters, int do_append, StepPtr k,
-                         StepPtr v, int* step_ctr, cudaStream_t s, long long* launches);
+                         StepPtr v, int* step_ctr, const NextFront& nf, cudaStream_t s, long long* launches);
 
 }  // namespace dkv

@@ -10,6 +10,7 @@
 
 #include "append_block.cuh"
 #include "common.cuh"
+#include "front_rows.cuh"
 
 namespace dkv {
 
@@ -61,45 +62,15 @@ __global__ void __launch_bounds__(FR_THREADS, 2) k_front(Tables t, StepPtr qp, S
         for (int i = 0; i < V4; i++)
             rv[it][i] = in ? __ldcs(reinterpret_cast<const float4*>(R + (size_t)j * HD + l8 * 4 + 32 * i)) : make_float4(0.f, 0.f, 0.f, 0.f);
     }
-    // sum of the unit's query heads: the four row groups of a warp take heads sub and sub + 4 and
-    // exchange their partial sums, so a thread loads G/4 heads instead of G
+    // the unit's query heads (summed) and the new key, as this lane's share of a row
     float qs[V4][4], kk[V4][4];
 #pragma unroll
     for (int i = 0; i < V4; i++)
 #pragma unroll
         for (int e = 0; e < 4; e++) { qs[i][e] = 0.f; kk[i][e] = 0.f; }
-    if (has_q) {
-        const float* q = reinterpret_cast<const float*>(qp.get()) + (size_t)u * t.G * HD;
-        static_assert(MAX_G <= 8, "two heads per row group");
-#pragma unroll
-        for (int h = 0; h < 2; h++) {
-            const int g = sub + 4 * h;
-            if (g < t.G) {
-#pragma unroll
-                for (int i = 0; i < V4; i++) {
-                    const float4 v = *reinterpret_cast<const float4*>(q + g * HD + l8 * 4 + 32 * i);
-                    qs[i][0] += v.x; qs[i][1] += v.y; qs[i][2] += v.z; qs[i][3] += v.w;
-                }
-            }
-        }
-    }
-    if (has_k) {
-        const KV* k = reinterpret_cast<const KV*>(kp.get()) + (size_t)u * HD;
-#pragma unroll
-        for (int i = 0; i < V4; i++) {
-            const float4 v = ld4(k, l8 * 4 + 32 * i);
-            kk[i][0] = v.x; kk[i][1] = v.y; kk[i][2] = v.z; kk[i][3] = v.w;
-        }
-    }
-    if (has_q) {
-#pragma unroll
-        for (int i = 0; i < V4; i++)
-#pragma unroll
-            for (int e = 0; e < 4; e++) {
-                qs[i][e] += __shfl_xor_sync(0xffffffffu, qs[i][e], 8);
-                qs[i][e] += __shfl_xor_sync(0xffffffffu, qs[i][e], 16);
-            }
-    }
+    if (has_q) front_qsum_load<HD>(reinterpret_cast<const float*>(qp.get()) + (size_t)u * t.G * HD, t.G, lane, qs);
+    if (has_k) front_key_load<KV, HD>(reinterpret_cast<const KV*>(kp.get()) + (size_t)u * HD, lane, kk);
+    if (has_q) front_qsum_finish<HD>(qs);
     const float invG = 1.0f / (float)t.G;
     float* SC = t.scores + (size_t)u * t.max_clusters;
     float* DS = t.dists + (size_t)u * t.max_clusters;
@@ -108,16 +79,8 @@ __global__ void __launch_bounds__(FR_THREADS, 2) k_front(Tables t, StepPtr qp, S
         const int j = j0 + warp * 4 + sub + it * (FR_THREADS / 32) * 4;
         const bool in = j < jend;
         const bool live = in && cn[it] > 0;
-        float s = 0.f, dd = 0.f;
-#pragma unroll
-        for (int i = 0; i < V4; i++) {
-            const float4 r4 = rv[it][i];
-            s = fmaf(qs[i][0], r4.x, s); s = fmaf(qs[i][1], r4.y, s); s = fmaf(qs[i][2], r4.z, s); s = fmaf(qs[i][3], r4.w, s);
-            float a = kk[i][0] - r4.x, b = kk[i][1] - r4.y, c = kk[i][2] - r4.z, e = kk[i][3] - r4.w;
-            dd = fmaf(a, a, dd); dd = fmaf(b, b, dd); dd = fmaf(c, c, dd); dd = fmaf(e, e, dd);
-        }
-#pragma unroll
-        for (int o = 4; o > 0; o >>= 1) { s += __shfl_xor_sync(0xffffffffu, s, o); dd += __shfl_xor_sync(0xffffffffu, dd, o); }
+        float s, dd;
+        front_row<HD>(rv[it], qs, kk, s, dd);
         if (in && l8 == 0) {
             if (has_q) SC[j] = live ? s * invG : -INFINITY;
             if (has_k) DS[j] = live ? dd : INFINITY;

@@ -8,6 +8,7 @@
 
 #include "append_block.cuh"
 #include "common.cuh"
+#include "front_unit.cuh"
 
 namespace dkv {
 
@@ -15,11 +16,28 @@ constexpr int SP_THREADS = 512;
 constexpr int SP_CACHE_BYTES = 32 * 1024;      // member keys of the cluster being split are staged here when they fit
 constexpr int SP_WARPS = SP_THREADS / 32;
 
+// Dynamic shared memory, in order: chain[maxch], newpg[maxch], trig[max_clusters] (ints); the staged member
+// keys (SP_CACHE_BYTES, 16-byte aligned; also stage 0 of the fused centroid pass) and their token ids; stage 1
+// of the fused centroid pass; one live flag per cluster id.
+template <int HD, int KVB> struct SplitSmem {
+    static constexpr int cache_rows = SP_CACHE_BYTES / (HD * KVB);
+    static constexpr int stage_bytes = FrontUnit<SP_THREADS, HD>::STAGE_BYTES;
+    static_assert(stage_bytes <= SP_CACHE_BYTES, "stage 0 of the centroid pass lives in the staging area");
+    __host__ __device__ static size_t keys_off(int maxch, int max_clusters) { return (((size_t)(2 * maxch + max_clusters) * sizeof(int)) + 127) & ~(size_t)127; }
+    __host__ __device__ static size_t stage1_off(int maxch, int max_clusters) {
+        return (keys_off(maxch, max_clusters) + SP_CACHE_BYTES + (size_t)cache_rows * sizeof(int) + 127) & ~(size_t)127;
+    }
+    __host__ __device__ static size_t live_off(int maxch, int max_clusters) { return stage1_off(maxch, max_clusters) + stage_bytes; }
+    __host__ __device__ static size_t total(int maxch, int max_clusters) { return live_off(maxch, max_clusters) + (size_t)max_clusters + 16; }
+};
+
 template <typename KV, int HD>
 __global__ void __launch_bounds__(SP_THREADS) k_split_check(Tables t, float gamma, int var_enabled, int min_size, int iters,
-                                                            int do_append, StepPtr app_k, StepPtr app_v, int* step_ctr) {
+                                                            int do_append, StepPtr app_k, StepPtr app_v, int* step_ctr,
+                                                            int do_front, StepPtr next_q, StepPtr next_k, const int* step_lim) {
     constexpr int EPL = HD / 32;
-    extern __shared__ int dyn[];
+    extern __shared__ __align__(128) int dyn[];
+    __shared__ unsigned long long fr_bars[2];
     const int maxch = t.max_tokens / PAGE + 2;
     int* chain = dyn;                 // pages of the cluster being split, in chain order
     int* newpg = dyn + maxch;         // pages allocated for the moving child
@@ -32,6 +50,12 @@ __global__ void __launch_bounds__(SP_THREADS) k_split_check(Tables t, float gamm
     __shared__ int s_a, s_ok;
 
     const int u = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    // the step this iteration belongs to: read once, before the last block of the iteration can advance it
+    const int t0 = step_ctr ? *step_ctr : 0;
+    if (do_front && tid == 0) {
+        mbar_init(smem_u32(&fr_bars[0]), 1); mbar_init(smem_u32(&fr_bars[1]), 1);
+        asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
+    }
     // fused loop iteration: the step's append for this unit comes first (Algorithm 1's order)
     if (do_append) { append_block<KV, HD>(t, u, app_k, app_v); __syncthreads(); }
     const int N = t.u_N[u], M0 = t.u_M[u], Mlive0 = t.u_Mlive[u];
@@ -54,9 +78,10 @@ __global__ void __launch_bounds__(SP_THREADS) k_split_check(Tables t, float gamm
     int* trig = dyn + 2 * maxch;
     // staged copy of the member keys (and their token ids) when the cluster fits: every pass below then
     // reads shared memory instead of walking the pages again
-    constexpr int CACHE_ROWS = SP_CACHE_BYTES / (HD * (int)sizeof(KV));
-    KV* krows = reinterpret_cast<KV*>(reinterpret_cast<unsigned char*>(dyn) +
-                                      (((size_t)(2 * maxch + t.max_clusters) * sizeof(int) + 15) & ~(size_t)15));
+    using Lay = SplitSmem<HD, (int)sizeof(KV)>;
+    constexpr int CACHE_ROWS = Lay::cache_rows;
+    unsigned char* dynb = reinterpret_cast<unsigned char*>(dyn);
+    KV* krows = reinterpret_cast<KV*>(dynb + Lay::keys_off(maxch, t.max_clusters));
     int* tok_s = reinterpret_cast<int*>(krows + (size_t)CACHE_ROWS * HD);
     __shared__ int s_ntrig, s_nsplit;
     if (tid == 0) { s_ntrig = 0; s_nsplit = 0; }
@@ -87,8 +112,20 @@ __global__ void __launch_bounds__(SP_THREADS) k_split_check(Tables t, float gamm
         __syncthreads();
     }
     const int ntrig = s_ntrig;
+    // ---- fused loop iteration: the unit's centroid pass for the NEXT step (its query scores and its new key's
+    // distances) on the state after this step's append.  It needs nothing from the gather-attention kernel that
+    // may still be running, and nothing from other units; a split below patches the two rows it changes.
+    const bool fronted = do_front && (t0 + 1 < *step_lim);
+    const float* q1 = nullptr; const KV* k1 = nullptr;
+    if (fronted) {
+        q1 = reinterpret_cast<const float*>(next_q.at(t0 + 1)) + (size_t)u * t.G * HD;
+        k1 = reinterpret_cast<const KV*>(next_k.at(t0 + 1)) + (size_t)u * HD;
+        front_unit<KV, HD, SP_THREADS>(t, u, q1, k1, reinterpret_cast<unsigned char*>(krows), dynb + Lay::stage1_off(maxch, t.max_clusters),
+                                       fr_bars, dynb + Lay::live_off(maxch, t.max_clusters));
+    }
     // Everything above reads and writes only what the gather-attention kernel before this one never touches
-    // (statistics, the new row beyond every listed row); the splits below move rows, so they wait for it.
+    // (statistics, the new row beyond every listed row, next step's scores); the splits below move rows, so
+    // they wait for it.
     if (ntrig > 0) pdl_wait();
     for (int li = 0; li < ntrig; li++) {
         const int j = trig[li];
@@ -359,6 +396,8 @@ __global__ void __launch_bounds__(SP_THREADS) k_split_check(Tables t, float gamm
             }
             __syncthreads();
         }
+        // next step's scores and distances of the two children
+        if (fronted && warp == 0) front_patch<KV, HD>(t, u, q1, k1, j, new_id);
     }
     __syncthreads();
     // No block leaves before the kernel ahead has completed: the next kernel on the stream (the next iteration's
@@ -376,30 +415,31 @@ __global__ void __launch_bounds__(SP_THREADS) k_split_check(Tables t, float gamm
 
 template <typename KV, int HD>
 static void split_t(const Tables& t, float gamma, int var_enabled, int min_size, int iters, int do_append, StepPtr k, StepPtr v,
-                    int* step_ctr, cudaStream_t s) {
-    size_t dyn = sizeof(int) * (2 * (size_t)(t.max_tokens / PAGE + 2) + (size_t)t.max_clusters);
-    dyn = ((dyn + 15) & ~(size_t)15) + SP_CACHE_BYTES + sizeof(int) * (SP_CACHE_BYTES / (HD * sizeof(KV))) + 16;
+                    int* step_ctr, const NextFront& nf, cudaStream_t s) {
+    const size_t dyn = SplitSmem<HD, (int)sizeof(KV)>::total(t.max_tokens / PAGE + 2, t.max_clusters);
     if (dyn > 32 * 1024)
         cudaFuncSetAttribute(k_split_check<KV, HD>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn);
-    launch_pdl(k_split_check<KV, HD>, dim3(t.U), dim3(SP_THREADS), dyn, s, t, gamma, var_enabled, min_size, iters, do_append, k, v, step_ctr);
+    launch_pdl(k_split_check<KV, HD>, dim3(t.U), dim3(SP_THREADS), dyn, s, t, gamma, var_enabled, min_size, iters, do_append, k, v, step_ctr,
+               nf.on, nf.q, nf.k, nf.step_lim);
 }
 
 void launch_split_check(const Tables& t, float gamma, int var_enabled, int min_size, int iters, cudaStream_t s,
                         long long* launches) {
-    launch_append_split(t, gamma, var_enabled, min_size, iters, 0, StepPtr{nullptr, 0, nullptr}, StepPtr{nullptr, 0, nullptr}, nullptr, s,
-                        launches);
+    launch_append_split(t, gamma, var_enabled, min_size, iters, 0, StepPtr{nullptr, 0, nullptr}, StepPtr{nullptr, 0, nullptr}, nullptr,
+                        NextFront{0, StepPtr{nullptr, 0, nullptr}, StepPtr{nullptr, 0, nullptr}, nullptr}, s, launches);
 }
 
-// The tail of a fused loop iteration in one launch: append (when do_append), split check, and, when step_ctr is
-// given, the increment of the device-side step index by the last block to finish.
+// The tail of a fused loop iteration in one launch: append (when do_append), the next step's centroid pass (when
+// nf.on and the next step exists), split check, and, when step_ctr is given, the increment of the device-side
+// step index by the last block to finish.
 void launch_append_split(const Tables& t, float gamma, int var_enabled, int min_size, int iters, int do_append, StepPtr k,
-                         StepPtr v, int* step_ctr, cudaStream_t s, long long* launches) {
+                         StepPtr v, int* step_ctr, const NextFront& nf, cudaStream_t s, long long* launches) {
     if (t.kv_dtype == DYNAKV_F32) {
-        if (t.d == 64) split_t<float, 64>(t, gamma, var_enabled, min_size, iters, do_append, k, v, step_ctr, s);
-        else split_t<float, 128>(t, gamma, var_enabled, min_size, iters, do_append, k, v, step_ctr, s);
+        if (t.d == 64) split_t<float, 64>(t, gamma, var_enabled, min_size, iters, do_append, k, v, step_ctr, nf, s);
+        else split_t<float, 128>(t, gamma, var_enabled, min_size, iters, do_append, k, v, step_ctr, nf, s);
     } else {
-        if (t.d == 64) split_t<__nv_bfloat16, 64>(t, gamma, var_enabled, min_size, iters, do_append, k, v, step_ctr, s);
-        else split_t<__nv_bfloat16, 128>(t, gamma, var_enabled, min_size, iters, do_append, k, v, step_ctr, s);
+        if (t.d == 64) split_t<__nv_bfloat16, 64>(t, gamma, var_enabled, min_size, iters, do_append, k, v, step_ctr, nf, s);
+        else split_t<__nv_bfloat16, 128>(t, gamma, var_enabled, min_size, iters, do_append, k, v, step_ctr, nf, s);
     }
     (*launches)++;
 }
