@@ -178,6 +178,11 @@ extern "C" int dynakv_create(const dynakv_config* cfg, void* cuda_stream, dynakv
     ALLOC(t.work_prefix, U + 1, true);
     ALLOC(t.unit_arrive, U, true);
     ALLOC(t.plan_counter, 2, true);
+    ALLOC(t.tail_sync, 4, true);
+    ALLOC(t.tail_queue, U, true);
+    ALLOC(t.front_done, U, true);
+    ALLOC(t.trig_n, U, true);
+    ALLOC(t.trig_list, U * Mx, false);
     if (cfg->kv_dtype == DYNAKV_BF16 && attn_tma_prepare(t) != 0) {
         snprintf(g_err, sizeof(g_err), "cannot reserve shared memory for the gather-attention kernel: %s", cudaGetErrorString(cudaGetLastError()));
         dynakv_destroy(c);
@@ -310,7 +315,12 @@ static void enqueue_loop_iteration(dynakv_ctx* c, StepPtr q, StepPtr k, StepPtr 
                         c->cfg.split_iters, 1, k, v, c->step_ctr, NextFront{1, q, k, c->step_lim}, c->stream, &c->launches);
 }
 
-__global__ void k_loop_begin(int* step_ctr, int* step_lim, int n_steps) { *step_ctr = 0; *step_lim = n_steps; }
+// Start of a captured loop: step index, step count, and the per-unit words the tail kernel's blocks exchange.
+__global__ void k_loop_begin(Tables t, int* step_ctr, int* step_lim, int n_steps) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i == 0) { *step_ctr = 0; *step_lim = n_steps; t.plan_counter[1] = 0; t.tail_sync[0] = 0; t.tail_sync[1] = 0; t.tail_sync[2] = 0; }
+    if (i < t.U) { t.front_done[i] = 0; t.tail_queue[i] = 0; }
+}
 
 extern "C" int dynakv_decode_step(dynakv_ctx* c, const float* q, int32_t token_budget, float* out, int32_t* selected_ids) {
     if (!c || !q || !out || token_budget < 0) return DYNAKV_ERR_ARG;
@@ -388,7 +398,7 @@ extern "C" int dynakv_decode_loop(dynakv_ctx* c, const float* q_steps, const voi
     if (n_steps == 0) return DYNAKV_OK;
     {
         const long long qs = (long long)t.U * t.G * t.d * 4, ks = (long long)t.U * t.d * (long long)kv_bytes(c->cfg);
-        k_loop_begin<<<1, 1, 0, c->stream>>>(c->step_ctr, c->step_lim, (int)n_steps);
+        k_loop_begin<<<(t.U + 255) / 256, 256, 0, c->stream>>>(t, c->step_ctr, c->step_lim, (int)n_steps);
         c->launches++;
         // step 0's centroid pass; every later one rides in the tail kernel of the step before it
         enqueue_front(c, StepPtr{q_steps, qs, c->step_ctr}, StepPtr{k_steps, ks, c->step_ctr}, 1, 1, false);

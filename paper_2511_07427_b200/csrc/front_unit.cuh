@@ -101,10 +101,11 @@ __device__ __forceinline__ bool front_unit(const Tables& t, int u, const float* 
     return true;
 }
 
-// The same two values for up to two single rows (the children of a split), by one full warp, out of
-// global memory with ordinary loads: the rows were written by this block before a block barrier.
+// The same two values for two single rows (the children of a split), by one full warp.  ra / rb point at the
+// rows' HD floats (shared or global memory, written before a block barrier); both clusters are live.
 template <typename KV, int HD>
-__device__ __forceinline__ void front_patch(const Tables& t, int u, const float* __restrict__ q, const KV* __restrict__ k, int ja, int jb) {
+__device__ __forceinline__ void front_patch(const Tables& t, int u, const float* __restrict__ q, const KV* __restrict__ k, int ja,
+                                            const float* ra, int jb, const float* rb) {
     constexpr int V4 = HD / 32;
     const int lane = threadIdx.x & 31, sub = lane >> 3, l8 = lane & 7;
     float qs[V4][4], kk[V4][4];
@@ -112,17 +113,16 @@ __device__ __forceinline__ void front_patch(const Tables& t, int u, const float*
     front_key_load<KV, HD>(k, lane, kk);
     front_qsum_finish<HD>(qs);
     const int j = sub == 0 ? ja : (sub == 1 ? jb : -1);
-    const float* R = t.cl_r + (size_t)u * t.max_clusters * HD;
+    const float* R = sub == 0 ? ra : rb;
     float4 rv[V4];
 #pragma unroll
     for (int i = 0; i < V4; i++)
-        rv[i] = j >= 0 ? *reinterpret_cast<const float4*>(R + (size_t)j * HD + l8 * 4 + 32 * i) : make_float4(0.f, 0.f, 0.f, 0.f);
+        rv[i] = j >= 0 ? *reinterpret_cast<const float4*>(R + l8 * 4 + 32 * i) : make_float4(0.f, 0.f, 0.f, 0.f);
     float s, dd;
     front_row<HD>(rv, qs, kk, s, dd);
     if (j >= 0 && l8 == 0) {
-        const bool live = t.cl_n[(size_t)u * t.max_clusters + j] > 0;
-        t.scores[(size_t)u * t.max_clusters + j] = live ? s * (1.0f / (float)t.G) : -INFINITY;
-        t.dists[(size_t)u * t.max_clusters + j] = live ? dd : INFINITY;
+        t.scores[(size_t)u * t.max_clusters + j] = s * (1.0f / (float)t.G);
+        t.dists[(size_t)u * t.max_clusters + j] = dd;
     }
 }
 

@@ -9,10 +9,12 @@
 #include "append_block.cuh"
 #include "common.cuh"
 #include "front_unit.cuh"
+#include "split_small.cuh"
 
 namespace dkv {
 
 constexpr int SP_THREADS = 512;
+constexpr int SP_HELPERS = 32;                 // extra blocks of a loop iteration's tail kernel that do the splits
 constexpr int SP_CACHE_BYTES = 32 * 1024;      // member keys of the cluster being split are staged here when they fit
 constexpr int SP_WARPS = SP_THREADS / 32;
 
@@ -27,12 +29,49 @@ template <int HD, int KVB> struct SplitSmem {
     __host__ __device__ static size_t stage1_off(int maxch, int max_clusters) {
         return (keys_off(maxch, max_clusters) + SP_CACHE_BYTES + (size_t)cache_rows * sizeof(int) + 127) & ~(size_t)127;
     }
-    __host__ __device__ static size_t live_off(int maxch, int max_clusters) { return stage1_off(maxch, max_clusters) + stage_bytes; }
+    // the second area holds stage 1 of the centroid pass or the staged V rows of a cluster being split
+    __host__ __device__ static size_t live_off(int maxch, int max_clusters) { return stage1_off(maxch, max_clusters) + SP_CACHE_BYTES; }
     __host__ __device__ static size_t total(int maxch, int max_clusters) { return live_off(maxch, max_clusters) + (size_t)max_clusters + 16; }
 };
 
+// ---- hand-over of triggered units from the unit blocks to the helper blocks of a loop iteration's tail kernel.
+// tail_sync[0] = queue slots reserved, [1] = slots claimed by helpers, [2] = unit blocks that have decided.
+// A unit block with triggered clusters reserves a slot and stores unit + 1 in it; a helper claims slots in
+// order.  Helpers never hold more than SP_HELPERS of the GPU's block slots, so the unit blocks they wait for
+// always get to run; all the same every wait here is bounded.
+__device__ __forceinline__ int ld_acquire(const int* p) {
+    int v;
+    asm volatile("ld.acquire.gpu.global.s32 %0, [%1];\n" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+// Called by one thread.  Returns the next unit to split, -1 when every unit block has decided and the queue is
+// drained, -2 when a bounded wait ran out (the status word is raised).
+__device__ int next_queued_unit(const Tables& t) {
+    unsigned long long t_begin = 0;
+    for (int i = 0;; i++) {
+        const int pushed = ld_acquire(t.tail_sync + 0);
+        const int taken = ld_acquire(t.tail_sync + 1);
+        if (taken < pushed) {
+            if (atomicCAS(t.tail_sync + 1, taken, taken + 1) != taken) continue;
+            for (int k = 0; k < (1 << 20); k++) {                 // the unit id lands right after its slot was reserved
+                const int v = ld_acquire(t.tail_queue + taken);
+                if (v != 0) { t.tail_queue[taken] = 0; return v - 1; }
+            }
+            atomicOr(t.status, DYNAKV_ST_INTERNAL);
+            return -2;
+        }
+        if (ld_acquire(t.tail_sync + 2) >= t.U && ld_acquire(t.tail_sync + 0) == pushed) return -1;
+        __nanosleep(200);
+        if ((i & 31) == 31) {
+            const unsigned long long now = global_ns();
+            if (t_begin == 0) t_begin = now;
+            else if (now - t_begin > 500000000ull) { atomicOr(t.status, DYNAKV_ST_INTERNAL); return -2; }
+        }
+    }
+}
+
 template <typename KV, int HD>
-__global__ void __launch_bounds__(SP_THREADS) k_split_check(Tables t, float gamma, int var_enabled, int min_size, int iters,
+__global__ void __launch_bounds__(SP_THREADS, 2) k_split_check(Tables t, float gamma, int var_enabled, int min_size, int iters,
                                                             int do_append, StepPtr app_k, StepPtr app_v, int* step_ctr,
                                                             int do_front, StepPtr next_q, StepPtr next_k, const int* step_lim) {
     constexpr int EPL = HD / 32;
@@ -49,24 +88,17 @@ __global__ void __launch_bounds__(SP_THREADS) k_split_check(Tables t, float gamm
     __shared__ int s_cnt[4];          // changed, nA, nB, misc
     __shared__ int s_a, s_ok;
 
-    const int u = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    // In a loop iteration (do_front) the grid is U unit blocks followed by SP_HELPERS helper blocks: a unit block
+    // appends, finds its triggered clusters, hands them to the helpers and runs the unit's centroid pass of the
+    // next step; the helpers split.  Otherwise block u does the whole job for unit u.
+    const bool loop_mode = do_front != 0;
+    const bool helper = loop_mode && (int)blockIdx.x >= t.U;
+    int u = helper ? 0 : (int)blockIdx.x;
     // the step this iteration belongs to: read once, before the last block of the iteration can advance it
     const int t0 = step_ctr ? *step_ctr : 0;
-    if (do_front && tid == 0) {
-        mbar_init(smem_u32(&fr_bars[0]), 1); mbar_init(smem_u32(&fr_bars[1]), 1);
-        asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
-    }
-    // fused loop iteration: the step's append for this unit comes first (Algorithm 1's order)
-    if (do_append) { append_block<KV, HD>(t, u, app_k, app_v); __syncthreads(); }
-    const int N = t.u_N[u], M0 = t.u_M[u], Mlive0 = t.u_Mlive[u];
-    const float tau = t.u_tau[u];
-    KV* kpg = reinterpret_cast<KV*>(t.kpages) + (size_t)u * t.P * PAGE * HD;
-    KV* vpg = reinterpret_cast<KV*>(t.vpages) + (size_t)u * t.P * PAGE * HD;
-    int* ptok = t.page_tok + (size_t)u * t.P * PAGE;
-    int* pnext = t.page_next + (size_t)u * t.P;
-    unsigned char* label_g = t.sp_label + (size_t)u * t.max_tokens;
-    int* rank_g = t.sp_pos + (size_t)u * 2 * t.max_tokens;      // per position
-    int* holes_g = rank_g + t.max_tokens;                       // hole positions, in order
+    const bool fronted = loop_mode && (t0 + 1 < *step_lim);
+    __shared__ int s_ntrig, s_nsplit, s_unit, s_flag;
     // the same three arrays in shared memory for a cluster small enough to be staged
     __shared__ unsigned char label_s[SP_CACHE_BYTES / 128];
     __shared__ int rank_s[SP_CACHE_BYTES / 128], holes_s[SP_CACHE_BYTES / 128];
@@ -83,10 +115,18 @@ __global__ void __launch_bounds__(SP_THREADS) k_split_check(Tables t, float gamm
     unsigned char* dynb = reinterpret_cast<unsigned char*>(dyn);
     KV* krows = reinterpret_cast<KV*>(dynb + Lay::keys_off(maxch, t.max_clusters));
     int* tok_s = reinterpret_cast<int*>(krows + (size_t)CACHE_ROWS * HD);
-    __shared__ int s_ntrig, s_nsplit;
     if (tid == 0) { s_ntrig = 0; s_nsplit = 0; }
-    __syncthreads();
-    {
+    int ntrig = 0;
+    if (!helper) {
+        if (loop_mode && tid == 0) {
+            mbar_init(smem_u32(&fr_bars[0]), 1); mbar_init(smem_u32(&fr_bars[1]), 1);
+            asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
+        }
+        // fused loop iteration: the step's append for this unit comes first (Algorithm 1's order)
+        if (do_append) append_block<KV, HD>(t, u, app_k, app_v);
+        __syncthreads();
+        const int N = t.u_N[u], M0 = t.u_M[u], Mlive0 = t.u_Mlive[u];
+        const float tau = t.u_tau[u];
         const int full = t.u_scan[u];
         const int last = t.u_last[u];
         int base = 0;
@@ -110,30 +150,107 @@ __global__ void __launch_bounds__(SP_THREADS) k_split_check(Tables t, float gamm
         }
         if (tid == 0) s_ntrig = base;
         __syncthreads();
+        ntrig = s_ntrig;
+        if (loop_mode) {
+            // ---- hand the triggered clusters to a helper block; this block goes on to the centroid pass
+            if (tid == 0) { t.u_scan[u] = 0; t.u_last[u] = -1; }
+            if (ntrig > 0) {
+                int* tl = t.trig_list + (size_t)u * t.max_clusters;
+                for (int i = tid; i < ntrig; i += SP_THREADS) tl[i] = trig[i];
+                if (tid == 0) t.trig_n[u] = ntrig;
+            }
+            __threadfence();
+            __syncthreads();
+            if (tid == 0) {
+                if (ntrig > 0) { const int slot = atomicAdd(t.tail_sync + 0, 1); __threadfence(); atomicExch(t.tail_queue + slot, u + 1); }
+                __threadfence();
+                atomicAdd(t.tail_sync + 2, 1);
+            }
+            // the unit's centroid pass for the NEXT step (its query scores and its new key's distances) on the
+            // state after this step's append.  It needs nothing from the gather-attention kernel that may still
+            // be running and nothing from other units; a helper that splits a cluster of this unit patches the
+            // two rows it changes once this pass has finished (front_done).
+            if (fronted) {
+                const float* q1 = reinterpret_cast<const float*>(next_q.at(t0 + 1)) + (size_t)u * t.G * HD;
+                const KV* k1 = reinterpret_cast<const KV*>(next_k.at(t0 + 1)) + (size_t)u * HD;
+                front_unit<KV, HD, SP_THREADS>(t, u, q1, k1, reinterpret_cast<unsigned char*>(krows),
+                                               dynb + Lay::stage1_off(maxch, t.max_clusters), fr_bars,
+                                               dynb + Lay::live_off(maxch, t.max_clusters));
+                __threadfence();
+                __syncthreads();
+                if (tid == 0) atomicExch(t.front_done + u, t0 + 1);
+            }
+            ntrig = 0;            // nothing is split here
+        }
     }
-    const int ntrig = s_ntrig;
-    // ---- fused loop iteration: the unit's centroid pass for the NEXT step (its query scores and its new key's
-    // distances) on the state after this step's append.  It needs nothing from the gather-attention kernel that
-    // may still be running, and nothing from other units; a split below patches the two rows it changes.
-    const bool fronted = do_front && (t0 + 1 < *step_lim);
-    const float* q1 = nullptr; const KV* k1 = nullptr;
-    if (fronted) {
-        q1 = reinterpret_cast<const float*>(next_q.at(t0 + 1)) + (size_t)u * t.G * HD;
-        k1 = reinterpret_cast<const KV*>(next_k.at(t0 + 1)) + (size_t)u * HD;
-        front_unit<KV, HD, SP_THREADS>(t, u, q1, k1, reinterpret_cast<unsigned char*>(krows), dynb + Lay::stage1_off(maxch, t.max_clusters),
-                                       fr_bars, dynb + Lay::live_off(maxch, t.max_clusters));
-    }
-    // Everything above reads and writes only what the gather-attention kernel before this one never touches
-    // (statistics, the new row beyond every listed row, next step's scores); the splits below move rows, so
-    // they wait for it.
+    // ---- splits: of the block's own unit, or (helper) of every unit taken from the queue
+    for (;;) {
+        if (helper) {
+            if (tid == 0) s_unit = next_queued_unit(t);
+            __syncthreads();
+            u = s_unit;
+            if (u < 0) break;
+            __threadfence();                 // the unit block's writes (append, trigger list) precede its queue entry
+            ntrig = t.trig_n[u];
+            const int* tl = t.trig_list + (size_t)u * t.max_clusters;
+            for (int i = tid; i < ntrig; i += SP_THREADS) trig[i] = tl[i];
+            if (tid == 0) s_nsplit = 0;
+            __syncthreads();
+        }
+    // Everything before this reads and writes only what the gather-attention kernel ahead never touches (statistics,
+    // the new row beyond every listed row, next step's scores); the splits move rows, so they wait for it.
     if (ntrig > 0) pdl_wait();
+    KV* kpg = reinterpret_cast<KV*>(t.kpages) + (size_t)u * t.P * PAGE * HD;
+    KV* vpg = reinterpret_cast<KV*>(t.vpages) + (size_t)u * t.P * PAGE * HD;
+    int* ptok = t.page_tok + (size_t)u * t.P * PAGE;
+    int* pnext = t.page_next + (size_t)u * t.P;
+    unsigned char* label_g = t.sp_label + (size_t)u * t.max_tokens;
+    int* rank_g = t.sp_pos + (size_t)u * 2 * t.max_tokens;      // per position
+    int* holes_g = rank_g + t.max_tokens;                       // hole positions, in order
+    bool front_seen = false;             // helper: the unit's centroid pass of the next step is known to be complete
+    // Next step's scores and distances of the two children of a split, once the unit's own pass (which read the
+    // rows as they were before, or half-way through, the split) can no longer overwrite them.  ra / rb: the
+    // children's means (written before a block barrier).
+    auto patch_children = [&](int ja, const float* ra, int jb, const float* rb) {
+        if (!front_seen) {
+            if (tid == 0) {
+                int ok = 0;
+                const unsigned long long t_begin = global_ns();
+                for (int i = 0; i < (1 << 24); i++) {
+                    if (ld_acquire(t.front_done + u) == t0 + 1) { ok = 1; break; }
+                    __nanosleep(200);
+                    if ((i & 31) == 31 && global_ns() - t_begin > 500000000ull) break;
+                }
+                if (!ok) atomicOr(t.status, DYNAKV_ST_INTERNAL);
+                s_flag = ok;
+            }
+            __syncthreads();
+            front_seen = true;
+        }
+        if (s_flag && warp == 0) {
+            const float* q1 = reinterpret_cast<const float*>(next_q.at(t0 + 1)) + (size_t)u * t.G * HD;
+            const KV* k1 = reinterpret_cast<const KV*>(next_k.at(t0 + 1)) + (size_t)u * HD;
+            front_patch<KV, HD>(t, u, q1, k1, ja, ra, jb, rb);
+        }
+    };
+    SplitScratch sc;
+    sc.cA = cA; sc.cB = cB; sc.label = label_s; sc.rank = rank_s; sc.holes = holes_s; sc.tok = tok_s; sc.newpg = newpg;
+    sc.cnt = s_cnt; sc.nsplit = &s_nsplit;
+    KV* vrows = reinterpret_cast<KV*>(dynb + Lay::stage1_off(maxch, t.max_clusters));
     for (int li = 0; li < ntrig; li++) {
         const int j = trig[li];
         const size_t cj = (size_t)u * t.max_clusters + j;
         const int c = t.cl_n[cj];
+        __syncthreads();    // previous cluster's work is complete
+        if (c <= CACHE_ROWS) {
+            // the common case: everything out of shared memory
+            int stay_side = 0;
+            const int nid = split_small<KV, HD, SP_THREADS, CACHE_ROWS>(t, u, j, c, iters, krows, vrows, sc, &stay_side);
+            if (nid >= 0 && helper && fronted) patch_children(j, stay_side ? cB : cA, nid, stay_side ? cA : cB);
+            continue;
+        }
         if (t.u_M[u] >= t.max_clusters) { if (tid == 0) atomicOr(t.status, DYNAKV_ST_MAX_CLUSTERS); continue; }
 
-        __syncthreads();    // previous cluster's work is complete
         const int npg = (c + PAGE - 1) / PAGE;
         if (tid == 0) {
             int p = t.cl_head[cj];
@@ -396,19 +513,26 @@ __global__ void __launch_bounds__(SP_THREADS) k_split_check(Tables t, float gamm
             }
             __syncthreads();
         }
-        // next step's scores and distances of the two children
-        if (fronted && warp == 0) front_patch<KV, HD>(t, u, q1, k1, j, new_id);
+        if (helper && fronted) patch_children(j, t.cl_r + cj * HD, new_id, t.cl_r + ((size_t)u * t.max_clusters + new_id) * HD);
+    }
+        if (!helper) break;
+        __syncthreads();
+        if (tid == 0 && s_nsplit > 0) t.u_scan[u] = 1;
     }
     __syncthreads();
     // No block leaves before the kernel ahead has completed: the next kernel on the stream (the next iteration's
     // centroid pass and selection, which rewrite the work lists) is ordered behind THIS kernel only.
     pdl_wait();
     if (tid == 0) {
-        t.u_scan[u] = s_nsplit > 0 ? 1 : 0; t.u_last[u] = -1;
+        if (!loop_mode) { t.u_scan[u] = s_nsplit > 0 ? 1 : 0; t.u_last[u] = -1; }
         if (step_ctr) {
-            // the last block of the iteration advances the device-side step index that every kernel of the loop reads
+            // the last block of the iteration advances the device-side step index that every kernel of the loop reads,
+            // and clears the hand-over words for the next iteration
             __threadfence();
-            if (atomicAdd(t.plan_counter + 1, 1) == (int)gridDim.x - 1) { t.plan_counter[1] = 0; *step_ctr += 1; }
+            if (atomicAdd(t.plan_counter + 1, 1) == (int)gridDim.x - 1) {
+                t.plan_counter[1] = 0; t.tail_sync[0] = 0; t.tail_sync[1] = 0; t.tail_sync[2] = 0;
+                *step_ctr += 1;
+            }
         }
     }
 }
@@ -419,7 +543,7 @@ static void split_t(const Tables& t, float gamma, int var_enabled, int min_size,
     const size_t dyn = SplitSmem<HD, (int)sizeof(KV)>::total(t.max_tokens / PAGE + 2, t.max_clusters);
     if (dyn > 32 * 1024)
         cudaFuncSetAttribute(k_split_check<KV, HD>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn);
-    launch_pdl(k_split_check<KV, HD>, dim3(t.U), dim3(SP_THREADS), dyn, s, t, gamma, var_enabled, min_size, iters, do_append, k, v, step_ctr,
+    launch_pdl(k_split_check<KV, HD>, dim3(t.U + (nf.on ? SP_HELPERS : 0)), dim3(SP_THREADS), dyn, s, t, gamma, var_enabled, min_size, iters, do_append, k, v, step_ctr,
                nf.on, nf.q, nf.k, nf.step_lim);
 }
 
