@@ -5,8 +5,9 @@
 //
 // The unit's representatives are one contiguous array, so the block streams them through a two-stage
 // shared-memory ring with bulk-asynchronous copies (TMA, 1-D) of one pass of rows each: thread 0 issues
-// the copies, every thread waits on the stage's mbarrier, the pass is computed out of shared memory
-// with the same row arithmetic as the stand-alone kernel, and a block barrier hands the stage back.
+// the copies, warp 0 waits on the stage's mbarrier with the rest of the block asleep in a barrier behind it,
+// the pass is computed out of shared memory with the same row arithmetic as the stand-alone kernel, and the
+// same barrier hands the stage back.
 #pragma once
 
 #include "bulk_copy.cuh"
@@ -20,40 +21,64 @@ template <int THREADS, int HD> struct FrontUnit {
     static constexpr int STAGE_BYTES = ROWS * HD * 4;
 };
 
-// Called by all THREADS threads of the block, after a __syncthreads() that follows the block's own
-// writes to the unit's tables.  stage0 / stage1: 16-byte aligned shared memory of STAGE_BYTES each;
-// bars: two mbarriers initialised with count 1; live_s: shared bytes, one per cluster id of the unit.
-// Returns false (in every thread) when a bounded wait ran out; the status word is raised then.
-template <typename KV, int HD, int THREADS>
-__device__ __forceinline__ bool front_unit(const Tables& t, int u, const float* __restrict__ q, const KV* __restrict__ k,
-                                           unsigned char* stage0, unsigned char* stage1, unsigned long long* bars, unsigned char* live_s) {
-    constexpr int V4 = HD / 32;
-    constexpr int ROWS = FrontUnit<THREADS, HD>::ROWS;
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int sub = lane >> 3, l8 = lane & 7;
-    const int Mcur = t.u_M[u];
-    const float* R = t.cl_r + (size_t)u * t.max_clusters * HD;
-    const int* CN = t.cl_n + (size_t)u * t.max_clusters;
-    const int nch = (Mcur + ROWS - 1) / ROWS;
-    // This block's append and splits wrote representatives with ordinary stores, and the ring's first stage
-    // may alias shared memory written the same way: order all of that before the asynchronous proxy.
-    __threadfence();
-    fence_proxy_async();
-    __syncthreads();
-    const unsigned bar0 = smem_u32(&bars[0]), bar1 = smem_u32(&bars[1]);
-    const unsigned dst0 = smem_u32(stage0), dst1 = smem_u32(stage1);
-    auto issue = [&](int c) {
+// The pass comes in two calls so that its first copies are in flight while the block does its append:
+// the append changes one row only (the representative of the cluster that took the new key), and that row
+// is recomputed afterwards from the values the block itself wrote.
+//
+// front_unit_begin: called by all THREADS threads at the start of the block (thread 0 has initialised the two
+// mbarriers `bars` with count 1).  stage0 / stage1: 16-byte aligned shared memory of STAGE_BYTES each;
+// live_s: shared bytes, one per cluster id of the unit.
+template <typename KV, int HD>
+__device__ __forceinline__ void front_patch(const Tables& t, int u, const float* __restrict__ q, const KV* __restrict__ k, int ja,
+                                            const float* ra, int jb, const float* rb);
+
+template <int HD, int THREADS> struct FrontIssue {
+    const float* R; int Mcur; unsigned bar0, bar1, dst0, dst1;
+    __device__ __forceinline__ void operator()(int c) const {
+        constexpr int ROWS = FrontUnit<THREADS, HD>::ROWS;
         const int rows = min(ROWS, Mcur - c * ROWS);
         const unsigned bytes = (unsigned)rows * HD * 4u;
         const unsigned bar = (c & 1) ? bar1 : bar0;
         mbar_arrive_expect_tx(bar, bytes);
         bulk_g2s((c & 1) ? dst1 : dst0, R + (size_t)c * ROWS * HD, bytes, bar);
-    };
-    if (tid == 0) {
-        if (nch > 0) issue(0);
-        if (nch > 1) issue(1);
     }
-    for (int j = tid; j < Mcur; j += THREADS) live_s[j] = CN[j] > 0 ? 1 : 0;
+};
+template <int HD, int THREADS>
+__device__ __forceinline__ FrontIssue<HD, THREADS> front_unit_begin(const Tables& t, int u, unsigned char* stage0, unsigned char* stage1,
+                                                                    unsigned long long* bars, unsigned char* live_s) {
+    constexpr int ROWS = FrontUnit<THREADS, HD>::ROWS;
+    FrontIssue<HD, THREADS> is;
+    is.Mcur = t.u_M[u];
+    is.R = t.cl_r + (size_t)u * t.max_clusters * HD;
+    is.bar0 = smem_u32(&bars[0]); is.bar1 = smem_u32(&bars[1]);
+    is.dst0 = smem_u32(stage0); is.dst1 = smem_u32(stage1);
+    const int nch = (is.Mcur + ROWS - 1) / ROWS;
+    if (threadIdx.x == 0) {
+        fence_proxy_async();
+        if (nch > 0) is(0);
+        if (nch > 1) is(1);
+    }
+    // which clusters are live does not change with an append (its target is live already)
+    const int* CN = t.cl_n + (size_t)u * t.max_clusters;
+    for (int j = threadIdx.x; j < is.Mcur; j += THREADS) live_s[j] = CN[j] > 0 ? 1 : 0;
+    return is;
+}
+
+// front_unit: the passes themselves, called by all THREADS threads after a __syncthreads() that follows
+// front_unit_begin (and the block's append).  `appended` is the cluster the block's append went to (-1: none):
+// its row is recomputed at the end from global memory.  Returns false (in every thread) when a bounded wait
+// ran out; the status word is raised then.
+template <typename KV, int HD, int THREADS>
+__device__ __forceinline__ bool front_unit(const Tables& t, int u, const float* __restrict__ q, const KV* __restrict__ k,
+                                           const FrontIssue<HD, THREADS>& issue, unsigned char* stage0, unsigned char* stage1,
+                                           unsigned char* live_s, int appended) {
+    constexpr int V4 = HD / 32;
+    constexpr int ROWS = FrontUnit<THREADS, HD>::ROWS;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int sub = lane >> 3, l8 = lane & 7;
+    const int Mcur = issue.Mcur;
+    const int nch = (Mcur + ROWS - 1) / ROWS;
+    const unsigned bar0 = issue.bar0, bar1 = issue.bar1;
     float qs[V4][4], kk[V4][4];
     front_qsum_load<HD>(q, t.G, lane, qs);
     front_key_load<KV, HD>(k, lane, kk);
@@ -61,13 +86,15 @@ __device__ __forceinline__ bool front_unit(const Tables& t, int u, const float* 
     const float invG = 1.0f / (float)t.G;
     float* SC = t.scores + (size_t)u * t.max_clusters;
     float* DS = t.dists + (size_t)u * t.max_clusters;
-    __syncthreads();                 // live_s is complete
-    int failed_at = -1;
-    for (int c = 0; c < nch; c++) {
-        // warp-uniform outcome: the row arithmetic below is executed by whole warps or not at all
-        const bool ok = __all_sync(0xffffffffu, mbar_wait((c & 1) ? bar1 : bar0, (unsigned)(c >> 1) & 1u) ? 1 : 0) != 0;
-        if (ok) {
-            // every lane of the warp goes through the row arithmetic (its shuffles name the full warp);
+    // Only warp 0 polls the mbarriers; everybody else sleeps in the block barrier behind it, so a block that
+    // waits for its data leaves the SM's issue slots to the block it shares the SM with.  One barrier per pass
+    // says both "every thread is done with this stage" and "the next stage has landed".
+    bool ok = true;
+    if (warp == 0 && nch > 0) ok = mbar_wait(bar0, 0u);
+    int failed_at = __syncthreads_or(ok ? 0 : 1) ? 0 : -1;        // also: live_s is complete
+    for (int c = 0; c < nch && failed_at < 0; c++) {
+        {
+            // every lane of a warp goes through the row arithmetic (its shuffles name the full warp);
             // lanes of rows beyond the unit's last one compute on zeros and store nothing
             const int j = c * ROWS + warp * 4 + sub;
             const bool in = j < Mcur;
@@ -84,20 +111,26 @@ __device__ __forceinline__ bool front_unit(const Tables& t, int u, const float* 
                 DS[j] = live ? dd : INFINITY;
             }
         }
-        if (__syncthreads_or(ok ? 0 : 1)) { failed_at = c; break; }      // also: every thread is done with the stage
+        ok = true;
+        if (warp == 0 && c + 1 < nch) ok = mbar_wait(((c + 1) & 1) ? bar1 : bar0, (unsigned)((c + 1) >> 1) & 1u);
+        if (__syncthreads_or(ok ? 0 : 1)) { failed_at = c + 1; break; }
         if (tid == 0 && c + 2 < nch) issue(c + 2);
     }
     if (failed_at >= 0) {
         // a bounded wait ran out: report it, and let the copies still in flight land before the block's
-        // shared memory can be handed to another block
+        // shared memory can be handed to another block (only the first two passes are ever in flight together
+        // with a pass that has not been waited for)
         if (tid == 0) {
             atomicOr(t.status, DYNAKV_ST_INTERNAL);
             mbar_wait((failed_at & 1) ? bar1 : bar0, (unsigned)(failed_at >> 1) & 1u);
-            if (failed_at + 1 < nch) mbar_wait(((failed_at + 1) & 1) ? bar1 : bar0, (unsigned)((failed_at + 1) >> 1) & 1u);
+            if (failed_at == 0 && nch > 1) mbar_wait(bar1, 0u);
         }
         __syncthreads();
         return false;
     }
+    // the appended cluster's row as the append left it (the pass may have seen it before, or half-way through, the update)
+    if (appended >= 0 && warp == 0)
+        front_patch<KV, HD>(t, u, q, k, appended, t.cl_r + ((size_t)u * t.max_clusters + appended) * HD, -1, nullptr);
     return true;
 }
 

@@ -118,9 +118,18 @@ __global__ void __launch_bounds__(SP_THREADS, 2) k_split_check(Tables t, float g
     if (tid == 0) { s_ntrig = 0; s_nsplit = 0; }
     int ntrig = 0;
     if (!helper) {
-        if (loop_mode && tid == 0) {
-            mbar_init(smem_u32(&fr_bars[0]), 1); mbar_init(smem_u32(&fr_bars[1]), 1);
-            asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
+        // The unit's centroid pass for the NEXT step starts here, ahead of the append: its first copies are in
+        // flight while the append runs, and the one row the append changes is recomputed at the end of the pass.
+        unsigned char* fr_stage0 = reinterpret_cast<unsigned char*>(krows);
+        unsigned char* fr_stage1 = dynb + Lay::stage1_off(maxch, t.max_clusters);
+        unsigned char* fr_live = dynb + Lay::live_off(maxch, t.max_clusters);
+        FrontIssue<HD, SP_THREADS> fr_issue = {};
+        if (fronted) {
+            if (tid == 0) {
+                mbar_init(smem_u32(&fr_bars[0]), 1); mbar_init(smem_u32(&fr_bars[1]), 1);
+                asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
+            }
+            fr_issue = front_unit_begin<HD, SP_THREADS>(t, u, fr_stage0, fr_stage1, fr_bars, fr_live);
         }
         // fused loop iteration: the step's append for this unit comes first (Algorithm 1's order)
         if (do_append) append_block<KV, HD>(t, u, app_k, app_v);
@@ -166,16 +175,14 @@ __global__ void __launch_bounds__(SP_THREADS, 2) k_split_check(Tables t, float g
                 __threadfence();
                 atomicAdd(t.tail_sync + 2, 1);
             }
-            // the unit's centroid pass for the NEXT step (its query scores and its new key's distances) on the
-            // state after this step's append.  It needs nothing from the gather-attention kernel that may still
-            // be running and nothing from other units; a helper that splits a cluster of this unit patches the
-            // two rows it changes once this pass has finished (front_done).
+            // the rest of the unit's centroid pass for the NEXT step (its query scores and its new key's distances).
+            // It needs nothing from the gather-attention kernel that may still be running and nothing from other
+            // units; a helper that splits a cluster of this unit patches the two rows it changes once this pass
+            // has finished (front_done).
             if (fronted) {
                 const float* q1 = reinterpret_cast<const float*>(next_q.at(t0 + 1)) + (size_t)u * t.G * HD;
                 const KV* k1 = reinterpret_cast<const KV*>(next_k.at(t0 + 1)) + (size_t)u * HD;
-                front_unit<KV, HD, SP_THREADS>(t, u, q1, k1, reinterpret_cast<unsigned char*>(krows),
-                                               dynb + Lay::stage1_off(maxch, t.max_clusters), fr_bars,
-                                               dynb + Lay::live_off(maxch, t.max_clusters));
+                front_unit<KV, HD, SP_THREADS>(t, u, q1, k1, fr_issue, fr_stage0, fr_stage1, fr_live, last);
                 __threadfence();
                 __syncthreads();
                 if (tid == 0) atomicExch(t.front_done + u, t0 + 1);
@@ -235,7 +242,7 @@ __global__ void __launch_bounds__(SP_THREADS, 2) k_split_check(Tables t, float g
     };
     SplitScratch sc;
     sc.cA = cA; sc.cB = cB; sc.label = label_s; sc.rank = rank_s; sc.holes = holes_s; sc.tok = tok_s; sc.newpg = newpg;
-    sc.cnt = s_cnt; sc.nsplit = &s_nsplit;
+    sc.part = &wsum[0][0][0]; sc.nsplit = &s_nsplit;
     KV* vrows = reinterpret_cast<KV*>(dynb + Lay::stage1_off(maxch, t.max_clusters));
     for (int li = 0; li < ntrig; li++) {
         const int j = trig[li];

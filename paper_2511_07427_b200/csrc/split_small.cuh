@@ -6,7 +6,8 @@
 // -- one for everything that depends only on the cluster id, the walk along its (short) page chain, one to
 // stage its K rows, V rows and token ids; after that global memory is only written; (2) few block barriers --
 // eight lanes share a row in every distance pass (three shuffle steps per reduction), a block-wide vote
-// doubles as the "did any label change" test, and the centre update is one thread per (side, dimension).
+// doubles as the "did any label change" test, and the member sums are taken by one thread per (row slice,
+// dimension) for both sides at once.
 //
 // What is computed is exactly the split rule: centre A = member farthest from the representative, centre B =
 // member farthest from A (ties: lowest token id); Lloyd on the two centres for at most `iters` rounds, ties to
@@ -26,7 +27,7 @@ struct SplitScratch {            // shared memory of the calling block
     int* holes;                  // [rows]
     int* tok;                    // [rows]
     int* newpg;                  // [>= rows / PAGE + 1]
-    int* cnt;                    // [4]
+    float* part;                 // [THREADS / HD][2][HD] partial member sums
     int* nsplit;                 // [1] splits done by this block for the current unit
 };
 
@@ -40,10 +41,12 @@ __device__ int split_small(const Tables& t, int u, int j, int c, int iters, KV* 
     constexpr int V16 = HD * (int)sizeof(KV) / 16;        // 16-byte pieces per row
     constexpr int MAXPG = MAXROWS / PAGE;                 // pages of a staged cluster
     constexpr int NW = THREADS / 32, NG = THREADS / 8;    // warps, row groups
-    static_assert(MAXROWS <= THREADS && 2 * HD <= THREADS && MAXROWS % PAGE == 0, "one thread per member, per (side, dimension)");
+    static_assert(MAXROWS <= THREADS && 2 * HD <= THREADS && THREADS % HD == 0 && MAXROWS % PAGE == 0, "one thread per member, per (side, dimension)");
     __shared__ float r_d[2][NW];
     __shared__ int r_t[2][NW], r_p[2][NW];
     __shared__ int s_ok;
+    constexpr int Q = THREADS / HD;                       // row slices of the member-sum pass
+    __shared__ int s_pcnt[Q];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, sub = lane >> 3, l8 = lane & 7;
     const int grp = warp * 4 + sub;
     const size_t cj = (size_t)u * t.max_clusters + j;
@@ -173,19 +176,35 @@ __device__ int split_small(const Tables& t, int u, int j, int c, int iters, KV* 
             }
         }
         const int changed = __syncthreads_or(chg);        // also: the labels are complete
-        // one thread per (side, dimension): the side's member count and, when labels moved, its new mean
-        if (tid < 2 * HD) {
-            const int side = tid / HD, x = tid % HD;
-            float s = 0.f; int n = 0;
-            for (int p = 0; p < c; p++)
-                if (sc.label[p] == side) { s += to_f(krows[(size_t)p * HD + x]); n++; }
-            if (x == 0) sc.cnt[1 + side] = n;
-            if (changed && n > 0) (side ? sc.cB : sc.cA)[x] = s / (float)n;
+        // Member sums: thread (slice, dimension) adds up its slice of the rows for both sides at once (a
+        // non-member contributes an exact + 0), the slices are combined in order afterwards.
+        {
+            const int x = tid % HD, qr = tid / HD;
+            const int per = (c + Q - 1) / Q, p_lo = min(c, qr * per), p_hi = min(c, p_lo + per);
+            float sA = 0.f, sB = 0.f; int nb = 0;
+            for (int p = p_lo; p < p_hi; p++) {
+                const float v = to_f(krows[(size_t)p * HD + x]);
+                const int l = sc.label[p];
+                sA += l ? 0.f : v; sB += l ? v : 0.f; nb += l;
+            }
+            sc.part[(qr * 2 + 0) * HD + x] = sA; sc.part[(qr * 2 + 1) * HD + x] = sB;
+            if (x == 0) s_pcnt[qr] = nb;
         }
         __syncthreads();
-        nA = sc.cnt[1]; nB = sc.cnt[2];
+        nB = 0;
+#pragma unroll
+        for (int q = 0; q < Q; q++) nB += s_pcnt[q];
+        nA = c - nB;
         if (nA == 0 || nB == 0) { abandoned = true; break; }
         if (!changed) break;
+        if (tid < 2 * HD) {
+            const int side = tid / HD, x = tid % HD;
+            float sum = 0.f;
+#pragma unroll
+            for (int q = 0; q < Q; q++) sum += sc.part[(q * 2 + side) * HD + x];
+            (side ? sc.cB : sc.cA)[x] = sum / (float)(side ? nB : nA);
+        }
+        __syncthreads();
     }
     if (abandoned) { if (tid == 0) t.cl_flags[cj] |= FLAG_HOLD; return -1; }
 
