@@ -13,14 +13,24 @@ namespace dkv {
 // the tail is full).  No stored entry moves.
 // Called by every thread of a block (any block size that is a multiple of 32, up to 1024); contains one
 // __syncthreads().  Global writes are made by warp 0; callers that go on reading them synchronise first.
+// What an append did, for a caller that goes on to the split decision without reading the tables back.
+struct AppendResult {
+    int cluster;      // cluster that took the new entry, -1 when nothing was appended
+    int n_new;        // its size after the append
+    float M2_new;     // its M2 after the append
+    int N_new;        // tokens of the unit after the append
+};
+
+// `res` (shared memory, may be null) is written by lane 0 of warp 0; the caller reads it after its own barrier.
 template <typename KV, int HD>
-__device__ __forceinline__ void append_block(const Tables& t, int u, StepPtr kp_, StepPtr vp_) {
+__device__ __forceinline__ void append_block(const Tables& t, int u, StepPtr kp_, StepPtr vp_, AppendResult* res = nullptr) {
     constexpr int EPL = HD / 32;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarp = blockDim.x >> 5;
     __shared__ float red_d[32];
     __shared__ int red_j[32];
     const int Mcur = t.u_M[u];
     const int N = t.u_N[u];
+    if (res && tid == 0) { res->cluster = -1; res->n_new = 0; res->M2_new = 0.f; res->N_new = N; }
     if (N >= t.max_tokens) { if (tid == 0) atomicOr(t.status, DYNAKV_ST_MAX_TOKENS); return; }
     const float* DS = t.dists + (size_t)u * t.max_clusters;
     float bd = INFINITY; int bj = 0x7fffffff;
@@ -78,7 +88,9 @@ __device__ __forceinline__ void append_block(const Tables& t, int u, StepPtr kp_
 #pragma unroll
     for (int e = 0; e < EPL; e++) { kpg[lane * EPL + e] = knew[lane * EPL + e]; vpg[lane * EPL + e] = vnew[lane * EPL + e]; }
     if (lane == 0) {
-        t.cl_M2[cj] += add;
+        const float m2_new = t.cl_M2[cj] + add;
+        t.cl_M2[cj] = m2_new;
+        if (res) { res->cluster = bj; res->n_new = n_old + 1; res->M2_new = m2_new; res->N_new = N + 1; }
         t.cl_n[cj] = n_old + 1;
         t.cl_flags[cj] &= ~FLAG_HOLD;
         t.page_tok[((size_t)u * t.P + page) * PAGE + row] = N;

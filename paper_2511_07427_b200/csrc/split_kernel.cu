@@ -14,6 +14,9 @@
 namespace dkv {
 
 constexpr int SP_THREADS = 512;
+#ifndef DKV_SP_MINBLOCKS
+#define DKV_SP_MINBLOCKS 2          // blocks per SM the register budget is held to (a loop iteration wants all units resident)
+#endif
 constexpr int SP_HELPERS = 32;                 // extra blocks of a loop iteration's tail kernel that do the splits
 constexpr int SP_CACHE_BYTES = 32 * 1024;      // member keys of the cluster being split are staged here when they fit
 constexpr int SP_WARPS = SP_THREADS / 32;
@@ -71,7 +74,7 @@ __device__ int next_queued_unit(const Tables& t) {
 }
 
 template <typename KV, int HD>
-__global__ void __launch_bounds__(SP_THREADS, 2) k_split_check(Tables t, float gamma, int var_enabled, int min_size, int iters,
+__global__ void __launch_bounds__(SP_THREADS, DKV_SP_MINBLOCKS) k_split_check(Tables t, float gamma, int var_enabled, int min_size, int iters,
                                                             int do_append, StepPtr app_k, StepPtr app_v, int* step_ctr,
                                                             int do_front, StepPtr next_q, StepPtr next_k, const int* step_lim) {
     constexpr int EPL = HD / 32;
@@ -80,7 +83,7 @@ __global__ void __launch_bounds__(SP_THREADS, 2) k_split_check(Tables t, float g
     const int maxch = t.max_tokens / PAGE + 2;
     int* chain = dyn;                 // pages of the cluster being split, in chain order
     int* newpg = dyn + maxch;         // pages allocated for the moving child
-    __shared__ float cA[HD], cB[HD];
+    __shared__ __align__(16) float cA[HD], cB[HD];
     __shared__ float wsum[SP_WARPS][2][HD];
     __shared__ float red_f[SP_WARPS];
     __shared__ int red_i[SP_WARPS], red_k[SP_WARPS];
@@ -99,6 +102,7 @@ __global__ void __launch_bounds__(SP_THREADS, 2) k_split_check(Tables t, float g
     const int t0 = step_ctr ? *step_ctr : 0;
     const bool fronted = loop_mode && (t0 + 1 < *step_lim);
     __shared__ int s_ntrig, s_nsplit, s_unit, s_flag;
+    __shared__ AppendResult s_app;
     // the same three arrays in shared memory for a cluster small enough to be staged
     __shared__ unsigned char label_s[SP_CACHE_BYTES / 128];
     __shared__ int rank_s[SP_CACHE_BYTES / 128], holes_s[SP_CACHE_BYTES / 128];
@@ -131,13 +135,29 @@ __global__ void __launch_bounds__(SP_THREADS, 2) k_split_check(Tables t, float g
             }
             fr_issue = front_unit_begin<HD, SP_THREADS>(t, u, fr_stage0, fr_stage1, fr_bars, fr_live);
         }
-        // fused loop iteration: the step's append for this unit comes first (Algorithm 1's order)
-        if (do_append) append_block<KV, HD>(t, u, app_k, app_v);
-        __syncthreads();
-        const int N = t.u_N[u], M0 = t.u_M[u], Mlive0 = t.u_Mlive[u];
-        const float tau = t.u_tau[u];
+        // what the trigger test needs and the append does not change: loaded ahead of the append's own chain of loads
         const int full = t.u_scan[u];
-        const int last = t.u_last[u];
+        const int Mlive0 = t.u_Mlive[u];
+        const float tau = t.u_tau[u];
+        // fused loop iteration: the step's append for this unit comes first (Algorithm 1's order)
+        if (do_append) append_block<KV, HD>(t, u, app_k, app_v, &s_app);
+        __syncthreads();
+        const int last = do_append ? s_app.cluster : t.u_last[u];
+        if (!full && do_append) {
+            // Only the cluster that took the append can have become triggered (for every other cluster n_j and M2_j
+            // are unchanged while N only grew), and the append has just computed its new statistics.
+            if (tid == 0 && last >= 0) {
+                const int c = s_app.n_new;
+                // the append cleared the cluster's hold flag
+                if (c >= min_size) {
+                    const bool by_var = var_enabled && (s_app.M2_new / (float)c > tau);
+                    const bool by_size = gamma > 0.f && ((double)c * (double)Mlive0 > (double)gamma * (double)s_app.N_new);
+                    if (by_var || by_size) { trig[0] = last; s_ntrig = 1; }
+                }
+            }
+            __syncthreads();
+        } else {
+        const int N = t.u_N[u], M0 = t.u_M[u];
         int base = 0;
         const int jlim = full ? M0 : (last >= 0 ? 1 : 0);
         for (int b0 = 0; b0 < jlim; b0 += SP_THREADS) {
@@ -159,6 +179,7 @@ __global__ void __launch_bounds__(SP_THREADS, 2) k_split_check(Tables t, float g
         }
         if (tid == 0) s_ntrig = base;
         __syncthreads();
+        }
         ntrig = s_ntrig;
         if (loop_mode) {
             // ---- hand the triggered clusters to a helper block; this block goes on to the centroid pass
