@@ -163,43 +163,73 @@ def test_duplicate_keys_leave_dead_clusters():
     ctx.destroy()
 
 
-def test_graph_loop_and_host_step_match_direct_calls():
-    cfg = CONFIGS[2].scaled(n_prefill=900, steps=48, M0=30, max_clusters=96, budget=256, T=4)
-    units = [0, 1, 2, 3, 4]
+def _loop_vs_direct(cfg, units, steps, modes=("direct", "graph", "host"), cut=None):
+    """The captured loop (and the host-buffer step) must leave the same state and outputs as direct calls."""
     s = [UnitStream(cfg, u) for u in units]
     K, V = make_prefill(s)
-    q, k, v = make_decode_chunk(s, 48)
+    q, k, v = make_decode_chunk(s, steps)
+    cut = steps // 2 - 3 if cut is None else cut
     side = torch.cuda.Stream()
     outs = {}
     states = {}
-    for mode in ("direct", "graph", "host"):
+    nsplit = {}
+    for mode in modes:
         with torch.cuda.stream(side):
             from parity_harness import make_ctx
             ctx = make_ctx(cfg, len(units), trace=0, assign_mode=1)
             ctx.build_index(K.cuda(), V.cuda(), cfg.M0, 7)
             qd, kd, vd = q.cuda(), k.cuda(), v.cuda()
             if mode == "direct":
-                out = torch.empty((48, len(units), cfg.G, cfg.d), device="cuda")
-                for t in range(48):
+                out = torch.empty((steps, len(units), cfg.G, cfg.d), device="cuda")
+                for t in range(steps):
                     ctx.decode_step(qd[t], cfg.budget, out=out[t]); ctx.append(kd[t], vd[t]); ctx.split_check()
             elif mode == "graph":
-                out = ctx.decode_loop(qd[:20], kd[:20], vd[:20], cfg.budget)
-                out2 = ctx.decode_loop(qd[20:], kd[20:], vd[20:], cfg.budget)
+                # two calls: the second one starts from the state the first one left (and a count that is not a
+                # multiple of the long graph's eight iterations)
+                out = ctx.decode_loop(qd[:cut], kd[:cut], vd[:cut], cfg.budget)
+                out2 = ctx.decode_loop(qd[cut:], kd[cut:], vd[cut:], cfg.budget)
                 out = torch.cat([out, out2])
             else:
-                out = torch.empty((48, len(units), cfg.G, cfg.d))
+                out = torch.empty((steps, len(units), cfg.G, cfg.d))
                 qh, kh, vh = q.pin_memory(), k.pin_memory(), v.pin_memory()
                 oh = torch.empty((len(units), cfg.G, cfg.d)).pin_memory()
-                for t in range(48):
+                for t in range(steps):
                     ctx.step_host(qh[t], kh[t], vh[t], cfg.budget, oh); out[t] = oh
             side.synchronize()
             outs[mode] = out.cpu().numpy()
             states[mode] = ctx.export_state()
-            assert ctx.get_status()["n_splits"] > 0
+            st = ctx.get_status()
+            nsplit[mode] = st["n_splits"]
+            assert st["error_bits"] & P.ST_INTERNAL == 0
             ctx.destroy()
-    for mode in ("graph", "host"):
+    for mode in modes[1:]:
+        assert nsplit[mode] == nsplit["direct"]
         assert np.array_equal(states[mode]["tok_cluster"], states["direct"]["tok_cluster"])
+        assert np.array_equal(states[mode]["counts"], states["direct"]["counts"])
         assert np.abs(outs[mode] - outs["direct"]).max() < 1e-4
+    return nsplit["direct"]
+
+
+def test_graph_loop_and_host_step_match_direct_calls():
+    cfg = CONFIGS[2].scaled(n_prefill=900, steps=48, M0=30, max_clusters=96, budget=256, T=4)
+    assert _loop_vs_direct(cfg, [0, 1, 2, 3, 4], 48, cut=20) > 0
+
+
+def test_graph_loop_with_clusters_too_large_to_stage():
+    # three clusters over 600 keys: the clusters that split hold about 200 rows, more than the shared-memory
+    # split path stages, so the loop's helper blocks take the general path and patch the children's rows from
+    # global memory; an eager size trigger gives several triggered clusters per unit and step
+    cfg = CONFIGS[2].scaled(n_prefill=600, steps=24, M0=3, max_clusters=40, budget=300, T=3, split_min_size=4,
+                            split_size_factor=1.05)
+    assert _loop_vs_direct(cfg, [0, 1, 2], 24, modes=("direct", "graph")) > 0
+
+
+def test_graph_loop_fp32_d64_and_more_triggered_units_than_helpers():
+    # the other instantiation of the tail kernel (fp32 K/V, d = 64), and 48 units that all split in the same
+    # steps: more hand-overs than there are helper blocks
+    cfg = CONFIGS[1].scaled(B=1, L=1, Hkv=48, Hq=48 * CONFIGS[1].G, n_prefill=256, steps=20, M0=6, max_clusters=40,
+                            budget=96, T=3, split_min_size=4, split_size_factor=1.2)
+    assert _loop_vs_direct(cfg, list(range(48)), 20, modes=("direct", "graph")) > 48
 
 
 def test_wrong_call_order_and_shapes():
