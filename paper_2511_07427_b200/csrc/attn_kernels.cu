@@ -104,8 +104,8 @@ __global__ void __launch_bounds__(AT_THREADS, 2) k_gather_attn_tma(Tables t, Ste
     float* mrg = reinterpret_cast<float*>(smem + AttnSmem<HD>::ring_bytes);
     unsigned long long* bars = reinterpret_cast<unsigned long long*>(smem + AttnSmem<HD>::ring_bytes + AttnSmem<HD>::merge_bytes);
     int* meta = reinterpret_cast<int*>(bars + 2 * AT_STAGES);
-    int* s_flag = meta + AT_STAGES;                  // [0] abort, [1] combine-here
-    int* pf_s = s_flag + 16;                         // copy of work_prefix when it fits
+    int* s_flag = meta + AT_STAGES;                  // [0] abort, [1] combine-here, [2..] warp totals of the prefix scan
+    int* pf_s = s_flag + 16;                         // the units' work-list prefix when it fits
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int U = t.U, G = t.G;
     const int nb = gridDim.x, b = blockIdx.x;
@@ -120,7 +120,25 @@ __global__ void __launch_bounds__(AT_THREADS, 2) k_gather_attn_tma(Tables t, Ste
     pdl_wait();          // the work lists and their prefix come from the selection kernel
     const int* pf = t.work_prefix;
     if (t.attn_pf_in_smem) {
-        for (int i = tid; i <= U; i += AT_THREADS) pf_s[i] = pf[i];
+        // Every CTA lays the units' work lists end to end itself: an exclusive prefix of their lengths, each
+        // thread taking a run of consecutive units (all its loads in flight together), then a block scan.
+        constexpr int MAXPER = 1024 / AT_THREADS;         // attn_pf_in_smem is set for at most 1024 units
+        const int per_t = (U + AT_THREADS - 1) / AT_THREADS;
+        const int b0 = min(tid * per_t, U);
+        int nw[MAXPER];
+        int sum = 0;
+#pragma unroll
+        for (int i = 0; i < MAXPER; i++) { nw[i] = (i < per_t && b0 + i < U) ? t.n_work[b0 + i] : 0; sum += nw[i]; }
+        int incl = sum;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) { const int y = __shfl_up_sync(0xffffffffu, incl, o); if (lane >= o) incl += y; }
+        if (lane == 31) s_flag[2 + warp] = incl;
+        __syncthreads();
+        int base = incl - sum;
+        for (int w = 0; w < warp; w++) base += s_flag[2 + w];
+#pragma unroll
+        for (int i = 0; i < MAXPER; i++) if (i < per_t && b0 + i < U) { pf_s[b0 + i] = base; base += nw[i]; }
+        if (tid == AT_THREADS - 1) pf_s[U] = base;
         pf = pf_s;
     }
     __syncthreads();

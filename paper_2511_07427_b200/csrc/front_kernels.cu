@@ -89,25 +89,27 @@ __global__ void __launch_bounds__(FR_THREADS, 2) k_front(Tables t, StepPtr qp, S
 
 constexpr int SL_THREADS = 1024;
 
-// One block per unit: see select_unit().  The last block to finish also writes the exclusive prefix of the
-// units' work-list lengths.
+// One block per unit: see select_unit().
 __global__ void __launch_bounds__(SL_THREADS) k_select(Tables t, int budget, int* __restrict__ user_ids) {
     __shared__ SelectSmem sm;
     __shared__ int s_last;
     pdl_wait();                          // the scores come from the kernel before
     select_unit<SL_THREADS>(t, blockIdx.x, budget, user_ids, sm);
-    // ---- the last unit block to finish lays the units' work lists end to end
-    __threadfence();
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        const int old = atomicAdd(t.plan_counter, 1);
-        s_last = (old == t.U - 1) ? 1 : 0;
-    }
-    __syncthreads();
-    if (s_last) {
+    // ---- With more units than the gather-attention CTAs keep in shared memory, the last unit block to finish lays
+    // the units' work lists end to end (otherwise every attention CTA does that itself from n_work).
+    if (!t.attn_pf_in_smem) {
         __threadfence();
-        work_prefix_block<SL_THREADS>(t, sm.sh);
-        if (threadIdx.x == 0) *t.plan_counter = 0;
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            const int old = atomicAdd(t.plan_counter, 1);
+            s_last = (old == t.U - 1) ? 1 : 0;
+        }
+        __syncthreads();
+        if (s_last) {
+            __threadfence();
+            work_prefix_block<SL_THREADS>(t, sm.sh);
+            if (threadIdx.x == 0) *t.plan_counter = 0;
+        }
     }
     pdl_trigger();
 }
