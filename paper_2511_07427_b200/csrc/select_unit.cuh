@@ -35,13 +35,18 @@ __device__ __forceinline__ unsigned int ord_key(float f) {
 template <int THREADS>
 __device__ void select_unit(const Tables& t, int u, int budget, int* __restrict__ user_ids, SelectSmem& sm) {
     const int tid = threadIdx.x;
-    const int Mcur = t.u_M[u];
     const float* SC = t.scores + (size_t)u * t.max_clusters;
     const int* CN = t.cl_n + (size_t)u * t.max_clusters;
+    // A unit never has fewer ids than the build gave it, so the first id of every thread below that count is
+    // loaded without waiting for the unit's current count.
+    const bool early = tid < t.M_floor;
+    int sz0 = 0; float sc0 = 0.f;
+    if (early) { sz0 = CN[tid]; sc0 = __ldcg(SC + tid); }
+    const int Mcur = t.u_M[u];
     unsigned long long best = 0ull;
     for (int j = tid; j < Mcur; j += THREADS) {
-        const int sz = CN[j];
-        const unsigned int key = sz > 0 ? ord_key(__ldcg(SC + j)) : 0u;
+        const int sz = (j == tid && early) ? sz0 : CN[j];
+        const unsigned int key = sz > 0 ? ord_key((j == tid && early) ? sc0 : __ldcg(SC + j)) : 0u;
         sm.keys[j] = key; sm.sizes[j] = sz;
         if (sz > 0) {
             const unsigned long long kk = ((unsigned long long)key << 32) | (unsigned long long)(0xffffffffu - (unsigned)j);
