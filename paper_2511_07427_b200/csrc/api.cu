@@ -179,7 +179,7 @@ extern "C" int dynakv_create(const dynakv_config* cfg, void* cuda_stream, dynakv
     ALLOC(t.unit_arrive, U, true);
     ALLOC(t.plan_counter, 2, true);
     ALLOC(t.tail_sync, 4, true);
-    ALLOC(t.tail_queue, U, true);
+    ALLOC(t.tail_queue, 2 * U, true);
     ALLOC(t.front_done, U, true);
     ALLOC(t.trig_n, U, true);
     ALLOC(t.trig_list, U * Mx, false);
@@ -319,7 +319,7 @@ static void enqueue_loop_iteration(dynakv_ctx* c, StepPtr q, StepPtr k, StepPtr 
 __global__ void k_loop_begin(Tables t, int* step_ctr, int* step_lim, int n_steps) {
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i == 0) { *step_ctr = 0; *step_lim = n_steps; t.plan_counter[1] = 0; t.tail_sync[0] = 0; t.tail_sync[1] = 0; t.tail_sync[2] = 0; }
-    if (i < t.U) { t.front_done[i] = 0; t.tail_queue[i] = 0; }
+    if (i < t.U) { t.front_done[i] = 0; t.tail_queue[2 * i] = 0; t.tail_queue[2 * i + 1] = 0; }
 }
 
 extern "C" int dynakv_decode_step(dynakv_ctx* c, const float* q, int32_t token_budget, float* out, int32_t* selected_ids) {

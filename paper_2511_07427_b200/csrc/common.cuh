@@ -52,7 +52,7 @@ struct Tables {
     int* plan_counter;               // [2] blocks finished in this step: [0] of the selection, [1] of the append/split kernel
     // hand-over of triggered units from the unit blocks to the helper blocks of a loop iteration's tail kernel
     int* tail_sync;                  // [4] queue slots reserved, slots claimed, unit blocks that have decided
-    int* tail_queue;                 // [U] unit + 1 per reserved slot (0 = not yet written / consumed)
+    int* tail_queue;                 // [U][2] per reserved slot: hint, unit + 1 (0 = not yet written / consumed)
     int* front_done;                 // [U] step + 1 of the last fused centroid pass the unit's block completed
     int* trig_n; int* trig_list;     // [U], [U][Mmax] triggered cluster ids of a unit, ascending
     int n_attn_ctas;                 // persistent gather-attention CTAs (2 per SM)

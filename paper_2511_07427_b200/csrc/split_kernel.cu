@@ -39,8 +39,9 @@ template <int HD, int KVB> struct SplitSmem {
 
 // ---- hand-over of triggered units from the unit blocks to the helper blocks of a loop iteration's tail kernel.
 // tail_sync[0] = queue slots reserved, [1] = slots claimed by helpers, [2] = unit blocks that have decided.
-// A unit block with triggered clusters reserves a slot and stores unit + 1 in it; a helper claims slots in
-// order.  Helpers never hold more than SP_HELPERS of the GPU's block slots, so the unit blocks they wait for
+// A unit block with triggered clusters reserves a slot (two words) and stores a hint, then unit + 1, in it; a
+// helper claims slots in order.  The hint spares the helper two trips to memory in the common case of one
+// triggered cluster whose size the unit block knows: (cluster id + 1) | (size << 13), else 0.  Helpers never hold more than SP_HELPERS of the GPU's block slots, so the unit blocks they wait for
 // always get to run; all the same every wait here is bounded.
 __device__ __forceinline__ int ld_acquire(const int* p) {
     int v;
@@ -49,7 +50,7 @@ __device__ __forceinline__ int ld_acquire(const int* p) {
 }
 // Called by one thread.  Returns the next unit to split, -1 when every unit block has decided and the queue is
 // drained, -2 when a bounded wait ran out (the status word is raised).
-__device__ int next_queued_unit(const Tables& t) {
+__device__ int next_queued_unit(const Tables& t, int* hint) {
     unsigned long long t_begin = 0;
     for (int i = 0;; i++) {
         const int pushed = ld_acquire(t.tail_sync + 0);
@@ -57,8 +58,8 @@ __device__ int next_queued_unit(const Tables& t) {
         if (taken < pushed) {
             if (atomicCAS(t.tail_sync + 1, taken, taken + 1) != taken) continue;
             for (int k = 0; k < (1 << 20); k++) {                 // the unit id lands right after its slot was reserved
-                const int v = ld_acquire(t.tail_queue + taken);
-                if (v != 0) { t.tail_queue[taken] = 0; return v - 1; }
+                const int v = ld_acquire(t.tail_queue + 2 * taken + 1);
+                if (v != 0) { *hint = t.tail_queue[2 * taken]; t.tail_queue[2 * taken + 1] = 0; return v - 1; }
             }
             atomicOr(t.status, DYNAKV_ST_INTERNAL);
             return -2;
@@ -101,7 +102,8 @@ __global__ void __launch_bounds__(SP_THREADS, DKV_SP_MINBLOCKS) k_split_check(Ta
     // the step this iteration belongs to: read once, before the last block of the iteration can advance it
     const int t0 = step_ctr ? *step_ctr : 0;
     const bool fronted = loop_mode && (t0 + 1 < *step_lim);
-    __shared__ int s_ntrig, s_nsplit, s_unit, s_flag;
+    __shared__ int s_ntrig, s_nsplit, s_unit, s_flag, s_hint;
+    int c_hint = 0;                  // helper: size of the single triggered cluster when the unit block passed it along
     __shared__ AppendResult s_app;
     // the same three arrays in shared memory for a cluster small enough to be staged
     __shared__ unsigned char label_s[SP_CACHE_BYTES / 128];
@@ -192,7 +194,14 @@ __global__ void __launch_bounds__(SP_THREADS, DKV_SP_MINBLOCKS) k_split_check(Ta
             __threadfence();
             __syncthreads();
             if (tid == 0) {
-                if (ntrig > 0) { const int slot = atomicAdd(t.tail_sync + 0, 1); __threadfence(); atomicExch(t.tail_queue + slot, u + 1); }
+                if (ntrig > 0) {
+                    const int slot = atomicAdd(t.tail_sync + 0, 1);
+                    int hint = 0;
+                    if (ntrig == 1 && !full && do_append && s_app.cluster == trig[0]) hint = (trig[0] + 1) | (s_app.n_new << 13);
+                    t.tail_queue[2 * slot] = hint;
+                    __threadfence();
+                    atomicExch(t.tail_queue + 2 * slot + 1, u + 1);
+                }
                 __threadfence();
                 atomicAdd(t.tail_sync + 2, 1);
             }
@@ -214,15 +223,21 @@ __global__ void __launch_bounds__(SP_THREADS, DKV_SP_MINBLOCKS) k_split_check(Ta
     // ---- splits: of the block's own unit, or (helper) of every unit taken from the queue
     for (;;) {
         if (helper) {
-            if (tid == 0) s_unit = next_queued_unit(t);
+            if (tid == 0) { int h = 0; s_unit = next_queued_unit(t, &h); s_hint = h; }
             __syncthreads();
             u = s_unit;
             if (u < 0) break;
             __threadfence();                 // the unit block's writes (append, trigger list) precede its queue entry
-            ntrig = t.trig_n[u];
-            const int* tl = t.trig_list + (size_t)u * t.max_clusters;
-            for (int i = tid; i < ntrig; i += SP_THREADS) trig[i] = tl[i];
-            if (tid == 0) s_nsplit = 0;
+            c_hint = 0;
+            if (s_hint != 0) {
+                ntrig = 1; c_hint = s_hint >> 13;
+                if (tid == 0) { trig[0] = (s_hint & 8191) - 1; s_nsplit = 0; }
+            } else {
+                ntrig = t.trig_n[u];
+                const int* tl = t.trig_list + (size_t)u * t.max_clusters;
+                for (int i = tid; i < ntrig; i += SP_THREADS) trig[i] = tl[i];
+                if (tid == 0) s_nsplit = 0;
+            }
             __syncthreads();
         }
     // Everything before this reads and writes only what the gather-attention kernel ahead never touches (statistics,
@@ -268,7 +283,7 @@ __global__ void __launch_bounds__(SP_THREADS, DKV_SP_MINBLOCKS) k_split_check(Ta
     for (int li = 0; li < ntrig; li++) {
         const int j = trig[li];
         const size_t cj = (size_t)u * t.max_clusters + j;
-        const int c = t.cl_n[cj];
+        const int c = c_hint > 0 ? c_hint : t.cl_n[cj];
         __syncthreads();    // previous cluster's work is complete
         if (c <= CACHE_ROWS) {
             // the common case: everything out of shared memory
