@@ -3,7 +3,7 @@
 // query of step t + 1 and measures the distances of the key of step t + 1, while other units' blocks
 // may still be splitting (units are independent, so nothing else has to be waited for).
 //
-// The unit's representatives are one contiguous array, so the block streams them through a two-stage
+// The unit's representatives are one contiguous array, so the block streams them through a three-stage
 // shared-memory ring with bulk-asynchronous copies (TMA, 1-D) of one pass of rows each: thread 0 issues
 // the copies, warp 0 waits on the stage's mbarrier with the rest of the block asleep in a barrier behind it,
 // the pass is computed out of shared memory with the same row arithmetic as the stand-alone kernel, and the
@@ -26,32 +26,37 @@ template <int THREADS, int HD> struct FrontUnit {
 // is recomputed afterwards from the values the block itself wrote.
 //
 // front_unit_begin: called by all THREADS threads at the start of the block (thread 0 has initialised the two
-// mbarriers `bars` with count 1).  stage0 / stage1: 16-byte aligned shared memory of STAGE_BYTES each;
+// FR_STAGES mbarriers `bars` with count 1).  stages: 16-byte aligned shared memory of STAGE_BYTES each;
 // live_s: shared bytes, one per cluster id of the unit.
 template <typename KV, int HD>
 __device__ __forceinline__ void front_patch(const Tables& t, int u, const float* __restrict__ q, const KV* __restrict__ k, int ja,
                                             const float* ra, int jb, const float* rb);
 
+constexpr int FR_STAGES = 3;
 template <int HD, int THREADS> struct FrontIssue {
-    const float* R; int Mcur; unsigned bar0, bar1, dst0, dst1;
+    const float* R; int Mcur; unsigned bar[FR_STAGES], dst[FR_STAGES];
+    static_assert(FR_STAGES == 3, "the selects below spell the stages out (no run-time indexing of register arrays)");
+    __device__ __forceinline__ unsigned bar_of(int st) const { return st == 0 ? bar[0] : (st == 1 ? bar[1] : bar[2]); }
     __device__ __forceinline__ void operator()(int c) const {
         constexpr int ROWS = FrontUnit<THREADS, HD>::ROWS;
         const int rows = min(ROWS, Mcur - c * ROWS);
         const unsigned bytes = (unsigned)rows * HD * 4u;
-        const unsigned bar = (c & 1) ? bar1 : bar0;
-        mbar_arrive_expect_tx(bar, bytes);
-        bulk_g2s((c & 1) ? dst1 : dst0, R + (size_t)c * ROWS * HD, bytes, bar);
+        const int st = c % FR_STAGES;
+        mbar_arrive_expect_tx(bar_of(st), bytes);
+        bulk_g2s(st == 0 ? dst[0] : (st == 1 ? dst[1] : dst[2]), R + (size_t)c * ROWS * HD, bytes, bar_of(st));
     }
 };
+// stages: FR_STAGES pointers; the first two must be free from the start of the block, the third from the call of
+// front_unit() on.
 template <int HD, int THREADS>
-__device__ __forceinline__ FrontIssue<HD, THREADS> front_unit_begin(const Tables& t, int u, unsigned char* stage0, unsigned char* stage1,
+__device__ __forceinline__ FrontIssue<HD, THREADS> front_unit_begin(const Tables& t, int u, unsigned char* const* stages,
                                                                     unsigned long long* bars, unsigned char* live_s) {
     constexpr int ROWS = FrontUnit<THREADS, HD>::ROWS;
     FrontIssue<HD, THREADS> is;
     is.Mcur = t.u_M[u];
     is.R = t.cl_r + (size_t)u * t.max_clusters * HD;
-    is.bar0 = smem_u32(&bars[0]); is.bar1 = smem_u32(&bars[1]);
-    is.dst0 = smem_u32(stage0); is.dst1 = smem_u32(stage1);
+#pragma unroll
+    for (int i = 0; i < FR_STAGES; i++) { is.bar[i] = smem_u32(&bars[i]); is.dst[i] = smem_u32(stages[i]); }
     const int nch = (is.Mcur + ROWS - 1) / ROWS;
     if (threadIdx.x == 0) {
         fence_proxy_async();
@@ -70,7 +75,7 @@ __device__ __forceinline__ FrontIssue<HD, THREADS> front_unit_begin(const Tables
 // ran out; the status word is raised then.
 template <typename KV, int HD, int THREADS>
 __device__ __forceinline__ bool front_unit(const Tables& t, int u, const float* __restrict__ q, const KV* __restrict__ k,
-                                           const FrontIssue<HD, THREADS>& issue, unsigned char* stage0, unsigned char* stage1,
+                                           const FrontIssue<HD, THREADS>& issue, unsigned char* const* stages,
                                            unsigned char* live_s, int appended) {
     constexpr int V4 = HD / 32;
     constexpr int ROWS = FrontUnit<THREADS, HD>::ROWS;
@@ -78,7 +83,8 @@ __device__ __forceinline__ bool front_unit(const Tables& t, int u, const float* 
     const int sub = lane >> 3, l8 = lane & 7;
     const int Mcur = issue.Mcur;
     const int nch = (Mcur + ROWS - 1) / ROWS;
-    const unsigned bar0 = issue.bar0, bar1 = issue.bar1;
+    // the third stage is free now (the caller's barrier is behind every earlier use of that memory)
+    if (tid == 0 && nch > 2) { fence_proxy_async(); issue(2); }
     float qs[V4][4], kk[V4][4];
     front_qsum_load<HD>(q, t.G, lane, qs);
     front_key_load<KV, HD>(k, lane, kk);
@@ -90,7 +96,7 @@ __device__ __forceinline__ bool front_unit(const Tables& t, int u, const float* 
     // waits for its data leaves the SM's issue slots to the block it shares the SM with.  One barrier per pass
     // says both "every thread is done with this stage" and "the next stage has landed".
     bool ok = true;
-    if (warp == 0 && nch > 0) ok = mbar_wait(bar0, 0u);
+    if (warp == 0 && nch > 0) ok = mbar_wait(issue.bar[0], 0u);
     int failed_at = __syncthreads_or(ok ? 0 : 1) ? 0 : -1;        // also: live_s is complete
     for (int c = 0; c < nch && failed_at < 0; c++) {
         {
@@ -98,7 +104,8 @@ __device__ __forceinline__ bool front_unit(const Tables& t, int u, const float* 
             // lanes of rows beyond the unit's last one compute on zeros and store nothing
             const int j = c * ROWS + warp * 4 + sub;
             const bool in = j < Mcur;
-            const unsigned char* row = ((c & 1) ? stage1 : stage0) + (size_t)(warp * 4 + sub) * HD * 4;
+            const int st = c % FR_STAGES;
+            const unsigned char* row = (st == 0 ? stages[0] : (st == 1 ? stages[1] : stages[2])) + (size_t)(warp * 4 + sub) * HD * 4;
             float4 rv[V4];
 #pragma unroll
             for (int i = 0; i < V4; i++)
@@ -112,18 +119,17 @@ __device__ __forceinline__ bool front_unit(const Tables& t, int u, const float* 
             }
         }
         ok = true;
-        if (warp == 0 && c + 1 < nch) ok = mbar_wait(((c + 1) & 1) ? bar1 : bar0, (unsigned)((c + 1) >> 1) & 1u);
+        if (warp == 0 && c + 1 < nch) ok = mbar_wait(issue.bar_of((c + 1) % FR_STAGES), (unsigned)((c + 1) / FR_STAGES) & 1u);
         if (__syncthreads_or(ok ? 0 : 1)) { failed_at = c + 1; break; }
-        if (tid == 0 && c + 2 < nch) issue(c + 2);
+        if (tid == 0 && c + FR_STAGES < nch) issue(c + FR_STAGES);
     }
     if (failed_at >= 0) {
-        // a bounded wait ran out: report it, and let the copies still in flight land before the block's
-        // shared memory can be handed to another block (only the first two passes are ever in flight together
-        // with a pass that has not been waited for)
+        // a bounded wait ran out: report it, and let the copies still in flight (at most FR_STAGES passes from the
+        // failed one on) land before the block's shared memory can be handed to another block
         if (tid == 0) {
             atomicOr(t.status, DYNAKV_ST_INTERNAL);
-            mbar_wait((failed_at & 1) ? bar1 : bar0, (unsigned)(failed_at >> 1) & 1u);
-            if (failed_at == 0 && nch > 1) mbar_wait(bar1, 0u);
+            for (int f = failed_at; f < nch && f < failed_at + FR_STAGES; f++)
+                mbar_wait(issue.bar_of(f % FR_STAGES), (unsigned)(f / FR_STAGES) & 1u);
         }
         __syncthreads();
         return false;

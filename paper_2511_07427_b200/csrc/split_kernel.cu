@@ -21,18 +21,26 @@ constexpr int SP_HELPERS = 32;                 // extra blocks of a loop iterati
 constexpr int SP_CACHE_BYTES = 32 * 1024;      // member keys of the cluster being split are staged here when they fit
 constexpr int SP_WARPS = SP_THREADS / 32;
 
-// Dynamic shared memory, in order: chain[maxch], newpg[maxch], trig[max_clusters] (ints); the staged member
-// keys (SP_CACHE_BYTES, 16-byte aligned; also stage 0 of the fused centroid pass) and their token ids; stage 1
-// of the fused centroid pass; one live flag per cluster id.
+// Dynamic shared memory, in order:
+//   area 0: chain[maxch], newpg[maxch], trig[max_clusters] (ints), the split code's partial sums
+//           wsum[SP_WARPS][2][HD] (floats); at least one ring stage long, because in a unit block of a loop
+//           iteration it becomes stage 2 of the fused centroid pass once the trigger list has been handed over;
+//   area 1: the staged member keys (SP_CACHE_BYTES; stage 0 of the pass) and their token ids;
+//   area 2: the staged member values (SP_CACHE_BYTES; stage 1 of the pass);
+//   one live flag per cluster id.
 template <int HD, int KVB> struct SplitSmem {
     static constexpr int cache_rows = SP_CACHE_BYTES / (HD * KVB);
     static constexpr int stage_bytes = FrontUnit<SP_THREADS, HD>::STAGE_BYTES;
-    static_assert(stage_bytes <= SP_CACHE_BYTES, "stage 0 of the centroid pass lives in the staging area");
-    __host__ __device__ static size_t keys_off(int maxch, int max_clusters) { return (((size_t)(2 * maxch + max_clusters) * sizeof(int)) + 127) & ~(size_t)127; }
+    static_assert(stage_bytes <= SP_CACHE_BYTES, "stages 0 and 1 of the centroid pass live in the staging areas");
+    __host__ __device__ static size_t wsum_off(int maxch, int max_clusters) { return (((size_t)(2 * maxch + max_clusters) * sizeof(int)) + 15) & ~(size_t)15; }
+    __host__ __device__ static size_t keys_off(int maxch, int max_clusters) {
+        size_t a = wsum_off(maxch, max_clusters) + (size_t)SP_WARPS * 2 * HD * sizeof(float);
+        if (a < (size_t)stage_bytes) a = stage_bytes;
+        return (a + 127) & ~(size_t)127;
+    }
     __host__ __device__ static size_t stage1_off(int maxch, int max_clusters) {
         return (keys_off(maxch, max_clusters) + SP_CACHE_BYTES + (size_t)cache_rows * sizeof(int) + 127) & ~(size_t)127;
     }
-    // the second area holds stage 1 of the centroid pass or the staged V rows of a cluster being split
     __host__ __device__ static size_t live_off(int maxch, int max_clusters) { return stage1_off(maxch, max_clusters) + SP_CACHE_BYTES; }
     __host__ __device__ static size_t total(int maxch, int max_clusters) { return live_off(maxch, max_clusters) + (size_t)max_clusters + 16; }
 };
@@ -80,12 +88,11 @@ __global__ void __launch_bounds__(SP_THREADS, DKV_SP_MINBLOCKS) k_split_check(Ta
                                                             int do_front, StepPtr next_q, StepPtr next_k, const int* step_lim) {
     constexpr int EPL = HD / 32;
     extern __shared__ __align__(128) int dyn[];
-    __shared__ unsigned long long fr_bars[2];
+    __shared__ unsigned long long fr_bars[FR_STAGES];
     const int maxch = t.max_tokens / PAGE + 2;
     int* chain = dyn;                 // pages of the cluster being split, in chain order
     int* newpg = dyn + maxch;         // pages allocated for the moving child
     __shared__ __align__(16) float cA[HD], cB[HD];
-    __shared__ float wsum[SP_WARPS][2][HD];
     __shared__ float red_f[SP_WARPS];
     __shared__ int red_i[SP_WARPS], red_k[SP_WARPS];
     __shared__ int sh[33];
@@ -119,6 +126,8 @@ __global__ void __launch_bounds__(SP_THREADS, DKV_SP_MINBLOCKS) k_split_check(Ta
     using Lay = SplitSmem<HD, (int)sizeof(KV)>;
     constexpr int CACHE_ROWS = Lay::cache_rows;
     unsigned char* dynb = reinterpret_cast<unsigned char*>(dyn);
+    float* wsum = reinterpret_cast<float*>(dynb + Lay::wsum_off(maxch, t.max_clusters));   // [SP_WARPS][2][HD]
+    auto WS = [&](int w, int side, int x) -> float& { return wsum[((size_t)w * 2 + side) * HD + x]; };
     KV* krows = reinterpret_cast<KV*>(dynb + Lay::keys_off(maxch, t.max_clusters));
     int* tok_s = reinterpret_cast<int*>(krows + (size_t)CACHE_ROWS * HD);
     if (tid == 0) { s_ntrig = 0; s_nsplit = 0; }
@@ -126,16 +135,15 @@ __global__ void __launch_bounds__(SP_THREADS, DKV_SP_MINBLOCKS) k_split_check(Ta
     if (!helper) {
         // The unit's centroid pass for the NEXT step starts here, ahead of the append: its first copies are in
         // flight while the append runs, and the one row the append changes is recomputed at the end of the pass.
-        unsigned char* fr_stage0 = reinterpret_cast<unsigned char*>(krows);
-        unsigned char* fr_stage1 = dynb + Lay::stage1_off(maxch, t.max_clusters);
+        unsigned char* const fr_stages[FR_STAGES] = {reinterpret_cast<unsigned char*>(krows), dynb + Lay::stage1_off(maxch, t.max_clusters), dynb};
         unsigned char* fr_live = dynb + Lay::live_off(maxch, t.max_clusters);
         FrontIssue<HD, SP_THREADS> fr_issue = {};
         if (fronted) {
             if (tid == 0) {
-                mbar_init(smem_u32(&fr_bars[0]), 1); mbar_init(smem_u32(&fr_bars[1]), 1);
+                for (int i = 0; i < FR_STAGES; i++) mbar_init(smem_u32(&fr_bars[i]), 1);
                 asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
             }
-            fr_issue = front_unit_begin<HD, SP_THREADS>(t, u, fr_stage0, fr_stage1, fr_bars, fr_live);
+            fr_issue = front_unit_begin<HD, SP_THREADS>(t, u, fr_stages, fr_bars, fr_live);
         }
         // what the trigger test needs and the append does not change: loaded ahead of the append's own chain of loads
         const int full = t.u_scan[u];
@@ -192,6 +200,7 @@ __global__ void __launch_bounds__(SP_THREADS, DKV_SP_MINBLOCKS) k_split_check(Ta
                 if (tid == 0) t.trig_n[u] = ntrig;
             }
             __threadfence();
+            fence_proxy_async();          // area 0 (written above with ordinary stores) becomes a ring stage below
             __syncthreads();
             if (tid == 0) {
                 if (ntrig > 0) {
@@ -212,7 +221,7 @@ __global__ void __launch_bounds__(SP_THREADS, DKV_SP_MINBLOCKS) k_split_check(Ta
             if (fronted) {
                 const float* q1 = reinterpret_cast<const float*>(next_q.at(t0 + 1)) + (size_t)u * t.G * HD;
                 const KV* k1 = reinterpret_cast<const KV*>(next_k.at(t0 + 1)) + (size_t)u * HD;
-                front_unit<KV, HD, SP_THREADS>(t, u, q1, k1, fr_issue, fr_stage0, fr_stage1, fr_live, last);
+                front_unit<KV, HD, SP_THREADS>(t, u, q1, k1, fr_issue, fr_stages, fr_live, last);
                 __threadfence();
                 __syncthreads();
                 if (tid == 0) atomicExch(t.front_done + u, t0 + 1);
@@ -278,7 +287,7 @@ __global__ void __launch_bounds__(SP_THREADS, DKV_SP_MINBLOCKS) k_split_check(Ta
     };
     SplitScratch sc;
     sc.cA = cA; sc.cB = cB; sc.label = label_s; sc.rank = rank_s; sc.holes = holes_s; sc.tok = tok_s; sc.newpg = newpg;
-    sc.part = &wsum[0][0][0]; sc.nsplit = &s_nsplit;
+    sc.part = wsum; sc.nsplit = &s_nsplit;
     KV* vrows = reinterpret_cast<KV*>(dynb + Lay::stage1_off(maxch, t.max_clusters));
     for (int li = 0; li < ntrig; li++) {
         const int j = trig[li];
@@ -383,7 +392,7 @@ __global__ void __launch_bounds__(SP_THREADS, DKV_SP_MINBLOCKS) k_split_check(Ta
                 for (int e = 0; e < EPL; e++) { if (l) sb[e] += kk[e]; else sa[e] += kk[e]; }
             }
 #pragma unroll
-            for (int e = 0; e < EPL; e++) { wsum[warp][0][lane * EPL + e] = sa[e]; wsum[warp][1][lane * EPL + e] = sb[e]; }
+            for (int e = 0; e < EPL; e++) { WS(warp, 0, lane * EPL + e) = sa[e]; WS(warp, 1, lane * EPL + e) = sb[e]; }
             if (lane == 0) { if (chg) atomicOr(&s_cnt[0], 1); atomicAdd(&s_cnt[1], ca); atomicAdd(&s_cnt[2], cb); }
             __syncthreads();
             nA = s_cnt[1]; nB = s_cnt[2];
@@ -393,7 +402,7 @@ __global__ void __launch_bounds__(SP_THREADS, DKV_SP_MINBLOCKS) k_split_check(Ta
             for (int e = tid; e < 2 * HD; e += SP_THREADS) {
                 int side = e / HD, x = e % HD;
                 float s = 0.f;
-                for (int w = 0; w < SP_WARPS; w++) s += wsum[w][side][x];
+                for (int w = 0; w < SP_WARPS; w++) s += WS(w, side, x);
                 if (side == 0) cA[x] = s / (float)nA; else cB[x] = s / (float)nB;
             }
             __syncthreads();
@@ -526,11 +535,11 @@ __global__ void __launch_bounds__(SP_THREADS, DKV_SP_MINBLOCKS) k_split_check(Ta
                 for (int e = 0; e < EPL; e++) sa[e] += to_f(k[e]);
             }
 #pragma unroll
-            for (int e = 0; e < EPL; e++) wsum[warp][0][lane * EPL + e] = sa[e];
+            for (int e = 0; e < EPL; e++) WS(warp, 0, lane * EPL + e) = sa[e];
             __syncthreads();
             for (int e = tid; e < HD; e += SP_THREADS) {
                 float s = 0.f;
-                for (int w = 0; w < SP_WARPS; w++) s += wsum[w][0][e];
+                for (int w = 0; w < SP_WARPS; w++) s += WS(w, 0, e);
                 s /= (float)cc;
                 cA[e] = s;
                 t.cl_r[cid * HD + e] = s;
