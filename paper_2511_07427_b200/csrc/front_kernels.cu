@@ -87,14 +87,16 @@ __global__ void __launch_bounds__(FR_THREADS, 2) k_front(Tables t, StepPtr qp, S
 
 // ------------------------------------------------------------------ k_select
 
-constexpr int SL_THREADS = 1024;
-
-// One block per unit: see select_unit().
-__global__ void __launch_bounds__(SL_THREADS) k_select(Tables t, int budget, int* __restrict__ user_ids) {
-    __shared__ SelectSmem sm;
+// One block per unit: see select_unit().  Block size: 1024 threads when all units fit the GPU in one wave (the
+// shortest chain per block), 256 threads when there are more units than that (more blocks resident per SM; a
+// block's time is latency, not work).
+template <int THREADS>
+__global__ void __launch_bounds__(THREADS) k_select(Tables t, int budget, int* __restrict__ user_ids) {
+    extern __shared__ __align__(16) unsigned char sel_dyn[];
     __shared__ int s_last;
+    const SelectSmem sm = select_smem_at(sel_dyn, t.max_clusters);
     pdl_wait();                          // the scores come from the kernel before
-    select_unit<SL_THREADS>(t, blockIdx.x, budget, user_ids, sm);
+    select_unit<THREADS>(t, blockIdx.x, budget, user_ids, sm);
     // ---- With more units than the gather-attention CTAs keep in shared memory, the last unit block to finish lays
     // the units' work lists end to end (otherwise every attention CTA does that itself from n_work).
     if (!t.attn_pf_in_smem) {
@@ -107,7 +109,7 @@ __global__ void __launch_bounds__(SL_THREADS) k_select(Tables t, int budget, int
         __syncthreads();
         if (s_last) {
             __threadfence();
-            work_prefix_block<SL_THREADS>(t, sm.sh);
+            work_prefix_block<THREADS>(t, sm.sh);
             if (threadIdx.x == 0) *t.plan_counter = 0;
         }
     }
@@ -137,7 +139,9 @@ void launch_front(const Tables& t, StepPtr q, StepPtr k, int has_q, int has_k, c
 }
 
 void launch_select(const Tables& t, int budget, int* user_sel_ids, cudaStream_t s, long long* launches) {
-    launch_pdl(k_select, dim3(t.U), dim3(SL_THREADS), 0, s, t, budget, user_sel_ids);
+    const size_t smem = select_smem_bytes(t.max_clusters);
+    if (t.U <= t.n_attn_ctas) launch_pdl(k_select<1024>, dim3(t.U), dim3(1024), smem, s, t, budget, user_sel_ids);
+    else launch_pdl(k_select<256>, dim3(t.U), dim3(256), smem, s, t, budget, user_sel_ids);
     (*launches)++;
 }
 

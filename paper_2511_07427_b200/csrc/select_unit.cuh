@@ -15,14 +15,35 @@ namespace dkv {
 
 constexpr int SL_MAXM = 4096;          // most cluster ids a unit can have (dynakv_create enforces it)
 
+// The block's working set, carved out of shared memory by the caller: `ids` is the unit's id capacity
+// (max_clusters), so small configurations leave room for more resident blocks.
 struct SelectSmem {
-    unsigned int keys[SL_MAXM];        // orderable score of every cluster id (0 = dead / beyond the unit's ids)
-    int sizes[SL_MAXM];                // cluster sizes; the sign bit marks "selected" at the end
-    int hist[2048];
-    int sh[33];
-    int bin, rem, done, eqtake, eqcnt, L, tok;
-    unsigned long long best;
+    unsigned int* keys;                // [ids] orderable score of every cluster id (0 = dead / beyond the unit's ids)
+    int* sizes;                        // [ids] cluster sizes; the sign bit marks "selected" at the end
+    int* hist;                         // [2048]
+    int* sh;                           // [33]
+    int* sc;                           // [8] scalars, see the names below
+    unsigned long long* best64;        // [1]
 };
+#define SEL_bin sm.sc[0]
+#define SEL_rem sm.sc[1]
+#define SEL_done sm.sc[2]
+#define SEL_eqtake sm.sc[3]
+#define SEL_eqcnt sm.sc[4]
+#define SEL_L sm.sc[5]
+#define SEL_tok sm.sc[6]
+#define SEL_best (*sm.best64)
+__host__ __device__ inline size_t select_smem_bytes(int ids) { return (size_t)ids * 8 + 2048 * 4 + 48 * 4 + 8 + 16; }
+__device__ __forceinline__ SelectSmem select_smem_at(unsigned char* base, int ids) {      // base: 8-byte aligned
+    SelectSmem sm;
+    sm.best64 = reinterpret_cast<unsigned long long*>(base);
+    sm.keys = reinterpret_cast<unsigned int*>(base + 8);
+    sm.sizes = reinterpret_cast<int*>(sm.keys + ids);
+    sm.hist = sm.sizes + ids;
+    sm.sh = sm.hist + 2048;
+    sm.sc = sm.sh + 36;
+    return sm;
+}
 
 __device__ __forceinline__ unsigned int ord_key(float f) {
     unsigned int b = __float_as_uint(f);
@@ -33,7 +54,7 @@ __device__ __forceinline__ unsigned int ord_key(float f) {
 // by an earlier kernel).  user_ids (may be null): the selection in score order, -1 padded, [max_clusters].
 // On return (all global writes issued; no trailing barrier) thread 0 has written sel_n / sel_tokens / n_work.
 template <int THREADS>
-__device__ void select_unit(const Tables& t, int u, int budget, int* __restrict__ user_ids, SelectSmem& sm) {
+__device__ void select_unit(const Tables& t, int u, int budget, int* __restrict__ user_ids, const SelectSmem& sm) {
     const int tid = threadIdx.x;
     const float* SC = t.scores + (size_t)u * t.max_clusters;
     const int* CN = t.cl_n + (size_t)u * t.max_clusters;
@@ -53,7 +74,7 @@ __device__ void select_unit(const Tables& t, int u, int budget, int* __restrict_
             best = kk > best ? kk : best;
         }
     }
-    if (tid == 0) { sm.rem = budget; sm.done = 0; sm.eqtake = 0; sm.eqcnt = 0; sm.L = 0; sm.tok = 0; sm.best = 0ull; }
+    if (tid == 0) { SEL_rem = budget; SEL_done = 0; SEL_eqtake = 0; SEL_eqcnt = 0; SEL_L = 0; SEL_tok = 0; SEL_best = 0ull; }
     __syncthreads();
     // ---- radix select: digits [31:21], [20:10], [9:0]
     unsigned int prefix = 0u, pmask = 0u;
@@ -62,7 +83,7 @@ __device__ void select_unit(const Tables& t, int u, int budget, int* __restrict_
     for (int lvl = 0; lvl < 3; lvl++) {
         for (int b = tid; b < 2048; b += THREADS) sm.hist[b] = 0;
         __syncthreads();
-        if (sm.done) break;
+        if (SEL_done) break;
         const int nb = nbins[lvl];
         for (int j = tid; j < Mcur; j += THREADS) {
             const int sz = sm.sizes[j];
@@ -77,45 +98,45 @@ __device__ void select_unit(const Tables& t, int u, int budget, int* __restrict_
         for (int k = 0; k < BPT; k++) { const int b = nb - 1 - (tid * BPT + k); mine += b >= 0 ? sm.hist[b] : 0; }
         int tot;
         const int before = block_scan_excl(mine, sm.sh, &tot);   // weight of all bins above this thread's first
-        const int rem = sm.rem;
+        const int rem = SEL_rem;
         __syncthreads();
-        if (tid == 0 && tot <= rem) sm.done = 1;                 // everything under this prefix fits
+        if (tid == 0 && tot <= rem) SEL_done = 1;                 // everything under this prefix fits
         // the boundary bin is the first (from the top) whose inclusive suffix sum exceeds rem
         int acc = before;
 #pragma unroll
         for (int k = 0; k < BPT; k++) {
             const int b = nb - 1 - (tid * BPT + k);
             const int h = b >= 0 ? sm.hist[b] : 0;
-            if (b >= 0 && acc <= rem && acc + h > rem) { sm.bin = b; sm.rem = rem - acc; }
+            if (b >= 0 && acc <= rem && acc + h > rem) { SEL_bin = b; SEL_rem = rem - acc; }
             acc += h;
         }
         __syncthreads();
-        if (sm.done) break;
-        prefix |= (unsigned int)sm.bin << shifts[lvl];
+        if (SEL_done) break;
+        prefix |= (unsigned int)SEL_bin << shifts[lvl];
         pmask |= (unsigned int)(nb - 1) << shifts[lvl];
     }
     __syncthreads();
     // Selected: key above the boundary key; among clusters exactly at the boundary key, the lowest ids while
     // they still fit.  With `done` every key >= the current prefix range is in.
-    const bool all_in = sm.done != 0;
+    const bool all_in = SEL_done != 0;
     const unsigned int kb = prefix;
     if (!all_in) {
         // a single cluster at the boundary key cannot fit (its bin overflowed the remaining budget);
         // only with several equal scores does the id-order walk matter
         int ne = 0;
         for (int j = tid; j < Mcur; j += THREADS) ne += (sm.sizes[j] > 0 && sm.keys[j] == kb) ? 1 : 0;
-        if (ne) atomicAdd(&sm.eqcnt, ne);
+        if (ne) atomicAdd(&SEL_eqcnt, ne);
         __syncthreads();
-        if (tid == 0 && sm.eqcnt > 1) {
-            int rem = sm.rem, take = 0;
+        if (tid == 0 && SEL_eqcnt > 1) {
+            int rem = SEL_rem, take = 0;
             for (int j = 0; j < Mcur; j++)
                 if (sm.keys[j] == kb && sm.sizes[j] > 0) { if (sm.sizes[j] <= rem) { rem -= sm.sizes[j]; take++; } else break; }
-            sm.eqtake = take;
+            SEL_eqtake = take;
         }
     }
     __syncthreads();
     // When all_in, pmask covers the levels already fixed: keys matching the prefix there, or larger, are selected.
-    const int eqtake = sm.eqtake;
+    const int eqtake = SEL_eqtake;
     int selc = 0, tokc = 0;
     for (int j = tid; j < Mcur; j += THREADS) {
         const int sz = sm.sizes[j];
@@ -130,15 +151,15 @@ __device__ void select_unit(const Tables& t, int u, int budget, int* __restrict_
         }
         if (in) { selc++; tokc += sz; sm.sizes[j] = sz | (int)0x80000000; }
     }
-    if (selc) { atomicAdd(&sm.L, selc); atomicAdd(&sm.tok, tokc); }
-    if (best) atomicMax(&sm.best, best);
+    if (selc) { atomicAdd(&SEL_L, selc); atomicAdd(&SEL_tok, tokc); }
+    if (best) atomicMax(&SEL_best, best);
     __syncthreads();
-    int L = sm.L;
-    if (L == 0 && budget > 0 && sm.best != 0ull) {
+    int L = SEL_L;
+    if (L == 0 && budget > 0 && SEL_best != 0ull) {
         // not even the best cluster fits: take it alone
-        const int jb = (int)(0xffffffffu - (unsigned)(sm.best & 0xffffffffull));
+        const int jb = (int)(0xffffffffu - (unsigned)(SEL_best & 0xffffffffull));
         __syncthreads();
-        if (tid == 0) { sm.tok = sm.sizes[jb]; sm.sizes[jb] |= (int)0x80000000; atomicOr(t.status, DYNAKV_ST_BUDGET_EXCEEDED); }
+        if (tid == 0) { SEL_tok = sm.sizes[jb]; sm.sizes[jb] |= (int)0x80000000; atomicOr(t.status, DYNAKV_ST_BUDGET_EXCEEDED); }
         L = 1;
     }
     __syncthreads();
@@ -172,9 +193,9 @@ __device__ void select_unit(const Tables& t, int u, int budget, int* __restrict_
     }
     if (tid == 0) {
         t.sel_n[u] = L;
-        t.sel_tokens[u] = sm.tok;
+        t.sel_tokens[u] = SEL_tok;
         t.n_work[u] = min(tw, t.W);
-        atomicAdd(&t.counters[CNT_TOKENS_ATTENDED], (unsigned long long)sm.tok);
+        atomicAdd(&t.counters[CNT_TOKENS_ATTENDED], (unsigned long long)SEL_tok);
         atomicAdd(&t.counters[CNT_CLUSTERS_SELECTED], (unsigned long long)L);
     }
     if (user_ids) {
