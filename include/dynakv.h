@@ -134,8 +134,11 @@ int dynakv_split_check(dynakv_ctx* ctx);
  * of Algorithm 1's loop body), replayed from one captured CUDA graph whose kernels read
  * the step index from device memory.  q_steps: [n_steps][U][G][d] fp32, k_steps,
  * v_steps: [n_steps][U][d] kv_dtype, out_steps: [n_steps][U][G][d] fp32, all device.
- * The context must have been created on a non-default stream (stream capture), else
- * DYNAKV_ERR_STATE. */
+ * All n_steps inputs must be complete before the call: units are independent, so a unit's
+ * centroid pass for step t+1 (query scores, new key's distances) runs as soon as that
+ * unit's own append of step t is done, while other units may still be splitting; results
+ * are those of the stated order.  The context must have been created on a non-default
+ * stream (stream capture), else DYNAKV_ERR_STATE. */
 int dynakv_decode_loop(dynakv_ctx* ctx, const float* q_steps, const void* k_steps,
                        const void* v_steps, int64_t n_steps, int32_t token_budget,
                        float* out_steps);
