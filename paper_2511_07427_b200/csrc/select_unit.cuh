@@ -22,7 +22,7 @@ struct SelectSmem {
     int* sizes;                        // [ids] cluster sizes; the sign bit marks "selected" at the end
     int* hist;                         // [2048]
     int* sh;                           // [33]
-    int* sc;                           // [8] scalars, see the names below
+    int* sc;                           // [8] scalars: SEL_bin .. SEL_tok below
     unsigned long long* best64;        // [1]
 };
 #define SEL_bin sm.sc[0]
@@ -216,6 +216,15 @@ __device__ void select_unit(const Tables& t, int u, int budget, int* __restrict_
         for (int p = L + tid; p < t.max_clusters; p += THREADS) uo[p] = -1;
     }
 }
+
+#undef SEL_bin
+#undef SEL_rem
+#undef SEL_done
+#undef SEL_eqtake
+#undef SEL_eqcnt
+#undef SEL_L
+#undef SEL_tok
+#undef SEL_best
 
 // Exclusive prefix of the units' work-list lengths, by one block (after every unit's n_work is visible).
 template <int THREADS>

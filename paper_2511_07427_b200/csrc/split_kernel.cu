@@ -49,8 +49,9 @@ template <int HD, int KVB> struct SplitSmem {
 // tail_sync[0] = queue slots reserved, [1] = slots claimed by helpers, [2] = unit blocks that have decided.
 // A unit block with triggered clusters reserves a slot (two words) and stores a hint, then unit + 1, in it; a
 // helper claims slots in order.  The hint spares the helper two trips to memory in the common case of one
-// triggered cluster whose size the unit block knows: (cluster id + 1) | (size << 13), else 0.  Helpers never hold more than SP_HELPERS of the GPU's block slots, so the unit blocks they wait for
-// always get to run; all the same every wait here is bounded.
+// triggered cluster whose size the unit block knows: (cluster id + 1) | (size << 13), else 0.  Helpers never hold
+// more than SP_HELPERS of the GPU's block slots, so the unit blocks they wait for always get to run; all the same
+// every wait here is bounded.
 __device__ __forceinline__ int ld_acquire(const int* p) {
     int v;
     asm volatile("ld.acquire.gpu.global.s32 %0, [%1];\n" : "=r"(v) : "l"(p) : "memory");
@@ -249,324 +250,324 @@ __global__ void __launch_bounds__(SP_THREADS, DKV_SP_MINBLOCKS) k_split_check(Ta
             }
             __syncthreads();
         }
-    // Everything before this reads and writes only what the gather-attention kernel ahead never touches (statistics,
-    // the new row beyond every listed row, next step's scores); the splits move rows, so they wait for it.
-    if (ntrig > 0) pdl_wait();
-    KV* kpg = reinterpret_cast<KV*>(t.kpages) + (size_t)u * t.P * PAGE * HD;
-    KV* vpg = reinterpret_cast<KV*>(t.vpages) + (size_t)u * t.P * PAGE * HD;
-    int* ptok = t.page_tok + (size_t)u * t.P * PAGE;
-    int* pnext = t.page_next + (size_t)u * t.P;
-    unsigned char* label_g = t.sp_label + (size_t)u * t.max_tokens;
-    int* rank_g = t.sp_pos + (size_t)u * 2 * t.max_tokens;      // per position
-    int* holes_g = rank_g + t.max_tokens;                       // hole positions, in order
-    bool front_seen = false;             // helper: the unit's centroid pass of the next step is known to be complete
-    // Next step's scores and distances of the two children of a split, once the unit's own pass (which read the
-    // rows as they were before, or half-way through, the split) can no longer overwrite them.  ra / rb: the
-    // children's means (written before a block barrier).
-    auto patch_children = [&](int ja, const float* ra, int jb, const float* rb) {
-        if (!front_seen) {
-            if (tid == 0) {
-                int ok = 0;
-                const unsigned long long t_begin = global_ns();
-                for (int i = 0; i < (1 << 24); i++) {
-                    if (ld_acquire(t.front_done + u) == t0 + 1) { ok = 1; break; }
-                    __nanosleep(200);
-                    if ((i & 31) == 31 && global_ns() - t_begin > 500000000ull) break;
+        // Everything before this reads and writes only what the gather-attention kernel ahead never touches (statistics,
+        // the new row beyond every listed row, next step's scores); the splits move rows, so they wait for it.
+        if (ntrig > 0) pdl_wait();
+        KV* kpg = reinterpret_cast<KV*>(t.kpages) + (size_t)u * t.P * PAGE * HD;
+        KV* vpg = reinterpret_cast<KV*>(t.vpages) + (size_t)u * t.P * PAGE * HD;
+        int* ptok = t.page_tok + (size_t)u * t.P * PAGE;
+        int* pnext = t.page_next + (size_t)u * t.P;
+        unsigned char* label_g = t.sp_label + (size_t)u * t.max_tokens;
+        int* rank_g = t.sp_pos + (size_t)u * 2 * t.max_tokens;      // per position
+        int* holes_g = rank_g + t.max_tokens;                       // hole positions, in order
+        bool front_seen = false;             // helper: the unit's centroid pass of the next step is known to be complete
+        // Next step's scores and distances of the two children of a split, once the unit's own pass (which read the
+        // rows as they were before, or half-way through, the split) can no longer overwrite them.  ra / rb: the
+        // children's means (written before a block barrier).
+        auto patch_children = [&](int ja, const float* ra, int jb, const float* rb) {
+            if (!front_seen) {
+                if (tid == 0) {
+                    int ok = 0;
+                    const unsigned long long t_begin = global_ns();
+                    for (int i = 0; i < (1 << 24); i++) {
+                        if (ld_acquire(t.front_done + u) == t0 + 1) { ok = 1; break; }
+                        __nanosleep(200);
+                        if ((i & 31) == 31 && global_ns() - t_begin > 500000000ull) break;
+                    }
+                    if (!ok) atomicOr(t.status, DYNAKV_ST_INTERNAL);
+                    s_flag = ok;
                 }
-                if (!ok) atomicOr(t.status, DYNAKV_ST_INTERNAL);
-                s_flag = ok;
+                __syncthreads();
+                front_seen = true;
             }
-            __syncthreads();
-            front_seen = true;
-        }
-        if (s_flag && warp == 0) {
-            const float* q1 = reinterpret_cast<const float*>(next_q.at(t0 + 1)) + (size_t)u * t.G * HD;
-            const KV* k1 = reinterpret_cast<const KV*>(next_k.at(t0 + 1)) + (size_t)u * HD;
-            front_patch<KV, HD>(t, u, q1, k1, ja, ra, jb, rb);
-        }
-    };
-    SplitScratch sc;
-    sc.cA = cA; sc.cB = cB; sc.label = label_s; sc.rank = rank_s; sc.holes = holes_s; sc.tok = tok_s; sc.newpg = newpg;
-    sc.part = wsum; sc.nsplit = &s_nsplit;
-    KV* vrows = reinterpret_cast<KV*>(dynb + Lay::stage1_off(maxch, t.max_clusters));
-    for (int li = 0; li < ntrig; li++) {
-        const int j = trig[li];
-        const size_t cj = (size_t)u * t.max_clusters + j;
-        const int c = c_hint > 0 ? c_hint : t.cl_n[cj];
-        __syncthreads();    // previous cluster's work is complete
-        if (c <= CACHE_ROWS) {
-            // the common case: everything out of shared memory
-            int stay_side = 0;
-            const int nid = split_small<KV, HD, SP_THREADS, CACHE_ROWS>(t, u, j, c, iters, krows, vrows, sc, &stay_side);
-            if (nid >= 0 && helper && fronted) patch_children(j, stay_side ? cB : cA, nid, stay_side ? cA : cB);
-            continue;
-        }
-        if (t.u_M[u] >= t.max_clusters) { if (tid == 0) atomicOr(t.status, DYNAKV_ST_MAX_CLUSTERS); continue; }
-
-        const int npg = (c + PAGE - 1) / PAGE;
-        if (tid == 0) {
-            int p = t.cl_head[cj];
-            for (int i = 0; i < npg; i++) { chain[i] = p; p = pnext[p]; }
-        }
-        for (int e = tid; e < HD; e += SP_THREADS) cA[e] = t.cl_r[cj * HD + e];
-        __syncthreads();
-        const bool cached = c <= CACHE_ROWS;
-        if (cached) {
-            constexpr int V16 = HD * (int)sizeof(KV) / 16;      // 16-byte pieces per row
-            for (int idx = tid; idx < c * V16; idx += SP_THREADS) {
-                const int p = idx / V16, v = idx % V16;
-                const size_t row = (size_t)chain[p >> 5] * PAGE + (p & 31);
-                reinterpret_cast<uint4*>(krows + (size_t)p * HD)[v] = reinterpret_cast<const uint4*>(kpg + row * HD)[v];
+            if (s_flag && warp == 0) {
+                const float* q1 = reinterpret_cast<const float*>(next_q.at(t0 + 1)) + (size_t)u * t.G * HD;
+                const KV* k1 = reinterpret_cast<const KV*>(next_k.at(t0 + 1)) + (size_t)u * HD;
+                front_patch<KV, HD>(t, u, q1, k1, ja, ra, jb, rb);
             }
-            for (int p = tid; p < c; p += SP_THREADS) tok_s[p] = ptok[(size_t)chain[p >> 5] * PAGE + (p & 31)];
-            __syncthreads();
-        }
-        unsigned char* label = cached ? label_s : label_g;
-        int* rank_of = cached ? rank_s : rank_g;
-        int* holes = cached ? holes_s : holes_g;
-        // key row and token id of member position p
-        auto key_of = [&](int p) -> const KV* {
-            return cached ? krows + (size_t)p * HD : kpg + ((size_t)chain[p >> 5] * PAGE + (p & 31)) * HD;
         };
-        auto tok_of = [&](int p) -> int { return cached ? tok_s[p] : ptok[(size_t)chain[p >> 5] * PAGE + (p & 31)]; };
-
-        // ---- centre A: member farthest from r_j; centre B: member farthest from A (ties: lowest token id)
-        for (int round = 0; round < 2; round++) {
-            float cen[EPL];
-#pragma unroll
-            for (int e = 0; e < EPL; e++) cen[e] = cA[lane * EPL + e];
-            float bd = -1.f; int bt = 0x7fffffff, bp = -1;
-            for (int p = warp; p < c; p += SP_WARPS) {
-                const KV* k = key_of(p) + lane * EPL;
-                float part = 0.f;
-#pragma unroll
-                for (int e = 0; e < EPL; e++) { float df = to_f(k[e]) - cen[e]; part = fmaf(df, df, part); }
-                part = warp_sum(part);
-                int tok = tok_of(p);
-                if (part > bd || (part == bd && tok < bt)) { bd = part; bt = tok; bp = p; }
+        SplitScratch sc;
+        sc.cA = cA; sc.cB = cB; sc.label = label_s; sc.rank = rank_s; sc.holes = holes_s; sc.tok = tok_s; sc.newpg = newpg;
+        sc.part = wsum; sc.nsplit = &s_nsplit;
+        KV* vrows = reinterpret_cast<KV*>(dynb + Lay::stage1_off(maxch, t.max_clusters));
+        for (int li = 0; li < ntrig; li++) {
+            const int j = trig[li];
+            const size_t cj = (size_t)u * t.max_clusters + j;
+            const int c = c_hint > 0 ? c_hint : t.cl_n[cj];
+            __syncthreads();    // previous cluster's work is complete
+            if (c <= CACHE_ROWS) {
+                // the common case: everything out of shared memory
+                int stay_side = 0;
+                const int nid = split_small<KV, HD, SP_THREADS, CACHE_ROWS>(t, u, j, c, iters, krows, vrows, sc, &stay_side);
+                if (nid >= 0 && helper && fronted) patch_children(j, stay_side ? cB : cA, nid, stay_side ? cA : cB);
+                continue;
             }
-            if (lane == 0) { red_f[warp] = bd; red_i[warp] = bt; red_k[warp] = bp; }
-            __syncthreads();
+            if (t.u_M[u] >= t.max_clusters) { if (tid == 0) atomicOr(t.status, DYNAKV_ST_MAX_CLUSTERS); continue; }
+
+            const int npg = (c + PAGE - 1) / PAGE;
             if (tid == 0) {
-                float d0 = red_f[0]; int t0 = red_i[0], p0 = red_k[0];
-                for (int w = 1; w < SP_WARPS; w++)
-                    if (red_f[w] > d0 || (red_f[w] == d0 && red_i[w] < t0)) { d0 = red_f[w]; t0 = red_i[w]; p0 = red_k[w]; }
-                s_a = p0;
+                int p = t.cl_head[cj];
+                for (int i = 0; i < npg; i++) { chain[i] = p; p = pnext[p]; }
             }
+            for (int e = tid; e < HD; e += SP_THREADS) cA[e] = t.cl_r[cj * HD + e];
             __syncthreads();
-            {
-                const KV* src = key_of(s_a);
-                float* dst = (round == 0) ? cA : cB;
-                __syncthreads();
-                for (int e = tid; e < HD; e += SP_THREADS) dst[e] = to_f(src[e]);
+            const bool cached = c <= CACHE_ROWS;
+            if (cached) {
+                constexpr int V16 = HD * (int)sizeof(KV) / 16;      // 16-byte pieces per row
+                for (int idx = tid; idx < c * V16; idx += SP_THREADS) {
+                    const int p = idx / V16, v = idx % V16;
+                    const size_t row = (size_t)chain[p >> 5] * PAGE + (p & 31);
+                    reinterpret_cast<uint4*>(krows + (size_t)p * HD)[v] = reinterpret_cast<const uint4*>(kpg + row * HD)[v];
+                }
+                for (int p = tid; p < c; p += SP_THREADS) tok_s[p] = ptok[(size_t)chain[p >> 5] * PAGE + (p & 31)];
                 __syncthreads();
             }
-        }
-        // After round 0, cA = key A and the second round measured distances to cA: correct.
+            unsigned char* label = cached ? label_s : label_g;
+            int* rank_of = cached ? rank_s : rank_g;
+            int* holes = cached ? holes_s : holes_g;
+            // key row and token id of member position p
+            auto key_of = [&](int p) -> const KV* {
+                return cached ? krows + (size_t)p * HD : kpg + ((size_t)chain[p >> 5] * PAGE + (p & 31)) * HD;
+            };
+            auto tok_of = [&](int p) -> int { return cached ? tok_s[p] : ptok[(size_t)chain[p >> 5] * PAGE + (p & 31)]; };
 
-        // ---- 2-means rounds
-        for (int p = tid; p < c; p += SP_THREADS) label[p] = 255;
-        __syncthreads();
-        int nA = 0, nB = 0;
-        bool abandoned = false;
-        for (int it = 0; it < iters; it++) {
-            if (tid < 4) s_cnt[tid] = 0;
-            __syncthreads();
-            float a_c[EPL], b_c[EPL], sa[EPL], sb[EPL];
+            // ---- centre A: member farthest from r_j; centre B: member farthest from A (ties: lowest token id)
+            for (int round = 0; round < 2; round++) {
+                float cen[EPL];
 #pragma unroll
-            for (int e = 0; e < EPL; e++) { a_c[e] = cA[lane * EPL + e]; b_c[e] = cB[lane * EPL + e]; sa[e] = 0.f; sb[e] = 0.f; }
-            int chg = 0, ca = 0, cb = 0;
+                for (int e = 0; e < EPL; e++) cen[e] = cA[lane * EPL + e];
+                float bd = -1.f; int bt = 0x7fffffff, bp = -1;
+                for (int p = warp; p < c; p += SP_WARPS) {
+                    const KV* k = key_of(p) + lane * EPL;
+                    float part = 0.f;
+#pragma unroll
+                    for (int e = 0; e < EPL; e++) { float df = to_f(k[e]) - cen[e]; part = fmaf(df, df, part); }
+                    part = warp_sum(part);
+                    int tok = tok_of(p);
+                    if (part > bd || (part == bd && tok < bt)) { bd = part; bt = tok; bp = p; }
+                }
+                if (lane == 0) { red_f[warp] = bd; red_i[warp] = bt; red_k[warp] = bp; }
+                __syncthreads();
+                if (tid == 0) {
+                    float d0 = red_f[0]; int t0 = red_i[0], p0 = red_k[0];
+                    for (int w = 1; w < SP_WARPS; w++)
+                        if (red_f[w] > d0 || (red_f[w] == d0 && red_i[w] < t0)) { d0 = red_f[w]; t0 = red_i[w]; p0 = red_k[w]; }
+                    s_a = p0;
+                }
+                __syncthreads();
+                {
+                    const KV* src = key_of(s_a);
+                    float* dst = (round == 0) ? cA : cB;
+                    __syncthreads();
+                    for (int e = tid; e < HD; e += SP_THREADS) dst[e] = to_f(src[e]);
+                    __syncthreads();
+                }
+            }
+            // After round 0, cA = key A and the second round measured distances to cA: correct.
+
+            // ---- 2-means rounds
+            for (int p = tid; p < c; p += SP_THREADS) label[p] = 255;
+            __syncthreads();
+            int nA = 0, nB = 0;
+            bool abandoned = false;
+            for (int it = 0; it < iters; it++) {
+                if (tid < 4) s_cnt[tid] = 0;
+                __syncthreads();
+                float a_c[EPL], b_c[EPL], sa[EPL], sb[EPL];
+#pragma unroll
+                for (int e = 0; e < EPL; e++) { a_c[e] = cA[lane * EPL + e]; b_c[e] = cB[lane * EPL + e]; sa[e] = 0.f; sb[e] = 0.f; }
+                int chg = 0, ca = 0, cb = 0;
+                for (int p = warp; p < c; p += SP_WARPS) {
+                    const KV* k = key_of(p) + lane * EPL;
+                    float kk[EPL], da = 0.f, db = 0.f;
+#pragma unroll
+                    for (int e = 0; e < EPL; e++) {
+                        kk[e] = to_f(k[e]);
+                        float x = kk[e] - a_c[e], y = kk[e] - b_c[e];
+                        da = fmaf(x, x, da); db = fmaf(y, y, db);
+                    }
+                    da = warp_sum(da); db = warp_sum(db);
+                    const int l = db < da ? 1 : 0;
+                    if (lane == 0) { if (label[p] != l) chg = 1; label[p] = (unsigned char)l; if (l) cb++; else ca++; }
+#pragma unroll
+                    for (int e = 0; e < EPL; e++) { if (l) sb[e] += kk[e]; else sa[e] += kk[e]; }
+                }
+#pragma unroll
+                for (int e = 0; e < EPL; e++) { WS(warp, 0, lane * EPL + e) = sa[e]; WS(warp, 1, lane * EPL + e) = sb[e]; }
+                if (lane == 0) { if (chg) atomicOr(&s_cnt[0], 1); atomicAdd(&s_cnt[1], ca); atomicAdd(&s_cnt[2], cb); }
+                __syncthreads();
+                nA = s_cnt[1]; nB = s_cnt[2];
+                const int changed = s_cnt[0];
+                if (nA == 0 || nB == 0) { abandoned = true; break; }
+                if (!changed) break;
+                for (int e = tid; e < 2 * HD; e += SP_THREADS) {
+                    int side = e / HD, x = e % HD;
+                    float s = 0.f;
+                    for (int w = 0; w < SP_WARPS; w++) s += WS(w, side, x);
+                    if (side == 0) cA[x] = s / (float)nA; else cB[x] = s / (float)nB;
+                }
+                __syncthreads();
+            }
+            if (abandoned) { if (tid == 0) t.cl_flags[cj] |= FLAG_HOLD; continue; }
+
+            // ---- which side stays: the one holding the smallest token id
+            {
+                int bt = 0x7fffffff, bl = 0;
+                for (int p = tid; p < c; p += SP_THREADS) {
+                    int tok = tok_of(p);
+                    if (tok < bt) { bt = tok; bl = label[p]; }
+                }
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) {
+                    int ot = __shfl_xor_sync(0xffffffffu, bt, o), ol = __shfl_xor_sync(0xffffffffu, bl, o);
+                    if (ot < bt) { bt = ot; bl = ol; }
+                }
+                if (lane == 0) { red_i[warp] = bt; red_k[warp] = bl; }
+                __syncthreads();
+                if (tid == 0) {
+                    int t0 = red_i[0], l0 = red_k[0];
+                    for (int w = 1; w < SP_WARPS; w++) if (red_i[w] < t0) { t0 = red_i[w]; l0 = red_k[w]; }
+                    s_a = l0;
+                }
+                __syncthreads();
+            }
+            const int stay = s_a;
+            const int s_n = stay ? nB : nA, m_n = c - s_n;
+            const int need = (m_n + PAGE - 1) / PAGE, keep = (s_n + PAGE - 1) / PAGE;
+
+            // ---- pages for the moving child
+            if (tid == 0) {
+                int fc = t.u_free_cnt[u], top = t.u_page_top[u];
+                int ok = (fc + (t.P - top) >= need) ? 1 : 0;
+                if (ok) {
+                    for (int i = 0; i < need; i++) {
+                        int pg;
+                        if (fc > 0) pg = t.free_stack[(size_t)u * t.P + --fc]; else pg = top++;
+                        newpg[i] = pg;
+                    }
+                    t.u_free_cnt[u] = fc; t.u_page_top[u] = top;
+                } else atomicOr(t.status, DYNAKV_ST_PAGE_POOL);
+                s_ok = ok;
+            }
+            __syncthreads();
+            if (!s_ok) continue;
+            const int new_id = t.u_M[u];
+
+            // ---- ranks: movers in position order; fillers (stayers at positions >= s_n); holes (movers at positions < s_n)
+            int base_m = 0, base_f = 0, base_h = 0;
+            for (int b0 = 0; b0 < c; b0 += SP_THREADS) {
+                const int p = b0 + tid;
+                const int mv = (p < c && label[p] != stay) ? 1 : 0;
+                const int fl = (p < c && !mv && p >= s_n) ? 1 : 0;
+                const int hl = (p < c && mv && p < s_n) ? 1 : 0;
+                int tm, tf, th;
+                const int rm = base_m + block_scan_excl(mv, sh, &tm);
+                const int rf = base_f + block_scan_excl(fl, sh, &tf);
+                const int rh = base_h + block_scan_excl(hl, sh, &th);
+                if (p < c) rank_of[p] = mv ? rm : (fl ? rf : -1);
+                if (hl) holes[rh] = p;
+                base_m += tm; base_f += tf; base_h += th;
+            }
+            __syncthreads();
+
+            // ---- phase 1: movers go to the new pages (one warp per row)
             for (int p = warp; p < c; p += SP_WARPS) {
-                const KV* k = key_of(p) + lane * EPL;
-                float kk[EPL], da = 0.f, db = 0.f;
+                if (label[p] == stay) continue;
+                const int r = rank_of[p];
+                const size_t src = (size_t)chain[p >> 5] * PAGE + (p & 31);
+                const size_t dst = (size_t)newpg[r >> 5] * PAGE + (r & 31);
 #pragma unroll
                 for (int e = 0; e < EPL; e++) {
-                    kk[e] = to_f(k[e]);
-                    float x = kk[e] - a_c[e], y = kk[e] - b_c[e];
-                    da = fmaf(x, x, da); db = fmaf(y, y, db);
+                    kpg[dst * HD + lane * EPL + e] = kpg[src * HD + lane * EPL + e];
+                    vpg[dst * HD + lane * EPL + e] = vpg[src * HD + lane * EPL + e];
                 }
-                da = warp_sum(da); db = warp_sum(db);
-                const int l = db < da ? 1 : 0;
-                if (lane == 0) { if (label[p] != l) chg = 1; label[p] = (unsigned char)l; if (l) cb++; else ca++; }
-#pragma unroll
-                for (int e = 0; e < EPL; e++) { if (l) sb[e] += kk[e]; else sa[e] += kk[e]; }
-            }
-#pragma unroll
-            for (int e = 0; e < EPL; e++) { WS(warp, 0, lane * EPL + e) = sa[e]; WS(warp, 1, lane * EPL + e) = sb[e]; }
-            if (lane == 0) { if (chg) atomicOr(&s_cnt[0], 1); atomicAdd(&s_cnt[1], ca); atomicAdd(&s_cnt[2], cb); }
-            __syncthreads();
-            nA = s_cnt[1]; nB = s_cnt[2];
-            const int changed = s_cnt[0];
-            if (nA == 0 || nB == 0) { abandoned = true; break; }
-            if (!changed) break;
-            for (int e = tid; e < 2 * HD; e += SP_THREADS) {
-                int side = e / HD, x = e % HD;
-                float s = 0.f;
-                for (int w = 0; w < SP_WARPS; w++) s += WS(w, side, x);
-                if (side == 0) cA[x] = s / (float)nA; else cB[x] = s / (float)nB;
-            }
-            __syncthreads();
-        }
-        if (abandoned) { if (tid == 0) t.cl_flags[cj] |= FLAG_HOLD; continue; }
-
-        // ---- which side stays: the one holding the smallest token id
-        {
-            int bt = 0x7fffffff, bl = 0;
-            for (int p = tid; p < c; p += SP_THREADS) {
-                int tok = tok_of(p);
-                if (tok < bt) { bt = tok; bl = label[p]; }
-            }
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) {
-                int ot = __shfl_xor_sync(0xffffffffu, bt, o), ol = __shfl_xor_sync(0xffffffffu, bl, o);
-                if (ot < bt) { bt = ot; bl = ol; }
-            }
-            if (lane == 0) { red_i[warp] = bt; red_k[warp] = bl; }
-            __syncthreads();
-            if (tid == 0) {
-                int t0 = red_i[0], l0 = red_k[0];
-                for (int w = 1; w < SP_WARPS; w++) if (red_i[w] < t0) { t0 = red_i[w]; l0 = red_k[w]; }
-                s_a = l0;
-            }
-            __syncthreads();
-        }
-        const int stay = s_a;
-        const int s_n = stay ? nB : nA, m_n = c - s_n;
-        const int need = (m_n + PAGE - 1) / PAGE, keep = (s_n + PAGE - 1) / PAGE;
-
-        // ---- pages for the moving child
-        if (tid == 0) {
-            int fc = t.u_free_cnt[u], top = t.u_page_top[u];
-            int ok = (fc + (t.P - top) >= need) ? 1 : 0;
-            if (ok) {
-                for (int i = 0; i < need; i++) {
-                    int pg;
-                    if (fc > 0) pg = t.free_stack[(size_t)u * t.P + --fc]; else pg = top++;
-                    newpg[i] = pg;
+                if (lane == 0) {
+                    int tok = ptok[src];
+                    ptok[dst] = tok;
+                    t.tok_cluster[(size_t)u * t.max_tokens + tok] = new_id;
                 }
-                t.u_free_cnt[u] = fc; t.u_page_top[u] = top;
-            } else atomicOr(t.status, DYNAKV_ST_PAGE_POOL);
-            s_ok = ok;
-        }
-        __syncthreads();
-        if (!s_ok) continue;
-        const int new_id = t.u_M[u];
-
-        // ---- ranks: movers in position order; fillers (stayers at positions >= s_n); holes (movers at positions < s_n)
-        int base_m = 0, base_f = 0, base_h = 0;
-        for (int b0 = 0; b0 < c; b0 += SP_THREADS) {
-            const int p = b0 + tid;
-            const int mv = (p < c && label[p] != stay) ? 1 : 0;
-            const int fl = (p < c && !mv && p >= s_n) ? 1 : 0;
-            const int hl = (p < c && mv && p < s_n) ? 1 : 0;
-            int tm, tf, th;
-            const int rm = base_m + block_scan_excl(mv, sh, &tm);
-            const int rf = base_f + block_scan_excl(fl, sh, &tf);
-            const int rh = base_h + block_scan_excl(hl, sh, &th);
-            if (p < c) rank_of[p] = mv ? rm : (fl ? rf : -1);
-            if (hl) holes[rh] = p;
-            base_m += tm; base_f += tf; base_h += th;
-        }
-        __syncthreads();
-
-        // ---- phase 1: movers go to the new pages (one warp per row)
-        for (int p = warp; p < c; p += SP_WARPS) {
-            if (label[p] == stay) continue;
-            const int r = rank_of[p];
-            const size_t src = (size_t)chain[p >> 5] * PAGE + (p & 31);
-            const size_t dst = (size_t)newpg[r >> 5] * PAGE + (r & 31);
-#pragma unroll
-            for (int e = 0; e < EPL; e++) {
-                kpg[dst * HD + lane * EPL + e] = kpg[src * HD + lane * EPL + e];
-                vpg[dst * HD + lane * EPL + e] = vpg[src * HD + lane * EPL + e];
-            }
-            if (lane == 0) {
-                int tok = ptok[src];
-                ptok[dst] = tok;
-                t.tok_cluster[(size_t)u * t.max_tokens + tok] = new_id;
-            }
-        }
-        __syncthreads();
-        // ---- phase 2: stayers beyond position s_n fill the holes
-        for (int p = s_n + warp; p < c; p += SP_WARPS) {
-            if (label[p] != stay) continue;
-            const int h = holes[rank_of[p]];
-            const size_t src = (size_t)chain[p >> 5] * PAGE + (p & 31);
-            const size_t dst = (size_t)chain[h >> 5] * PAGE + (h & 31);
-#pragma unroll
-            for (int e = 0; e < EPL; e++) {
-                kpg[dst * HD + lane * EPL + e] = kpg[src * HD + lane * EPL + e];
-                vpg[dst * HD + lane * EPL + e] = vpg[src * HD + lane * EPL + e];
-            }
-            if (lane == 0) ptok[dst] = ptok[src];
-        }
-        __syncthreads();
-        // ---- phase 3: chains, ids, allocator
-        const size_t cn = (size_t)u * t.max_clusters + new_id;
-        if (tid == 0) {
-            pnext[chain[keep - 1]] = -1;
-            t.cl_tail[cj] = chain[keep - 1];
-            int fc = t.u_free_cnt[u];
-            for (int i = keep; i < npg; i++) t.free_stack[(size_t)u * t.P + fc++] = chain[i];
-            t.u_free_cnt[u] = fc;
-            for (int i = 0; i < need; i++) pnext[newpg[i]] = (i + 1 < need) ? newpg[i + 1] : -1;
-            t.cl_head[cn] = newpg[0]; t.cl_tail[cn] = newpg[need - 1];
-            t.cl_n[cj] = s_n; t.cl_n[cn] = m_n;
-            t.cl_flags[cj] = 0; t.cl_flags[cn] = 0;
-            t.u_M[u] = new_id + 1; t.u_Mlive[u] = t.u_Mlive[u] + 1;
-            atomicAdd(&t.counters[CNT_SPLITS], 1ull);
-            s_nsplit = s_nsplit + 1;
-        }
-        __syncthreads();
-        // ---- phase 4: exact statistics of both children (mean, then M2 about the mean)
-        for (int child = 0; child < 2; child++) {
-            const int cc = child == 0 ? s_n : m_n;
-            const int* pages = child == 0 ? chain : newpg;
-            const size_t cid = child == 0 ? cj : cn;
-            float sa[EPL];
-#pragma unroll
-            for (int e = 0; e < EPL; e++) sa[e] = 0.f;
-            // staged members of this child (by label) when the cluster was staged, else its rows in their new place
-            const int n_scan = cached ? c : cc;
-            for (int p = warp; p < n_scan; p += SP_WARPS) {
-                if (cached && ((label[p] == stay) != (child == 0))) continue;
-                const KV* k = (cached ? krows + (size_t)p * HD : kpg + ((size_t)pages[p >> 5] * PAGE + (p & 31)) * HD) + lane * EPL;
-#pragma unroll
-                for (int e = 0; e < EPL; e++) sa[e] += to_f(k[e]);
-            }
-#pragma unroll
-            for (int e = 0; e < EPL; e++) WS(warp, 0, lane * EPL + e) = sa[e];
-            __syncthreads();
-            for (int e = tid; e < HD; e += SP_THREADS) {
-                float s = 0.f;
-                for (int w = 0; w < SP_WARPS; w++) s += WS(w, 0, e);
-                s /= (float)cc;
-                cA[e] = s;
-                t.cl_r[cid * HD + e] = s;
             }
             __syncthreads();
-            float mean[EPL], m2 = 0.f;
+            // ---- phase 2: stayers beyond position s_n fill the holes
+            for (int p = s_n + warp; p < c; p += SP_WARPS) {
+                if (label[p] != stay) continue;
+                const int h = holes[rank_of[p]];
+                const size_t src = (size_t)chain[p >> 5] * PAGE + (p & 31);
+                const size_t dst = (size_t)chain[h >> 5] * PAGE + (h & 31);
 #pragma unroll
-            for (int e = 0; e < EPL; e++) mean[e] = cA[lane * EPL + e];
-            for (int p = warp; p < n_scan; p += SP_WARPS) {
-                if (cached && ((label[p] == stay) != (child == 0))) continue;
-                const KV* k = (cached ? krows + (size_t)p * HD : kpg + ((size_t)pages[p >> 5] * PAGE + (p & 31)) * HD) + lane * EPL;
-                float part = 0.f;
-#pragma unroll
-                for (int e = 0; e < EPL; e++) { float df = to_f(k[e]) - mean[e]; part = fmaf(df, df, part); }
-                m2 += warp_sum(part);
+                for (int e = 0; e < EPL; e++) {
+                    kpg[dst * HD + lane * EPL + e] = kpg[src * HD + lane * EPL + e];
+                    vpg[dst * HD + lane * EPL + e] = vpg[src * HD + lane * EPL + e];
+                }
+                if (lane == 0) ptok[dst] = ptok[src];
             }
-            if (lane == 0) red_f[warp] = m2;
             __syncthreads();
+            // ---- phase 3: chains, ids, allocator
+            const size_t cn = (size_t)u * t.max_clusters + new_id;
             if (tid == 0) {
-                float s = 0.f;
-                for (int w = 0; w < SP_WARPS; w++) s += red_f[w];
-                t.cl_M2[cid] = s;
+                pnext[chain[keep - 1]] = -1;
+                t.cl_tail[cj] = chain[keep - 1];
+                int fc = t.u_free_cnt[u];
+                for (int i = keep; i < npg; i++) t.free_stack[(size_t)u * t.P + fc++] = chain[i];
+                t.u_free_cnt[u] = fc;
+                for (int i = 0; i < need; i++) pnext[newpg[i]] = (i + 1 < need) ? newpg[i + 1] : -1;
+                t.cl_head[cn] = newpg[0]; t.cl_tail[cn] = newpg[need - 1];
+                t.cl_n[cj] = s_n; t.cl_n[cn] = m_n;
+                t.cl_flags[cj] = 0; t.cl_flags[cn] = 0;
+                t.u_M[u] = new_id + 1; t.u_Mlive[u] = t.u_Mlive[u] + 1;
+                atomicAdd(&t.counters[CNT_SPLITS], 1ull);
+                s_nsplit = s_nsplit + 1;
             }
             __syncthreads();
+            // ---- phase 4: exact statistics of both children (mean, then M2 about the mean)
+            for (int child = 0; child < 2; child++) {
+                const int cc = child == 0 ? s_n : m_n;
+                const int* pages = child == 0 ? chain : newpg;
+                const size_t cid = child == 0 ? cj : cn;
+                float sa[EPL];
+#pragma unroll
+                for (int e = 0; e < EPL; e++) sa[e] = 0.f;
+                // staged members of this child (by label) when the cluster was staged, else its rows in their new place
+                const int n_scan = cached ? c : cc;
+                for (int p = warp; p < n_scan; p += SP_WARPS) {
+                    if (cached && ((label[p] == stay) != (child == 0))) continue;
+                    const KV* k = (cached ? krows + (size_t)p * HD : kpg + ((size_t)pages[p >> 5] * PAGE + (p & 31)) * HD) + lane * EPL;
+#pragma unroll
+                    for (int e = 0; e < EPL; e++) sa[e] += to_f(k[e]);
+                }
+#pragma unroll
+                for (int e = 0; e < EPL; e++) WS(warp, 0, lane * EPL + e) = sa[e];
+                __syncthreads();
+                for (int e = tid; e < HD; e += SP_THREADS) {
+                    float s = 0.f;
+                    for (int w = 0; w < SP_WARPS; w++) s += WS(w, 0, e);
+                    s /= (float)cc;
+                    cA[e] = s;
+                    t.cl_r[cid * HD + e] = s;
+                }
+                __syncthreads();
+                float mean[EPL], m2 = 0.f;
+#pragma unroll
+                for (int e = 0; e < EPL; e++) mean[e] = cA[lane * EPL + e];
+                for (int p = warp; p < n_scan; p += SP_WARPS) {
+                    if (cached && ((label[p] == stay) != (child == 0))) continue;
+                    const KV* k = (cached ? krows + (size_t)p * HD : kpg + ((size_t)pages[p >> 5] * PAGE + (p & 31)) * HD) + lane * EPL;
+                    float part = 0.f;
+#pragma unroll
+                    for (int e = 0; e < EPL; e++) { float df = to_f(k[e]) - mean[e]; part = fmaf(df, df, part); }
+                    m2 += warp_sum(part);
+                }
+                if (lane == 0) red_f[warp] = m2;
+                __syncthreads();
+                if (tid == 0) {
+                    float s = 0.f;
+                    for (int w = 0; w < SP_WARPS; w++) s += red_f[w];
+                    t.cl_M2[cid] = s;
+                }
+                __syncthreads();
+            }
+            if (helper && fronted) patch_children(j, t.cl_r + cj * HD, new_id, t.cl_r + ((size_t)u * t.max_clusters + new_id) * HD);
         }
-        if (helper && fronted) patch_children(j, t.cl_r + cj * HD, new_id, t.cl_r + ((size_t)u * t.max_clusters + new_id) * HD);
-    }
         if (!helper) break;
         __syncthreads();
         if (tid == 0 && s_nsplit > 0) t.u_scan[u] = 1;
