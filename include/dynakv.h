@@ -144,8 +144,12 @@ int dynakv_decode_loop(dynakv_ctx* ctx, const float* q_steps, const void* k_step
                        float* out_steps);
 
 /* One loop iteration as above with HOST buffers (pinned memory recommended): copies
- * q, k, v to the device, runs the three calls, copies out back and synchronises the
- * stream.  q_host [U][G][d] fp32, k_host, v_host [U][d] kv_dtype, out_host [U][G][d]. */
+ * q, k, v to the device, runs the three calls and copies out back.  Returns when out_host
+ * holds the step's result; the step's append and split check may still be running on the
+ * context's stream then, and every later call on the context is ordered behind them (a call
+ * that synchronises, e.g. dynakv_get_status, sees them complete).  q_host, k_host, v_host
+ * must stay unchanged until the call returns.  q_host [U][G][d] fp32, k_host, v_host
+ * [U][d] kv_dtype, out_host [U][G][d]. */
 int dynakv_step_host(dynakv_ctx* ctx, const float* q_host, const void* k_host,
                      const void* v_host, int32_t token_budget, float* out_host);
 

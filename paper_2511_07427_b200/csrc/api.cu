@@ -42,6 +42,8 @@ struct dynakv_ctx {
     long long graph_nodes = 0;
     // staging for dynakv_step_host
     float* st_q = nullptr; void* st_k = nullptr; void* st_v = nullptr; float* st_out = nullptr;
+    cudaStream_t copy_stream = nullptr;      // carries the result copy of a host step past the step's append / split
+    cudaEvent_t ev_attended = nullptr;
     // optional per-kernel event timing (off inside graph capture)
     bool timing = false;
     struct Span { int kc; cudaEvent_t e0, e1; };
@@ -208,6 +210,8 @@ extern "C" int dynakv_create(const dynakv_config* cfg, void* cuda_stream, dynakv
 extern "C" void dynakv_destroy(dynakv_ctx* c) {
     if (!c) return;
     cudaStreamSynchronize(c->stream);
+    if (c->copy_stream) { cudaStreamSynchronize(c->copy_stream); cudaStreamDestroy(c->copy_stream); }
+    if (c->ev_attended) cudaEventDestroy(c->ev_attended);
     if (c->graph_exec) cudaGraphExecDestroy(c->graph_exec);
     if (c->graph_exec_long) cudaGraphExecDestroy(c->graph_exec_long);
     for (auto& sp : c->spans) { cudaEventDestroy(sp.e0); cudaEventDestroy(sp.e1); }
@@ -294,16 +298,6 @@ static void enqueue_append_apply(dynakv_ctx* c, StepPtr k, StepPtr v, bool timed
 }
 
 static const NextFront kNoNextFront = {0, StepPtr{nullptr, 0, nullptr}, StepPtr{nullptr, 0, nullptr}, nullptr};
-
-// One whole loop iteration in four launches: a single centroid pass serves both the query scores and the new
-// key's distances; selection; gather-attention with its combine; then append + split check in one kernel.
-static void enqueue_step(dynakv_ctx* c, StepPtr q, StepPtr k, StepPtr v, int budget, StepPtrW out, bool timed) {
-    enqueue_front(c, q, k, 1, 1, timed);
-    enqueue_retrieve(c, q, budget, out, nullptr, timed);
-    TimeScope ts(c, KC_SPLIT, timed);
-    launch_append_split(c->t, c->cfg.split_size_factor, c->cfg.split_var_factor > 0.f ? 1 : 0, c->cfg.split_min_size,
-                        c->cfg.split_iters, 1, k, v, nullptr, kNoNextFront, c->stream, &c->launches);
-}
 
 // One iteration of a captured loop in three launches.  The centroid pass of step t + 1 is part of the tail kernel
 // of step t (every unit's block runs it as soon as the unit's own append is done), so an iteration starts at the
@@ -419,10 +413,25 @@ extern "C" int dynakv_step_host(dynakv_ctx* c, const float* q_host, const void* 
     CK(cudaMemcpyAsync(c->st_q, q_host, qb, cudaMemcpyHostToDevice, c->stream));
     CK(cudaMemcpyAsync(c->st_k, k_host, kb, cudaMemcpyHostToDevice, c->stream));
     CK(cudaMemcpyAsync(c->st_v, v_host, kb, cudaMemcpyHostToDevice, c->stream));
-    enqueue_step(c, StepPtr{c->st_q, 0, nullptr}, StepPtr{c->st_k, 0, nullptr}, StepPtr{c->st_v, 0, nullptr},
-                 token_budget, StepPtrW{c->st_out, 0, nullptr}, true);
-    CK(cudaMemcpyAsync(out_host, c->st_out, qb, cudaMemcpyDeviceToHost, c->stream));
-    CK(cudaStreamSynchronize(c->stream));
+    // The result depends on the attention kernel only: its copy back runs on a second stream beside the step's
+    // append and split check, and the call returns when the result is on the host.  Whatever is called next on
+    // the context is ordered behind the append and split check by the context's stream.
+    if (!c->copy_stream) {
+        CK(cudaStreamCreateWithFlags(&c->copy_stream, cudaStreamNonBlocking));
+        CK(cudaEventCreateWithFlags(&c->ev_attended, cudaEventDisableTiming));
+    }
+    const StepPtr q{c->st_q, 0, nullptr}, k{c->st_k, 0, nullptr}, v{c->st_v, 0, nullptr};
+    enqueue_front(c, q, k, 1, 1, true);
+    enqueue_retrieve(c, q, token_budget, StepPtrW{c->st_out, 0, nullptr}, nullptr, true);
+    CK(cudaEventRecord(c->ev_attended, c->stream));
+    CK(cudaStreamWaitEvent(c->copy_stream, c->ev_attended, 0));
+    CK(cudaMemcpyAsync(out_host, c->st_out, qb, cudaMemcpyDeviceToHost, c->copy_stream));
+    {
+        TimeScope ts(c, KC_SPLIT, true);
+        launch_append_split(c->t, c->cfg.split_size_factor, c->cfg.split_var_factor > 0.f ? 1 : 0, c->cfg.split_min_size,
+                            c->cfg.split_iters, 1, k, v, nullptr, kNoNextFront, c->stream, &c->launches);
+    }
+    CK(cudaStreamSynchronize(c->copy_stream));
     return DYNAKV_OK;
 }
 
