@@ -13,7 +13,10 @@
 
 namespace dkv {
 
-constexpr int SP_THREADS = 512;
+#ifndef DKV_SP_THREADS
+#define DKV_SP_THREADS 512
+#endif
+constexpr int SP_THREADS = DKV_SP_THREADS;    // a multiple of 128 (one thread per (side, dimension) and per staged member)
 #ifndef DKV_SP_MINBLOCKS
 #define DKV_SP_MINBLOCKS 2          // blocks per SM the register budget is held to (a loop iteration wants all units resident)
 #endif
