@@ -108,17 +108,26 @@ __device__ __forceinline__ void tc_ld_wait() { asm volatile("tcgen05.wait::ld.sy
 
 constexpr int TC_D = 128;                 // head dimension = contraction length
 constexpr int TC_BM = 128;                // keys per item (one TMEM lane each)
-constexpr int TC_BN = 256;                // centres per accumulator
+#ifndef DKV_TC_BN
+#define DKV_TC_BN 256
+#endif
+constexpr int TC_BN = DKV_TC_BN;          // centres per accumulator: 256 (two accumulators) or 128 (four)
+constexpr int TC_NACC = 512 / TC_BN;      // accumulators in the 512 columns of tensor memory
+constexpr int TC_NB = (2 * 256) / TC_BN;  // centre-tile stages (128 KB of shared memory in all)
 constexpr int TC_A_BYTES = TC_BM * TC_D * 2;          // 32 KB: two [128 rows x 128 B] swizzle panels
-constexpr int TC_B_BYTES = TC_BN * TC_D * 2;          // 64 KB: two [256 rows x 128 B] swizzle panels
+constexpr int TC_B_BYTES = TC_BN * TC_D * 2;          // 64 KB or 32 KB: two [TC_BN rows x 128 B] swizzle panels
 constexpr int TC_XCHG_BYTES = 2 * 3 * TC_BM * 5 * 4;      // hand-over of (g1, g2, g3, j1, j2) between the drain groups
-constexpr int TC_SMEM_BYTES = 2 * TC_A_BYTES + 2 * TC_B_BYTES + 1024 /* alignment */ + 256 /* barriers */ + TC_XCHG_BYTES;
+constexpr int TC_SMEM_BYTES = 2 * TC_A_BYTES + TC_NB * TC_B_BYTES + 1024 /* alignment */ + 256 /* barriers */ + TC_XCHG_BYTES;
 #ifndef DKV_TC_GROUPS
 #define DKV_TC_GROUPS 4
 #endif
 constexpr int TC_GROUPS = DKV_TC_GROUPS;  // drain groups of four warps: 2 (one per accumulator) or 4 (two per accumulator, half the columns each)
 constexpr int TC_THREADS = 64 + 128 * TC_GROUPS;   // warp 0 loads, warp 1 issues MMAs, the rest drain the accumulators
-constexpr unsigned TC_TMEM_COLS = 512;    // two 256-column fp32 accumulators
+constexpr unsigned TC_TMEM_COLS = 512;    // TC_NACC fp32 accumulators of TC_BN columns
+// mbarriers: key block full / empty (2 each), centre stage full / empty (TC_NB each), accumulator full / empty
+constexpr int BAR_AF = 0, BAR_AE = 2, BAR_BF = 4, BAR_BE = 4 + TC_NB, BAR_CF = 4 + 2 * TC_NB, BAR_CE = BAR_CF + TC_NACC,
+              BAR_COUNT = BAR_CE + TC_NACC;
+static_assert((BAR_COUNT + 2) * 8 <= 256, "barrier block");
 
 // Shared-memory matrix descriptor of a K-major panel with 128-byte rows under the 128-byte swizzle:
 // start address / 16, leading offset unused (1), 1024 B between 8-row groups, descriptor version 1,
@@ -277,21 +286,19 @@ __global__ void __launch_bounds__(TC_THREADS, 1) k_tc_assign(const __grid_consta
     const unsigned base = (raw + 1023u) & ~1023u;                    // swizzle panels need 1024-byte alignment
     unsigned char* gen = tc_smem_raw + (base - raw);
     const unsigned sA = base, sB = base + 2 * TC_A_BYTES;
-    unsigned long long* bars = reinterpret_cast<unsigned long long*>(gen + 2 * TC_A_BYTES + 2 * TC_B_BYTES);
-    // barrier indices: 0,1 a_full; 2,3 a_empty; 4,5 b_full; 6,7 b_empty; 8,9 acc_full; 10,11 acc_empty
+    unsigned long long* bars = reinterpret_cast<unsigned long long*>(gen + 2 * TC_A_BYTES + TC_NB * TC_B_BYTES);
     auto bar = [&](int i) { return tc_smem_u32(&bars[i]); };
-    volatile unsigned* s_tmem = reinterpret_cast<volatile unsigned*>(&bars[12]);
-    volatile int* s_abort = reinterpret_cast<volatile int*>(&bars[13]);
-    float* xchg = reinterpret_cast<float*>(gen + 2 * TC_A_BYTES + 2 * TC_B_BYTES + 256);
+    volatile unsigned* s_tmem = reinterpret_cast<volatile unsigned*>(&bars[BAR_COUNT]);
+    volatile int* s_abort = reinterpret_cast<volatile int*>(&bars[BAR_COUNT + 1]);
+    float* xchg = reinterpret_cast<float*>(gen + 2 * TC_A_BYTES + TC_NB * TC_B_BYTES + 256);
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int NT = p.Mpad / TC_BN;
     const long long n_items = (long long)p.U * p.KB;
 
     if (tid == 0) {
-        for (int i = 0; i < 8; i++) tc_mbar_init(bar(i), 1);
-        tc_mbar_init(bar(8), 1); tc_mbar_init(bar(9), 1);
-        tc_mbar_init(bar(10), 2 * TC_GROUPS); tc_mbar_init(bar(11), 2 * TC_GROUPS);   // one arrival per draining warp
+        for (int i = 0; i < BAR_CE; i++) tc_mbar_init(bar(i), 1);
+        for (int i = 0; i < TC_NACC; i++) tc_mbar_init(bar(BAR_CE + i), 2 * TC_GROUPS);   // one arrival per draining warp of the accumulator
         *s_abort = 0;
         asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
     }
@@ -309,32 +316,33 @@ __global__ void __launch_bounds__(TC_THREADS, 1) k_tc_assign(const __grid_consta
         // =============================== TMA producer ===============================
         if (lane == 0) {
             long long ia = 0, tb = 0;
-            long long lastA[2] = {-1, -1}, lastB[2] = {-1, -1};
+            long long lastA[2] = {-1, -1}, lastB[TC_NB];
+            for (int i = 0; i < TC_NB; i++) lastB[i] = -1;
             for (long long it = blockIdx.x; it < n_items && !*s_abort; it += gridDim.x, ia++) {
                 const int u = (int)(it / p.KB), kb = (int)(it % p.KB);
                 const int ab = (int)(ia & 1);
-                if (!tc_mbar_wait(bar(2 + ab), (unsigned)((ia >> 1) & 1) ^ 1u)) { *s_abort = 1; break; }
-                tc_mbar_expect_tx(bar(ab), TC_A_BYTES);
+                if (!tc_mbar_wait(bar(BAR_AE + ab), (unsigned)((ia >> 1) & 1) ^ 1u)) { *s_abort = 1; break; }
+                tc_mbar_expect_tx(bar(BAR_AF + ab), TC_A_BYTES);
                 const int rowA = u * p.n + kb * TC_BM;
-                tc_tma_load_2d(sA + ab * TC_A_BYTES, &mapA, 0, rowA, bar(ab));
-                tc_tma_load_2d(sA + ab * TC_A_BYTES + TC_A_BYTES / 2, &mapA, 64, rowA, bar(ab));
+                tc_tma_load_2d(sA + ab * TC_A_BYTES, &mapA, 0, rowA, bar(BAR_AF + ab));
+                tc_tma_load_2d(sA + ab * TC_A_BYTES + TC_A_BYTES / 2, &mapA, 64, rowA, bar(BAR_AF + ab));
                 lastA[ab] = ia;
                 for (int nt = 0; nt < NT; nt++, tb++) {
-                    const int st = (int)(tb & 1);
-                    if (!tc_mbar_wait(bar(6 + st), (unsigned)((tb >> 1) & 1) ^ 1u)) { *s_abort = 1; break; }
-                    tc_mbar_expect_tx(bar(4 + st), TC_B_BYTES);
+                    const int st = (int)(tb % TC_NB);
+                    if (!tc_mbar_wait(bar(BAR_BE + st), (unsigned)((tb / TC_NB) & 1) ^ 1u)) { *s_abort = 1; break; }
+                    tc_mbar_expect_tx(bar(BAR_BF + st), TC_B_BYTES);
                     const int rowB = u * p.Mpad + nt * TC_BN;
-                    tc_tma_load_2d(sB + st * TC_B_BYTES, &mapB, 0, rowB, bar(4 + st));
-                    tc_tma_load_2d(sB + st * TC_B_BYTES + TC_B_BYTES / 2, &mapB, 64, rowB, bar(4 + st));
+                    tc_tma_load_2d(sB + st * TC_B_BYTES, &mapB, 0, rowB, bar(BAR_BF + st));
+                    tc_tma_load_2d(sB + st * TC_B_BYTES + TC_B_BYTES / 2, &mapB, 64, rowB, bar(BAR_BF + st));
                     lastB[st] = tb;
                 }
             }
             if (*s_abort) {
                 // let the copies already issued land before the shared memory can be reused
-                for (int i = 0; i < 2; i++) {
-                    if (lastA[i] >= 0) tc_mbar_wait(bar(i), (unsigned)((lastA[i] >> 1) & 1));
-                    if (lastB[i] >= 0) tc_mbar_wait(bar(4 + i), (unsigned)((lastB[i] >> 1) & 1));
-                }
+                for (int i = 0; i < 2; i++)
+                    if (lastA[i] >= 0) tc_mbar_wait(bar(BAR_AF + i), (unsigned)((lastA[i] >> 1) & 1));
+                for (int i = 0; i < TC_NB; i++)
+                    if (lastB[i] >= 0) tc_mbar_wait(bar(BAR_BF + i), (unsigned)((lastB[i] / TC_NB) & 1));
             }
         }
     } else if (warp == 1) {
@@ -343,23 +351,23 @@ __global__ void __launch_bounds__(TC_THREADS, 1) k_tc_assign(const __grid_consta
             long long ia = 0, tb = 0;
             for (long long it = blockIdx.x; it < n_items && !*s_abort; it += gridDim.x, ia++) {
                 const int ab = (int)(ia & 1);
-                if (!tc_mbar_wait(bar(ab), (unsigned)((ia >> 1) & 1))) { *s_abort = 1; break; }
+                if (!tc_mbar_wait(bar(BAR_AF + ab), (unsigned)((ia >> 1) & 1))) { *s_abort = 1; break; }
                 for (int nt = 0; nt < NT; nt++, tb++) {
-                    const int st = (int)(tb & 1);
-                    if (!tc_mbar_wait(bar(4 + st), (unsigned)((tb >> 1) & 1)) ||
-                        !tc_mbar_wait(bar(10 + st), (unsigned)((tb >> 1) & 1) ^ 1u)) { *s_abort = 1; break; }
+                    const int st = (int)(tb % TC_NB), ac = (int)(tb % TC_NACC);
+                    if (!tc_mbar_wait(bar(BAR_BF + st), (unsigned)((tb / TC_NB) & 1)) ||
+                        !tc_mbar_wait(bar(BAR_CE + ac), (unsigned)((tb / TC_NACC) & 1) ^ 1u)) { *s_abort = 1; break; }
                     tc_fence_after();
 #pragma unroll
                     for (int k = 0; k < TC_D / 16; k++) {
                         const unsigned a_addr = sA + ab * TC_A_BYTES + (k >> 2) * (TC_A_BYTES / 2) + (k & 3) * 32;
                         const unsigned b_addr = sB + st * TC_B_BYTES + (k >> 2) * (TC_B_BYTES / 2) + (k & 3) * 32;
-                        tc_mma_f16(tmem + st * TC_BN, tc_panel_desc(a_addr), tc_panel_desc(b_addr), TC_IDESC, k > 0 ? 1u : 0u);
+                        tc_mma_f16(tmem + ac * TC_BN, tc_panel_desc(a_addr), tc_panel_desc(b_addr), TC_IDESC, k > 0 ? 1u : 0u);
                     }
-                    tc_commit(bar(6 + st));       // centre tile may be overwritten
-                    tc_commit(bar(8 + st));       // accumulator is complete
+                    tc_commit(bar(BAR_BE + st));  // centre tile may be overwritten
+                    tc_commit(bar(BAR_CF + ac));  // accumulator is complete
                 }
                 if (*s_abort) break;
-                tc_commit(bar(2 + ab));           // key block may be overwritten
+                tc_commit(bar(BAR_AE + ab));      // key block may be overwritten
             }
         }
     } else {
@@ -371,7 +379,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) k_tc_assign(const __grid_consta
         // them into its best two (with indices) and third value; at the end of an item the other groups hand
         // their triples to group 0 through shared memory, and group 0 decides.
         const int grp = (warp - 2) >> 2;              // drain group
-        const int my_st = grp & 1;                    // accumulator this group drains
+        const int team = grp & 1;                     // tiles of this parity are this group's (accumulators team, team + 2, ...)
         constexpr int CPG = (TC_BN / 32) / (TC_GROUPS / 2);   // 32-column chunks per group and tile
         const int c_first = (grp >> 1) * CPG;         // first chunk of this group's column range
         const int q = warp & 3;                       // TMEM lane quarter this warp may read
@@ -386,9 +394,9 @@ __global__ void __launch_bounds__(TC_THREADS, 1) k_tc_assign(const __grid_consta
             const float2 sc = p.scale[u];
             const float m2S = -2.f * sc.x;
             for (int nt = 0; nt < NT; nt++, tb++) {
-                const int st = (int)(tb & 1);
-                if (st != my_st) continue;
-                if (*s_abort || !tc_mbar_wait(bar(8 + st), (unsigned)((tb >> 1) & 1))) { *s_abort = 1; dead = true; break; }
+                if ((int)(tb & 1) != team) continue;
+                const int st = (int)(tb % TC_NACC);
+                if (*s_abort || !tc_mbar_wait(bar(BAR_CF + st), (unsigned)((tb / TC_NACC) & 1))) { *s_abort = 1; dead = true; break; }
                 tc_fence_after();
                 float ch[4][3];                                        // four independent chains of three smallest
 #pragma unroll
@@ -427,7 +435,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) k_tc_assign(const __grid_consta
                 }
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) tc_mbar_arrive(bar(10 + st));          // accumulator may be overwritten
+                if (lane == 0) tc_mbar_arrive(bar(BAR_CE + st));      // accumulator may be overwritten
                 // the tile's three smallest out of the four chains
                 tc_merge3(ch[0], ch[1]);
                 tc_merge3(ch[2], ch[3]);
