@@ -96,6 +96,9 @@ __device__ __forceinline__ void append_block(const Tables& t, int u, StepPtr kp_
         t.page_tok[((size_t)u * t.P + page) * PAGE + row] = N;
         t.tok_cluster[(size_t)u * t.max_tokens + N] = bj;
         t.u_N[u] = N + 1;
+        // an append whose split check is still owed, to another cluster: the next check has to scan them all
+        const int owed = t.u_last[u];
+        if (owed >= 0 && owed != bj) t.u_scan[u] = 1;
         t.u_last[u] = bj;
         atomicAdd(&t.counters[CNT_APPENDED], 1ull);
     }

@@ -150,13 +150,15 @@ __global__ void __launch_bounds__(SP_THREADS, DKV_SP_MINBLOCKS) k_split_check(Ta
             fr_issue = front_unit_begin<HD, SP_THREADS>(t, u, fr_stages, fr_bars, fr_live);
         }
         // what the trigger test needs and the append does not change: loaded ahead of the append's own chain of loads
-        const int full = t.u_scan[u];
+        const int owed = t.u_last[u];            // an earlier append whose check is still owed (-1 in a loop's steady state)
+        int full = t.u_scan[u];
         const int Mlive0 = t.u_Mlive[u];
         const float tau = t.u_tau[u];
         // fused loop iteration: the step's append for this unit comes first (Algorithm 1's order)
         if (do_append) append_block<KV, HD>(t, u, app_k, app_v, &s_app);
         __syncthreads();
-        const int last = do_append ? s_app.cluster : t.u_last[u];
+        const int last = do_append ? s_app.cluster : owed;
+        if (do_append && owed >= 0 && owed != last) full = 1;
         if (!full && do_append) {
             // Only the cluster that took the append can have become triggered (for every other cluster n_j and M2_j
             // are unchanged while N only grew), and the append has just computed its new statistics.

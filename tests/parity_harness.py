@@ -90,9 +90,10 @@ def check_state(o: O.OracleUnit, st: dict, ui: int, rep: ParityReport, where: st
 
 def run_parity(cfg: WorkloadConfig, units: Sequence[int], steps: int, *, assign_mode: int = 0,
                state_every: int = 1, budget: Optional[int] = None, ctx_units: Optional[Sequence[int]] = None,
-               seed: int = 1234, device: str = "cuda") -> ParityReport:
+               seed: int = 1234, device: str = "cuda", check_every: int = 1) -> ParityReport:
     """Run `steps` decode iterations of `cfg`.  The GPU context holds `ctx_units` (default:
-    `units`); the oracle follows the units listed in `units` (a subset of ctx_units)."""
+    `units`); the oracle follows the units listed in `units` (a subset of ctx_units).  With check_every > 1 the
+    split check is called only after every check_every-th append (on both sides)."""
     rep = ParityReport()
     ctx_units = list(ctx_units) if ctx_units is not None else list(units)
     pos = {u: i for i, u in enumerate(ctx_units)}
@@ -150,6 +151,8 @@ def run_parity(cfg: WorkloadConfig, units: Sequence[int], steps: int, *, assign_
                              hint_cluster=int(st["tok_cluster"][ui, n0]))
                 assert o.violations == v0 and j == int(st["tok_cluster"][ui, n0]), \
                     f"step {done + t} unit {ui}: append target gpu {st['tok_cluster'][ui, n0]} oracle {j}"
+            if (done + t + 1) % check_every != 0:
+                continue
             ctx.split_check()
             st = ctx.export_state()
             for ui in watch:

@@ -89,6 +89,17 @@ def test_few_clusters_long_chains_and_capacity_bits():
     assert rep.status_bits & P.ST_MAX_CLUSTERS
 
 
+def test_split_check_owed_for_several_appends():
+    # The split check runs only after every third append: clusters that took the earlier appends must still be
+    # examined (the oracle examines every cluster at every check).  Few clusters and a size trigger of 1.5 x the
+    # mean make "an append pushes its cluster over the threshold, and it is not the last append before the check"
+    # happen several times in this run (a library that examines only the last appended cluster fails it).
+    cfg = CONFIGS[2].scaled(n_prefill=120, steps=399, M0=6, max_clusters=128, budget=120, T=3, split_min_size=4,
+                            split_size_factor=1.5, split_var_factor=0.0)
+    rep = _run(cfg, [0, 1, 2, 3], cfg.steps, assign_mode=1, check_every=3, state_every=30)
+    assert rep.gpu_splits >= 8
+
+
 def _single_ctx(cfg, K, V, **kw):
     from parity_harness import make_ctx
     ctx = make_ctx(cfg, K.shape[0], trace=0, **kw)
