@@ -240,7 +240,8 @@ def test_graph_loop_fp32_d64_and_more_triggered_units_than_helpers():
     # steps: more hand-overs than there are helper blocks
     cfg = CONFIGS[1].scaled(B=1, L=1, Hkv=48, Hq=48 * CONFIGS[1].G, n_prefill=256, steps=20, M0=6, max_clusters=40,
                             budget=96, T=3, split_min_size=4, split_size_factor=1.2)
-    assert _loop_vs_direct(cfg, list(range(48)), 20, modes=("direct", "graph")) > 48
+    # first call of one step only: the loop's single iteration has no next step to prepare
+    assert _loop_vs_direct(cfg, list(range(48)), 20, modes=("direct", "graph"), cut=1) > 48
 
 
 def test_wrong_call_order_and_shapes():
