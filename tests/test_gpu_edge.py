@@ -244,6 +244,14 @@ def test_graph_loop_fp32_d64_and_more_triggered_units_than_helpers():
     assert _loop_vs_direct(cfg, list(range(48)), 20, modes=("direct", "graph"), cut=1) > 48
 
 
+def test_graph_loop_with_more_units_than_block_slots():
+    # 1100 units: the tail kernel's unit blocks run in several waves with the helper blocks last, the selection
+    # runs with 256-thread blocks and its last block lays out the work lists (more than 1024 units)
+    cfg = CONFIGS[2].scaled(B=1, L=1, Hkv=1100, Hq=1100 * CONFIGS[2].G, n_prefill=96, steps=12, M0=6, max_clusters=24,
+                            budget=64, T=2, split_min_size=4, split_size_factor=1.3)
+    assert _loop_vs_direct(cfg, list(range(1100)), 12, modes=("direct", "graph"), cut=5) > 100
+
+
 def test_wrong_call_order_and_shapes():
     cfg = P.DynaKVConfig(n_units=1, gqa_group=2, head_dim=64, kv_dtype=P.F32, max_tokens=64, max_clusters=8)
     ctx = P.DynaKV(cfg)
