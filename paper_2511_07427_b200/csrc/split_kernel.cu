@@ -599,8 +599,14 @@ template <typename KV, int HD>
 static void split_t(const Tables& t, float gamma, int var_enabled, int min_size, int iters, int do_append, StepPtr k, StepPtr v,
                     int* step_ctr, const NextFront& nf, cudaStream_t s) {
     const size_t dyn = SplitSmem<HD, (int)sizeof(KV)>::total(t.max_tokens / PAGE + 2, t.max_clusters);
-    if (dyn > 32 * 1024)
+    // the opt-in to more than 48 KB of dynamic shared memory: once per size, device and kernel instance
+    static size_t opted[64] = {0};
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (dyn > 32 * 1024 && (dev < 0 || dev >= 64 || opted[dev] != dyn)) {
         cudaFuncSetAttribute(k_split_check<KV, HD>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn);
+        if (dev >= 0 && dev < 64) opted[dev] = dyn;
+    }
     launch_pdl(k_split_check<KV, HD>, dim3(t.U + (nf.on ? SP_HELPERS : 0)), dim3(SP_THREADS), dyn, s, t, gamma, var_enabled, min_size, iters, do_append, k, v, step_ctr,
                nf.on, nf.q, nf.k, nf.step_lim);
 }
