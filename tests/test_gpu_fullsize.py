@@ -1,5 +1,5 @@
-"""Config 4 at its full size (256 units x 32768 keys, 1024 clusters, budget 2048), in the launch configuration
-that bench.py times (tensor-core build, one launch per kernel for all units, CUDA-graph decode loop), checked on
+"""Configs 2 to 5 at their full sizes (config 4: 256 units x 32768 keys, 1024 clusters, budget 2048; config 5: 1792
+units), in the launch configuration that bench.py times (tensor-core build, one launch per kernel for all units, CUDA-graph decode loop), checked on
 sampled units.  The oracle's own k-means would take minutes per unit at this size, so it continues from the
 library's partition (installed, with representatives and M2 recomputed from the members, which checks Eq. 4 and
 the statistics on the way) and then follows every decode call exactly as in the small parity runs."""
@@ -14,12 +14,12 @@ from parity_harness import (TOL_OUT_ABS, TOL_OUT_L2, ParityReport, check_state, 
 
 pytestmark = pytest.mark.gpu
 
-SAMPLED = [0, 101, 255]
 DIRECT_STEPS, GRAPH_STEPS = 3, 3
 
 
-def test_config4_full_size_sampled_units():
-    cfg = CONFIGS[4]
+@pytest.mark.parametrize("cid,SAMPLED", [(4, [0, 101, 255]), (2, [0, 77, 255]), (3, [0, 130, 255]), (5, [0, 900, 1791])])
+def test_full_size_sampled_units(cid, SAMPLED):
+    cfg = CONFIGS[cid]
     U, n = cfg.U, cfg.n_prefill
     side = torch.cuda.Stream()
     with torch.cuda.stream(side):
@@ -98,7 +98,7 @@ def test_config4_full_size_first_assignment_sampled_keys():
     st = ctx.export_state()
     status = ctx.get_status()
     rng = np.random.default_rng(9)
-    for u in SAMPLED:
+    for u in [0, 101, 255]:
         Ku = K[u].double().cpu().numpy()
         picks = O.init_random(n, M, 4321, unit=u)
         C0 = Ku[picks]
