@@ -14,7 +14,7 @@ from parity_harness import (TOL_OUT_ABS, TOL_OUT_L2, ParityReport, check_state, 
 
 pytestmark = pytest.mark.gpu
 
-DIRECT_STEPS, GRAPH_STEPS = 3, 3
+DIRECT_STEPS, GRAPH_STEPS = 3, 13
 
 
 @pytest.mark.parametrize("cid,SAMPLED", [(4, [0, 101, 255]), (2, [0, 77, 255]), (3, [0, 130, 255]), (5, [0, 900, 1791])])
@@ -81,6 +81,39 @@ def test_full_size_sampled_units(cid, SAMPLED):
         for u in SAMPLED:
             check_state(oracles[u], st, u, rep, f"after the graph loop, unit {u}")
         assert status["error_bits"] & (P.ST_INTERNAL | P.ST_PAGE_POOL | P.ST_MAX_TOKENS) == 0
+        # ---- properties that must hold for EVERY unit, sampled or not (Eq. 3 and Eq. 4 on the final state): every token
+        # in exactly one live cluster, sizes equal to the membership counts, representatives equal to the member means,
+        # M2 equal to the members' squared distances to them
+        steps = DIRECT_STEPS + GRAPH_STEPS
+        K_all = torch.cat([K, k[:steps].transpose(0, 1)], dim=1)                  # [U, n + steps, d]
+        Mx, nt = cfg.max_clusters, n + steps
+        assert np.all(st["n_tokens"] == nt)
+        tokc = torch.from_numpy(st["tok_cluster"][:, :nt].astype(np.int64)).cuda()
+        counts = torch.from_numpy(st["counts"].astype(np.int64)).cuda()
+        cent = torch.from_numpy(st["centroids"]).cuda().double()
+        M2 = torch.from_numpy(st["M2"]).cuda().double()
+        n_ids = torch.from_numpy(st["n_ids"].astype(np.int64)).cuda()
+        assert int(tokc.min()) >= 0 and bool((tokc < n_ids[:, None]).all())
+        worst_c, worst_m = 0.0, 0.0
+        for u0 in range(0, U, 64):
+            u1 = min(U, u0 + 64)
+            nu = u1 - u0
+            gid = (torch.arange(nu, device="cuda")[:, None] * Mx + tokc[u0:u1]).reshape(-1)
+            Kd = K_all[u0:u1].double().reshape(-1, cfg.d)
+            cnt = torch.zeros(nu * Mx, dtype=torch.int64, device="cuda").index_add_(0, gid, torch.ones_like(gid))
+            assert torch.equal(cnt.reshape(nu, Mx), counts[u0:u1]), "sizes differ from the membership counts"
+            sums = torch.zeros((nu * Mx, cfg.d), dtype=torch.float64, device="cuda").index_add_(0, gid, Kd)
+            live = cnt > 0
+            mean = sums[live] / cnt[live][:, None]
+            cg = cent[u0:u1].reshape(nu * Mx, cfg.d)[live]
+            err = ((cg - mean).norm(dim=1) / mean.norm(dim=1).clamp_min(1e-30)).max()
+            worst_c = max(worst_c, float(err))
+            m2 = torch.zeros(nu * Mx, dtype=torch.float64, device="cuda").index_add_(0, gid, ((Kd - sums[gid] / cnt[gid][:, None]) ** 2).sum(1))
+            mg = M2[u0:u1].reshape(-1)[live]
+            scale = m2[live].clamp_min(1e-6)
+            worst_m = max(worst_m, float(((mg - m2[live]).abs() / scale).max()))
+        assert worst_c <= 1e-4, f"representatives differ from the member means: {worst_c:.2e}"
+        assert worst_m <= 2e-3, f"M2 differs from the members' spread: {worst_m:.2e}"
         assert status["assign_rechecked"] < 0.1 * U * n * cfg.T          # the filter decides most keys
         ctx.destroy()
 
