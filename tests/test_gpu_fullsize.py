@@ -114,6 +114,44 @@ def test_full_size_sampled_units(cid, SAMPLED):
             worst_m = max(worst_m, float(((mg - m2[live]).abs() / scale).max()))
         assert worst_c <= 1e-4, f"representatives differ from the member means: {worst_c:.2e}"
         assert worst_m <= 2e-3, f"M2 differs from the members' spread: {worst_m:.2e}"
+        # ---- one more decode step on that state, checked for EVERY unit against plain torch: the selection is a score
+        # prefix that fills the budget (Section 4.1), and the output is softmax attention over exactly the selected
+        # clusters' tokens (Section 2.1)
+        V_all = torch.cat([V, v[:steps].transpose(0, 1)], dim=1)
+        qx = q[steps - 1]
+        out = ctx.decode_step(qx, cfg.budget, selected_ids=sel)
+        nsel, ntok = ctx.get_selection()
+        nsel_t = torch.from_numpy(nsel.astype(np.int64)).cuda()
+        selmask = torch.zeros((U, Mx + 1), dtype=torch.bool, device="cuda")
+        selmask.scatter_(1, torch.where(sel >= 0, sel.long(), torch.full_like(sel, Mx).long()), True)
+        selmask = selmask[:, :Mx]
+        assert torch.equal(selmask.sum(1), nsel_t)
+        live = counts > 0
+        assert bool((selmask <= live).all())
+        tok_sel = (counts * selmask).sum(1)
+        assert torch.equal(tok_sel.cpu(), torch.from_numpy(ntok.astype(np.int64)))
+        assert bool(((tok_sel <= cfg.budget) | (nsel_t == 1)).all())
+        sc = torch.einsum("ud,umd->um", qx.double().mean(1), cent)
+        s_sel_min = torch.where(selmask, sc, torch.full_like(sc, float("inf"))).min(1).values
+        rest = live & ~selmask
+        s_rest = torch.where(rest, sc, torch.full_like(sc, float("-inf")))
+        s_rest_max, j_rest = s_rest.max(1)
+        has_rest = rest.any(1)
+        tol = 1e-5 * sc.abs().max(1).values + 1e-12
+        assert bool((~has_rest | (s_rest_max <= s_sel_min + tol)).all()), "an unselected cluster scores above a selected one"
+        next_fits = tok_sel + counts.gather(1, j_rest[:, None])[:, 0] <= cfg.budget
+        near_tie = (s_sel_min - s_rest_max).abs() <= tol
+        assert bool((~has_rest | ~next_fits | near_tie | (nsel_t == 1)).all()), "the selection stops before the budget is filled"
+        worst_o = 0.0
+        for u0 in range(0, U, 32):
+            u1 = min(U, u0 + 32)
+            tm = selmask[u0:u1].gather(1, tokc[u0:u1])                                   # [nu, nt] token attended?
+            lg = torch.einsum("ugd,utd->ugt", qx[u0:u1].float(), K_all[u0:u1].float()) / float(np.sqrt(cfg.d))
+            lg = lg.masked_fill(~tm[:, None, :], float("-inf"))
+            ref = torch.einsum("ugt,utd->ugd", torch.softmax(lg, dim=2), V_all[u0:u1].float())
+            ref = torch.where(tm.any(1)[:, None, None], ref, torch.zeros_like(ref))
+            worst_o = max(worst_o, float((out[u0:u1] - ref).abs().max()))
+        assert worst_o <= TOL_OUT_ABS, f"attention over the selected tokens: max abs {worst_o:.3e}"
         assert status["assign_rechecked"] < 0.1 * U * n * cfg.T          # the filter decides most keys
         ctx.destroy()
 
