@@ -18,7 +18,9 @@
  *
  * Pins (tests, CPU only): brute-force argmin, inertia monotonicity, blob recovery,
  * scikit-learn Lloyd cross-check, D^2-sampling frequencies, Welford vs two-pass,
- * full-budget retrieval == dense softmax attention, split invariants.
+ * full-budget retrieval == dense softmax attention, split invariants, the round cap of
+ * the split's 2-means (hand-worked fixture), validity of a selection hint (including the
+ * over-budget single-cluster case).
  * Conventions the paper leaves open (score metric, GQA reduction, threshold
  * calibration, split seeding, id rule, budget boundary) are "parity unpinned" by the
  * paper: they are pinned only to their stated definitions.
@@ -287,7 +289,9 @@ void ork_score(const ork_unit *u, const double *q, double *scores) {
  * With a hint (another implementation's ordered selection) the hint is accepted, and a
  * tie counted, if it is a valid answer up to `tol` on the scores: non-increasing up to
  * tol, within budget, no unselected cluster scoring above the last selected one by more
- * than tol, and some unselected cluster tied for next place does not fit. */
+ * than tol, and some unselected cluster tied for next place does not fit.  A hint that
+ * exceeds the budget is valid only as one cluster that ties the best live score, when the
+ * oracle's own answer is the over-budget case as well. */
 int ork_select(ork_unit *u, const double *scores, int budget, const int *hint_ids, int hint_n,
                int *out_ids, int *out_tokens) {
     int M = u->M, nsel = 0, tokens = 0;
@@ -318,16 +322,26 @@ int ork_select(ork_unit *u, const double *scores, int budget, const int *hint_id
                 if (a > 0) {
                     double sp = scores[hint_ids[a - 1]], sc = scores[j];
                     if (sc > sp && !near_tie(sc, sp, u->tol)) ok = 0;
-                    if (sc == sp && j < hint_ids[a - 1]) { /* equal scores out of id order: still a tie */ }
                 }
             }
-            if (ok && htok > budget && !(hint_n == 1)) ok = 0;
+            int over = ok && htok > budget;
+            if (over) {
+                /* Over budget: valid only as the "best cluster taken alone" case.  The hint must be a single
+                 * cluster, the oracle's own answer must be that case too, and the hinted cluster must tie the
+                 * best live score. */
+                int own_over = (nsel == 1 && tokens > budget);
+                if (hint_n != 1 || !own_over) ok = 0;
+                else {
+                    double sh = scores[hint_ids[0]], sb = scores[out_ids[0]];
+                    if (!(sh == sb || near_tie(sh, sb, u->tol))) ok = 0;
+                }
+            }
             if (ok && hint_n == 0) {
                 /* nothing selected: valid only if nothing fits at the top */
                 int any = 0; for (int j = 0; j < M; j++) any |= u->live[j];
                 if (any && budget > 0) ok = 0;
             }
-            if (ok && hint_n > 0 && !(hint_n == 1 && htok > budget)) {
+            if (ok && hint_n > 0 && !over) {
                 double slast = scores[hint_ids[hint_n - 1]];
                 double snext = -INFINITY; int have = 0;
                 for (int j = 0; j < M; j++)

@@ -429,6 +429,69 @@ def test_select_hint_validation():
     assert list(ids) == [1, 0] and u.violations == 2
 
 
+def _unit_with_sizes(sizes):
+    """A unit whose cluster j holds sizes[j] copies of the 1-D key 10 * j (three Lloyd rounds from the first keys
+    of a seed that picks one key per value)."""
+    K = np.concatenate([np.full(s, 10.0 * j) for j, s in enumerate(sizes)])[:, None]
+    M = len(sizes)
+    for seed in range(2000):
+        picks = O.init_random(len(K), M, seed, 0)
+        if len({K[p, 0] for p in picks}) == M:
+            break
+    else:
+        raise AssertionError("no seed found")
+    u = O.OracleUnit(1, 1, len(K) + 2, M + 2, gamma=0, alpha=0)
+    u.build(K, K, M, 2, seed=seed, init_mode=O.INIT_RANDOM)
+    assert sorted(u.counts()) == sorted(sizes)
+    # cluster ids follow the picks' order, not the values: map value -> id
+    ids = {int(round(u.centroids()[j, 0] / 10.0)): j for j in range(M)}
+    return u, ids
+
+
+def test_select_hint_of_one_over_budget_cluster_is_checked():
+    # three clusters of 3 tokens, scores (3, 2, 1), budget 2: nothing fits, the best cluster is taken alone.
+    # A hint naming the worst cluster alone is over budget too, but it is not the best: a violation.
+    u, ids = _unit_with_sizes([3, 3, 3])
+    s = np.zeros(3); s[ids[0]], s[ids[1]], s[ids[2]] = 3.0, 2.0, 1.0
+    own, tok = u.select(s, 2)
+    assert list(own) == [ids[0]] and tok == 3
+    got, _ = u.select(s, 2, hint_ids=[ids[2]])
+    assert list(got) == [ids[0]] and u.violations == 1 and u.ties == 0
+    # the same over-budget answer with a near-tied score is a tie
+    s2 = s.copy(); s2[ids[1]] = 3.0 - 1e-8
+    got, _ = u.select(s2, 2, hint_ids=[ids[1]])
+    assert list(got) == [ids[1]] and u.violations == 1 and u.ties == 1
+    # sizes (2, 9, 2), budget 5: the two small clusters fit (4 tokens); the 9-token, lowest-scoring cluster
+    # alone is no valid answer
+    u, ids = _unit_with_sizes([2, 9, 2])
+    s = np.zeros(3); s[ids[0]], s[ids[1]], s[ids[2]] = 3.0, 1.0, 2.0
+    own, tok = u.select(s, 5)
+    assert list(own) == [ids[0], ids[2]] and tok == 4
+    got, tok = u.select(s, 5, hint_ids=[ids[1]])
+    assert list(got) == [ids[0], ids[2]] and tok == 4 and u.violations == 1 and u.ties == 0
+    # an over-budget hint of one cluster that DOES tie the best score, while the oracle's own answer is within
+    # budget, is not an answer the selection rule can give either
+    s3 = s.copy(); s3[ids[1]] = 3.0
+    got, _ = u.select(s3, 5, hint_ids=[ids[1]])
+    assert u.violations == 2
+
+
+def test_two_means_round_cap_hand_worked_fixture():
+    """The round cap of the split's local clustering: with split_iters = 1 or 2 the partition is the capped one,
+    not the converged one (hand-worked in the fixture)."""
+    g = _gold("two_means_cap_1d.txt")
+    K = g["members"][:, None]
+    for cap in (1, 2, 3, 8):
+        u = O.OracleUnit(1, 1, 16, 4, gamma=0.5, alpha=0, split_min_size=2, split_iters=cap)
+        u.build(K, K, 1, 1, seed=0, init_mode=O.INIT_RANDOM)
+        assert u.split_check() == 1
+        assert list(u.assign()) == list(g[f"assign_cap{cap}"].astype(int)), f"cap {cap}"
+        if f"centres_cap{cap}" in g:
+            # children's representatives are the member means of the final labels (UpdateStats)
+            assert np.allclose(u.centroids()[:2, 0], g[f"centres_cap{cap}"], atol=1e-12)
+    assert not np.array_equal(g["assign_cap1"], g["assign_cap2"]) and not np.array_equal(g["assign_cap2"], g["assign_cap8"])
+
+
 def test_two_means_equidistant_member_goes_to_centre_a():
     # members 0, 10, 5 around r = 5: A = token 0 (first of the two farthest), B = token 1;
     # token 2 is equidistant and must join A, so the moved child is {10} alone.
