@@ -95,21 +95,21 @@ int dynakv_create(const dynakv_config* cfg, void* cuda_stream, dynakv_ctx** out)
  * (squared Euclidean, ties to the lowest id) and mean update (an empty cluster keeps its
  * centre).  Then the members of each cluster are stored contiguously in 32-token pages
  * (Section 5.1, intra-cluster placement), n_j, r_j and M2_j = sum ||k - r_j||^2 are
- * initialised (Algorithm 1, "Initialize cluster size, centroid, variance") and the unit's
+ * initialised (Algorithm 1, the initialisation of size, centroid and variance) and the unit's
  * variance threshold tau is set.  Token id = row index.  Requires
  * n_clusters <= n <= max_tokens, n_clusters <= max_clusters, d == head_dim.
  * May be called once per context. */
 int dynakv_build_index(dynakv_ctx* ctx, const void* K, const void* V, int64_t n, int32_t d,
                        int32_t n_clusters, uint64_t seed);
 
-/* Algorithm 1, "Assign new KV entry to its nearest cluster", UpdateVar, AddEntry,
+/* Algorithm 1, nearest-cluster assignment of the new entry, UpdateVar, AddEntry,
  * UpdateStats: for every unit, the new key k [U][d] joins the live cluster with the
  * nearest representative; n_j, r_j, M2_j are updated incrementally and the (k, v) row is
  * written into the tail page of that cluster (no existing entry moves).  The new token id
  * is the unit's token count before the call. */
 int dynakv_append(dynakv_ctx* ctx, const void* k, const void* v);
 
-/* Section 4.1 / Algorithm 1 "Load top-k clusters by query-centroid similarity", then
+/* Section 4.1 / Algorithm 1, retrieval of the top clusters by query-centroid similarity, then
  * attention over the retrieved entries only (Section 2.1).  q: [U][G][d] fp32.
  * score_j = mean over the G heads of q_g . r_j; clusters are taken in (score descending,
  * id ascending) order while their sizes sum to <= token_budget (the best cluster is taken

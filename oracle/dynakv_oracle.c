@@ -162,7 +162,7 @@ void ork_assign(const double *K, int n, int d, const double *C, int M, const uns
 }
 
 /* c_j = mean of the keys assigned to j (Eq. 4).  A cluster with no member keeps its
- * previous centre (the reading taken for "robust to empty-cluster cases", Section 7). */
+ * previous centre (the reading taken for Section 7's remark that the k-means copes with empty clusters). */
 void ork_update(const double *K, int n, int d, const int *assign, int M, double *C, int *cnt) {
     double *sum = (double *)calloc((size_t)M * d, sizeof(double));
     for (int j = 0; j < M; j++) cnt[j] = 0;
@@ -227,7 +227,7 @@ static void recompute_stats(ork_unit *u, int j) {
     free(sum);
 }
 
-/* Prefill (Algorithm 1, "build the initial partition"): init, then exactly T rounds of
+/* Prefill (Algorithm 1, NewCluster on the prefill cache): init, then exactly T rounds of
  * assign + update; membership is the T-th assignment and the representatives are its
  * means, so Eq. 4 holds exactly.  Clusters empty at the end are dead: never scored,
  * never appended to; their ids stay reserved.  The unit's variance threshold is
@@ -268,8 +268,8 @@ int ork_build(ork_unit *u, const double *K, const double *V, int n, int n_cluste
 
 /* ------------------------------------------------------ decode: score, select */
 
-/* s_j = (1/G) sum_g q_g . r_j for live clusters ("similarity scores between q and all
- * representatives", Section 4.1).  Inner product, averaged over the G query heads that
+/* s_j = (1/G) sum_g q_g . r_j for live clusters (Section 4.1: the query is scored against
+ * every representative).  Inner product, averaged over the G query heads that
  * share this KV head so the group retrieves one set.  Dead clusters get -infinity. */
 void ork_score(const ork_unit *u, const double *q, double *scores) {
     int d = u->d;
@@ -284,7 +284,7 @@ void ork_score(const ork_unit *u, const double *q, double *scores) {
 /* Top clusters under a token budget: order live clusters by (score descending, id
  * ascending) and take the longest prefix whose sizes sum to <= budget; if the first
  * cluster alone is larger it is taken whole and BUDGET_EXCEEDED is raised (the budget
- * form of the paper's top-k active set, Section 4.1 / Algorithm 1 "Load top-k clusters").
+ * form of the paper's top-k active set, Section 4.1 / Algorithm 1, the step that loads the top clusters).
  * Returns the selection in that order.
  * With a hint (another implementation's ordered selection) the hint is accepted, and a
  * tie counted, if it is a valid answer up to `tol` on the scores: non-increasing up to
@@ -369,8 +369,8 @@ int ork_select(ork_unit *u, const double *scores, int budget, const int *hint_id
 
 /* ------------------------------------------------------ decode: attention */
 
-/* Attention restricted to the retrieved entries (Section 2.1, "only the most relevant KV
- * entries ... are accessed"): for each of the G heads, logits q_g.k_i / sqrt(d) over the
+/* Attention restricted to the retrieved entries (Section 2.1: attention reads
+ * only the retrieved part of the cache): for each of the G heads, logits q_g.k_i / sqrt(d) over the
  * members of the selected clusters (token-id order), softmax, weighted sum of values.
  * Written as the definition: max, exponentials, normalise.  Empty selection -> zeros. */
 void ork_attend(const ork_unit *u, const double *q, const int *ids, int n_ids, double *out) {
@@ -415,11 +415,11 @@ int ork_decode_step(ork_unit *u, const double *q, int budget, const int *hint_id
 
 /* ------------------------------------------------------ decode: append */
 
-/* Algorithm 1, "Assign new KV entry to its nearest cluster", UpdateVar, AddEntry,
+/* Algorithm 1, the nearest-cluster assignment of the new entry, UpdateVar, AddEntry,
  * UpdateStats: nearest live representative in squared Euclidean distance, then the
  * incremental mean / sum-of-squares update
  *     n <- n+1;  delta = k - r;  r <- r + delta/n;  M2 <- M2 + delta.(k - r_new),
- * which is what "computed from the centroid, the variance, and the new entry" allows.
+ * which needs only the centroid, the running sum of squares and the new entry, as Section 4.2 says the update should.
  * Returns the cluster id, or -1 if the unit is full. */
 int ork_append(ork_unit *u, const double *k, const double *v, int hint_cluster) {
     int d = u->d;
@@ -455,9 +455,8 @@ int ork_append(ork_unit *u, const double *k, const double *v, int hint_cluster) 
 
 /* ------------------------------------------------------ decode: split check */
 
-/* SplitCluster (Algorithm 1; Section 4.2 "a local clustering algorithm is executed";
- * Section 5.2 "split into two new clusters ... one continues to grow from the original
- * head, the other is migrated").  Two-means over the members of cluster j, members in
+/* SplitCluster (Algorithm 1; Section 4.2: a flagged cluster is re-clustered locally; Section 5.2: one child keeps
+ * growing where the parent was, the other is written elsewhere).  Two-means over the members of cluster j, members in
  * token-id order: centre A = the member farthest from r_j, centre B = the member
  * farthest from A; at most split_iters rounds of (label by nearer centre, ties to A;
  * recompute the two means), stopping early when no label changes.  labels[m] = 0 for A,

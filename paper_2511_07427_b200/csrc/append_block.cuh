@@ -1,6 +1,6 @@
 // The append of one decode step for one unit, as a block-level device function shared by the stand-alone
 // append kernel and by the split-check kernel of the fused loop iteration (arXiv 2511.07427, Algorithm 1:
-// "Assign new KV entry to its nearest cluster", UpdateVar, AddEntry, UpdateStats).
+// nearest-cluster assignment of the new entry, UpdateVar, AddEntry, UpdateStats).
 #pragma once
 
 #include "common.cuh"

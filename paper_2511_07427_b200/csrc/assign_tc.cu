@@ -588,13 +588,16 @@ bool tc_assign_begin(const Tables& t, const void* K, long long n, int M, void* s
     if (cudaMemcpyAsync(&h_bad, bad, sizeof(int), cudaMemcpyDeviceToHost, s) != cudaSuccess) return false;
     if (cudaStreamSynchronize(s) != cudaSuccess) return false;
     if (h_bad) return false;
-    static bool attr_set = false;
-    if (!attr_set) {
+    // the opt-in to more than 48 KB of dynamic shared memory is a per-device attribute of the kernel
+    static bool opted[64] = {false};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return false; }
+    if (dev < 0 || dev >= 64 || !opted[dev]) {
         if (cudaFuncSetAttribute(k_tc_assign, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_SMEM_BYTES) != cudaSuccess) {
             cudaGetLastError();
             return false;
         }
-        attr_set = true;
+        if (dev >= 0 && dev < 64) opted[dev] = true;
     }
     return true;
 }

@@ -402,10 +402,13 @@ template <typename KV, int HD>
 static void assign_f32_t(const Tables& t, const void* K, long long n, int M, const float* C, int* assign,
                          const int* list, const unsigned* counts, unsigned long long* listed_total,
                          cudaStream_t s, long long* launches) {
-    static bool attr_set = false;
-    if (!attr_set) {
+    // the opt-in to more than 48 KB of dynamic shared memory is a per-device attribute of the kernel instance
+    static bool opted[64] = {false};
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (dev < 0 || dev >= 64 || !opted[dev]) {
         cudaFuncSetAttribute(k_assign_f32<KV, HD>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)AssignSmem<HD>::bytes);
-        attr_set = true;
+        if (dev >= 0 && dev < 64) opted[dev] = true;
     }
     dim3 grid((unsigned)((n + AS_BK - 1) / AS_BK), t.U);
     k_assign_f32<KV, HD><<<grid, AS_THREADS, AssignSmem<HD>::bytes, s>>>((const KV*)K, (int)n, M, C, assign, list, counts,

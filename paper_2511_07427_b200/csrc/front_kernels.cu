@@ -1,8 +1,8 @@
 // Front half of a decode step (arXiv 2511.07427, Section 4.1 and Algorithm 1):
 //   k_front          one streaming pass over the fp32 representatives that produces both
-//                    the query scores ("similarity scores between q and all
-//                    representatives") and the new key's squared distances ("assign new KV
-//                    entry to its nearest cluster"), so the centroid table is read once;
+//                    the query's score against every representative and the new key's
+//                    squared distance to every representative (for its nearest-cluster
+//                    assignment), so the centroid table is read once;
 //   k_select         budgeted top-cluster selection by weighted radix select on the scores,
 //                    then the flat (page, rows) work list of the selected clusters;
 //   k_append_apply   argmin of the distances, incremental statistics, slot claim.

@@ -13,6 +13,7 @@
 // instead of from cluster pages, and the split-K partial records (acc, m, l) -- the scratch
 // memory of that kernel pair -- live in a file-scope __device__ array of fixed size that every
 // GPU loading the library carries until the process exits.
+#include <atomic>
 #include <float.h>
 
 #include "common.cuh"
@@ -147,25 +148,26 @@ using namespace dkv;
 // Device address of the scratch array, looked up once per device (with that device current).
 static float* na_scratch_for_current_device(int* rc) {
     constexpr int MAX_DEV = 64;
-    static float* ptr[MAX_DEV] = {nullptr};
+    // threads may race to fill a device's slot; they all store the same address, and the slot is atomic
+    static std::atomic<float*> ptr[MAX_DEV];
     int dev = -1;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess || dev < 0 || dev >= MAX_DEV) {
         *rc = DYNAKV_ERR_CUDA;
         return nullptr;
     }
-    if (!ptr[dev]) {
-        float* p = nullptr;
+    float* p = ptr[dev].load(std::memory_order_acquire);
+    if (!p) {
         e = cudaGetSymbolAddress((void**)&p, g_noalloc_scratch);
         if (e != cudaSuccess || !p) {
             cudaGetLastError();
             *rc = DYNAKV_ERR_CUDA;
             return nullptr;
         }
-        ptr[dev] = p;
+        ptr[dev].store(p, std::memory_order_release);
     }
     *rc = DYNAKV_OK;
-    return ptr[dev];
+    return p;
 }
 
 extern "C" int dynakv_attend_rows_noalloc(const float* q, const void* K, const void* V, int32_t n_units, int64_t n,
@@ -180,6 +182,8 @@ extern "C" int dynakv_attend_rows_noalloc(const float* q, const void* K, const v
     float* scratch = na_scratch_for_current_device(&rc);
     if (!scratch) return rc;
     cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
+    // an error left behind by an earlier, unrelated call on this thread must not be reported as this call's
+    cudaGetLastError();
     if (kv_dtype == DYNAKV_F32) {
         if (d == 64) na_launch<float, 64>(q, K, V, n_units, n, gqa_group, scratch, out, st);
         else na_launch<float, 128>(q, K, V, n_units, n, gqa_group, scratch, out, st);

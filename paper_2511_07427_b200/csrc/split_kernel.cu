@@ -1,7 +1,6 @@
 // Split check: Algorithm 1's split decision and SplitCluster of arXiv 2511.07427
-// (Section 4.2 "a local clustering algorithm is executed", Section 5.2 "one of the
-// resulting sub-clusters continues to grow from the original head, the other is
-// migrated").  One block per unit walks the unit's clusters in ascending id; a triggered
+// (Section 4.2: a flagged cluster is re-clustered locally; Section 5.2: one child keeps
+// growing where the parent was and the other is written elsewhere).  One block per unit walks the unit's clusters in ascending id; a triggered
 // cluster is 2-means-partitioned, the staying child is compacted inside the pages it
 // already owns, and the moving child is written to fresh pages under the next free id.
 #include <float.h>
@@ -52,7 +51,7 @@ template <int HD, int KVB> struct SplitSmem {
 // tail_sync[0] = queue slots reserved, [1] = slots claimed by helpers, [2] = unit blocks that have decided.
 // A unit block with triggered clusters reserves a slot (two words) and stores a hint, then unit + 1, in it; a
 // helper claims slots in order.  The hint spares the helper two trips to memory in the common case of one
-// triggered cluster whose size the unit block knows: (cluster id + 1) | (size << 13), else 0.  Helpers never hold
+// triggered cluster whose size the unit block knows and that has fewer than 2^18 members: (cluster id + 1) | (size << 13), else 0.  Helpers never hold
 // more than SP_HELPERS of the GPU's block slots, so the unit blocks they wait for always get to run; all the same
 // every wait here is bounded.
 __device__ __forceinline__ int ld_acquire(const int* p) {
@@ -212,7 +211,7 @@ __global__ void __launch_bounds__(SP_THREADS, DKV_SP_MINBLOCKS) k_split_check(Ta
                 if (ntrig > 0) {
                     const int slot = atomicAdd(t.tail_sync + 0, 1);
                     int hint = 0;
-                    if (ntrig == 1 && !full && do_append && s_app.cluster == trig[0]) hint = (trig[0] + 1) | (s_app.n_new << 13);
+                    if (ntrig == 1 && !full && do_append && s_app.cluster == trig[0] && s_app.n_new < (1 << 18)) hint = (trig[0] + 1) | (s_app.n_new << 13);
                     t.tail_queue[2 * slot] = hint;
                     __threadfence();
                     atomicExch(t.tail_queue + 2 * slot + 1, u + 1);
@@ -316,25 +315,13 @@ __global__ void __launch_bounds__(SP_THREADS, DKV_SP_MINBLOCKS) k_split_check(Ta
             }
             for (int e = tid; e < HD; e += SP_THREADS) cA[e] = t.cl_r[cj * HD + e];
             __syncthreads();
-            const bool cached = c <= CACHE_ROWS;
-            if (cached) {
-                constexpr int V16 = HD * (int)sizeof(KV) / 16;      // 16-byte pieces per row
-                for (int idx = tid; idx < c * V16; idx += SP_THREADS) {
-                    const int p = idx / V16, v = idx % V16;
-                    const size_t row = (size_t)chain[p >> 5] * PAGE + (p & 31);
-                    reinterpret_cast<uint4*>(krows + (size_t)p * HD)[v] = reinterpret_cast<const uint4*>(kpg + row * HD)[v];
-                }
-                for (int p = tid; p < c; p += SP_THREADS) tok_s[p] = ptok[(size_t)chain[p >> 5] * PAGE + (p & 31)];
-                __syncthreads();
-            }
-            unsigned char* label = cached ? label_s : label_g;
-            int* rank_of = cached ? rank_s : rank_g;
-            int* holes = cached ? holes_s : holes_g;
+            // general path (the cluster does not fit the staging area): every pass walks the pages
+            unsigned char* label = label_g;
+            int* rank_of = rank_g;
+            int* holes = holes_g;
             // key row and token id of member position p
-            auto key_of = [&](int p) -> const KV* {
-                return cached ? krows + (size_t)p * HD : kpg + ((size_t)chain[p >> 5] * PAGE + (p & 31)) * HD;
-            };
-            auto tok_of = [&](int p) -> int { return cached ? tok_s[p] : ptok[(size_t)chain[p >> 5] * PAGE + (p & 31)]; };
+            auto key_of = [&](int p) -> const KV* { return kpg + ((size_t)chain[p >> 5] * PAGE + (p & 31)) * HD; };
+            auto tok_of = [&](int p) -> int { return ptok[(size_t)chain[p >> 5] * PAGE + (p & 31)]; };
 
             // ---- centre A: member farthest from r_j; centre B: member farthest from A (ties: lowest token id)
             for (int round = 0; round < 2; round++) {
@@ -532,11 +519,9 @@ __global__ void __launch_bounds__(SP_THREADS, DKV_SP_MINBLOCKS) k_split_check(Ta
                 float sa[EPL];
 #pragma unroll
                 for (int e = 0; e < EPL; e++) sa[e] = 0.f;
-                // staged members of this child (by label) when the cluster was staged, else its rows in their new place
-                const int n_scan = cached ? c : cc;
-                for (int p = warp; p < n_scan; p += SP_WARPS) {
-                    if (cached && ((label[p] == stay) != (child == 0))) continue;
-                    const KV* k = (cached ? krows + (size_t)p * HD : kpg + ((size_t)pages[p >> 5] * PAGE + (p & 31)) * HD) + lane * EPL;
+                // the child's rows in their new place
+                for (int p = warp; p < cc; p += SP_WARPS) {
+                    const KV* k = kpg + ((size_t)pages[p >> 5] * PAGE + (p & 31)) * HD + lane * EPL;
 #pragma unroll
                     for (int e = 0; e < EPL; e++) sa[e] += to_f(k[e]);
                 }
@@ -554,9 +539,8 @@ __global__ void __launch_bounds__(SP_THREADS, DKV_SP_MINBLOCKS) k_split_check(Ta
                 float mean[EPL], m2 = 0.f;
 #pragma unroll
                 for (int e = 0; e < EPL; e++) mean[e] = cA[lane * EPL + e];
-                for (int p = warp; p < n_scan; p += SP_WARPS) {
-                    if (cached && ((label[p] == stay) != (child == 0))) continue;
-                    const KV* k = (cached ? krows + (size_t)p * HD : kpg + ((size_t)pages[p >> 5] * PAGE + (p & 31)) * HD) + lane * EPL;
+                for (int p = warp; p < cc; p += SP_WARPS) {
+                    const KV* k = kpg + ((size_t)pages[p >> 5] * PAGE + (p & 31)) * HD + lane * EPL;
                     float part = 0.f;
 #pragma unroll
                     for (int e = 0; e < EPL; e++) { float df = to_f(k[e]) - mean[e]; part = fmaf(df, df, part); }

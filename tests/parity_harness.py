@@ -40,6 +40,26 @@ class ParityReport:
     tokens_selected: List[int] = field(default_factory=list)
     status_bits: int = 0
     rechecked: int = 0
+    decisions: int = 0          # discrete decisions offered to the oracle as hints (assignments, selections, appends, checks)
+
+
+def tie_bound(rep: "ParityReport") -> int:
+    """Most followed ties a run may show: two, plus one per 10 000 decisions.  A tie needs two candidates within
+    1e-5 relative in the oracle's fp64 numbers; on continuous random data that is rare, so a count above this bound
+    means the library leans on the tie rule instead of deciding correctly."""
+    return 2 + rep.decisions // 10000
+
+
+def log_ties(name: str, rep: "ParityReport") -> None:
+    """Append one JSON line per parity run to gpurun_out/parity_ties.jsonl (when that folder exists), so the tie
+    counts of a test session can be read afterwards."""
+    import json
+    import os
+    folder = os.path.join(os.path.dirname(os.path.dirname(os.path.abspath(__file__))), "gpurun_out")
+    if os.path.isdir(folder):
+        with open(os.path.join(folder, "parity_ties.jsonl"), "a") as f:
+            f.write(json.dumps({"run": name, "ties": rep.ties, "violations": rep.violations, "decisions": rep.decisions,
+                                "bound": tie_bound(rep), "steps": rep.steps, "splits": rep.splits}) + "\n")
 
 
 def make_ctx(cfg: WorkloadConfig, n_units: int, trace: int = 1, assign_mode: int = 0) -> P.DynaKV:
@@ -167,6 +187,8 @@ def run_parity(cfg: WorkloadConfig, units: Sequence[int], steps: int, *, assign_
         done += nb
     status = ctx.get_status()
     rep.steps = steps
+    n_checks = steps // check_every
+    rep.decisions = len(watch) * (cfg.n_prefill * cfg.T + (cfg.M0 if cfg.init_mode == "kmeanspp" else 0) + 2 * steps + n_checks)
     rep.status_bits = status["error_bits"]
     rep.rechecked = status["assign_rechecked"]
     for ui in watch:

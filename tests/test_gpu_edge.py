@@ -12,7 +12,11 @@ pytestmark = pytest.mark.gpu
 
 def _run(cfg, units, steps, **kw):
     from parity_harness import run_parity
+    import inspect
+    from parity_harness import log_ties, tie_bound
     rep = run_parity(cfg, units, steps, **kw)
+    log_ties(f"{inspect.stack()[1].function}:{cfg.name}", rep)
+    assert rep.ties <= tie_bound(rep), f"{rep.ties} ties followed in {rep.decisions} decisions"
     assert rep.violations == 0
     return rep
 

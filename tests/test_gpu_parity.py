@@ -10,7 +10,11 @@ pytestmark = pytest.mark.gpu
 
 def _run(cfg, units, steps, **kw):
     from parity_harness import run_parity
+    import inspect
+    from parity_harness import log_ties, tie_bound
     rep = run_parity(cfg, units, steps, **kw)
+    log_ties(f"{inspect.stack()[1].function}:{cfg.name}", rep)
+    assert rep.ties <= tie_bound(rep), f"{rep.ties} ties followed in {rep.decisions} decisions"
     print(f"\n[{cfg.name}] steps={rep.steps} ties={rep.ties} splits={rep.splits} max_abs={rep.max_out_abs:.2e} "
           f"max_relL2={rep.max_out_l2:.2e} centroid_rel={rep.max_centroid_rel:.2e} "
           f"tokens/step={np.mean(rep.tokens_selected):.0f} status={rep.status_bits} rechecked={rep.rechecked}")

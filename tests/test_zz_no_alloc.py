@@ -8,6 +8,7 @@ import numpy as np
 import pytest
 import torch
 
+import oracle as O
 import paper_2511_07427_b200 as P
 from gen import CONFIGS, UnitStream, make_decode_chunk, make_prefill
 
@@ -27,15 +28,31 @@ def _reference_and_noalloc(cfg, n_units):
         init_mode=P.INIT_RANDOM, assign_mode=1))
     ctx.build_index(Kd, Vd, cfg.M0, 11)
     out = torch.empty((n_units, cfg.G, cfg.d), dtype=torch.float32, device="cuda")   # caller-owned output, reused
+    # the fp64 oracle's attention over all rows of unit 0 (one cluster holding everything), as a second reference
+    o = O.OracleUnit(cfg.d, cfg.G, cfg.n_prefill, 1)
+    o.install(K[0].double().numpy(), V[0].double().numpy(), np.zeros(cfg.n_prefill, np.int32), 1)
     for t in range(2):                                                              # two calls in a row
         ref = ctx.decode_step(qd[t], 10 ** 9).cpu().numpy().astype(np.float64)       # budget covers every cluster
         _, ntok = ctx.get_selection()
         assert int(ntok.min()) == cfg.n_prefill
+        torch.cuda.synchronize()
+        if t == 1:
+            # the first call on a device looks the scratch array's address up; from then on a call must leave the
+            # device's free memory and torch's allocator untouched
+            free0, alloc0 = torch.cuda.mem_get_info()[0], torch.cuda.memory_allocated()
         P.attend_rows_noalloc(qd[t], Kd, Vd, out=out)
+        torch.cuda.synchronize()
+        if t == 1:
+            assert torch.cuda.mem_get_info()[0] == free0 and torch.cuda.memory_allocated() == alloc0, \
+                "dynakv_attend_rows_noalloc changed the device's free memory"
         got = out.cpu().numpy().astype(np.float64)
         err = np.abs(got - ref).max()
         l2 = np.linalg.norm(got - ref) / np.linalg.norm(ref)
         assert err <= TOL_ABS and l2 <= TOL_L2, f"call {t}: max abs {err:.3e}, relative L2 {l2:.3e}"
+        want = o.attend(q[t, 0].double().numpy(), [0])
+        err = np.abs(got[0] - want).max()
+        l2 = np.linalg.norm(got[0] - want) / np.linalg.norm(want)
+        assert err <= TOL_ABS and l2 <= TOL_L2, f"call {t} against the oracle: max abs {err:.3e}, relative L2 {l2:.3e}"
     ctx.destroy()
 
 
