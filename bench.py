@@ -161,9 +161,23 @@ class OracleSample:
 
     def describe(self, steps: int, dt: float) -> str:
         cfg = self.cfg
-        return (f"{self.n_units} of {cfg.U} units of config {cfg.cfg_id} at full size (index built by the oracle with "
-                f"1 Lloyd round, untimed), {steps} decode steps in {dt:.1f} s on {self.cores} threads, scaled per unit "
-                f"to all {cfg.U} units")
+        return (f"{self.n_units} of {cfg.U} units of config {cfg.cfg_id} at full size, {steps} decode steps in {dt:.1f} s on "
+                f"{self.cores} threads, scaled per unit to all {cfg.U} units; the index under the timed steps is built by "
+                f"the oracle, untimed, with 1 Lloyd round instead of the config's {cfg.T} (a full-size oracle build is "
+                f"about a minute per unit and round; the decode steps' cost does not depend on how converged the partition is)")
+
+
+def _host_info() -> dict:
+    model = None
+    try:
+        with open("/proc/cpuinfo") as f:
+            for line in f:
+                if line.startswith("model name"):
+                    model = line.split(":", 1)[1].strip()
+                    break
+    except OSError:
+        pass
+    return {"nproc": os.cpu_count(), "cpu_model": model}
 
 
 def _cpu_baseline(cfg, target_seconds: float = 12.0) -> dict:
@@ -174,8 +188,15 @@ def _cpu_baseline(cfg, target_seconds: float = 12.0) -> dict:
     dt = smp.run(probe)
     steps = int(max(8, min(cap - probe - 1, target_seconds / max(dt / probe, 1e-6))))
     dt = smp.run(steps)
-    return {"value": smp.steps_per_s(dt, steps), "unit": "steps/s", "cores": smp.cores, "kind": "oracle",
-            "sample": smp.describe(steps, dt)}
+    out = {"value": smp.steps_per_s(dt, steps), "unit": "steps/s", "cores": smp.cores, "kind": "oracle",
+           "sample": smp.describe(steps, dt), "host": _host_info()}
+    # the same on ONE host thread (one unit), scaled per unit like the figure above
+    one = OracleSample(cfg, 1, cap)
+    dt1 = one.run(probe)
+    steps1 = int(max(8, min(cap - probe - 1, 4.0 / max(dt1 / probe, 1e-6))))
+    dt1 = one.run(steps1)
+    out["one_thread"] = {"value": one.steps_per_s(dt1, steps1), "unit": "steps/s", "cores": 1, "sample": one.describe(steps1, dt1)}
+    return out
 
 
 def run_reference(args, cfg):
@@ -196,7 +217,7 @@ def run_reference(args, cfg):
         "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
         "config": config_dict(cfg, args.warmup),
         "cpu_baseline": {"value": value, "unit": "steps/s", "cores": smp.cores, "kind": "oracle",
-                         "sample": smp.describe(args.steps, dt)},
+                         "sample": smp.describe(args.steps, dt), "host": _host_info()},
         "e2e": {"value": value, "unit": "steps/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }
     print(json.dumps(line), flush=True)
@@ -206,7 +227,7 @@ def config_dict(cfg, warmup: int) -> dict:
     """The `config` object of the JSON line, the same for both arms."""
     return {"workload": f"config{cfg.cfg_id}:{cfg.name}", "units_per_gpu": cfg.U, "layers": cfg.L, "kv_heads": cfg.Hkv,
             "gqa_group": cfg.G, "head_dim": cfg.d, "context": cfg.n_prefill + warmup, "clusters": cfg.M0, "budget": cfg.budget,
-            "l2": "inputs_larger_than_l2", "loop": "cuda_graph_replay(decode_step,append,split_check)"}
+            "l2": "inputs_larger_than_l2"}
 
 
 def rank_units(cfg, rank: int):
@@ -250,10 +271,15 @@ def run_ours(args, cfg):
     torch.cuda.set_stream(side)
     peaks = _peaks()
     K_steps, W = args.steps, args.warmup
-    n_e2e = min(args.e2e_steps, K_steps)
-    n_prof = min(args.profile_steps, K_steps)
-    total_steps = W + K_steps + n_e2e + n_prof
-    assert total_steps <= cfg.steps, "not enough decode capacity in this config for the requested steps"
+    n_e2e = min(args.e2e_steps, max(K_steps, 16))
+    n_prof = min(args.profile_steps, max(K_steps, 16))
+    # the timed region of K steps is run `repeats` times on consecutive slices of the stream (the median is the
+    # value); what is left of the config's decode length, up to 512 steps, goes to one long call
+    room = cfg.steps - W - n_e2e - n_prof
+    assert room >= K_steps, "not enough decode capacity in this config for the requested steps"
+    repeats = max(1, min(args.repeats, room // K_steps))
+    n_steady = max(0, min(args.steady_steps, room - repeats * K_steps))
+    total_steps = W + repeats * K_steps + n_steady + n_e2e + n_prof
 
     # ---- synthetic inputs, generated on the device (seeded per unit and rank)
     U = cfg.U
@@ -308,26 +334,40 @@ def run_ours(args, cfg):
     st0 = ctx.get_status()
     if st0["error_bits"] & P.ST_INTERNAL:
         raise RuntimeError("a bounded wait ran out inside a kernel during warm-up (status bit INTERNAL); not timing")
-    launches0 = ctx.launch_count()
     sampler = ClockSampler(local) if rank == 0 else None
     if sampler:
         sampler.start()
     torch.cuda.synchronize()
     t_wall0 = time.perf_counter()
-    e0.record()
-    loop(pos, pos + K_steps)
-    e1.record()
-    torch.cuda.synchronize()
+    ms_runs, gpu_launches = [], 0
+    for r in range(repeats):
+        launches0 = ctx.launch_count()
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+        e0.record()
+        loop(pos, pos + K_steps)
+        e1.record()
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        ms_runs.append(max_over_ranks(e0.elapsed_time(e1), dev))
+        gpu_launches = ctx.launch_count() - launches0
+        pos += K_steps
     t_wall1 = time.perf_counter()
-    if world > 1:
-        dist.barrier()
-    ms = e0.elapsed_time(e1)
-    clocks = sampler.stop(t_wall0, t_wall1) if sampler else None
-    pos += K_steps
     st1 = ctx.get_status()
-    gpu_launches = ctx.launch_count() - launches0
-    ms = max_over_ranks(ms, dev)
+    ms = statistics.median(ms_runs)
     value = whole_job_steps_per_s(world, K_steps, ms)
+    steady_us = None
+    if n_steady > 0:
+        e0.record()
+        loop(pos, pos + n_steady)
+        e1.record()
+        torch.cuda.synchronize()
+        steady_us = max_over_ranks(e0.elapsed_time(e1), dev) * 1e3 / n_steady
+        pos += n_steady
+    clocks = sampler.stop(t_wall0, time.perf_counter()) if sampler else None
+    timed_steps = repeats * K_steps
 
     # ---- per-kernel breakdown with CUDA events around every launch (direct calls, same stream)
     ctx.set_timing(True)
@@ -387,9 +427,12 @@ def run_ours(args, cfg):
             "config": config_dict(cfg, W),
             "e2e": e2e, "gpu_launches": int(gpu_launches), "clocks": clocks, "roofline": roofline,
             "cpu_baseline": cpu_baseline, "build": build,
+            "timing": {"repeats": repeats, "ms_per_repeat": ms_runs, "value_is": "median of the repeats",
+                       "steady_us_per_iteration": steady_us, "steady_steps": n_steady,
+                       "loop": "cuda_graph_replay(decode_step,append,split_check)"},
             "counters": {"splits_in_timed_region": st1["n_splits"] - st0["n_splits"],
-                         "tokens_attended_per_step": (st1["tokens_attended_total"] - st0["tokens_attended_total"]) / K_steps,
-                         "clusters_selected_per_step": (st1["clusters_selected_total"] - st0["clusters_selected_total"]) / K_steps,
+                         "tokens_attended_per_step": (st1["tokens_attended_total"] - st0["tokens_attended_total"]) / timed_steps,
+                         "clusters_selected_per_step": (st1["clusters_selected_total"] - st0["clusters_selected_total"]) / timed_steps,
                          "status_bits": status["error_bits"], "assign_rechecked": status["assign_rechecked"]},
         }
         print(json.dumps(line), flush=True)
@@ -400,7 +443,9 @@ def run_ours(args, cfg):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=1024)
+    ap.add_argument("--steps", type=int, default=256)
+    ap.add_argument("--repeats", type=int, default=5, help="timed regions of --steps steps each; the median is reported")
+    ap.add_argument("--steady-steps", type=int, default=512, help="one more long call after the repeats (start-up share visible)")
     ap.add_argument("--warmup", type=int, default=16)
     ap.add_argument("--config", type=int, default=4)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])

@@ -131,8 +131,9 @@ int dynakv_decode_step(dynakv_ctx* ctx, const float* q, int32_t token_budget, fl
 int dynakv_split_check(dynakv_ctx* ctx);
 
 /* n_steps iterations of { decode_step(q_t); append(k_t, v_t); split_check() } (the order
- * of Algorithm 1's loop body), replayed from one captured CUDA graph whose kernels read
- * the step index from device memory.  q_steps: [n_steps][U][G][d] fp32, k_steps,
+ * of Algorithm 1's loop body), replayed from CUDA graphs (of 8, 4, 2 and 1 iterations,
+ * captured once per token budget) whose kernels read the step index and the addresses of
+ * the caller's arrays from device memory, so later calls may pass other arrays at no cost.  q_steps: [n_steps][U][G][d] fp32, k_steps,
  * v_steps: [n_steps][U][d] kv_dtype, out_steps: [n_steps][U][G][d] fp32, all device.
  * All n_steps inputs must be complete before the call: units are independent, so a unit's
  * centroid pass for step t+1 (query scores, new key's distances) runs as soon as that

@@ -36,10 +36,11 @@ struct dynakv_ctx {
     // graph loop
     int* step_ctr = nullptr;          // device: step index of the captured loop
     int* step_lim = nullptr;          // device: number of steps of the loop in flight
-    cudaGraphExec_t graph_exec = nullptr, graph_exec_long = nullptr;   // one iteration / eight iterations
-    const void* g_q = nullptr; const void* g_k = nullptr; const void* g_v = nullptr; void* g_out = nullptr;
+    static constexpr int N_GRAPHS = 4;            // captured loops of 8, 4, 2 and 1 iterations
+    cudaGraphExec_t graph_exec[N_GRAPHS] = {nullptr, nullptr, nullptr, nullptr};
+    const void** loop_args = nullptr; // device: [4] q, k, v, out arrays of the loop in flight (read by the captured kernels)
     int g_budget = -1;
-    long long graph_nodes = 0;
+    long long graph_nodes = 0;        // kernel launches per captured iteration
     // staging for dynakv_step_host
     float* st_q = nullptr; void* st_k = nullptr; void* st_v = nullptr; float* st_out = nullptr;
     cudaStream_t copy_stream = nullptr;      // carries the result copy of a host step past the step's append / split
@@ -170,8 +171,8 @@ extern "C" int dynakv_create(const dynakv_config* cfg, void* cuda_stream, dynakv
     ALLOC(t.u_scan, U, true); ALLOC(t.u_last, U, true);
     ALLOC(t.sel_ids, U * Mx, true);
     ALLOC(t.sel_n, U, true); ALLOC(t.sel_tokens, U, true);
-    ALLOC(t.work, U * (size_t)t.W, false);
-    ALLOC(t.n_work, U, true);
+    ALLOC(t.work, 2 * U * (size_t)t.W, false);
+    ALLOC(t.n_work, 2 * U, true);
     {
         size_t recs = U * (size_t)t.n_splits_attn;
         if (recs < 2 * (size_t)t.n_attn_ctas) recs = 2 * (size_t)t.n_attn_ctas;
@@ -196,6 +197,7 @@ extern "C" int dynakv_create(const dynakv_config* cfg, void* cuda_stream, dynakv
     ALLOC(t.counters, 8, true);
     ALLOC(c->step_ctr, 1, true);
     ALLOC(c->step_lim, 1, true);
+    ALLOC(c->loop_args, 4, true);
     ALLOC(c->st_q, U * t.G * d, false);
     ALLOC(c->st_out, U * t.G * d, false);
     {
@@ -212,8 +214,7 @@ extern "C" void dynakv_destroy(dynakv_ctx* c) {
     cudaStreamSynchronize(c->stream);
     if (c->copy_stream) { cudaStreamSynchronize(c->copy_stream); cudaStreamDestroy(c->copy_stream); }
     if (c->ev_attended) cudaEventDestroy(c->ev_attended);
-    if (c->graph_exec) cudaGraphExecDestroy(c->graph_exec);
-    if (c->graph_exec_long) cudaGraphExecDestroy(c->graph_exec_long);
+    for (cudaGraphExec_t g : c->graph_exec) if (g) cudaGraphExecDestroy(g);
     for (auto& sp : c->spans) { cudaEventDestroy(sp.e0); cudaEventDestroy(sp.e1); }
     for (cudaEvent_t e : c->event_pool) cudaEventDestroy(e);
     for (void* p : c->allocs) cudaFree(p);
@@ -279,9 +280,16 @@ static void enqueue_front(dynakv_ctx* c, StepPtr q, StepPtr k, int has_q, int ha
     launch_front(c->t, q, k, has_q, has_k, c->stream, &c->launches);
 }
 
+// gather attention -> combine, on work lists already written by a selection
+static void enqueue_attend(dynakv_ctx* c, StepPtr q, StepPtrW out, bool timed);
+
 // select -> gather attention -> combine, on scores already written by the front pass
 static void enqueue_retrieve(dynakv_ctx* c, StepPtr q, int budget, StepPtrW out, int* sel_ids, bool timed) {
     { TimeScope ts(c, KC_SELECT, timed); launch_select(c->t, budget, sel_ids, c->stream, &c->launches); }
+    enqueue_attend(c, q, out, timed);
+}
+
+static void enqueue_attend(dynakv_ctx* c, StepPtr q, StepPtrW out, bool timed) {
     if (c->t.kv_dtype == DYNAKV_BF16 && c->cfg.attn_mode == 0) {
         // gather, attend and combine in one persistent kernel
         TimeScope ts(c, KC_ATTN, timed);
@@ -297,23 +305,16 @@ static void enqueue_append_apply(dynakv_ctx* c, StepPtr k, StepPtr v, bool timed
     launch_append_apply(c->t, k, v, c->stream, &c->launches);
 }
 
-static const NextFront kNoNextFront = {0, StepPtr{nullptr, 0, nullptr}, StepPtr{nullptr, 0, nullptr}, nullptr};
+static const NextFront kNoNextFront = {0, StepPtr{nullptr, 0, nullptr}, StepPtr{nullptr, 0, nullptr}, nullptr, 0};
 
-// One iteration of a captured loop in three launches.  The centroid pass of step t + 1 is part of the tail kernel
-// of step t (every unit's block runs it as soon as the unit's own append is done), so an iteration starts at the
-// selection; the pass of step 0 is launched once ahead of the loop.  The tail kernel's last block advances the
-// device-side step index that all kernels of the loop read.
+// One iteration of a captured loop in two launches: gather-attention of step t, then the tail kernel, in which every
+// unit's block appends the step's key, runs the centroid pass of step t + 1 and the selection of step t + 1 (helper
+// blocks do the splits, and the selection of the units they split).  The pass and the selection of step 0 are launched
+// once ahead of the loop.  The tail kernel's last block advances the device-side step index that all kernels read.
 static void enqueue_loop_iteration(dynakv_ctx* c, StepPtr q, StepPtr k, StepPtr v, int budget, StepPtrW out) {
-    enqueue_retrieve(c, q, budget, out, nullptr, false);
+    enqueue_attend(c, q, out, false);
     launch_append_split(c->t, c->cfg.split_size_factor, c->cfg.split_var_factor > 0.f ? 1 : 0, c->cfg.split_min_size,
-                        c->cfg.split_iters, 1, k, v, c->step_ctr, NextFront{1, q, k, c->step_lim}, c->stream, &c->launches);
-}
-
-// Start of a captured loop: step index, step count, and the per-unit words the tail kernel's blocks exchange.
-__global__ void k_loop_begin(Tables t, int* step_ctr, int* step_lim, int n_steps) {
-    const int i = blockIdx.x * blockDim.x + threadIdx.x;
-    if (i == 0) { *step_ctr = 0; *step_lim = n_steps; t.plan_counter[1] = 0; t.tail_sync[0] = 0; t.tail_sync[1] = 0; t.tail_sync[2] = 0; }
-    if (i < t.U) { t.front_done[i] = 0; t.tail_queue[2 * i] = 0; t.tail_queue[2 * i + 1] = 0; }
+                        c->cfg.split_iters, 1, k, v, c->step_ctr, NextFront{1, q, k, c->step_lim, budget}, c->stream, &c->launches);
 }
 
 extern "C" int dynakv_decode_step(dynakv_ctx* c, const float* q, int32_t token_budget, float* out, int32_t* selected_ids) {
@@ -357,49 +358,54 @@ extern "C" int dynakv_decode_loop(dynakv_ctx* c, const float* q_steps, const voi
         return DYNAKV_ERR_STATE;
     }
     const Tables& t = c->t;
-    constexpr int UNROLL = 8;            // iterations in the long graph; the remainder runs the one-iteration graph
-    if (!c->graph_exec || c->g_q != q_steps || c->g_k != k_steps || c->g_v != v_steps || c->g_out != out_steps ||
-        c->g_budget != token_budget) {
-        if (c->graph_exec) { cudaGraphExecDestroy(c->graph_exec); c->graph_exec = nullptr; }
-        if (c->graph_exec_long) { cudaGraphExecDestroy(c->graph_exec_long); c->graph_exec_long = nullptr; }
-        const long long qs = (long long)t.U * t.G * t.d * 4, ks = (long long)t.U * t.d * (long long)kv_bytes(c->cfg);
-        for (int which = 0; which < 2; which++) {
-            const int reps = which == 0 ? 1 : UNROLL;
+    const long long qs = (long long)t.U * t.G * t.d * 4, ks = (long long)t.U * t.d * (long long)kv_bytes(c->cfg);
+    // The loop is captured once per token budget as graphs of 8, 4, 2 and 1 iterations.  The captured kernels read
+    // the caller's arrays through c->loop_args (stored by the pass that opens the loop), so the same graphs serve
+    // every later call whatever arrays it passes.
+    if (!c->graph_exec[0] || c->g_budget != token_budget) {
+        for (cudaGraphExec_t& g : c->graph_exec) if (g) { cudaGraphExecDestroy(g); g = nullptr; }
+        const StepPtr gq{nullptr, qs, c->step_ctr, c->loop_args + 0}, gk{nullptr, ks, c->step_ctr, c->loop_args + 1},
+                      gv{nullptr, ks, c->step_ctr, c->loop_args + 2};
+        const StepPtrW go{nullptr, qs, c->step_ctr, (void* const*)(c->loop_args + 3)};
+        for (int which = 0; which < dynakv_ctx::N_GRAPHS; which++) {
+            const int reps = 8 >> which;
             cudaGraph_t graph = nullptr;
             long long before = c->launches;
             CK(cudaStreamBeginCapture(c->stream, cudaStreamCaptureModeThreadLocal));
-            for (int r = 0; r < reps; r++)
-                enqueue_loop_iteration(c, StepPtr{q_steps, qs, c->step_ctr}, StepPtr{k_steps, ks, c->step_ctr},
-                                       StepPtr{v_steps, ks, c->step_ctr}, token_budget, StepPtrW{out_steps, qs, c->step_ctr});
+            for (int r = 0; r < reps; r++) enqueue_loop_iteration(c, gq, gk, gv, token_budget, go);
             cudaError_t e = cudaStreamEndCapture(c->stream, &graph);
-            if (which == 0) c->graph_nodes = c->launches - before;
+            c->graph_nodes = (c->launches - before) / reps;
             c->launches = before;
-            if (e != cudaSuccess || !graph) {
-                snprintf(g_err, sizeof(g_err), "graph capture failed: %s", cudaGetErrorString(e));
-                return DYNAKV_ERR_CUDA;
+            if (e == cudaSuccess && graph) {
+                e = cudaGraphInstantiate(&c->graph_exec[which], graph, 0);
+                cudaGraphDestroy(graph);
+                // send the executable graph to the device now, not inside the first timed launch
+                if (e == cudaSuccess) e = cudaGraphUpload(c->graph_exec[which], c->stream);
             }
-            e = cudaGraphInstantiate(which == 0 ? &c->graph_exec : &c->graph_exec_long, graph, 0);
-            cudaGraphDestroy(graph);
             if (e != cudaSuccess) {
-                if (c->graph_exec) { cudaGraphExecDestroy(c->graph_exec); c->graph_exec = nullptr; }
-                c->graph_exec_long = nullptr;
-                snprintf(g_err, sizeof(g_err), "graph instantiate failed: %s", cudaGetErrorString(e));
+                for (cudaGraphExec_t& g : c->graph_exec) if (g) { cudaGraphExecDestroy(g); g = nullptr; }
+                snprintf(g_err, sizeof(g_err), "graph capture / instantiate failed: %s", cudaGetErrorString(e));
+                cudaGetLastError();
                 return DYNAKV_ERR_CUDA;
             }
         }
-        c->g_q = q_steps; c->g_k = k_steps; c->g_v = v_steps; c->g_out = out_steps; c->g_budget = token_budget;
+        c->g_budget = token_budget;
     }
     if (n_steps == 0) return DYNAKV_OK;
     {
-        const long long qs = (long long)t.U * t.G * t.d * 4, ks = (long long)t.U * t.d * (long long)kv_bytes(c->cfg);
-        k_loop_begin<<<(t.U + 255) / 256, 256, 0, c->stream>>>(t, c->step_ctr, c->step_lim, (int)n_steps);
-        c->launches++;
-        // step 0's centroid pass; every later one rides in the tail kernel of the step before it
-        enqueue_front(c, StepPtr{q_steps, qs, c->step_ctr}, StepPtr{k_steps, ks, c->step_ctr}, 1, 1, false);
+        // step 0's centroid pass opens the loop (step index, hand-over words, the caller's arrays); every later
+        // pass rides in the tail kernel of the step before it
+        LoopBegin lb;
+        lb.on = 1; lb.step_ctr = c->step_ctr; lb.step_lim = c->step_lim; lb.n_steps = (int)n_steps; lb.args = c->loop_args;
+        lb.q = q_steps; lb.k = k_steps; lb.v = v_steps; lb.out = out_steps;
+        launch_front(c->t, StepPtr{q_steps, qs, nullptr}, StepPtr{k_steps, ks, nullptr}, 1, 1, c->stream, &c->launches, &lb);
+        launch_select(c->t, token_budget, nullptr, c->stream, &c->launches);     // step 0's selection (work lists of parity 0)
     }
-    int64_t s = 0;
-    for (; s + UNROLL <= n_steps; s += UNROLL) CK(cudaGraphLaunch(c->graph_exec_long, c->stream));
-    for (; s < n_steps; s++) CK(cudaGraphLaunch(c->graph_exec, c->stream));
+    int64_t left = n_steps;
+    for (int which = 0; which < dynakv_ctx::N_GRAPHS; which++) {
+        const int reps = 8 >> which;
+        for (; left >= reps; left -= reps) CK(cudaGraphLaunch(c->graph_exec[which], c->stream));
+    }
     c->launches += c->graph_nodes * n_steps;
     return DYNAKV_OK;
 }

@@ -117,7 +117,12 @@ __global__ void __launch_bounds__(AT_THREADS, 2) k_gather_attn_tma(Tables t, Ste
         asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
     }
     pdl_trigger();       // the append/split kernel may move in as CTAs of this grid retire; it waits before it moves rows
-    pdl_wait();          // the work lists and their prefix come from the selection kernel
+    pdl_wait();          // the work lists and their prefix come from the selection (the kernel before)
+    // inside a captured loop the step's work lists are the copy of the step's parity (the other copy is being
+    // written for the next step while this kernel runs)
+    const int buf = qp.ctr ? (*qp.ctr & 1) : 0;
+    const int* n_work = t.n_work + (size_t)buf * U;
+    const int2* work = t.work + (size_t)buf * U * t.W;
     const int* pf = t.work_prefix;
     if (t.attn_pf_in_smem) {
         // Every CTA lays the units' work lists end to end itself: an exclusive prefix of their lengths, each
@@ -128,7 +133,7 @@ __global__ void __launch_bounds__(AT_THREADS, 2) k_gather_attn_tma(Tables t, Ste
         int nw[MAXPER];
         int sum = 0;
 #pragma unroll
-        for (int i = 0; i < MAXPER; i++) { nw[i] = (i < per_t && b0 + i < U) ? t.n_work[b0 + i] : 0; sum += nw[i]; }
+        for (int i = 0; i < MAXPER; i++) { nw[i] = (i < per_t && b0 + i < U) ? n_work[b0 + i] : 0; sum += nw[i]; }
         int incl = sum;
 #pragma unroll
         for (int o = 1; o < 32; o <<= 1) { const int y = __shfl_up_sync(0xffffffffu, incl, o); if (lane >= o) incl += y; }
@@ -165,14 +170,14 @@ __global__ void __launch_bounds__(AT_THREADS, 2) k_gather_attn_tma(Tables t, Ste
             const unsigned full = smem_u32(&bars[lane]), empty = smem_u32(&bars[AT_STAGES + lane]);
             const unsigned dst = smem_u32(ring + (size_t)lane * AttnSmem<HD>::stage_bytes);
             int u = unit_of_bisect(pf, U, lo + lane);
-            int2 ent = t.work[(size_t)u * t.W + (lo + lane - pf[u])];
+            int2 ent = work[(size_t)u * t.W + (lo + lane - pf[u])];
             int last_issued = -1;
             for (int it = lane; it < n_items; it += AT_STAGES) {
                 const int2 cur = ent;
                 const int cu = u;
                 if (it + AT_STAGES < n_items) {          // next entry: its load is in flight during the wait below
                     u = unit_of(pf, u, lo + it + AT_STAGES);
-                    ent = t.work[(size_t)u * t.W + (lo + it + AT_STAGES - pf[u])];
+                    ent = work[(size_t)u * t.W + (lo + it + AT_STAGES - pf[u])];
                 }
                 const unsigned ph = (unsigned)(it / AT_STAGES) & 1u;
                 if (!mbar_wait(empty, ph ^ 1u)) { s_flag[0] = 1; break; }

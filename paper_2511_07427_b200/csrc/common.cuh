@@ -44,8 +44,10 @@ struct Tables {
     float* dists;                    // [U][Mmax] squared distance of the step's new key to every representative
     int* sel_ids;                    // [U][Mmax]
     int* sel_n; int* sel_tokens;     // [U]
-    int2* work;                      // [U][W] (first row = page * PAGE + offset, rows <= ENTRY_ROWS)
-    int* n_work;                     // [U]
+    // The work lists exist twice: inside a captured loop the selection of step t + 1 is written (buffer (t + 1) & 1)
+    // while the gather-attention kernel of step t still reads its own (buffer t & 1); direct calls use buffer 0.
+    int2* work;                      // [2][U][W] (first row = page * PAGE + offset, rows <= ENTRY_ROWS)
+    int* n_work;                     // [2][U]
     float* part;                     // partial (acc, m, l) records of [G][d + 2] floats: [U][S] (plain kernel) or [2 * n_attn_ctas]
     int* work_prefix;                // [U + 1] exclusive prefix of n_work over the units (written by the last select block)
     int* unit_arrive;                // [U] arrival counters of the split-K combine (zero between steps)
@@ -68,25 +70,30 @@ struct Tables {
 enum { CNT_APPENDED = 0, CNT_SPLITS = 1, CNT_RECHECKED = 2, CNT_TOKENS_ATTENDED = 3, CNT_CLUSTERS_SELECTED = 7 };
 
 // A per-step operand: base pointer plus a stride applied with the device-side step index,
-// so the same kernel serves a direct call (ctr == nullptr) and a captured graph replay.
+// so the same kernel serves a direct call (ctr == nullptr) and a captured graph replay.  With
+// `ind` set the base pointer itself is read from device memory (written at the start of a loop),
+// so one captured graph serves every call of the loop whatever arrays the caller passes.
 struct StepPtr {
     const void* base;
     long long stride_bytes;
     const int* ctr;
+    const void* const* ind;
+    __device__ __forceinline__ const char* origin() const { return ind ? (const char*)(*ind) : (const char*)base; }
     __device__ __forceinline__ const void* get() const {
         long long t = ctr ? (long long)(*ctr) : 0;
-        return (const char*)base + t * stride_bytes;
+        return origin() + t * stride_bytes;
     }
     // the operand of step `step`, whatever the step index says
-    __device__ __forceinline__ const void* at(long long step) const { return (const char*)base + step * stride_bytes; }
+    __device__ __forceinline__ const void* at(long long step) const { return origin() + step * stride_bytes; }
 };
 struct StepPtrW {
     void* base;
     long long stride_bytes;
     const int* ctr;
+    void* const* ind;
     __device__ __forceinline__ void* get() const {
         long long t = ctr ? (long long)(*ctr) : 0;
-        return (char*)base + t * stride_bytes;
+        return (ind ? (char*)(*ind) : (char*)base) + t * stride_bytes;
     }
 };
 
@@ -191,7 +198,17 @@ void launch_update(const Tables& t, const void* K, long long n, int M, const int
                    cudaStream_t s, long long* launches);
 void launch_finalize(const Tables& t, const void* K, const void* V, long long n, int M, const BuildScratch& b,
                      float alpha, cudaStream_t s, long long* launches);
-void launch_front(const Tables& t, StepPtr q, StepPtr k, int has_q, int has_k, cudaStream_t s, long long* launches);
+// What the stand-alone centroid pass does in addition when it opens a captured loop: it resets the device-side
+// step index and the hand-over words of the loop's tail kernel, and stores the caller's arrays where the
+// captured kernels look them up.
+struct LoopBegin {
+    int on;                   // 0: an ordinary pass
+    int* step_ctr; int* step_lim; int n_steps;
+    const void** args;        // device: [4] q, k, v, out of the loop in flight
+    const void* q; const void* k; const void* v; void* out;
+};
+void launch_front(const Tables& t, StepPtr q, StepPtr k, int has_q, int has_k, cudaStream_t s, long long* launches,
+                  const LoopBegin* lb = nullptr);
 void launch_select(const Tables& t, int budget, int* user_sel_ids, cudaStream_t s, long long* launches);
 void launch_append_apply(const Tables& t, StepPtr k, StepPtr v, cudaStream_t s, long long* launches);
 void launch_gather_attn_tma(const Tables& t, StepPtr q, StepPtrW out, cudaStream_t s, long long* launches);
@@ -205,6 +222,7 @@ struct NextFront {
     int on;                  // 0: no fused pass
     StepPtr q, k;            // per-step query and key arrays (indexed with step + 1)
     const int* step_lim;     // device: number of steps of the loop; the pass is skipped when step + 1 reaches it
+    int budget;              // token budget of the next step's selection, which follows the pass unit by unit
 };
 void launch_append_split(const Tables& t, float gamma, int var_enabled, int min_size, int iters, int do_append, StepPtr k,
                          StepPtr v, int* step_ctr, const NextFront& nf, cudaStream_t s, long long* launches);

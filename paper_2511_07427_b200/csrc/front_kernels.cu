@@ -28,7 +28,7 @@ constexpr int FR_ROWS = DKV_FR_ROWS;      // representatives per block (a multip
 // thread -- its rows, their cluster sizes, its share of the query heads, the new key -- is issued
 // before the first use of any of them, so a block pays one memory latency, not a chain of them.
 template <typename KV, int HD>
-__global__ void __launch_bounds__(FR_THREADS, 2) k_front(Tables t, StepPtr qp, StepPtr kp, int has_q, int has_k) {
+__global__ void __launch_bounds__(FR_THREADS, 2) k_front(Tables t, StepPtr qp, StepPtr kp, int has_q, int has_k, LoopBegin lb) {
     constexpr int V4 = HD / 32;   // float4 loads per lane per row
     constexpr int NIT = FR_ROWS / ((FR_THREADS / 32) * 4);
     const int u = blockIdx.y;
@@ -36,6 +36,15 @@ __global__ void __launch_bounds__(FR_THREADS, 2) k_front(Tables t, StepPtr qp, S
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int sub = lane >> 3, l8 = lane & 7;
     pdl_wait();                          // inside a captured loop the representatives come from the iteration before
+    if (lb.on && blockIdx.x == 0 && threadIdx.x == 0) {
+        // opening a captured loop: this pass is step 0's and runs on the caller's arrays directly
+        t.front_done[u] = 0; t.tail_queue[2 * u] = 0; t.tail_queue[2 * u + 1] = 0;
+        if (u == 0) {
+            *lb.step_ctr = 0; *lb.step_lim = lb.n_steps;
+            t.plan_counter[1] = 0; t.tail_sync[0] = 0; t.tail_sync[1] = 0; t.tail_sync[2] = 0;
+            lb.args[0] = lb.q; lb.args[1] = lb.k; lb.args[2] = lb.v; lb.args[3] = lb.out;
+        }
+    }
     // A unit never has fewer clusters than the build gave it: blocks wholly below that count need not
     // wait for the unit's current count before they issue their row loads.
     int jend = j0 + FR_ROWS;
@@ -126,14 +135,17 @@ __global__ void __launch_bounds__(256) k_append_apply(Tables t, StepPtr kp_, Ste
 
 // ------------------------------------------------------------------ launchers
 
-void launch_front(const Tables& t, StepPtr q, StepPtr k, int has_q, int has_k, cudaStream_t s, long long* launches) {
+void launch_front(const Tables& t, StepPtr q, StepPtr k, int has_q, int has_k, cudaStream_t s, long long* launches,
+                  const LoopBegin* lbp) {
+    LoopBegin lb = {};
+    if (lbp) lb = *lbp;
     dim3 grid((t.max_clusters + FR_ROWS - 1) / FR_ROWS, t.U);
     if (t.kv_dtype == DYNAKV_F32) {
-        if (t.d == 64) launch_pdl(k_front<float, 64>, grid, dim3(FR_THREADS), 0, s, t, q, k, has_q, has_k);
-        else launch_pdl(k_front<float, 128>, grid, dim3(FR_THREADS), 0, s, t, q, k, has_q, has_k);
+        if (t.d == 64) launch_pdl(k_front<float, 64>, grid, dim3(FR_THREADS), 0, s, t, q, k, has_q, has_k, lb);
+        else launch_pdl(k_front<float, 128>, grid, dim3(FR_THREADS), 0, s, t, q, k, has_q, has_k, lb);
     } else {
-        if (t.d == 64) launch_pdl(k_front<__nv_bfloat16, 64>, grid, dim3(FR_THREADS), 0, s, t, q, k, has_q, has_k);
-        else launch_pdl(k_front<__nv_bfloat16, 128>, grid, dim3(FR_THREADS), 0, s, t, q, k, has_q, has_k);
+        if (t.d == 64) launch_pdl(k_front<__nv_bfloat16, 64>, grid, dim3(FR_THREADS), 0, s, t, q, k, has_q, has_k, lb);
+        else launch_pdl(k_front<__nv_bfloat16, 128>, grid, dim3(FR_THREADS), 0, s, t, q, k, has_q, has_k, lb);
     }
     (*launches)++;
 }

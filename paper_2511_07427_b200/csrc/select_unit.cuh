@@ -33,7 +33,7 @@ struct SelectSmem {
 #define SEL_L sm.sc[5]
 #define SEL_tok sm.sc[6]
 #define SEL_best (*sm.best64)
-__host__ __device__ inline size_t select_smem_bytes(int ids) { return (size_t)ids * 8 + 2048 * 4 + 48 * 4 + 8 + 16; }
+__host__ __device__ constexpr size_t select_smem_bytes(int ids) { return (size_t)ids * 8 + 2048 * 4 + 48 * 4 + 8 + 16; }
 __device__ __forceinline__ SelectSmem select_smem_at(unsigned char* base, int ids) {      // base: 8-byte aligned
     SelectSmem sm;
     sm.best64 = reinterpret_cast<unsigned long long*>(base);
@@ -53,8 +53,9 @@ __device__ __forceinline__ unsigned int ord_key(float f) {
 // Called by every thread of the block.  scores: the unit's scores in global memory (written before a barrier or
 // by an earlier kernel).  user_ids (may be null): the selection in score order, -1 padded, [max_clusters].
 // On return (all global writes issued; no trailing barrier) thread 0 has written sel_n / sel_tokens / n_work.
+// buf: which copy of the work lists to write (0 outside a captured loop).
 template <int THREADS>
-__device__ void select_unit(const Tables& t, int u, int budget, int* __restrict__ user_ids, const SelectSmem& sm) {
+__device__ void select_unit(const Tables& t, int u, int budget, int* __restrict__ user_ids, const SelectSmem& sm, int buf = 0) {
     const int tid = threadIdx.x;
     const float* SC = t.scores + (size_t)u * t.max_clusters;
     const int* CN = t.cl_n + (size_t)u * t.max_clusters;
@@ -62,11 +63,11 @@ __device__ void select_unit(const Tables& t, int u, int budget, int* __restrict_
     // loaded without waiting for the unit's current count.
     const bool early = tid < t.M_floor;
     int sz0 = 0; float sc0 = 0.f;
-    if (early) { sz0 = CN[tid]; sc0 = __ldcg(SC + tid); }
-    const int Mcur = t.u_M[u];
+    if (early) { sz0 = __ldcg(CN + tid); sc0 = __ldcg(SC + tid); }
+    const int Mcur = __ldcg(&t.u_M[u]);
     unsigned long long best = 0ull;
     for (int j = tid; j < Mcur; j += THREADS) {
-        const int sz = (j == tid && early) ? sz0 : CN[j];
+        const int sz = (j == tid && early) ? sz0 : __ldcg(CN + j);
         const unsigned int key = sz > 0 ? ord_key((j == tid && early) ? sc0 : __ldcg(SC + j)) : 0u;
         sm.keys[j] = key; sm.sizes[j] = sz;
         if (sz > 0) {
@@ -165,7 +166,7 @@ __device__ void select_unit(const Tables& t, int u, int budget, int* __restrict_
     __syncthreads();
     // ---- compaction in id order + work list: every thread owns a run of consecutive ids
     int* sel = t.sel_ids + (size_t)u * t.max_clusters;
-    int2* work = t.work + (size_t)u * t.W;
+    int2* work = t.work + ((size_t)buf * t.U + u) * t.W;
     const int per = (Mcur + THREADS - 1) / THREADS;
     const int j_lo = min(Mcur, tid * per), j_hi = min(Mcur, j_lo + per);
     int my_sel = 0, my_w = 0;
@@ -183,18 +184,18 @@ __device__ void select_unit(const Tables& t, int u, int budget, int* __restrict_
         const int sz = szs & 0x7fffffff;
         const int np = (sz + ENTRY_ROWS - 1) / ENTRY_ROWS;     // work entries: runs of <= ENTRY_ROWS rows inside one page
         sel[spos++] = j;
-        int page = t.cl_head[(size_t)u * t.max_clusters + j];
+        int page = __ldcg(&t.cl_head[(size_t)u * t.max_clusters + j]);
         for (int i = 0; i < np && wpos + i < t.W; i++) {
             constexpr int EPP = PAGE / ENTRY_ROWS;       // entries per page
             work[wpos + i] = make_int2(page * PAGE + (i % EPP) * ENTRY_ROWS, min(ENTRY_ROWS, sz - ENTRY_ROWS * i));
-            if (i % EPP == EPP - 1) page = t.page_next[(size_t)u * t.P + page];
+            if (i % EPP == EPP - 1) page = __ldcg(&t.page_next[(size_t)u * t.P + page]);
         }
         wpos += np;
     }
     if (tid == 0) {
         t.sel_n[u] = L;
         t.sel_tokens[u] = SEL_tok;
-        t.n_work[u] = min(tw, t.W);
+        t.n_work[(size_t)buf * t.U + u] = min(tw, t.W);
         atomicAdd(&t.counters[CNT_TOKENS_ATTENDED], (unsigned long long)SEL_tok);
         atomicAdd(&t.counters[CNT_CLUSTERS_SELECTED], (unsigned long long)L);
     }
@@ -228,15 +229,16 @@ __device__ void select_unit(const Tables& t, int u, int budget, int* __restrict_
 
 // Exclusive prefix of the units' work-list lengths, by one block (after every unit's n_work is visible).
 template <int THREADS>
-__device__ void work_prefix_block(const Tables& t, int* sh) {
+__device__ void work_prefix_block(const Tables& t, int* sh, int buf = 0) {
     const int tid = threadIdx.x;
+    const int* n_work = t.n_work + (size_t)buf * t.U;
     const int per_t = (t.U + THREADS - 1) / THREADS;
     const int b0 = min(tid * per_t, t.U), b1 = min(b0 + per_t, t.U);
     int sum = 0;
-    for (int i = b0; i < b1; i++) sum += __ldcg(&t.n_work[i]);
+    for (int i = b0; i < b1; i++) sum += __ldcg(&n_work[i]);
     int tot;
     int base = block_scan_excl(sum, sh, &tot);
-    for (int i = b0; i < b1; i++) { t.work_prefix[i] = base; base += __ldcg(&t.n_work[i]); }
+    for (int i = b0; i < b1; i++) { t.work_prefix[i] = base; base += __ldcg(&n_work[i]); }
     if (tid == 0) t.work_prefix[t.U] = tot;
 }
 

@@ -10,3 +10,13 @@ if ROOT not in sys.path:
 
 def pytest_configure(config):
     config.addinivalue_line("markers", "gpu: needs a CUDA device (run on the B200 box)")
+    config.addinivalue_line("markers", "slow: takes many minutes (full decode lengths); runs only with DYNAKV_RUN_SLOW=1")
+
+
+def pytest_collection_modifyitems(config, items):
+    if os.environ.get("DYNAKV_RUN_SLOW") == "1":
+        return
+    skip = pytest.mark.skip(reason="slow: set DYNAKV_RUN_SLOW=1 to run the full decode lengths")
+    for item in items:
+        if "slow" in item.keywords:
+            item.add_marker(skip)

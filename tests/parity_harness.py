@@ -197,3 +197,43 @@ def run_parity(cfg: WorkloadConfig, units: Sequence[int], steps: int, *, assign_
     rep.gpu_splits = status["n_splits"]
     ctx.destroy()
     return rep
+
+
+def check_every_unit(cfg: WorkloadConfig, st: dict, K_all: "torch.Tensor", nt: int) -> dict:
+    """Eq. 3 and Eq. 4 on an exported state, for EVERY unit: every token in exactly one live cluster id below the
+    unit's id count, sizes equal to the membership counts, representatives equal to the member means, M2 equal to
+    the members' squared distances to their mean.  K_all: [U, >= nt, d] keys in token-id order on the GPU (plain
+    torch in fp64; no library code).  Returns the worst relative deviations seen."""
+    U, Mx, d = K_all.shape[0], cfg.max_clusters, cfg.d
+    assert np.all(st["n_tokens"] == nt), "token counts"
+    tokc = torch.from_numpy(st["tok_cluster"][:, :nt].astype(np.int64)).cuda()
+    counts = torch.from_numpy(st["counts"].astype(np.int64)).cuda()
+    cent = torch.from_numpy(st["centroids"]).cuda()
+    M2 = torch.from_numpy(st["M2"]).cuda().double()
+    n_ids = torch.from_numpy(st["n_ids"].astype(np.int64)).cuda()
+    assert int(tokc.min()) >= 0 and bool((tokc < n_ids[:, None]).all()), "a token outside the unit's ids"
+    worst_c, worst_m = 0.0, 0.0
+    step = max(1, min(64, (1 << 28) // max(nt * d, 1)))
+    for u0 in range(0, U, step):
+        u1 = min(U, u0 + step)
+        nu = u1 - u0
+        gid = (torch.arange(nu, device="cuda")[:, None] * Mx + tokc[u0:u1]).reshape(-1)
+        Kd = K_all[u0:u1, :nt].double().reshape(-1, d)
+        cnt = torch.zeros(nu * Mx, dtype=torch.int64, device="cuda").index_add_(0, gid, torch.ones_like(gid))
+        assert torch.equal(cnt.reshape(nu, Mx), counts[u0:u1]), "sizes differ from the membership counts"
+        sums = torch.zeros((nu * Mx, d), dtype=torch.float64, device="cuda").index_add_(0, gid, Kd)
+        live = cnt > 0
+        mean = sums[live] / cnt[live][:, None]
+        cg = cent[u0:u1].reshape(nu * Mx, d)[live].double()
+        err = ((cg - mean).norm(dim=1) / mean.norm(dim=1).clamp_min(1e-30)).max()
+        worst_c = max(worst_c, float(err))
+        m2 = torch.zeros(nu * Mx, dtype=torch.float64, device="cuda").index_add_(0, gid, ((Kd - sums[gid] / cnt[gid][:, None]) ** 2).sum(1))
+        mg = M2[u0:u1].reshape(-1)[live]
+        # floor: the fp32 rounding of a representative leaves about n |r|^2 2^-46 in M2 even when the members coincide
+        scale = torch.maximum(m2[live], 1e-6 * cnt[live] * (mean.norm(dim=1) ** 2)).clamp_min(1e-6)
+        worst_m = max(worst_m, float(((mg - m2[live]).abs() / scale).max()))
+        del Kd, sums, m2
+    assert worst_c <= TOL_CENTROID, f"representatives differ from the member means: {worst_c:.2e}"
+    assert worst_m <= 2e-3, f"M2 differs from the members' spread: {worst_m:.2e}"
+    return {"centroid_rel": worst_c, "M2_rel": worst_m, "live_clusters": int((counts > 0).sum()),
+            "ids_max": int(n_ids.max()), "ids_min": int(n_ids.min())}
