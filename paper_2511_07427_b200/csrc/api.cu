@@ -136,6 +136,11 @@ extern "C" int dynakv_create(const dynakv_config* cfg, void* cuda_stream, dynakv
     int slack = full_pages / 8; if (slack < 64) slack = 64;
     t.P = full_pages + cfg->max_clusters + slack;
     t.W = (PAGE / ENTRY_ROWS) * t.P;
+    if (t.W >= (1 << 19)) {          // the selection packs a work-list position and a cluster count into one word
+        snprintf(g_err, sizeof(g_err), "max_tokens too large: a unit's work list would have %d entries (limit %d)", t.W, (1 << 19) - 1);
+        delete c;
+        return DYNAKV_ERR_ARG;
+    }
     t.n_splits_attn = 8;
     {
         int dev = 0, sms = 0;
@@ -171,8 +176,8 @@ extern "C" int dynakv_create(const dynakv_config* cfg, void* cuda_stream, dynakv
     ALLOC(t.u_scan, U, true); ALLOC(t.u_last, U, true);
     ALLOC(t.sel_ids, U * Mx, true);
     ALLOC(t.sel_n, U, true); ALLOC(t.sel_tokens, U, true);
-    ALLOC(t.work, 2 * U * (size_t)t.W, false);
-    ALLOC(t.n_work, 2 * U, true);
+    ALLOC(t.work, U * (size_t)t.W, false);
+    ALLOC(t.n_work, U, true);
     {
         size_t recs = U * (size_t)t.n_splits_attn;
         if (recs < 2 * (size_t)t.n_attn_ctas) recs = 2 * (size_t)t.n_attn_ctas;
@@ -305,16 +310,16 @@ static void enqueue_append_apply(dynakv_ctx* c, StepPtr k, StepPtr v, bool timed
     launch_append_apply(c->t, k, v, c->stream, &c->launches);
 }
 
-static const NextFront kNoNextFront = {0, StepPtr{nullptr, 0, nullptr}, StepPtr{nullptr, 0, nullptr}, nullptr, 0};
+static const NextFront kNoNextFront = {0, StepPtr{nullptr, 0, nullptr}, StepPtr{nullptr, 0, nullptr}, nullptr};
 
-// One iteration of a captured loop in two launches: gather-attention of step t, then the tail kernel, in which every
-// unit's block appends the step's key, runs the centroid pass of step t + 1 and the selection of step t + 1 (helper
-// blocks do the splits, and the selection of the units they split).  The pass and the selection of step 0 are launched
-// once ahead of the loop.  The tail kernel's last block advances the device-side step index that all kernels read.
+// One iteration of a captured loop in three launches.  The centroid pass of step t + 1 is part of the tail kernel
+// of step t (every unit's block runs it as soon as the unit's own append is done), so an iteration starts at the
+// selection; the pass of step 0 is launched once ahead of the loop.  The tail kernel's last block advances the
+// device-side step index that all kernels of the loop read.
 static void enqueue_loop_iteration(dynakv_ctx* c, StepPtr q, StepPtr k, StepPtr v, int budget, StepPtrW out) {
-    enqueue_attend(c, q, out, false);
+    enqueue_retrieve(c, q, budget, out, nullptr, false);
     launch_append_split(c->t, c->cfg.split_size_factor, c->cfg.split_var_factor > 0.f ? 1 : 0, c->cfg.split_min_size,
-                        c->cfg.split_iters, 1, k, v, c->step_ctr, NextFront{1, q, k, c->step_lim, budget}, c->stream, &c->launches);
+                        c->cfg.split_iters, 1, k, v, c->step_ctr, NextFront{1, q, k, c->step_lim}, c->stream, &c->launches);
 }
 
 extern "C" int dynakv_decode_step(dynakv_ctx* c, const float* q, int32_t token_budget, float* out, int32_t* selected_ids) {
@@ -399,7 +404,6 @@ extern "C" int dynakv_decode_loop(dynakv_ctx* c, const float* q_steps, const voi
         lb.on = 1; lb.step_ctr = c->step_ctr; lb.step_lim = c->step_lim; lb.n_steps = (int)n_steps; lb.args = c->loop_args;
         lb.q = q_steps; lb.k = k_steps; lb.v = v_steps; lb.out = out_steps;
         launch_front(c->t, StepPtr{q_steps, qs, nullptr}, StepPtr{k_steps, ks, nullptr}, 1, 1, c->stream, &c->launches, &lb);
-        launch_select(c->t, token_budget, nullptr, c->stream, &c->launches);     // step 0's selection (work lists of parity 0)
     }
     int64_t left = n_steps;
     for (int which = 0; which < dynakv_ctx::N_GRAPHS; which++) {

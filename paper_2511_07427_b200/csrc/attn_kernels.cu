@@ -118,11 +118,8 @@ __global__ void __launch_bounds__(AT_THREADS, 2) k_gather_attn_tma(Tables t, Ste
     }
     pdl_trigger();       // the append/split kernel may move in as CTAs of this grid retire; it waits before it moves rows
     pdl_wait();          // the work lists and their prefix come from the selection (the kernel before)
-    // inside a captured loop the step's work lists are the copy of the step's parity (the other copy is being
-    // written for the next step while this kernel runs)
-    const int buf = qp.ctr ? (*qp.ctr & 1) : 0;
-    const int* n_work = t.n_work + (size_t)buf * U;
-    const int2* work = t.work + (size_t)buf * U * t.W;
+    const int* n_work = t.n_work;
+    const int2* work = t.work;
     const int* pf = t.work_prefix;
     if (t.attn_pf_in_smem) {
         // Every CTA lays the units' work lists end to end itself: an exclusive prefix of their lengths, each

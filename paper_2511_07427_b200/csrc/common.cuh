@@ -44,10 +44,8 @@ struct Tables {
     float* dists;                    // [U][Mmax] squared distance of the step's new key to every representative
     int* sel_ids;                    // [U][Mmax]
     int* sel_n; int* sel_tokens;     // [U]
-    // The work lists exist twice: inside a captured loop the selection of step t + 1 is written (buffer (t + 1) & 1)
-    // while the gather-attention kernel of step t still reads its own (buffer t & 1); direct calls use buffer 0.
-    int2* work;                      // [2][U][W] (first row = page * PAGE + offset, rows <= ENTRY_ROWS)
-    int* n_work;                     // [2][U]
+    int2* work;                      // [U][W] (first row = page * PAGE + offset, rows <= ENTRY_ROWS)
+    int* n_work;                     // [U]
     float* part;                     // partial (acc, m, l) records of [G][d + 2] floats: [U][S] (plain kernel) or [2 * n_attn_ctas]
     int* work_prefix;                // [U + 1] exclusive prefix of n_work over the units (written by the last select block)
     int* unit_arrive;                // [U] arrival counters of the split-K combine (zero between steps)
@@ -222,7 +220,6 @@ struct NextFront {
     int on;                  // 0: no fused pass
     StepPtr q, k;            // per-step query and key arrays (indexed with step + 1)
     const int* step_lim;     // device: number of steps of the loop; the pass is skipped when step + 1 reaches it
-    int budget;              // token budget of the next step's selection, which follows the pass unit by unit
 };
 void launch_append_split(const Tables& t, float gamma, int var_enabled, int min_size, int iters, int do_append, StepPtr k,
                          StepPtr v, int* step_ctr, const NextFront& nf, cudaStream_t s, long long* launches);

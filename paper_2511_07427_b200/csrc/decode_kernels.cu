@@ -32,11 +32,10 @@ __global__ void __launch_bounds__(128) k_gather_attn_v1(Tables t, StepPtr qp) {
 #pragma unroll
         for (int e = 0; e < EPL; e++) acc[g][e] = 0.f;
     }
-    const int buf = qp.ctr ? (*qp.ctr & 1) : 0;      // inside a captured loop: the work lists of the step's parity
-    const int nw = t.n_work[(size_t)buf * t.U + u];
+    const int nw = t.n_work[u];
     const int per = (nw + S - 1) / S;
     const int w0 = s * per, w1 = min(nw, w0 + per);
-    const int2* work = t.work + ((size_t)buf * t.U + u) * t.W;
+    const int2* work = t.work + (size_t)u * t.W;
     const KV* kp = reinterpret_cast<const KV*>(t.kpages);
     const KV* vp = reinterpret_cast<const KV*>(t.vpages);
     for (int w = w0 + warp; w < w1; w += 4) {

@@ -96,7 +96,7 @@ __global__ void __launch_bounds__(FR_THREADS, 2) k_front(Tables t, StepPtr qp, S
 
 // ------------------------------------------------------------------ k_select
 
-// One block per unit: see select_unit().  Block size: 1024 threads when all units fit the GPU in one wave (the
+// One block per unit: see select_unit().  Block size: 512 threads when all units fit the GPU in one wave (the
 // shortest chain per block), 256 threads when there are more units than that (more blocks resident per SM; a
 // block's time is latency, not work).
 template <int THREADS>
@@ -152,7 +152,7 @@ void launch_front(const Tables& t, StepPtr q, StepPtr k, int has_q, int has_k, c
 
 void launch_select(const Tables& t, int budget, int* user_sel_ids, cudaStream_t s, long long* launches) {
     const size_t smem = select_smem_bytes(t.max_clusters);
-    if (t.U <= t.n_attn_ctas) launch_pdl(k_select<1024>, dim3(t.U), dim3(1024), smem, s, t, budget, user_sel_ids);
+    if (t.U <= t.n_attn_ctas) launch_pdl(k_select<512>, dim3(t.U), dim3(512), smem, s, t, budget, user_sel_ids);
     else launch_pdl(k_select<256>, dim3(t.U), dim3(256), smem, s, t, budget, user_sel_ids);
     (*launches)++;
 }

@@ -8,7 +8,6 @@
 #include "append_block.cuh"
 #include "common.cuh"
 #include "front_unit.cuh"
-#include "select_unit.cuh"
 #include "split_small.cuh"
 
 namespace dkv {
@@ -35,7 +34,6 @@ template <int HD, int KVB> struct SplitSmem {
     static constexpr int cache_rows = SP_CACHE_BYTES / (HD * KVB);
     static constexpr int stage_bytes = FrontUnit<SP_THREADS, HD>::STAGE_BYTES;
     static_assert(stage_bytes <= SP_CACHE_BYTES, "stages 0 and 1 of the centroid pass live in the staging areas");
-    static_assert(select_smem_bytes(SL_MAXM) <= 2 * (size_t)SP_CACHE_BYTES, "the selection's working set lies over the two staging areas");
     __host__ __device__ static size_t wsum_off(int maxch, int max_clusters) { return (((size_t)(2 * maxch + max_clusters) * sizeof(int)) + 15) & ~(size_t)15; }
     __host__ __device__ static size_t keys_off(int maxch, int max_clusters) {
         size_t a = wsum_off(maxch, max_clusters) + (size_t)SP_WARPS * 2 * HD * sizeof(float);
@@ -90,8 +88,7 @@ __device__ int next_queued_unit(const Tables& t, int* hint) {
 template <typename KV, int HD>
 __global__ void __launch_bounds__(SP_THREADS, DKV_SP_MINBLOCKS) k_split_check(Tables t, float gamma, int var_enabled, int min_size, int iters,
                                                             int do_append, StepPtr app_k, StepPtr app_v, int* step_ctr,
-                                                            int do_front, StepPtr next_q, StepPtr next_k, const int* step_lim,
-                                                            int next_budget) {
+                                                            int do_front, StepPtr next_q, StepPtr next_k, const int* step_lim) {
     constexpr int EPL = HD / 32;
     extern __shared__ __align__(128) int dyn[];
     __shared__ unsigned long long fr_bars[FR_STAGES];
@@ -106,6 +103,9 @@ __global__ void __launch_bounds__(SP_THREADS, DKV_SP_MINBLOCKS) k_split_check(Ta
     __shared__ int s_a, s_ok;
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    // The next kernel on the stream may be scheduled as soon as every block of this grid has started: its blocks move
+    // in as blocks of this grid retire, set themselves up and wait for this grid's completion before they read anything.
+    pdl_trigger();
     // In a loop iteration (do_front) the grid is U unit blocks followed by SP_HELPERS helper blocks: a unit block
     // appends, finds its triggered clusters, hands them to the helpers and runs the unit's centroid pass of the
     // next step; the helpers split.  Otherwise block u does the whole job for unit u.
@@ -138,10 +138,6 @@ __global__ void __launch_bounds__(SP_THREADS, DKV_SP_MINBLOCKS) k_split_check(Ta
     int* tok_s = reinterpret_cast<int*>(krows + (size_t)CACHE_ROWS * HD);
     if (tid == 0) { s_ntrig = 0; s_nsplit = 0; }
     int ntrig = 0;
-    // The next step's selection of a unit follows the unit's centroid pass inside this kernel (by the unit's block,
-    // or by the helper that split one of its clusters); its working set lies over the staging areas, which are
-    // free by then.  It writes the work lists of the next step's parity.
-    const SelectSmem sel_sm = select_smem_at(dynb + Lay::keys_off(maxch, t.max_clusters), t.max_clusters);
     if (!helper) {
         // The unit's centroid pass for the NEXT step starts here, ahead of the append: its first copies are in
         // flight while the append runs, and the one row the append changes is recomputed at the end of the pass.
@@ -233,12 +229,10 @@ __global__ void __launch_bounds__(SP_THREADS, DKV_SP_MINBLOCKS) k_split_check(Ta
             if (fronted) {
                 const float* q1 = reinterpret_cast<const float*>(next_q.at(t0 + 1)) + (size_t)u * t.G * HD;
                 const KV* k1 = reinterpret_cast<const KV*>(next_k.at(t0 + 1)) + (size_t)u * HD;
-                const bool passed = front_unit<KV, HD, SP_THREADS>(t, u, q1, k1, fr_issue, fr_stages, fr_live, last);
+                front_unit<KV, HD, SP_THREADS>(t, u, q1, k1, fr_issue, fr_stages, fr_live, last);
                 __threadfence();
                 __syncthreads();
                 if (tid == 0) atomicExch(t.front_done + u, t0 + 1);
-                // no split pending for this unit: nothing the selection reads can change any more
-                if (ntrig == 0 && passed) select_unit<SP_THREADS>(t, u, next_budget, nullptr, sel_sm, (t0 + 1) & 1);
             }
             ntrig = 0;            // nothing is split here
         }
@@ -277,7 +271,7 @@ __global__ void __launch_bounds__(SP_THREADS, DKV_SP_MINBLOCKS) k_split_check(Ta
         // Next step's scores and distances of the two children of a split, once the unit's own pass (which read the
         // rows as they were before, or half-way through, the split) can no longer overwrite them.  ra / rb: the
         // children's means (written before a block barrier).
-        auto wait_front = [&]() {
+        auto patch_children = [&](int ja, const float* ra, int jb, const float* rb) {
             if (!front_seen) {
                 if (tid == 0) {
                     int ok = 0;
@@ -293,9 +287,6 @@ __global__ void __launch_bounds__(SP_THREADS, DKV_SP_MINBLOCKS) k_split_check(Ta
                 __syncthreads();
                 front_seen = true;
             }
-        };
-        auto patch_children = [&](int ja, const float* ra, int jb, const float* rb) {
-            wait_front();
             if (s_flag && warp == 0) {
                 const float* q1 = reinterpret_cast<const float*>(next_q.at(t0 + 1)) + (size_t)u * t.G * HD;
                 const KV* k1 = reinterpret_cast<const KV*>(next_k.at(t0 + 1)) + (size_t)u * HD;
@@ -572,33 +563,18 @@ __global__ void __launch_bounds__(SP_THREADS, DKV_SP_MINBLOCKS) k_split_check(Ta
         if (!helper) break;
         __syncthreads();
         if (tid == 0 && s_nsplit > 0) t.u_scan[u] = 1;
-        if (fronted) {
-            // the unit's selection for the next step, on the clusters as the splits left them and on the scores as the
-            // unit's own pass and the patches above left them
-            wait_front();
-            __syncthreads();
-            if (s_flag) select_unit<SP_THREADS>(t, u, next_budget, nullptr, sel_sm, (t0 + 1) & 1);
-            __syncthreads();
-        }
     }
     __syncthreads();
     // No block leaves before the kernel ahead has completed: the next kernel on the stream (the next iteration's
     // centroid pass and selection, which rewrite the work lists) is ordered behind THIS kernel only.
     pdl_wait();
-    if (tid == 0 && !loop_mode) { t.u_scan[u] = s_nsplit > 0 ? 1 : 0; t.u_last[u] = -1; }
-    if (step_ctr) {
-        // the last block of the iteration lays the units' new work lists end to end when the gather-attention
-        // kernel does not do that itself (more than 1024 units), clears the hand-over words for the next iteration
-        // and advances the device-side step index that every kernel of the loop reads
-        if (tid == 0) {
+    if (tid == 0) {
+        if (!loop_mode) { t.u_scan[u] = s_nsplit > 0 ? 1 : 0; t.u_last[u] = -1; }
+        if (step_ctr) {
+            // the last block of the iteration advances the device-side step index that every kernel of the loop reads,
+            // and clears the hand-over words for the next iteration
             __threadfence();
-            s_flag = (atomicAdd(t.plan_counter + 1, 1) == (int)gridDim.x - 1) ? 1 : 0;
-        }
-        __syncthreads();
-        if (s_flag) {
-            __threadfence();
-            if (fronted && !t.attn_pf_in_smem) work_prefix_block<SP_THREADS>(t, sh, (t0 + 1) & 1);
-            if (tid == 0) {
+            if (atomicAdd(t.plan_counter + 1, 1) == (int)gridDim.x - 1) {
                 t.plan_counter[1] = 0; t.tail_sync[0] = 0; t.tail_sync[1] = 0; t.tail_sync[2] = 0;
                 *step_ctr += 1;
             }
@@ -619,13 +595,13 @@ static void split_t(const Tables& t, float gamma, int var_enabled, int min_size,
         if (dev >= 0 && dev < 64) opted[dev] = dyn;
     }
     launch_pdl(k_split_check<KV, HD>, dim3(t.U + (nf.on ? SP_HELPERS : 0)), dim3(SP_THREADS), dyn, s, t, gamma, var_enabled, min_size, iters, do_append, k, v, step_ctr,
-               nf.on, nf.q, nf.k, nf.step_lim, nf.budget);
+               nf.on, nf.q, nf.k, nf.step_lim);
 }
 
 void launch_split_check(const Tables& t, float gamma, int var_enabled, int min_size, int iters, cudaStream_t s,
                         long long* launches) {
     launch_append_split(t, gamma, var_enabled, min_size, iters, 0, StepPtr{nullptr, 0, nullptr}, StepPtr{nullptr, 0, nullptr}, nullptr,
-                        NextFront{0, StepPtr{nullptr, 0, nullptr}, StepPtr{nullptr, 0, nullptr}, nullptr, 0}, s, launches);
+                        NextFront{0, StepPtr{nullptr, 0, nullptr}, StepPtr{nullptr, 0, nullptr}, nullptr}, s, launches);
 }
 
 // The tail of a fused loop iteration in one launch: append (when do_append), the next step's centroid pass (when

@@ -153,6 +153,44 @@ def test_zero_query_breaks_score_ties_by_id():
     ctx.destroy()
 
 
+def test_selection_with_bunched_scores_and_outliers():
+    """The selection's short way ranks the few clusters of one histogram bin against each other and leaves the job
+    to the general radix version when that bin holds more than 64 clusters.  Queries are crafted so that: all
+    scores are equal (every cluster in one bin, ties by id); one cluster scores far above a bunch of nearly equal
+    ones (the bunch shares a bin); scores are spread out (the common case); and budgets fall on both sides of the
+    boundaries.  Every selection must equal the oracle's."""
+    from parity_harness import make_oracle
+    cfg = CONFIGS[2].scaled(B=1, L=1, Hkv=1, Hq=4, n_prefill=3000, steps=4, M0=150, max_clusters=256, budget=400, T=3)
+    s = [UnitStream(cfg, 0)]
+    K, V = make_prefill(s)
+    ctx = _single_ctx(cfg, K, V, assign_mode=1)
+    st = ctx.export_state()
+    o = make_oracle(cfg)
+    o.install(K[0].double().numpy(), V[0].double().numpy(), st["tok_cluster"][0, :cfg.n_prefill], int(st["n_ids"][0]))
+    C = torch.from_numpy(st["centroids"][0, :cfg.M0]).float()
+    g = torch.Generator().manual_seed(5)
+    # a direction nearly orthogonal to every representative, plus a large multiple of one representative's own direction
+    r = torch.randn(cfg.d, generator=g)
+    r = r - C.T @ torch.linalg.lstsq(C @ C.T + 1e-3 * torch.eye(cfg.M0), C @ r).solution
+    queries = {
+        "equal": torch.zeros(cfg.G, cfg.d),
+        "bunched": (1e-4 * r + 50.0 * C[7] / C[7].norm() ** 2).repeat(cfg.G, 1),
+        "spread": torch.randn(cfg.G, cfg.d, generator=g),
+    }
+    sel = torch.full((1, cfg.max_clusters), -1, dtype=torch.int32, device="cuda")
+    for name, q in queries.items():
+        q = q.to(torch.bfloat16).float()
+        for budget in (1, 25, 400, 1500, 2999, 3000, 10 ** 6):
+            ctx.decode_step(q[None].cuda(), budget, selected_ids=sel)
+            nsel, ntok = ctx.get_selection()
+            ids = sel[0].cpu().numpy()[: nsel[0]]
+            v0 = o.violations
+            _, ids_o, tok_o = o.decode_step(q.double().numpy(), budget, hint_ids=ids)
+            assert o.violations == v0 and list(ids_o) == list(ids) and tok_o == int(ntok[0]), \
+                f"{name}, budget {budget}: gpu {ids[:10]} oracle {ids_o[:10]}"
+    ctx.destroy()
+
+
 def test_duplicate_keys_leave_dead_clusters():
     cfg = CONFIGS[1].scaled(n_prefill=256, steps=16, M0=12, max_clusters=32, budget=80, T=4, init_mode="random")
     from parity_harness import make_ctx, make_oracle, check_state, ParityReport
