@@ -19,6 +19,7 @@ _LIB = os.path.join(_HERE, "libdynakv_oracle.so")
 
 INIT_KMEANSPP = 0
 INIT_RANDOM = 1
+MODE_ADAPTIVE, MODE_STATIC, MODE_LOCAL = 0, 1, 2
 ST_BUDGET_EXCEEDED = 1
 ST_MAX_CLUSTERS = 2
 ST_MAX_TOKENS = 4
@@ -82,6 +83,7 @@ def lib() -> C.CDLL:
         L.ork_get_M2.argtypes = [C.c_void_p, dp]
         L.ork_get_live.argtypes = [C.c_void_p, bp]
         L.ork_set_tau.argtypes = [C.c_void_p, C.c_double]
+        L.ork_set_mode.argtypes = [C.c_void_p, C.c_int, C.c_int]
     return _lib
 
 
@@ -150,10 +152,12 @@ class OracleUnit:
     """One unit (one KV head) of the oracle: the four verbs of the library plus getters."""
 
     def __init__(self, d: int, G: int, max_tokens: int, max_clusters: int, gamma: float = 2.0,
-                 alpha: float = 2.0, split_min_size: int = 8, split_iters: int = 8, tol: float = 1e-5):
+                 alpha: float = 2.0, split_min_size: int = 8, split_iters: int = 8, tol: float = 1e-5,
+                 mode: int = MODE_ADAPTIVE, local_max: int = 64):
         self.d, self.G, self.max_tokens, self.max_clusters = d, G, max_tokens, max_clusters
         self._h = C.c_void_p(lib().ork_create(d, G, max_tokens, max_clusters, gamma, alpha,
                                                split_min_size, split_iters, tol))
+        lib().ork_set_mode(self._h, mode, local_max)
 
     def __del__(self):
         try:

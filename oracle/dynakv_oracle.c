@@ -20,7 +20,8 @@
  * scikit-learn Lloyd cross-check, D^2-sampling frequencies, Welford vs two-pass,
  * full-budget retrieval == dense softmax attention, split invariants, the round cap of
  * the split's 2-means (hand-worked fixture), validity of a selection hint (including the
- * over-budget single-cluster case).
+ * over-budget single-cluster case), the static and local update modes (frozen build, brute-force
+ * append targets, separation of two new blobs).
  * Conventions the paper leaves open (score metric, GQA reduction, threshold
  * calibration, split seeding, id rule, budget boundary) are "parity unpinned" by the
  * paper: they are pinned only to their stated definitions.
@@ -32,6 +33,16 @@
 
 #define ORK_INIT_KMEANSPP 0
 #define ORK_INIT_RANDOM 1
+
+/* How the partition follows the decode stream (Section 3.1 and the baselines of Section 8.1):
+ *   ADAPTIVE  append to the nearest cluster, split clusters that grow too large or too spread out (the paper's method);
+ *   STATIC    append to the nearest cluster, never split ("static update");
+ *   LOCAL     new entries are clustered among themselves only ("local update"): clusters of the prefill build never
+ *             change; a new entry joins the nearest cluster born during decoding (the first one founds it), and such a
+ *             cluster is split by the same 2-means once it holds more than local_max entries. */
+#define ORK_MODE_ADAPTIVE 0
+#define ORK_MODE_STATIC 1
+#define ORK_MODE_LOCAL 2
 
 #define ORK_ST_BUDGET_EXCEEDED 1u
 #define ORK_ST_MAX_CLUSTERS 2u
@@ -54,6 +65,8 @@ typedef struct {
     long ties, violations;
     unsigned status;
     long n_splits;
+    int mode, local_max;  /* update mode; LOCAL: size above which a decode-born cluster splits */
+    int M_build;          /* ids handed out by the build (or installed): the "old" clusters of LOCAL mode */
 } ork_unit;
 
 /* ---------------------------------------------------------------- helpers */
@@ -241,7 +254,7 @@ int ork_build(ork_unit *u, const double *K, const double *V, int n, int n_cluste
     if (n > u->max_tokens || M > u->max_clusters || n < M || M < 1) return -1;
     memcpy(u->K, K, sizeof(double) * (size_t)n * d);
     memcpy(u->V, V, sizeof(double) * (size_t)n * d);
-    u->n = n; u->M = M;
+    u->n = n; u->M = M; u->M_build = M;
     int *picks = (int *)malloc(sizeof(int) * (size_t)M);
     if (init_mode == ORK_INIT_KMEANSPP)
         ork_init_kmeanspp(u->K, n, d, M, seed, unit_index, hint_picks, u->tol, picks, &u->ties, &u->violations);
@@ -425,14 +438,37 @@ int ork_append(ork_unit *u, const double *k, const double *v, int hint_cluster) 
     int d = u->d;
     if (u->n >= u->max_tokens) { u->status |= ORK_ST_MAX_TOKENS; return -1; }
     int best = -1; double bd = 0.0;
-    for (int j = 0; j < u->M; j++) {
+    /* LOCAL mode: only clusters born during decoding are candidates */
+    int j0 = (u->mode == ORK_MODE_LOCAL) ? u->M_build : 0;
+    for (int j = j0; j < u->M; j++) {
         if (!u->live[j]) continue;
         double dd = sqdist(k, u->r + (size_t)j * d, d);
         if (best < 0 || dd < bd) { bd = dd; best = j; }
     }
+    if (best < 0 && u->mode == ORK_MODE_LOCAL) {
+        if (u->M < u->max_clusters) {
+            /* the first new entry founds a cluster of its own: r = k, M2 = 0 */
+            int id = u->M++;
+            int i = u->n++;
+            memcpy(u->K + (size_t)i * d, k, sizeof(double) * d);
+            memcpy(u->V + (size_t)i * d, v, sizeof(double) * d);
+            u->assign[i] = id;
+            memcpy(u->r + (size_t)id * d, k, sizeof(double) * d);
+            u->M2[id] = 0.0; u->cnt[id] = 1; u->live[id] = 1; u->hold[id] = 0;
+            return id;
+        }
+        /* no id left: fall back to the nearest cluster of all */
+        u->status |= ORK_ST_MAX_CLUSTERS;
+        for (int j = 0; j < u->M; j++) {
+            if (!u->live[j]) continue;
+            double dd = sqdist(k, u->r + (size_t)j * d, d);
+            if (best < 0 || dd < bd) { bd = dd; best = j; }
+        }
+        j0 = 0;
+    }
     if (best < 0) return -1;
     if (hint_cluster >= 0 && hint_cluster != best) {
-        if (hint_cluster < u->M && u->live[hint_cluster] &&
+        if (hint_cluster >= j0 && hint_cluster < u->M && u->live[hint_cluster] &&
             near_tie(sqdist(k, u->r + (size_t)hint_cluster * d, d), bd, u->tol)) { best = hint_cluster; u->ties++; }
         else u->violations++;
     }
@@ -509,6 +545,7 @@ static int two_means(const ork_unit *u, const int *mem, int nm, unsigned char *l
  * its own split check.  Returns the number of splits performed. */
 int ork_split_check(ork_unit *u, const int *hint_assign_after) {
     int d = u->d, n = u->n, M0 = u->M, done = 0;
+    if (u->mode == ORK_MODE_STATIC) return 0;
     int Mlive = 0;
     for (int j = 0; j < M0; j++) Mlive += u->live[j];
     int *mem = (int *)malloc(sizeof(int) * (size_t)(n > 0 ? n : 1));
@@ -519,6 +556,11 @@ int ork_split_check(ork_unit *u, const int *hint_assign_after) {
     unsigned char *vartie = (unsigned char *)calloc((size_t)M0, 1);
     for (int j = 0; j < M0; j++) {
         if (!u->live[j] || u->hold[j] || u->cnt[j] < u->split_min_size) continue;
+        if (u->mode == ORK_MODE_LOCAL) {
+            /* only decode-born clusters split, and only by their absolute size */
+            trig[j] = j >= u->M_build && u->cnt[j] > u->local_max;
+            continue;
+        }
         double var = u->M2[j] / u->cnt[j];
         int by_var = u->alpha > 0.0 && var > u->tau;
         int by_size = u->gamma > 0.0 && (double)u->cnt[j] * (double)Mlive > u->gamma * (double)n;
@@ -585,7 +627,7 @@ int ork_install(ork_unit *u, const double *K, const double *V, int n, const int 
     memcpy(u->K, K, sizeof(double) * (size_t)n * d);
     memcpy(u->V, V, sizeof(double) * (size_t)n * d);
     memcpy(u->assign, assign, sizeof(int) * (size_t)n);
-    u->n = n; u->M = M;
+    u->n = n; u->M = M; u->M_build = M;
     double vs = 0.0; int nl = 0;
     for (int j = 0; j < M; j++) {
         u->hold[j] = 0;
@@ -612,3 +654,4 @@ void ork_get_counts(const ork_unit *u, int *out) { memcpy(out, u->cnt, sizeof(in
 void ork_get_M2(const ork_unit *u, double *out) { memcpy(out, u->M2, sizeof(double) * (size_t)u->M); }
 void ork_get_live(const ork_unit *u, unsigned char *out) { memcpy(out, u->live, (size_t)u->M); }
 void ork_set_tau(ork_unit *u, double tau) { u->tau = tau; }
+void ork_set_mode(ork_unit *u, int mode, int local_max) { u->mode = mode; u->local_max = local_max; }

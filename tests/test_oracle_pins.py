@@ -553,3 +553,79 @@ def test_install_reproduces_the_state_of_a_build():
     # centroid of an installed cluster is the plain mean of its members
     j = int(np.argmax(b.counts()))
     assert np.allclose(b.centroids()[j], K[a.assign() == j].mean(0), atol=1e-13)
+
+
+# ------------------------------------------------------------------ update modes (static / local)
+
+def _mode_stream(seed=3, n0=300, d=8, steps=160):
+    rng = np.random.default_rng(seed)
+    means = rng.normal(size=(6, d)) * 4.0
+    K0 = means[rng.integers(0, 6, n0)] + 0.3 * rng.normal(size=(n0, d))
+    # decode keys drift away from the prefill mixture
+    Kd = means[rng.integers(0, 6, steps)] + 0.3 * rng.normal(size=(steps, d)) + np.linspace(0, 6, steps)[:, None]
+    return K0, Kd
+
+
+def test_static_mode_never_splits_and_appends_to_the_nearest_representative():
+    K0, Kd = _mode_stream()
+    u = O.OracleUnit(K0.shape[1], 1, 600, 64, gamma=1.2, alpha=1.2, split_min_size=4, mode=O.MODE_STATIC)
+    u.build(K0, K0, 8, 3, seed=2, init_mode=O.INIT_RANDOM)
+    for k in Kd:
+        C, live = u.centroids(), u.live()
+        dist = ((C - k[None]) ** 2).sum(1)
+        dist[~live] = np.inf
+        j = u.append(k, k)
+        assert j == int(np.argmin(dist))                       # brute force over the representatives as they were
+        assert u.split_check() == 0
+    assert u.M == 8 and u.n_splits == 0
+    # the same stream with the split rules on does split: the mode is what keeps the partition static
+    a = O.OracleUnit(K0.shape[1], 1, 600, 64, gamma=1.2, alpha=1.2, split_min_size=4)
+    a.build(K0, K0, 8, 3, seed=2, init_mode=O.INIT_RANDOM)
+    for k in Kd:
+        a.append(k, k); a.split_check()
+    assert a.n_splits > 0
+
+
+def test_local_mode_keeps_the_build_frozen_and_clusters_new_entries_among_themselves():
+    K0, Kd = _mode_stream()
+    M0, local_max = 8, 24
+    u = O.OracleUnit(K0.shape[1], 1, 600, 64, gamma=1.2, alpha=1.2, split_min_size=4, mode=O.MODE_LOCAL, local_max=local_max)
+    u.build(K0, K0, M0, 3, seed=2, init_mode=O.INIT_RANDOM)
+    C0, n0, m20, a0 = u.centroids().copy(), u.counts().copy(), u.M2().copy(), u.assign().copy()
+    first = u.append(Kd[0], Kd[0])
+    assert first == M0 and u.M == M0 + 1                       # the first new entry founds a cluster of its own
+    assert np.array_equal(u.centroids()[M0], Kd[0]) and u.M2()[M0] == 0.0 and u.counts()[M0] == 1
+    u.split_check()
+    for k in Kd[1:]:
+        C, live = u.centroids(), u.live()
+        dist = ((C - k[None]) ** 2).sum(1)
+        dist[~live] = np.inf
+        dist[:M0] = np.inf                                      # only decode-born clusters are candidates
+        j = u.append(k, k)
+        assert j == int(np.argmin(dist)) and j >= M0
+        u.split_check()
+        assert u.counts()[M0:].max() <= local_max               # a cluster above the limit has just been split
+    # the clusters of the build are exactly as the build left them
+    assert np.array_equal(u.centroids()[:M0], C0) and np.array_equal(u.counts()[:M0], n0)
+    assert np.array_equal(u.M2()[:M0], m20) and np.array_equal(u.assign()[: len(a0)], a0)
+    assert np.all(u.assign()[len(a0):] >= M0) and u.n_splits > 0
+    # Eq. 3 / Eq. 4 hold for the new clusters too
+    A = u.assign(); Kall = np.concatenate([K0, Kd])
+    for j in range(M0, u.M):
+        mem = Kall[A == j]
+        assert len(mem) == u.counts()[j] and np.allclose(mem.mean(0), u.centroids()[j], atol=1e-10)
+
+
+def test_local_mode_separates_two_new_blobs_when_the_size_limit_is_reached():
+    rng = np.random.default_rng(8)
+    K0 = rng.normal(size=(100, 4))
+    blobs = np.array([[50.0, 0, 0, 0], [0, 50.0, 0, 0]])
+    lab = np.arange(41) % 2
+    Kd = blobs[lab] + 0.1 * rng.normal(size=(41, 4))
+    u = O.OracleUnit(4, 1, 200, 16, split_min_size=4, mode=O.MODE_LOCAL, local_max=40)
+    u.build(K0, K0, 4, 2, seed=1, init_mode=O.INIT_RANDOM)
+    for k in Kd:
+        u.append(k, k); u.split_check()
+    A = u.assign()[100:]
+    assert u.M == 6 and u.n_splits == 1                          # one founding, one split at 41 entries
+    assert len(set(A[lab == 0])) == 1 and len(set(A[lab == 1])) == 1 and A[0] != A[1]
