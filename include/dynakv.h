@@ -68,7 +68,19 @@ typedef struct dynakv_config {
     int32_t trace;             /* 1: keep every Lloyd round's assignment for dynakv_get_build_trace */
     int32_t assign_mode;       /* 0: auto (tensor-core distance GEMM for bf16, d=128), 1: force fp32 path */
     int32_t attn_mode;         /* 0: auto (tensor-core gather-attention for bf16 K/V), 1: force the plain fp32 kernel */
+    int32_t update_mode;       /* DYNAKV_MODE_ADAPTIVE (0, the paper's method), DYNAKV_MODE_STATIC or DYNAKV_MODE_LOCAL */
+    int32_t local_max;         /* DYNAKV_MODE_LOCAL: a cluster born during decoding splits above this size (>= 2)    */
 } dynakv_config;
+
+/* How the partition follows the decode stream (Section 3.1; the baselines of Section 8.1):
+ *   ADAPTIVE  append to the nearest cluster; split_check splits clusters by the variance and size rules;
+ *   STATIC    append to the nearest cluster; split_check never splits ("static update");
+ *   LOCAL     new entries are clustered among themselves only ("local update"): the clusters of the build never
+ *             change; append joins the nearest cluster born during decoding (the first new entry founds one), and
+ *             split_check splits such a cluster by the same 2-means once it holds more than local_max entries. */
+#define DYNAKV_MODE_ADAPTIVE 0
+#define DYNAKV_MODE_STATIC 1
+#define DYNAKV_MODE_LOCAL 2
 
 typedef struct dynakv_status {
     uint32_t error_bits;       /* OR of DYNAKV_ST_*                                              */

@@ -124,6 +124,8 @@ extern "C" int dynakv_create(const dynakv_config* cfg, void* cuda_stream, dynakv
     if (cfg->max_tokens < 1 || cfg->max_clusters < 1 || cfg->max_clusters > 4096) return DYNAKV_ERR_ARG;
     if (cfg->kmeans_iters < 1 || cfg->split_iters < 1) return DYNAKV_ERR_ARG;
     if (cfg->init_mode != DYNAKV_INIT_KMEANSPP && cfg->init_mode != DYNAKV_INIT_RANDOM) return DYNAKV_ERR_ARG;
+    if (cfg->update_mode < DYNAKV_MODE_ADAPTIVE || cfg->update_mode > DYNAKV_MODE_LOCAL) return DYNAKV_ERR_ARG;
+    if (cfg->update_mode == DYNAKV_MODE_LOCAL && cfg->local_max < 2) return DYNAKV_ERR_ARG;
     dynakv_ctx* c = new (std::nothrow) dynakv_ctx();
     if (!c) return DYNAKV_ERR_NOMEM;
     c->cfg = *cfg;
@@ -132,6 +134,7 @@ extern "C" int dynakv_create(const dynakv_config* cfg, void* cuda_stream, dynakv
     memset(&t, 0, sizeof(t));
     t.U = cfg->n_units; t.G = cfg->gqa_group; t.d = cfg->head_dim; t.kv_dtype = cfg->kv_dtype;
     t.max_tokens = cfg->max_tokens; t.max_clusters = cfg->max_clusters;
+    t.update_mode = cfg->update_mode; t.local_max = cfg->local_max;
     const int full_pages = (cfg->max_tokens + PAGE - 1) / PAGE;
     int slack = full_pages / 8; if (slack < 64) slack = 64;
     t.P = full_pages + cfg->max_clusters + slack;

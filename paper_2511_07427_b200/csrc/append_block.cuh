@@ -7,7 +7,8 @@
 
 namespace dkv {
 
-// One block per unit: argmin over the distances written by k_front (ties to the lowest id),
+// One block per unit: argmin over the distances written by k_front (ties to the lowest id; in the local-update
+// mode only over the clusters born during decoding, and a first new entry founds a cluster of its own),
 // then n <- n+1, delta = k - r, r <- r + delta/n, M2 <- M2 + delta.(k - r_new), and the
 // (k, v) row goes to the next slot of the cluster's tail page (a fresh page is linked when
 // the tail is full).  No stored entry moves.
@@ -34,7 +35,9 @@ __device__ __forceinline__ void append_block(const Tables& t, int u, StepPtr kp_
     if (N >= t.max_tokens) { if (tid == 0) atomicOr(t.status, DYNAKV_ST_MAX_TOKENS); return; }
     const float* DS = t.dists + (size_t)u * t.max_clusters;
     float bd = INFINITY; int bj = 0x7fffffff;
-    for (int j = tid; j < Mcur; j += blockDim.x) {
+    // local-update mode: the clusters of the build (ids below M_floor) take no new entries
+    const int j_first = t.update_mode == DYNAKV_MODE_LOCAL ? t.M_floor : 0;
+    for (int j = j_first + tid; j < Mcur; j += blockDim.x) {
         const float dd = DS[j];
         if (dd < bd) { bd = dd; bj = j; }
     }
@@ -49,21 +52,40 @@ __device__ __forceinline__ void append_block(const Tables& t, int u, StepPtr kp_
     bd = red_d[0]; bj = red_j[0];
 #pragma unroll
     for (int w = 1; w < nwarp; w++) if (red_d[w] < bd || (red_d[w] == bd && red_j[w] < bj)) { bd = red_d[w]; bj = red_j[w]; }
-    if (bj == 0x7fffffff) return;    // no live cluster
     const KV* knew = reinterpret_cast<const KV*>(kp_.get()) + (size_t)u * HD;
     const KV* vnew = reinterpret_cast<const KV*>(vp_.get()) + (size_t)u * HD;
+    bool found = false;              // local-update mode: the entry founds a new cluster
+    if (bj == 0x7fffffff && t.update_mode == DYNAKV_MODE_LOCAL) {
+        if (Mcur < t.max_clusters) { bj = Mcur; found = true; }
+        else {
+            // no id left: the nearest cluster of all takes the entry
+            if (lane == 0) atomicOr(t.status, DYNAKV_ST_MAX_CLUSTERS);
+            for (int j = lane; j < Mcur; j += 32) {
+                const float dd = DS[j];
+                if (dd < bd || (dd == bd && j < bj)) { bd = dd; bj = j; }
+            }
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) {
+                const float od = __shfl_xor_sync(0xffffffffu, bd, o); const int oj = __shfl_xor_sync(0xffffffffu, bj, o);
+                if (od < bd || (od == bd && oj < bj)) { bd = od; bj = oj; }
+            }
+        }
+    }
+    if (bj == 0x7fffffff) return;    // no live cluster
     const size_t cj = (size_t)u * t.max_clusters + bj;
-    const int n_old = t.cl_n[cj];
-    int page = t.cl_tail[cj];
+    const int n_old = found ? 0 : t.cl_n[cj];
+    int page = found ? -1 : t.cl_tail[cj];
     const int row = n_old % PAGE;
-    if (row == 0) {   // tail is full: link a fresh page
+    if (row == 0) {   // tail is full (or there is no page yet): link a fresh page
         int np = -1;
         if (lane == 0) {
             int fc = t.u_free_cnt[u];
             if (fc > 0) { np = t.free_stack[(size_t)u * t.P + fc - 1]; t.u_free_cnt[u] = fc - 1; }
             else { int top = t.u_page_top[u]; if (top < t.P) { np = top; t.u_page_top[u] = top + 1; } }
-            if (np >= 0) { t.page_next[(size_t)u * t.P + page] = np; t.page_next[(size_t)u * t.P + np] = -1; t.cl_tail[cj] = np; }
-            else atomicOr(t.status, DYNAKV_ST_PAGE_POOL);
+            if (np >= 0) {
+                if (page >= 0) t.page_next[(size_t)u * t.P + page] = np; else t.cl_head[cj] = np;
+                t.page_next[(size_t)u * t.P + np] = -1; t.cl_tail[cj] = np;
+            } else atomicOr(t.status, DYNAKV_ST_PAGE_POOL);
         }
         np = __shfl_sync(0xffffffffu, np, 0);
         if (np < 0) return;
@@ -76,7 +98,7 @@ __device__ __forceinline__ void append_block(const Tables& t, int u, StepPtr kp_
 #pragma unroll
     for (int e = 0; e < EPL; e++) {
         kk[e] = to_f(knew[lane * EPL + e]);
-        const float ro = r[lane * EPL + e];
+        const float ro = found ? kk[e] : r[lane * EPL + e];          // a founded cluster starts at r = k, M2 = 0
         const float delta = kk[e] - ro;
         const float rn = ro + delta / n_new;
         r[lane * EPL + e] = rn;
@@ -88,11 +110,12 @@ __device__ __forceinline__ void append_block(const Tables& t, int u, StepPtr kp_
 #pragma unroll
     for (int e = 0; e < EPL; e++) { kpg[lane * EPL + e] = knew[lane * EPL + e]; vpg[lane * EPL + e] = vnew[lane * EPL + e]; }
     if (lane == 0) {
-        const float m2_new = t.cl_M2[cj] + add;
+        const float m2_new = found ? 0.f : t.cl_M2[cj] + add;
         t.cl_M2[cj] = m2_new;
+        if (found) { t.u_M[u] = Mcur + 1; t.u_Mlive[u] = t.u_Mlive[u] + 1; }
         if (res) { res->cluster = bj; res->n_new = n_old + 1; res->M2_new = m2_new; res->N_new = N + 1; }
         t.cl_n[cj] = n_old + 1;
-        t.cl_flags[cj] &= ~FLAG_HOLD;
+        t.cl_flags[cj] = found ? 0 : (t.cl_flags[cj] & ~FLAG_HOLD);
         t.page_tok[((size_t)u * t.P + page) * PAGE + row] = N;
         t.tok_cluster[(size_t)u * t.max_tokens + N] = bj;
         t.u_N[u] = N + 1;

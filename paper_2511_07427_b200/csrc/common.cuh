@@ -25,6 +25,7 @@ constexpr int FLAG_HOLD = 1;        // split abandoned; not retried until the ne
 //   full, so cluster members are contiguous page by page (intra-cluster placement).
 struct Tables {
     int U, G, d, kv_dtype, max_tokens, max_clusters, P, n_splits_attn;
+    int update_mode, local_max;      // DYNAKV_MODE_*; LOCAL: size above which a decode-born cluster splits
     int W;                           // work-list capacity per unit (entries)
     int M_floor;                     // clusters every unit has had since the build (ids never go away); 0 before it
     void* kpages; void* vpages;

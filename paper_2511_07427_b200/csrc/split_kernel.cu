@@ -168,9 +168,15 @@ __global__ void __launch_bounds__(SP_THREADS, DKV_SP_MINBLOCKS) k_split_check(Ta
                 const int c = s_app.n_new;
                 // the append cleared the cluster's hold flag
                 if (c >= min_size) {
-                    const bool by_var = var_enabled && (s_app.M2_new / (float)c > tau);
-                    const bool by_size = gamma > 0.f && ((double)c * (double)Mlive0 > (double)gamma * (double)s_app.N_new);
-                    if (by_var || by_size) { trig[0] = last; s_ntrig = 1; }
+                    bool hit;
+                    if (t.update_mode == DYNAKV_MODE_LOCAL) hit = last >= t.M_floor && c > t.local_max;   // decode-born clusters, by absolute size
+                    else if (t.update_mode == DYNAKV_MODE_STATIC) hit = false;
+                    else {
+                        const bool by_var = var_enabled && (s_app.M2_new / (float)c > tau);
+                        const bool by_size = gamma > 0.f && ((double)c * (double)Mlive0 > (double)gamma * (double)s_app.N_new);
+                        hit = by_var || by_size;
+                    }
+                    if (hit) { trig[0] = last; s_ntrig = 1; }
                 }
             }
             __syncthreads();
@@ -185,9 +191,13 @@ __global__ void __launch_bounds__(SP_THREADS, DKV_SP_MINBLOCKS) k_split_check(Ta
                 const size_t cj = (size_t)u * t.max_clusters + j;
                 const int c = t.cl_n[cj];
                 if (c > 0 && c >= min_size && !(t.cl_flags[cj] & FLAG_HOLD)) {
-                    const bool by_var = var_enabled && (t.cl_M2[cj] / (float)c > tau);
-                    const bool by_size = gamma > 0.f && ((double)c * (double)Mlive0 > (double)gamma * (double)N);
-                    hit = (by_var || by_size) ? 1 : 0;
+                    if (t.update_mode == DYNAKV_MODE_LOCAL) hit = (j >= t.M_floor && c > t.local_max) ? 1 : 0;
+                    else if (t.update_mode == DYNAKV_MODE_STATIC) hit = 0;
+                    else {
+                        const bool by_var = var_enabled && (t.cl_M2[cj] / (float)c > tau);
+                        const bool by_size = gamma > 0.f && ((double)c * (double)Mlive0 > (double)gamma * (double)N);
+                        hit = (by_var || by_size) ? 1 : 0;
+                    }
                 }
             }
             int tot;

@@ -216,6 +216,14 @@ def test_duplicate_keys_leave_dead_clusters():
     ctx.destroy()
 
 
+def test_graph_loop_in_local_update_mode():
+    # the captured loop founds a cluster for the first new entry inside the tail kernel (an id beyond the ones the
+    # unit's centroid pass covered) and splits decode-born clusters above 20 entries
+    cfg = CONFIGS[2].scaled(B=1, L=1, Hkv=1, Hq=4, n_prefill=400, steps=90, M0=10, max_clusters=64, budget=200, T=3,
+                            update_mode="local", local_max=20)
+    assert _loop_vs_direct(cfg, [0, 1, 2, 3, 4], 90, cut=31) >= 5
+
+
 def _loop_vs_direct(cfg, units, steps, modes=("direct", "graph", "host"), cut=None):
     """The captured loop (and the host-buffer step) must leave the same state and outputs as direct calls."""
     s = [UnitStream(cfg, u) for u in units]

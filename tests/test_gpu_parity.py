@@ -37,6 +37,20 @@ def test_scaled_bf16_configs(cid):
     _run(cfg, [0, 1, 2], cfg.steps, assign_mode=1)
 
 
+@pytest.mark.parametrize("mode", ["static", "local"])
+def test_update_modes(mode):
+    """The static-update and local-update modes (Section 3.1; the baselines of Section 8.1) against the oracle's: drifting
+    keys with new mixture components, so that the adaptive rule would split; static never does, local founds clusters
+    for the new entries, keeps the build frozen and splits the new clusters above 24 entries."""
+    cfg = CONFIGS[3].scaled(n_prefill=500, steps=200, M0=12, max_clusters=96, budget=300, T=4, new_every=64,
+                            update_mode=mode, local_max=24)
+    rep = _run(cfg, [0, 1, 2], cfg.steps, assign_mode=1)
+    if mode == "static":
+        assert rep.gpu_splits == 0 and rep.splits == 0
+    else:
+        assert rep.splits >= 3 * 4          # 200 new entries in clusters of at most 24: several splits per unit
+
+
 @pytest.mark.parametrize("cid", [2, 5])
 def test_tensor_core_assign_ragged(cid):
     """Distance GEMM on the tensor cores (assign_mode 0): 1111 keys = 8 full 128-key blocks + 87, 37 centres
