@@ -166,6 +166,13 @@ int dynakv_decode_loop(dynakv_ctx* ctx, const float* q_steps, const void* k_step
 int dynakv_step_host(dynakv_ctx* ctx, const float* q_host, const void* k_host,
                      const void* v_host, int32_t token_budget, float* out_host);
 
+/* dynakv_decode_loop with HOST arrays (same shapes; pinned memory for the copies to overlap): the steps are taken in
+ * chunks of 32; while the loop runs one chunk on the device, the next chunk's q, k, v are copied in and the
+ * previous chunk's outputs copied out on two more streams.  Returns when every output is in out_steps.  For a
+ * caller that has its inputs step by step, dynakv_step_host is the call. */
+int dynakv_decode_loop_host(dynakv_ctx* ctx, const float* q_steps, const void* k_steps, const void* v_steps,
+                            int64_t n_steps, int32_t token_budget, float* out_steps);
+
 /* Synchronises the stream and fills *host_out (host memory). */
 int dynakv_get_status(dynakv_ctx* ctx, dynakv_status* host_out);
 
@@ -177,6 +184,20 @@ int dynakv_get_status(dynakv_ctx* ctx, dynakv_status* host_out);
  *   n_tokens    [U] int32,  n_ids [U] int32 (ids handed out),  tau [U] fp32 */
 int dynakv_export_state(dynakv_ctx* ctx, int32_t* tok_cluster, float* centroids, int32_t* counts,
                         float* M2, int32_t* n_tokens, int32_t* n_ids, float* tau);
+
+/* Checkpoint and resume (the paper keeps its KV store on flash but describes no resume; these two calls make the
+ * index restartable).  dynakv_export_kv synchronises and writes the first n tokens' K and V rows of every unit,
+ * in token-id order, to DEVICE arrays [U][n][d] of cfg.kv_dtype (n = the units' common token count).  Together
+ * with dynakv_export_state's tok_cluster, n_ids and tau that is a complete checkpoint.
+ * dynakv_import_state takes such a checkpoint into a freshly created context INSTEAD of dynakv_build_index:
+ * K, V and tok_cluster [U][n] are DEVICE arrays, n_ids [U] and tau [U] HOST arrays; n_build_clusters is the
+ * n_clusters of the original build (ids below it are the build's clusters, which matters in
+ * DYNAKV_MODE_LOCAL).  Members are laid out cluster by cluster in pages as after a build, and n_j, r_j
+ * (member means, Eq. 4) and M2_j are recomputed from the members, so they equal the exported ones up to
+ * fp32 rounding; ids without members stay unused; a split that had been abandoned may be tried again. */
+int dynakv_export_kv(dynakv_ctx* ctx, void* K_out, void* V_out, int64_t n);
+int dynakv_import_state(dynakv_ctx* ctx, const void* K, const void* V, int64_t n, const int32_t* tok_cluster,
+                        const int32_t* n_ids, const float* tau, int32_t n_build_clusters);
 
 /* Synchronises and copies the last decode step's selection sizes to HOST arrays:
  * n_selected [U], tokens_selected [U]; either may be NULL. */

@@ -20,7 +20,7 @@ EXPORTED_SYMBOLS = [
     "dynakv_create", "dynakv_build_index", "dynakv_append", "dynakv_decode_step", "dynakv_split_check",
     "dynakv_decode_loop", "dynakv_step_host", "dynakv_get_status", "dynakv_export_state", "dynakv_get_selection",
     "dynakv_get_build_trace", "dynakv_set_timing", "dynakv_get_kernel_times", "dynakv_launch_count", "dynakv_last_error", "dynakv_destroy",
-    "dynakv_attend_rows_noalloc",
+    "dynakv_attend_rows_noalloc", "dynakv_export_kv", "dynakv_import_state", "dynakv_decode_loop_host",
 ]
 ERR_TOO_LARGE = -5
 NOALLOC_SCRATCH_BYTES = 4 * 1024 * 1024
@@ -101,6 +101,12 @@ def load_library() -> C.CDLL:
     L.dynakv_export_state.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp]
     L.dynakv_get_selection.restype = C.c_int
     L.dynakv_get_selection.argtypes = [vp, vp, vp]
+    L.dynakv_decode_loop_host.restype = C.c_int
+    L.dynakv_decode_loop_host.argtypes = [vp, vp, vp, vp, i64, i32, vp]
+    L.dynakv_export_kv.restype = C.c_int
+    L.dynakv_export_kv.argtypes = [vp, vp, vp, i64]
+    L.dynakv_import_state.restype = C.c_int
+    L.dynakv_import_state.argtypes = [vp, vp, vp, i64, vp, vp, vp, i32]
     L.dynakv_get_build_trace.restype = C.c_int
     L.dynakv_get_build_trace.argtypes = [vp, vp, vp]
     L.dynakv_set_timing.restype = C.c_int
@@ -245,6 +251,15 @@ class DynaKV:
         self._keep = [q_steps, k_steps, v_steps, out_steps]
         return out_steps
 
+    def decode_loop_host(self, q_host, k_host, v_host, token_budget: int, out_host) -> None:
+        """The captured loop on HOST tensors [n, U, ...] (pinned for the copies to overlap the loop)."""
+        U, G, d = self.cfg.n_units, self.cfg.gqa_group, self.cfg.head_dim
+        n = q_host.shape[0]
+        assert not q_host.is_cuda and not out_host.is_cuda
+        self._check(self._L.dynakv_decode_loop_host(self._h, self._f32(q_host, (n, U, G, d)), self._kv(k_host, (n, U, d)),
+                                                    self._kv(v_host, (n, U, d)), n, token_budget, self._f32(out_host, (n, U, G, d))),
+                    "dynakv_decode_loop_host")
+
     def step_host(self, q_host, k_host, v_host, token_budget: int, out_host) -> None:
         U, G, d = self.cfg.n_units, self.cfg.gqa_group, self.cfg.head_dim
         assert not q_host.is_cuda and not out_host.is_cuda
@@ -267,6 +282,33 @@ class DynaKV:
         self._check(self._L.dynakv_export_state(self._h, *[_np_ptr(out[k]) for k in
                     ("tok_cluster", "centroids", "counts", "M2", "n_tokens", "n_ids", "tau")]), "dynakv_export_state")
         return out
+
+    def export_kv(self, n: int):
+        """K, V rows of the first n tokens of every unit in token-id order: two device tensors [U, n, d]."""
+        import torch
+        U, d = self.cfg.n_units, self.cfg.head_dim
+        dt = torch.float32 if self.cfg.kv_dtype == F32 else torch.bfloat16
+        with torch.cuda.stream(self._stream):
+            K = torch.empty((U, n, d), dtype=dt, device="cuda")
+            V = torch.empty_like(K)
+        self._check(self._L.dynakv_export_kv(self._h, C.c_void_p(K.data_ptr()), C.c_void_p(V.data_ptr()), n), "dynakv_export_kv")
+        return K, V
+
+    def import_state(self, K, V, tok_cluster, n_ids, tau, n_build_clusters: int) -> None:
+        """Resume from a checkpoint (export_state + export_kv) instead of building: K, V [U, n, d] device tensors,
+        tok_cluster [U, n] (device tensor or array), n_ids [U] and tau [U] arrays."""
+        import torch
+        U, d = self.cfg.n_units, self.cfg.head_dim
+        n = K.shape[1]
+        tc = torch.as_tensor(np.ascontiguousarray(tok_cluster), dtype=torch.int32) if not torch.is_tensor(tok_cluster) else tok_cluster
+        with torch.cuda.stream(self._stream):
+            tc = tc.to(device="cuda", dtype=torch.int32).contiguous()
+        self._stream.synchronize()
+        if tuple(tc.shape) != (U, n):
+            raise DynaKVError(f"expected tok_cluster of shape {(U, n)}, got {tuple(tc.shape)}")
+        ids = np.ascontiguousarray(n_ids, dtype=np.int32); ta = np.ascontiguousarray(tau, dtype=np.float32)
+        self._check(self._L.dynakv_import_state(self._h, self._kv(K, (U, n, d)), self._kv(V, (U, n, d)), n, C.c_void_p(tc.data_ptr()),
+                                                _np_ptr(ids), _np_ptr(ta), n_build_clusters), "dynakv_import_state")
 
     def get_selection(self):
         U = self.cfg.n_units

@@ -45,6 +45,21 @@ struct dynakv_ctx {
     float* st_q = nullptr; void* st_k = nullptr; void* st_v = nullptr; float* st_out = nullptr;
     cudaStream_t copy_stream = nullptr;      // carries the result copy of a host step past the step's append / split
     cudaEvent_t ev_attended = nullptr;
+    // the front half of a host step as one executable graph (per token budget): three copy-in nodes and the kernels up
+    // to the attention output
+    cudaGraphExec_t host_exec = nullptr;
+    cudaGraph_t host_graph = nullptr;            // kept: its node handles name the copy nodes in later updates
+    cudaGraphNode_t host_nodes[3] = {nullptr, nullptr, nullptr};    // copy nodes: q, k, v
+    const void* host_ptrs[3] = {nullptr, nullptr, nullptr};         // the host addresses the nodes hold now
+    int host_budget = -1;
+    long long host_launches = 0;
+    // dynakv_decode_loop_host: two sets of device staging arrays for chunks of steps, a stream for the copies in and
+    // one for the copies out, and the events that order them against the loop
+    static constexpr int HOST_CHUNK = 32;
+    char* hl_q[2] = {nullptr, nullptr}; char* hl_k[2] = {nullptr, nullptr}; char* hl_v[2] = {nullptr, nullptr};
+    char* hl_out[2] = {nullptr, nullptr};
+    cudaStream_t in_stream = nullptr, out_stream = nullptr;
+    cudaEvent_t ev_in[2] = {nullptr, nullptr}, ev_done[2] = {nullptr, nullptr}, ev_out[2] = {nullptr, nullptr};
     // optional per-kernel event timing (off inside graph capture)
     bool timing = false;
     struct Span { int kc; cudaEvent_t e0, e1; };
@@ -222,6 +237,10 @@ extern "C" void dynakv_destroy(dynakv_ctx* c) {
     cudaStreamSynchronize(c->stream);
     if (c->copy_stream) { cudaStreamSynchronize(c->copy_stream); cudaStreamDestroy(c->copy_stream); }
     if (c->ev_attended) cudaEventDestroy(c->ev_attended);
+    for (cudaStream_t s : {c->in_stream, c->out_stream}) if (s) { cudaStreamSynchronize(s); cudaStreamDestroy(s); }
+    for (int i = 0; i < 2; i++) for (cudaEvent_t e : {c->ev_in[i], c->ev_done[i], c->ev_out[i]}) if (e) cudaEventDestroy(e);
+    if (c->host_exec) cudaGraphExecDestroy(c->host_exec);
+    if (c->host_graph) cudaGraphDestroy(c->host_graph);
     for (cudaGraphExec_t g : c->graph_exec) if (g) cudaGraphExecDestroy(g);
     for (auto& sp : c->spans) { cudaEventDestroy(sp.e0); cudaEventDestroy(sp.e1); }
     for (cudaEvent_t e : c->event_pool) cudaEventDestroy(e);
@@ -423,9 +442,6 @@ extern "C" int dynakv_step_host(dynakv_ctx* c, const float* q_host, const void* 
     if (!c->built) return DYNAKV_ERR_STATE;
     const Tables& t = c->t;
     const size_t qb = (size_t)t.U * t.G * t.d * 4, kb = (size_t)t.U * t.d * kv_bytes(c->cfg);
-    CK(cudaMemcpyAsync(c->st_q, q_host, qb, cudaMemcpyHostToDevice, c->stream));
-    CK(cudaMemcpyAsync(c->st_k, k_host, kb, cudaMemcpyHostToDevice, c->stream));
-    CK(cudaMemcpyAsync(c->st_v, v_host, kb, cudaMemcpyHostToDevice, c->stream));
     // The result depends on the attention kernel only: its copy back runs on a second stream beside the step's
     // append and split check, and the call returns when the result is on the host.  Whatever is called next on
     // the context is ordered behind the append and split check by the context's stream.
@@ -434,8 +450,72 @@ extern "C" int dynakv_step_host(dynakv_ctx* c, const float* q_host, const void* 
         CK(cudaEventCreateWithFlags(&c->ev_attended, cudaEventDisableTiming));
     }
     const StepPtr q{c->st_q, 0, nullptr}, k{c->st_k, 0, nullptr}, v{c->st_v, 0, nullptr};
-    enqueue_front(c, q, k, 1, 1, true);
-    enqueue_retrieve(c, q, token_budget, StepPtrW{c->st_out, 0, nullptr}, nullptr, true);
+    const bool can_graph = !c->timing && c->stream != nullptr && c->stream != cudaStreamLegacy;
+    if (can_graph) {
+        // ---- the three copies in and the kernels up to the attention output as ONE graph launch.  Captured once per
+        // budget; a later call with other host arrays only rewrites the copy nodes' addresses.
+        const void* now[3] = {q_host, k_host, v_host};
+        if (!c->host_exec || c->host_budget != token_budget) {
+            if (c->host_exec) { cudaGraphExecDestroy(c->host_exec); c->host_exec = nullptr; }
+            if (c->host_graph) { cudaGraphDestroy(c->host_graph); c->host_graph = nullptr; }
+            cudaGraph_t graph = nullptr;
+            const long long before = c->launches;
+            CK(cudaStreamBeginCapture(c->stream, cudaStreamCaptureModeThreadLocal));
+            cudaMemcpyAsync(c->st_q, q_host, qb, cudaMemcpyHostToDevice, c->stream);
+            cudaMemcpyAsync(c->st_k, k_host, kb, cudaMemcpyHostToDevice, c->stream);
+            cudaMemcpyAsync(c->st_v, v_host, kb, cudaMemcpyHostToDevice, c->stream);
+            enqueue_front(c, q, k, 1, 1, false);
+            enqueue_retrieve(c, q, token_budget, StepPtrW{c->st_out, 0, nullptr}, nullptr, false);
+            cudaError_t e = cudaStreamEndCapture(c->stream, &graph);
+            c->host_launches = c->launches - before;
+            c->launches = before;
+            if (e == cudaSuccess && graph) e = cudaGraphInstantiate(&c->host_exec, graph, 0);
+            if (e == cudaSuccess) {
+                // find the three copy nodes by the device staging buffer they write
+                size_t nn = 0;
+                cudaGraphGetNodes(graph, nullptr, &nn);
+                std::vector<cudaGraphNode_t> nodes(nn);
+                cudaGraphGetNodes(graph, nodes.data(), &nn);
+                for (int i = 0; i < 3; i++) c->host_nodes[i] = nullptr;
+                for (cudaGraphNode_t nd : nodes) {
+                    cudaGraphNodeType ty;
+                    if (cudaGraphNodeGetType(nd, &ty) != cudaSuccess || ty != cudaGraphNodeTypeMemcpy) continue;
+                    cudaMemcpy3DParms mp;
+                    if (cudaGraphMemcpyNodeGetParams(nd, &mp) != cudaSuccess) continue;
+                    if (mp.dstPtr.ptr == (void*)c->st_q) c->host_nodes[0] = nd;
+                    else if (mp.dstPtr.ptr == c->st_k) c->host_nodes[1] = nd;
+                    else if (mp.dstPtr.ptr == c->st_v) c->host_nodes[2] = nd;
+                }
+                if (!c->host_nodes[0] || !c->host_nodes[1] || !c->host_nodes[2]) e = cudaErrorUnknown;
+            }
+            if (e != cudaSuccess) {
+                if (graph) cudaGraphDestroy(graph);
+                if (c->host_exec) { cudaGraphExecDestroy(c->host_exec); c->host_exec = nullptr; }
+                snprintf(g_err, sizeof(g_err), "host-step graph capture / instantiate failed: %s", cudaGetErrorString(e));
+                cudaGetLastError();
+                return DYNAKV_ERR_CUDA;
+            }
+            c->host_graph = graph;
+            cudaGraphUpload(c->host_exec, c->stream);
+            c->host_budget = token_budget;
+            for (int i = 0; i < 3; i++) c->host_ptrs[i] = now[i];
+        }
+        const size_t bytes[3] = {qb, kb, kb};
+        void* const dev[3] = {c->st_q, c->st_k, c->st_v};
+        for (int i = 0; i < 3; i++) {
+            if (c->host_ptrs[i] == now[i]) continue;
+            CK(cudaGraphExecMemcpyNodeSetParams1D(c->host_exec, c->host_nodes[i], dev[i], now[i], bytes[i], cudaMemcpyHostToDevice));
+            c->host_ptrs[i] = now[i];
+        }
+        CK(cudaGraphLaunch(c->host_exec, c->stream));
+        c->launches += c->host_launches;
+    } else {
+        CK(cudaMemcpyAsync(c->st_q, q_host, qb, cudaMemcpyHostToDevice, c->stream));
+        CK(cudaMemcpyAsync(c->st_k, k_host, kb, cudaMemcpyHostToDevice, c->stream));
+        CK(cudaMemcpyAsync(c->st_v, v_host, kb, cudaMemcpyHostToDevice, c->stream));
+        enqueue_front(c, q, k, 1, 1, true);
+        enqueue_retrieve(c, q, token_budget, StepPtrW{c->st_out, 0, nullptr}, nullptr, true);
+    }
     CK(cudaEventRecord(c->ev_attended, c->stream));
     CK(cudaStreamWaitEvent(c->copy_stream, c->ev_attended, 0));
     CK(cudaMemcpyAsync(out_host, c->st_out, qb, cudaMemcpyDeviceToHost, c->copy_stream));
@@ -445,6 +525,54 @@ extern "C" int dynakv_step_host(dynakv_ctx* c, const float* q_host, const void* 
                             c->cfg.split_iters, 1, k, v, nullptr, kNoNextFront, c->stream, &c->launches);
     }
     CK(cudaStreamSynchronize(c->copy_stream));
+    return DYNAKV_OK;
+}
+
+extern "C" int dynakv_decode_loop_host(dynakv_ctx* c, const float* q_host, const void* k_host, const void* v_host,
+                                       int64_t n_steps, int32_t token_budget, float* out_host) {
+    if (!c || !q_host || !k_host || !v_host || !out_host || n_steps < 0 || token_budget < 0) return DYNAKV_ERR_ARG;
+    if (!c->built) return DYNAKV_ERR_STATE;
+    const Tables& t = c->t;
+    const size_t qs = (size_t)t.U * t.G * t.d * 4, ks = (size_t)t.U * t.d * kv_bytes(c->cfg);
+    constexpr int CH = dynakv_ctx::HOST_CHUNK;
+    if (!c->in_stream) {
+        // first call: staging arrays (kept until destroy), streams, events
+        for (int b = 0; b < 2; b++) {
+            ALLOC_B(c->hl_q[b], CH * qs, false); ALLOC_B(c->hl_k[b], CH * ks, false); ALLOC_B(c->hl_v[b], CH * ks, false);
+            ALLOC_B(c->hl_out[b], CH * qs, false);
+        }
+        CK(cudaStreamCreateWithFlags(&c->in_stream, cudaStreamNonBlocking));
+        CK(cudaStreamCreateWithFlags(&c->out_stream, cudaStreamNonBlocking));
+        for (int b = 0; b < 2; b++)
+            for (cudaEvent_t* e : {&c->ev_in[b], &c->ev_done[b], &c->ev_out[b]}) CK(cudaEventCreateWithFlags(e, cudaEventDisableTiming));
+    }
+    // Chunks of CH steps: chunk i + 1 is copied in and chunk i - 1 copied out while the loop runs chunk i.
+    const int64_t n_chunks = (n_steps + CH - 1) / CH;
+    // whatever ran on the context's stream before must be complete before its inputs are overwritten
+    CK(cudaEventRecord(c->ev_done[0], c->stream)); CK(cudaEventRecord(c->ev_done[1], c->stream));
+    CK(cudaEventRecord(c->ev_out[0], c->out_stream)); CK(cudaEventRecord(c->ev_out[1], c->out_stream));
+    for (int64_t i = 0; i < n_chunks; i++) {
+        const int b = (int)(i & 1);
+        const int64_t s0 = i * CH, nb = (n_steps - s0 < CH) ? n_steps - s0 : CH;
+        // copy in: the staging set is free once the loop over the chunk that used it before has finished
+        CK(cudaStreamWaitEvent(c->in_stream, c->ev_done[b], 0));
+        CK(cudaMemcpyAsync(c->hl_q[b], (const char*)q_host + s0 * qs, nb * qs, cudaMemcpyHostToDevice, c->in_stream));
+        CK(cudaMemcpyAsync(c->hl_k[b], (const char*)k_host + s0 * ks, nb * ks, cudaMemcpyHostToDevice, c->in_stream));
+        CK(cudaMemcpyAsync(c->hl_v[b], (const char*)v_host + s0 * ks, nb * ks, cudaMemcpyHostToDevice, c->in_stream));
+        CK(cudaEventRecord(c->ev_in[b], c->in_stream));
+        // the loop: needs the chunk's inputs, and its output set copied out (two chunks ago)
+        CK(cudaStreamWaitEvent(c->stream, c->ev_in[b], 0));
+        CK(cudaStreamWaitEvent(c->stream, c->ev_out[b], 0));
+        int rc = dynakv_decode_loop(c, (const float*)c->hl_q[b], c->hl_k[b], c->hl_v[b], nb, token_budget, (float*)c->hl_out[b]);
+        if (rc != DYNAKV_OK) return rc;
+        CK(cudaEventRecord(c->ev_done[b], c->stream));
+        // copy out
+        CK(cudaStreamWaitEvent(c->out_stream, c->ev_done[b], 0));
+        CK(cudaMemcpyAsync((char*)out_host + s0 * qs, c->hl_out[b], nb * qs, cudaMemcpyDeviceToHost, c->out_stream));
+        CK(cudaEventRecord(c->ev_out[b], c->out_stream));
+    }
+    CK(cudaStreamSynchronize(c->out_stream));
+    CK(cudaStreamSynchronize(c->stream));
     return DYNAKV_OK;
 }
 
@@ -494,6 +622,56 @@ extern "C" int dynakv_export_state(dynakv_ctx* c, int32_t* tok_cluster, float* c
     if (n_ids) CK(cudaMemcpyAsync(n_ids, t.u_M, sizeof(int) * U, cudaMemcpyDeviceToHost, s));
     if (tau) CK(cudaMemcpyAsync(tau, t.u_tau, sizeof(float) * U, cudaMemcpyDeviceToHost, s));
     CK(cudaStreamSynchronize(s));
+    return DYNAKV_OK;
+}
+
+extern "C" int dynakv_export_kv(dynakv_ctx* c, void* K_out, void* V_out, int64_t n) {
+    if (!c || !K_out || !V_out || n < 1 || n > c->t.max_tokens) return DYNAKV_ERR_ARG;
+    if (!c->built) return DYNAKV_ERR_STATE;
+    launch_export_rows(c->t, K_out, V_out, n, c->stream, &c->launches);
+    CK(cudaGetLastError());
+    CK(cudaStreamSynchronize(c->stream));
+    return DYNAKV_OK;
+}
+
+extern "C" int dynakv_import_state(dynakv_ctx* c, const void* K, const void* V, int64_t n, const int32_t* tok_cluster,
+                                   const int32_t* n_ids, const float* tau, int32_t n_build_clusters) {
+    if (!c || !K || !V || !tok_cluster || !n_ids || !tau) return DYNAKV_ERR_ARG;
+    if (c->built) return DYNAKV_ERR_STATE;
+    Tables& t = c->t;
+    if (n < 1 || n > t.max_tokens || n_build_clusters < 1 || n_build_clusters > t.max_clusters) return DYNAKV_ERR_ARG;
+    const size_t U = t.U;
+    int M = 0, Mmin = t.max_clusters;
+    for (size_t u = 0; u < U; u++) {
+        if (n_ids[u] < 1 || n_ids[u] > t.max_clusters) return DYNAKV_ERR_ARG;
+        M = n_ids[u] > M ? n_ids[u] : M;
+        Mmin = n_ids[u] < Mmin ? n_ids[u] : Mmin;
+    }
+    if (n_build_clusters > Mmin) return DYNAKV_ERR_ARG;
+    const int d = t.d;
+    BuildScratch b;
+    memset(&b, 0, sizeof(b));
+    const size_t mark = c->allocs.size();
+    int* ids_dev = nullptr; float* tau_dev = nullptr;
+    ALLOC_B(b.C, U * M * d, true);
+    ALLOC_B(b.sums, U * M * d, false);
+    ALLOC_B(b.counts, U * M, false);
+    ALLOC_B(b.cursor, U * M, false);
+    ALLOC_B(ids_dev, U, false);
+    ALLOC_B(tau_dev, U, false);
+    b.assign = const_cast<int*>(tok_cluster);
+    CK(cudaMemcpyAsync(ids_dev, n_ids, sizeof(int) * U, cudaMemcpyHostToDevice, c->stream));
+    CK(cudaMemcpyAsync(tau_dev, tau, sizeof(float) * U, cudaMemcpyHostToDevice, c->stream));
+    // representatives = member means (Eq. 4), then the layout and the exact statistics, as at the end of a build
+    launch_update(t, K, n, M, b.assign, b, c->stream, &c->launches);
+    launch_finalize(t, K, V, n, M, b, c->cfg.split_var_factor, c->stream, &c->launches);
+    launch_import_units(t, ids_dev, tau_dev, c->stream, &c->launches);
+    CK(cudaGetLastError());
+    CK(cudaStreamSynchronize(c->stream));
+    for (size_t i = mark; i < c->allocs.size(); i++) cudaFree(c->allocs[i]);
+    c->allocs.resize(mark);
+    c->built = true; c->n_prefill = n; c->M0 = n_build_clusters;
+    t.M_floor = n_build_clusters;
     return DYNAKV_OK;
 }
 

@@ -372,6 +372,47 @@ __global__ void __launch_bounds__(256) k_fin_tau(Tables t, int M, float alpha) {
     if (threadIdx.x == 0) t.u_tau[u] = alpha * red[0] / (float)max(t.u_Mlive[u], 1);
 }
 
+// ------------------------------------------------------------------ checkpoint: rows out in token order, partition in
+
+// One block per (cluster, unit): the members' K and V rows go to [U][n][d] arrays at their token ids.
+template <typename KV, int HD>
+__global__ void __launch_bounds__(128) k_export_rows(Tables t, KV* __restrict__ Kout, KV* __restrict__ Vout, long long n) {
+    const int j = blockIdx.x, u = blockIdx.y;
+    if (j >= t.u_M[u]) return;
+    const size_t cj = (size_t)u * t.max_clusters + j;
+    const int c = t.cl_n[cj];
+    const KV* kp = reinterpret_cast<const KV*>(t.kpages);
+    const KV* vp = reinterpret_cast<const KV*>(t.vpages);
+    int page = t.cl_head[cj];
+    constexpr int V16 = HD * (int)sizeof(KV) / 16;        // 16-byte pieces per row
+    for (int s0 = 0; s0 < c; s0 += PAGE) {
+        const int rows = min(PAGE, c - s0);
+        for (int idx = threadIdx.x; idx < rows * V16; idx += blockDim.x) {
+            const int r = idx / V16, v = idx % V16;
+            const size_t slot = ((size_t)u * t.P + page) * PAGE + r;
+            const int tok = t.page_tok[slot];
+            if (tok < 0 || tok >= n) continue;
+            reinterpret_cast<uint4*>(Kout + ((size_t)u * n + tok) * HD)[v] = reinterpret_cast<const uint4*>(kp + slot * HD)[v];
+            reinterpret_cast<uint4*>(Vout + ((size_t)u * n + tok) * HD)[v] = reinterpret_cast<const uint4*>(vp + slot * HD)[v];
+        }
+        page = t.page_next[(size_t)u * t.P + page];
+    }
+}
+
+// A given partition's per-unit bookkeeping after the layout kernels have run with a common id count M: every unit
+// gets its own number of ids in use and its threshold back.
+__global__ void k_import_units(Tables t, const int* __restrict__ n_ids, const float* __restrict__ tau) {
+    const int u = blockIdx.x * blockDim.x + threadIdx.x;
+    if (u >= t.U) return;
+    t.u_M[u] = n_ids[u];
+    t.u_tau[u] = tau[u];
+}
+
+template <typename KV, int HD>
+static void export_rows_t(const Tables& t, void* K, void* V, long long n, cudaStream_t s) {
+    k_export_rows<KV, HD><<<dim3(t.max_clusters, t.U), 128, 0, s>>>(t, (KV*)K, (KV*)V, n);
+}
+
 // ------------------------------------------------------------------ launchers
 
 template <typename KV, int HD>
@@ -464,6 +505,16 @@ static void finalize_t(const Tables& t, const void* K, const void* V, long long 
 void launch_finalize(const Tables& t, const void* K, const void* V, long long n, int M, const BuildScratch& b,
                      float alpha, cudaStream_t s, long long* launches) {
     DKV_DISPATCH(finalize_t, t, K, V, n, M, b, alpha, s, launches);
+}
+
+void launch_export_rows(const Tables& t, void* K, void* V, long long n, cudaStream_t s, long long* launches) {
+    DKV_DISPATCH(export_rows_t, t, K, V, n, s);
+    (*launches)++;
+}
+
+void launch_import_units(const Tables& t, const int* n_ids, const float* tau, cudaStream_t s, long long* launches) {
+    k_import_units<<<(t.U + 255) / 256, 256, 0, s>>>(t, n_ids, tau);
+    (*launches)++;
 }
 
 }  // namespace dkv

@@ -206,6 +206,8 @@ struct LoopBegin {
     const void** args;        // device: [4] q, k, v, out of the loop in flight
     const void* q; const void* k; const void* v; void* out;
 };
+void launch_export_rows(const Tables& t, void* K, void* V, long long n, cudaStream_t s, long long* launches);
+void launch_import_units(const Tables& t, const int* n_ids, const float* tau, cudaStream_t s, long long* launches);
 void launch_front(const Tables& t, StepPtr q, StepPtr k, int has_q, int has_k, cudaStream_t s, long long* launches,
                   const LoopBegin* lb = nullptr);
 void launch_select(const Tables& t, int budget, int* user_sel_ids, cudaStream_t s, long long* launches);

@@ -216,6 +216,54 @@ def test_duplicate_keys_leave_dead_clusters():
     ctx.destroy()
 
 
+@pytest.mark.parametrize("mode", ["adaptive", "local"])
+def test_checkpoint_and_resume(mode):
+    """export_state + export_kv after some decode steps, import into a fresh context, and both contexts must go on
+    identically: same membership and ids after more steps (splits included), outputs equal up to the rounding of
+    the recomputed statistics."""
+    from parity_harness import make_ctx
+    cfg = CONFIGS[2].scaled(B=1, L=1, Hkv=1, Hq=4, n_prefill=700, steps=120, M0=20, max_clusters=128, budget=300, T=3,
+                            update_mode=mode, local_max=20)
+    units = [0, 1, 2]
+    s = [UnitStream(cfg, u) for u in units]
+    K, V = make_prefill(s)
+    q, k, v = make_decode_chunk(s, 120)
+    qd, kd, vd = q.cuda(), k.cuda(), v.cuda()
+    a = make_ctx(cfg, 3, trace=0, assign_mode=1)
+    a.build_index(K.cuda(), V.cuda(), cfg.M0, 5)
+    for t in range(60):
+        a.decode_step(qd[t], cfg.budget); a.append(kd[t], vd[t]); a.split_check()
+    st = a.export_state()
+    n = int(st["n_tokens"][0])
+    assert n == 760 and np.all(st["n_tokens"] == n)
+    Kx, Vx = a.export_kv(n)
+    Kref = torch.cat([K, k[:60].transpose(0, 1)], dim=1)
+    assert torch.equal(Kx.cpu(), Kref)                                      # rows come back in token order
+    b = make_ctx(cfg, 3, trace=0, assign_mode=1)
+    b.import_state(Kx, Vx, st["tok_cluster"][:, :n], st["n_ids"], st["tau"], cfg.M0)
+    sb = b.export_state()
+    assert np.array_equal(sb["tok_cluster"], st["tok_cluster"]) and np.array_equal(sb["counts"], st["counts"])
+    assert np.array_equal(sb["n_ids"], st["n_ids"]) and np.array_equal(sb["tau"], st["tau"])
+    live = st["counts"] > 0
+    assert np.abs(sb["centroids"][live] - st["centroids"][live]).max() <= 1e-4 * np.abs(st["centroids"][live]).max()
+    worst = 0.0
+    for t in range(60, 120):
+        oa = a.decode_step(qd[t], cfg.budget); ob = b.decode_step(qd[t], cfg.budget)
+        worst = max(worst, float((oa - ob).abs().max()))
+        a.append(kd[t], vd[t]); b.append(kd[t], vd[t])
+        a.split_check(); b.split_check()
+    sa, sb = a.export_state(), b.export_state()
+    assert np.array_equal(sa["tok_cluster"], sb["tok_cluster"]) and np.array_equal(sa["counts"], sb["counts"])
+    assert a.get_status()["n_splits"] > 0 and worst < 1e-4
+    a.destroy(); b.destroy()
+
+
+def test_host_array_loop_matches_direct_calls():
+    cfg = CONFIGS[2].scaled(B=1, L=1, Hkv=1, Hq=4, n_prefill=500, steps=70, M0=12, max_clusters=64, budget=200, T=3,
+                            split_size_factor=1.3)
+    assert _loop_vs_direct(cfg, [0, 1, 2, 3], 70, modes=("direct", "hostloop")) > 0
+
+
 def test_graph_loop_in_local_update_mode():
     # the captured loop founds a cluster for the first new entry inside the tail kernel (an id beyond the ones the
     # unit's centroid pass covered) and splits decode-born clusters above 20 entries
@@ -250,6 +298,11 @@ def _loop_vs_direct(cfg, units, steps, modes=("direct", "graph", "host"), cut=No
                 out = ctx.decode_loop(qd[:cut], kd[:cut], vd[:cut], cfg.budget)
                 out2 = ctx.decode_loop(qd[cut:], kd[cut:], vd[cut:], cfg.budget)
                 out = torch.cat([out, out2])
+            elif mode == "hostloop":
+                # host arrays through the chunked, double-buffered loop (70 steps = two full chunks of 32 and a rest)
+                qh, kh, vh = q.pin_memory(), k.pin_memory(), v.pin_memory()
+                out = torch.empty((steps, len(units), cfg.G, cfg.d)).pin_memory()
+                ctx.decode_loop_host(qh, kh, vh, cfg.budget, out)
             else:
                 out = torch.empty((steps, len(units), cfg.G, cfg.d))
                 qh, kh, vh = q.pin_memory(), k.pin_memory(), v.pin_memory()
