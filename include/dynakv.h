@@ -208,6 +208,19 @@ int dynakv_get_selection(dynakv_ctx* ctx, int32_t* n_selected, int32_t* tokens_s
  * either may be NULL.  Returns DYNAKV_ERR_STATE if tracing was off. */
 int dynakv_get_build_trace(dynakv_ctx* ctx, int32_t* picks, int32_t* assign);
 
+/* Self-test of the device-side bounded waits (no counterpart in the paper).  Every wait on a shared-memory barrier in
+ * this library gives up after a bounded number of polls, sets DYNAKV_ST_INTERNAL and lets the kernel return.  This
+ * call runs a one-thread kernel that waits, with a limit of 4096 polls, on a barrier nobody arrives at: *gave_up
+ * (HOST) becomes 1, DYNAKV_ST_INTERNAL is set in the status word, and the context stays usable.  Synchronises. */
+int dynakv_selftest_wait_expiry(dynakv_ctx* ctx, int32_t* gave_up);
+
+/* Measurement aid (no counterpart in the paper).  Runs the gather-attention kernel `reps` times back to back on the
+ * selection of the LAST dynakv_decode_step (same work lists, q as given, results to out), as ordinary launches
+ * bracketed by two CUDA events on the context's stream, after one untimed launch.  *ms_per_launch (HOST) = elapsed
+ * time / reps: the kernel's duration without the cost of an event pair around every launch.  bf16 K/V only.
+ * Synchronises. */
+int dynakv_time_gather_attention(dynakv_ctx* ctx, const float* q, float* out, int32_t reps, float* ms_per_launch);
+
 /* Measurement aid (no counterpart in the paper).  With timing on, every kernel launched
  * by a direct call (not by dynakv_decode_loop's graph replay) is bracketed by CUDA events on
  * the context's stream.  dynakv_get_kernel_times synchronises and returns, per kernel class,

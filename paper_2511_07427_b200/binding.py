@@ -20,7 +20,7 @@ EXPORTED_SYMBOLS = [
     "dynakv_create", "dynakv_build_index", "dynakv_append", "dynakv_decode_step", "dynakv_split_check",
     "dynakv_decode_loop", "dynakv_step_host", "dynakv_get_status", "dynakv_export_state", "dynakv_get_selection",
     "dynakv_get_build_trace", "dynakv_set_timing", "dynakv_get_kernel_times", "dynakv_launch_count", "dynakv_last_error", "dynakv_destroy",
-    "dynakv_attend_rows_noalloc", "dynakv_export_kv", "dynakv_import_state", "dynakv_decode_loop_host",
+    "dynakv_attend_rows_noalloc", "dynakv_export_kv", "dynakv_import_state", "dynakv_decode_loop_host", "dynakv_selftest_wait_expiry", "dynakv_time_gather_attention",
 ]
 ERR_TOO_LARGE = -5
 NOALLOC_SCRATCH_BYTES = 4 * 1024 * 1024
@@ -103,6 +103,10 @@ def load_library() -> C.CDLL:
     L.dynakv_get_selection.argtypes = [vp, vp, vp]
     L.dynakv_decode_loop_host.restype = C.c_int
     L.dynakv_decode_loop_host.argtypes = [vp, vp, vp, vp, i64, i32, vp]
+    L.dynakv_time_gather_attention.restype = C.c_int
+    L.dynakv_time_gather_attention.argtypes = [vp, vp, vp, i32, vp]
+    L.dynakv_selftest_wait_expiry.restype = C.c_int
+    L.dynakv_selftest_wait_expiry.argtypes = [vp, vp]
     L.dynakv_export_kv.restype = C.c_int
     L.dynakv_export_kv.argtypes = [vp, vp, vp, i64]
     L.dynakv_import_state.restype = C.c_int
@@ -309,6 +313,20 @@ class DynaKV:
         ids = np.ascontiguousarray(n_ids, dtype=np.int32); ta = np.ascontiguousarray(tau, dtype=np.float32)
         self._check(self._L.dynakv_import_state(self._h, self._kv(K, (U, n, d)), self._kv(V, (U, n, d)), n, C.c_void_p(tc.data_ptr()),
                                                 _np_ptr(ids), _np_ptr(ta), n_build_clusters), "dynakv_import_state")
+
+    def time_gather_attention(self, q, out, reps: int) -> float:
+        """Milliseconds per launch of the gather-attention kernel over `reps` back-to-back launches on the last selection."""
+        U, G, d = self.cfg.n_units, self.cfg.gqa_group, self.cfg.head_dim
+        ms = np.zeros(1, np.float32)
+        self._check(self._L.dynakv_time_gather_attention(self._h, self._f32(q, (U, G, d)), self._f32(out, (U, G, d)), reps,
+                                                         _np_ptr(ms)), "dynakv_time_gather_attention")
+        return float(ms[0])
+
+    def selftest_wait_expiry(self) -> int:
+        """Runs the bounded-wait self-test; returns 1 when the wait gave up as it must."""
+        flag = np.zeros(1, np.int32)
+        self._check(self._L.dynakv_selftest_wait_expiry(self._h, _np_ptr(flag)), "dynakv_selftest_wait_expiry")
+        return int(flag[0])
 
     def get_selection(self):
         U = self.cfg.n_units

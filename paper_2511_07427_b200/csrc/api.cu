@@ -695,6 +695,38 @@ extern "C" int dynakv_get_build_trace(dynakv_ctx* c, int32_t* picks, int32_t* as
     return DYNAKV_OK;
 }
 
+extern "C" int dynakv_selftest_wait_expiry(dynakv_ctx* c, int32_t* gave_up) {
+    if (!c || !gave_up) return DYNAKV_ERR_ARG;
+    int* flag = reinterpret_cast<int*>(c->t.plan_counter);      // a scratch word that is zero between calls
+    launch_selftest_wait_expiry(c->t, flag, c->stream, &c->launches);
+    CK(cudaGetLastError());
+    CK(cudaMemcpyAsync(gave_up, flag, sizeof(int), cudaMemcpyDeviceToHost, c->stream));
+    CK(cudaMemsetAsync(flag, 0, sizeof(int), c->stream));
+    CK(cudaStreamSynchronize(c->stream));
+    return DYNAKV_OK;
+}
+
+extern "C" int dynakv_time_gather_attention(dynakv_ctx* c, const float* q, float* out, int32_t reps, float* ms_per_launch) {
+    if (!c || !q || !out || !ms_per_launch || reps < 1) return DYNAKV_ERR_ARG;
+    if (!c->built) return DYNAKV_ERR_STATE;
+    if (c->t.kv_dtype != DYNAKV_BF16 || c->cfg.attn_mode != 0) return DYNAKV_ERR_ARG;
+    cudaEvent_t e0, e1;
+    CK(cudaEventCreate(&e0)); CK(cudaEventCreate(&e1));
+    const StepPtr qp{q, 0, nullptr};
+    const StepPtrW op{out, 0, nullptr};
+    launch_gather_attn_plain(c->t, qp, op, c->stream, &c->launches);       // one untimed launch first
+    CK(cudaEventRecord(e0, c->stream));
+    for (int i = 0; i < reps; i++) launch_gather_attn_plain(c->t, qp, op, c->stream, &c->launches);
+    CK(cudaEventRecord(e1, c->stream));
+    CK(cudaGetLastError());
+    CK(cudaEventSynchronize(e1));
+    float ms = 0.f;
+    CK(cudaEventElapsedTime(&ms, e0, e1));
+    *ms_per_launch = ms / (float)reps;
+    cudaEventDestroy(e0); cudaEventDestroy(e1);
+    return DYNAKV_OK;
+}
+
 extern "C" int dynakv_set_timing(dynakv_ctx* c, int32_t on) {
     if (!c) return DYNAKV_ERR_ARG;
     c->timing = on != 0;

@@ -412,6 +412,24 @@ __global__ void __launch_bounds__(AT_THREADS, 2) k_gather_attn_tma(Tables t, Ste
     }
 }
 
+// Self-test of the bounded waits: one thread waits on an mbarrier that nobody ever arrives at, with a limit of a few
+// thousand polls.  The wait must give up, the kernel raises the same status bit the production kernels raise on an
+// expired wait, and returns normally; nothing faults, traps or spins on.
+__global__ void k_selftest_wait_expiry(unsigned int* status, int* gave_up) {
+    __shared__ unsigned long long bar;
+    if (threadIdx.x == 0) {
+        mbar_init(smem_u32(&bar), 1);
+        asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
+        const bool ok = mbar_wait(smem_u32(&bar), 0u, 4096);
+        if (!ok) { atomicOr(status, DYNAKV_ST_INTERNAL); *gave_up = 1; }
+    }
+}
+
+void launch_selftest_wait_expiry(const Tables& t, int* gave_up, cudaStream_t s, long long* launches) {
+    k_selftest_wait_expiry<<<1, 32, 0, s>>>(t.status, gave_up);
+    (*launches)++;
+}
+
 size_t attn_tma_smem_bytes(const Tables& t) {
     const size_t fixed = t.d == 64 ? AttnSmem<64>::fixed_bytes : AttnSmem<128>::fixed_bytes;
     return fixed + (t.attn_pf_in_smem ? (size_t)(t.U + 1) * 4 : 0) + 64;
@@ -423,6 +441,14 @@ int attn_tma_prepare(const Tables& t) {
         ? cudaFuncSetAttribute(k_gather_attn_tma<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes)
         : cudaFuncSetAttribute(k_gather_attn_tma<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
     return e == cudaSuccess ? 0 : -1;
+}
+
+// The same kernel as an ordinary launch (no programmatic dependence on its neighbours): for timing it alone.
+void launch_gather_attn_plain(const Tables& t, StepPtr q, StepPtrW out, cudaStream_t s, long long* launches) {
+    const size_t bytes = attn_tma_smem_bytes(t);
+    if (t.d == 64) k_gather_attn_tma<64><<<t.n_attn_ctas, AT_THREADS, bytes, s>>>(t, q, out);
+    else k_gather_attn_tma<128><<<t.n_attn_ctas, AT_THREADS, bytes, s>>>(t, q, out);
+    (*launches)++;
 }
 
 void launch_gather_attn_tma(const Tables& t, StepPtr q, StepPtrW out, cudaStream_t s, long long* launches) {

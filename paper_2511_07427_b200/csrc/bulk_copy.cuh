@@ -28,10 +28,11 @@ __device__ __forceinline__ unsigned long long global_ns() {
     asm volatile("mov.u64 %0, %%globaltimer;\n" : "=l"(v));
     return v;
 }
-// Bounded wait: gives up after 2^22 polls or about 0.2 s, whichever comes first.
-__device__ __forceinline__ bool mbar_wait(unsigned bar, unsigned parity) {
+// Bounded wait: gives up after max_polls polls (2^22 unless the caller says otherwise) or about 0.2 s, whichever
+// comes first.
+__device__ __forceinline__ bool mbar_wait(unsigned bar, unsigned parity, int max_polls = 1 << 22) {
     unsigned long long t0 = 0;
-    for (int i = 0; i < (1 << 22); i++) {
+    for (int i = 0; i < max_polls; i++) {
         if (mbar_try_wait(bar, parity)) return true;
         if ((i & 63) == 63) {
             const unsigned long long now = global_ns();

@@ -213,7 +213,9 @@ void launch_front(const Tables& t, StepPtr q, StepPtr k, int has_q, int has_k, c
 void launch_select(const Tables& t, int budget, int* user_sel_ids, cudaStream_t s, long long* launches);
 void launch_append_apply(const Tables& t, StepPtr k, StepPtr v, cudaStream_t s, long long* launches);
 void launch_gather_attn_tma(const Tables& t, StepPtr q, StepPtrW out, cudaStream_t s, long long* launches);
+void launch_gather_attn_plain(const Tables& t, StepPtr q, StepPtrW out, cudaStream_t s, long long* launches);
 int attn_tma_prepare(const Tables& t);
+void launch_selftest_wait_expiry(const Tables& t, int* gave_up, cudaStream_t s, long long* launches);
 void launch_gather_attn_v1(const Tables& t, StepPtr q, cudaStream_t s, long long* launches);
 void launch_attn_combine(const Tables& t, StepPtrW out, cudaStream_t s, long long* launches);
 void launch_split_check(const Tables& t, float gamma, int var_enabled, int min_size, int iters, cudaStream_t s,

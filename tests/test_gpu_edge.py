@@ -264,6 +264,25 @@ def test_host_array_loop_matches_direct_calls():
     assert _loop_vs_direct(cfg, [0, 1, 2, 3], 70, modes=("direct", "hostloop")) > 0
 
 
+def test_a_bounded_wait_that_runs_out_raises_the_status_bit_and_returns():
+    """A wait on a barrier nobody arrives at gives up after its poll limit: the status word gets INTERNAL, the kernel
+    returns, and the context goes on working (no fault, no hang)."""
+    cfg = CONFIGS[2].scaled(B=1, L=1, Hkv=1, Hq=4, n_prefill=300, steps=4, M0=8, max_clusters=32, budget=100, T=2)
+    s_ = [UnitStream(cfg, 0)]
+    K, V = make_prefill(s_)
+    q, k, v = make_decode_chunk(s_, 2)
+    ctx = _single_ctx(cfg, K, V, assign_mode=1)
+    out0 = ctx.decode_step(q[0].cuda(), cfg.budget).cpu()
+    assert ctx.get_status()["error_bits"] & P.ST_INTERNAL == 0
+    assert ctx.selftest_wait_expiry() == 1
+    assert ctx.get_status()["error_bits"] & P.ST_INTERNAL
+    out1 = ctx.decode_step(q[0].cuda(), cfg.budget).cpu()       # the context is still usable and gives the same answer
+    assert torch.equal(out0, out1)
+    ctx.append(k[0].cuda(), v[0].cuda()); ctx.split_check()
+    assert ctx.export_state()["n_tokens"][0] == cfg.n_prefill + 1
+    ctx.destroy()
+
+
 def test_graph_loop_in_local_update_mode():
     # the captured loop founds a cluster for the first new entry inside the tail kernel (an id beyond the ones the
     # unit's centroid pass covered) and splits decode-born clusters above 20 entries
