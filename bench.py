@@ -31,7 +31,7 @@ METRIC = "decode steps/s at 32-layer 32K ctx; retrieval-attention HBM GB/s vs pe
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch, and the tokens that launch attended.  Traffic
 # is proportional to the rows attended, so a launch's traffic is scaled by its own token count.  Set
 # NCU_ATTN_CAPTURE to None whenever the kernel changes after the capture.
-NCU_ATTN_CAPTURE = {"dram_bytes": 100.3156e6 + 3.0356e6, "tokens": 195006.5}
+NCU_ATTN_CAPTURE = {"dram_bytes": 100.3295e6 + 3.1793e6, "tokens": 195006.5}
 
 
 def _peaks():

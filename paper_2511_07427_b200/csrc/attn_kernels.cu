@@ -370,9 +370,49 @@ __global__ void __launch_bounds__(AT_THREADS, 2) k_gather_attn_tma(Tables t, Ste
             consumer_sync();
             if (s_flag[1]) {
                 __threadfence();
-                // every thread merges one float4 column of one head; the pieces are read four at a time
-                // so that their loads are in flight together
-                for (int i4 = ctid; i4 < G * HD / 4; i4 += AT_CONSUMERS * 32) {
+                // every thread merges up to three float4 columns (one head each); a unit is rarely cut into more than
+                // four pieces, and then ALL loads of the thread -- every column, every piece -- are issued before the first
+                // use, so the merge costs one trip to memory
+                constexpr int NC = (MAX_G * HD / 4 + AT_CONSUMERS * 32 - 1) / (AT_CONSUMERS * 32);
+                const int ncols = G * HD / 4;
+                if (c_hi - c_lo < 4) {
+                    float mv[NC][4], lv[NC][4]; float4 pv[NC][4];
+#pragma unroll
+                    for (int x = 0; x < NC; x++) {
+                        const int i4 = ctid + x * AT_CONSUMERS * 32;
+                        const int g = (i4 * 4) / HD;
+#pragma unroll
+                        for (int j = 0; j < 4; j++) {
+                            const int cc = c_lo + j;
+                            mv[x][j] = -INFINITY; lv[x][j] = 0.f; pv[x][j] = make_float4(0.f, 0.f, 0.f, 0.f);
+                            if (i4 < ncols && cc <= c_hi) {
+                                const int slot = (cc == c_lo && cc * per != pf[u]) ? 1 : 0;
+                                const float* ps = t.part + (size_t)(2 * cc + slot) * rec_floats;
+                                mv[x][j] = __ldcg(ps + G * HD + g); lv[x][j] = __ldcg(ps + G * HD + 8 + g);
+                                pv[x][j] = __ldcg(reinterpret_cast<const float4*>(ps) + i4);
+                            }
+                        }
+                    }
+#pragma unroll
+                    for (int x = 0; x < NC; x++) {
+                        const int i4 = ctid + x * AT_CONSUMERS * 32;
+                        if (i4 >= ncols) continue;
+                        const float mm = fmaxf(fmaxf(mv[x][0], mv[x][1]), fmaxf(mv[x][2], mv[x][3]));
+                        float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
+                        float ll = 0.f;
+                        if (mm != -INFINITY) {
+#pragma unroll
+                            for (int j = 0; j < 4; j++) {
+                                const float f = mv[x][j] == -INFINITY ? 0.f : exp2f(mv[x][j] - mm);
+                                a.x += pv[x][j].x * f; a.y += pv[x][j].y * f; a.z += pv[x][j].z * f; a.w += pv[x][j].w * f;
+                                ll += lv[x][j] * f;
+                            }
+                        }
+                        const float inv = ll > 0.f ? 1.f / ll : 0.f;
+                        reinterpret_cast<float4*>(out + (size_t)u * G * HD)[i4] = make_float4(a.x * inv, a.y * inv, a.z * inv, a.w * inv);
+                    }
+                } else
+                for (int i4 = ctid; i4 < ncols; i4 += AT_CONSUMERS * 32) {
                     const int g = (i4 * 4) / HD;
                     float mm = -INFINITY, ll = 0.f;
                     float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
