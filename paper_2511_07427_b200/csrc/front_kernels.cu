@@ -99,13 +99,13 @@ __global__ void __launch_bounds__(FR_THREADS, 2) k_front(Tables t, StepPtr qp, S
 // One block per unit: see select_unit().  Block size: 512 threads when all units fit the GPU in one wave (the
 // shortest chain per block), 256 threads when there are more units than that (more blocks resident per SM; a
 // block's time is latency, not work).
-template <int THREADS>
+template <int THREADS, int MAXPER>
 __global__ void __launch_bounds__(THREADS) k_select(Tables t, int budget, int* __restrict__ user_ids) {
     extern __shared__ __align__(16) unsigned char sel_dyn[];
     __shared__ int s_last;
     const SelectSmem sm = select_smem_at(sel_dyn, t.max_clusters);
     pdl_wait();                          // the scores come from the kernel before
-    select_unit<THREADS>(t, blockIdx.x, budget, user_ids, sm);
+    select_unit<THREADS, MAXPER>(t, blockIdx.x, budget, user_ids, sm);
     // ---- With more units than the gather-attention CTAs keep in shared memory, the last unit block to finish lays
     // the units' work lists end to end (otherwise every attention CTA does that itself from n_work).
     if (!t.attn_pf_in_smem) {
@@ -152,8 +152,14 @@ void launch_front(const Tables& t, StepPtr q, StepPtr k, int has_q, int has_k, c
 
 void launch_select(const Tables& t, int budget, int* user_sel_ids, cudaStream_t s, long long* launches) {
     const size_t smem = select_smem_bytes(t.max_clusters);
-    if (t.U <= t.n_attn_ctas) launch_pdl(k_select<512>, dim3(t.U), dim3(512), smem, s, t, budget, user_sel_ids);
-    else launch_pdl(k_select<256>, dim3(t.U), dim3(256), smem, s, t, budget, user_sel_ids);
+    // threads x ids per thread >= the unit's id capacity.  One wave of units: the shortest chain per block (512
+    // threads, few ids each); more units than that: small blocks with few registers, many per SM.
+    const bool one_wave = t.U <= t.n_attn_ctas;
+    if (t.max_clusters > 2048 && one_wave) launch_pdl(k_select<512, 8>, dim3(t.U), dim3(512), smem, s, t, budget, user_sel_ids);
+    else if (t.max_clusters > 2048) launch_pdl(k_select<256, 16>, dim3(t.U), dim3(256), smem, s, t, budget, user_sel_ids);
+    else if (one_wave) launch_pdl(k_select<512, 4>, dim3(t.U), dim3(512), smem, s, t, budget, user_sel_ids);
+    else if (t.max_clusters <= 1024) launch_pdl(k_select<256, 4>, dim3(t.U), dim3(256), smem, s, t, budget, user_sel_ids);
+    else launch_pdl(k_select<256, 8>, dim3(t.U), dim3(256), smem, s, t, budget, user_sel_ids);
     (*launches)++;
 }
 

@@ -261,17 +261,19 @@ __device__ __forceinline__ unsigned int block_scan_excl_1sync(unsigned int v, un
 // Then the selection is written in id order, with the work list of the selected clusters' rows.
 // Nothing here waits for the unit's current id count: ids not yet handed out have size 0, like dead clusters, so
 // every load of the per-cluster tables is issued at once over the unit's whole id capacity.
-template <int THREADS>
+// MAXPER: most consecutive ids a thread owns; the caller picks THREADS * MAXPER >= max_clusters.
+template <int THREADS, int MAXPER>
 __device__ void select_unit(const Tables& t, int u, int budget, int* __restrict__ user_ids, const SelectSmem& sm) {
     static_assert(2048 % THREADS == 0 && THREADS % 32 == 0 && THREADS <= 1024, "bins are dealt out evenly to the threads");
     constexpr int BPT = 2048 / THREADS;           // histogram bins per thread
     constexpr int NW = THREADS / 32;
-    constexpr int MAXPER = (SL_MAXM + THREADS - 1) / THREADS;     // most consecutive ids a thread owns
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int Mlim = t.max_clusters;
-    const float* SC = t.scores + (size_t)u * Mlim;
-    const int* CN = t.cl_n + (size_t)u * Mlim;
-    const int* HEAD = t.cl_head + (size_t)u * Mlim;
+    // ids to look at: the whole id capacity, so that no load waits for the unit's id count -- unless the capacity is
+    // far above what the build handed out (a unit that may grow a lot): then the count is fetched first
+    const int Mlim = (t.max_clusters > 2 * t.M_floor + 64) ? min(t.max_clusters, __ldcg(&t.u_M[u])) : t.max_clusters;
+    const float* SC = t.scores + (size_t)u * t.max_clusters;
+    const int* CN = t.cl_n + (size_t)u * t.max_clusters;
+    const int* HEAD = t.cl_head + (size_t)u * t.max_clusters;
     const int* NEXT = t.page_next + (size_t)u * t.P;
     unsigned int* wtot = reinterpret_cast<unsigned int*>(sm.wtot);
     // ---- every thread owns a run of consecutive ids; all its loads are issued together (through L2: other blocks of a
@@ -393,7 +395,7 @@ __device__ void select_unit(const Tables& t, int u, int budget, int* __restrict_
     __syncthreads();                                                        // (6) selection marks final
     const int L = SEL_L;
     // ---- compaction in id order + work list
-    int* sel = t.sel_ids + (size_t)u * Mlim;
+    int* sel = t.sel_ids + (size_t)u * t.max_clusters;
     int2* work = t.work + (size_t)u * t.W;
     unsigned int my = 0;                          // work entries << 13 | selected clusters (at most 4096 ids, W < 2^19)
     bool on[MAXPER];
@@ -430,7 +432,7 @@ __device__ void select_unit(const Tables& t, int u, int budget, int* __restrict_
     if (user_ids) {
         // score order: rank = number of selected clusters that come first
         __syncthreads();
-        int* uo = user_ids + (size_t)u * Mlim;
+        int* uo = user_ids + (size_t)u * t.max_clusters;
         for (int a = tid; a < L; a += THREADS) {
             const int j = sel[a];
             const unsigned int kj = sm.keys[j];
@@ -442,7 +444,7 @@ __device__ void select_unit(const Tables& t, int u, int budget, int* __restrict_
             }
             uo[rank] = j;
         }
-        for (int p = L + tid; p < Mlim; p += THREADS) uo[p] = -1;
+        for (int p = L + tid; p < t.max_clusters; p += THREADS) uo[p] = -1;
     }
 }
 
