@@ -45,7 +45,7 @@ def _peaks():
 
 class ClockSampler:
     """Reads SM clock, power and clock-event reasons from NVML on a background thread
-    (read-only queries, about every 20 ms) between start() and stop()."""
+    (read-only queries, a few hundred per second) between start() and stop()."""
 
     def __init__(self, torch_device_index: int):
         import threading
@@ -80,7 +80,7 @@ class ClockSampler:
                 self.samples.append((time.perf_counter(), sm, pw, rs))
             except Exception:
                 pass
-            self._stop.wait(0.02)
+            self._stop.wait(0.003)
 
     def start(self):
         if self._thread is not None:
