@@ -328,10 +328,17 @@ __global__ void __launch_bounds__(SP_THREADS, DKV_SP_MINBLOCKS) k_split_check(Ta
             }
             for (int e = tid; e < HD; e += SP_THREADS) cA[e] = t.cl_r[cj * HD + e];
             __syncthreads();
-            // general path (the cluster does not fit the staging area): every pass walks the pages
-            unsigned char* label = label_g;
-            int* rank_of = rank_g;
-            int* holes = holes_g;
+            // general path (the cluster does not fit the staging area): every pass walks the pages.  The labels, ranks
+            // and hole list of a cluster of up to GEN_ROWS members live in the two staging areas, which this path does
+            // not use otherwise (every member's label is read and written once per 2-means round); beyond that in
+            // global memory.
+            constexpr int GEN_ROWS = 6144;
+            static_assert(8192 + 2 * GEN_ROWS * 4 <= 2 * SP_CACHE_BYTES, "labels, ranks and holes fit the two staging areas");
+            unsigned char* area = reinterpret_cast<unsigned char*>(krows);
+            const bool on_chip = c <= GEN_ROWS;
+            unsigned char* label = on_chip ? area : label_g;
+            int* rank_of = on_chip ? reinterpret_cast<int*>(area + 8192) : rank_g;
+            int* holes = on_chip ? reinterpret_cast<int*>(area + 8192) + GEN_ROWS : holes_g;
             // key row and token id of member position p
             auto key_of = [&](int p) -> const KV* { return kpg + ((size_t)chain[p >> 5] * PAGE + (p & 31)) * HD; };
             auto tok_of = [&](int p) -> int { return ptok[(size_t)chain[p >> 5] * PAGE + (p & 31)]; };
