@@ -389,20 +389,33 @@ __global__ void __launch_bounds__(SP_THREADS, DKV_SP_MINBLOCKS) k_split_check(Ta
 #pragma unroll
                 for (int e = 0; e < EPL; e++) { a_c[e] = cA[lane * EPL + e]; b_c[e] = cB[lane * EPL + e]; sa[e] = 0.f; sb[e] = 0.f; }
                 int chg = 0, ca = 0, cb = 0;
-                for (int p = warp; p < c; p += SP_WARPS) {
-                    const KV* k = key_of(p) + lane * EPL;
-                    float kk[EPL], da = 0.f, db = 0.f;
+                // two rows of the warp at a time, their loads issued together (the rows live in global memory)
+                for (int p0 = warp; p0 < c; p0 += 2 * SP_WARPS) {
+                    const int p1 = p0 + SP_WARPS;
+                    float k0[EPL], k1[EPL];
+                    {
+                        const KV* r0 = key_of(p0) + lane * EPL;
+                        const KV* r1 = key_of(p1 < c ? p1 : p0) + lane * EPL;
 #pragma unroll
-                    for (int e = 0; e < EPL; e++) {
-                        kk[e] = to_f(k[e]);
-                        float x = kk[e] - a_c[e], y = kk[e] - b_c[e];
-                        da = fmaf(x, x, da); db = fmaf(y, y, db);
+                        for (int e = 0; e < EPL; e++) { k0[e] = to_f(r0[e]); k1[e] = to_f(r1[e]); }
                     }
-                    da = warp_sum(da); db = warp_sum(db);
-                    const int l = db < da ? 1 : 0;
-                    if (lane == 0) { if (label[p] != l) chg = 1; label[p] = (unsigned char)l; if (l) cb++; else ca++; }
 #pragma unroll
-                    for (int e = 0; e < EPL; e++) { if (l) sb[e] += kk[e]; else sa[e] += kk[e]; }
+                    for (int b2 = 0; b2 < 2; b2++) {
+                        const int p = b2 ? p1 : p0;
+                        if (p >= c) break;
+                        float da = 0.f, db = 0.f;
+#pragma unroll
+                        for (int e = 0; e < EPL; e++) {
+                            const float kv = b2 ? k1[e] : k0[e];
+                            float x = kv - a_c[e], y = kv - b_c[e];
+                            da = fmaf(x, x, da); db = fmaf(y, y, db);
+                        }
+                        da = warp_sum(da); db = warp_sum(db);
+                        const int l = db < da ? 1 : 0;
+                        if (lane == 0) { if (label[p] != l) chg = 1; label[p] = (unsigned char)l; if (l) cb++; else ca++; }
+#pragma unroll
+                        for (int e = 0; e < EPL; e++) { const float kv = b2 ? k1[e] : k0[e]; if (l) sb[e] += kv; else sa[e] += kv; }
+                    }
                 }
 #pragma unroll
                 for (int e = 0; e < EPL; e++) { WS(warp, 0, lane * EPL + e) = sa[e]; WS(warp, 1, lane * EPL + e) = sb[e]; }
