@@ -39,7 +39,7 @@ class WorkloadConfig:
     Hq: int
     Hkv: int
     d: int
-    kv_dtype: str          # "f32" | "bf16"
+    kv_dtype: str          # "f32" | "bf16" | "fp8" (bf16 rows handed over, stored as e4m3 bytes with a scale per row)
     n_prefill: int
     steps: int
     M0: int                # clusters per unit at build time
@@ -115,7 +115,7 @@ def _round_storage(x: torch.Tensor, cfg: WorkloadConfig) -> torch.Tensor:
 
 
 def _round_query(x: torch.Tensor, cfg: WorkloadConfig) -> torch.Tensor:
-    if cfg.kv_dtype == "bf16":
+    if cfg.kv_dtype != "f32":
         return x.to(torch.bfloat16).to(torch.float32)
     return x
 

@@ -32,6 +32,14 @@ extern "C" {
 
 #define DYNAKV_F32 0
 #define DYNAKV_BF16 1
+/* DYNAKV_FP8: K and V are PASSED as bf16 arrays (like DYNAKV_BF16) and kept in the precision the paper evaluates in
+ * (Section 8.1): every row is rounded, where it enters the library, to e4m3 values (OCP 8-bit float: 4 exponent
+ * bits, 3 mantissa bits, largest value 448) times one power-of-two scale per row, the smallest 2^e with
+ * max|x| / 2^e <= 448, round to nearest even.  All arithmetic of the method then runs on those rounded values
+ * (they are exact in bf16), and the gather-attention kernel streams a one-byte-per-element copy of the pages: half
+ * the bytes of DYNAKV_BF16 per retrieved token.  The context keeps the bf16 pages as well, for the paths that move or
+ * re-read rows (splits, statistics, export).  head_dim 128 only. */
+#define DYNAKV_FP8 2
 
 #define DYNAKV_INIT_KMEANSPP 0
 #define DYNAKV_INIT_RANDOM 1
@@ -56,7 +64,7 @@ typedef struct dynakv_config {
     int32_t n_units;           /* U = sequences x layers x KV heads                              */
     int32_t gqa_group;         /* G, 1..8                                                        */
     int32_t head_dim;          /* d: 64 or 128                                                   */
-    int32_t kv_dtype;          /* DYNAKV_F32 or DYNAKV_BF16 for K, V; q, out, centroids are fp32 */
+    int32_t kv_dtype;          /* DYNAKV_F32, DYNAKV_BF16 or DYNAKV_FP8 for K, V; q, out, centroids are fp32 */
     int32_t max_tokens;        /* capacity per unit (prefill + decode)                           */
     int32_t max_clusters;      /* cluster ids per unit, <= 4096                                  */
     int32_t kmeans_iters;      /* T: Lloyd rounds at build time (all are run, no early exit)     */

@@ -5,11 +5,11 @@ marshals ``torch`` device tensors (memory and streams) into the C ABI declared i
 ``include/dynakv.h``.  There is no CPU fallback: importing the binding without the built
 library raises.
 """
-from .binding import (DynaKV, DynaKVConfig, DynaKVError, load_library, F32, BF16, INIT_KMEANSPP, INIT_RANDOM,
+from .binding import (DynaKV, DynaKVConfig, DynaKVError, load_library, F32, BF16, FP8, INIT_KMEANSPP, INIT_RANDOM,
                       MODE_ADAPTIVE, MODE_STATIC, MODE_LOCAL,
                       ST_BUDGET_EXCEEDED, ST_MAX_CLUSTERS, ST_MAX_TOKENS, ST_PAGE_POOL, ST_INTERNAL, EXPORTED_SYMBOLS, attend_rows_noalloc)
 
-__all__ = ["DynaKV", "DynaKVConfig", "DynaKVError", "load_library", "F32", "BF16", "INIT_KMEANSPP", "INIT_RANDOM",
+__all__ = ["DynaKV", "DynaKVConfig", "DynaKVError", "load_library", "F32", "BF16", "FP8", "INIT_KMEANSPP", "INIT_RANDOM",
            "MODE_ADAPTIVE", "MODE_STATIC", "MODE_LOCAL",
            "ST_BUDGET_EXCEEDED", "ST_MAX_CLUSTERS", "ST_MAX_TOKENS", "ST_PAGE_POOL", "ST_INTERNAL", "EXPORTED_SYMBOLS",
            "attend_rows_noalloc"]

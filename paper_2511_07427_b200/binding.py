@@ -11,7 +11,7 @@ import numpy as np
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _LIB_PATH = os.path.join(_HERE, "libdynakv.so")
 
-F32, BF16 = 0, 1
+F32, BF16, FP8 = 0, 1, 2
 INIT_KMEANSPP, INIT_RANDOM = 0, 1
 MODE_ADAPTIVE, MODE_STATIC, MODE_LOCAL = 0, 1, 2
 ST_BUDGET_EXCEEDED, ST_MAX_CLUSTERS, ST_MAX_TOKENS, ST_PAGE_POOL, ST_INTERNAL = 1, 2, 4, 8, 16

@@ -135,7 +135,8 @@ extern "C" int dynakv_create(const dynakv_config* cfg, void* cuda_stream, dynakv
     *out = nullptr;
     if (cfg->n_units < 1 || cfg->gqa_group < 1 || cfg->gqa_group > MAX_G) return DYNAKV_ERR_ARG;
     if (cfg->head_dim != 64 && cfg->head_dim != 128) return DYNAKV_ERR_ARG;
-    if (cfg->kv_dtype != DYNAKV_F32 && cfg->kv_dtype != DYNAKV_BF16) return DYNAKV_ERR_ARG;
+    if (cfg->kv_dtype != DYNAKV_F32 && cfg->kv_dtype != DYNAKV_BF16 && cfg->kv_dtype != DYNAKV_FP8) return DYNAKV_ERR_ARG;
+    if (cfg->kv_dtype == DYNAKV_FP8 && cfg->head_dim != 128) return DYNAKV_ERR_ARG;
     if (cfg->max_tokens < 1 || cfg->max_clusters < 1 || cfg->max_clusters > 4096) return DYNAKV_ERR_ARG;
     if (cfg->kmeans_iters < 1 || cfg->split_iters < 1) return DYNAKV_ERR_ARG;
     if (cfg->init_mode != DYNAKV_INIT_KMEANSPP && cfg->init_mode != DYNAKV_INIT_RANDOM) return DYNAKV_ERR_ARG;
@@ -147,7 +148,9 @@ extern "C" int dynakv_create(const dynakv_config* cfg, void* cuda_stream, dynakv
     c->stream = reinterpret_cast<cudaStream_t>(cuda_stream);
     Tables& t = c->t;
     memset(&t, 0, sizeof(t));
-    t.U = cfg->n_units; t.G = cfg->gqa_group; t.d = cfg->head_dim; t.kv_dtype = cfg->kv_dtype;
+    t.U = cfg->n_units; t.G = cfg->gqa_group; t.d = cfg->head_dim;
+    t.fp8 = cfg->kv_dtype == DYNAKV_FP8 ? 1 : 0;
+    t.kv_dtype = t.fp8 ? DYNAKV_BF16 : cfg->kv_dtype;
     t.max_tokens = cfg->max_tokens; t.max_clusters = cfg->max_clusters;
     t.update_mode = cfg->update_mode; t.local_max = cfg->local_max;
     const int full_pages = (cfg->max_tokens + PAGE - 1) / PAGE;
@@ -172,6 +175,10 @@ extern "C" int dynakv_create(const dynakv_config* cfg, void* cuda_stream, dynakv
     }
     const size_t U = t.U, P = t.P, Mx = t.max_clusters, d = t.d;
     const size_t page_elems = U * P * PAGE * d;
+    if (t.fp8) {
+        ALLOC(t.k8, page_elems, false); ALLOC(t.v8, page_elems, false);
+        ALLOC(t.k8e, U * P * PAGE, true); ALLOC(t.v8e, U * P * PAGE, true);
+    }
     if (cfg->kv_dtype == DYNAKV_F32) {
         float *a, *b; ALLOC(a, page_elems, false); ALLOC(b, page_elems, false); t.kpages = a; t.vpages = b;
     } else {
@@ -209,7 +216,7 @@ extern "C" int dynakv_create(const dynakv_config* cfg, void* cuda_stream, dynakv
     ALLOC(t.front_done, U, true);
     ALLOC(t.trig_n, U, true);
     ALLOC(t.trig_list, U * Mx, false);
-    if (cfg->kv_dtype == DYNAKV_BF16 && attn_tma_prepare(t) != 0) {
+    if (t.kv_dtype == DYNAKV_BF16 && attn_tma_prepare(t) != 0) {
         snprintf(g_err, sizeof(g_err), "cannot reserve shared memory for the gather-attention kernel: %s", cudaGetErrorString(cudaGetLastError()));
         dynakv_destroy(c);
         return DYNAKV_ERR_CUDA;
@@ -268,6 +275,14 @@ extern "C" int dynakv_build_index(dynakv_ctx* c, const void* K, const void* V, i
     int* assign_buf = nullptr;
     if (c->cfg.trace) { ALLOC_B(c->trace_assign, (size_t)T * U * n, false); }
     else ALLOC_B(assign_buf, U * (size_t)n, false);
+    if (t.fp8) {
+        // FP8 mode: the rows are rounded to the storage grid first; everything below works on the rounded copies
+        __nv_bfloat16 *kq, *vq;
+        ALLOC_B(kq, U * (size_t)n * d, false); ALLOC_B(vq, U * (size_t)n * d, false);
+        launch_fp8_round_rows(K, kq, (long long)U * n, c->stream, &c->launches);
+        launch_fp8_round_rows(V, vq, (long long)U * n, c->stream, &c->launches);
+        K = kq; V = vq;
+    }
     bool use_tc = c->cfg.assign_mode == 0 && tc_assign_supported(t, n, M);
     void* tc_scratch = nullptr;
     if (use_tc) { char* p; ALLOC_B(p, tc_assign_scratch_bytes(t, n, M), false); tc_scratch = p; }
@@ -317,7 +332,7 @@ static void enqueue_retrieve(dynakv_ctx* c, StepPtr q, int budget, StepPtrW out,
 }
 
 static void enqueue_attend(dynakv_ctx* c, StepPtr q, StepPtrW out, bool timed) {
-    if (c->t.kv_dtype == DYNAKV_BF16 && c->cfg.attn_mode == 0) {
+    if (c->t.kv_dtype == DYNAKV_BF16 && c->cfg.attn_mode == 0 && !c->t.fp8) {
         // gather, attend and combine in one persistent kernel
         TimeScope ts(c, KC_ATTN, timed);
         launch_gather_attn_tma(c->t, q, out, c->stream, &c->launches);
@@ -660,6 +675,13 @@ extern "C" int dynakv_import_state(dynakv_ctx* c, const void* K, const void* V, 
     ALLOC_B(ids_dev, U, false);
     ALLOC_B(tau_dev, U, false);
     b.assign = const_cast<int*>(tok_cluster);
+    if (t.fp8) {
+        __nv_bfloat16 *kq, *vq;
+        ALLOC_B(kq, U * (size_t)n * d, false); ALLOC_B(vq, U * (size_t)n * d, false);
+        launch_fp8_round_rows(K, kq, (long long)U * n, c->stream, &c->launches);
+        launch_fp8_round_rows(V, vq, (long long)U * n, c->stream, &c->launches);
+        K = kq; V = vq;
+    }
     CK(cudaMemcpyAsync(ids_dev, n_ids, sizeof(int) * U, cudaMemcpyHostToDevice, c->stream));
     CK(cudaMemcpyAsync(tau_dev, tau, sizeof(float) * U, cudaMemcpyHostToDevice, c->stream));
     // representatives = member means (Eq. 4), then the layout and the exact statistics, as at the end of a build
@@ -709,7 +731,7 @@ extern "C" int dynakv_selftest_wait_expiry(dynakv_ctx* c, int32_t* gave_up) {
 extern "C" int dynakv_time_gather_attention(dynakv_ctx* c, const float* q, float* out, int32_t reps, float* ms_per_launch) {
     if (!c || !q || !out || !ms_per_launch || reps < 1) return DYNAKV_ERR_ARG;
     if (!c->built) return DYNAKV_ERR_STATE;
-    if (c->t.kv_dtype != DYNAKV_BF16 || c->cfg.attn_mode != 0) return DYNAKV_ERR_ARG;
+    if (c->t.kv_dtype != DYNAKV_BF16 || c->cfg.attn_mode != 0 || c->t.fp8) return DYNAKV_ERR_ARG;
     cudaEvent_t e0, e1;
     CK(cudaEventCreate(&e0)); CK(cudaEventCreate(&e1));
     const StepPtr qp{q, 0, nullptr};

@@ -4,6 +4,7 @@
 #pragma once
 
 #include "common.cuh"
+#include "fp8_rows.cuh"
 
 namespace dkv {
 
@@ -94,10 +95,29 @@ __device__ __forceinline__ void append_block(const Tables& t, int u, StepPtr kp_
     const float n_new = (float)(n_old + 1);
     float* r = t.cl_r + cj * HD;
     float add = 0.f;
-    float kk[EPL];
+    float kk[EPL], vv[EPL];
+#pragma unroll
+    for (int e = 0; e < EPL; e++) { kk[e] = to_f(knew[lane * EPL + e]); vv[e] = to_f(vnew[lane * EPL + e]); }
+    unsigned k8w = 0, v8w = 0;        // FP8 mode: the row's four bytes of this lane, and the rows' scale exponents
+    int k8x = 0, v8x = 0;
+    if (t.fp8) {
+        // the new row enters the library here: round it to the storage grid (a warp holds the whole row)
+        if constexpr (EPL == 4) {
+            float am = fmaxf(fmaxf(fabsf(kk[0]), fabsf(kk[1])), fmaxf(fabsf(kk[2]), fabsf(kk[3])));
+            k8x = fp8_row_exp(group_max(am, 32));
+            am = fmaxf(fmaxf(fabsf(vv[0]), fabsf(vv[1])), fmaxf(fabsf(vv[2]), fabsf(vv[3])));
+            v8x = fp8_row_exp(group_max(am, 32));
+            const float ki = pow2f(-k8x), ks = pow2f(k8x), vi = pow2f(-v8x), vs = pow2f(v8x);
+            k8w = (unsigned)fp8_pack2(kk[0], kk[1], ki) | ((unsigned)fp8_pack2(kk[2], kk[3], ki) << 16);
+            v8w = (unsigned)fp8_pack2(vv[0], vv[1], vi) | ((unsigned)fp8_pack2(vv[2], vv[3], vi) << 16);
+            float2 a = fp8_unpack2((unsigned short)(k8w & 0xffffu), ks), b = fp8_unpack2((unsigned short)(k8w >> 16), ks);
+            kk[0] = a.x; kk[1] = a.y; kk[2] = b.x; kk[3] = b.y;
+            a = fp8_unpack2((unsigned short)(v8w & 0xffffu), vs); b = fp8_unpack2((unsigned short)(v8w >> 16), vs);
+            vv[0] = a.x; vv[1] = a.y; vv[2] = b.x; vv[3] = b.y;
+        }
+    }
 #pragma unroll
     for (int e = 0; e < EPL; e++) {
-        kk[e] = to_f(knew[lane * EPL + e]);
         const float ro = found ? kk[e] : r[lane * EPL + e];          // a founded cluster starts at r = k, M2 = 0
         const float delta = kk[e] - ro;
         const float rn = ro + delta / n_new;
@@ -108,7 +128,13 @@ __device__ __forceinline__ void append_block(const Tables& t, int u, StepPtr kp_
     KV* kpg = reinterpret_cast<KV*>(t.kpages) + (((size_t)u * t.P + page) * PAGE + row) * HD;
     KV* vpg = reinterpret_cast<KV*>(t.vpages) + (((size_t)u * t.P + page) * PAGE + row) * HD;
 #pragma unroll
-    for (int e = 0; e < EPL; e++) { kpg[lane * EPL + e] = knew[lane * EPL + e]; vpg[lane * EPL + e] = vnew[lane * EPL + e]; }
+    for (int e = 0; e < EPL; e++) { kpg[lane * EPL + e] = (KV)kk[e]; vpg[lane * EPL + e] = (KV)vv[e]; }
+    if (t.fp8) {
+        const size_t slot = ((size_t)u * t.P + page) * PAGE + row;
+        *reinterpret_cast<unsigned*>(t.k8 + slot * HD + lane * 4) = k8w;
+        *reinterpret_cast<unsigned*>(t.v8 + slot * HD + lane * 4) = v8w;
+        if (lane == 0) { t.k8e[slot] = (signed char)k8x; t.v8e[slot] = (signed char)v8x; }
+    }
     if (lane == 0) {
         const float m2_new = found ? 0.f : t.cl_M2[cj] + add;
         t.cl_M2[cj] = m2_new;

@@ -4,8 +4,37 @@
 #include <float.h>
 
 #include "common.cuh"
+#include "fp8_rows.cuh"
 
 namespace dkv {
+
+// ------------------------------------------------------------------ FP8 mode: rows rounded where they enter
+
+// One warp per row of 128 bf16 elements: the row rounded to e4m3 values times the row's power-of-two scale, written
+// back as bf16 (exact).  Every later kernel of the build works on these rows.
+__global__ void __launch_bounds__(256) k_fp8_round_rows(const __nv_bfloat16* __restrict__ X, __nv_bfloat16* __restrict__ Y, long long rows) {
+    const int lane = threadIdx.x & 31;
+    long long w = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const long long nw = ((long long)gridDim.x * blockDim.x) >> 5;
+    for (; w < rows; w += nw) {
+        const float4 v = ld4(X + (size_t)w * 128, lane * 4);
+        const float amax = group_max(fmaxf(fmaxf(fabsf(v.x), fabsf(v.y)), fmaxf(fabsf(v.z), fabsf(v.w))), 32);
+        const int e = fp8_row_exp(amax);
+        const float sc = pow2f(e), inv = pow2f(-e);
+        const float2 a = fp8_round2(v.x, v.y, inv, sc), b = fp8_round2(v.z, v.w, inv, sc);
+        __nv_bfloat162 o0 = __floats2bfloat162_rn(a.x, a.y), o1 = __floats2bfloat162_rn(b.x, b.y);
+        uint2 pk;
+        pk.x = *reinterpret_cast<unsigned*>(&o0); pk.y = *reinterpret_cast<unsigned*>(&o1);
+        *reinterpret_cast<uint2*>(Y + (size_t)w * 128 + lane * 4) = pk;
+    }
+}
+
+void launch_fp8_round_rows(const void* X, void* Y, long long rows, cudaStream_t s, long long* launches) {
+    long long blocks = (rows + 7) / 8;
+    if (blocks > 148LL * 32) blocks = 148LL * 32;
+    k_fp8_round_rows<<<(unsigned)blocks, 256, 0, s>>>(reinterpret_cast<const __nv_bfloat16*>(X), reinterpret_cast<__nv_bfloat16*>(Y), rows);
+    (*launches)++;
+}
 
 // ------------------------------------------------------------------ init: k-means++
 
@@ -318,6 +347,22 @@ __global__ void __launch_bounds__(256) k_fin_scatter(Tables t, const KV* __restr
         const KV* vs = V + (size_t)w * HD + lane * EPL;
 #pragma unroll
         for (int e = 0; e < EPL; e++) { kp[dst + lane * EPL + e] = ks[e]; vp[dst + lane * EPL + e] = vs[e]; }
+        if (t.fp8) {
+            // the one-byte copy of the row (the rows are on the grid already, so this conversion is exact)
+            if constexpr (HD == 128 && sizeof(KV) == 2) {
+                const size_t slot = ((size_t)u * t.P + page) * PAGE + row;
+#pragma unroll
+                for (int side = 0; side < 2; side++) {
+                    const KV* src = side == 0 ? ks : vs;
+                    const float x0 = to_f(src[0]), x1 = to_f(src[1]), x2 = to_f(src[2]), x3 = to_f(src[3]);
+                    const int ex = fp8_row_exp(group_max(fmaxf(fmaxf(fabsf(x0), fabsf(x1)), fmaxf(fabsf(x2), fabsf(x3))), 32));
+                    const float inv = pow2f(-ex);
+                    const unsigned pk = (unsigned)fp8_pack2(x0, x1, inv) | ((unsigned)fp8_pack2(x2, x3, inv) << 16);
+                    *reinterpret_cast<unsigned*>((side == 0 ? t.k8 : t.v8) + slot * HD + lane * 4) = pk;
+                    if (lane == 0) (side == 0 ? t.k8e : t.v8e)[slot] = (signed char)ex;
+                }
+            }
+        }
         if (lane == 0) {
             t.page_tok[((size_t)u * t.P + page) * PAGE + row] = i;
             t.tok_cluster[(size_t)u * t.max_tokens + i] = j;

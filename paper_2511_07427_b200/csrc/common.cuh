@@ -26,6 +26,11 @@ constexpr int FLAG_HOLD = 1;        // split abandoned; not retried until the ne
 struct Tables {
     int U, G, d, kv_dtype, max_tokens, max_clusters, P, n_splits_attn;
     int update_mode, local_max;      // DYNAKV_MODE_*; LOCAL: size above which a decode-born cluster splits
+    // FP8 mode (fp8 != 0): kv_dtype is DYNAKV_BF16 for every kernel, all rows lie on the e4m3-times-power-of-two grid,
+    // and a one-byte copy of the pages is kept for the gather-attention kernel
+    int fp8;
+    unsigned char* k8; unsigned char* v8;          // [U][P][PAGE][d] e4m3 bytes
+    signed char* k8e; signed char* v8e;            // [U][P][PAGE] exponent of the row's power-of-two scale
     int W;                           // work-list capacity per unit (entries)
     int M_floor;                     // clusters every unit has had since the build (ids never go away); 0 before it
     void* kpages; void* vpages;
@@ -206,6 +211,7 @@ struct LoopBegin {
     const void** args;        // device: [4] q, k, v, out of the loop in flight
     const void* q; const void* k; const void* v; void* out;
 };
+void launch_fp8_round_rows(const void* X, void* Y, long long rows, cudaStream_t s, long long* launches);
 void launch_export_rows(const Tables& t, void* K, void* V, long long n, cudaStream_t s, long long* launches);
 void launch_import_units(const Tables& t, const int* n_ids, const float* tau, cudaStream_t s, long long* launches);
 void launch_front(const Tables& t, StepPtr q, StepPtr k, int has_q, int has_k, cudaStream_t s, long long* launches,

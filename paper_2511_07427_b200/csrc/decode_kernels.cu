@@ -4,6 +4,7 @@
 #include <float.h>
 
 #include "common.cuh"
+#include "fp8_rows.cuh"
 
 namespace dkv {
 
@@ -45,8 +46,22 @@ __global__ void __launch_bounds__(128) k_gather_attn_v1(Tables t, StepPtr qp) {
             const KV* k = kp + pbase + (size_t)r * HD + lane * EPL;
             const KV* v = vp + pbase + (size_t)r * HD + lane * EPL;
             float kk[EPL], vv[EPL];
+            if (t.fp8) {
+                // FP8 mode: the row's one-byte copy (four bytes per lane) and its two scale exponents
+                if constexpr (EPL == 4) {
+                    const size_t slot = (size_t)u * t.P * PAGE + ent.x + r;
+                    const unsigned kb = *reinterpret_cast<const unsigned*>(t.k8 + slot * HD + lane * 4);
+                    const unsigned vb = *reinterpret_cast<const unsigned*>(t.v8 + slot * HD + lane * 4);
+                    const float ks = pow2f(t.k8e[slot]), vs = pow2f(t.v8e[slot]);
+                    float2 a = fp8_unpack2((unsigned short)(kb & 0xffffu), ks), b = fp8_unpack2((unsigned short)(kb >> 16), ks);
+                    kk[0] = a.x; kk[1] = a.y; kk[2] = b.x; kk[3] = b.y;
+                    a = fp8_unpack2((unsigned short)(vb & 0xffffu), vs); b = fp8_unpack2((unsigned short)(vb >> 16), vs);
+                    vv[0] = a.x; vv[1] = a.y; vv[2] = b.x; vv[3] = b.y;
+                }
+            } else {
 #pragma unroll
             for (int e = 0; e < EPL; e++) { kk[e] = to_f(k[e]); vv[e] = to_f(v[e]); }
+            }
 #pragma unroll
             for (int g = 0; g < G; g++) {
                 float p = 0.f;

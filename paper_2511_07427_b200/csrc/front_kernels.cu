@@ -74,7 +74,7 @@ __global__ void __launch_bounds__(FR_THREADS, 2) k_front(Tables t, StepPtr qp, S
 #pragma unroll
         for (int e = 0; e < 4; e++) { qs[i][e] = 0.f; kk[i][e] = 0.f; }
     if (has_q) front_qsum_load<HD>(reinterpret_cast<const float*>(qp.get()) + (size_t)u * t.G * HD, t.G, lane, qs);
-    if (has_k) front_key_load<KV, HD>(reinterpret_cast<const KV*>(kp.get()) + (size_t)u * HD, lane, kk);
+    if (has_k) front_key_load<KV, HD>(reinterpret_cast<const KV*>(kp.get()) + (size_t)u * HD, lane, kk, t.fp8);
     if (has_q) front_qsum_finish<HD>(qs);
     const float invG = 1.0f / (float)t.G;
     float* SC = t.scores + (size_t)u * t.max_clusters;

@@ -6,6 +6,7 @@
 #pragma once
 
 #include "common.cuh"
+#include "fp8_rows.cuh"
 
 namespace dkv {
 
@@ -42,13 +43,28 @@ __device__ __forceinline__ void front_qsum_finish(float (&qs)[HD / 32][4]) {
         }
 }
 
+// fp8: the key is rounded to the FP8 storage grid first (the eight lanes of a row group hold the whole row).
 template <typename KV, int HD>
-__device__ __forceinline__ void front_key_load(const KV* __restrict__ k, int lane, float (&kk)[HD / 32][4]) {
+__device__ __forceinline__ void front_key_load(const KV* __restrict__ k, int lane, float (&kk)[HD / 32][4], int fp8 = 0) {
     const int l8 = lane & 7;
 #pragma unroll
     for (int i = 0; i < HD / 32; i++) {
         const float4 v = ld4(k, l8 * 4 + 32 * i);
         kk[i][0] = v.x; kk[i][1] = v.y; kk[i][2] = v.z; kk[i][3] = v.w;
+    }
+    if (fp8) {
+        float am = 0.f;
+#pragma unroll
+        for (int i = 0; i < HD / 32; i++)
+#pragma unroll
+            for (int e = 0; e < 4; e++) am = fmaxf(am, fabsf(kk[i][e]));
+        const int ex = fp8_row_exp(group_max(am, 8));
+        const float sc = pow2f(ex), inv = pow2f(-ex);
+#pragma unroll
+        for (int i = 0; i < HD / 32; i++) {
+            const float2 a = fp8_round2(kk[i][0], kk[i][1], inv, sc), b = fp8_round2(kk[i][2], kk[i][3], inv, sc);
+            kk[i][0] = a.x; kk[i][1] = a.y; kk[i][2] = b.x; kk[i][3] = b.y;
+        }
     }
 }
 

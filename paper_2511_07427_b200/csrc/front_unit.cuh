@@ -87,7 +87,7 @@ __device__ __forceinline__ bool front_unit(const Tables& t, int u, const float* 
     if (tid == 0 && nch > 2) { fence_proxy_async(); issue(2); }
     float qs[V4][4], kk[V4][4];
     front_qsum_load<HD>(q, t.G, lane, qs);
-    front_key_load<KV, HD>(k, lane, kk);
+    front_key_load<KV, HD>(k, lane, kk, t.fp8);
     front_qsum_finish<HD>(qs);
     const float invG = 1.0f / (float)t.G;
     float* SC = t.scores + (size_t)u * t.max_clusters;
@@ -149,7 +149,7 @@ __device__ __forceinline__ void front_patch(const Tables& t, int u, const float*
     const int lane = threadIdx.x & 31, sub = lane >> 3, l8 = lane & 7;
     float qs[V4][4], kk[V4][4];
     front_qsum_load<HD>(q, t.G, lane, qs);
-    front_key_load<KV, HD>(k, lane, kk);
+    front_key_load<KV, HD>(k, lane, kk, t.fp8);
     front_qsum_finish<HD>(qs);
     const int j = sub == 0 ? ja : (sub == 1 ? jb : -1);
     const float* R = sub == 0 ? ra : rb;

@@ -47,6 +47,15 @@ template <int HD, int KVB> struct SplitSmem {
     __host__ __device__ static size_t total(int maxch, int max_clusters) { return live_off(maxch, max_clusters) + (size_t)max_clusters + 16; }
 };
 
+// FP8 mode: the one-byte copy of a row (128 bytes and the two scale exponents) follows the row from slot src to slot
+// dst of unit u's pages; called by a full warp.
+__device__ __forceinline__ void fp8_move_row(const Tables& t, int u, size_t src, size_t dst, int lane) {
+    const size_t gs = (size_t)u * t.P * PAGE + src, gd = (size_t)u * t.P * PAGE + dst;
+    reinterpret_cast<unsigned*>(t.k8 + gd * t.d)[lane] = reinterpret_cast<const unsigned*>(t.k8 + gs * t.d)[lane];
+    reinterpret_cast<unsigned*>(t.v8 + gd * t.d)[lane] = reinterpret_cast<const unsigned*>(t.v8 + gs * t.d)[lane];
+    if (lane == 0) { t.k8e[gd] = t.k8e[gs]; t.v8e[gd] = t.v8e[gs]; }
+}
+
 // ---- hand-over of triggered units from the unit blocks to the helper blocks of a loop iteration's tail kernel.
 // tail_sync[0] = queue slots reserved, [1] = slots claimed by helpers, [2] = unit blocks that have decided.
 // A unit block with triggered clusters reserves a slot (two words) and stores a hint, then unit + 1, in it; a
@@ -506,6 +515,7 @@ __global__ void __launch_bounds__(SP_THREADS, DKV_SP_MINBLOCKS) k_split_check(Ta
                     kpg[dst * HD + lane * EPL + e] = kpg[src * HD + lane * EPL + e];
                     vpg[dst * HD + lane * EPL + e] = vpg[src * HD + lane * EPL + e];
                 }
+                if (t.fp8) fp8_move_row(t, u, src, dst, lane);
                 if (lane == 0) {
                     int tok = ptok[src];
                     ptok[dst] = tok;
@@ -524,6 +534,7 @@ __global__ void __launch_bounds__(SP_THREADS, DKV_SP_MINBLOCKS) k_split_check(Ta
                     kpg[dst * HD + lane * EPL + e] = kpg[src * HD + lane * EPL + e];
                     vpg[dst * HD + lane * EPL + e] = vpg[src * HD + lane * EPL + e];
                 }
+                if (t.fp8) fp8_move_row(t, u, src, dst, lane);
                 if (lane == 0) ptok[dst] = ptok[src];
             }
             __syncthreads();

@@ -17,6 +17,7 @@
 #pragma once
 
 #include "common.cuh"
+#include "fp8_rows.cuh"
 
 namespace dkv {
 
@@ -47,6 +48,7 @@ __device__ int split_small(const Tables& t, int u, int j, int c, int iters, KV* 
     __shared__ int s_ok;
     constexpr int Q = THREADS / HD;                       // row slices of the member-sum pass
     __shared__ int s_pcnt[Q];
+    __shared__ signed char s_kx[MAXROWS], s_vx[MAXROWS];     // FP8 mode: the staged rows' scale exponents
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, sub = lane >> 3, l8 = lane & 7;
     const int grp = warp * 4 + sub;
     const size_t cj = (size_t)u * t.max_clusters + j;
@@ -85,7 +87,11 @@ __device__ int split_small(const Tables& t, int u, int j, int c, int iters, KV* 
         reinterpret_cast<uint4*>(krows + (size_t)p * HD)[v] = reinterpret_cast<const uint4*>(kpg + row * HD)[v];
         reinterpret_cast<uint4*>(vrows + (size_t)p * HD)[v] = reinterpret_cast<const uint4*>(vpg + row * HD)[v];
     }
-    if (tid < c) { sc.tok[tid] = ptok[(size_t)page_of(tid >> 5) * PAGE + (tid & 31)]; sc.label[tid] = 255; }
+    if (tid < c) {
+        const size_t slot = (size_t)page_of(tid >> 5) * PAGE + (tid & 31);
+        sc.tok[tid] = ptok[slot]; sc.label[tid] = 255;
+        if (t.fp8) { s_kx[tid] = t.k8e[(size_t)u * t.P * PAGE + slot]; s_vx[tid] = t.v8e[(size_t)u * t.P * PAGE + slot]; }
+    }
     __syncthreads();
 
     // ---- member farthest from a centre (ties: lowest token id).  The centre arrives in registers, as this
@@ -269,6 +275,23 @@ __device__ int split_small(const Tables& t, int u, int j, int c, int iters, KV* 
         else { const int h = sc.holes[-2 - code]; dst = (size_t)page_of(h >> 5) * PAGE + (h & 31); }
         reinterpret_cast<uint4*>(kpg + dst * HD)[v] = reinterpret_cast<const uint4*>(krows + (size_t)p * HD)[v];
         reinterpret_cast<uint4*>(vpg + dst * HD)[v] = reinterpret_cast<const uint4*>(vrows + (size_t)p * HD)[v];
+        if (t.fp8) {
+            // the one-byte copy follows the row: the staged values are on the grid, so packing them with the row's own
+            // scale gives the row's bytes back
+            if constexpr (sizeof(KV) == 2) {
+                const size_t g = (size_t)u * t.P * PAGE + dst;
+#pragma unroll
+                for (int side = 0; side < 2; side++) {
+                    const KV* src = (side == 0 ? krows : vrows) + (size_t)p * HD + v * 8;
+                    const float inv = pow2f(-(int)(side == 0 ? s_kx[p] : s_vx[p]));
+                    uint2 pk;
+                    pk.x = (unsigned)fp8_pack2(to_f(src[0]), to_f(src[1]), inv) | ((unsigned)fp8_pack2(to_f(src[2]), to_f(src[3]), inv) << 16);
+                    pk.y = (unsigned)fp8_pack2(to_f(src[4]), to_f(src[5]), inv) | ((unsigned)fp8_pack2(to_f(src[6]), to_f(src[7]), inv) << 16);
+                    *reinterpret_cast<uint2*>((side == 0 ? t.k8 : t.v8) + g * HD + v * 8) = pk;
+                    if (v == 0) (side == 0 ? t.k8e : t.v8e)[g] = side == 0 ? s_kx[p] : s_vx[p];
+                }
+            }
+        }
     }
     if (tid < c) {
         const int code = sc.rank[tid], tok = sc.tok[tid];

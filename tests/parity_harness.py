@@ -65,13 +65,34 @@ def log_ties(name: str, rep: "ParityReport") -> None:
 def make_ctx(cfg: WorkloadConfig, n_units: int, trace: int = 1, assign_mode: int = 0) -> P.DynaKV:
     return P.DynaKV(P.DynaKVConfig(
         n_units=n_units, gqa_group=cfg.G, head_dim=cfg.d,
-        kv_dtype=P.F32 if cfg.kv_dtype == "f32" else P.BF16,
+        kv_dtype={"f32": P.F32, "bf16": P.BF16, "fp8": P.FP8}[cfg.kv_dtype],
         max_tokens=cfg.max_tokens, max_clusters=cfg.max_clusters, kmeans_iters=cfg.T,
         init_mode=P.INIT_KMEANSPP if cfg.init_mode == "kmeanspp" else P.INIT_RANDOM,
         split_size_factor=cfg.split_size_factor, split_var_factor=cfg.split_var_factor,
         split_min_size=cfg.split_min_size, split_iters=cfg.split_iters, trace=trace, assign_mode=assign_mode,
         update_mode={"adaptive": P.MODE_ADAPTIVE, "static": P.MODE_STATIC, "local": P.MODE_LOCAL}[cfg.update_mode],
         local_max=cfg.local_max))
+
+
+def fp8_round_rows(x: "torch.Tensor") -> "torch.Tensor":
+    """Rows of x (last axis) as the FP8 storage mode keeps them: e4m3 elements (round to nearest even, largest finite
+    value 448) times one power-of-two scale per row, 2^e with e the smallest integer that brings the row's largest
+    magnitude to at most 448 (0 for a zero row).  Returned as float64.  The byte conversion is torch's own
+    float8_e4m3fn cast; only the scale rule is written out here."""
+    xf = x.to(torch.float64)
+    amax = xf.abs().amax(dim=-1, keepdim=True)
+    safe = torch.where(amax > 0, amax, torch.ones_like(amax))
+    e = torch.floor(torch.log2(safe)) - 8                    # 2^8 <= amax / 2^e < 2^9 up to log2's rounding ...
+    e = torch.where(safe / torch.exp2(e) > 448.0, e + 1, e)   # ... settled by testing the bound itself
+    e = torch.where(safe / torch.exp2(e - 1) <= 448.0, e - 1, e)
+    e = torch.where(amax > 0, e.clamp(-120, 120), torch.zeros_like(e))
+    scale = torch.exp2(e)
+    return (xf / scale).to(torch.float32).to(torch.float8_e4m3fn).to(torch.float64) * scale
+
+
+def stored(x: "torch.Tensor", cfg: WorkloadConfig) -> np.ndarray:
+    """The values the library keeps for rows x under cfg's storage type, as float64 (what the oracle is given)."""
+    return (fp8_round_rows(x) if cfg.kv_dtype == "fp8" else x.double()).numpy()
 
 
 def make_oracle(cfg: WorkloadConfig) -> O.OracleUnit:
@@ -132,7 +153,7 @@ def run_parity(cfg: WorkloadConfig, units: Sequence[int], steps: int, *, assign_
     oracles = {}
     for ui in watch:
         o = make_oracle(cfg)
-        o.build(K[ui].double().numpy(), V[ui].double().numpy(), cfg.M0, cfg.T, seed, unit_index=ui,
+        o.build(stored(K[ui], cfg), stored(V[ui], cfg), cfg.M0, cfg.T, seed, unit_index=ui,
                 init_mode=O.INIT_KMEANSPP if cfg.init_mode == "kmeanspp" else O.INIT_RANDOM,
                 hint_picks=picks[ui] if cfg.init_mode == "kmeanspp" else None, hint_assign=trace[:, ui, :])
         assert o.violations == 0, f"build unit {ui}: {o.violations} decisions differ beyond the tie tolerance"
@@ -171,7 +192,7 @@ def run_parity(cfg: WorkloadConfig, units: Sequence[int], steps: int, *, assign_
                 o = oracles[ui]
                 n0 = o.n
                 v0 = o.violations
-                j = o.append(k[t, ui].double().numpy(), v[t, ui].double().numpy(),
+                j = o.append(stored(k[t, ui], cfg), stored(v[t, ui], cfg),
                              hint_cluster=int(st["tok_cluster"][ui, n0]))
                 assert o.violations == v0 and j == int(st["tok_cluster"][ui, n0]), \
                     f"step {done + t} unit {ui}: append target gpu {st['tok_cluster'][ui, n0]} oracle {j}"

@@ -104,3 +104,52 @@ def test_tensor_core_assign_adversarial_keys():
     assert st["error_bits"] & P.ST_INTERNAL == 0 and st["assign_rechecked"] > 0
     print(f"\n[adversarial] ties followed {o.ties}, re-decided exactly {st['assign_rechecked']} of {n * T}")
     ctx.destroy()
+
+
+@pytest.mark.parametrize("cid,assign_mode", [(2, 1), (3, 1), (2, 0)])
+def test_fp8_storage(cid, assign_mode):
+    """FP8 storage of the K/V rows (the precision of Section 8.1's runs): the library is handed bf16 rows and keeps them
+    as e4m3 bytes with a power-of-two scale per row; the oracle is handed the same rows rounded by the test-side
+    quantiser.  Decisions, statistics and attention outputs then agree to the same bounds as in bf16 storage; config 3's
+    drifting stream makes clusters split, so rows also move between pages."""
+    base = CONFIGS[cid]
+    cfg = base.scaled(n_prefill=1111 if cid != 3 else 333, steps=96 if cid != 3 else 200, M0=37 if cid != 3 else 13,
+                      max_clusters=160, budget=300, T=6, new_every=32 if base.new_every else 0, kv_dtype="fp8")
+    rep = _run(cfg, [0, 1, 2], cfg.steps, assign_mode=assign_mode)
+    if cid == 3:
+        assert rep.splits > 0
+
+
+def test_fp8_storage_keeps_rows_on_the_grid_and_resumes():
+    """The rows an FP8 context exports are the handed-over rows rounded to the storage grid, bit for bit, also after
+    appends and splits; a context resumed from that export continues with the same outputs."""
+    import paper_2511_07427_b200 as P
+    from gen import UnitStream, make_prefill, make_decode_chunk
+    from parity_harness import fp8_round_rows, make_ctx
+    cfg = CONFIGS[3].scaled(n_prefill=333, steps=160, M0=13, max_clusters=160, budget=300, T=4, new_every=32, kv_dtype="fp8",
+                            split_size_factor=1.3)
+    U = 4
+    streams = [UnitStream(cfg, u) for u in range(U)]
+    K, V = make_prefill(streams)
+    q, k, v = make_decode_chunk(streams, cfg.steps)
+    ctx = make_ctx(cfg, U, trace=0, assign_mode=1)
+    ctx.build_index(K.cuda(), V.cuda(), cfg.M0, 7)
+    half = 100
+    qd, kd, vd = q.cuda(), k.cuda(), v.cuda()
+    for t in range(half):
+        ctx.decode_step(qd[t], cfg.budget); ctx.append(kd[t], vd[t]); ctx.split_check()
+    assert ctx.get_status()["n_splits"] > 0
+    n = cfg.n_prefill + half
+    Ke, Ve = ctx.export_kv(n)
+    K_all = torch.cat([K, k[:half].transpose(0, 1)], dim=1); V_all = torch.cat([V, v[:half].transpose(0, 1)], dim=1)
+    assert torch.equal(Ke.cpu().double(), fp8_round_rows(K_all)) and torch.equal(Ve.cpu().double(), fp8_round_rows(V_all))
+    st = ctx.export_state()
+    ctx2 = make_ctx(cfg, U, trace=0, assign_mode=1)
+    ctx2.import_state(Ke, Ve, st["tok_cluster"][:, :n], st["n_ids"], st["tau"], cfg.M0)
+    for t in range(half, cfg.steps):
+        a = ctx.decode_step(qd[t], cfg.budget).clone(); b = ctx2.decode_step(qd[t], cfg.budget).clone()
+        assert (a - b).abs().max().item() <= 2e-3
+        for c in (ctx, ctx2):
+            c.append(kd[t], vd[t]); c.split_check()
+    assert np.array_equal(ctx.export_state()["tok_cluster"], ctx2.export_state()["tok_cluster"])
+    ctx.destroy(); ctx2.destroy()
