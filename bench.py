@@ -290,7 +290,7 @@ def run_ours(args, cfg):
     torch.cuda.synchronize()
 
     ctx = P.DynaKV(P.DynaKVConfig(
-        n_units=U, gqa_group=cfg.G, head_dim=cfg.d, kv_dtype=P.F32 if cfg.kv_dtype == "f32" else P.BF16,
+        n_units=U, gqa_group=cfg.G, head_dim=cfg.d, kv_dtype={"f32": P.F32, "bf16": P.BF16, "fp8": P.FP8}[cfg.kv_dtype],
         max_tokens=cfg.max_tokens, max_clusters=cfg.max_clusters, kmeans_iters=cfg.T,
         init_mode=P.INIT_KMEANSPP if cfg.init_mode == "kmeanspp" else P.INIT_RANDOM,
         split_size_factor=cfg.split_size_factor, split_var_factor=cfg.split_var_factor,
@@ -352,11 +352,12 @@ def run_ours(args, cfg):
     ctx.set_timing(False)
     tok1 = ctx.get_status()["tokens_attended_total"]
     pos += n_prof
-    bytes_kv = 4 if cfg.kv_dtype == "f32" else 2
+    # bytes the kernel must read per attended row: K and V rows, in FP8 storage one byte per element and a scale byte each
+    row_bytes = {"f32": 8 * cfg.d, "bf16": 4 * cfg.d, "fp8": 2 * cfg.d + 2}[cfg.kv_dtype]
     attn_ms_each = kt["attn"]["ms"] / max(kt["attn"]["launches"], 1)      # an event pair around every launch
     attn_ms, attn_how, tokens_per_launch = attn_ms_each, "CUDA events around every launch of %d direct-call steps" % n_prof, \
         (tok1 - tok0) / max(n_prof, 1)
-    if cfg.kv_dtype == "bf16" and n_prof > 0:
+    if cfg.kv_dtype != "f32" and n_prof > 0:
         # the kernel alone: 50 back-to-back ordinary launches on one selection between two events (the step's rows,
         # 267 MB in config 4, are more than twice the L2, so every launch streams from HBM)
         ctx.decode_step(q_all[pos - 1], cfg.budget, out=out_all[pos - 1])
@@ -364,7 +365,7 @@ def run_ours(args, cfg):
         attn_ms = ctx.time_gather_attention(q_all[pos - 1], out_all[pos - 1], 50)
         tokens_per_launch = float(ntok_sel.sum())
         attn_how = "two CUDA events around 50 back-to-back launches on one step's selection (one untimed launch first)"
-    attn_bytes = tokens_per_launch * 2 * cfg.d * bytes_kv + 2 * U * cfg.G * cfg.d * 4
+    attn_bytes = tokens_per_launch * row_bytes + 2 * U * cfg.G * cfg.d * 4
     achieved = attn_bytes / (attn_ms * 1e-3) / 1e9 if attn_ms > 0 else 0.0
     kernels = {k: (v["ms"] / v["launches"] * 1e3 if v["launches"] else None) for k, v in kt.items()
                if k in ("front", "select", "attn", "combine", "append", "split")}
@@ -423,7 +424,7 @@ def run_ours(args, cfg):
             ctx.step_host(qh[t], kh[t], vh[t], cfg.budget, oh)
         torch.cuda.synchronize()
         dt_sync = max_over_ranks(time.perf_counter() - t0, dev)
-        h2d = int(qh[0].numel() * 4 + 2 * kh[0].numel() * bytes_kv)
+        h2d = int(qh[0].numel() * 4 + 2 * kh[0].numel() * kh.element_size())
         d2h = int(oh.numel() * 4)
         e2e = {"value": None, "unit": "steps/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                "call": "dynakv_decode_loop_host", "steps": n_loop,
@@ -464,7 +465,8 @@ def run_ours(args, cfg):
         line = {
             "metric": METRIC, "value": value, "unit": "steps/s", "n_gpus": world, "steps": K_steps, "warmup": W,
             "ms_per_step": ms / K_steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-            "dtype": "f32" if cfg.kv_dtype == "f32" else "bf16 KV / f32 math", "data": "synthetic",
+            "dtype": {"f32": "f32", "bf16": "bf16 KV / f32 math", "fp8": "fp8 (e4m3, scale per row) KV / f32 math"}[cfg.kv_dtype],
+            "data": "synthetic",
             "config": config_dict(cfg, W),
             "e2e": e2e, "gpu_launches": int(gpu_launches), "clocks": clocks, "roofline": roofline,
             "cpu_baseline": cpu_baseline, "build": build,
@@ -491,6 +493,7 @@ def main():
     ap.add_argument("--config", type=int, default=4)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--assign-mode", type=int, default=0)
+    ap.add_argument("--kv", default="", choices=["", "fp8"], help="fp8: the config's bf16 K/V rows kept in FP8 storage")
     ap.add_argument("--e2e-steps", type=int, default=160)
     ap.add_argument("--profile-steps", type=int, default=64)
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -507,6 +510,9 @@ def main():
         cfg = cfg.scaled(B=1, L=1, Hkv=args.units, Hq=args.units * cfg.G, name=cfg.name + f"[first {args.units} units]")
     if args.budget > 0:
         cfg = cfg.scaled(budget=args.budget, name=cfg.name + f"[budget {args.budget}]")
+    if args.kv == "fp8":
+        assert cfg.kv_dtype == "bf16" and cfg.d == 128, "FP8 storage is for the bf16 configurations with d = 128"
+        cfg = cfg.scaled(kv_dtype="fp8", name=cfg.name + "[fp8 K/V]")
     if args.impl == "reference":
         run_reference(args, cfg)
     else:

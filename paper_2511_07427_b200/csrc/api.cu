@@ -332,7 +332,7 @@ static void enqueue_retrieve(dynakv_ctx* c, StepPtr q, int budget, StepPtrW out,
 }
 
 static void enqueue_attend(dynakv_ctx* c, StepPtr q, StepPtrW out, bool timed) {
-    if (c->t.kv_dtype == DYNAKV_BF16 && c->cfg.attn_mode == 0 && !c->t.fp8) {
+    if (c->t.kv_dtype == DYNAKV_BF16 && c->cfg.attn_mode == 0) {
         // gather, attend and combine in one persistent kernel
         TimeScope ts(c, KC_ATTN, timed);
         launch_gather_attn_tma(c->t, q, out, c->stream, &c->launches);
@@ -731,7 +731,7 @@ extern "C" int dynakv_selftest_wait_expiry(dynakv_ctx* c, int32_t* gave_up) {
 extern "C" int dynakv_time_gather_attention(dynakv_ctx* c, const float* q, float* out, int32_t reps, float* ms_per_launch) {
     if (!c || !q || !out || !ms_per_launch || reps < 1) return DYNAKV_ERR_ARG;
     if (!c->built) return DYNAKV_ERR_STATE;
-    if (c->t.kv_dtype != DYNAKV_BF16 || c->cfg.attn_mode != 0 || c->t.fp8) return DYNAKV_ERR_ARG;
+    if (c->t.kv_dtype != DYNAKV_BF16 || c->cfg.attn_mode != 0) return DYNAKV_ERR_ARG;
     cudaEvent_t e0, e1;
     CK(cudaEventCreate(&e0)); CK(cudaEventCreate(&e1));
     const StepPtr qp{q, 0, nullptr};

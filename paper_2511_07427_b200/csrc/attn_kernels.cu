@@ -23,10 +23,20 @@
 // written by that CTA.  A unit cut by slice boundaries leaves one unnormalised partial per
 // CTA; each such CTA bumps the unit's arrival counter and the last one to arrive merges
 // the partials and writes the output, so no CTA ever waits for another.
+//
+// FP8 storage (F8 = true, d = 128): the producer streams the one-byte copy of the pages -- e4m3 rows of 128 bytes and the
+// rows' scale exponents -- so a row costs 258 bytes instead of 512.  The consumers turn the bytes into f16 operands
+// (exact: e4m3 has four significant bits) with the paired conversion instruction and use f16 MMAs; Q, divided by a
+// power of two per head so that it fits f16 whatever its size, and the softmax weights are split into f16 hi + lo
+// parts.  A K row's scale multiplies its logit; a V row's scale 2^e is folded into the softmax: the running maximum is
+// kept over (logit + e), the MMA weight is 2^(logit + e - max) <= 1 and the denominator adds that weight times 2^-e,
+// so numerator and denominator carry the same factor and every merge below works unchanged.
+#include <cuda_fp16.h>
 #include <float.h>
 
 #include "bulk_copy.cuh"
 #include "common.cuh"
+#include "fp8_rows.cuh"
 
 namespace dkv {
 
@@ -46,6 +56,35 @@ __device__ __forceinline__ void split2(float x, float y, unsigned& hi, unsigned&
     lo = (unsigned)__bfloat16_as_ushort(xl) | ((unsigned)__bfloat16_as_ushort(yl) << 16);
 }
 
+__device__ __forceinline__ void mma_f16(float (&c)[4], unsigned a0, unsigned a1, unsigned a2, unsigned a3,
+                                        unsigned b0, unsigned b1) {
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"
+        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+// (hi, lo) f16 split of two floats in [-1, 1], packed as f16x2 (first value in the low half).
+__device__ __forceinline__ void split2h(float x, float y, unsigned& hi, unsigned& lo) {
+    const __half2 h = __floats2half2_rn(x, y);
+    const float2 hf = __half22float2(h);
+    const __half2 l = __floats2half2_rn(x - hf.x, y - hf.y);
+    hi = *reinterpret_cast<const unsigned*>(&h);
+    lo = *reinterpret_cast<const unsigned*>(&l);
+}
+
+// Four e4m3 bytes as two f16x2 registers: lo from bytes 0 and 1, hi from bytes 2 and 3.
+__device__ __forceinline__ void e4m3x4_to_f16x2(unsigned b, unsigned& lo, unsigned& hi) {
+    asm("{\n .reg .b16 l, h;\n mov.b32 {l, h}, %2;\n cvt.rn.f16x2.e4m3x2 %0, l;\n cvt.rn.f16x2.e4m3x2 %1, h;\n}\n"
+        : "=r"(lo), "=r"(hi) : "r"(b));
+}
+
+__device__ __forceinline__ int lds_s8x2(unsigned addr) {      // two signed bytes: low byte in .x of the result pair
+    unsigned short v;
+    asm volatile("ld.shared.u16 %0, [%1];\n" : "=h"(v) : "r"(addr));
+    return (int)v;
+}
+
 __device__ __forceinline__ uint4 lds16(unsigned addr) {
     uint4 v;
     asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];\n" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
@@ -61,18 +100,26 @@ __device__ __forceinline__ uint4 lds16(unsigned addr) {
 constexpr int AT_CONSUMERS = DKV_AT_CONSUMERS;      // consumer warps
 constexpr int AT_THREADS = (AT_CONSUMERS + 1) * 32; // + one producer warp
 constexpr int AT_STAGES = DKV_AT_STAGES;                      // work entries (runs of <= ENTRY_ROWS rows) in flight per CTA
-// Item i of a CTA's slice is consumed by warp i % AT_CONSUMERS from ring stage i % AT_STAGES.  A stage
+#ifndef DKV_AT_STAGES_F8
+#define DKV_AT_STAGES_F8 9
+#endif
+constexpr int AT_STAGES_F8 = DKV_AT_STAGES_F8;                // the same for the one-byte rows (stages half the size)
+// Item i of a CTA's slice is consumed by warp i % AT_CONSUMERS from ring stage i % stages.  A stage
 // must always be consumed by the same warp: a parity wait cannot tell phase p from phase p + 2, so a
 // warp must never be able to run two phases ahead of another warp on a shared stage.
 static_assert(AT_STAGES <= 32 && AT_STAGES % AT_CONSUMERS == 0, "each ring stage belongs to one consumer warp");
+static_assert(AT_STAGES_F8 <= 32 && AT_STAGES_F8 % AT_CONSUMERS == 0, "each ring stage belongs to one consumer warp");
 
 __device__ __forceinline__ void consumer_sync() { asm volatile("bar.sync 1, %0;\n" ::"n"(AT_CONSUMERS * 32) : "memory"); }
 
-template <int HD> struct AttnSmem {
-    static constexpr int stage_bytes = 2 * ENTRY_ROWS * HD * 2;                 // K rows then V rows of one entry
-    static constexpr int ring_bytes = AT_STAGES * stage_bytes;
+template <int HD, bool F8> struct AttnSmem {
+    static constexpr int stages = F8 ? AT_STAGES_F8 : AT_STAGES;
+    static constexpr int row_bytes = F8 ? HD : HD * 2;
+    // K rows then V rows of one entry; FP8: then the K rows' and the V rows' scale exponents (ENTRY_ROWS bytes each)
+    static constexpr int stage_bytes = 2 * ENTRY_ROWS * row_bytes + (F8 ? 128 : 0);
+    static constexpr int ring_bytes = stages * stage_bytes;
     static constexpr int merge_bytes = AT_CONSUMERS * 8 * (HD + 2) * 4;   // per warp: acc[8][HD], m[8], l[8]
-    static constexpr int fixed_bytes = ring_bytes + merge_bytes + 2 * AT_STAGES * 8 + AT_STAGES * 4 + 64;
+    static constexpr int fixed_bytes = ring_bytes + merge_bytes + 2 * stages * 8 + stages * 4 + 64;
 };
 
 // Smallest u with pf[u+1] > k, starting the search at u0 (pf non-decreasing).
@@ -92,17 +139,20 @@ __device__ __forceinline__ int unit_of_bisect(const int* pf, int U, int k) {
     return a;
 }
 
-template <int HD>
+template <int HD, bool F8>
 __global__ void __launch_bounds__(AT_THREADS, 2) k_gather_attn_tma(Tables t, StepPtr qp, StepPtrW outp) {
+    static_assert(!F8 || HD == 128, "the one-byte rows are kept for d = 128");
+    using SM = AttnSmem<HD, F8>;
+    constexpr int AT_STAGES = SM::stages;
     constexpr int KS = HD / 16;       // k-steps of Q.K^T
-    constexpr int KJ = KS / 2;        // 16-byte chunks a thread loads per K row
+    constexpr int KJ = F8 ? KS / 4 : KS / 2;   // 16-byte chunks a thread loads per K row
     constexpr int NT = HD / 8;        // n-tiles of P.V
-    constexpr int VI = HD / 64;       // 16-byte chunks a thread loads per V row
-    constexpr int ROWB = HD * 2;      // bytes per K or V row
+    constexpr int VI = F8 ? 1 : HD / 64;       // 16-byte chunks a thread loads per V row
+    constexpr int ROWB = SM::row_bytes;        // bytes per K or V row
     extern __shared__ __align__(128) unsigned char smem[];
     unsigned char* ring = smem;
-    float* mrg = reinterpret_cast<float*>(smem + AttnSmem<HD>::ring_bytes);
-    unsigned long long* bars = reinterpret_cast<unsigned long long*>(smem + AttnSmem<HD>::ring_bytes + AttnSmem<HD>::merge_bytes);
+    float* mrg = reinterpret_cast<float*>(smem + SM::ring_bytes);
+    unsigned long long* bars = reinterpret_cast<unsigned long long*>(smem + SM::ring_bytes + SM::merge_bytes);
     int* meta = reinterpret_cast<int*>(bars + 2 * AT_STAGES);
     int* s_flag = meta + AT_STAGES;                  // [0] abort, [1] combine-here, [2..] warp totals of the prefix scan
     int* pf_s = s_flag + 16;                         // the units' work-list prefix when it fits
@@ -162,10 +212,10 @@ __global__ void __launch_bounds__(AT_THREADS, 2) k_gather_attn_tma(Tables t, Ste
         // Lane j owns ring stage j: it fetches the work entries of items j, j + AT_STAGES, ... and issues
         // their copies as soon as the stage's consumer has released it, independently of the other lanes.
         if (lane < AT_STAGES && lane < n_items) {
-            const __nv_bfloat16* kp = reinterpret_cast<const __nv_bfloat16*>(t.kpages);
-            const __nv_bfloat16* vp = reinterpret_cast<const __nv_bfloat16*>(t.vpages);
+            const unsigned char* kp = F8 ? t.k8 : reinterpret_cast<const unsigned char*>(t.kpages);
+            const unsigned char* vp = F8 ? t.v8 : reinterpret_cast<const unsigned char*>(t.vpages);
             const unsigned full = smem_u32(&bars[lane]), empty = smem_u32(&bars[AT_STAGES + lane]);
-            const unsigned dst = smem_u32(ring + (size_t)lane * AttnSmem<HD>::stage_bytes);
+            const unsigned dst = smem_u32(ring + (size_t)lane * SM::stage_bytes);
             int u = unit_of_bisect(pf, U, lo + lane);
             int2 ent = work[(size_t)u * t.W + (lo + lane - pf[u])];
             int last_issued = -1;
@@ -179,11 +229,17 @@ __global__ void __launch_bounds__(AT_THREADS, 2) k_gather_attn_tma(Tables t, Ste
                 const unsigned ph = (unsigned)(it / AT_STAGES) & 1u;
                 if (!mbar_wait(empty, ph ^ 1u)) { s_flag[0] = 1; break; }
                 const unsigned bytes = (unsigned)cur.y * ROWB;
-                const size_t src = ((size_t)cu * t.P * PAGE + cur.x) * HD;
+                const size_t row0 = (size_t)cu * t.P * PAGE + cur.x;
+                const size_t src = row0 * ROWB;
                 meta[lane] = cur.y;
-                mbar_arrive_expect_tx(full, 2 * bytes);
+                mbar_arrive_expect_tx(full, 2 * bytes + (F8 ? 2 * ENTRY_ROWS : 0));
                 bulk_g2s(dst, kp + src, bytes, full);
                 bulk_g2s(dst + ENTRY_ROWS * ROWB, vp + src, bytes, full);
+                if constexpr (F8) {
+                    // the run's scale exponents: first row a multiple of ENTRY_ROWS, so source and size are multiples of 16
+                    bulk_g2s(dst + 2 * ENTRY_ROWS * ROWB, t.k8e + row0, ENTRY_ROWS, full);
+                    bulk_g2s(dst + 2 * ENTRY_ROWS * ROWB + ENTRY_ROWS, t.v8e + row0, ENTRY_ROWS, full);
+                }
                 last_issued = it;
             }
             if (*(volatile int*)&s_flag[0]) {
@@ -214,6 +270,31 @@ __global__ void __launch_bounds__(AT_THREADS, 2) k_gather_attn_tma(Tables t, Ste
         // ---- Q fragments of unit u: rows 0..7 = hi part of head r, rows 8..15 = lo part of head r
         const float* q = qbase + (size_t)u * G * HD;
         unsigned qa[KS][4];
+        float head_scale = 0.f;          // FP8: what a logit of head r is multiplied by besides the K row's scale
+        if constexpr (F8) {
+            // k-step ks takes elements 16 (c + 4 (ks / 4)) + 4 (ks % 4) .. + 3: the 16 bytes a thread loads from a K row
+            // are its B fragments of four k-steps.  Head r is divided by 2^ex, ex the exponent of its largest magnitude.
+            float4 qv[KS];
+            float amax = 0.f;
+#pragma unroll
+            for (int ks = 0; ks < KS; ks++) {
+                const int base = 16 * (c + 4 * (ks >> 2)) + 4 * (ks & 3);
+                qv[ks] = r < G ? *reinterpret_cast<const float4*>(q + r * HD + base) : make_float4(0.f, 0.f, 0.f, 0.f);
+                amax = fmaxf(fmaxf(amax, fmaxf(fabsf(qv[ks].x), fabsf(qv[ks].y))), fmaxf(fabsf(qv[ks].z), fabsf(qv[ks].w)));
+            }
+            amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 1));
+            amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 2));
+            int ex = 0;
+            if (amax > 0.f && amax < INFINITY) frexpf(amax, &ex);
+            ex = max(-100, min(100, ex));
+            const float inv = pow2f(-ex);
+            head_scale = pow2f(ex) * scale;
+#pragma unroll
+            for (int ks = 0; ks < KS; ks++) {
+                split2h(qv[ks].x * inv, qv[ks].y * inv, qa[ks][0], qa[ks][1]);
+                split2h(qv[ks].z * inv, qv[ks].w * inv, qa[ks][2], qa[ks][3]);
+            }
+        } else {
 #pragma unroll
         for (int ks = 0; ks < KS; ks++) {
             const int base = 8 * (c + 4 * (ks >> 1)) + 4 * (ks & 1);
@@ -224,6 +305,7 @@ __global__ void __launch_bounds__(AT_THREADS, 2) k_gather_attn_tma(Tables t, Ste
             }
             split2(x0, x1, qa[ks][0], qa[ks][1]);
             split2(x2, x3, qa[ks][2], qa[ks][3]);
+        }
         }
         float o[NT][4];
 #pragma unroll
@@ -238,30 +320,125 @@ __global__ void __launch_bounds__(AT_THREADS, 2) k_gather_attn_tma(Tables t, Ste
             const unsigned ph = (unsigned)(it / AT_STAGES) & 1u;
             if (!mbar_wait(smem_u32(&bars[stage]), ph)) { s_flag[0] = 1; dead = true; break; }
             const int rows = meta[stage];
-            const unsigned kbase = smem_u32(ring + (size_t)stage * AttnSmem<HD>::stage_bytes);
+            const unsigned kbase = smem_u32(ring + (size_t)stage * SM::stage_bytes);
             const unsigned vbase = kbase + ENTRY_ROWS * ROWB;
 #pragma unroll 1
             for (int sub = 0; sub < ENTRY_ROWS / 16; sub++) {
                 const int nvalid = rows - sub * 16;
                 if (nvalid <= 0) break;
                 const unsigned krow0 = kbase + (unsigned)(sub * 16) * ROWB, vrow0 = vbase + (unsigned)(sub * 16) * ROWB;
-                // ---- loads: K rows (tile*8 + r), chunks c + 4j; V rows 2c, 2c+1, 2c+8, 2c+9, chunks r + 8i
+                if constexpr (F8) {
+                // ---- loads: K rows (tile*8 + r), chunks c + 4j; V rows 2c, 2c+1, 2c+8, 2c+9, chunk r; the scale exponents
+                // of this thread's four tokens (tile*8 + 2c, + 1)
+                // (rows past the run's end are read from its last row instead: their logits are masked and their weights
+                // are zero, so all they must be is finite)
                 uint4 kw[2][KJ];
 #pragma unroll
                 for (int tile = 0; tile < 2; tile++) {
-                    const bool ok = tile * 8 + r < nvalid;
+                    const unsigned row = (unsigned)min(tile * 8 + r, nvalid - 1);
 #pragma unroll
-                    for (int j = 0; j < KJ; j++)
-                        kw[tile][j] = ok ? lds16(krow0 + (unsigned)(tile * 8 + r) * ROWB + 16u * (c + 4 * j)) : make_uint4(0, 0, 0, 0);
+                    for (int j = 0; j < KJ; j++) kw[tile][j] = lds16(krow0 + row * ROWB + 16u * (c + 4 * j));
+                }
+                uint4 vw[4];
+#pragma unroll
+                for (int rr = 0; rr < 4; rr++) {
+                    const unsigned tok = (unsigned)min(2 * c + (rr & 1) + 8 * (rr >> 1), nvalid - 1);
+                    vw[rr] = lds16(vrow0 + tok * ROWB + 16u * r);
+                }
+                const unsigned xbase = kbase + 2 * ENTRY_ROWS * ROWB + (unsigned)(sub * 16);
+                int kx[4], vx[4];
+#pragma unroll
+                for (int tile = 0; tile < 2; tile++) {
+                    const int kp2 = lds_s8x2(xbase + tile * 8 + 2 * c), vp2 = lds_s8x2(xbase + ENTRY_ROWS + tile * 8 + 2 * c);
+                    kx[tile * 2] = (int)(signed char)(kp2 & 0xff); kx[tile * 2 + 1] = (int)(signed char)(kp2 >> 8);
+                    vx[tile * 2] = (int)(signed char)(vp2 & 0xff); vx[tile * 2 + 1] = (int)(signed char)(vp2 >> 8);
+                }
+                // ---- S = Q K^T for the two 8-token tiles: word w of chunk j holds the B fragments of k-step 4j + w
+                float sc[2][4];
+#pragma unroll
+                for (int tile = 0; tile < 2; tile++) {
+                    sc[tile][0] = 0.f; sc[tile][1] = 0.f; sc[tile][2] = 0.f; sc[tile][3] = 0.f;
+#pragma unroll
+                    for (int j = 0; j < KJ; j++) {
+                        const unsigned* w4 = reinterpret_cast<const unsigned*>(&kw[tile][j]);
+#pragma unroll
+                        for (int w = 0; w < 4; w++) {
+                            const int ks = 4 * j + w;
+                            unsigned b0, b1;
+                            e4m3x4_to_f16x2(w4[w], b0, b1);
+                            mma_f16(sc[tile], qa[ks][0], qa[ks][1], qa[ks][2], qa[ks][3], b0, b1);
+                        }
+                    }
+                }
+                // logits of head r (hi row + lo row) times the head's and the K row's scales; for the softmax the V row's
+                // exponent is added
+                float lg[4];
+#pragma unroll
+                for (int tile = 0; tile < 2; tile++) {
+                    const int tok = tile * 8 + 2 * c;
+#pragma unroll
+                    for (int h = 0; h < 2; h++) {
+                        const int e = tile * 2 + h;
+                        const bool ok = tok + h < nvalid;
+                        if (!ok) { kx[e] = 0; vx[e] = 0; }
+                        lg[e] = ok ? (sc[tile][h] + sc[tile][2 + h]) * head_scale * pow2f(kx[e]) + (float)vx[e] : -INFINITY;
+                    }
+                }
+                float mx = fmaxf(fmaxf(lg[0], lg[1]), fmaxf(lg[2], lg[3]));
+                mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+                mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+                // the reference point of the exponentials follows the running maximum lazily: it moves only when the maximum
+                // has grown by more than 2^8, so weights stay below 2^8 and the accumulators are rarely rescaled
+                const float mn = mx > m + 8.f ? mx : m;        // finite: row 0 of the entry is valid
+                const float corr = exp2f(m - mn);
+                m = mn;
+                float p[4];
+#pragma unroll
+                for (int e = 0; e < 4; e++) p[e] = exp2f(lg[e] - mn);
+                l = l * corr + (p[0] * pow2f(-vx[0]) + p[1] * pow2f(-vx[1])) + (p[2] * pow2f(-vx[2]) + p[3] * pow2f(-vx[3]));
+                unsigned pa[4];
+                split2h(p[0], p[1], pa[0], pa[1]);   // a0 = hi(tile 0), a1 = lo(tile 0)
+                split2h(p[2], p[3], pa[2], pa[3]);   // a2 = hi(tile 1), a3 = lo(tile 1)
+                if (__any_sync(0xffffffffu, corr != 1.f)) {
+#pragma unroll
+                    for (int x = 0; x < NT; x++) { o[x][0] *= corr; o[x][1] *= corr; o[x][2] *= corr; o[x][3] *= corr; }
+                }
+                // ---- O += P V : n-tile e takes byte e of the chunk of the thread's four rows (column 16 r + e)
+                const unsigned* a0 = reinterpret_cast<const unsigned*>(&vw[0]);
+                const unsigned* a1 = reinterpret_cast<const unsigned*>(&vw[1]);
+                const unsigned* a2 = reinterpret_cast<const unsigned*>(&vw[2]);
+                const unsigned* a3 = reinterpret_cast<const unsigned*>(&vw[3]);
+#pragma unroll
+                for (int w = 0; w < 4; w++) {
+#pragma unroll
+                    for (int h = 0; h < 2; h++) {
+                        // bytes (2h, 2h+1) of word w of two rows, interleaved: row A byte, row B byte, row A next, row B next
+                        const unsigned sel = h ? 0x7362u : 0x5140u;
+                        const unsigned t01 = __byte_perm(a0[w], a1[w], sel), t23 = __byte_perm(a2[w], a3[w], sel);
+                        unsigned b0e, b0o, b1e, b1o;      // even / odd byte of the pair
+                        e4m3x4_to_f16x2(t01, b0e, b0o);
+                        e4m3x4_to_f16x2(t23, b1e, b1o);
+                        mma_f16(o[4 * w + 2 * h], pa[0], pa[1], pa[2], pa[3], b0e, b1e);
+                        mma_f16(o[4 * w + 2 * h + 1], pa[0], pa[1], pa[2], pa[3], b0o, b1o);
+                    }
+                }
+                } else {
+                // ---- loads: K rows (tile*8 + r), chunks c + 4j; V rows 2c, 2c+1, 2c+8, 2c+9, chunks r + 8i
+                uint4 kw[2][KJ];
+#pragma unroll
+                // (rows past the run's end are read from its last row instead: their logits are masked and their weights
+                // are zero, so all they must be is finite)
+                for (int tile = 0; tile < 2; tile++) {
+                    const unsigned row = (unsigned)min(tile * 8 + r, nvalid - 1);
+#pragma unroll
+                    for (int j = 0; j < KJ; j++) kw[tile][j] = lds16(krow0 + row * ROWB + 16u * (c + 4 * j));
                 }
                 uint4 vw[4][VI];
 #pragma unroll
                 for (int rr = 0; rr < 4; rr++) {
-                    const int tok = 2 * c + (rr & 1) + 8 * (rr >> 1);
-                    const bool ok = tok < nvalid;
+                    const unsigned tok = (unsigned)min(2 * c + (rr & 1) + 8 * (rr >> 1), nvalid - 1);
 #pragma unroll
-                    for (int i = 0; i < VI; i++)
-                        vw[rr][i] = ok ? lds16(vrow0 + (unsigned)tok * ROWB + 16u * (r + 8 * i)) : make_uint4(0, 0, 0, 0);
+                    for (int i = 0; i < VI; i++) vw[rr][i] = lds16(vrow0 + tok * ROWB + 16u * (r + 8 * i));
                 }
                 // ---- S = Q K^T for the two 8-token tiles
                 float sc[2][4];
@@ -285,7 +462,9 @@ __global__ void __launch_bounds__(AT_THREADS, 2) k_gather_attn_tma(Tables t, Ste
                 float mx = fmaxf(fmaxf(lg[0], lg[1]), fmaxf(lg[2], lg[3]));
                 mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
                 mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
-                const float mn = fmaxf(m, mx);                 // finite: row 0 of the entry is valid
+                // the reference point of the exponentials follows the running maximum lazily: it moves only when the maximum
+                // has grown by more than 2^8, so weights stay below 2^8 and the accumulators are rarely rescaled
+                const float mn = mx > m + 8.f ? mx : m;        // finite: row 0 of the entry is valid
                 const float corr = exp2f(m - mn);
                 m = mn;
                 float p[4];
@@ -314,6 +493,7 @@ __global__ void __launch_bounds__(AT_THREADS, 2) k_gather_attn_tma(Tables t, Ste
                         mma_bf16(o[i * 8 + e], pa[0], pa[1], pa[2], pa[3], b0, b1);
                     }
                 }
+                }
             }
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(&bars[AT_STAGES + stage]));
@@ -325,9 +505,14 @@ __global__ void __launch_bounds__(AT_THREADS, 2) k_gather_attn_tma(Tables t, Ste
         if (c == 0) { mrg_m[cw * 8 + r] = m; mrg_l[cw * 8 + r] = l; }
 #pragma unroll
         for (int x = 0; x < NT; x++) {
+            if constexpr (F8) {           // n-tile x, accumulator columns 2c and 2c+1: output columns 16 (2c) + x and 16 (2c+1) + x
+                mrg_o[(cw * 8 + r) * HD + 16 * (2 * c) + x] = o[x][0] + o[x][2];
+                mrg_o[(cw * 8 + r) * HD + 16 * (2 * c + 1) + x] = o[x][1] + o[x][3];
+            } else {
             const int i = x >> 3, e = x & 7;
             mrg_o[(cw * 8 + r) * HD + 8 * (2 * c + 8 * i) + e] = o[x][0] + o[x][2];
             mrg_o[(cw * 8 + r) * HD + 8 * (2 * c + 1 + 8 * i) + e] = o[x][1] + o[x][3];
+            }
         }
         consumer_sync();
         if (*(volatile int*)&s_flag[0] || dead) {
@@ -471,30 +656,32 @@ void launch_selftest_wait_expiry(const Tables& t, int* gave_up, cudaStream_t s, 
 }
 
 size_t attn_tma_smem_bytes(const Tables& t) {
-    const size_t fixed = t.d == 64 ? AttnSmem<64>::fixed_bytes : AttnSmem<128>::fixed_bytes;
+    const size_t fixed = t.fp8 ? AttnSmem<128, true>::fixed_bytes : t.d == 64 ? AttnSmem<64, false>::fixed_bytes : AttnSmem<128, false>::fixed_bytes;
     return fixed + (t.attn_pf_in_smem ? (size_t)(t.U + 1) * 4 : 0) + 64;
 }
 
 int attn_tma_prepare(const Tables& t) {
     const int bytes = (int)attn_tma_smem_bytes(t);
-    cudaError_t e = t.d == 64
-        ? cudaFuncSetAttribute(k_gather_attn_tma<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes)
-        : cudaFuncSetAttribute(k_gather_attn_tma<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+    cudaError_t e = t.fp8 ? cudaFuncSetAttribute(k_gather_attn_tma<128, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes)
+        : t.d == 64 ? cudaFuncSetAttribute(k_gather_attn_tma<64, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes)
+        : cudaFuncSetAttribute(k_gather_attn_tma<128, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
     return e == cudaSuccess ? 0 : -1;
 }
 
 // The same kernel as an ordinary launch (no programmatic dependence on its neighbours): for timing it alone.
 void launch_gather_attn_plain(const Tables& t, StepPtr q, StepPtrW out, cudaStream_t s, long long* launches) {
     const size_t bytes = attn_tma_smem_bytes(t);
-    if (t.d == 64) k_gather_attn_tma<64><<<t.n_attn_ctas, AT_THREADS, bytes, s>>>(t, q, out);
-    else k_gather_attn_tma<128><<<t.n_attn_ctas, AT_THREADS, bytes, s>>>(t, q, out);
+    if (t.fp8) k_gather_attn_tma<128, true><<<t.n_attn_ctas, AT_THREADS, bytes, s>>>(t, q, out);
+    else if (t.d == 64) k_gather_attn_tma<64, false><<<t.n_attn_ctas, AT_THREADS, bytes, s>>>(t, q, out);
+    else k_gather_attn_tma<128, false><<<t.n_attn_ctas, AT_THREADS, bytes, s>>>(t, q, out);
     (*launches)++;
 }
 
 void launch_gather_attn_tma(const Tables& t, StepPtr q, StepPtrW out, cudaStream_t s, long long* launches) {
     const size_t bytes = attn_tma_smem_bytes(t);
-    if (t.d == 64) launch_pdl(k_gather_attn_tma<64>, dim3(t.n_attn_ctas), dim3(AT_THREADS), bytes, s, t, q, out);
-    else launch_pdl(k_gather_attn_tma<128>, dim3(t.n_attn_ctas), dim3(AT_THREADS), bytes, s, t, q, out);
+    if (t.fp8) launch_pdl(k_gather_attn_tma<128, true>, dim3(t.n_attn_ctas), dim3(AT_THREADS), bytes, s, t, q, out);
+    else if (t.d == 64) launch_pdl(k_gather_attn_tma<64, false>, dim3(t.n_attn_ctas), dim3(AT_THREADS), bytes, s, t, q, out);
+    else launch_pdl(k_gather_attn_tma<128, false>, dim3(t.n_attn_ctas), dim3(AT_THREADS), bytes, s, t, q, out);
     (*launches)++;
 }
 

@@ -59,23 +59,8 @@ def test_more_than_1024_units_keep_the_work_prefix_in_global_memory():
 
 
 def test_plain_attention_kernel_on_bf16():
-    cfg = CONFIGS[5].scaled(B=1, L=1, n_prefill=600, steps=16, M0=24, max_clusters=64, budget=200, T=3)
-    from parity_harness import make_ctx
-    import parity_harness as H
-    orig = H.make_ctx
-
-    def forced(cfg_, n_units, trace=1, assign_mode=0):
-        c = P.DynaKVConfig(n_units=n_units, gqa_group=cfg_.G, head_dim=cfg_.d, kv_dtype=P.BF16, max_tokens=cfg_.max_tokens,
-                           max_clusters=cfg_.max_clusters, kmeans_iters=cfg_.T, init_mode=P.INIT_RANDOM,
-                           split_size_factor=cfg_.split_size_factor, split_var_factor=cfg_.split_var_factor,
-                           split_min_size=cfg_.split_min_size, split_iters=cfg_.split_iters, trace=trace, assign_mode=1,
-                           attn_mode=1)
-        return P.DynaKV(c)
-    H.make_ctx = forced
-    try:
-        _run(cfg, [0, 1, 2, 3], cfg.steps)
-    finally:
-        H.make_ctx = orig
+    cfg = CONFIGS[5].scaled(B=1, L=1, n_prefill=600, steps=16, M0=24, max_clusters=64, budget=200, T=3, init_mode="random")
+    _run(cfg, [0, 1, 2, 3], cfg.steps, assign_mode=1, attn_mode=1)
 
 
 def test_every_key_its_own_cluster_and_page_boundaries():

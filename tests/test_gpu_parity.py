@@ -106,16 +106,17 @@ def test_tensor_core_assign_adversarial_keys():
     ctx.destroy()
 
 
-@pytest.mark.parametrize("cid,assign_mode", [(2, 1), (3, 1), (2, 0)])
-def test_fp8_storage(cid, assign_mode):
+@pytest.mark.parametrize("cid,assign_mode,attn_mode", [(2, 1, 0), (3, 1, 0), (2, 0, 0), (3, 1, 1), (5, 1, 0)])
+def test_fp8_storage(cid, assign_mode, attn_mode):
     """FP8 storage of the K/V rows (the precision of Section 8.1's runs): the library is handed bf16 rows and keeps them
     as e4m3 bytes with a power-of-two scale per row; the oracle is handed the same rows rounded by the test-side
     quantiser.  Decisions, statistics and attention outputs then agree to the same bounds as in bf16 storage; config 3's
-    drifting stream makes clusters split, so rows also move between pages."""
+    drifting stream makes clusters split, so rows also move between pages.  attn_mode 0 is the streaming kernel on the
+    one-byte rows, 1 the plain one."""
     base = CONFIGS[cid]
     cfg = base.scaled(n_prefill=1111 if cid != 3 else 333, steps=96 if cid != 3 else 200, M0=37 if cid != 3 else 13,
                       max_clusters=160, budget=300, T=6, new_every=32 if base.new_every else 0, kv_dtype="fp8")
-    rep = _run(cfg, [0, 1, 2], cfg.steps, assign_mode=assign_mode)
+    rep = _run(cfg, [0, 1, 2], cfg.steps, assign_mode=assign_mode, attn_mode=attn_mode)
     if cid == 3:
         assert rep.splits > 0
 
