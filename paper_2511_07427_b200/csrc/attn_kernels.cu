@@ -50,10 +50,9 @@ __device__ __forceinline__ void mma_bf16(float (&c)[4], unsigned a0, unsigned a1
 
 // (hi, lo) bf16 split of two floats packed as bf16x2 (first value in the low half).
 __device__ __forceinline__ void split2(float x, float y, unsigned& hi, unsigned& lo) {
-    __nv_bfloat16 xh = __float2bfloat16_rn(x), yh = __float2bfloat16_rn(y);
-    __nv_bfloat16 xl = __float2bfloat16_rn(x - __bfloat162float(xh)), yl = __float2bfloat16_rn(y - __bfloat162float(yh));
-    hi = (unsigned)__bfloat16_as_ushort(xh) | ((unsigned)__bfloat16_as_ushort(yh) << 16);
-    lo = (unsigned)__bfloat16_as_ushort(xl) | ((unsigned)__bfloat16_as_ushort(yl) << 16);
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;\n" : "=r"(hi) : "f"(y), "f"(x));          // first source operand goes to the upper half
+    const float xr = x - __uint_as_float(hi << 16), yr = y - __uint_as_float(hi & 0xffff0000u);
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;\n" : "=r"(lo) : "f"(yr), "f"(xr));
 }
 
 __device__ __forceinline__ void mma_f16(float (&c)[4], unsigned a0, unsigned a1, unsigned a2, unsigned a3,
@@ -83,6 +82,13 @@ __device__ __forceinline__ int lds_s8x2(unsigned addr) {      // two signed byte
     unsigned short v;
     asm volatile("ld.shared.u16 %0, [%1];\n" : "=h"(v) : "r"(addr));
     return (int)v;
+}
+
+// 2^x for x <= 8 or so (flushes tiny results to zero; -inf gives 0): one special-function instruction.
+__device__ __forceinline__ float ex2(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;\n" : "=f"(y) : "f"(x));
+    return y;
 }
 
 __device__ __forceinline__ uint4 lds16(unsigned addr) {
@@ -209,29 +215,40 @@ __global__ void __launch_bounds__(AT_THREADS, 2) k_gather_attn_tma(Tables t, Ste
 
     if (warp == 0) {
         // =============================== producer ===============================
-        // Lane j owns ring stage j: it fetches the work entries of items j, j + AT_STAGES, ... and issues
-        // their copies as soon as the stage's consumer has released it, independently of the other lanes.
-        if (lane < AT_STAGES && lane < n_items) {
-            const unsigned char* kp = F8 ? t.k8 : reinterpret_cast<const unsigned char*>(t.kpages);
-            const unsigned char* vp = F8 ? t.v8 : reinterpret_cast<const unsigned char*>(t.vpages);
-            const unsigned full = smem_u32(&bars[lane]), empty = smem_u32(&bars[AT_STAGES + lane]);
-            const unsigned dst = smem_u32(ring + (size_t)lane * SM::stage_bytes);
-            int u = unit_of_bisect(pf, U, lo + lane);
-            int2 ent = work[(size_t)u * t.W + (lo + lane - pf[u])];
-            int last_issued = -1;
-            for (int it = lane; it < n_items; it += AT_STAGES) {
+        // Lane j owns ring stage j: it fetches the work entries of items j, j + stages, ... and issues their copies as
+        // soon as the stage's consumer has released it.  The lanes stay in lockstep: every turn of the loop each lane
+        // takes one non-suspending look at its own stage's barrier and the lanes whose stage is free refill it, so a lane
+        // whose stage is still in use never holds up one whose stage has just been released.
+        const bool mine = lane < AT_STAGES && lane < n_items;
+        const int sl = lane < AT_STAGES ? lane : 0;
+        const unsigned char* kp = F8 ? t.k8 : reinterpret_cast<const unsigned char*>(t.kpages);
+        const unsigned char* vp = F8 ? t.v8 : reinterpret_cast<const unsigned char*>(t.vpages);
+        const unsigned full = smem_u32(&bars[sl]), empty = smem_u32(&bars[AT_STAGES + sl]);
+        const unsigned dst = smem_u32(ring + (size_t)sl * SM::stage_bytes);
+        int it = lane;                     // this lane's next item
+        int u = 0;
+        int2 ent = make_int2(0, 0);
+        if (mine) {
+            u = unit_of_bisect(pf, U, lo + lane);
+            ent = work[(size_t)u * t.W + (lo + lane - pf[u])];
+        }
+        bool active = mine, failed = false;
+        int last_issued = -1, idle = 0;
+        unsigned long long t_idle = 0;
+        while (__any_sync(0xffffffffu, active)) {
+            const bool ready = active && mbar_test_wait(empty, (((unsigned)(it / AT_STAGES)) & 1u) ^ 1u);
+            if (ready) {
                 const int2 cur = ent;
                 const int cu = u;
-                if (it + AT_STAGES < n_items) {          // next entry: its load is in flight during the wait below
-                    u = unit_of(pf, u, lo + it + AT_STAGES);
-                    ent = work[(size_t)u * t.W + (lo + it + AT_STAGES - pf[u])];
+                const int nx = it + AT_STAGES;
+                if (nx < n_items) {          // next entry: its load is in flight until the stage comes round again
+                    u = unit_of(pf, u, lo + nx);
+                    ent = work[(size_t)u * t.W + (lo + nx - pf[u])];
                 }
-                const unsigned ph = (unsigned)(it / AT_STAGES) & 1u;
-                if (!mbar_wait(empty, ph ^ 1u)) { s_flag[0] = 1; break; }
                 const unsigned bytes = (unsigned)cur.y * ROWB;
                 const size_t row0 = (size_t)cu * t.P * PAGE + cur.x;
                 const size_t src = row0 * ROWB;
-                meta[lane] = cur.y;
+                meta[sl] = cur.y;
                 mbar_arrive_expect_tx(full, 2 * bytes + (F8 ? 2 * ENTRY_ROWS : 0));
                 bulk_g2s(dst, kp + src, bytes, full);
                 bulk_g2s(dst + ENTRY_ROWS * ROWB, vp + src, bytes, full);
@@ -241,13 +258,27 @@ __global__ void __launch_bounds__(AT_THREADS, 2) k_gather_attn_tma(Tables t, Ste
                     bulk_g2s(dst + 2 * ENTRY_ROWS * ROWB + ENTRY_ROWS, t.v8e + row0, ENTRY_ROWS, full);
                 }
                 last_issued = it;
+                it = nx;
+                active = nx < n_items;
             }
-            if (*(volatile int*)&s_flag[0]) {
-                // a bounded wait ran out: report it, and let this lane's last copy land before the CTA's
-                // shared memory can be handed to another CTA
-                atomicOr(t.status, DYNAKV_ST_INTERNAL);
-                if (last_issued >= 0) mbar_wait(full, (unsigned)(last_issued / AT_STAGES) & 1u);
+            if (__any_sync(0xffffffffu, ready)) { idle = 0; t_idle = 0; continue; }
+            // nothing was free this turn: the wait is bounded by turns and by time, and ends when a consumer gave up
+            idle++;
+            if ((idle & 63) == 0) {
+                bool stop = idle >= (1 << 22) || *(volatile int*)&s_flag[0] != 0;
+                if (lane == 0) {
+                    const unsigned long long now = global_ns();
+                    if (t_idle == 0) t_idle = now;
+                    else if (now - t_idle > 200000000ull) stop = true;
+                }
+                if (__any_sync(0xffffffffu, stop)) { failed = true; break; }
             }
+        }
+        if (failed || *(volatile int*)&s_flag[0]) {
+            // a bounded wait ran out: report it, and let every lane's last copy land before the CTA's shared memory can
+            // be handed to another CTA
+            if (lane == 0) { s_flag[0] = 1; atomicOr(t.status, DYNAKV_ST_INTERNAL); }
+            if (mine && last_issued >= 0) mbar_wait(full, (unsigned)(last_issued / AT_STAGES) & 1u);
         }
         return;
     }
@@ -357,6 +388,7 @@ __global__ void __launch_bounds__(AT_THREADS, 2) k_gather_attn_tma(Tables t, Ste
                 float sc[2][4];
 #pragma unroll
                 for (int tile = 0; tile < 2; tile++) {
+                    float s2[4] = {0.f, 0.f, 0.f, 0.f};      // two chains of four MMAs instead of one of eight
                     sc[tile][0] = 0.f; sc[tile][1] = 0.f; sc[tile][2] = 0.f; sc[tile][3] = 0.f;
 #pragma unroll
                     for (int j = 0; j < KJ; j++) {
@@ -366,9 +398,12 @@ __global__ void __launch_bounds__(AT_THREADS, 2) k_gather_attn_tma(Tables t, Ste
                             const int ks = 4 * j + w;
                             unsigned b0, b1;
                             e4m3x4_to_f16x2(w4[w], b0, b1);
-                            mma_f16(sc[tile], qa[ks][0], qa[ks][1], qa[ks][2], qa[ks][3], b0, b1);
+                            if (w & 1) mma_f16(s2, qa[ks][0], qa[ks][1], qa[ks][2], qa[ks][3], b0, b1);
+                            else mma_f16(sc[tile], qa[ks][0], qa[ks][1], qa[ks][2], qa[ks][3], b0, b1);
                         }
                     }
+#pragma unroll
+                    for (int e = 0; e < 4; e++) sc[tile][e] += s2[e];
                 }
                 // logits of head r (hi row + lo row) times the head's and the K row's scales; for the softmax the V row's
                 // exponent is added
@@ -390,11 +425,11 @@ __global__ void __launch_bounds__(AT_THREADS, 2) k_gather_attn_tma(Tables t, Ste
                 // the reference point of the exponentials follows the running maximum lazily: it moves only when the maximum
                 // has grown by more than 2^8, so weights stay below 2^8 and the accumulators are rarely rescaled
                 const float mn = mx > m + 8.f ? mx : m;        // finite: row 0 of the entry is valid
-                const float corr = exp2f(m - mn);
+                const float corr = ex2(m - mn);
                 m = mn;
                 float p[4];
 #pragma unroll
-                for (int e = 0; e < 4; e++) p[e] = exp2f(lg[e] - mn);
+                for (int e = 0; e < 4; e++) p[e] = ex2(lg[e] - mn);
                 l = l * corr + (p[0] * pow2f(-vx[0]) + p[1] * pow2f(-vx[1])) + (p[2] * pow2f(-vx[2]) + p[3] * pow2f(-vx[3]));
                 unsigned pa[4];
                 split2h(p[0], p[1], pa[0], pa[1]);   // a0 = hi(tile 0), a1 = lo(tile 0)
@@ -444,12 +479,15 @@ __global__ void __launch_bounds__(AT_THREADS, 2) k_gather_attn_tma(Tables t, Ste
                 float sc[2][4];
 #pragma unroll
                 for (int tile = 0; tile < 2; tile++) {
+                    float s2[4] = {0.f, 0.f, 0.f, 0.f};      // two chains of MMAs instead of one twice as long
                     sc[tile][0] = 0.f; sc[tile][1] = 0.f; sc[tile][2] = 0.f; sc[tile][3] = 0.f;
 #pragma unroll
                     for (int j = 0; j < KJ; j++) {
                         mma_bf16(sc[tile], qa[2 * j][0], qa[2 * j][1], qa[2 * j][2], qa[2 * j][3], kw[tile][j].x, kw[tile][j].y);
-                        mma_bf16(sc[tile], qa[2 * j + 1][0], qa[2 * j + 1][1], qa[2 * j + 1][2], qa[2 * j + 1][3], kw[tile][j].z, kw[tile][j].w);
+                        mma_bf16(s2, qa[2 * j + 1][0], qa[2 * j + 1][1], qa[2 * j + 1][2], qa[2 * j + 1][3], kw[tile][j].z, kw[tile][j].w);
                     }
+#pragma unroll
+                    for (int e = 0; e < 4; e++) sc[tile][e] += s2[e];
                 }
                 // logits of head r for tokens tile*8 + 2c + {0,1}: hi row + lo row
                 float lg[4];
@@ -465,11 +503,11 @@ __global__ void __launch_bounds__(AT_THREADS, 2) k_gather_attn_tma(Tables t, Ste
                 // the reference point of the exponentials follows the running maximum lazily: it moves only when the maximum
                 // has grown by more than 2^8, so weights stay below 2^8 and the accumulators are rarely rescaled
                 const float mn = mx > m + 8.f ? mx : m;        // finite: row 0 of the entry is valid
-                const float corr = exp2f(m - mn);
+                const float corr = ex2(m - mn);
                 m = mn;
                 float p[4];
 #pragma unroll
-                for (int e = 0; e < 4; e++) p[e] = exp2f(lg[e] - mn);
+                for (int e = 0; e < 4; e++) p[e] = ex2(lg[e] - mn);
                 l = l * corr + (p[0] + p[1]) + (p[2] + p[3]);
                 unsigned pa[4];
                 split2(p[0], p[1], pa[0], pa[1]);   // a0 = hi(tile 0), a1 = lo(tile 0)
