@@ -127,12 +127,14 @@ __device__ __forceinline__ void append_block(const Tables& t, int u, StepPtr kp_
     add = warp_sum(add);
     KV* kpg = reinterpret_cast<KV*>(t.kpages) + (((size_t)u * t.P + page) * PAGE + row) * HD;
     KV* vpg = reinterpret_cast<KV*>(t.vpages) + (((size_t)u * t.P + page) * PAGE + row) * HD;
+    const size_t aslot = ((size_t)u * t.P + page) * PAGE + row;
+    const int apos = row_pos<Epc<KV>::v>(aslot, lane * EPL);
 #pragma unroll
-    for (int e = 0; e < EPL; e++) { kpg[lane * EPL + e] = (KV)kk[e]; vpg[lane * EPL + e] = (KV)vv[e]; }
+    for (int e = 0; e < EPL; e++) { kpg[apos + e] = (KV)kk[e]; vpg[apos + e] = (KV)vv[e]; }
     if (t.fp8) {
         const size_t slot = ((size_t)u * t.P + page) * PAGE + row;
-        *reinterpret_cast<unsigned*>(t.k8 + slot * HD + lane * 4) = k8w;
-        *reinterpret_cast<unsigned*>(t.v8 + slot * HD + lane * 4) = v8w;
+        *reinterpret_cast<unsigned*>(t.k8 + slot * HD + row_pos<16>(slot, lane * 4)) = k8w;
+        *reinterpret_cast<unsigned*>(t.v8 + slot * HD + row_pos<16>(slot, lane * 4)) = v8w;
         if (lane == 0) { t.k8e[slot] = (signed char)k8x; t.v8e[slot] = (signed char)v8x; }
     }
     if (lane == 0) {

@@ -303,13 +303,13 @@ __global__ void __launch_bounds__(AT_THREADS, 2) k_gather_attn_tma(Tables t, Ste
         unsigned qa[KS][4];
         float head_scale = 0.f;          // FP8: what a logit of head r is multiplied by besides the K row's scale
         if constexpr (F8) {
-            // k-step ks takes elements 16 (c + 4 (ks / 4)) + 4 (ks % 4) .. + 3: the 16 bytes a thread loads from a K row
+            // k-step ks takes elements 16 (2c + ks / 4) + 4 (ks % 4) .. + 3: the 16 bytes a thread loads from a K row
             // are its B fragments of four k-steps.  Head r is divided by 2^ex, ex the exponent of its largest magnitude.
             float4 qv[KS];
             float amax = 0.f;
 #pragma unroll
             for (int ks = 0; ks < KS; ks++) {
-                const int base = 16 * (c + 4 * (ks >> 2)) + 4 * (ks & 3);
+                const int base = 16 * (2 * c + (ks >> 2)) + 4 * (ks & 3);
                 qv[ks] = r < G ? *reinterpret_cast<const float4*>(q + r * HD + base) : make_float4(0.f, 0.f, 0.f, 0.f);
                 amax = fmaxf(fmaxf(amax, fmaxf(fabsf(qv[ks].x), fabsf(qv[ks].y))), fmaxf(fabsf(qv[ks].z), fabsf(qv[ks].w)));
             }
@@ -328,7 +328,7 @@ __global__ void __launch_bounds__(AT_THREADS, 2) k_gather_attn_tma(Tables t, Ste
         } else {
 #pragma unroll
         for (int ks = 0; ks < KS; ks++) {
-            const int base = 8 * (c + 4 * (ks >> 1)) + 4 * (ks & 1);
+            const int base = 8 * (2 * c + ((ks >> 1) & 1) + (KJ > 2 ? 8 : 2) * (ks >> 2)) + 4 * (ks & 1);
             float x0 = 0.f, x1 = 0.f, x2 = 0.f, x3 = 0.f;
             if (r < G) {
                 const float4 v = *reinterpret_cast<const float4*>(q + r * HD + base);
@@ -359,7 +359,8 @@ __global__ void __launch_bounds__(AT_THREADS, 2) k_gather_attn_tma(Tables t, Ste
                 if (nvalid <= 0) break;
                 const unsigned krow0 = kbase + (unsigned)(sub * 16) * ROWB, vrow0 = vbase + (unsigned)(sub * 16) * ROWB;
                 if constexpr (F8) {
-                // ---- loads: K rows (tile*8 + r), chunks c + 4j; V rows 2c, 2c+1, 2c+8, 2c+9, chunk r; the scale exponents
+                // ---- loads: K rows (tile*8 + r), chunks 2c + j; V rows 2c, 2c+1, 2c+8, 2c+9, chunk r (each at its place in
+                // the row's stored chunk order, which keeps the lanes of one load on distinct banks); the scale exponents
                 // of this thread's four tokens (tile*8 + 2c, + 1)
                 // (rows past the run's end are read from its last row instead: their logits are masked and their weights
                 // are zero, so all they must be is finite)
@@ -368,13 +369,13 @@ __global__ void __launch_bounds__(AT_THREADS, 2) k_gather_attn_tma(Tables t, Ste
                 for (int tile = 0; tile < 2; tile++) {
                     const unsigned row = (unsigned)min(tile * 8 + r, nvalid - 1);
 #pragma unroll
-                    for (int j = 0; j < KJ; j++) kw[tile][j] = lds16(krow0 + row * ROWB + 16u * (c + 4 * j));
+                    for (int j = 0; j < KJ; j++) kw[tile][j] = lds16(krow0 + row * ROWB + 16u * ((2 * c + j) ^ (row & 7)));
                 }
                 uint4 vw[4];
 #pragma unroll
                 for (int rr = 0; rr < 4; rr++) {
                     const unsigned tok = (unsigned)min(2 * c + (rr & 1) + 8 * (rr >> 1), nvalid - 1);
-                    vw[rr] = lds16(vrow0 + tok * ROWB + 16u * r);
+                    vw[rr] = lds16(vrow0 + tok * ROWB + 16u * (r ^ (tok & 7)));
                 }
                 const unsigned xbase = kbase + 2 * ENTRY_ROWS * ROWB + (unsigned)(sub * 16);
                 int kx[4], vx[4];
@@ -458,7 +459,8 @@ __global__ void __launch_bounds__(AT_THREADS, 2) k_gather_attn_tma(Tables t, Ste
                     }
                 }
                 } else {
-                // ---- loads: K rows (tile*8 + r), chunks c + 4j; V rows 2c, 2c+1, 2c+8, 2c+9, chunks r + 8i
+                // ---- loads: K rows (tile*8 + r), chunks 2c, 2c+1, 2c+8, 2c+9; V rows 2c, 2c+1, 2c+8, 2c+9, chunks r + 8i
+                // (each at its place in the row's stored chunk order, which keeps the lanes of one load on distinct banks)
                 uint4 kw[2][KJ];
 #pragma unroll
                 // (rows past the run's end are read from its last row instead: their logits are masked and their weights
@@ -466,14 +468,15 @@ __global__ void __launch_bounds__(AT_THREADS, 2) k_gather_attn_tma(Tables t, Ste
                 for (int tile = 0; tile < 2; tile++) {
                     const unsigned row = (unsigned)min(tile * 8 + r, nvalid - 1);
 #pragma unroll
-                    for (int j = 0; j < KJ; j++) kw[tile][j] = lds16(krow0 + row * ROWB + 16u * (c + 4 * j));
+                    for (int j = 0; j < KJ; j++)
+                        kw[tile][j] = lds16(krow0 + row * ROWB + 16u * ((2 * c + (j & 1) + (KJ > 2 ? 8 : 2) * (j >> 1)) ^ (row & 7)));
                 }
                 uint4 vw[4][VI];
 #pragma unroll
                 for (int rr = 0; rr < 4; rr++) {
                     const unsigned tok = (unsigned)min(2 * c + (rr & 1) + 8 * (rr >> 1), nvalid - 1);
 #pragma unroll
-                    for (int i = 0; i < VI; i++) vw[rr][i] = lds16(vrow0 + tok * ROWB + 16u * (r + 8 * i));
+                    for (int i = 0; i < VI; i++) vw[rr][i] = lds16(vrow0 + tok * ROWB + 16u * ((r + 8 * i) ^ (tok & 7)));
                 }
                 // ---- S = Q K^T for the two 8-token tiles
                 float sc[2][4];

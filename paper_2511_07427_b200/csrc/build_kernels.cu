@@ -341,12 +341,14 @@ __global__ void __launch_bounds__(256) k_fin_scatter(Tables t, const KV* __restr
         if (lane == 0) slot = atomicAdd(&cursor[(size_t)u * M + j], 1);
         slot = __shfl_sync(0xffffffffu, slot, 0);
         int page = t.cl_head[(size_t)u * t.max_clusters + j] + slot / PAGE, row = slot % PAGE;
-        size_t dst = (((size_t)u * t.P + page) * PAGE + row) * HD;
+        const size_t dslot = ((size_t)u * t.P + page) * PAGE + row;
+        size_t dst = dslot * HD;
         constexpr int EPL = HD / 32;   // elements per lane
+        const int pos = row_pos<Epc<KV>::v>(dslot, lane * EPL);      // EPL elements stay inside one chunk
         const KV* ks = K + (size_t)w * HD + lane * EPL;
         const KV* vs = V + (size_t)w * HD + lane * EPL;
 #pragma unroll
-        for (int e = 0; e < EPL; e++) { kp[dst + lane * EPL + e] = ks[e]; vp[dst + lane * EPL + e] = vs[e]; }
+        for (int e = 0; e < EPL; e++) { kp[dst + pos + e] = ks[e]; vp[dst + pos + e] = vs[e]; }
         if (t.fp8) {
             // the one-byte copy of the row (the rows are on the grid already, so this conversion is exact)
             if constexpr (HD == 128 && sizeof(KV) == 2) {
@@ -358,7 +360,7 @@ __global__ void __launch_bounds__(256) k_fin_scatter(Tables t, const KV* __restr
                     const int ex = fp8_row_exp(group_max(fmaxf(fmaxf(fabsf(x0), fabsf(x1)), fmaxf(fabsf(x2), fabsf(x3))), 32));
                     const float inv = pow2f(-ex);
                     const unsigned pk = (unsigned)fp8_pack2(x0, x1, inv) | ((unsigned)fp8_pack2(x2, x3, inv) << 16);
-                    *reinterpret_cast<unsigned*>((side == 0 ? t.k8 : t.v8) + slot * HD + lane * 4) = pk;
+                    *reinterpret_cast<unsigned*>((side == 0 ? t.k8 : t.v8) + slot * HD + row_pos<16>(slot, lane * 4)) = pk;
                     if (lane == 0) (side == 0 ? t.k8e : t.v8e)[slot] = (signed char)ex;
                 }
             }
@@ -392,7 +394,8 @@ __global__ void __launch_bounds__(256) k_fin_stats(Tables t, int M, const float*
     for (int s = 0; s < c; s++) {
         int row = s % PAGE;
         if (s > 0 && row == 0) page = t.page_next[(size_t)u * t.P + page];
-        const KV* k = kp + (((size_t)u * t.P + page) * PAGE + row) * HD + lane * EPL;
+        const size_t kslot = ((size_t)u * t.P + page) * PAGE + row;
+        const KV* k = kp + kslot * HD + row_pos<Epc<KV>::v>(kslot, lane * EPL);
         float part = 0.f;
 #pragma unroll
         for (int e = 0; e < EPL; e++) { float df = to_f(k[e]) - r[e]; part = fmaf(df, df, part); }
@@ -437,8 +440,9 @@ __global__ void __launch_bounds__(128) k_export_rows(Tables t, KV* __restrict__ 
             const size_t slot = ((size_t)u * t.P + page) * PAGE + r;
             const int tok = t.page_tok[slot];
             if (tok < 0 || tok >= n) continue;
-            reinterpret_cast<uint4*>(Kout + ((size_t)u * n + tok) * HD)[v] = reinterpret_cast<const uint4*>(kp + slot * HD)[v];
-            reinterpret_cast<uint4*>(Vout + ((size_t)u * n + tok) * HD)[v] = reinterpret_cast<const uint4*>(vp + slot * HD)[v];
+            const int pv = row_pos<1>(slot, v);          // in chunks
+            reinterpret_cast<uint4*>(Kout + ((size_t)u * n + tok) * HD)[v] = reinterpret_cast<const uint4*>(kp + slot * HD)[pv];
+            reinterpret_cast<uint4*>(Vout + ((size_t)u * n + tok) * HD)[v] = reinterpret_cast<const uint4*>(vp + slot * HD)[pv];
         }
         page = t.page_next[(size_t)u * t.P + page];
     }

@@ -15,6 +15,14 @@ constexpr int PAGE = 32;            // tokens per page
 #ifndef DKV_ENTRY_ROWS
 #define DKV_ENTRY_ROWS 32
 #endif
+// Storage order inside a page row.  The row in slot s (its index in the unit's page pool) keeps its 16-byte chunks
+// permuted: logical chunk q sits at position q ^ (s & 7).  A run of rows that a bulk copy drops into shared memory
+// unchanged can then be read by the attention kernel's fragment loads -- several rows at one logical chunk, or one
+// row at several -- without two lanes of a load hitting the same banks.  Every reader and writer of the pages goes
+// through row_pos(); a row has at least eight chunks for every supported (type, d).
+//   row_pos<EPC>(s, e): position, in elements, of logical element e; EPC = elements per 16-byte chunk
+template <int EPC> __device__ __forceinline__ int row_pos(size_t slot, int e) { return e ^ (((int)slot & 7) * EPC); }
+template <typename KV> struct Epc { static constexpr int v = 16 / (int)sizeof(KV); };
 constexpr int ENTRY_ROWS = DKV_ENTRY_ROWS;   // rows per gather work entry (16 or 32: a run inside one page)
 constexpr int MAX_G = 8;
 constexpr int FLAG_HOLD = 1;        // split abandoned; not retried until the next append

@@ -43,15 +43,16 @@ __global__ void __launch_bounds__(128) k_gather_attn_v1(Tables t, StepPtr qp) {
         int2 ent = work[w];
         size_t pbase = ((size_t)u * t.P * PAGE + ent.x) * HD;
         for (int r = 0; r < ent.y; r++) {
-            const KV* k = kp + pbase + (size_t)r * HD + lane * EPL;
-            const KV* v = vp + pbase + (size_t)r * HD + lane * EPL;
+            const int pos = row_pos<Epc<KV>::v>((size_t)(ent.x + r), lane * EPL);      // the row's stored chunk order
+            const KV* k = kp + pbase + (size_t)r * HD + pos;
+            const KV* v = vp + pbase + (size_t)r * HD + pos;
             float kk[EPL], vv[EPL];
             if (t.fp8) {
                 // FP8 mode: the row's one-byte copy (four bytes per lane) and its two scale exponents
                 if constexpr (EPL == 4) {
                     const size_t slot = (size_t)u * t.P * PAGE + ent.x + r;
-                    const unsigned kb = *reinterpret_cast<const unsigned*>(t.k8 + slot * HD + lane * 4);
-                    const unsigned vb = *reinterpret_cast<const unsigned*>(t.v8 + slot * HD + lane * 4);
+                    const unsigned kb = *reinterpret_cast<const unsigned*>(t.k8 + slot * HD + row_pos<16>(slot, lane * 4));
+                    const unsigned vb = *reinterpret_cast<const unsigned*>(t.v8 + slot * HD + row_pos<16>(slot, lane * 4));
                     const float ks = pow2f(t.k8e[slot]), vs = pow2f(t.v8e[slot]);
                     float2 a = fp8_unpack2((unsigned short)(kb & 0xffffu), ks), b = fp8_unpack2((unsigned short)(kb >> 16), ks);
                     kk[0] = a.x; kk[1] = a.y; kk[2] = b.x; kk[3] = b.y;

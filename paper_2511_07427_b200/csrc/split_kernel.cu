@@ -51,8 +51,9 @@ template <int HD, int KVB> struct SplitSmem {
 // dst of unit u's pages; called by a full warp.
 __device__ __forceinline__ void fp8_move_row(const Tables& t, int u, size_t src, size_t dst, int lane) {
     const size_t gs = (size_t)u * t.P * PAGE + src, gd = (size_t)u * t.P * PAGE + dst;
-    reinterpret_cast<unsigned*>(t.k8 + gd * t.d)[lane] = reinterpret_cast<const unsigned*>(t.k8 + gs * t.d)[lane];
-    reinterpret_cast<unsigned*>(t.v8 + gd * t.d)[lane] = reinterpret_cast<const unsigned*>(t.v8 + gs * t.d)[lane];
+    const int ps = row_pos<16>(gs, lane * 4), pd = row_pos<16>(gd, lane * 4);      // each slot's own chunk order
+    *reinterpret_cast<unsigned*>(t.k8 + gd * t.d + pd) = *reinterpret_cast<const unsigned*>(t.k8 + gs * t.d + ps);
+    *reinterpret_cast<unsigned*>(t.v8 + gd * t.d + pd) = *reinterpret_cast<const unsigned*>(t.v8 + gs * t.d + ps);
     if (lane == 0) { t.k8e[gd] = t.k8e[gs]; t.v8e[gd] = t.v8e[gs]; }
 }
 
@@ -349,7 +350,11 @@ __global__ void __launch_bounds__(SP_THREADS, DKV_SP_MINBLOCKS) k_split_check(Ta
             int* rank_of = on_chip ? reinterpret_cast<int*>(area + 8192) : rank_g;
             int* holes = on_chip ? reinterpret_cast<int*>(area + 8192) + GEN_ROWS : holes_g;
             // key row and token id of member position p
-            auto key_of = [&](int p) -> const KV* { return kpg + ((size_t)chain[p >> 5] * PAGE + (p & 31)) * HD; };
+            // (key_at(p, e): logical element e of the row, in the row's stored chunk order)
+            auto key_at = [&](int p, int e) -> const KV* {
+                const size_t slot = (size_t)chain[p >> 5] * PAGE + (p & 31);
+                return kpg + slot * HD + row_pos<Epc<KV>::v>(slot, e);
+            };
             auto tok_of = [&](int p) -> int { return ptok[(size_t)chain[p >> 5] * PAGE + (p & 31)]; };
 
             // ---- centre A: member farthest from r_j; centre B: member farthest from A (ties: lowest token id)
@@ -359,7 +364,7 @@ __global__ void __launch_bounds__(SP_THREADS, DKV_SP_MINBLOCKS) k_split_check(Ta
                 for (int e = 0; e < EPL; e++) cen[e] = cA[lane * EPL + e];
                 float bd = -1.f; int bt = 0x7fffffff, bp = -1;
                 for (int p = warp; p < c; p += SP_WARPS) {
-                    const KV* k = key_of(p) + lane * EPL;
+                    const KV* k = key_at(p, lane * EPL);
                     float part = 0.f;
 #pragma unroll
                     for (int e = 0; e < EPL; e++) { float df = to_f(k[e]) - cen[e]; part = fmaf(df, df, part); }
@@ -377,10 +382,9 @@ __global__ void __launch_bounds__(SP_THREADS, DKV_SP_MINBLOCKS) k_split_check(Ta
                 }
                 __syncthreads();
                 {
-                    const KV* src = key_of(s_a);
                     float* dst = (round == 0) ? cA : cB;
                     __syncthreads();
-                    for (int e = tid; e < HD; e += SP_THREADS) dst[e] = to_f(src[e]);
+                    for (int e = tid; e < HD; e += SP_THREADS) dst[e] = to_f(*key_at(s_a, e));
                     __syncthreads();
                 }
             }
@@ -403,8 +407,8 @@ __global__ void __launch_bounds__(SP_THREADS, DKV_SP_MINBLOCKS) k_split_check(Ta
                     const int p1 = p0 + SP_WARPS;
                     float k0[EPL], k1[EPL];
                     {
-                        const KV* r0 = key_of(p0) + lane * EPL;
-                        const KV* r1 = key_of(p1 < c ? p1 : p0) + lane * EPL;
+                        const KV* r0 = key_at(p0, lane * EPL);
+                        const KV* r1 = key_at(p1 < c ? p1 : p0, lane * EPL);
 #pragma unroll
                         for (int e = 0; e < EPL; e++) { k0[e] = to_f(r0[e]); k1[e] = to_f(r1[e]); }
                     }
@@ -510,10 +514,11 @@ __global__ void __launch_bounds__(SP_THREADS, DKV_SP_MINBLOCKS) k_split_check(Ta
                 const int r = rank_of[p];
                 const size_t src = (size_t)chain[p >> 5] * PAGE + (p & 31);
                 const size_t dst = (size_t)newpg[r >> 5] * PAGE + (r & 31);
+                const int ps = row_pos<Epc<KV>::v>(src, lane * EPL), pd = row_pos<Epc<KV>::v>(dst, lane * EPL);
 #pragma unroll
                 for (int e = 0; e < EPL; e++) {
-                    kpg[dst * HD + lane * EPL + e] = kpg[src * HD + lane * EPL + e];
-                    vpg[dst * HD + lane * EPL + e] = vpg[src * HD + lane * EPL + e];
+                    kpg[dst * HD + pd + e] = kpg[src * HD + ps + e];
+                    vpg[dst * HD + pd + e] = vpg[src * HD + ps + e];
                 }
                 if (t.fp8) fp8_move_row(t, u, src, dst, lane);
                 if (lane == 0) {
@@ -529,10 +534,11 @@ __global__ void __launch_bounds__(SP_THREADS, DKV_SP_MINBLOCKS) k_split_check(Ta
                 const int h = holes[rank_of[p]];
                 const size_t src = (size_t)chain[p >> 5] * PAGE + (p & 31);
                 const size_t dst = (size_t)chain[h >> 5] * PAGE + (h & 31);
+                const int ps = row_pos<Epc<KV>::v>(src, lane * EPL), pd = row_pos<Epc<KV>::v>(dst, lane * EPL);
 #pragma unroll
                 for (int e = 0; e < EPL; e++) {
-                    kpg[dst * HD + lane * EPL + e] = kpg[src * HD + lane * EPL + e];
-                    vpg[dst * HD + lane * EPL + e] = vpg[src * HD + lane * EPL + e];
+                    kpg[dst * HD + pd + e] = kpg[src * HD + ps + e];
+                    vpg[dst * HD + pd + e] = vpg[src * HD + ps + e];
                 }
                 if (t.fp8) fp8_move_row(t, u, src, dst, lane);
                 if (lane == 0) ptok[dst] = ptok[src];
@@ -565,7 +571,8 @@ __global__ void __launch_bounds__(SP_THREADS, DKV_SP_MINBLOCKS) k_split_check(Ta
                 for (int e = 0; e < EPL; e++) sa[e] = 0.f;
                 // the child's rows in their new place
                 for (int p = warp; p < cc; p += SP_WARPS) {
-                    const KV* k = kpg + ((size_t)pages[p >> 5] * PAGE + (p & 31)) * HD + lane * EPL;
+                    const size_t kslot = (size_t)pages[p >> 5] * PAGE + (p & 31);
+                    const KV* k = kpg + kslot * HD + row_pos<Epc<KV>::v>(kslot, lane * EPL);
 #pragma unroll
                     for (int e = 0; e < EPL; e++) sa[e] += to_f(k[e]);
                 }
@@ -584,7 +591,8 @@ __global__ void __launch_bounds__(SP_THREADS, DKV_SP_MINBLOCKS) k_split_check(Ta
 #pragma unroll
                 for (int e = 0; e < EPL; e++) mean[e] = cA[lane * EPL + e];
                 for (int p = warp; p < cc; p += SP_WARPS) {
-                    const KV* k = kpg + ((size_t)pages[p >> 5] * PAGE + (p & 31)) * HD + lane * EPL;
+                    const size_t kslot = (size_t)pages[p >> 5] * PAGE + (p & 31);
+                    const KV* k = kpg + kslot * HD + row_pos<Epc<KV>::v>(kslot, lane * EPL);
                     float part = 0.f;
 #pragma unroll
                     for (int e = 0; e < EPL; e++) { float df = to_f(k[e]) - mean[e]; part = fmaf(df, df, part); }

@@ -84,8 +84,9 @@ __device__ int split_small(const Tables& t, int u, int j, int c, int iters, KV* 
     for (int idx = tid; idx < c * V16; idx += THREADS) {
         const int p = idx / V16, v = idx % V16;
         const size_t row = (size_t)page_of(p >> 5) * PAGE + (p & 31);
-        reinterpret_cast<uint4*>(krows + (size_t)p * HD)[v] = reinterpret_cast<const uint4*>(kpg + row * HD)[v];
-        reinterpret_cast<uint4*>(vrows + (size_t)p * HD)[v] = reinterpret_cast<const uint4*>(vpg + row * HD)[v];
+        const int pv = row_pos<1>(row, v);       // the staged copies are in logical chunk order
+        reinterpret_cast<uint4*>(krows + (size_t)p * HD)[v] = reinterpret_cast<const uint4*>(kpg + row * HD)[pv];
+        reinterpret_cast<uint4*>(vrows + (size_t)p * HD)[v] = reinterpret_cast<const uint4*>(vpg + row * HD)[pv];
     }
     if (tid < c) {
         const size_t slot = (size_t)page_of(tid >> 5) * PAGE + (tid & 31);
@@ -273,8 +274,9 @@ __device__ int split_small(const Tables& t, int u, int j, int c, int iters, KV* 
         size_t dst;
         if (code >= 0) dst = (size_t)sc.newpg[code >> 5] * PAGE + (code & 31);
         else { const int h = sc.holes[-2 - code]; dst = (size_t)page_of(h >> 5) * PAGE + (h & 31); }
-        reinterpret_cast<uint4*>(kpg + dst * HD)[v] = reinterpret_cast<const uint4*>(krows + (size_t)p * HD)[v];
-        reinterpret_cast<uint4*>(vpg + dst * HD)[v] = reinterpret_cast<const uint4*>(vrows + (size_t)p * HD)[v];
+        const int pv = row_pos<1>(dst, v);       // the destination slot's chunk order
+        reinterpret_cast<uint4*>(kpg + dst * HD)[pv] = reinterpret_cast<const uint4*>(krows + (size_t)p * HD)[v];
+        reinterpret_cast<uint4*>(vpg + dst * HD)[pv] = reinterpret_cast<const uint4*>(vrows + (size_t)p * HD)[v];
         if (t.fp8) {
             // the one-byte copy follows the row: the staged values are on the grid, so packing them with the row's own
             // scale gives the row's bytes back
@@ -287,7 +289,7 @@ __device__ int split_small(const Tables& t, int u, int j, int c, int iters, KV* 
                     uint2 pk;
                     pk.x = (unsigned)fp8_pack2(to_f(src[0]), to_f(src[1]), inv) | ((unsigned)fp8_pack2(to_f(src[2]), to_f(src[3]), inv) << 16);
                     pk.y = (unsigned)fp8_pack2(to_f(src[4]), to_f(src[5]), inv) | ((unsigned)fp8_pack2(to_f(src[6]), to_f(src[7]), inv) << 16);
-                    *reinterpret_cast<uint2*>((side == 0 ? t.k8 : t.v8) + g * HD + v * 8) = pk;
+                    *reinterpret_cast<uint2*>((side == 0 ? t.k8 : t.v8) + g * HD + row_pos<16>(g, v * 8)) = pk;
                     if (v == 0) (side == 0 ? t.k8e : t.v8e)[g] = side == 0 ? s_kx[p] : s_vx[p];
                 }
             }
