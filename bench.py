@@ -31,7 +31,9 @@ METRIC = "decode steps/s at 32-layer 32K ctx; retrieval-attention HBM GB/s vs pe
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch, and the tokens that launch attended.  Traffic
 # is proportional to the rows attended, so a launch's traffic is scaled by its own token count.  Set
 # NCU_ATTN_CAPTURE to None whenever the kernel changes after the capture.
-NCU_ATTN_CAPTURE = {"dram_bytes": 100.3295e6 + 3.1793e6, "tokens": 195006.5}
+NCU_ATTN_CAPTURE = {"dram_bytes": 100.3539e6 + 2.9870e6, "tokens": 195006.5}
+# the same for the kernel on FP8 rows (profiles/gather_attn_fp8_config4_96units.txt)
+NCU_ATTN_CAPTURE_FP8 = {"dram_bytes": 51.9986e6 + 0.2985e6, "tokens": 194980.75}
 
 
 def _peaks():
@@ -373,7 +375,9 @@ def run_ours(args, cfg):
                 "frac": achieved / peaks["hbm_gbs"],
                 "traffic": (args.attn_traffic_bytes if args.attn_traffic_bytes is not None else
                             (NCU_ATTN_CAPTURE["dram_bytes"] * tokens_per_launch / NCU_ATTN_CAPTURE["tokens"]
-                             if NCU_ATTN_CAPTURE and cfg.kv_dtype == "bf16" and cfg.d == 128 else None)),
+                             if NCU_ATTN_CAPTURE and cfg.kv_dtype == "bf16" and cfg.d == 128 else
+                             NCU_ATTN_CAPTURE_FP8["dram_bytes"] * tokens_per_launch / NCU_ATTN_CAPTURE_FP8["tokens"]
+                             if NCU_ATTN_CAPTURE_FP8 and cfg.kv_dtype == "fp8" else None)),
                 "kernel": "gather_attn", "us_per_launch": attn_ms * 1e3, "timed_how": attn_how,
                 "us_per_launch_event_pair_each": attn_ms_each * 1e3, "algorithmic_bytes_per_launch": attn_bytes,
                 "tokens_per_launch": tokens_per_launch, "frac_of_8TBs_nominal": achieved / 8000.0,
