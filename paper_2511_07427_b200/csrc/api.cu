@@ -561,14 +561,20 @@ extern "C" int dynakv_decode_loop_host(dynakv_ctx* c, const float* q_host, const
         for (int b = 0; b < 2; b++)
             for (cudaEvent_t* e : {&c->ev_in[b], &c->ev_done[b], &c->ev_out[b]}) CK(cudaEventCreateWithFlags(e, cudaEventDisableTiming));
     }
-    // Chunks of CH steps: chunk i + 1 is copied in and chunk i - 1 copied out while the loop runs chunk i.
-    const int64_t n_chunks = (n_steps + CH - 1) / CH;
+    // Chunks of up to CH steps: chunk i + 1 is copied in and chunk i - 1 copied out while the loop runs chunk i.
+    // The first chunk's copy in and the last chunk's copy out have nothing to hide behind, so the chunks start at
+    // 4 steps and double up to CH, and halve again towards the end of the call.
     // whatever ran on the context's stream before must be complete before its inputs are overwritten
     CK(cudaEventRecord(c->ev_done[0], c->stream)); CK(cudaEventRecord(c->ev_done[1], c->stream));
     CK(cudaEventRecord(c->ev_out[0], c->out_stream)); CK(cudaEventRecord(c->ev_out[1], c->out_stream));
-    for (int64_t i = 0; i < n_chunks; i++) {
+    int64_t s0 = 0;
+    for (int64_t i = 0; s0 < n_steps; i++) {
         const int b = (int)(i & 1);
-        const int64_t s0 = i * CH, nb = (n_steps - s0 < CH) ? n_steps - s0 : CH;
+        const int64_t left = n_steps - s0;
+        int64_t nb = i < 3 ? (int64_t)4 << i : CH;
+        if (nb > CH) nb = CH;
+        if (nb > (left + 1) / 2) nb = (left + 1) / 2 > 4 ? (left + 1) / 2 : 4;
+        if (nb > left) nb = left;
         // copy in: the staging set is free once the loop over the chunk that used it before has finished
         CK(cudaStreamWaitEvent(c->in_stream, c->ev_done[b], 0));
         CK(cudaMemcpyAsync(c->hl_q[b], (const char*)q_host + s0 * qs, nb * qs, cudaMemcpyHostToDevice, c->in_stream));
@@ -585,6 +591,7 @@ extern "C" int dynakv_decode_loop_host(dynakv_ctx* c, const float* q_host, const
         CK(cudaStreamWaitEvent(c->out_stream, c->ev_done[b], 0));
         CK(cudaMemcpyAsync((char*)out_host + s0 * qs, c->hl_out[b], nb * qs, cudaMemcpyDeviceToHost, c->out_stream));
         CK(cudaEventRecord(c->ev_out[b], c->out_stream));
+        s0 += nb;
     }
     CK(cudaStreamSynchronize(c->out_stream));
     CK(cudaStreamSynchronize(c->stream));
