@@ -175,7 +175,8 @@ int dynakv_step_host(dynakv_ctx* ctx, const float* q_host, const void* k_host,
                      const void* v_host, int32_t token_budget, float* out_host);
 
 /* dynakv_decode_loop with HOST arrays (same shapes; pinned memory for the copies to overlap): the steps are taken in
- * chunks of 32; while the loop runs one chunk on the device, the next chunk's q, k, v are copied in and the
+ * chunks of up to 32 (shorter ones at both ends of the call, so that the first copy in and the last copy out are
+ * short); while the loop runs one chunk on the device, the next chunk's q, k, v are copied in and the
  * previous chunk's outputs copied out on two more streams.  Returns when every output is in out_steps.  For a
  * caller that has its inputs step by step, dynakv_step_host is the call. */
 int dynakv_decode_loop_host(dynakv_ctx* ctx, const float* q_steps, const void* k_steps, const void* v_steps,
