@@ -78,6 +78,12 @@ typedef struct dynakv_config {
     int32_t attn_mode;         /* 0: auto (tensor-core gather-attention for bf16 K/V), 1: force the plain fp32 kernel */
     int32_t update_mode;       /* DYNAKV_MODE_ADAPTIVE (0, the paper's method), DYNAKV_MODE_STATIC or DYNAKV_MODE_LOCAL */
     int32_t local_max;         /* DYNAKV_MODE_LOCAL: a cluster born during decoding splits above this size (>= 2)    */
+    int32_t det_sums;          /* 1: the build's centroid sums (Eq. 4) accumulate in 64-bit fixed point, units of 2^-24:
+                                  the sum does not depend on the order in which keys arrive, so the centroids and every
+                                  Lloyd round's assignment are reproducible bit for bit from run to run (the order of a
+                                  cluster's rows inside its pages still follows arrival).  Needs |key element| < 2^18 (else DYNAKV_ST_INTERNAL is
+                                  set and the element is clamped) and at most 2^20 keys per cluster.  0: fp32 atomic adds
+                                  in arrival order (last bits of the centroids may differ between runs)             */
 } dynakv_config;
 
 /* How the partition follows the decode stream (Section 3.1; the baselines of Section 8.1):

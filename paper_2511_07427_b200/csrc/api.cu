@@ -153,6 +153,7 @@ extern "C" int dynakv_create(const dynakv_config* cfg, void* cuda_stream, dynakv
     t.kv_dtype = t.fp8 ? DYNAKV_BF16 : cfg->kv_dtype;
     t.max_tokens = cfg->max_tokens; t.max_clusters = cfg->max_clusters;
     t.update_mode = cfg->update_mode; t.local_max = cfg->local_max;
+    t.det_sums = cfg->det_sums ? 1 : 0;
     const int full_pages = (cfg->max_tokens + PAGE - 1) / PAGE;
     int slack = full_pages / 8; if (slack < 64) slack = 64;
     t.P = full_pages + cfg->max_clusters + slack;
@@ -267,7 +268,7 @@ extern "C" int dynakv_build_index(dynakv_ctx* c, const void* K, const void* V, i
     memset(&b, 0, sizeof(b));
     const size_t mark = c->allocs.size();
     ALLOC_B(b.C, U * M * d, false);
-    ALLOC_B(b.sums, U * M * d, false);
+    ALLOC_B(b.sums, U * M * d * (t.det_sums ? 2 : 1), false);      // 64-bit sums in the order-independent mode
     ALLOC_B(b.counts, U * M, false);
     ALLOC_B(b.cursor, U * M, false);
     ALLOC_B(b.picks, U * M, false);
@@ -676,7 +677,7 @@ extern "C" int dynakv_import_state(dynakv_ctx* c, const void* K, const void* V, 
     const size_t mark = c->allocs.size();
     int* ids_dev = nullptr; float* tau_dev = nullptr;
     ALLOC_B(b.C, U * M * d, true);
-    ALLOC_B(b.sums, U * M * d, false);
+    ALLOC_B(b.sums, U * M * d * (t.det_sums ? 2 : 1), false);      // 64-bit sums in the order-independent mode
     ALLOC_B(b.counts, U * M, false);
     ALLOC_B(b.cursor, U * M, false);
     ALLOC_B(ids_dev, U, false);

@@ -275,6 +275,42 @@ __global__ void __launch_bounds__(256) k_update_sums(const KV* __restrict__ K, l
     }
 }
 
+// The same with sums that do not depend on the order of arrival: every element is rounded to a multiple of 2^-24 and
+// added as a 64-bit integer.  Elements of 2^18 or more are clamped and reported.
+constexpr float DET_SCALE = 16777216.f;     // 2^24
+template <typename KV, int HD>
+__global__ void __launch_bounds__(256) k_update_sums_det(const KV* __restrict__ K, long long n_total, int n, int M,
+                                                          const int* __restrict__ assign, long long* __restrict__ sums,
+                                                          int* __restrict__ counts, unsigned int* __restrict__ status) {
+    const int lane = threadIdx.x & 31;
+    long long w = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const long long nwarps = ((long long)gridDim.x * blockDim.x) >> 5;
+    for (; w < n_total; w += nwarps) {
+        int u = (int)(w / n);
+        int j = assign[w];
+        const KV* k = K + (size_t)w * HD;
+        unsigned long long* dst = reinterpret_cast<unsigned long long*>(sums + ((size_t)u * M + j) * HD);
+        if (lane * 4 < HD) {
+            float4 v = ld4(k, lane * 4);
+            const float x[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+            for (int e = 0; e < 4; e++) {
+                float xe = x[e];
+                if (!(fabsf(xe) < 262144.f)) { atomicOr(status, DYNAKV_ST_INTERNAL); xe = xe != xe ? 0.f : copysignf(262143.f, xe); }
+                atomicAdd(dst + lane * 4 + e, (unsigned long long)__float2ll_rn(xe * DET_SCALE));
+            }
+        }
+        if (lane == 0) atomicAdd(&counts[(size_t)u * M + j], 1);
+    }
+}
+__global__ void k_centroid_div_det(float* __restrict__ C, const long long* __restrict__ sums, const int* __restrict__ counts,
+                                   long long total, int d) {
+    long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= total) return;
+    int c = counts[i / d];
+    if (c > 0) C[i] = (float)(((double)sums[i] * (1.0 / 16777216.0)) / (double)c);
+}
+
 // c_j = sum_j / count_j; an empty cluster keeps its previous centre.
 __global__ void k_centroid_div(float* __restrict__ C, const float* __restrict__ sums, const int* __restrict__ counts,
                                long long total, int d) {
@@ -522,12 +558,19 @@ template <typename KV, int HD>
 static void update_t(const Tables& t, const void* K, long long n, int M, const int* assign, const BuildScratch& b,
                      cudaStream_t s, long long* launches) {
     long long total = (long long)t.U * n;
-    cudaMemsetAsync(b.sums, 0, sizeof(float) * (size_t)t.U * M * HD, s);
+    cudaMemsetAsync(b.sums, 0, sizeof(float) * (size_t)t.U * M * HD * (t.det_sums ? 2 : 1), s);
     cudaMemsetAsync(b.counts, 0, sizeof(int) * (size_t)t.U * M, s);
     long long blocks = (total + 7) / 8;
     if (blocks > 148LL * 64) blocks = 148LL * 64;
-    k_update_sums<KV, HD><<<(unsigned)blocks, 256, 0, s>>>((const KV*)K, total, (int)n, M, assign, b.sums, b.counts);
     long long cd = (long long)t.U * M * HD;
+    if (t.det_sums) {
+        long long* isums = reinterpret_cast<long long*>(b.sums);
+        k_update_sums_det<KV, HD><<<(unsigned)blocks, 256, 0, s>>>((const KV*)K, total, (int)n, M, assign, isums, b.counts, t.status);
+        k_centroid_div_det<<<(unsigned)((cd + 255) / 256), 256, 0, s>>>(b.C, isums, b.counts, cd, HD);
+        (*launches) += 2;
+        return;
+    }
+    k_update_sums<KV, HD><<<(unsigned)blocks, 256, 0, s>>>((const KV*)K, total, (int)n, M, assign, b.sums, b.counts);
     k_centroid_div<<<(unsigned)((cd + 255) / 256), 256, 0, s>>>(b.C, b.sums, b.counts, cd, HD);
     (*launches) += 2;
 }

@@ -34,6 +34,7 @@ constexpr int FLAG_HOLD = 1;        // split abandoned; not retried until the ne
 struct Tables {
     int U, G, d, kv_dtype, max_tokens, max_clusters, P, n_splits_attn;
     int update_mode, local_max;      // DYNAKV_MODE_*; LOCAL: size above which a decode-born cluster splits
+    int det_sums;                    // 1: centroid sums of the build in 64-bit fixed point (order-independent)
     // FP8 mode (fp8 != 0): kv_dtype is DYNAKV_BF16 for every kernel, all rows lie on the e4m3-times-power-of-two grid,
     // and a one-byte copy of the pages is kept for the gather-attention kernel
     int fp8;

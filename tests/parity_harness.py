@@ -62,7 +62,8 @@ def log_ties(name: str, rep: "ParityReport") -> None:
                                 "bound": tie_bound(rep), "steps": rep.steps, "splits": rep.splits}) + "\n")
 
 
-def make_ctx(cfg: WorkloadConfig, n_units: int, trace: int = 1, assign_mode: int = 0, attn_mode: int = 0) -> P.DynaKV:
+def make_ctx(cfg: WorkloadConfig, n_units: int, trace: int = 1, assign_mode: int = 0, attn_mode: int = 0,
+             det_sums: int = 0) -> P.DynaKV:
     return P.DynaKV(P.DynaKVConfig(
         n_units=n_units, gqa_group=cfg.G, head_dim=cfg.d,
         kv_dtype={"f32": P.F32, "bf16": P.BF16, "fp8": P.FP8}[cfg.kv_dtype],
@@ -71,7 +72,7 @@ def make_ctx(cfg: WorkloadConfig, n_units: int, trace: int = 1, assign_mode: int
         split_size_factor=cfg.split_size_factor, split_var_factor=cfg.split_var_factor,
         split_min_size=cfg.split_min_size, split_iters=cfg.split_iters, trace=trace, assign_mode=assign_mode, attn_mode=attn_mode,
         update_mode={"adaptive": P.MODE_ADAPTIVE, "static": P.MODE_STATIC, "local": P.MODE_LOCAL}[cfg.update_mode],
-        local_max=cfg.local_max))
+        local_max=cfg.local_max, det_sums=det_sums))
 
 
 def fp8_round_rows(x: "torch.Tensor") -> "torch.Tensor":
@@ -135,7 +136,8 @@ def check_state(o: O.OracleUnit, st: dict, ui: int, rep: ParityReport, where: st
 
 def run_parity(cfg: WorkloadConfig, units: Sequence[int], steps: int, *, assign_mode: int = 0,
                state_every: int = 1, budget: Optional[int] = None, ctx_units: Optional[Sequence[int]] = None,
-               seed: int = 1234, device: str = "cuda", check_every: int = 1, attn_mode: int = 0) -> ParityReport:
+               seed: int = 1234, device: str = "cuda", check_every: int = 1, attn_mode: int = 0,
+               det_sums: int = 0) -> ParityReport:
     """Run `steps` decode iterations of `cfg`.  The GPU context holds `ctx_units` (default:
     `units`); the oracle follows the units listed in `units` (a subset of ctx_units).  With check_every > 1 the
     split check is called only after every check_every-th append (on both sides)."""
@@ -146,7 +148,7 @@ def run_parity(cfg: WorkloadConfig, units: Sequence[int], steps: int, *, assign_
     budget = cfg.budget if budget is None else budget
     streams = [UnitStream(cfg, u) for u in ctx_units]
     K, V = make_prefill(streams)
-    ctx = make_ctx(cfg, len(ctx_units), trace=1, assign_mode=assign_mode, attn_mode=attn_mode)
+    ctx = make_ctx(cfg, len(ctx_units), trace=1, assign_mode=assign_mode, attn_mode=attn_mode, det_sums=det_sums)
     ctx.build_index(K.to(device), V.to(device), cfg.M0, seed)
     picks, trace = ctx.get_build_trace()
     st = ctx.export_state()

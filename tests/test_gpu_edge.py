@@ -376,3 +376,28 @@ def test_wrong_call_order_and_shapes():
     with pytest.raises(P.DynaKVError):
         ctx.decode_loop(q[None], K[:, 0][None], K[:, 0][None], 8)   # default stream: no graph capture
     ctx.destroy()
+
+
+def test_order_independent_centroid_sums_reproduce_bit_for_bit_and_match_the_oracle():
+    """det_sums = 1: the build's centroid sums (Eq. 4) are accumulated as 64-bit integers in units of 2^-24, so they do
+    not depend on the order in which the keys' atomic adds arrive.  Two builds of the same input give the same
+    assignment in every Lloyd round and the same centroids bit for bit, and the mode passes the same parity run as
+    the default one."""
+    from parity_harness import make_ctx
+    cfg = CONFIGS[2].scaled(B=1, L=1, n_prefill=3000, steps=24, M0=50, max_clusters=128, budget=300, T=6)
+    streams = [UnitStream(cfg, u) for u in range(6)]
+    K, V = make_prefill(streams)
+    res = []
+    for _ in range(2):
+        ctx = make_ctx(cfg, 6, trace=1, assign_mode=1, det_sums=1)
+        ctx.build_index(K.cuda(), V.cuda(), cfg.M0, 11)
+        _, trace = ctx.get_build_trace()
+        st = ctx.export_state()
+        assert ctx.get_status()["error_bits"] == 0
+        res.append((trace.copy(), st["centroids"].copy(), st["counts"].copy()))
+        ctx.destroy()
+    assert np.array_equal(res[0][0], res[1][0]) and np.array_equal(res[0][2], res[1][2])
+    assert np.array_equal(res[0][1].view(np.uint32), res[1][1].view(np.uint32))
+    rep = _run(cfg, [0, 1, 2], cfg.steps, assign_mode=1, det_sums=1)
+    assert rep.status_bits == 0
+    _run(cfg, [0, 1], 8, assign_mode=0, det_sums=1)          # with the tensor-core assignment
