@@ -10,7 +10,7 @@ import torch
 import oracle as O
 import paper_2511_07427_b200 as P
 from gen import CONFIGS, UnitStream, make_decode_chunk, make_prefill
-from parity_harness import (TOL_OUT_ABS, TOL_OUT_L2, ParityReport, check_state, make_ctx, make_oracle, rel_l2)
+from parity_harness import (TOL_OUT_ABS, TOL_OUT_L2, ParityReport, check_state, make_ctx, make_oracle, rel_l2, stored, fp8_round_rows)
 
 pytestmark = pytest.mark.gpu
 
@@ -18,10 +18,12 @@ DIRECT_STEPS = 3
 
 
 # config 3 (1K prefill, drifting keys, 64 clusters to start with) runs 200 loop iterations: its clusters split all the time
-@pytest.mark.parametrize("cid,SAMPLED,GRAPH_STEPS", [(4, [0, 101, 255], 13), (2, [0, 77, 255], 13), (3, [0, 130, 255], 200),
-                                                    (5, [0, 900, 1791], 13)])
-def test_full_size_sampled_units(cid, SAMPLED, GRAPH_STEPS):
-    cfg = CONFIGS[cid]
+# (the last case is config 4 with its rows in FP8 storage: the oracle is handed the rows as the library keeps them)
+@pytest.mark.parametrize("cid,SAMPLED,GRAPH_STEPS,kv", [(4, [0, 101, 255], 13, ""), (2, [0, 77, 255], 13, ""), (3, [0, 130, 255], 200, ""),
+                                                       (5, [0, 900, 1791], 13, ""), (4, [3, 128, 250], 13, "fp8")])
+def test_full_size_sampled_units(cid, SAMPLED, GRAPH_STEPS, kv):
+    cfg = CONFIGS[cid] if not kv else CONFIGS[cid].scaled(kv_dtype=kv)
+    rows = lambda x: stored(x.cpu(), cfg)
     U, n = cfg.U, cfg.n_prefill
     side = torch.cuda.Stream()
     with torch.cuda.stream(side):
@@ -38,7 +40,7 @@ def test_full_size_sampled_units(cid, SAMPLED, GRAPH_STEPS):
             # Eq. 3: every key in exactly one cluster, sizes add up
             assert a.min() >= 0 and a.max() < cfg.M0 and np.array_equal(np.bincount(a, minlength=cfg.M0), st["counts"][u, :cfg.M0])
             o = make_oracle(cfg)
-            o.install(K[u].double().cpu().numpy(), V[u].double().cpu().numpy(), a, int(st["n_ids"][u]))
+            o.install(rows(K[u]), rows(V[u]), a, int(st["n_ids"][u]))
             check_state(o, st, u, rep, f"full-size build unit {u}")          # Eq. 4 centroids, M2, sizes
             assert abs(float(st["tau"][u]) - o.tau) <= 1e-4 * o.tau
             oracles[u] = o
@@ -61,7 +63,7 @@ def test_full_size_sampled_units(cid, SAMPLED, GRAPH_STEPS):
                 o = oracles[u]
                 n0 = o.n
                 # the append target is read from the map before the split may have moved the token
-                o.append(k[t, u].double().cpu().numpy(), v[t, u].double().cpu().numpy(), hint_cluster=-1)
+                o.append(rows(k[t, u]), rows(v[t, u]), hint_cluster=-1)
                 o.split_check(hint_assign_after=st["tok_cluster"][u, : o.n])
                 assert o.violations == 0 and o.n == n0 + 1
                 check_state(o, st, u, rep, f"full-size step {t} unit {u}")
@@ -78,7 +80,7 @@ def test_full_size_sampled_units(cid, SAMPLED, GRAPH_STEPS):
                 out_o, _, _ = o.decode_step(q[a + t, u].double().cpu().numpy(), cfg.budget)
                 ea, el = float(np.abs(outs[t, u] - out_o).max()), rel_l2(outs[t, u], out_o)
                 assert ea <= TOL_OUT_ABS and el <= TOL_OUT_L2, f"graph step {t} unit {u}: abs {ea:.3e} relL2 {el:.3e}"
-                o.append(k[a + t, u].double().cpu().numpy(), v[a + t, u].double().cpu().numpy())
+                o.append(rows(k[a + t, u]), rows(v[a + t, u]))
                 o.split_check()
         for u in SAMPLED:
             check_state(oracles[u], st, u, rep, f"after the graph loop, unit {u}")
@@ -89,6 +91,8 @@ def test_full_size_sampled_units(cid, SAMPLED, GRAPH_STEPS):
         # M2 equal to the members' squared distances to them
         steps = DIRECT_STEPS + GRAPH_STEPS
         K_all = torch.cat([K, k[:steps].transpose(0, 1)], dim=1)                  # [U, n + steps, d]
+        as_kept = lambda X: X if kv != "fp8" else torch.cat([fp8_round_rows(X[i:i + 32]).to(X.dtype) for i in range(0, U, 32)])
+        K_all = as_kept(K_all)                                                    # the rows as the library keeps them
         Mx, nt = cfg.max_clusters, n + steps
         assert np.all(st["n_tokens"] == nt)
         tokc = torch.from_numpy(st["tok_cluster"][:, :nt].astype(np.int64)).cuda()
@@ -120,7 +124,7 @@ def test_full_size_sampled_units(cid, SAMPLED, GRAPH_STEPS):
         # ---- one more decode step on that state, checked for EVERY unit against plain torch: the selection is a score
         # prefix that fills the budget (Section 4.1), and the output is softmax attention over exactly the selected
         # clusters' tokens (Section 2.1)
-        V_all = torch.cat([V, v[:steps].transpose(0, 1)], dim=1)
+        V_all = as_kept(torch.cat([V, v[:steps].transpose(0, 1)], dim=1))
         qx = q[steps - 1]
         out = ctx.decode_step(qx, cfg.budget, selected_ids=sel)
         nsel, ntok = ctx.get_selection()
