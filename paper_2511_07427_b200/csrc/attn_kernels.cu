@@ -124,7 +124,8 @@ template <int HD, bool F8> struct AttnSmem {
     // K rows then V rows of one entry; FP8: then the K rows' and the V rows' scale exponents (ENTRY_ROWS bytes each)
     static constexpr int stage_bytes = 2 * ENTRY_ROWS * row_bytes + (F8 ? 128 : 0);
     static constexpr int ring_bytes = stages * stage_bytes;
-    static constexpr int merge_bytes = AT_CONSUMERS * 8 * (HD + 2) * 4;   // per warp: acc[8][HD], m[8], l[8]
+    static constexpr int merge_row = HD + 2;                              // floats between rows of the merge scratch
+    static constexpr int merge_bytes = AT_CONSUMERS * 8 * (merge_row + 2) * 4;   // per warp: acc[8][HD + 2], m[8], l[8]
     static constexpr int fixed_bytes = ring_bytes + merge_bytes + 2 * stages * 8 + stages * 4 + 64;
 };
 
@@ -288,8 +289,14 @@ __global__ void __launch_bounds__(AT_THREADS, 2) k_gather_attn_tma(Tables t, Ste
     const int r = lane >> 2, c = lane & 3;
     const float scale = rsqrtf((float)HD) * 1.4426950408889634f;
     const float* qbase = reinterpret_cast<const float*>(qp.get());
-    float* mrg_o = mrg;                                   // [AT_CONSUMERS][8][HD]
-    float* mrg_m = mrg + AT_CONSUMERS * 8 * HD;           // [AT_CONSUMERS][8]
+    // Merge scratch.  A warp's accumulator fragments go out with lanes (r, c) writing row r at columns 16 or 32 apart:
+    // with rows HD floats apart every lane of such a store would hit one of two banks (or one).  Rows are HD + 2
+    // floats apart and column x sits at x ^ bit5(x) ^ (bit6(x) << 4), which spreads the 32 lanes of every store over
+    // the 32 banks and leaves the merge loop's row-wise reads conflict-free.
+    constexpr int MR = SM::merge_row;
+    auto mcol = [](int x) -> int { return x ^ ((x >> 5) & 1) ^ (((x >> 6) & 1) << 4); };
+    float* mrg_o = mrg;                                   // [AT_CONSUMERS][8][MR]
+    float* mrg_m = mrg + AT_CONSUMERS * 8 * MR;           // [AT_CONSUMERS][8]
     float* mrg_l = mrg_m + AT_CONSUMERS * 8;              // [AT_CONSUMERS][8]
 
     int u = unit_of_bisect(pf, U, lo);
@@ -547,12 +554,12 @@ __global__ void __launch_bounds__(AT_THREADS, 2) k_gather_attn_tma(Tables t, Ste
 #pragma unroll
         for (int x = 0; x < NT; x++) {
             if constexpr (F8) {           // n-tile x, accumulator columns 2c and 2c+1: output columns 16 (2c) + x and 16 (2c+1) + x
-                mrg_o[(cw * 8 + r) * HD + 16 * (2 * c) + x] = o[x][0] + o[x][2];
-                mrg_o[(cw * 8 + r) * HD + 16 * (2 * c + 1) + x] = o[x][1] + o[x][3];
+                mrg_o[(cw * 8 + r) * MR + mcol(16 * (2 * c) + x)] = o[x][0] + o[x][2];
+                mrg_o[(cw * 8 + r) * MR + mcol(16 * (2 * c + 1) + x)] = o[x][1] + o[x][3];
             } else {
             const int i = x >> 3, e = x & 7;
-            mrg_o[(cw * 8 + r) * HD + 8 * (2 * c + 8 * i) + e] = o[x][0] + o[x][2];
-            mrg_o[(cw * 8 + r) * HD + 8 * (2 * c + 1 + 8 * i) + e] = o[x][1] + o[x][3];
+            mrg_o[(cw * 8 + r) * MR + mcol(8 * (2 * c + 8 * i) + e)] = o[x][0] + o[x][2];
+            mrg_o[(cw * 8 + r) * MR + mcol(8 * (2 * c + 1 + 8 * i) + e)] = o[x][1] + o[x][3];
             }
         }
         consumer_sync();
@@ -574,7 +581,7 @@ __global__ void __launch_bounds__(AT_THREADS, 2) k_gather_attn_tma(Tables t, Ste
 #pragma unroll
                 for (int w = 0; w < AT_CONSUMERS; w++) {
                     const float f = exp2f(mrg_m[w * 8 + g] - mm);
-                    a += mrg_o[(w * 8 + g) * HD + e] * f; ll += mrg_l[w * 8 + g] * f;
+                    a += mrg_o[(w * 8 + g) * MR + mcol(e)] * f; ll += mrg_l[w * 8 + g] * f;
                 }
             }
             if (whole) out[(size_t)u * G * HD + idx] = ll > 0.f ? a / ll : 0.f;
