@@ -88,13 +88,14 @@ class ClockSampler:
         if self._thread is not None:
             self._thread.start()
 
-    def stop(self, t0: float = None, t1: float = None) -> dict:
+    def stop(self, windows=None) -> dict:
+        """windows: list of (t0, t1) perf_counter intervals; samples inside any of them are summarised."""
         out = {"sm_mhz": None, "sm_max_mhz": self.sm_max, "reasons": [], "samples": 0, "power_w_max": None}
         if self._thread is None:
             return out
         self._stop.set(); self._thread.join(timeout=2)
         nv = self._nv
-        rows = [r for r in self.samples if (t0 is None or r[0] >= t0) and (t1 is None or r[0] <= t1)]
+        rows = [r for r in self.samples if windows is None or any(a <= r[0] <= b for a, b in windows)]
         if not rows:
             rows = self.samples
         if rows:
@@ -408,7 +409,7 @@ def run_ours(args, cfg):
     st1 = ctx.get_status()
     ms = statistics.median(ms_runs)
     value = whole_job_steps_per_s(world, K_steps, ms)
-    clocks = sampler.stop(t_wall0, time.perf_counter()) if sampler else None
+    clock_windows = [(t_wall0, t_wall1)]
     timed_steps = repeats * K_steps
 
     # ---- end to end through the C ABI with host buffers (pinned), copies inside the timed region.  Two calls a user
@@ -453,12 +454,19 @@ def run_ours(args, cfg):
     # variance rule fire more often (the start-up share of the short timed regions is visible against it too)
     steady_us = None
     if n_steady > 0:
+        torch.cuda.synchronize()
+        ts0 = time.perf_counter()
         e0.record()
         loop(pos, pos + n_steady)
         e1.record()
         torch.cuda.synchronize()
+        clock_windows.append((ts0, time.perf_counter()))
         steady_us = max_over_ranks(e0.elapsed_time(e1), dev) * 1e3 / n_steady
         pos += n_steady
+    # clocks sampled while the graph loop ran: the timed repeats and the long call above
+    clocks = sampler.stop(clock_windows) if sampler else None
+    if clocks is not None:
+        clocks["sampled_during"] = "the timed repeats and the steady run of the same loop"
     status = ctx.get_status()
     ctx.destroy()
 
