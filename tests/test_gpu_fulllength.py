@@ -21,7 +21,7 @@ import torch
 import paper_2511_07427_b200 as P
 from gen import CONFIGS, UnitStream, make_decode_chunk, make_prefill
 from parity_harness import (TOL_OUT_ABS, TOL_OUT_L2, ParityReport, check_every_unit, check_state, make_ctx,
-                            make_oracle, rel_l2)
+                            make_oracle, rel_l2, stored, fp8_round_rows)
 
 pytestmark = [pytest.mark.gpu, pytest.mark.slow]
 
@@ -36,10 +36,13 @@ def _log(rec):
             f.write(json.dumps(rec) + "\n")
 
 
-@pytest.mark.parametrize("cid,sampled,chunk", [(2, [0, 77, 255], 512), (4, [0, 101, 255], 256), (5, [0, 900, 1791], 512),
-                                               (3, [0, 130, 255], 4096)])
-def test_whole_decode_length(cid, sampled, chunk):
-    cfg = CONFIGS[cid]
+# (the last case is config 4 with its rows in FP8 storage: the oracle is handed the rows as the library keeps them)
+@pytest.mark.parametrize("cid,sampled,chunk,kv", [(2, [0, 77, 255], 512, ""), (4, [0, 101, 255], 256, ""), (5, [0, 900, 1791], 512, ""),
+                                                  (3, [0, 130, 255], 4096, ""), (4, [3, 128, 250], 256, "fp8")])
+def test_whole_decode_length(cid, sampled, chunk, kv):
+    cfg = CONFIGS[cid] if not kv else CONFIGS[cid].scaled(kv_dtype=kv)
+    rows = lambda x: stored(x.cpu(), cfg)
+    as_kept = lambda X: X if kv != "fp8" else torch.cat([fp8_round_rows(X[i:i + 32]).to(X.dtype) for i in range(0, X.shape[0], 32)])
     U, n0 = cfg.U, cfg.n_prefill
     steps_total = int(os.environ.get("DYNAKV_FULL_STEPS", cfg.steps))
     side = torch.cuda.Stream()
@@ -56,18 +59,18 @@ def test_whole_decode_length(cid, sampled, chunk):
         oracles = {}
         for u in sampled:
             o = make_oracle(cfg)
-            o.install(K[u].double().cpu().numpy(), V[u].double().cpu().numpy(), st["tok_cluster"][u, :n0], int(st["n_ids"][u]))
+            o.install(rows(K[u]), rows(V[u]), st["tok_cluster"][u, :n0], int(st["n_ids"][u]))
             check_state(o, st, u, rep, f"build unit {u}")
             oracles[u] = o
         K_all = torch.empty((U, n0 + steps_total, cfg.d), dtype=K.dtype, device="cuda")
-        K_all[:, :n0] = K
+        K_all[:, :n0] = as_kept(K)
         del K, V
         done, worst_abs, worst_l2 = 0, 0.0, 0.0
         gpu_ms = 0.0
         while done < steps_total:
             nb = min(chunk, steps_total - done)
             q, k, v = make_decode_chunk(streams, nb)
-            K_all[:, n0 + done: n0 + done + nb] = k.transpose(0, 1)
+            K_all[:, n0 + done: n0 + done + nb] = as_kept(k.transpose(0, 1).contiguous())
             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             e0.record()
             outs = ctx.decode_loop(q, k, v, cfg.budget)
@@ -78,8 +81,8 @@ def test_whole_decode_length(cid, sampled, chunk):
             status = ctx.get_status()
             outs_s = {u: outs[:, u].cpu().numpy().astype(np.float64) for u in sampled}
             qs = {u: q[:, u].double().cpu().numpy() for u in sampled}
-            ks = {u: k[:, u].double().cpu().numpy() for u in sampled}
-            vs = {u: v[:, u].double().cpu().numpy() for u in sampled}
+            ks = {u: rows(k[:, u]) for u in sampled}
+            vs = {u: rows(v[:, u]) for u in sampled}
             del outs, q, k, v
 
             def follow(u):
