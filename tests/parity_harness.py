@@ -12,6 +12,7 @@ output (max abs <= 2e-3, relative L2 <= 1e-3).
 """
 from __future__ import annotations
 
+import os
 from dataclasses import dataclass, field
 from typing import List, Optional, Sequence
 
@@ -43,6 +44,11 @@ class ParityReport:
     decisions: int = 0          # discrete decisions offered to the oracle as hints (assignments, selections, appends, checks)
 
 
+# where test runs leave their one-line summaries: a folder at the repository root, overridable by the environment
+LOG_DIR = os.environ.get("DYNAKV_LOG_DIR",
+                         os.path.join(os.path.dirname(os.path.dirname(os.path.abspath(__file__))), "gpurun_out"))
+
+
 def tie_bound(rep: "ParityReport") -> int:
     """Most followed ties a run may show: two, plus one per 10 000 decisions.  A tie needs two candidates within
     1e-5 relative in the oracle's fp64 numbers; on continuous random data that is rare, so a count above this bound
@@ -51,11 +57,11 @@ def tie_bound(rep: "ParityReport") -> int:
 
 
 def log_ties(name: str, rep: "ParityReport") -> None:
-    """Append one JSON line per parity run to gpurun_out/parity_ties.jsonl (when that folder exists), so the tie
-    counts of a test session can be read afterwards."""
+    """Append one JSON line per parity run to parity_ties.jsonl in the run's log folder (LOG_DIR below, when that
+    folder exists), so the tie counts of a test session can be read afterwards."""
     import json
     import os
-    folder = os.path.join(os.path.dirname(os.path.dirname(os.path.abspath(__file__))), "gpurun_out")
+    folder = LOG_DIR
     if os.path.isdir(folder):
         with open(os.path.join(folder, "parity_ties.jsonl"), "a") as f:
             f.write(json.dumps({"run": name, "ties": rep.ties, "violations": rep.violations, "decisions": rep.decisions,

@@ -8,7 +8,8 @@ loop, all units, in the launch configuration the benchmark times.  The stream is
   * the status word must show no capacity or internal bit.
 
 These runs take minutes (the oracle is a scalar fp64 program), so they carry the `slow` marker and run only with
-DYNAKV_RUN_SLOW=1.  Each run appends a one-line summary per checkpoint to gpurun_out/fulllength.jsonl."""
+DYNAKV_RUN_SLOW=1.  Each run appends a one-line summary per checkpoint to fulllength.jsonl in the log folder
+(parity_harness.LOG_DIR)."""
 import json
 import os
 import time
@@ -21,7 +22,7 @@ import torch
 import paper_2511_07427_b200 as P
 from gen import CONFIGS, UnitStream, make_decode_chunk, make_prefill
 from parity_harness import (TOL_OUT_ABS, TOL_OUT_L2, ParityReport, check_every_unit, check_state, make_ctx,
-                            make_oracle, rel_l2, stored, fp8_round_rows)
+                            make_oracle, rel_l2, stored, fp8_round_rows, LOG_DIR)
 
 pytestmark = [pytest.mark.gpu, pytest.mark.slow]
 
@@ -29,7 +30,7 @@ ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 
 
 def _log(rec):
-    folder = os.path.join(ROOT, "gpurun_out")
+    folder = LOG_DIR
     print(json.dumps(rec), flush=True)
     if os.path.isdir(folder):
         with open(os.path.join(folder, "fulllength.jsonl"), "a") as f:
