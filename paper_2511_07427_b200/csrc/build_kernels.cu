@@ -384,7 +384,11 @@ __global__ void __launch_bounds__(256) k_fin_scatter(Tables t, const KV* __restr
         const KV* ks = K + (size_t)w * HD + lane * EPL;
         const KV* vs = V + (size_t)w * HD + lane * EPL;
 #pragma unroll
-        for (int e = 0; e < EPL; e++) { kp[dst + pos + e] = ks[e]; vp[dst + pos + e] = vs[e]; }
+        for (int e = 0; e < EPL; e++) kp[dst + pos + e] = ks[e];
+        if (!t.fp8) {
+#pragma unroll
+            for (int e = 0; e < EPL; e++) vp[dst + pos + e] = vs[e];
+        }
         if (t.fp8) {
             // the one-byte copy of the row (the rows are on the grid already, so this conversion is exact)
             if constexpr (HD == 128 && sizeof(KV) == 2) {
@@ -478,6 +482,20 @@ __global__ void __launch_bounds__(128) k_export_rows(Tables t, KV* __restrict__ 
             if (tok < 0 || tok >= n) continue;
             const int pv = row_pos<1>(slot, v);          // in chunks
             reinterpret_cast<uint4*>(Kout + ((size_t)u * n + tok) * HD)[v] = reinterpret_cast<const uint4*>(kp + slot * HD)[pv];
+            if (t.fp8) {
+                // FP8 storage keeps V as bytes: eight of them and the row's scale give this 16-byte piece back exactly
+                if constexpr (HD == 128 && sizeof(KV) == 2) {
+                    const uint2 by = *reinterpret_cast<const uint2*>(t.v8 + slot * HD + row_pos<16>(slot, v * 8));
+                    const float sc = pow2f(t.v8e[slot]);
+                    KV* o8 = Vout + ((size_t)u * n + tok) * HD + v * 8;
+                    const unsigned w[2] = {by.x, by.y};
+#pragma unroll
+                    for (int h = 0; h < 2; h++) {
+                        const float2 a = fp8_unpack2((unsigned short)(w[h] & 0xffffu), sc), b = fp8_unpack2((unsigned short)(w[h] >> 16), sc);
+                        o8[4 * h] = (KV)a.x; o8[4 * h + 1] = (KV)a.y; o8[4 * h + 2] = (KV)b.x; o8[4 * h + 3] = (KV)b.y;
+                    }
+                }
+            } else
             reinterpret_cast<uint4*>(Vout + ((size_t)u * n + tok) * HD)[v] = reinterpret_cast<const uint4*>(vp + slot * HD)[pv];
         }
         page = t.page_next[(size_t)u * t.P + page];

@@ -518,7 +518,7 @@ __global__ void __launch_bounds__(SP_THREADS, DKV_SP_MINBLOCKS) k_split_check(Ta
 #pragma unroll
                 for (int e = 0; e < EPL; e++) {
                     kpg[dst * HD + pd + e] = kpg[src * HD + ps + e];
-                    vpg[dst * HD + pd + e] = vpg[src * HD + ps + e];
+                    if (!t.fp8) vpg[dst * HD + pd + e] = vpg[src * HD + ps + e];
                 }
                 if (t.fp8) fp8_move_row(t, u, src, dst, lane);
                 if (lane == 0) {
@@ -538,7 +538,7 @@ __global__ void __launch_bounds__(SP_THREADS, DKV_SP_MINBLOCKS) k_split_check(Ta
 #pragma unroll
                 for (int e = 0; e < EPL; e++) {
                     kpg[dst * HD + pd + e] = kpg[src * HD + ps + e];
-                    vpg[dst * HD + pd + e] = vpg[src * HD + ps + e];
+                    if (!t.fp8) vpg[dst * HD + pd + e] = vpg[src * HD + ps + e];
                 }
                 if (t.fp8) fp8_move_row(t, u, src, dst, lane);
                 if (lane == 0) ptok[dst] = ptok[src];

@@ -86,7 +86,12 @@ __device__ int split_small(const Tables& t, int u, int j, int c, int iters, KV* 
         const size_t row = (size_t)page_of(p >> 5) * PAGE + (p & 31);
         const int pv = row_pos<1>(row, v);       // the staged copies are in logical chunk order
         reinterpret_cast<uint4*>(krows + (size_t)p * HD)[v] = reinterpret_cast<const uint4*>(kpg + row * HD)[pv];
-        reinterpret_cast<uint4*>(vrows + (size_t)p * HD)[v] = reinterpret_cast<const uint4*>(vpg + row * HD)[pv];
+        if (!t.fp8) reinterpret_cast<uint4*>(vrows + (size_t)p * HD)[v] = reinterpret_cast<const uint4*>(vpg + row * HD)[pv];
+        else if (v < HD / 16) {
+            // FP8 storage keeps V as bytes only: HD bytes per row, staged as they are (logical chunk order)
+            const unsigned char* v8r = t.v8 + ((size_t)u * t.P * PAGE + row) * HD;
+            reinterpret_cast<uint4*>(reinterpret_cast<unsigned char*>(vrows) + (size_t)p * HD)[v] = reinterpret_cast<const uint4*>(v8r)[row_pos<1>(row, v)];
+        }
     }
     if (tid < c) {
         const size_t slot = (size_t)page_of(tid >> 5) * PAGE + (tid & 31);
@@ -276,22 +281,25 @@ __device__ int split_small(const Tables& t, int u, int j, int c, int iters, KV* 
         else { const int h = sc.holes[-2 - code]; dst = (size_t)page_of(h >> 5) * PAGE + (h & 31); }
         const int pv = row_pos<1>(dst, v);       // the destination slot's chunk order
         reinterpret_cast<uint4*>(kpg + dst * HD)[pv] = reinterpret_cast<const uint4*>(krows + (size_t)p * HD)[v];
-        reinterpret_cast<uint4*>(vpg + dst * HD)[pv] = reinterpret_cast<const uint4*>(vrows + (size_t)p * HD)[v];
+        if (!t.fp8) reinterpret_cast<uint4*>(vpg + dst * HD)[pv] = reinterpret_cast<const uint4*>(vrows + (size_t)p * HD)[v];
         if (t.fp8) {
-            // the one-byte copy follows the row: the staged values are on the grid, so packing them with the row's own
-            // scale gives the row's bytes back
             if constexpr (sizeof(KV) == 2) {
                 const size_t g = (size_t)u * t.P * PAGE + dst;
-#pragma unroll
-                for (int side = 0; side < 2; side++) {
-                    const KV* src = (side == 0 ? krows : vrows) + (size_t)p * HD + v * 8;
-                    const float inv = pow2f(-(int)(side == 0 ? s_kx[p] : s_vx[p]));
+                // K's one-byte copy follows the row: the staged values are on the grid, so packing them with the row's
+                // own scale gives the row's bytes back
+                {
+                    const KV* src = krows + (size_t)p * HD + v * 8;
+                    const float inv = pow2f(-(int)s_kx[p]);
                     uint2 pk;
                     pk.x = (unsigned)fp8_pack2(to_f(src[0]), to_f(src[1]), inv) | ((unsigned)fp8_pack2(to_f(src[2]), to_f(src[3]), inv) << 16);
                     pk.y = (unsigned)fp8_pack2(to_f(src[4]), to_f(src[5]), inv) | ((unsigned)fp8_pack2(to_f(src[6]), to_f(src[7]), inv) << 16);
-                    *reinterpret_cast<uint2*>((side == 0 ? t.k8 : t.v8) + g * HD + row_pos<16>(g, v * 8)) = pk;
-                    if (v == 0) (side == 0 ? t.k8e : t.v8e)[g] = side == 0 ? s_kx[p] : s_vx[p];
+                    *reinterpret_cast<uint2*>(t.k8 + g * HD + row_pos<16>(g, v * 8)) = pk;
+                    if (v == 0) { t.k8e[g] = s_kx[p]; t.v8e[g] = s_vx[p]; }
                 }
+                // V's bytes go from the staging area to the destination slot as they are
+                if (v < HD / 16)
+                    reinterpret_cast<uint4*>(t.v8 + g * HD)[row_pos<1>(dst, v)] =
+                        reinterpret_cast<const uint4*>(reinterpret_cast<const unsigned char*>(vrows) + (size_t)p * HD)[v];
             }
         }
     }
