@@ -7,7 +7,7 @@
 // power of two and e4m3 has four significant bits, every stored value is exactly representable in bf16, so the
 // rest of the library (k-means, representatives, statistics, splits) works on bf16 rows that already lie on this
 // grid: keys and values are rounded to it once, where they enter the library, and the gather-attention kernel reads
-// the one-byte copy of the pages.
+// the one-byte pages.  K keeps bf16 pages beside its bytes (for the splits and the statistics); V is bytes only.
 //
 // The helpers below do the rounding for the register layouts the kernels use.  Conversions go through the
 // conversion intrinsics of cuda_fp8.h.
