@@ -292,6 +292,7 @@ def run_ours(args, cfg):
     del streams
     torch.cuda.synchronize()
 
+    free_before = torch.cuda.mem_get_info(dev)[0]
     ctx = P.DynaKV(P.DynaKVConfig(
         n_units=U, gqa_group=cfg.G, head_dim=cfg.d, kv_dtype={"f32": P.F32, "bf16": P.BF16, "fp8": P.FP8}[cfg.kv_dtype],
         max_tokens=cfg.max_tokens, max_clusters=cfg.max_clusters, kmeans_iters=cfg.T,
@@ -299,6 +300,8 @@ def run_ours(args, cfg):
         split_size_factor=cfg.split_size_factor, split_var_factor=cfg.split_var_factor,
         split_min_size=cfg.split_min_size, split_iters=cfg.split_iters, trace=0, assign_mode=args.assign_mode))
 
+    # device memory the context holds (page pool, index, scratch), from the driver's free-memory figure
+    context_gb = (free_before - torch.cuda.mem_get_info(dev)[0]) / 1e9
     # ---- build (prefill indexing), timed on its own
     ctx.set_timing(True)
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -314,6 +317,7 @@ def run_ours(args, cfg):
     round_ms = assign_ms + update_ms
     assign_flop = 2.0 * cfg.n_prefill * cfg.M0 * cfg.d * U
     build = {
+        "context_device_gb": context_gb,
         "seconds": build_ms / 1e3, "lloyd_rounds": cfg.T,
         "assign_ms_per_round": assign_ms, "update_ms_per_round": update_ms,
         "init_ms": kt["init"]["ms"], "finalize_ms": kt["finalize"]["ms"],

@@ -37,9 +37,9 @@ extern "C" {
  * bits, 3 mantissa bits, largest value 448) times one power-of-two scale per row, the smallest 2^e with
  * max|x| / 2^e <= 448, round to nearest even.  All arithmetic of the method then runs on those rounded values
  * (they are exact in bf16), and the gather-attention kernel streams a one-byte-per-element copy of the pages: half
- * the bytes of DYNAKV_BF16 per retrieved token.  The context keeps K's rows in bf16 as well, for the paths that
- * re-read keys (the splits' 2-means, the statistics); V is kept as bytes only, so the pages take the memory they take
- * with DYNAKV_BF16.  head_dim 128 only. */
+ * the bytes of DYNAKV_BF16 per retrieved token.  The bytes and one scale exponent per row are all the context keeps of
+ * a row (the paths that re-read keys decode them, exactly), so the pages take half the memory they take with
+ * DYNAKV_BF16.  head_dim 128 only. */
 #define DYNAKV_FP8 2
 
 #define DYNAKV_INIT_KMEANSPP 0

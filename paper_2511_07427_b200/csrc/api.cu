@@ -183,9 +183,9 @@ extern "C" int dynakv_create(const dynakv_config* cfg, void* cuda_stream, dynakv
     if (cfg->kv_dtype == DYNAKV_F32) {
         float *a, *b; ALLOC(a, page_elems, false); ALLOC(b, page_elems, false); t.kpages = a; t.vpages = b;
     } else if (t.fp8) {
-        // FP8 storage: V lives in its one-byte form only (nothing but attention, moves and export ever reads V rows);
-        // K keeps its bf16 rows beside the bytes for the splits' 2-means and the exact statistics
-        __nv_bfloat16* a; ALLOC(a, page_elems, false); t.kpages = a; t.vpages = nullptr;
+        // FP8 storage: the rows live in their one-byte form only; whoever re-reads keys (the splits' 2-means, the exact
+        // statistics, export) decodes them, which is exact
+        t.kpages = nullptr; t.vpages = nullptr;
     } else {
         __nv_bfloat16 *a, *b; ALLOC(a, page_elems, false); ALLOC(b, page_elems, false); t.kpages = a; t.vpages = b;
     }

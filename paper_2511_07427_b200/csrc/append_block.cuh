@@ -130,11 +130,7 @@ __device__ __forceinline__ void append_block(const Tables& t, int u, StepPtr kp_
     const size_t aslot = ((size_t)u * t.P + page) * PAGE + row;
     const int apos = row_pos<Epc<KV>::v>(aslot, lane * EPL);
 #pragma unroll
-    for (int e = 0; e < EPL; e++) kpg[apos + e] = (KV)kk[e];
-    if (!t.fp8) {
-#pragma unroll
-        for (int e = 0; e < EPL; e++) vpg[apos + e] = (KV)vv[e];
-    }
+    for (int e = 0; e < EPL; e++) if (!t.fp8) { kpg[apos + e] = (KV)kk[e]; vpg[apos + e] = (KV)vv[e]; }
     if (t.fp8) {
         const size_t slot = ((size_t)u * t.P + page) * PAGE + row;
         *reinterpret_cast<unsigned*>(t.k8 + slot * HD + row_pos<16>(slot, lane * 4)) = k8w;

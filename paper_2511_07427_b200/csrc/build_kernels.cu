@@ -384,11 +384,7 @@ __global__ void __launch_bounds__(256) k_fin_scatter(Tables t, const KV* __restr
         const KV* ks = K + (size_t)w * HD + lane * EPL;
         const KV* vs = V + (size_t)w * HD + lane * EPL;
 #pragma unroll
-        for (int e = 0; e < EPL; e++) kp[dst + pos + e] = ks[e];
-        if (!t.fp8) {
-#pragma unroll
-            for (int e = 0; e < EPL; e++) vp[dst + pos + e] = vs[e];
-        }
+        for (int e = 0; e < EPL; e++) if (!t.fp8) { kp[dst + pos + e] = ks[e]; vp[dst + pos + e] = vs[e]; }
         if (t.fp8) {
             // the one-byte copy of the row (the rows are on the grid already, so this conversion is exact)
             if constexpr (HD == 128 && sizeof(KV) == 2) {
@@ -435,10 +431,11 @@ __global__ void __launch_bounds__(256) k_fin_stats(Tables t, int M, const float*
         int row = s % PAGE;
         if (s > 0 && row == 0) page = t.page_next[(size_t)u * t.P + page];
         const size_t kslot = ((size_t)u * t.P + page) * PAGE + row;
-        const KV* k = kp + kslot * HD + row_pos<Epc<KV>::v>(kslot, lane * EPL);
+        float kx[EPL];
+        load_key<KV, HD, EPL>(t, kslot, lane * EPL, kx);
         float part = 0.f;
 #pragma unroll
-        for (int e = 0; e < EPL; e++) { float df = to_f(k[e]) - r[e]; part = fmaf(df, df, part); }
+        for (int e = 0; e < EPL; e++) { float df = kx[e] - r[e]; part = fmaf(df, df, part); }
         m2 += warp_sum(part);
     }
     if (lane == 0) t.cl_M2[cj] = m2;
@@ -481,22 +478,26 @@ __global__ void __launch_bounds__(128) k_export_rows(Tables t, KV* __restrict__ 
             const int tok = t.page_tok[slot];
             if (tok < 0 || tok >= n) continue;
             const int pv = row_pos<1>(slot, v);          // in chunks
-            reinterpret_cast<uint4*>(Kout + ((size_t)u * n + tok) * HD)[v] = reinterpret_cast<const uint4*>(kp + slot * HD)[pv];
             if (t.fp8) {
-                // FP8 storage keeps V as bytes: eight of them and the row's scale give this 16-byte piece back exactly
+                // FP8 storage keeps the rows as bytes: eight of them and the row's scale give this 16-byte piece back exactly
                 if constexpr (HD == 128 && sizeof(KV) == 2) {
-                    const uint2 by = *reinterpret_cast<const uint2*>(t.v8 + slot * HD + row_pos<16>(slot, v * 8));
-                    const float sc = pow2f(t.v8e[slot]);
-                    KV* o8 = Vout + ((size_t)u * n + tok) * HD + v * 8;
-                    const unsigned w[2] = {by.x, by.y};
 #pragma unroll
-                    for (int h = 0; h < 2; h++) {
-                        const float2 a = fp8_unpack2((unsigned short)(w[h] & 0xffffu), sc), b = fp8_unpack2((unsigned short)(w[h] >> 16), sc);
-                        o8[4 * h] = (KV)a.x; o8[4 * h + 1] = (KV)a.y; o8[4 * h + 2] = (KV)b.x; o8[4 * h + 3] = (KV)b.y;
+                    for (int side = 0; side < 2; side++) {
+                        const uint2 by = *reinterpret_cast<const uint2*>((side == 0 ? t.k8 : t.v8) + slot * HD + row_pos<16>(slot, v * 8));
+                        const float sc = pow2f((side == 0 ? t.k8e : t.v8e)[slot]);
+                        KV* o8 = (side == 0 ? Kout : Vout) + ((size_t)u * n + tok) * HD + v * 8;
+                        const unsigned w[2] = {by.x, by.y};
+#pragma unroll
+                        for (int h = 0; h < 2; h++) {
+                            const float2 a = fp8_unpack2((unsigned short)(w[h] & 0xffffu), sc), b = fp8_unpack2((unsigned short)(w[h] >> 16), sc);
+                            o8[4 * h] = (KV)a.x; o8[4 * h + 1] = (KV)a.y; o8[4 * h + 2] = (KV)b.x; o8[4 * h + 3] = (KV)b.y;
+                        }
                     }
                 }
-            } else
-            reinterpret_cast<uint4*>(Vout + ((size_t)u * n + tok) * HD)[v] = reinterpret_cast<const uint4*>(vp + slot * HD)[pv];
+            } else {
+                reinterpret_cast<uint4*>(Kout + ((size_t)u * n + tok) * HD)[v] = reinterpret_cast<const uint4*>(kp + slot * HD)[pv];
+                reinterpret_cast<uint4*>(Vout + ((size_t)u * n + tok) * HD)[v] = reinterpret_cast<const uint4*>(vp + slot * HD)[pv];
+            }
         }
         page = t.page_next[(size_t)u * t.P + page];
     }

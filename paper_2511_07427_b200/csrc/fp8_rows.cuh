@@ -7,7 +7,8 @@
 // power of two and e4m3 has four significant bits, every stored value is exactly representable in bf16, so the
 // rest of the library (k-means, representatives, statistics, splits) works on bf16 rows that already lie on this
 // grid: keys and values are rounded to it once, where they enter the library, and the gather-attention kernel reads
-// the one-byte pages.  K keeps bf16 pages beside its bytes (for the splits and the statistics); V is bytes only.
+// the one-byte pages.  No wider copy of a row is kept: the paths that re-read keys (splits, statistics, export)
+// decode the bytes through load_key below, which gives the rounded values back exactly.
 //
 // The helpers below do the rounding for the register layouts the kernels use.  Conversions go through the
 // conversion intrinsics of cuda_fp8.h.
@@ -48,6 +49,31 @@ __device__ __forceinline__ float2 fp8_round2(float x, float y, float inv_scale, 
 __device__ __forceinline__ float group_max(float v, int group) {
     for (int o = group >> 1; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
     return v;
+}
+
+// N consecutive elements (logical index e0; N = 1, 2 or 4, inside one 4-element group) of the K row in global slot
+// `gslot` (its index in the whole page pool), as floats: from the row's bf16 / fp32 page, or -- FP8 storage, which keeps
+// no such page -- decoded from the row's bytes and scale exponent (exact).
+template <typename KV, int HD, int N>
+__device__ __forceinline__ void load_key(const Tables& t, size_t gslot, int e0, float (&x)[N]) {
+    if (t.fp8) {
+        if constexpr (HD == 128 && sizeof(KV) == 2) {
+            const unsigned char* p = t.k8 + gslot * HD + row_pos<16>(gslot, e0);
+            const float sc = pow2f(t.k8e[gslot]);
+            if constexpr (N == 4) {
+                const unsigned w = *reinterpret_cast<const unsigned*>(p);
+                const float2 a = fp8_unpack2((unsigned short)(w & 0xffffu), sc), b = fp8_unpack2((unsigned short)(w >> 16), sc);
+                x[0] = a.x; x[1] = a.y; x[2] = b.x; x[3] = b.y;
+            } else {
+#pragma unroll
+                for (int i = 0; i < N; i++) x[i] = fp8_unpack2((unsigned short)p[i], sc).x;
+            }
+        }
+        return;
+    }
+    const KV* k = reinterpret_cast<const KV*>(t.kpages) + gslot * HD + row_pos<Epc<KV>::v>(gslot, e0);
+#pragma unroll
+    for (int i = 0; i < N; i++) x[i] = to_f(k[i]);
 }
 
 }  // namespace dkv

@@ -7,6 +7,7 @@
 
 #include "append_block.cuh"
 #include "common.cuh"
+#include "fp8_rows.cuh"
 #include "front_unit.cuh"
 #include "split_small.cuh"
 
@@ -350,11 +351,9 @@ __global__ void __launch_bounds__(SP_THREADS, DKV_SP_MINBLOCKS) k_split_check(Ta
             int* rank_of = on_chip ? reinterpret_cast<int*>(area + 8192) : rank_g;
             int* holes = on_chip ? reinterpret_cast<int*>(area + 8192) + GEN_ROWS : holes_g;
             // key row and token id of member position p
-            // (key_at(p, e): logical element e of the row, in the row's stored chunk order)
-            auto key_at = [&](int p, int e) -> const KV* {
-                const size_t slot = (size_t)chain[p >> 5] * PAGE + (p & 31);
-                return kpg + slot * HD + row_pos<Epc<KV>::v>(slot, e);
-            };
+            // (keys are read through load_key: from the row's page, or decoded from its bytes in FP8 storage)
+            const size_t gbase = (size_t)u * t.P * PAGE;          // the unit's first slot in the whole pool
+            auto gslot_of = [&](int p) -> size_t { return gbase + (size_t)chain[p >> 5] * PAGE + (p & 31); };
             auto tok_of = [&](int p) -> int { return ptok[(size_t)chain[p >> 5] * PAGE + (p & 31)]; };
 
             // ---- centre A: member farthest from r_j; centre B: member farthest from A (ties: lowest token id)
@@ -364,10 +363,11 @@ __global__ void __launch_bounds__(SP_THREADS, DKV_SP_MINBLOCKS) k_split_check(Ta
                 for (int e = 0; e < EPL; e++) cen[e] = cA[lane * EPL + e];
                 float bd = -1.f; int bt = 0x7fffffff, bp = -1;
                 for (int p = warp; p < c; p += SP_WARPS) {
-                    const KV* k = key_at(p, lane * EPL);
+                    float kx[EPL];
+                    load_key<KV, HD, EPL>(t, gslot_of(p), lane * EPL, kx);
                     float part = 0.f;
 #pragma unroll
-                    for (int e = 0; e < EPL; e++) { float df = to_f(k[e]) - cen[e]; part = fmaf(df, df, part); }
+                    for (int e = 0; e < EPL; e++) { float df = kx[e] - cen[e]; part = fmaf(df, df, part); }
                     part = warp_sum(part);
                     int tok = tok_of(p);
                     if (part > bd || (part == bd && tok < bt)) { bd = part; bt = tok; bp = p; }
@@ -384,7 +384,7 @@ __global__ void __launch_bounds__(SP_THREADS, DKV_SP_MINBLOCKS) k_split_check(Ta
                 {
                     float* dst = (round == 0) ? cA : cB;
                     __syncthreads();
-                    for (int e = tid; e < HD; e += SP_THREADS) dst[e] = to_f(*key_at(s_a, e));
+                    for (int e = tid; e < HD; e += SP_THREADS) { float x1[1]; load_key<KV, HD, 1>(t, gslot_of(s_a), e, x1); dst[e] = x1[0]; }
                     __syncthreads();
                 }
             }
@@ -407,10 +407,8 @@ __global__ void __launch_bounds__(SP_THREADS, DKV_SP_MINBLOCKS) k_split_check(Ta
                     const int p1 = p0 + SP_WARPS;
                     float k0[EPL], k1[EPL];
                     {
-                        const KV* r0 = key_at(p0, lane * EPL);
-                        const KV* r1 = key_at(p1 < c ? p1 : p0, lane * EPL);
-#pragma unroll
-                        for (int e = 0; e < EPL; e++) { k0[e] = to_f(r0[e]); k1[e] = to_f(r1[e]); }
+                        load_key<KV, HD, EPL>(t, gslot_of(p0), lane * EPL, k0);
+                        load_key<KV, HD, EPL>(t, gslot_of(p1 < c ? p1 : p0), lane * EPL, k1);
                     }
 #pragma unroll
                     for (int b2 = 0; b2 < 2; b2++) {
@@ -517,8 +515,7 @@ __global__ void __launch_bounds__(SP_THREADS, DKV_SP_MINBLOCKS) k_split_check(Ta
                 const int ps = row_pos<Epc<KV>::v>(src, lane * EPL), pd = row_pos<Epc<KV>::v>(dst, lane * EPL);
 #pragma unroll
                 for (int e = 0; e < EPL; e++) {
-                    kpg[dst * HD + pd + e] = kpg[src * HD + ps + e];
-                    if (!t.fp8) vpg[dst * HD + pd + e] = vpg[src * HD + ps + e];
+                    if (!t.fp8) { kpg[dst * HD + pd + e] = kpg[src * HD + ps + e]; vpg[dst * HD + pd + e] = vpg[src * HD + ps + e]; }
                 }
                 if (t.fp8) fp8_move_row(t, u, src, dst, lane);
                 if (lane == 0) {
@@ -537,8 +534,7 @@ __global__ void __launch_bounds__(SP_THREADS, DKV_SP_MINBLOCKS) k_split_check(Ta
                 const int ps = row_pos<Epc<KV>::v>(src, lane * EPL), pd = row_pos<Epc<KV>::v>(dst, lane * EPL);
 #pragma unroll
                 for (int e = 0; e < EPL; e++) {
-                    kpg[dst * HD + pd + e] = kpg[src * HD + ps + e];
-                    if (!t.fp8) vpg[dst * HD + pd + e] = vpg[src * HD + ps + e];
+                    if (!t.fp8) { kpg[dst * HD + pd + e] = kpg[src * HD + ps + e]; vpg[dst * HD + pd + e] = vpg[src * HD + ps + e]; }
                 }
                 if (t.fp8) fp8_move_row(t, u, src, dst, lane);
                 if (lane == 0) ptok[dst] = ptok[src];
@@ -572,9 +568,10 @@ __global__ void __launch_bounds__(SP_THREADS, DKV_SP_MINBLOCKS) k_split_check(Ta
                 // the child's rows in their new place
                 for (int p = warp; p < cc; p += SP_WARPS) {
                     const size_t kslot = (size_t)pages[p >> 5] * PAGE + (p & 31);
-                    const KV* k = kpg + kslot * HD + row_pos<Epc<KV>::v>(kslot, lane * EPL);
+                    float kx[EPL];
+                    load_key<KV, HD, EPL>(t, (size_t)u * t.P * PAGE + kslot, lane * EPL, kx);
 #pragma unroll
-                    for (int e = 0; e < EPL; e++) sa[e] += to_f(k[e]);
+                    for (int e = 0; e < EPL; e++) sa[e] += kx[e];
                 }
 #pragma unroll
                 for (int e = 0; e < EPL; e++) WS(warp, 0, lane * EPL + e) = sa[e];
@@ -592,10 +589,11 @@ __global__ void __launch_bounds__(SP_THREADS, DKV_SP_MINBLOCKS) k_split_check(Ta
                 for (int e = 0; e < EPL; e++) mean[e] = cA[lane * EPL + e];
                 for (int p = warp; p < cc; p += SP_WARPS) {
                     const size_t kslot = (size_t)pages[p >> 5] * PAGE + (p & 31);
-                    const KV* k = kpg + kslot * HD + row_pos<Epc<KV>::v>(kslot, lane * EPL);
+                    float kx[EPL];
+                    load_key<KV, HD, EPL>(t, (size_t)u * t.P * PAGE + kslot, lane * EPL, kx);
                     float part = 0.f;
 #pragma unroll
-                    for (int e = 0; e < EPL; e++) { float df = to_f(k[e]) - mean[e]; part = fmaf(df, df, part); }
+                    for (int e = 0; e < EPL; e++) { float df = kx[e] - mean[e]; part = fmaf(df, df, part); }
                     m2 += warp_sum(part);
                 }
                 if (lane == 0) red_f[warp] = m2;

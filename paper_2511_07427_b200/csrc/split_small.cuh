@@ -85,12 +85,27 @@ __device__ int split_small(const Tables& t, int u, int j, int c, int iters, KV* 
         const int p = idx / V16, v = idx % V16;
         const size_t row = (size_t)page_of(p >> 5) * PAGE + (p & 31);
         const int pv = row_pos<1>(row, v);       // the staged copies are in logical chunk order
-        reinterpret_cast<uint4*>(krows + (size_t)p * HD)[v] = reinterpret_cast<const uint4*>(kpg + row * HD)[pv];
-        if (!t.fp8) reinterpret_cast<uint4*>(vrows + (size_t)p * HD)[v] = reinterpret_cast<const uint4*>(vpg + row * HD)[pv];
-        else if (v < HD / 16) {
-            // FP8 storage keeps V as bytes only: HD bytes per row, staged as they are (logical chunk order)
-            const unsigned char* v8r = t.v8 + ((size_t)u * t.P * PAGE + row) * HD;
-            reinterpret_cast<uint4*>(reinterpret_cast<unsigned char*>(vrows) + (size_t)p * HD)[v] = reinterpret_cast<const uint4*>(v8r)[row_pos<1>(row, v)];
+        if (!t.fp8) {
+            reinterpret_cast<uint4*>(krows + (size_t)p * HD)[v] = reinterpret_cast<const uint4*>(kpg + row * HD)[pv];
+            reinterpret_cast<uint4*>(vrows + (size_t)p * HD)[v] = reinterpret_cast<const uint4*>(vpg + row * HD)[pv];
+        } else {
+            // FP8 storage keeps the rows as bytes only.  K is staged decoded (exact), eight elements per piece, so that
+            // everything below works on the same bf16 rows as in bf16 storage; V's HD bytes are staged as they are.
+            if constexpr (sizeof(KV) == 2) {
+                const size_t g = (size_t)u * t.P * PAGE + row;
+                const uint2 by = *reinterpret_cast<const uint2*>(t.k8 + g * HD + row_pos<16>(g, v * 8));
+                const float sck = pow2f(t.k8e[g]);
+                KV* o8 = krows + (size_t)p * HD + v * 8;
+                const unsigned w2[2] = {by.x, by.y};
+#pragma unroll
+                for (int h = 0; h < 2; h++) {
+                    const float2 a = fp8_unpack2((unsigned short)(w2[h] & 0xffffu), sck), b = fp8_unpack2((unsigned short)(w2[h] >> 16), sck);
+                    o8[4 * h] = (KV)a.x; o8[4 * h + 1] = (KV)a.y; o8[4 * h + 2] = (KV)b.x; o8[4 * h + 3] = (KV)b.y;
+                }
+                if (v < HD / 16)
+                    reinterpret_cast<uint4*>(reinterpret_cast<unsigned char*>(vrows) + (size_t)p * HD)[v] =
+                        reinterpret_cast<const uint4*>(t.v8 + g * HD)[row_pos<1>(row, v)];
+            }
         }
     }
     if (tid < c) {
@@ -280,8 +295,10 @@ __device__ int split_small(const Tables& t, int u, int j, int c, int iters, KV* 
         if (code >= 0) dst = (size_t)sc.newpg[code >> 5] * PAGE + (code & 31);
         else { const int h = sc.holes[-2 - code]; dst = (size_t)page_of(h >> 5) * PAGE + (h & 31); }
         const int pv = row_pos<1>(dst, v);       // the destination slot's chunk order
-        reinterpret_cast<uint4*>(kpg + dst * HD)[pv] = reinterpret_cast<const uint4*>(krows + (size_t)p * HD)[v];
-        if (!t.fp8) reinterpret_cast<uint4*>(vpg + dst * HD)[pv] = reinterpret_cast<const uint4*>(vrows + (size_t)p * HD)[v];
+        if (!t.fp8) {
+            reinterpret_cast<uint4*>(kpg + dst * HD)[pv] = reinterpret_cast<const uint4*>(krows + (size_t)p * HD)[v];
+            reinterpret_cast<uint4*>(vpg + dst * HD)[pv] = reinterpret_cast<const uint4*>(vrows + (size_t)p * HD)[v];
+        }
         if (t.fp8) {
             if constexpr (sizeof(KV) == 2) {
                 const size_t g = (size_t)u * t.P * PAGE + dst;

@@ -154,3 +154,16 @@ def test_fp8_storage_keeps_rows_on_the_grid_and_resumes():
             c.append(kd[t], vd[t]); c.split_check()
     assert np.array_equal(ctx.export_state()["tok_cluster"], ctx2.export_state()["tok_cluster"])
     ctx.destroy(); ctx2.destroy()
+
+
+def test_fp8_storage_with_clusters_too_large_to_stage():
+    """FP8 storage where the clusters that split hold about 200 rows: more than the shared-memory split path stages, so
+    the general path runs -- its 2-means and statistics read keys decoded from the one-byte pages, and its row moves
+    copy bytes slot to slot.  Direct calls against the oracle, then the same stream through the graph loop, whose
+    helper blocks take that path too."""
+    cfg = CONFIGS[2].scaled(n_prefill=600, steps=24, M0=3, max_clusters=40, budget=300, T=3, split_min_size=4,
+                            split_size_factor=1.05, kv_dtype="fp8")
+    rep = _run(cfg, [0, 1, 2], cfg.steps, assign_mode=1)
+    assert rep.splits > 0
+    from test_gpu_edge import _loop_vs_direct
+    assert _loop_vs_direct(cfg, [0, 1, 2], 24, modes=("direct", "graph")) > 0
