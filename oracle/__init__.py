@@ -19,7 +19,7 @@ _LIB = os.path.join(_HERE, "libdynakv_oracle.so")
 
 INIT_KMEANSPP = 0
 INIT_RANDOM = 1
-MODE_ADAPTIVE, MODE_STATIC, MODE_LOCAL = 0, 1, 2
+MODE_ADAPTIVE, MODE_STATIC, MODE_LOCAL, MODE_DELAYED = 0, 1, 2, 3
 ST_BUDGET_EXCEEDED = 1
 ST_MAX_CLUSTERS = 2
 ST_MAX_TOKENS = 4
@@ -84,6 +84,8 @@ def lib() -> C.CDLL:
         L.ork_get_live.argtypes = [C.c_void_p, bp]
         L.ork_set_tau.argtypes = [C.c_void_p, C.c_double]
         L.ork_set_mode.argtypes = [C.c_void_p, C.c_int, C.c_int]
+        L.ork_set_buf_max.argtypes = [C.c_void_p, C.c_int]
+        L.ork_get_flags.argtypes = [C.c_void_p, bp, ip]
     return _lib
 
 
@@ -153,11 +155,12 @@ class OracleUnit:
 
     def __init__(self, d: int, G: int, max_tokens: int, max_clusters: int, gamma: float = 2.0,
                  alpha: float = 2.0, split_min_size: int = 8, split_iters: int = 8, tol: float = 1e-5,
-                 mode: int = MODE_ADAPTIVE, local_max: int = 64):
+                 mode: int = MODE_ADAPTIVE, local_max: int = 64, buf_max: int = 64):
         self.d, self.G, self.max_tokens, self.max_clusters = d, G, max_tokens, max_clusters
         self._h = C.c_void_p(lib().ork_create(d, G, max_tokens, max_clusters, gamma, alpha,
                                                split_min_size, split_iters, tol))
         lib().ork_set_mode(self._h, mode, local_max)
+        lib().ork_set_buf_max(self._h, buf_max)
 
     def __del__(self):
         try:
@@ -251,6 +254,12 @@ class OracleUnit:
 
     def M2(self) -> np.ndarray:
         c = np.zeros(max(self.M, 1), np.float64); lib().ork_get_M2(self._h, _dp(c)); return c[: self.M]
+
+    def flags(self):
+        """DELAYED mode: (flag [M] bool: a split is owed, buf [M]: entries buffered for the cluster)."""
+        f = np.zeros(max(self.M, 1), np.uint8); b = np.zeros(max(self.M, 1), np.int32)
+        lib().ork_get_flags(self._h, _bp(f), _ip(b))
+        return f[: self.M].astype(bool), b[: self.M]
 
     def live(self) -> np.ndarray:
         c = np.zeros(max(self.M, 1), np.uint8); lib().ork_get_live(self._h, _bp(c)); return c[: self.M].astype(bool)

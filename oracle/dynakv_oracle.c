@@ -39,10 +39,16 @@
  *   STATIC    append to the nearest cluster, never split ("static update");
  *   LOCAL     new entries are clustered among themselves only ("local update"): clusters of the prefill build never
  *             change; a new entry joins the nearest cluster born during decoding (the first one founds it), and such a
- *             cluster is split by the same 2-means once it holds more than local_max entries. */
+ *             cluster is split by the same 2-means once it holds more than local_max entries;
+ *   DELAYED   the adaptive rule with Algorithm 1's delayed split (Section 4.2): a cluster whose trigger fires is split
+ *             at once only if it is among the clusters the step's query retrieved; otherwise it is flagged, entries
+ *             it takes from then on count as buffered, and it is split at the first later check at which it is among
+ *             the retrieved clusters.  When the buffered entries of all flagged clusters reach buf_max, the flagged
+ *             cluster with the most buffered entries (lowest id among equals) is split as well, after the others. */
 #define ORK_MODE_ADAPTIVE 0
 #define ORK_MODE_STATIC 1
 #define ORK_MODE_LOCAL 2
+#define ORK_MODE_DELAYED 3
 
 #define ORK_ST_BUDGET_EXCEEDED 1u
 #define ORK_ST_MAX_CLUSTERS 2u
@@ -67,6 +73,12 @@ typedef struct {
     long n_splits;
     int mode, local_max;  /* update mode; LOCAL: size above which a decode-born cluster splits */
     int M_build;          /* ids handed out by the build (or installed): the "old" clusters of LOCAL mode */
+    /* DELAYED mode */
+    int buf_max;          /* B_max: buffered entries over all flagged clusters that force a split */
+    unsigned char *flag;  /* [max_clusters] f_j: a split of cluster j is owed */
+    int *buf;             /* [max_clusters] |Buf_j|: the entry that raised the flag and every entry taken since */
+    int *req;             /* the clusters the last decode step retrieved, n_req of them */
+    int n_req;
 } ork_unit;
 
 /* ---------------------------------------------------------------- helpers */
@@ -211,6 +223,10 @@ ork_unit *ork_create(int d, int G, int max_tokens, int max_clusters, double gamm
     u->cnt = (int *)calloc((size_t)max_clusters, sizeof(int));
     u->live = (unsigned char *)calloc((size_t)max_clusters, 1);
     u->hold = (unsigned char *)calloc((size_t)max_clusters, 1);
+    u->flag = (unsigned char *)calloc((size_t)max_clusters, 1);
+    u->buf = (int *)calloc((size_t)max_clusters, sizeof(int));
+    u->req = (int *)calloc((size_t)max_clusters, sizeof(int));
+    u->buf_max = 1 << 30;
     u->gamma = gamma; u->alpha = alpha;
     u->split_min_size = split_min_size; u->split_iters = split_iters;
     u->tol = tol;
@@ -220,7 +236,7 @@ ork_unit *ork_create(int d, int G, int max_tokens, int max_clusters, double gamm
 void ork_destroy(ork_unit *u) {
     if (!u) return;
     free(u->K); free(u->V); free(u->assign); free(u->r); free(u->M2); free(u->cnt);
-    free(u->live); free(u->hold); free(u);
+    free(u->live); free(u->hold); free(u->flag); free(u->buf); free(u->req); free(u);
 }
 
 /* UpdateStats (Algorithm 1): n_j, r_j = member mean, M2_j = sum ||k - r_j||^2 recomputed
@@ -422,6 +438,9 @@ int ork_decode_step(ork_unit *u, const double *q, int budget, const int *hint_id
     ork_score(u, q, scores);
     int nsel = ork_select(u, scores, budget, hint_ids, hint_n, out_ids, out_tokens);
     ork_attend(u, q, out_ids, nsel, out);
+    /* the retrieved set of this step, for the delayed split */
+    u->n_req = nsel;
+    for (int i = 0; i < nsel; i++) u->req[i] = out_ids[i];
     free(scores);
     return nsel;
 }
@@ -486,6 +505,7 @@ int ork_append(ork_unit *u, const double *k, const double *v, int hint_cluster) 
     }
     u->M2[best] += add;
     u->hold[best] = 0;
+    if (u->mode == ORK_MODE_DELAYED && u->flag[best]) u->buf[best]++;     /* an entry for a flagged cluster is buffered */
     return best;
 }
 
@@ -567,7 +587,34 @@ int ork_split_check(ork_unit *u, const int *hint_assign_after) {
         trig[j] = by_var || by_size;
         vartie[j] = u->alpha > 0.0 && !by_size && near_tie(var, u->tau, u->tol);
     }
-    for (int j = 0; j < M0; j++) {
+    int *order = (int *)malloc(sizeof(int) * (size_t)(M0 + 1));
+    int n_order = 0;
+    if (u->mode == ORK_MODE_DELAYED) {
+        /* Algorithm 1, delayed split.  In the retrieved set: split now, whether the trigger fires at this check or
+         * the flag is owed from an earlier one.  Outside it: a firing trigger raises the flag (that entry is the first
+         * buffered one).  Then, if the buffered entries of the clusters still flagged reach buf_max, the one with the
+         * most of them follows. */
+        unsigned char *inreq = (unsigned char *)calloc((size_t)M0, 1);
+        for (int i = 0; i < u->n_req; i++) if (u->req[i] >= 0 && u->req[i] < M0) inreq[u->req[i]] = 1;
+        for (int j = 0; j < M0; j++) {
+            int owed = u->live[j] && u->flag[j];
+            if ((trig[j] || owed) && inreq[j]) { trig[j] = 1; order[n_order++] = j; continue; }
+            if (trig[j] && !u->flag[j]) { u->flag[j] = 1; u->buf[j] = 1; }
+            trig[j] = 0;
+        }
+        long total = 0; int jmax = -1;
+        for (int j = 0; j < M0; j++) {
+            if (!u->live[j] || !u->flag[j] || trig[j]) continue;
+            total += u->buf[j];
+            if (jmax < 0 || u->buf[j] > u->buf[jmax]) jmax = j;
+        }
+        if (jmax >= 0 && total >= u->buf_max) { trig[jmax] = 1; order[n_order++] = jmax; }
+        free(inreq);
+    } else {
+        for (int j = 0; j < M0; j++) order[n_order++] = j;
+    }
+    for (int oi = 0; oi < n_order; oi++) {
+        int j = order[oi];
         if (!u->live[j]) continue;
         int hinted = 0, hint_split = 0;
         if (hint_assign_after) {
@@ -586,11 +633,11 @@ int ork_split_check(ork_unit *u, const int *hint_assign_after) {
         int ok = two_means(u, mem, nm, labels, cA, cB);
         if (hinted && !hint_split) {
             /* the other side did not split j: acceptable only as a trigger tie */
-            if (!ok) { u->hold[j] = 1; continue; }
+            if (!ok) { u->hold[j] = 1; u->flag[j] = 0; u->buf[j] = 0; continue; }
             if (vartie[j]) { u->ties++; continue; }
             u->violations++;
         }
-        if (!ok) { u->hold[j] = 1; continue; }
+        if (!ok) { u->hold[j] = 1; u->flag[j] = 0; u->buf[j] = 0; continue; }
         /* stay = the side holding the smallest token id (mem[0]) */
         unsigned char stay = labels[0];
         if (hinted && hint_split) {
@@ -606,12 +653,13 @@ int ork_split_check(ork_unit *u, const int *hint_assign_after) {
         }
         int id = u->M++;
         u->live[id] = 1; u->hold[id] = 0; u->hold[j] = 0;
+        u->flag[j] = 0; u->buf[j] = 0; u->flag[id] = 0; u->buf[id] = 0;
         for (int m = 0; m < nm; m++) if (labels[m] != stay) u->assign[mem[m]] = id;
         recompute_stats(u, j);
         recompute_stats(u, id);
         done++; u->n_splits++;
     }
-    free(mem); free(labels); free(cA); free(cB); free(trig); free(vartie);
+    free(mem); free(labels); free(cA); free(cB); free(trig); free(vartie); free(order);
     return done;
 }
 
@@ -655,3 +703,7 @@ void ork_get_M2(const ork_unit *u, double *out) { memcpy(out, u->M2, sizeof(doub
 void ork_get_live(const ork_unit *u, unsigned char *out) { memcpy(out, u->live, (size_t)u->M); }
 void ork_set_tau(ork_unit *u, double tau) { u->tau = tau; }
 void ork_set_mode(ork_unit *u, int mode, int local_max) { u->mode = mode; u->local_max = local_max; }
+void ork_set_buf_max(ork_unit *u, int buf_max) { u->buf_max = buf_max; }
+void ork_get_flags(const ork_unit *u, unsigned char *flag, int *buf) {
+    memcpy(flag, u->flag, (size_t)u->M); memcpy(buf, u->buf, sizeof(int) * (size_t)u->M);
+}

@@ -629,3 +629,87 @@ def test_local_mode_separates_two_new_blobs_when_the_size_limit_is_reached():
     A = u.assign()[100:]
     assert u.M == 6 and u.n_splits == 1                          # one founding, one split at 41 entries
     assert len(set(A[lab == 0])) == 1 and len(set(A[lab == 1])) == 1 and A[0] != A[1]
+
+
+# ---------------------------------------------------------------------------------------------------------------
+# Delayed split (Algorithm 1, its last two blocks; Section 4.2): hand-built clusters on a line, so that which cluster a
+# query retrieves, which cluster an entry joins and when a variance trigger fires can all be read off the numbers.
+
+def _delayed_unit(buf_max, extra_cluster=False, mode=None):
+    """Cluster A: six entries at x = -0.05 .. 0.05; cluster B: six at 9.95 .. 10.05; optionally C: six around 30.
+    tau = 0.5: an entry 4 away from B's (or C's) centre lifts that cluster's variance over it."""
+    xs = [np.linspace(-0.05, 0.05, 6), 10 + np.linspace(-0.05, 0.05, 6)] + ([30 + np.linspace(-0.05, 0.05, 6)] if extra_cluster else [])
+    K = np.stack([np.concatenate(xs), np.zeros(6 * len(xs))], axis=1)
+    assign = np.repeat(np.arange(len(xs)), 6).astype(np.int32)
+    u = O.OracleUnit(2, 1, 64, 16, gamma=0.0, alpha=1.0, split_min_size=2,
+                     mode=O.MODE_DELAYED if mode is None else mode, buf_max=buf_max)
+    u.install(K, K, assign, len(xs))
+    u.tau = 0.5
+    return u
+
+
+def _retrieve(u, x):
+    """A query that scores cluster centres by x * centre: positive x retrieves the cluster farthest right, negative x
+    cluster A (score 0 against negative scores); the budget holds one cluster."""
+    _, ids, _ = u.decode_step(np.array([[x, 0.0]]), 9)
+    return list(ids)
+
+
+def test_delayed_split_waits_until_the_flagged_cluster_is_retrieved():
+    u = _delayed_unit(buf_max=100)
+    assert _retrieve(u, -1.0) == [0]                      # the query retrieves A
+    assert u.append(np.array([14.0, 0.0]), np.zeros(2)) == 1    # the entry joins B and lifts its variance over tau
+    assert u.counts()[1] == 7 and u.M2()[1] / 7 > 0.5
+    assert u.split_check() == 0                           # B is not among the retrieved clusters: flagged, not split
+    f, b = u.flags()
+    assert list(f) == [False, True] and list(b) == [0, 1] and u.M == 2
+    assert _retrieve(u, -1.0) == [0]
+    assert u.append(np.array([14.5, 0.0]), np.zeros(2)) == 1    # buffered for the flagged cluster
+    assert u.split_check() == 0
+    f, b = u.flags()
+    assert list(b) == [0, 2] and u.M == 2
+    assert _retrieve(u, 1.0) == [1]                       # now the query retrieves B (8 entries, budget 9)
+    assert u.append(np.array([10.0, 0.1]), np.zeros(2)) == 1
+    assert u.split_check() == 1                           # the owed split happens, on the cluster with its buffered entries
+    f, b = u.flags()
+    assert not f.any() and not b.any() and u.M == 3
+    a = u.assign()
+    assert list(a[:6]) == [0] * 6 and list(a[6:12]) == [1] * 6 and a[14] == 1      # the entries near 10 stay cluster 1
+    assert a[12] == 2 and a[13] == 2                      # the two far entries are the new cluster
+    # the same members split by the adaptive rule (no delay) give the same partition
+    v = _delayed_unit(buf_max=100, mode=O.MODE_ADAPTIVE)
+    for x, y in ((14.0, 0.0), (14.5, 0.0), (10.0, 0.1)):
+        v.append(np.array([x, y]), np.zeros(2))
+    assert v.split_check() == 1 and np.array_equal(v.assign(), a)
+
+
+def test_delayed_split_is_immediate_for_a_retrieved_cluster():
+    u = _delayed_unit(buf_max=100)
+    assert _retrieve(u, 1.0) == [1]
+    u.append(np.array([14.0, 0.0]), np.zeros(2))
+    assert u.split_check() == 1 and u.M == 3 and not u.flags()[0].any()
+
+
+def test_buffered_entries_reaching_buf_max_force_the_split_of_the_fullest_flagged_cluster():
+    u = _delayed_unit(buf_max=3, extra_cluster=True)
+    _retrieve(u, -1.0)
+    assert u.append(np.array([14.0, 0.0]), np.zeros(2)) == 1 and u.split_check() == 0       # B flagged, 1 buffered
+    _retrieve(u, -1.0)
+    assert u.append(np.array([34.0, 0.0]), np.zeros(2)) == 2 and u.split_check() == 0       # C flagged, 1 buffered; total 2 < 3
+    f, b = u.flags()
+    assert list(f) == [False, True, True] and list(b) == [0, 1, 1]
+    _retrieve(u, -1.0)
+    assert u.append(np.array([34.5, 0.0]), np.zeros(2)) == 2                                # C: 2 buffered; total 3
+    assert u.split_check() == 1                           # nothing flagged is retrieved, but the buffers are full: C goes
+    f, b = u.flags()
+    assert list(f[:3]) == [False, True, False] and list(b[:3]) == [0, 1, 0] and u.M == 4
+    a = u.assign()
+    assert a[19] == 3 and a[20] == 3 and list(a[12:18]) == [2] * 6
+    # with equal buffers the lower id goes first
+    w = _delayed_unit(buf_max=2, extra_cluster=True)
+    _retrieve(w, -1.0)
+    w.append(np.array([14.0, 0.0]), np.zeros(2)); assert w.split_check() == 0
+    _retrieve(w, -1.0)
+    w.append(np.array([34.0, 0.0]), np.zeros(2)); assert w.split_check() == 1               # total 2: B (id 1) before C
+    f, b = w.flags()
+    assert list(f[:3]) == [False, False, True]
