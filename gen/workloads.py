@@ -60,8 +60,9 @@ class WorkloadConfig:
     split_var_factor: float = 2.0    # alpha
     split_min_size: int = 8
     split_iters: int = 8
-    update_mode: str = "adaptive"    # "adaptive" | "static" | "local" (how the partition follows the decode stream)
+    update_mode: str = "adaptive"    # "adaptive" | "static" | "local" | "delayed" (how the partition follows the decode stream)
     local_max: int = 64              # "local": size above which a cluster born during decoding splits
+    buf_max: int = 64                # "delayed": buffered entries per unit that force a split
 
     @property
     def U(self) -> int:

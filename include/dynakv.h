@@ -77,7 +77,7 @@ typedef struct dynakv_config {
     int32_t trace;             /* 1: keep every Lloyd round's assignment for dynakv_get_build_trace */
     int32_t assign_mode;       /* 0: auto (tensor-core distance GEMM for bf16, d=128), 1: force fp32 path */
     int32_t attn_mode;         /* 0: auto (tensor-core gather-attention for bf16 K/V), 1: force the plain fp32 kernel */
-    int32_t update_mode;       /* DYNAKV_MODE_ADAPTIVE (0, the paper's method), DYNAKV_MODE_STATIC or DYNAKV_MODE_LOCAL */
+    int32_t update_mode;       /* DYNAKV_MODE_ADAPTIVE (0, the paper's method), _STATIC, _LOCAL or _DELAYED          */
     int32_t local_max;         /* DYNAKV_MODE_LOCAL: a cluster born during decoding splits above this size (>= 2)    */
     int32_t det_sums;          /* 1: the build's centroid sums (Eq. 4) accumulate in 64-bit fixed point, units of 2^-24:
                                   the sum does not depend on the order in which keys arrive, so the centroids and every
@@ -85,6 +85,8 @@ typedef struct dynakv_config {
                                   cluster's rows inside its pages still follows arrival).  Needs |key element| < 2^18 (else DYNAKV_ST_INTERNAL is
                                   set and the element is clamped) and at most 2^20 keys per cluster.  0: fp32 atomic adds
                                   in arrival order (last bits of the centroids may differ between runs)             */
+    int32_t buf_max;           /* DYNAKV_MODE_DELAYED: B_max of Algorithm 1, per unit -- entries buffered for flagged
+                                  clusters that force a split (>= 1)                                                  */
 } dynakv_config;
 
 /* How the partition follows the decode stream (Section 3.1; the baselines of Section 8.1):
@@ -96,6 +98,14 @@ typedef struct dynakv_config {
 #define DYNAKV_MODE_ADAPTIVE 0
 #define DYNAKV_MODE_STATIC 1
 #define DYNAKV_MODE_LOCAL 2
+/*   DELAYED   the adaptive rule with the delayed split of Algorithm 1 / Section 4.2 (there it saves the transfer of a
+ *             cluster that is not in fast memory; here every cluster is resident and the mode only reproduces the
+ *             policy): at a split check a cluster whose trigger fires is split only if the last decode step retrieved
+ *             it; otherwise it is flagged, the entries it takes from then on count as buffered, and it is split at the
+ *             first later check at which it is among the retrieved clusters.  When the buffered entries of a unit's
+ *             flagged clusters reach buf_max, the flagged cluster with the most of them (lowest id among equals) is
+ *             split as well, after the others.  Flags are not part of a checkpoint. */
+#define DYNAKV_MODE_DELAYED 3
 
 typedef struct dynakv_status {
     uint32_t error_bits;       /* OR of DYNAKV_ST_*                                              */

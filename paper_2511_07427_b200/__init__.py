@@ -6,10 +6,10 @@ marshals ``torch`` device tensors (memory and streams) into the C ABI declared i
 library raises.
 """
 from .binding import (DynaKV, DynaKVConfig, DynaKVError, load_library, F32, BF16, FP8, INIT_KMEANSPP, INIT_RANDOM,
-                      MODE_ADAPTIVE, MODE_STATIC, MODE_LOCAL,
+                      MODE_ADAPTIVE, MODE_STATIC, MODE_LOCAL, MODE_DELAYED,
                       ST_BUDGET_EXCEEDED, ST_MAX_CLUSTERS, ST_MAX_TOKENS, ST_PAGE_POOL, ST_INTERNAL, EXPORTED_SYMBOLS, attend_rows_noalloc)
 
 __all__ = ["DynaKV", "DynaKVConfig", "DynaKVError", "load_library", "F32", "BF16", "FP8", "INIT_KMEANSPP", "INIT_RANDOM",
-           "MODE_ADAPTIVE", "MODE_STATIC", "MODE_LOCAL",
+           "MODE_ADAPTIVE", "MODE_STATIC", "MODE_LOCAL", "MODE_DELAYED",
            "ST_BUDGET_EXCEEDED", "ST_MAX_CLUSTERS", "ST_MAX_TOKENS", "ST_PAGE_POOL", "ST_INTERNAL", "EXPORTED_SYMBOLS",
            "attend_rows_noalloc"]

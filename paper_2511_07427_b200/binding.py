@@ -13,7 +13,7 @@ _LIB_PATH = os.path.join(_HERE, "libdynakv.so")
 
 F32, BF16, FP8 = 0, 1, 2
 INIT_KMEANSPP, INIT_RANDOM = 0, 1
-MODE_ADAPTIVE, MODE_STATIC, MODE_LOCAL = 0, 1, 2
+MODE_ADAPTIVE, MODE_STATIC, MODE_LOCAL, MODE_DELAYED = 0, 1, 2, 3
 ST_BUDGET_EXCEEDED, ST_MAX_CLUSTERS, ST_MAX_TOKENS, ST_PAGE_POOL, ST_INTERNAL = 1, 2, 4, 8, 16
 
 EXPORTED_SYMBOLS = [
@@ -35,7 +35,7 @@ class _Config(C.Structure):
                 ("max_tokens", C.c_int32), ("max_clusters", C.c_int32), ("kmeans_iters", C.c_int32),
                 ("init_mode", C.c_int32), ("split_size_factor", C.c_float), ("split_var_factor", C.c_float),
                 ("split_min_size", C.c_int32), ("split_iters", C.c_int32), ("trace", C.c_int32),
-                ("assign_mode", C.c_int32), ("attn_mode", C.c_int32), ("update_mode", C.c_int32), ("local_max", C.c_int32), ("det_sums", C.c_int32)]
+                ("assign_mode", C.c_int32), ("attn_mode", C.c_int32), ("update_mode", C.c_int32), ("local_max", C.c_int32), ("det_sums", C.c_int32), ("buf_max", C.c_int32)]
 
 
 class _Status(C.Structure):
@@ -67,6 +67,7 @@ class DynaKVConfig:
     update_mode: int = 0
     local_max: int = 64
     det_sums: int = 0
+    buf_max: int = 64
 
 
 _lib = None
@@ -185,7 +186,7 @@ class DynaKV:
         self._stream = stream if stream is not None else torch.cuda.current_stream()
         c = _Config(cfg.n_units, cfg.gqa_group, cfg.head_dim, cfg.kv_dtype, cfg.max_tokens, cfg.max_clusters,
                     cfg.kmeans_iters, cfg.init_mode, cfg.split_size_factor, cfg.split_var_factor,
-                    cfg.split_min_size, cfg.split_iters, cfg.trace, cfg.assign_mode, cfg.attn_mode, cfg.update_mode, cfg.local_max, cfg.det_sums)
+                    cfg.split_min_size, cfg.split_iters, cfg.trace, cfg.assign_mode, cfg.attn_mode, cfg.update_mode, cfg.local_max, cfg.det_sums, cfg.buf_max)
         h = C.c_void_p()
         self._check(self._L.dynakv_create(C.byref(c), C.c_void_p(self._stream.cuda_stream), C.byref(h)), "dynakv_create")
         self._h = h

@@ -140,7 +140,8 @@ extern "C" int dynakv_create(const dynakv_config* cfg, void* cuda_stream, dynakv
     if (cfg->max_tokens < 1 || cfg->max_clusters < 1 || cfg->max_clusters > 4096) return DYNAKV_ERR_ARG;
     if (cfg->kmeans_iters < 1 || cfg->split_iters < 1) return DYNAKV_ERR_ARG;
     if (cfg->init_mode != DYNAKV_INIT_KMEANSPP && cfg->init_mode != DYNAKV_INIT_RANDOM) return DYNAKV_ERR_ARG;
-    if (cfg->update_mode < DYNAKV_MODE_ADAPTIVE || cfg->update_mode > DYNAKV_MODE_LOCAL) return DYNAKV_ERR_ARG;
+    if (cfg->update_mode < DYNAKV_MODE_ADAPTIVE || cfg->update_mode > DYNAKV_MODE_DELAYED) return DYNAKV_ERR_ARG;
+    if (cfg->update_mode == DYNAKV_MODE_DELAYED && cfg->buf_max < 1) return DYNAKV_ERR_ARG;
     if (cfg->update_mode == DYNAKV_MODE_LOCAL && cfg->local_max < 2) return DYNAKV_ERR_ARG;
     dynakv_ctx* c = new (std::nothrow) dynakv_ctx();
     if (!c) return DYNAKV_ERR_NOMEM;
@@ -154,6 +155,7 @@ extern "C" int dynakv_create(const dynakv_config* cfg, void* cuda_stream, dynakv
     t.max_tokens = cfg->max_tokens; t.max_clusters = cfg->max_clusters;
     t.update_mode = cfg->update_mode; t.local_max = cfg->local_max;
     t.det_sums = cfg->det_sums ? 1 : 0;
+    t.buf_max = cfg->buf_max;
     const int full_pages = (cfg->max_tokens + PAGE - 1) / PAGE;
     int slack = full_pages / 8; if (slack < 64) slack = 64;
     t.P = full_pages + cfg->max_clusters + slack;
@@ -198,6 +200,7 @@ extern "C" int dynakv_create(const dynakv_config* cfg, void* cuda_stream, dynakv
     ALLOC(t.cl_head, U * Mx, true);
     ALLOC(t.cl_tail, U * Mx, true);
     ALLOC(t.cl_flags, U * Mx, true);
+    ALLOC(t.cl_buf, U * Mx, true);
     ALLOC(t.u_N, U, true); ALLOC(t.u_M, U, true); ALLOC(t.u_Mlive, U, true); ALLOC(t.u_tau, U, true);
     ALLOC(t.u_page_top, U, true); ALLOC(t.u_free_cnt, U, true);
     ALLOC(t.tok_cluster, U * (size_t)t.max_tokens, false);

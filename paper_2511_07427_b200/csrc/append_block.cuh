@@ -143,7 +143,9 @@ __device__ __forceinline__ void append_block(const Tables& t, int u, StepPtr kp_
         if (found) { t.u_M[u] = Mcur + 1; t.u_Mlive[u] = t.u_Mlive[u] + 1; }
         if (res) { res->cluster = bj; res->n_new = n_old + 1; res->M2_new = m2_new; res->N_new = N + 1; }
         t.cl_n[cj] = n_old + 1;
-        t.cl_flags[cj] = found ? 0 : (t.cl_flags[cj] & ~FLAG_HOLD);
+        const int fl = found ? 0 : t.cl_flags[cj];
+        t.cl_flags[cj] = (unsigned char)(fl & ~FLAG_HOLD);
+        if (fl & FLAG_SPLIT) t.cl_buf[cj] = t.cl_buf[cj] + 1;      // delayed-split mode: an entry for a flagged cluster is buffered
         t.page_tok[((size_t)u * t.P + page) * PAGE + row] = N;
         t.tok_cluster[(size_t)u * t.max_tokens + N] = bj;
         t.u_N[u] = N + 1;

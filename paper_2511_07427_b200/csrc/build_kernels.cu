@@ -341,7 +341,7 @@ __global__ void __launch_bounds__(1024) k_fin_layout(Tables t, int n, int M, con
         if (j < t.max_clusters) {
             size_t cj = (size_t)u * t.max_clusters + j;
             t.cl_n[cj] = c;
-            t.cl_flags[cj] = 0;
+            t.cl_flags[cj] = 0; t.cl_buf[cj] = 0;
             t.cl_M2[cj] = 0.f;
             t.cl_head[cj] = c > 0 ? first : -1;
             t.cl_tail[cj] = c > 0 ? first + np - 1 : -1;

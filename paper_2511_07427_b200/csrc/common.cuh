@@ -26,6 +26,7 @@ template <typename KV> struct Epc { static constexpr int v = 16 / (int)sizeof(KV
 constexpr int ENTRY_ROWS = DKV_ENTRY_ROWS;   // rows per gather work entry (16 or 32: a run inside one page)
 constexpr int MAX_G = 8;
 constexpr int FLAG_HOLD = 1;        // split abandoned; not retried until the next append
+constexpr int FLAG_SPLIT = 2;       // delayed-split mode: a split is owed (Algorithm 1's f_j)
 
 // Device-resident state of a context.  All arrays are unit-major.
 //   KV store: kpages/vpages [U][P][PAGE][d] in kv dtype; every cluster owns a chain of
@@ -35,6 +36,8 @@ struct Tables {
     int U, G, d, kv_dtype, max_tokens, max_clusters, P, n_splits_attn;
     int update_mode, local_max;      // DYNAKV_MODE_*; LOCAL: size above which a decode-born cluster splits
     int det_sums;                    // 1: centroid sums of the build in 64-bit fixed point (order-independent)
+    int buf_max;                     // delayed-split mode: buffered entries per unit that force a split
+    int* cl_buf;                     // [U][Mmax] delayed-split mode: entries buffered for a flagged cluster
     // FP8 mode (fp8 != 0): kv_dtype is DYNAKV_BF16 for every kernel, all rows lie on the e4m3-times-power-of-two grid,
     // and a one-byte copy of the pages is kept for the gather-attention kernel
     int fp8;

@@ -233,7 +233,7 @@ __device__ int split_small(const Tables& t, int u, int j, int c, int iters, KV* 
         }
         __syncthreads();
     }
-    if (abandoned) { if (tid == 0) t.cl_flags[cj] |= FLAG_HOLD; return -1; }
+    if (abandoned) { if (tid == 0) { t.cl_flags[cj] = FLAG_HOLD; t.cl_buf[cj] = 0; } return -1; }
 
     // ---- which side stays: the one holding the smallest token id
     int stay;
@@ -341,7 +341,7 @@ __device__ int split_small(const Tables& t, int u, int j, int c, int iters, KV* 
         for (int i = 0; i < need; i++) pnext[sc.newpg[i]] = (i + 1 < need) ? sc.newpg[i + 1] : -1;
         t.cl_head[cn] = sc.newpg[0]; t.cl_tail[cn] = sc.newpg[need - 1];
         t.cl_n[cj] = s_n; t.cl_n[cn] = m_n;
-        t.cl_flags[cj] = 0; t.cl_flags[cn] = 0;
+        t.cl_flags[cj] = 0; t.cl_flags[cn] = 0; t.cl_buf[cj] = 0; t.cl_buf[cn] = 0;
         t.u_M[u] = new_id + 1; t.u_Mlive[u] = mlive + 1;
         atomicAdd(&t.counters[CNT_SPLITS], 1ull);
         *sc.nsplit = *sc.nsplit + 1;

@@ -77,8 +77,9 @@ def make_ctx(cfg: WorkloadConfig, n_units: int, trace: int = 1, assign_mode: int
         init_mode=P.INIT_KMEANSPP if cfg.init_mode == "kmeanspp" else P.INIT_RANDOM,
         split_size_factor=cfg.split_size_factor, split_var_factor=cfg.split_var_factor,
         split_min_size=cfg.split_min_size, split_iters=cfg.split_iters, trace=trace, assign_mode=assign_mode, attn_mode=attn_mode,
-        update_mode={"adaptive": P.MODE_ADAPTIVE, "static": P.MODE_STATIC, "local": P.MODE_LOCAL}[cfg.update_mode],
-        local_max=cfg.local_max, det_sums=det_sums))
+        update_mode={"adaptive": P.MODE_ADAPTIVE, "static": P.MODE_STATIC, "local": P.MODE_LOCAL,
+                     "delayed": P.MODE_DELAYED}[cfg.update_mode],
+        local_max=cfg.local_max, det_sums=det_sums, buf_max=cfg.buf_max))
 
 
 def fp8_round_rows(x: "torch.Tensor") -> "torch.Tensor":
@@ -106,8 +107,9 @@ def make_oracle(cfg: WorkloadConfig) -> O.OracleUnit:
     return O.OracleUnit(cfg.d, cfg.G, cfg.max_tokens, cfg.max_clusters,
                         gamma=float(np.float32(cfg.split_size_factor)), alpha=float(np.float32(cfg.split_var_factor)),
                         split_min_size=cfg.split_min_size, split_iters=cfg.split_iters, tol=TOL_TIE,
-                        mode={"adaptive": O.MODE_ADAPTIVE, "static": O.MODE_STATIC, "local": O.MODE_LOCAL}[cfg.update_mode],
-                        local_max=cfg.local_max)
+                        mode={"adaptive": O.MODE_ADAPTIVE, "static": O.MODE_STATIC, "local": O.MODE_LOCAL,
+                              "delayed": O.MODE_DELAYED}[cfg.update_mode],
+                        local_max=cfg.local_max, buf_max=cfg.buf_max)
 
 
 def rel_l2(a: np.ndarray, b: np.ndarray) -> float:

@@ -276,6 +276,14 @@ def test_graph_loop_in_local_update_mode():
     assert _loop_vs_direct(cfg, [0, 1, 2, 3, 4], 90, cut=31) >= 5
 
 
+def test_graph_loop_in_delayed_split_mode():
+    # the tail kernel's unit blocks decide, from the step's retrieved clusters and the flags, which splits happen now,
+    # which are owed and whether the buffer limit forces one; the helper blocks split; the host-buffer step does the same
+    cfg = CONFIGS[3].scaled(n_prefill=500, steps=96, M0=12, max_clusters=256, budget=120, T=4, new_every=32,
+                            split_size_factor=1.3, split_var_factor=1.3, update_mode="delayed", buf_max=8)
+    assert _loop_vs_direct(cfg, [0, 1, 2, 3, 4], 96, cut=37) > 50
+
+
 def _loop_vs_direct(cfg, units, steps, modes=("direct", "graph", "host"), cut=None):
     """The captured loop (and the host-buffer step) must leave the same state and outputs as direct calls."""
     s = [UnitStream(cfg, u) for u in units]

@@ -167,3 +167,16 @@ def test_fp8_storage_with_clusters_too_large_to_stage():
     assert rep.splits > 0
     from test_gpu_edge import _loop_vs_direct
     assert _loop_vs_direct(cfg, [0, 1, 2], 24, modes=("direct", "graph")) > 0
+
+
+@pytest.mark.parametrize("buf_max,budget", [(1000, 120), (6, 60), (1000, 300)])
+def test_delayed_split_mode(buf_max, budget):
+    """The delayed split of Algorithm 1 (Section 4.2) against the oracle's: with a small budget most triggered clusters
+    are not among the retrieved ones, so their splits wait until a query retrieves them (buf_max 1000) or until the
+    buffered entries force them (buf_max 6); with a large budget nearly every trigger is split at once.  Membership,
+    ids, statistics and outputs must agree at every step, so every deferral and every forced split happens in the same
+    step on both sides."""
+    cfg = CONFIGS[3].scaled(n_prefill=500, steps=160, M0=12, max_clusters=256, budget=budget, T=4, new_every=64,
+                            split_size_factor=1.3, split_var_factor=1.3, update_mode="delayed", buf_max=buf_max)
+    rep = _run(cfg, [0, 1, 2], cfg.steps, assign_mode=1)
+    assert rep.splits > 20 and rep.gpu_splits >= rep.splits

@@ -41,7 +41,9 @@ def _cfg(**kw):
 
 @pytest.mark.parametrize("bad", [dict(n_units=0), dict(gqa_group=0), dict(gqa_group=9), dict(head_dim=96),
                                  dict(kv_dtype=3), dict(kv_dtype=2, head_dim=64), dict(max_tokens=0), dict(max_clusters=0), dict(max_clusters=5000),
-                                 dict(kmeans_iters=0), dict(split_iters=0), dict(init_mode=2)])
+                                 dict(kmeans_iters=0), dict(split_iters=0), dict(init_mode=2),
+                                 dict(update_mode=4), dict(update_mode=-1), dict(update_mode=2, local_max=1),
+                                 dict(update_mode=3, buf_max=0)])
 def test_create_rejects_bad_config_without_a_device(bad):
     L = P.load_library()
     h = C.c_void_p()
