@@ -96,6 +96,70 @@ __device__ int next_queued_unit(const Tables& t, int* hint) {
     }
 }
 
+// Delayed-split mode (Algorithm 1, its last two blocks): the trigger scan of one unit, by all SP_THREADS threads of its
+// block.  A cluster whose trigger fires or whose flag is owed is listed for a split now if the step's query retrieved it
+// (sel[0..L), the selection's id list); a firing trigger outside that set raises the flag, and that entry is the first
+// buffered one.  Then, if the buffered entries of the clusters left flagged reach buf_max, the one with the most of
+// them (lowest id among equals) is listed as well, after the others.  Returns the number of listed clusters (the same
+// in every thread).  Kept out of line: it runs in this mode only and must not weigh on the kernel's registers.
+__device__ __noinline__ int delayed_scan(const int* cl_n, unsigned char* cl_flags, const float* cl_M2, int* cl_buf, const int* sel, int L,
+                                         int M0, int min_size, int var_enabled, float tau, float gamma, int Mlive0, int N,
+                                         int buf_max, int* trig, int* sh, float* red_f, int* red_i, int* red_k) {
+    __shared__ unsigned int req_bits[128];     // the retrieved clusters of the step, one bit per id (ids are below 4096)
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    for (int i = tid; i < 128; i += SP_THREADS) req_bits[i] = 0u;
+    __syncthreads();
+    for (int i = tid; i < L; i += SP_THREADS) { const int j = sel[i]; if (j >= 0 && j < 4096) atomicOr(&req_bits[j >> 5], 1u << (j & 31)); }
+    __syncthreads();
+    int base = 0, buf_sum = 0, buf_best = 0, buf_id = 0x7fffffff;
+    for (int b0 = 0; b0 < M0; b0 += SP_THREADS) {
+        const int j = b0 + tid;
+        int hit = 0;
+        if (j < M0) {
+            const int c = cl_n[j];
+            const int fl = cl_flags[j];
+            if (c > 0 && c >= min_size && !(fl & FLAG_HOLD)) {
+                const bool by_var = var_enabled && (cl_M2[j] / (float)c > tau);
+                const bool by_size = gamma > 0.f && ((double)c * (double)Mlive0 > (double)gamma * (double)N);
+                hit = (by_var || by_size) ? 1 : 0;
+            }
+            const bool owed_j = c > 0 && (fl & FLAG_SPLIT);
+            const bool inreq = j < 4096 && ((req_bits[j >> 5] >> (j & 31)) & 1u);
+            int bufj = owed_j ? cl_buf[j] : 0;
+            if ((hit || owed_j) && inreq) hit = 1;
+            else {
+                if (hit && !owed_j) { cl_flags[j] = (unsigned char)(fl | FLAG_SPLIT); cl_buf[j] = 1; bufj = 1; }
+                if (hit || owed_j) {
+                    buf_sum += bufj;
+                    if (bufj > buf_best || (bufj == buf_best && j < buf_id)) { buf_best = bufj; buf_id = j; }
+                }
+                hit = 0;
+            }
+        }
+        int tot;
+        const int pos = base + block_scan_excl(hit, sh, &tot);
+        if (hit) trig[pos] = j;
+        base += tot;
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        buf_sum += __shfl_xor_sync(0xffffffffu, buf_sum, o);
+        const int ob = __shfl_xor_sync(0xffffffffu, buf_best, o), oi = __shfl_xor_sync(0xffffffffu, buf_id, o);
+        if (ob > buf_best || (ob == buf_best && oi < buf_id)) { buf_best = ob; buf_id = oi; }
+    }
+    __syncthreads();
+    if (lane == 0) { red_f[warp] = __int_as_float(buf_sum); red_i[warp] = buf_best; red_k[warp] = buf_id; }
+    __syncthreads();
+    int tot = 0, bb = 0, bi = 0x7fffffff;
+    for (int w = 0; w < SP_WARPS; w++) {
+        tot += __float_as_int(red_f[w]);
+        if (red_i[w] > bb || (red_i[w] == bb && red_k[w] < bi)) { bb = red_i[w]; bi = red_k[w]; }
+    }
+    if (bb > 0 && tot >= buf_max) { if (tid == 0) trig[base] = bi; base++; }
+    __syncthreads();
+    return base;
+}
+
 template <typename KV, int HD>
 __global__ void __launch_bounds__(SP_THREADS, DKV_SP_MINBLOCKS) k_split_check(Tables t, float gamma, int var_enabled, int min_size, int iters,
                                                             int do_append, StepPtr app_k, StepPtr app_v, int* step_ctr,
@@ -112,7 +176,6 @@ __global__ void __launch_bounds__(SP_THREADS, DKV_SP_MINBLOCKS) k_split_check(Ta
     __shared__ int sh[33];
     __shared__ int s_cnt[4];          // changed, nA, nB, misc
     __shared__ int s_a, s_ok;
-    __shared__ unsigned int req_bits[128];     // delayed-split mode: the retrieved clusters of the step, one bit per id
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     // The next kernel on the stream may be scheduled as soon as every block of this grid has started: its blocks move
@@ -167,16 +230,7 @@ __global__ void __launch_bounds__(SP_THREADS, DKV_SP_MINBLOCKS) k_split_check(Ta
         const int owed = t.u_last[u];            // an earlier append whose check is still owed (-1 in a loop's steady state)
         int full = t.u_scan[u];
         const bool delayed = t.update_mode == DYNAKV_MODE_DELAYED;
-        if (delayed) {
-            // delayed-split mode looks at every cluster at every check (flags owed from earlier checks, the buffer
-            // limit), and needs to know which clusters the step's query retrieved: one bit per cluster id
-            full = 1;
-            for (int i = tid; i < 128; i += SP_THREADS) req_bits[i] = 0u;
-            __syncthreads();
-            const int L = t.sel_n[u];
-            const int* sel = t.sel_ids + (size_t)u * t.max_clusters;
-            for (int i = tid; i < L; i += SP_THREADS) { const int j = sel[i]; if (j >= 0 && j < 4096) atomicOr(&req_bits[j >> 5], 1u << (j & 31)); }
-        }
+        if (delayed) full = 1;       // every cluster is looked at at every check (flags owed from earlier checks, the buffer limit)
         const int Mlive0 = t.u_Mlive[u];
         const float tau = t.u_tau[u];
         // fused loop iteration: the step's append for this unit comes first (Algorithm 1's order)
@@ -203,19 +257,23 @@ __global__ void __launch_bounds__(SP_THREADS, DKV_SP_MINBLOCKS) k_split_check(Ta
                 }
             }
             __syncthreads();
+        } else if (delayed) {
+            const size_t c0 = (size_t)u * t.max_clusters;
+            const int nt = delayed_scan(t.cl_n + c0, t.cl_flags + c0, t.cl_M2 + c0, t.cl_buf + c0, t.sel_ids + c0, t.sel_n[u], t.u_M[u],
+                                        min_size, var_enabled, tau, gamma, Mlive0, t.u_N[u], t.buf_max, trig, sh, red_f, red_i, red_k);
+            if (tid == 0) s_ntrig = nt;
+            __syncthreads();
         } else {
         const int N = t.u_N[u], M0 = t.u_M[u];
         int base = 0;
         const int jlim = full ? M0 : (last >= 0 ? 1 : 0);
-        int buf_sum = 0, buf_best = 0, buf_id = 0x7fffffff;       // delayed mode: buffered entries of the clusters left flagged
         for (int b0 = 0; b0 < jlim; b0 += SP_THREADS) {
             const int j = full ? b0 + tid : (tid == 0 ? last : -1);
             int hit = 0;
             if (j >= 0 && j < M0) {
                 const size_t cj = (size_t)u * t.max_clusters + j;
                 const int c = t.cl_n[cj];
-                const int fl = t.cl_flags[cj];
-                if (c > 0 && c >= min_size && !(fl & FLAG_HOLD)) {
+                if (c > 0 && c >= min_size && !(t.cl_flags[cj] & FLAG_HOLD)) {
                     if (t.update_mode == DYNAKV_MODE_LOCAL) hit = (j >= t.M_floor && c > t.local_max) ? 1 : 0;
                     else if (t.update_mode == DYNAKV_MODE_STATIC) hit = 0;
                     else {
@@ -224,48 +282,11 @@ __global__ void __launch_bounds__(SP_THREADS, DKV_SP_MINBLOCKS) k_split_check(Ta
                         hit = (by_var || by_size) ? 1 : 0;
                     }
                 }
-                if (delayed) {
-                    // Algorithm 1, delayed split: inside the retrieved set a firing trigger or an owed flag is split now;
-                    // outside it a firing trigger raises the flag, and that entry is the first buffered one
-                    const bool owed_j = c > 0 && (fl & FLAG_SPLIT);
-                    const bool inreq = j < 4096 && ((req_bits[j >> 5] >> (j & 31)) & 1u);
-                    int bufj = owed_j ? t.cl_buf[cj] : 0;
-                    if ((hit || owed_j) && inreq) hit = 1;
-                    else {
-                        if (hit && !owed_j) { t.cl_flags[cj] = (unsigned char)(fl | FLAG_SPLIT); t.cl_buf[cj] = 1; bufj = 1; }
-                        if (hit || owed_j) {
-                            buf_sum += bufj;
-                            if (bufj > buf_best || (bufj == buf_best && j < buf_id)) { buf_best = bufj; buf_id = j; }
-                        }
-                        hit = 0;
-                    }
-                }
             }
             int tot;
             const int pos = base + block_scan_excl(hit, sh, &tot);
             if (hit) trig[pos] = j;
             base += tot;
-        }
-        if (delayed) {
-            // the buffer limit: when the entries buffered for the clusters left flagged reach buf_max, the one with the
-            // most of them (lowest id among equals) is split as well, after the others
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) {
-                buf_sum += __shfl_xor_sync(0xffffffffu, buf_sum, o);
-                const int ob = __shfl_xor_sync(0xffffffffu, buf_best, o), oi = __shfl_xor_sync(0xffffffffu, buf_id, o);
-                if (ob > buf_best || (ob == buf_best && oi < buf_id)) { buf_best = ob; buf_id = oi; }
-            }
-            __syncthreads();
-            if (lane == 0) { red_f[warp] = (float)buf_sum; red_i[warp] = buf_best; red_k[warp] = buf_id; }
-            __syncthreads();
-            if (tid == 0) {
-                int tot = 0, bb = 0, bi = 0x7fffffff;
-                for (int w = 0; w < SP_WARPS; w++) {
-                    tot += (int)red_f[w];
-                    if (red_i[w] > bb || (red_i[w] == bb && red_k[w] < bi)) { bb = red_i[w]; bi = red_k[w]; }
-                }
-                if (bb > 0 && tot >= t.buf_max) trig[base++] = bi;
-            }
         }
         if (tid == 0) s_ntrig = base;
         __syncthreads();
