@@ -4,7 +4,8 @@ the dense attention mass that the budgeted retrieval keeps.
     python -m paper_2511_07427_b200.mode_report [--config 3] [--steps 8192] [--units 64] [--every 2048]
 
 For every mode (adaptive = the paper's append + split rule, static = append only, local = new entries clustered
-among themselves; arXiv 2511.07427 Section 3.1 and the baselines of Section 8.1) the same seeded stream is run
+among themselves; arXiv 2511.07427 Section 3.1 and the baselines of Section 8.1; with --buf-max also the delayed split
+of Algorithm 1, which defers a triggered cluster's split until a query retrieves it) the same seeded stream is run
 through the library's CUDA-graph decode loop.  At every checkpoint the exported state gives
 
   * the mean over live clusters of sigma_j^2 = M2_j / n_j (the scalar the paper's variance table reports per
@@ -38,7 +39,8 @@ from gen import CONFIGS, UnitStream, make_decode_chunk, make_prefill  # noqa: E4
 
 
 def run_mode(cfg, mode: str, local_max: int, units: int, steps: int, every: int):
-    name = mode if mode != "local" else f"local(max {local_max})"
+    # (for the delayed-split mode the second argument is buf_max)
+    name = f"local(max {local_max})" if mode == "local" else f"delayed(B {local_max})" if mode == "delayed" else mode
     side = torch.cuda.Stream()
     rows = []
     with torch.cuda.stream(side):
@@ -49,7 +51,8 @@ def run_mode(cfg, mode: str, local_max: int, units: int, steps: int, every: int)
             n_units=units, gqa_group=cfg.G, head_dim=cfg.d, kv_dtype=P.BF16, max_tokens=n0 + steps, max_clusters=cfg.max_clusters,
             kmeans_iters=cfg.T, init_mode=P.INIT_RANDOM, split_size_factor=cfg.split_size_factor,
             split_var_factor=cfg.split_var_factor, split_min_size=cfg.split_min_size, split_iters=cfg.split_iters,
-            update_mode={"adaptive": P.MODE_ADAPTIVE, "static": P.MODE_STATIC, "local": P.MODE_LOCAL}[mode], local_max=local_max))
+            update_mode={"adaptive": P.MODE_ADAPTIVE, "static": P.MODE_STATIC, "local": P.MODE_LOCAL,
+                         "delayed": P.MODE_DELAYED}[mode], local_max=local_max, buf_max=local_max))
         ctx.build_index(K, V, cfg.M0, 1234)
         K_all = torch.empty((units, n0 + steps, cfg.d), dtype=K.dtype, device="cuda")
         V_all = torch.empty_like(K_all)
@@ -111,9 +114,10 @@ def main():
     ap.add_argument("--units", type=int, default=64)
     ap.add_argument("--every", type=int, default=2048)
     ap.add_argument("--local-max", type=int, nargs="*", default=[64, 512])
+    ap.add_argument("--buf-max", type=int, nargs="*", default=[], help="also run the delayed-split mode with these buffer limits")
     args = ap.parse_args()
     cfg = CONFIGS[args.config]
-    runs = [("adaptive", 0), ("static", 0)] + [("local", m) for m in args.local_max]
+    runs = [("adaptive", 0), ("static", 0)] + [("local", m) for m in args.local_max] + [("delayed", b) for b in args.buf_max]
     table = []
     for mode, lm in runs:
         table += run_mode(cfg, mode, max(lm, 2), args.units, args.steps, args.every)
