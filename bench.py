@@ -306,7 +306,11 @@ def run_ours(args, cfg):
     ctx.set_timing(True)
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record()
-    ctx.build_index(Kp, Vp, cfg.M0, 1234)
+    if args.placed > 0:
+        # correlation-aware placement from the first decode queries of the stream (they are used again as decode steps)
+        ctx.build_index(Kp, Vp, cfg.M0, 1234, placement_queries=q_all[:args.placed].contiguous(), placement_budget=cfg.budget)
+    else:
+        ctx.build_index(Kp, Vp, cfg.M0, 1234)
     e1.record(); torch.cuda.synchronize()
     build_ms = e0.elapsed_time(e1)
     kt = ctx.get_kernel_times(reset=True)
@@ -472,6 +476,9 @@ def run_ours(args, cfg):
     if clocks is not None:
         clocks["sampled_during"] = "the timed repeats and the steady run of the same loop"
     status = ctx.get_status()
+    # access contiguity of the last step's gather list (rows read per run of consecutive pages of the pool)
+    from paper_2511_07427_b200.placement import mean_contiguous_rows
+    contiguous_rows = mean_contiguous_rows(*ctx.get_work_list())
     ctx.destroy()
 
     if rank == 0:
@@ -492,7 +499,8 @@ def run_ours(args, cfg):
             "counters": {"splits_in_timed_region": st1["n_splits"] - st0["n_splits"],
                          "tokens_attended_per_step": (st1["tokens_attended_total"] - st0["tokens_attended_total"]) / timed_steps,
                          "clusters_selected_per_step": (st1["clusters_selected_total"] - st0["clusters_selected_total"]) / timed_steps,
-                         "status_bits": status["error_bits"], "assign_rechecked": status["assign_rechecked"]},
+                         "status_bits": status["error_bits"], "assign_rechecked": status["assign_rechecked"],
+                         "mean_contiguous_rows_per_stretch": contiguous_rows, "placement_queries": args.placed},
         }
         print(json.dumps(line), flush=True)
     if world > 1:
@@ -510,6 +518,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--assign-mode", type=int, default=0)
     ap.add_argument("--kv", default="", choices=["", "fp8"], help="fp8: the config's bf16 K/V rows kept in FP8 storage")
+    ap.add_argument("--placed", type=int, default=0,
+                    help="build with correlation-aware placement from this many reference queries (0: clusters in id order)")
     ap.add_argument("--e2e-steps", type=int, default=160)
     ap.add_argument("--profile-steps", type=int, default=64)
     ap.add_argument("--no-cpu-baseline", action="store_true")

@@ -139,6 +139,21 @@ int dynakv_create(const dynakv_config* cfg, void* cuda_stream, dynakv_ctx** out)
 int dynakv_build_index(dynakv_ctx* ctx, const void* K, const void* V, int64_t n, int32_t d,
                        int32_t n_clusters, uint64_t seed);
 
+/* dynakv_build_index followed by the correlation-aware placement of Section 5.1 (Eq. 8): the reference queries q_ref
+ * (DEVICE, [n_ref][U][G][d] fp32 -- the paper uses the initial input) are scored and selected under token_budget on
+ * the finished index, every pair of clusters retrieved by the same query is counted (the adjacency matrix of retrieval
+ * frequencies; Eq. 8 divides it by one constant, which does not change an ordering), and the clusters' pages are
+ * laid out again so that a cluster is followed by the not yet placed cluster it was co-retrieved with most often
+ * (greedy chain from the most co-retrieved cluster; lowest id among equals).  Clusters stay contiguous page by page;
+ * only the order of the clusters in the page pool changes, so every later call gives the results it gives after
+ * dynakv_build_index.  In HBM the order of pages has no cost of its own (there is no seek, and a copy never spans two
+ * pages); the call exists so that the placement can be run and its effect on access contiguity measured
+ * (dynakv_get_work_list).  Needs n_clusters^2 * 4 bytes of scratch per unit during the call.  Counters and status
+ * word are left as a plain build leaves them. */
+int dynakv_build_index_placed(dynakv_ctx* ctx, const void* K, const void* V, int64_t n, int32_t d,
+                              int32_t n_clusters, uint64_t seed, const float* q_ref, int64_t n_ref,
+                              int32_t token_budget);
+
 /* Algorithm 1, nearest-cluster assignment of the new entry, UpdateVar, AddEntry,
  * UpdateStats: for every unit, the new key k [U][d] joins the live cluster with the
  * nearest representative; n_j, r_j, M2_j are updated incrementally and the (k, v) row is
@@ -228,6 +243,12 @@ int dynakv_import_state(dynakv_ctx* ctx, const void* K, const void* V, int64_t n
 /* Synchronises and copies the last decode step's selection sizes to HOST arrays:
  * n_selected [U], tokens_selected [U]; either may be NULL. */
 int dynakv_get_selection(dynakv_ctx* ctx, int32_t* n_selected, int32_t* tokens_selected);
+
+/* The last decode step's gather list, to HOST arrays: n_entries [U] and, if entries is not NULL, entries
+ * [U][entries_per_unit][2] = (first row in the unit's page pool, rows <= 32) of every run of rows the attention kernel
+ * copied, in the order it took them; entries_per_unit >= dynakv_work_list_capacity(ctx).  Synchronises. */
+int dynakv_get_work_list(dynakv_ctx* ctx, int32_t* n_entries, int32_t* entries, int64_t entries_per_unit);
+int dynakv_work_list_capacity(dynakv_ctx* ctx);
 
 /* With cfg.trace = 1: HOST arrays picks [U][n_clusters] (token ids chosen as initial
  * centres, in centre order) and assign [T][U][n] (assignment of every Lloyd round);

@@ -21,6 +21,7 @@ EXPORTED_SYMBOLS = [
     "dynakv_decode_loop", "dynakv_step_host", "dynakv_get_status", "dynakv_export_state", "dynakv_get_selection",
     "dynakv_get_build_trace", "dynakv_set_timing", "dynakv_get_kernel_times", "dynakv_launch_count", "dynakv_last_error", "dynakv_destroy",
     "dynakv_attend_rows_noalloc", "dynakv_export_kv", "dynakv_import_state", "dynakv_decode_loop_host", "dynakv_selftest_wait_expiry", "dynakv_time_gather_attention",
+    "dynakv_build_index_placed", "dynakv_get_work_list", "dynakv_work_list_capacity",
 ]
 ERR_TOO_LARGE = -5
 NOALLOC_SCRATCH_BYTES = 4 * 1024 * 1024
@@ -87,6 +88,12 @@ def load_library() -> C.CDLL:
     L.dynakv_create.argtypes = [C.POINTER(_Config), vp, C.POINTER(vp)]
     L.dynakv_build_index.restype = C.c_int
     L.dynakv_build_index.argtypes = [vp, vp, vp, i64, i32, i32, u64]
+    L.dynakv_build_index_placed.restype = C.c_int
+    L.dynakv_build_index_placed.argtypes = [vp, vp, vp, i64, i32, i32, u64, vp, i64, i32]
+    L.dynakv_get_work_list.restype = C.c_int
+    L.dynakv_get_work_list.argtypes = [vp, vp, vp, i64]
+    L.dynakv_work_list_capacity.restype = C.c_int
+    L.dynakv_work_list_capacity.argtypes = [vp]
     L.dynakv_append.restype = C.c_int
     L.dynakv_append.argtypes = [vp, vp, vp]
     L.dynakv_decode_step.restype = C.c_int
@@ -214,12 +221,20 @@ class DynaKV:
         return C.c_void_p(t.data_ptr())
 
     # ---- the C ABI, one method per entry point
-    def build_index(self, K, V, n_clusters: int, seed: int) -> None:
+    def build_index(self, K, V, n_clusters: int, seed: int, placement_queries=None, placement_budget: int = 0) -> None:
+        """placement_queries ([n_ref, U, G, d] fp32 on the device) selects the build with correlation-aware placement:
+        the clusters' pages are ordered by how often the reference queries retrieve clusters together."""
         U, d = self.cfg.n_units, self.cfg.head_dim
         n = K.shape[1]
         assert K.is_cuda and V.is_cuda
-        self._check(self._L.dynakv_build_index(self._h, self._kv(K, (U, n, d)), self._kv(V, (U, n, d)), n, d,
-                                               n_clusters, seed), "dynakv_build_index")
+        if placement_queries is None:
+            self._check(self._L.dynakv_build_index(self._h, self._kv(K, (U, n, d)), self._kv(V, (U, n, d)), n, d,
+                                                   n_clusters, seed), "dynakv_build_index")
+        else:
+            qr = placement_queries
+            self._check(self._L.dynakv_build_index_placed(
+                self._h, self._kv(K, (U, n, d)), self._kv(V, (U, n, d)), n, d, n_clusters, seed,
+                self._f32(qr, (qr.shape[0], U, self.cfg.gqa_group, d)), qr.shape[0], placement_budget), "dynakv_build_index_placed")
         self.n_prefill, self.n_clusters0 = n, n_clusters
 
     def append(self, k, v) -> None:
@@ -335,6 +350,15 @@ class DynaKV:
         a, b = np.empty(U, np.int32), np.empty(U, np.int32)
         self._check(self._L.dynakv_get_selection(self._h, _np_ptr(a), _np_ptr(b)), "dynakv_get_selection")
         return a, b
+
+    def get_work_list(self):
+        """The last decode step's gather list: (n_entries [U], entries [U, W, 2] = first row in the unit's page pool and
+        row count of every run the attention kernel copied)."""
+        U = self.cfg.n_units
+        W = self._L.dynakv_work_list_capacity(self._h)
+        n = np.empty(U, np.int32); e = np.empty((U, W, 2), np.int32)
+        self._check(self._L.dynakv_get_work_list(self._h, _np_ptr(n), _np_ptr(e), W), "dynakv_get_work_list")
+        return n, e
 
     def get_build_trace(self):
         U, T = self.cfg.n_units, self.cfg.kmeans_iters

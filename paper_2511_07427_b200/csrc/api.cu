@@ -263,8 +263,8 @@ extern "C" void dynakv_destroy(dynakv_ctx* c) {
     delete c;
 }
 
-extern "C" int dynakv_build_index(dynakv_ctx* c, const void* K, const void* V, int64_t n, int32_t d,
-                                  int32_t n_clusters, uint64_t seed) {
+static int build_index_impl(dynakv_ctx* c, const void* K, const void* V, int64_t n, int32_t d, int32_t n_clusters,
+                            uint64_t seed, const float* q_ref, int64_t n_ref, int32_t ref_budget) {
     if (!c || !K || !V) return DYNAKV_ERR_ARG;
     if (c->built) return DYNAKV_ERR_STATE;
     Tables& t = c->t;
@@ -308,6 +308,31 @@ extern "C" int dynakv_build_index(dynakv_ctx* c, const void* K, const void* V, i
         { TimeScope ts(c, KC_UPDATE); launch_update(t, K, n, M, b.assign, b, c->stream, &c->launches); }
     }
     { TimeScope ts(c, KC_FINALIZE); launch_finalize(t, K, V, n, M, b, c->cfg.split_var_factor, c->stream, &c->launches); }
+    if (q_ref && n_ref > 0) {
+        // Correlation-aware placement (Section 5.1): the reference queries are run through the scoring and the
+        // selection on the index as it stands, every pair of clusters retrieved together is counted, a placement
+        // order is derived from the counts, and the pages are laid out once more in that order.  Counters and status
+        // word are put back afterwards: the reference queries are not decode steps.
+        unsigned int* f = nullptr; int* order = nullptr;
+        ALLOC_B(f, U * (size_t)M * M, true);
+        ALLOC_B(order, U * M, false);
+        unsigned long long cnt_save[8]; unsigned int st_save = 0;
+        CK(cudaStreamSynchronize(c->stream));
+        CK(cudaMemcpy(cnt_save, t.counters, sizeof(cnt_save), cudaMemcpyDeviceToHost));
+        CK(cudaMemcpy(&st_save, t.status, sizeof(st_save), cudaMemcpyDeviceToHost));
+        t.M_floor = M;
+        const long long qs = (long long)t.U * t.G * t.d * 4;
+        for (int64_t r = 0; r < n_ref; r++) {
+            launch_front(t, StepPtr{(const char*)q_ref + r * qs, 0, nullptr}, StepPtr{nullptr, 0, nullptr}, 1, 0, c->stream, &c->launches);
+            launch_select(t, ref_budget, nullptr, c->stream, &c->launches);
+            launch_pair_count(t, M, f, c->stream, &c->launches);
+        }
+        launch_place_order(t, M, f, order, c->stream, &c->launches);
+        { TimeScope ts(c, KC_FINALIZE); launch_finalize(t, K, V, n, M, b, c->cfg.split_var_factor, c->stream, &c->launches, order); }
+        CK(cudaStreamSynchronize(c->stream));
+        CK(cudaMemcpy(t.counters, cnt_save, sizeof(cnt_save), cudaMemcpyHostToDevice));
+        CK(cudaMemcpy(t.status, &st_save, sizeof(st_save), cudaMemcpyHostToDevice));
+    }
     CK(cudaGetLastError());
     CK(cudaStreamSynchronize(c->stream));
     // keep the picks for the trace; free the rest of the build scratch
@@ -365,6 +390,19 @@ static void enqueue_loop_iteration(dynakv_ctx* c, StepPtr q, StepPtr k, StepPtr 
     enqueue_retrieve(c, q, budget, out, nullptr, false);
     launch_append_split(c->t, c->cfg.split_size_factor, c->cfg.split_var_factor > 0.f ? 1 : 0, c->cfg.split_min_size,
                         c->cfg.split_iters, 1, k, v, c->step_ctr, NextFront{1, q, k, c->step_lim}, c->stream, &c->launches);
+}
+
+
+extern "C" int dynakv_build_index(dynakv_ctx* c, const void* K, const void* V, int64_t n, int32_t d,
+                                  int32_t n_clusters, uint64_t seed) {
+    return build_index_impl(c, K, V, n, d, n_clusters, seed, nullptr, 0, 0);
+}
+
+extern "C" int dynakv_build_index_placed(dynakv_ctx* c, const void* K, const void* V, int64_t n, int32_t d,
+                                         int32_t n_clusters, uint64_t seed, const float* q_ref, int64_t n_ref,
+                                         int32_t token_budget) {
+    if (!q_ref || n_ref < 1 || token_budget < 0) return DYNAKV_ERR_ARG;
+    return build_index_impl(c, K, V, n, d, n_clusters, seed, q_ref, n_ref, token_budget);
 }
 
 extern "C" int dynakv_decode_step(dynakv_ctx* c, const float* q, int32_t token_budget, float* out, int32_t* selected_ids) {
@@ -720,6 +758,21 @@ extern "C" int dynakv_get_selection(dynakv_ctx* c, int32_t* n_selected, int32_t*
     CK(cudaStreamSynchronize(c->stream));
     return DYNAKV_OK;
 }
+
+extern "C" int dynakv_get_work_list(dynakv_ctx* c, int32_t* n_entries, int32_t* entries, int64_t entries_per_unit) {
+    if (!c || !n_entries) return DYNAKV_ERR_ARG;
+    if (!c->built) return DYNAKV_ERR_STATE;
+    const Tables& t = c->t;
+    if (entries && entries_per_unit < t.W) return DYNAKV_ERR_ARG;
+    CK(cudaMemcpyAsync(n_entries, t.n_work, sizeof(int) * t.U, cudaMemcpyDeviceToHost, c->stream));
+    if (entries)
+        CK(cudaMemcpy2DAsync(entries, (size_t)entries_per_unit * 8, t.work, (size_t)t.W * 8, (size_t)t.W * 8, t.U,
+                             cudaMemcpyDeviceToHost, c->stream));
+    CK(cudaStreamSynchronize(c->stream));
+    return DYNAKV_OK;
+}
+
+extern "C" int dynakv_work_list_capacity(dynakv_ctx* c) { return c ? c->t.W : DYNAKV_ERR_ARG; }
 
 extern "C" int dynakv_get_build_trace(dynakv_ctx* c, int32_t* picks, int32_t* assign) {
     if (!c) return DYNAKV_ERR_ARG;

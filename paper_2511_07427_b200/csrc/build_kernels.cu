@@ -324,8 +324,10 @@ __global__ void k_centroid_div(float* __restrict__ C, const float* __restrict__ 
 
 // One block per unit: page chains for every non-empty cluster (consecutive pages at build
 // time), per-unit counters, cursors zeroed.
+// `order` (optional, [U][M]): the clusters of the build in the order in which their pages follow one another in the
+// pool (correlation-aware placement, Section 5.1); without it they follow one another by id.
 __global__ void __launch_bounds__(1024) k_fin_layout(Tables t, int n, int M, const int* __restrict__ counts,
-                                                     int* __restrict__ cursor) {
+                                                     int* __restrict__ cursor, const int* __restrict__ order) {
     const int u = blockIdx.x, tid = threadIdx.x;
     __shared__ int sh[33];
     __shared__ int s_live;
@@ -333,7 +335,8 @@ __global__ void __launch_bounds__(1024) k_fin_layout(Tables t, int n, int M, con
     __syncthreads();
     int page_base = 0, live = 0;
     for (int base = 0; base < t.max_clusters; base += blockDim.x) {
-        int j = base + tid;
+        const int pos = base + tid;                                   // position in the pool's order
+        int j = (order && pos < M) ? order[(size_t)u * M + pos] : pos;
         int c = (j < M) ? counts[(size_t)u * M + j] : 0;
         int np = (c + PAGE - 1) / PAGE;
         int tot;
@@ -601,8 +604,8 @@ void launch_update(const Tables& t, const void* K, long long n, int M, const int
 
 template <typename KV, int HD>
 static void finalize_t(const Tables& t, const void* K, const void* V, long long n, int M, const BuildScratch& b,
-                       float alpha, cudaStream_t s, long long* launches) {
-    k_fin_layout<<<t.U, 1024, 0, s>>>(t, (int)n, M, b.counts, b.cursor);
+                       float alpha, const int* order, cudaStream_t s, long long* launches) {
+    k_fin_layout<<<t.U, 1024, 0, s>>>(t, (int)n, M, b.counts, b.cursor, order);
     long long total = (long long)t.U * n;
     long long blocks = (total + 7) / 8;
     if (blocks > 148LL * 64) blocks = 148LL * 64;
@@ -614,8 +617,81 @@ static void finalize_t(const Tables& t, const void* K, const void* V, long long 
 }
 
 void launch_finalize(const Tables& t, const void* K, const void* V, long long n, int M, const BuildScratch& b,
-                     float alpha, cudaStream_t s, long long* launches) {
-    DKV_DISPATCH(finalize_t, t, K, V, n, M, b, alpha, s, launches);
+                     float alpha, cudaStream_t s, long long* launches, const int* order) {
+    DKV_DISPATCH(finalize_t, t, K, V, n, M, b, alpha, order, s, launches);
+}
+
+// ------------------------------------------------------------------ correlation-aware placement (Section 5.1, Eq. 8)
+
+// One block per unit, after a selection: every pair of clusters the query retrieved together is counted once, in both
+// directions of the unit's M x M frequency matrix f (the adjacency matrix of retrieval frequencies).
+__global__ void __launch_bounds__(256) k_pair_count(Tables t, int M, unsigned int* __restrict__ f) {
+    const int u = blockIdx.x;
+    const int L = t.sel_n[u];
+    const int* sel = t.sel_ids + (size_t)u * t.max_clusters;
+    unsigned int* fu = f + (size_t)u * M * M;
+    for (int p = threadIdx.x; p < L * L; p += blockDim.x) {
+        const int a = sel[p / L], b = sel[p % L];
+        if (a != b && a < M && b < M) atomicAdd(&fu[(size_t)a * M + b], 1u);
+    }
+}
+
+// One block per unit: a placement order from the frequencies.  The co-retrieval probability of Eq. 8 is f divided by
+// one constant per unit, so ordering by f is ordering by it.  The order is a greedy chain: it starts at the cluster
+// that was co-retrieved most often in all, and every next cluster is the one not yet placed that was co-retrieved
+// most often with the one just placed (lowest id among equals; the lowest unplaced id when none ever was).
+__global__ void __launch_bounds__(256) k_place_order(int M, const unsigned int* __restrict__ f, int* __restrict__ order) {
+    const int u = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const unsigned int* fu = f + (size_t)u * M * M;
+    int* ou = order + (size_t)u * M;
+    __shared__ unsigned int placed[128];           // one bit per cluster id (ids are below 4096)
+    __shared__ unsigned long long best_s[8];
+    __shared__ int cur_s;
+    for (int i = tid; i < 128; i += 256) placed[i] = 0u;
+    // key of a candidate: (frequency, then the lower id) as one 64-bit value to maximise
+    auto key = [](unsigned long long freq, int id) -> unsigned long long { return (freq << 32) | (unsigned)(0x7fffffff - id); };
+    auto block_max = [&](unsigned long long k) -> unsigned long long {
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) { const unsigned long long y = __shfl_xor_sync(0xffffffffu, k, o); if (y > k) k = y; }
+        __syncthreads();
+        if (lane == 0) best_s[warp] = k;
+        __syncthreads();
+        unsigned long long r = best_s[0];
+#pragma unroll
+        for (int w = 1; w < 8; w++) if (best_s[w] > r) r = best_s[w];
+        return r;
+    };
+    __syncthreads();
+    // start: the largest row sum
+    unsigned long long k0 = 0;
+    for (int j = tid; j < M; j += 256) {
+        unsigned long long sum = 0;
+        for (int i = 0; i < M; i++) sum += fu[(size_t)j * M + i];
+        const unsigned long long kj = key(sum > 0xffffffffull ? 0xffffffffull : sum, j);
+        if (kj > k0) k0 = kj;
+    }
+    int cur = 0x7fffffff - (int)(block_max(k0) & 0xffffffffull);
+    for (int p = 0; p < M; p++) {
+        if (tid == 0) { ou[p] = cur; placed[cur >> 5] |= 1u << (cur & 31); }
+        __syncthreads();
+        if (p + 1 == M) break;
+        unsigned long long kb = 0;
+        for (int j = tid; j < M; j += 256) {
+            if ((placed[j >> 5] >> (j & 31)) & 1u) continue;
+            const unsigned long long kj = key(fu[(size_t)cur * M + j], j) | (1ull << 63);      // any unplaced id beats "none"
+            if (kj > kb) kb = kj;
+        }
+        cur = 0x7fffffff - (int)(block_max(kb) & 0xffffffffull);
+    }
+}
+
+void launch_pair_count(const Tables& t, int M, unsigned int* f, cudaStream_t s, long long* launches) {
+    k_pair_count<<<t.U, 256, 0, s>>>(t, M, f);
+    (*launches)++;
+}
+void launch_place_order(const Tables& t, int M, const unsigned int* f, int* order, cudaStream_t s, long long* launches) {
+    k_place_order<<<t.U, 256, 0, s>>>(M, f, order);
+    (*launches)++;
 }
 
 void launch_export_rows(const Tables& t, void* K, void* V, long long n, cudaStream_t s, long long* launches) {

@@ -213,7 +213,9 @@ void launch_assign_f32_listed(const Tables& t, const void* K, long long n, int M
 void launch_update(const Tables& t, const void* K, long long n, int M, const int* assign, const BuildScratch& b,
                    cudaStream_t s, long long* launches);
 void launch_finalize(const Tables& t, const void* K, const void* V, long long n, int M, const BuildScratch& b,
-                     float alpha, cudaStream_t s, long long* launches);
+                     float alpha, cudaStream_t s, long long* launches, const int* order = nullptr);
+void launch_pair_count(const Tables& t, int M, unsigned int* f, cudaStream_t s, long long* launches);
+void launch_place_order(const Tables& t, int M, const unsigned int* f, int* order, cudaStream_t s, long long* launches);
 // What the stand-alone centroid pass does in addition when it opens a captured loop: it resets the device-side
 // step index and the hand-over words of the loop's tail kernel, and stores the caller's arrays where the
 // captured kernels look them up.

@@ -145,7 +145,7 @@ def check_state(o: O.OracleUnit, st: dict, ui: int, rep: ParityReport, where: st
 def run_parity(cfg: WorkloadConfig, units: Sequence[int], steps: int, *, assign_mode: int = 0,
                state_every: int = 1, budget: Optional[int] = None, ctx_units: Optional[Sequence[int]] = None,
                seed: int = 1234, device: str = "cuda", check_every: int = 1, attn_mode: int = 0,
-               det_sums: int = 0) -> ParityReport:
+               det_sums: int = 0, placement_queries: int = 0) -> ParityReport:
     """Run `steps` decode iterations of `cfg`.  The GPU context holds `ctx_units` (default:
     `units`); the oracle follows the units listed in `units` (a subset of ctx_units).  With check_every > 1 the
     split check is called only after every check_every-th append (on both sides)."""
@@ -157,7 +157,13 @@ def run_parity(cfg: WorkloadConfig, units: Sequence[int], steps: int, *, assign_
     streams = [UnitStream(cfg, u) for u in ctx_units]
     K, V = make_prefill(streams)
     ctx = make_ctx(cfg, len(ctx_units), trace=1, assign_mode=assign_mode, attn_mode=attn_mode, det_sums=det_sums)
-    ctx.build_index(K.to(device), V.to(device), cfg.M0, seed)
+    if placement_queries > 0:
+        # the build with correlation-aware placement: the pages' order in the pool changes, nothing else may
+        g = torch.Generator().manual_seed(99)
+        q_ref = torch.randn((placement_queries, len(ctx_units), cfg.G, cfg.d), generator=g).to(device)
+        ctx.build_index(K.to(device), V.to(device), cfg.M0, seed, placement_queries=q_ref, placement_budget=budget)
+    else:
+        ctx.build_index(K.to(device), V.to(device), cfg.M0, seed)
     picks, trace = ctx.get_build_trace()
     st = ctx.export_state()
     oracles = {}

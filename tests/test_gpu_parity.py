@@ -180,3 +180,45 @@ def test_delayed_split_mode(buf_max, budget):
                             split_size_factor=1.3, split_var_factor=1.3, update_mode="delayed", buf_max=buf_max)
     rep = _run(cfg, [0, 1, 2], cfg.steps, assign_mode=1)
     assert rep.splits > 20 and rep.gpu_splits >= rep.splits
+
+
+def test_correlation_aware_placement_changes_nothing_but_the_page_order():
+    """dynakv_build_index_placed against the oracle: the partition, the statistics and every decode result are those of
+    a plain build (the oracle knows nothing of pages); splits and appends work on the re-ordered pool."""
+    base = CONFIGS[2]
+    cfg = base.scaled(n_prefill=1111, steps=64, M0=37, max_clusters=160, budget=300, T=6, split_size_factor=1.3)
+    rep = _run(cfg, [0, 1, 2], cfg.steps, assign_mode=1, placement_queries=24)
+    assert rep.splits > 0
+
+
+def test_correlation_aware_placement_lengthens_contiguous_access():
+    """Queries near the mixture components' means retrieve the same few clusters together again and again; placing the
+    clusters by those co-retrieval counts (Section 5.1, Eq. 8) must lengthen the contiguous stretches of the page pool
+    that a step reads, measured on queries the placement has not seen, and must leave the outputs alone."""
+    from gen import UnitStream, make_decode_chunk, make_prefill
+    from parity_harness import make_ctx
+    from paper_2511_07427_b200.placement import mean_contiguous_rows
+    cfg = CONFIGS[2].scaled(B=1, L=1, n_prefill=4096, steps=128, M0=128, max_clusters=256, budget=512, T=6)
+    U = 8
+    streams = [UnitStream(cfg, u) for u in range(U)]
+    K, V = make_prefill(streams)
+    q, _, _ = make_decode_chunk(streams, 128)
+    q = q.cuda()
+    res = {}
+    for placed in (False, True):
+        ctx = make_ctx(cfg, U, trace=0, assign_mode=1)
+        if placed:
+            ctx.build_index(K.cuda(), V.cuda(), cfg.M0, 5, placement_queries=q[:64].contiguous(), placement_budget=cfg.budget)
+        else:
+            ctx.build_index(K.cuda(), V.cuda(), cfg.M0, 5)
+        runs, outs = [], []
+        for t in range(64, 128):
+            outs.append(ctx.decode_step(q[t], cfg.budget).clone())
+            runs.append(mean_contiguous_rows(*ctx.get_work_list()))
+        st = ctx.export_state()
+        res[placed] = (float(np.mean(runs)), torch.stack(outs), st["tok_cluster"].copy(), ctx.get_status()["error_bits"])
+        ctx.destroy()
+    print(f"\nmean contiguous rows per stretch: id order {res[False][0]:.1f}, placed {res[True][0]:.1f}")
+    assert np.array_equal(res[False][2], res[True][2]) and res[True][3] == res[False][3]
+    assert (res[False][1] - res[True][1]).abs().max().item() <= 1e-4
+    assert res[True][0] >= 1.15 * res[False][0]
