@@ -298,7 +298,8 @@ def run_ours(args, cfg):
         max_tokens=cfg.max_tokens, max_clusters=cfg.max_clusters, kmeans_iters=cfg.T,
         init_mode=P.INIT_KMEANSPP if cfg.init_mode == "kmeanspp" else P.INIT_RANDOM,
         split_size_factor=cfg.split_size_factor, split_var_factor=cfg.split_var_factor,
-        split_min_size=cfg.split_min_size, split_iters=cfg.split_iters, trace=0, assign_mode=args.assign_mode))
+        split_min_size=cfg.split_min_size, split_iters=cfg.split_iters, trace=0, assign_mode=args.assign_mode,
+        tier=1 if args.tier > 0 else 0, cache_pages=args.tier))
 
     # device memory the context holds (page pool, index, scratch), from the driver's free-memory figure
     context_gb = (free_before - torch.cuda.mem_get_info(dev)[0]) / 1e9
@@ -478,7 +479,18 @@ def run_ours(args, cfg):
     status = ctx.get_status()
     # access contiguity of the last step's gather list (rows read per run of consecutive pages of the pool)
     from paper_2511_07427_b200.placement import mean_contiguous_rows
-    contiguous_rows = mean_contiguous_rows(*ctx.get_work_list())
+    # (two-tier runs: the list names cache frames, whose order says nothing about the pool's)
+    contiguous_rows = None if args.tier > 0 else mean_contiguous_rows(*ctx.get_work_list())
+    tier = None
+    if args.tier > 0:
+        tier = ctx.get_tier_stats()
+        tier["cache_pages_per_unit"] = args.tier
+        tier["pool_pages_per_unit_in_use"] = status["pages_in_use"] / U
+        n_decode = max(pos, 1)
+        tier["pages_fetched_per_step"] = tier["pages_fetched"] / n_decode
+        tier["host_to_device_mb_per_step"] = tier["pages_fetched"] * 32 * cfg.d * 2 * (4 if cfg.kv_dtype == "f32" else 2) / n_decode / 1e6
+        looked_up = tier["clusters_hit"] + tier["clusters_refreshed"] + tier["clusters_fetched"]
+        tier["cluster_hit_rate"] = (tier["clusters_hit"] + tier["clusters_refreshed"]) / max(looked_up, 1)
     ctx.destroy()
 
     if rank == 0:
@@ -502,6 +514,9 @@ def run_ours(args, cfg):
                          "status_bits": status["error_bits"], "assign_rechecked": status["assign_rechecked"],
                          "mean_contiguous_rows_per_stretch": contiguous_rows, "placement_queries": args.placed},
         }
+        if tier is not None:
+            line["tier"] = tier
+            line["config"]["two_tier_cache_pages"] = args.tier
         print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()
@@ -520,6 +535,8 @@ def main():
     ap.add_argument("--kv", default="", choices=["", "fp8"], help="fp8: the config's bf16 K/V rows kept in FP8 storage")
     ap.add_argument("--placed", type=int, default=0,
                     help="build with correlation-aware placement from this many reference queries (0: clusters in id order)")
+    ap.add_argument("--tier", type=int, default=0,
+                    help="two-tier mode: the page pool in pinned host memory and this many 32-token page frames per unit in HBM")
     ap.add_argument("--e2e-steps", type=int, default=160)
     ap.add_argument("--profile-steps", type=int, default=64)
     ap.add_argument("--no-cpu-baseline", action="store_true")

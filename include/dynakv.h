@@ -58,6 +58,8 @@ extern "C" {
 #define DYNAKV_ST_MAX_TOKENS 4u       /* an append was dropped: unit holds max_tokens            */
 #define DYNAKV_ST_PAGE_POOL 8u        /* a split or append was skipped: no free page             */
 #define DYNAKV_ST_INTERNAL 16u        /* an internal bound was hit (bounded wait ran out, ...)   */
+#define DYNAKV_ST_TIER_CACHE 32u      /* two-tier mode: a step's clusters did not fit a unit's cache; that unit's output
+                                         of the step is meaningless                              */
 
 typedef struct dynakv_ctx dynakv_ctx;
 
@@ -87,6 +89,13 @@ typedef struct dynakv_config {
                                   in arrival order (last bits of the centroids may differ between runs)             */
     int32_t buf_max;           /* DYNAKV_MODE_DELAYED: B_max of Algorithm 1, per unit -- entries buffered for flagged
                                   clusters that force a split (>= 1)                                                  */
+    int32_t tier;              /* 1: two memory tiers (Section 6; Section 7 on CPU-GPU platforms).  The page pool lives in
+                                  pinned host memory; device memory holds a cache of cache_pages page frames per unit.
+                                  Each step's selected clusters are brought into the cache whole before the attention
+                                  reads them, replacing whole clusters (Section 6.2); results are those of tier = 0.
+                                  F32 / BF16 only                                                                      */
+    int32_t cache_pages;       /* tier = 1: 32-token page frames per unit in device memory; must hold the clusters of
+                                  any one step (about token_budget / 32 plus one per selected cluster)                */
 } dynakv_config;
 
 /* How the partition follows the decode stream (Section 3.1; the baselines of Section 8.1):
@@ -119,6 +128,21 @@ typedef struct dynakv_status {
     int64_t tokens_attended_total;   /* tokens attended, summed over units and all decode steps  */
     int64_t clusters_selected_total; /* clusters selected, summed over units and all decode steps */
 } dynakv_status;
+
+/* Counters of the two-tier mode since dynakv_create, summed over units (dynakv_get_tier_stats):
+ * a selected cluster is a hit (its copy in the cache is current), refreshed (it only took appends since it was copied:
+ * the pages from its former last page on are copied) or fetched (all its pages are copied); evicted counts clusters
+ * that made room, dropped_stale copies made void by a split. */
+typedef struct dynakv_tier_stats {
+    int64_t pages_fetched;
+    int64_t clusters_hit;
+    int64_t clusters_fetched;
+    int64_t clusters_refreshed;
+    int64_t clusters_evicted;
+    int64_t copies_dropped_stale;
+    int64_t frames_in_use;     /* now, summed over units */
+    int64_t frames_total;      /* n_units * cache_pages  */
+} dynakv_tier_stats;
 
 /* Create a context on the current CUDA device; all later work runs on `cuda_stream`
  * (a cudaStream_t passed as void*, NULL = the legacy default stream).  Allocates the
@@ -246,8 +270,17 @@ int dynakv_get_selection(dynakv_ctx* ctx, int32_t* n_selected, int32_t* tokens_s
 
 /* The last decode step's gather list, to HOST arrays: n_entries [U] and, if entries is not NULL, entries
  * [U][entries_per_unit][2] = (first row in the unit's page pool, rows <= 32) of every run of rows the attention kernel
- * copied, in the order it took them; entries_per_unit >= dynakv_work_list_capacity(ctx).  Synchronises. */
+ * copied, in the order it took them; entries_per_unit >= dynakv_work_list_capacity(ctx).  With tier = 1 the rows are
+ * rows of the unit's cache frames.  Synchronises. */
 int dynakv_get_work_list(dynakv_ctx* ctx, int32_t* n_entries, int32_t* entries, int64_t entries_per_unit);
+
+/* Two-tier mode: the cache counters (HOST struct).  DYNAKV_ERR_STATE when the context has tier = 0.  Synchronises.
+ * Section 6.2 defines the replacement policy by two principles (small clusters are the ones worth caching; recently
+ * updated clusters are retained); the order this library evicts in: copies made void by a split, then clusters
+ * unchanged since they were copied -- more pages first, the longest unused first among equals, then the lowest id --
+ * then clusters that took appends since.  Clusters the current step selected are never evicted. */
+int dynakv_get_tier_stats(dynakv_ctx* ctx, dynakv_tier_stats* host_out);
+
 int dynakv_work_list_capacity(dynakv_ctx* ctx);
 
 /* With cfg.trace = 1: HOST arrays picks [U][n_clusters] (token ids chosen as initial
@@ -283,7 +316,8 @@ int dynakv_time_gather_attention(dynakv_ctx* ctx, const float* q, float* out, in
 #define DYNAKV_KC_APPEND 7
 #define DYNAKV_KC_SPLIT 8
 #define DYNAKV_KC_FRONT 9
-#define DYNAKV_KC_COUNT 10
+#define DYNAKV_KC_TIER 10       /* two-tier mode: cache bookkeeping and the page copies of a step */
+#define DYNAKV_KC_COUNT 11
 int dynakv_set_timing(dynakv_ctx* ctx, int32_t on);
 int dynakv_get_kernel_times(dynakv_ctx* ctx, double* ms_total, int64_t* launches, int32_t reset);
 

@@ -14,14 +14,14 @@ _LIB_PATH = os.path.join(_HERE, "libdynakv.so")
 F32, BF16, FP8 = 0, 1, 2
 INIT_KMEANSPP, INIT_RANDOM = 0, 1
 MODE_ADAPTIVE, MODE_STATIC, MODE_LOCAL, MODE_DELAYED = 0, 1, 2, 3
-ST_BUDGET_EXCEEDED, ST_MAX_CLUSTERS, ST_MAX_TOKENS, ST_PAGE_POOL, ST_INTERNAL = 1, 2, 4, 8, 16
+ST_BUDGET_EXCEEDED, ST_MAX_CLUSTERS, ST_MAX_TOKENS, ST_PAGE_POOL, ST_INTERNAL, ST_TIER_CACHE = 1, 2, 4, 8, 16, 32
 
 EXPORTED_SYMBOLS = [
     "dynakv_create", "dynakv_build_index", "dynakv_append", "dynakv_decode_step", "dynakv_split_check",
     "dynakv_decode_loop", "dynakv_step_host", "dynakv_get_status", "dynakv_export_state", "dynakv_get_selection",
     "dynakv_get_build_trace", "dynakv_set_timing", "dynakv_get_kernel_times", "dynakv_launch_count", "dynakv_last_error", "dynakv_destroy",
     "dynakv_attend_rows_noalloc", "dynakv_export_kv", "dynakv_import_state", "dynakv_decode_loop_host", "dynakv_selftest_wait_expiry", "dynakv_time_gather_attention",
-    "dynakv_build_index_placed", "dynakv_get_work_list", "dynakv_work_list_capacity",
+    "dynakv_build_index_placed", "dynakv_get_work_list", "dynakv_work_list_capacity", "dynakv_get_tier_stats",
 ]
 ERR_TOO_LARGE = -5
 NOALLOC_SCRATCH_BYTES = 4 * 1024 * 1024
@@ -36,7 +36,8 @@ class _Config(C.Structure):
                 ("max_tokens", C.c_int32), ("max_clusters", C.c_int32), ("kmeans_iters", C.c_int32),
                 ("init_mode", C.c_int32), ("split_size_factor", C.c_float), ("split_var_factor", C.c_float),
                 ("split_min_size", C.c_int32), ("split_iters", C.c_int32), ("trace", C.c_int32),
-                ("assign_mode", C.c_int32), ("attn_mode", C.c_int32), ("update_mode", C.c_int32), ("local_max", C.c_int32), ("det_sums", C.c_int32), ("buf_max", C.c_int32)]
+                ("assign_mode", C.c_int32), ("attn_mode", C.c_int32), ("update_mode", C.c_int32), ("local_max", C.c_int32), ("det_sums", C.c_int32), ("buf_max", C.c_int32),
+                ("tier", C.c_int32), ("cache_pages", C.c_int32)]
 
 
 class _Status(C.Structure):
@@ -45,7 +46,12 @@ class _Status(C.Structure):
                 ("pages_in_use", C.c_int64), ("assign_rechecked", C.c_int64), ("tokens_attended_total", C.c_int64),
                 ("clusters_selected_total", C.c_int64)]
 
-KERNEL_CLASSES = ["init", "assign", "update", "finalize", "select", "attn", "combine", "append", "split", "front"]
+class _TierStats(C.Structure):
+    _fields_ = [(k, C.c_int64) for k in ("pages_fetched", "clusters_hit", "clusters_fetched", "clusters_refreshed",
+                                         "clusters_evicted", "copies_dropped_stale", "frames_in_use", "frames_total")]
+
+
+KERNEL_CLASSES = ["init", "assign", "update", "finalize", "select", "attn", "combine", "append", "split", "front", "tier"]
 
 
 @dataclass
@@ -69,6 +75,8 @@ class DynaKVConfig:
     local_max: int = 64
     det_sums: int = 0
     buf_max: int = 64
+    tier: int = 0
+    cache_pages: int = 0
 
 
 _lib = None
@@ -94,6 +102,8 @@ def load_library() -> C.CDLL:
     L.dynakv_get_work_list.argtypes = [vp, vp, vp, i64]
     L.dynakv_work_list_capacity.restype = C.c_int
     L.dynakv_work_list_capacity.argtypes = [vp]
+    L.dynakv_get_tier_stats.restype = C.c_int
+    L.dynakv_get_tier_stats.argtypes = [vp, C.POINTER(_TierStats)]
     L.dynakv_append.restype = C.c_int
     L.dynakv_append.argtypes = [vp, vp, vp]
     L.dynakv_decode_step.restype = C.c_int
@@ -193,7 +203,8 @@ class DynaKV:
         self._stream = stream if stream is not None else torch.cuda.current_stream()
         c = _Config(cfg.n_units, cfg.gqa_group, cfg.head_dim, cfg.kv_dtype, cfg.max_tokens, cfg.max_clusters,
                     cfg.kmeans_iters, cfg.init_mode, cfg.split_size_factor, cfg.split_var_factor,
-                    cfg.split_min_size, cfg.split_iters, cfg.trace, cfg.assign_mode, cfg.attn_mode, cfg.update_mode, cfg.local_max, cfg.det_sums, cfg.buf_max)
+                    cfg.split_min_size, cfg.split_iters, cfg.trace, cfg.assign_mode, cfg.attn_mode, cfg.update_mode, cfg.local_max, cfg.det_sums, cfg.buf_max,
+                    cfg.tier, cfg.cache_pages)
         h = C.c_void_p()
         self._check(self._L.dynakv_create(C.byref(c), C.c_void_p(self._stream.cuda_stream), C.byref(h)), "dynakv_create")
         self._h = h
@@ -359,6 +370,12 @@ class DynaKV:
         n = np.empty(U, np.int32); e = np.empty((U, W, 2), np.int32)
         self._check(self._L.dynakv_get_work_list(self._h, _np_ptr(n), _np_ptr(e), W), "dynakv_get_work_list")
         return n, e
+
+    def get_tier_stats(self) -> dict:
+        """Two-tier mode: the cache counters since the context was created, summed over units."""
+        st = _TierStats()
+        self._check(self._L.dynakv_get_tier_stats(self._h, C.byref(st)), "dynakv_get_tier_stats")
+        return {k: int(getattr(st, k)) for k, _ in _TierStats._fields_}
 
     def get_build_trace(self):
         U, T = self.cfg.n_units, self.cfg.kmeans_iters

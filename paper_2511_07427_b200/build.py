@@ -10,7 +10,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(_HERE, "csrc")
 LIB = os.path.join(_HERE, "libdynakv.so")
 OBJ = os.path.join(_HERE, "_build")
-SOURCES = ["api.cu", "build_kernels.cu", "decode_kernels.cu", "split_kernel.cu", "assign_tc.cu", "attn_kernels.cu", "front_kernels.cu", "noalloc_attend.cu"]
+SOURCES = ["api.cu", "build_kernels.cu", "decode_kernels.cu", "split_kernel.cu", "assign_tc.cu", "attn_kernels.cu", "front_kernels.cu", "noalloc_attend.cu", "tier.cu"]
 NVCC_FLAGS = ["-O3", "-std=c++17", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
               "-Xcompiler", "-fPIC", "-Xptxas", "-v"]
 

@@ -26,6 +26,9 @@ struct dynakv_ctx {
     cudaStream_t stream;
     Tables t;
     std::vector<void*> allocs;
+    std::vector<void*> host_allocs;   // pinned host memory (the page pool of the two-tier mode)
+    bool tier = false;
+    TierState ts;
     bool built = false;
     long long n_prefill = 0;
     int M0 = 0;
@@ -143,6 +146,8 @@ extern "C" int dynakv_create(const dynakv_config* cfg, void* cuda_stream, dynakv
     if (cfg->update_mode < DYNAKV_MODE_ADAPTIVE || cfg->update_mode > DYNAKV_MODE_DELAYED) return DYNAKV_ERR_ARG;
     if (cfg->update_mode == DYNAKV_MODE_DELAYED && cfg->buf_max < 1) return DYNAKV_ERR_ARG;
     if (cfg->update_mode == DYNAKV_MODE_LOCAL && cfg->local_max < 2) return DYNAKV_ERR_ARG;
+    if (cfg->tier != 0 && cfg->tier != 1) return DYNAKV_ERR_ARG;
+    if (cfg->tier && (cfg->kv_dtype == DYNAKV_FP8 || cfg->cache_pages < 1 || cfg->n_units > 65535)) return DYNAKV_ERR_ARG;
     dynakv_ctx* c = new (std::nothrow) dynakv_ctx();
     if (!c) return DYNAKV_ERR_NOMEM;
     c->cfg = *cfg;
@@ -182,7 +187,44 @@ extern "C" int dynakv_create(const dynakv_config* cfg, void* cuda_stream, dynakv
         ALLOC(t.k8, page_elems, false); ALLOC(t.v8, page_elems, false);
         ALLOC(t.k8e, U * P * PAGE, true); ALLOC(t.v8e, U * P * PAGE, true);
     }
-    if (cfg->kv_dtype == DYNAKV_F32) {
+    if (cfg->tier) {
+        // two tiers: the page pool is pinned host memory the device reads and writes in place; device memory holds the
+        // frame cache only
+        c->tier = true;
+        memset(&c->ts, 0, sizeof(c->ts));
+        for (void** pp : {&t.kpages, &t.vpages}) {
+            void* h = nullptr;
+            cudaError_t e = cudaHostAlloc(&h, page_elems * kv_bytes(*cfg), cudaHostAllocMapped | cudaHostAllocPortable);
+            void* dptr = nullptr;
+            if (e == cudaSuccess) { c->host_allocs.push_back(h); e = cudaHostGetDevicePointer(&dptr, h, 0); }
+            if (e != cudaSuccess) {
+                snprintf(g_err, sizeof(g_err), "pinned host allocation of %zu bytes for the page pool failed: %s",
+                         page_elems * kv_bytes(*cfg), cudaGetErrorString(e));
+                cudaGetLastError();
+                dynakv_destroy(c);
+                return DYNAKV_ERR_NOMEM;
+            }
+            *pp = dptr;
+        }
+        TierState& ts = c->ts;
+        ts.Fc = cfg->cache_pages;
+        const size_t Fc = ts.Fc;
+        char *ka, *va;
+        ALLOC(ka, U * Fc * PAGE * d * kv_bytes(*cfg), true); ALLOC(va, U * Fc * PAGE * d * kv_bytes(*cfg), true);
+        ts.kcache = ka; ts.vcache = va;
+        ALLOC(ts.cl_fr_head, U * Mx, false); ALLOC(ts.cl_fr_tail, U * Mx, false);
+        ALLOC(ts.cl_snap, U * Mx * 4, true);
+        ALLOC(ts.cl_lru, U * Mx, false);
+        ALLOC(ts.page_frame, U * P, false);
+        ALLOC(ts.frame_page, U * Fc, false); ALLOC(ts.frame_next, U * Fc, false);
+        ALLOC(ts.fr_free, U * Fc, false); ALLOC(ts.fr_free_cnt, U, false);
+        ALLOC(ts.miss_list, U * Mx, false);
+        ALLOC(ts.jobs, U * (Fc + Mx), false); ALLOC(ts.n_jobs, U, false);
+        ALLOC(ts.clock, U, false);
+        ALLOC(ts.counters, TIER_COUNTERS, false);
+        ALLOC(t.cl_ver, U * Mx, false);
+        launch_tier_init(t, ts, c->stream, &c->launches);
+    } else if (cfg->kv_dtype == DYNAKV_F32) {
         float *a, *b; ALLOC(a, page_elems, false); ALLOC(b, page_elems, false); t.kpages = a; t.vpages = b;
     } else if (t.fp8) {
         // FP8 storage: the rows live in their one-byte form only; whoever re-reads keys (the splits' 2-means, the exact
@@ -260,6 +302,7 @@ extern "C" void dynakv_destroy(dynakv_ctx* c) {
     for (auto& sp : c->spans) { cudaEventDestroy(sp.e0); cudaEventDestroy(sp.e1); }
     for (cudaEvent_t e : c->event_pool) cudaEventDestroy(e);
     for (void* p : c->allocs) cudaFree(p);
+    for (void* p : c->host_allocs) cudaFreeHost(p);
     delete c;
 }
 
@@ -361,17 +404,27 @@ static void enqueue_attend(dynakv_ctx* c, StepPtr q, StepPtrW out, bool timed);
 // select -> gather attention -> combine, on scores already written by the front pass
 static void enqueue_retrieve(dynakv_ctx* c, StepPtr q, int budget, StepPtrW out, int* sel_ids, bool timed) {
     { TimeScope ts(c, KC_SELECT, timed); launch_select(c->t, budget, sel_ids, c->stream, &c->launches); }
+    // two tiers: bring the selected clusters into the frame cache and point the gather list at the frames
+    if (c->tier) { TimeScope ts(c, KC_TIER, timed); launch_tier_resolve_fetch(c->t, c->ts, c->stream, &c->launches); }
     enqueue_attend(c, q, out, timed);
 }
 
+// The tables the attention kernels read rows through: the page pool, or in the two-tier mode the frame cache.
+static Tables attn_tables(const dynakv_ctx* c) {
+    Tables a = c->t;
+    if (c->tier) { a.kpages = c->ts.kcache; a.vpages = c->ts.vcache; a.P = c->ts.Fc; }
+    return a;
+}
+
 static void enqueue_attend(dynakv_ctx* c, StepPtr q, StepPtrW out, bool timed) {
+    const Tables at = attn_tables(c);
     if (c->t.kv_dtype == DYNAKV_BF16 && c->cfg.attn_mode == 0) {
         // gather, attend and combine in one persistent kernel
         TimeScope ts(c, KC_ATTN, timed);
-        launch_gather_attn_tma(c->t, q, out, c->stream, &c->launches);
+        launch_gather_attn_tma(at, q, out, c->stream, &c->launches);
     } else {
-        { TimeScope ts(c, KC_ATTN, timed); launch_gather_attn_v1(c->t, q, c->stream, &c->launches); }
-        { TimeScope ts(c, KC_COMBINE, timed); launch_attn_combine(c->t, out, c->stream, &c->launches); }
+        { TimeScope ts(c, KC_ATTN, timed); launch_gather_attn_v1(at, q, c->stream, &c->launches); }
+        { TimeScope ts(c, KC_COMBINE, timed); launch_attn_combine(at, out, c->stream, &c->launches); }
     }
 }
 
@@ -772,6 +825,26 @@ extern "C" int dynakv_get_work_list(dynakv_ctx* c, int32_t* n_entries, int32_t* 
     return DYNAKV_OK;
 }
 
+extern "C" int dynakv_get_tier_stats(dynakv_ctx* c, dynakv_tier_stats* out) {
+    if (!c || !out) return DYNAKV_ERR_ARG;
+    if (!c->tier) return DYNAKV_ERR_STATE;
+    unsigned long long cnt[TIER_COUNTERS];
+    std::vector<int> free_cnt(c->t.U);
+    CK(cudaMemcpyAsync(cnt, c->ts.counters, sizeof(cnt), cudaMemcpyDeviceToHost, c->stream));
+    CK(cudaMemcpyAsync(free_cnt.data(), c->ts.fr_free_cnt, sizeof(int) * c->t.U, cudaMemcpyDeviceToHost, c->stream));
+    CK(cudaStreamSynchronize(c->stream));
+    out->pages_fetched = (int64_t)cnt[TIER_PAGES_FETCHED];
+    out->clusters_hit = (int64_t)cnt[TIER_HITS];
+    out->clusters_fetched = (int64_t)cnt[TIER_FETCHED];
+    out->clusters_refreshed = (int64_t)cnt[TIER_REFRESHED];
+    out->clusters_evicted = (int64_t)cnt[TIER_EVICTED];
+    out->copies_dropped_stale = (int64_t)cnt[TIER_STALE];
+    out->frames_total = (int64_t)c->t.U * c->ts.Fc;
+    out->frames_in_use = out->frames_total;
+    for (int f : free_cnt) out->frames_in_use -= f;
+    return DYNAKV_OK;
+}
+
 extern "C" int dynakv_work_list_capacity(dynakv_ctx* c) { return c ? c->t.W : DYNAKV_ERR_ARG; }
 
 extern "C" int dynakv_get_build_trace(dynakv_ctx* c, int32_t* picks, int32_t* assign) {
@@ -804,9 +877,10 @@ extern "C" int dynakv_time_gather_attention(dynakv_ctx* c, const float* q, float
     CK(cudaEventCreate(&e0)); CK(cudaEventCreate(&e1));
     const StepPtr qp{q, 0, nullptr};
     const StepPtrW op{out, 0, nullptr};
-    launch_gather_attn_plain(c->t, qp, op, c->stream, &c->launches);       // one untimed launch first
+    const Tables at = attn_tables(c);
+    launch_gather_attn_plain(at, qp, op, c->stream, &c->launches);       // one untimed launch first
     CK(cudaEventRecord(e0, c->stream));
-    for (int i = 0; i < reps; i++) launch_gather_attn_plain(c->t, qp, op, c->stream, &c->launches);
+    for (int i = 0; i < reps; i++) launch_gather_attn_plain(at, qp, op, c->stream, &c->launches);
     CK(cudaEventRecord(e1, c->stream));
     CK(cudaGetLastError());
     CK(cudaEventSynchronize(e1));

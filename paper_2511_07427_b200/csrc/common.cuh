@@ -38,6 +38,7 @@ struct Tables {
     int det_sums;                    // 1: centroid sums of the build in 64-bit fixed point (order-independent)
     int buf_max;                     // delayed-split mode: buffered entries per unit that force a split
     int* cl_buf;                     // [U][Mmax] delayed-split mode: entries buffered for a flagged cluster
+    int* cl_ver;                     // [U][Mmax] two-tier mode (else null): splits the cluster id has been through
     // FP8 mode (fp8 != 0): kv_dtype is DYNAKV_BF16 for every kernel, all rows lie on the e4m3-times-power-of-two grid,
     // and a one-byte copy of the pages is kept for the gather-attention kernel
     int fp8;
@@ -190,7 +191,7 @@ inline cudaError_t launch_pdl(void (*kern)(KArgs...), dim3 grid, dim3 block, siz
 
 // Kernel classes for the optional per-kernel event timing.
 enum { KC_INIT = 0, KC_ASSIGN = 1, KC_UPDATE = 2, KC_FINALIZE = 3, KC_SELECT = 4, KC_ATTN = 5, KC_COMBINE = 6,
-       KC_APPEND = 7, KC_SPLIT = 8, KC_FRONT = 9, KC_COUNT = 10 };
+       KC_APPEND = 7, KC_SPLIT = 8, KC_FRONT = 9, KC_TIER = 10, KC_COUNT = 11 };
 
 // ---- host launchers (defined in the kernel files) ---------------------------------------
 struct BuildScratch {
@@ -248,5 +249,26 @@ struct NextFront {
 };
 void launch_append_split(const Tables& t, float gamma, int var_enabled, int min_size, int iters, int do_append, StepPtr k,
                          StepPtr v, int* step_ctr, const NextFront& nf, cudaStream_t s, long long* launches);
+
+// Two-tier mode: the page pool (Tables::kpages / vpages) is pinned host memory and this is the HBM cache of page
+// frames over it, per unit, filled and replaced in whole clusters.
+enum { TIER_PAGES_FETCHED = 0, TIER_HITS = 1, TIER_FETCHED = 2, TIER_REFRESHED = 3, TIER_EVICTED = 4, TIER_STALE = 5,
+       TIER_COUNTERS = 8 };
+struct TierState {
+    int Fc;                          // frames per unit
+    void* kcache; void* vcache;      // [U][Fc][PAGE][d]
+    int* cl_fr_head; int* cl_fr_tail;   // [U][Mmax] first / last frame of the cluster's copy (-1: no copy)
+    int* cl_snap;                    // [U][Mmax][4] the cluster when it was copied: n, version, first page, last page
+    unsigned int* cl_lru;            // [U][Mmax] resolve turn that last used the copy
+    int* page_frame;                 // [U][P] frame holding a copy of the page (-1: none)
+    int* frame_page; int* frame_next;   // [U][Fc] page the frame copies; next frame of the same cluster's copy
+    int* fr_free; int* fr_free_cnt;  // [U][Fc] stack of free frames, [U] its height
+    int* miss_list;                  // [U][Mmax] selected clusters that need frames this turn
+    int2* jobs; int* n_jobs;         // [U][Fc + Mmax] (page, frame) copies of this turn, [U] how many
+    unsigned int* clock;             // [U] resolve turns so far
+    unsigned long long* counters;    // [TIER_COUNTERS]
+};
+void launch_tier_init(const Tables& t, const TierState& ts, cudaStream_t s, long long* launches);
+void launch_tier_resolve_fetch(const Tables& t, const TierState& ts, cudaStream_t s, long long* launches);
 
 }  // namespace dkv

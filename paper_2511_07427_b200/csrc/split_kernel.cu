@@ -624,6 +624,7 @@ __global__ void __launch_bounds__(SP_THREADS, DKV_SP_MINBLOCKS) k_split_check(Ta
                 t.cl_head[cn] = newpg[0]; t.cl_tail[cn] = newpg[need - 1];
                 t.cl_n[cj] = s_n; t.cl_n[cn] = m_n;
                 t.cl_flags[cj] = 0; t.cl_flags[cn] = 0; t.cl_buf[cj] = 0; t.cl_buf[cn] = 0;
+                if (t.cl_ver) t.cl_ver[cj] = t.cl_ver[cj] + 1;      // two-tier mode: copies of the cluster made before now are void
                 t.u_M[u] = new_id + 1; t.u_Mlive[u] = t.u_Mlive[u] + 1;
                 atomicAdd(&t.counters[CNT_SPLITS], 1ull);
                 s_nsplit = s_nsplit + 1;

@@ -342,6 +342,7 @@ __device__ int split_small(const Tables& t, int u, int j, int c, int iters, KV* 
         t.cl_head[cn] = sc.newpg[0]; t.cl_tail[cn] = sc.newpg[need - 1];
         t.cl_n[cj] = s_n; t.cl_n[cn] = m_n;
         t.cl_flags[cj] = 0; t.cl_flags[cn] = 0; t.cl_buf[cj] = 0; t.cl_buf[cn] = 0;
+        if (t.cl_ver) t.cl_ver[cj] = t.cl_ver[cj] + 1;      // two-tier mode: copies of the cluster made before now are void
         t.u_M[u] = new_id + 1; t.u_Mlive[u] = mlive + 1;
         atomicAdd(&t.counters[CNT_SPLITS], 1ull);
         *sc.nsplit = *sc.nsplit + 1;

@@ -20,6 +20,7 @@ import numpy as np
 import torch
 
 import oracle as O
+from oracle.cluster_cache import ClusterCacheModel
 import paper_2511_07427_b200 as P
 from gen import UnitStream, WorkloadConfig, make_decode_chunk, make_prefill
 
@@ -41,6 +42,9 @@ class ParityReport:
     tokens_selected: List[int] = field(default_factory=list)
     status_bits: int = 0
     rechecked: int = 0
+    gpu_splits: int = 0
+    tier_stats: Optional[dict] = None     # two-tier runs: the library's cache counters and the model's
+    tier_model: Optional[dict] = None
     decisions: int = 0          # discrete decisions offered to the oracle as hints (assignments, selections, appends, checks)
 
 
@@ -69,7 +73,7 @@ def log_ties(name: str, rep: "ParityReport") -> None:
 
 
 def make_ctx(cfg: WorkloadConfig, n_units: int, trace: int = 1, assign_mode: int = 0, attn_mode: int = 0,
-             det_sums: int = 0) -> P.DynaKV:
+             det_sums: int = 0, cache_pages: int = 0) -> P.DynaKV:
     return P.DynaKV(P.DynaKVConfig(
         n_units=n_units, gqa_group=cfg.G, head_dim=cfg.d,
         kv_dtype={"f32": P.F32, "bf16": P.BF16, "fp8": P.FP8}[cfg.kv_dtype],
@@ -79,7 +83,8 @@ def make_ctx(cfg: WorkloadConfig, n_units: int, trace: int = 1, assign_mode: int
         split_min_size=cfg.split_min_size, split_iters=cfg.split_iters, trace=trace, assign_mode=assign_mode, attn_mode=attn_mode,
         update_mode={"adaptive": P.MODE_ADAPTIVE, "static": P.MODE_STATIC, "local": P.MODE_LOCAL,
                      "delayed": P.MODE_DELAYED}[cfg.update_mode],
-        local_max=cfg.local_max, det_sums=det_sums, buf_max=cfg.buf_max))
+        local_max=cfg.local_max, det_sums=det_sums, buf_max=cfg.buf_max,
+        tier=1 if cache_pages > 0 else 0, cache_pages=cache_pages))
 
 
 def fp8_round_rows(x: "torch.Tensor") -> "torch.Tensor":
@@ -145,10 +150,12 @@ def check_state(o: O.OracleUnit, st: dict, ui: int, rep: ParityReport, where: st
 def run_parity(cfg: WorkloadConfig, units: Sequence[int], steps: int, *, assign_mode: int = 0,
                state_every: int = 1, budget: Optional[int] = None, ctx_units: Optional[Sequence[int]] = None,
                seed: int = 1234, device: str = "cuda", check_every: int = 1, attn_mode: int = 0,
-               det_sums: int = 0, placement_queries: int = 0) -> ParityReport:
+               det_sums: int = 0, placement_queries: int = 0, cache_pages: int = 0) -> ParityReport:
     """Run `steps` decode iterations of `cfg`.  The GPU context holds `ctx_units` (default:
     `units`); the oracle follows the units listed in `units` (a subset of ctx_units).  With check_every > 1 the
-    split check is called only after every check_every-th append (on both sides)."""
+    split check is called only after every check_every-th append (on both sides).  With cache_pages > 0 the context
+    runs in its two-tier mode with that many page frames per unit, every unit is watched, and the library's cache
+    counters must equal those of the oracle's cache model fed with the oracle's own selections, sizes and splits."""
     rep = ParityReport()
     ctx_units = list(ctx_units) if ctx_units is not None else list(units)
     pos = {u: i for i, u in enumerate(ctx_units)}
@@ -156,7 +163,12 @@ def run_parity(cfg: WorkloadConfig, units: Sequence[int], steps: int, *, assign_
     budget = cfg.budget if budget is None else budget
     streams = [UnitStream(cfg, u) for u in ctx_units]
     K, V = make_prefill(streams)
-    ctx = make_ctx(cfg, len(ctx_units), trace=1, assign_mode=assign_mode, attn_mode=attn_mode, det_sums=det_sums)
+    ctx = make_ctx(cfg, len(ctx_units), trace=1, assign_mode=assign_mode, attn_mode=attn_mode, det_sums=det_sums,
+                   cache_pages=cache_pages)
+    caches = {}
+    if cache_pages > 0:
+        assert len(watch) == len(ctx_units), "the cache counters are summed over the context's units: watch them all"
+        caches = {ui: ClusterCacheModel(cache_pages) for ui in watch}
     if placement_queries > 0:
         # the build with correlation-aware placement: the pages' order in the pool changes, nothing else may
         g = torch.Generator().manual_seed(99)
@@ -197,6 +209,8 @@ def run_parity(cfg: WorkloadConfig, units: Sequence[int], steps: int, *, assign_
                 assert o.violations == v0 and list(ids_o) == list(ids_gpu), \
                     f"step {done + t} unit {ui}: selection differs: gpu {ids_gpu[:12]} oracle {ids_o[:12]}"
                 assert tok_o == int(ntok[ui])
+                if caches:
+                    caches[ui].retrieve(ids_o, o.counts())
                 rep.tokens_selected.append(tok_o)
                 ea = float(np.abs(out_np[ui] - out_o).max()); el = rel_l2(out_np[ui], out_o)
                 rep.max_out_abs = max(rep.max_out_abs, ea); rep.max_out_l2 = max(rep.max_out_l2, el)
@@ -219,7 +233,11 @@ def run_parity(cfg: WorkloadConfig, units: Sequence[int], steps: int, *, assign_
             for ui in watch:
                 o = oracles[ui]
                 v0 = o.violations
+                sizes_before = o.counts().copy()
                 o.split_check(hint_assign_after=st["tok_cluster"][ui, : o.n])
+                if caches:
+                    for j in np.nonzero(o.counts()[: len(sizes_before)] < sizes_before)[0]:      # a cluster that lost entries was split
+                        caches[ui].note_split(int(j))
                 assert o.violations == v0, f"step {done + t} unit {ui}: split decisions differ beyond the tie tolerance"
                 if (done + t) % state_every == 0 or done + t == steps - 1:
                     check_state(o, st, ui, rep, f"step {done + t} unit {ui}")
@@ -236,6 +254,12 @@ def run_parity(cfg: WorkloadConfig, units: Sequence[int], steps: int, *, assign_
         o = oracles[ui]
         rep.ties += o.ties; rep.violations += o.violations; rep.splits += o.n_splits
     rep.gpu_splits = status["n_splits"]
+    if caches:
+        rep.tier_stats = ctx.get_tier_stats()
+        rep.tier_model = {k: sum(m.c[k] for m in caches.values()) for k in next(iter(caches.values())).c}
+        rep.tier_model["frames_in_use"] = sum(m.frames_in_use for m in caches.values())
+        for k, v in rep.tier_model.items():
+            assert rep.tier_stats[k] == v, f"cache counter {k}: library {rep.tier_stats[k]}, model {v}\n{rep.tier_stats}\n{rep.tier_model}"
     ctx.destroy()
     return rep
 

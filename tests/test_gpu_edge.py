@@ -284,7 +284,15 @@ def test_graph_loop_in_delayed_split_mode():
     assert _loop_vs_direct(cfg, [0, 1, 2, 3, 4], 96, cut=37) > 50
 
 
-def _loop_vs_direct(cfg, units, steps, modes=("direct", "graph", "host"), cut=None):
+def test_graph_loop_and_host_steps_in_two_tier_mode():
+    # the cache bookkeeping and the page copies are part of the captured iteration and of the host step's graph; a
+    # stream that splits often, so copies are voided between steps, and helper blocks split rows that live in host memory
+    cfg = CONFIGS[3].scaled(n_prefill=500, steps=96, M0=12, max_clusters=256, budget=300, T=4, new_every=32,
+                            split_size_factor=1.3, split_var_factor=1.3)
+    assert _loop_vs_direct(cfg, [0, 1, 2, 3, 4], 96, modes=("direct", "graph", "host", "hostloop"), cut=37, cache_pages=96) > 50
+
+
+def _loop_vs_direct(cfg, units, steps, modes=("direct", "graph", "host"), cut=None, cache_pages=0):
     """The captured loop (and the host-buffer step) must leave the same state and outputs as direct calls."""
     s = [UnitStream(cfg, u) for u in units]
     K, V = make_prefill(s)
@@ -294,10 +302,11 @@ def _loop_vs_direct(cfg, units, steps, modes=("direct", "graph", "host"), cut=No
     outs = {}
     states = {}
     nsplit = {}
+    tier = {}
     for mode in modes:
         with torch.cuda.stream(side):
             from parity_harness import make_ctx
-            ctx = make_ctx(cfg, len(units), trace=0, assign_mode=1)
+            ctx = make_ctx(cfg, len(units), trace=0, assign_mode=1, cache_pages=cache_pages)
             ctx.build_index(K.cuda(), V.cuda(), cfg.M0, 7)
             qd, kd, vd = q.cuda(), k.cuda(), v.cuda()
             if mode == "direct":
@@ -327,9 +336,14 @@ def _loop_vs_direct(cfg, units, steps, modes=("direct", "graph", "host"), cut=No
             st = ctx.get_status()
             nsplit[mode] = st["n_splits"]
             assert st["error_bits"] & P.ST_INTERNAL == 0
+            if cache_pages:
+                assert st["error_bits"] == 0
+                tier[mode] = ctx.get_tier_stats()
             ctx.destroy()
     for mode in modes[1:]:
         assert nsplit[mode] == nsplit["direct"]
+        if cache_pages:         # the cache sees the same steps whichever way they are launched
+            assert tier[mode] == tier["direct"], f"{mode}: {tier[mode]} vs {tier['direct']}" 
         assert np.array_equal(states[mode]["tok_cluster"], states["direct"]["tok_cluster"])
         assert np.array_equal(states[mode]["counts"], states["direct"]["counts"])
         assert np.abs(outs[mode] - outs["direct"]).max() < 1e-4

@@ -222,3 +222,52 @@ def test_correlation_aware_placement_lengthens_contiguous_access():
     assert np.array_equal(res[False][2], res[True][2]) and res[True][3] == res[False][3]
     assert (res[False][1] - res[True][1]).abs().max().item() <= 1e-4
     assert res[True][0] >= 1.15 * res[False][0]
+
+
+@pytest.mark.parametrize("cid,cache_pages,attn_mode", [(3, 20, 0), (2, 24, 0), (2, 48, 1), (1, 24, 0), (30, 96, 0)])
+def test_two_tier_mode(cid, cache_pages, attn_mode):
+    """The two-tier mode (Section 6; Section 7 on CPU-GPU platforms): the page pool in pinned host memory, a cache of
+    cache_pages frames per unit in device memory, whole clusters brought in and replaced (Section 6.2).  The cache is
+    invisible in the results: selections, appends, splits, statistics and attention outputs agree with the oracle as
+    they do without it, at cache sizes that force evictions every few steps.  And the library's cache counters (pages
+    copied, hits, refreshes, fetches, evictions, copies voided by splits, frames in use) equal those of the oracle's
+    cache model, fed with the oracle's own selections, sizes and splits.  Case 30 is config 3 set to split often;
+    config 1 stores fp32 rows; attn_mode 1 reads the frames with the plain kernel."""
+    if cid == 30:
+        cfg = CONFIGS[3].scaled(n_prefill=500, steps=160, M0=12, max_clusters=256, budget=300, T=4, new_every=32,
+                                split_size_factor=1.3, split_var_factor=1.3)
+    elif cid == 1:
+        cfg = CONFIGS[1].scaled(n_prefill=700, steps=120, M0=24, max_clusters=128, budget=300, T=4)
+    else:
+        base = CONFIGS[cid]
+        cfg = base.scaled(n_prefill=1111 if cid != 3 else 333, steps=96 if cid != 3 else 200, M0=37 if cid != 3 else 13,
+                          max_clusters=160, budget=300, T=6, new_every=32 if base.new_every else 0)
+    rep = _run(cfg, [0] if cid == 1 else [0, 1, 2], cfg.steps, assign_mode=1, attn_mode=attn_mode, cache_pages=cache_pages)
+    ts = rep.tier_stats
+    print(f"[two tiers, {cache_pages} frames] {ts}")
+    assert rep.status_bits == 0
+    assert ts["clusters_hit"] > 0 and ts["clusters_refreshed"] > 0 and ts["clusters_evicted"] > 0
+    if cid in (3, 30):
+        assert rep.splits > 0 and ts["copies_dropped_stale"] > 0
+
+
+def test_two_tier_mode_reports_a_cache_that_is_too_small():
+    """A cache that cannot hold one step's clusters: the status word says so, nothing is read out of bounds, and the
+    context keeps working (with a larger budget than the cache, every step of that unit is flagged)."""
+    import paper_2511_07427_b200 as P
+    from gen import UnitStream, make_prefill, make_decode_chunk
+    from parity_harness import make_ctx
+    cfg = CONFIGS[2].scaled(n_prefill=1111, steps=8, M0=37, max_clusters=160, budget=300, T=3)
+    streams = [UnitStream(cfg, u) for u in range(2)]
+    K, V = make_prefill(streams)
+    q, k, v = make_decode_chunk(streams, cfg.steps)
+    ctx = make_ctx(cfg, 2, trace=0, assign_mode=1, cache_pages=4)
+    ctx.build_index(K.cuda(), V.cuda(), cfg.M0, 7)
+    for t in range(cfg.steps):
+        out = ctx.decode_step(q[t].cuda(), cfg.budget)
+        assert torch.isfinite(out).all()
+        ctx.append(k[t].cuda(), v[t].cuda()); ctx.split_check()
+    st = ctx.get_status()
+    assert st["error_bits"] & P.ST_TIER_CACHE
+    assert st["n_appended"] == 2 * cfg.steps
+    ctx.destroy()
