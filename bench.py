@@ -488,7 +488,8 @@ def run_ours(args, cfg):
         tier["pool_pages_per_unit_in_use"] = status["pages_in_use"] / U
         n_decode = max(pos, 1)
         tier["pages_fetched_per_step"] = tier["pages_fetched"] / n_decode
-        tier["host_to_device_mb_per_step"] = tier["pages_fetched"] * 32 * cfg.d * 2 * (4 if cfg.kv_dtype == "f32" else 2) / n_decode / 1e6
+        page_bytes = 2 * 32 * (cfg.d * {"f32": 4, "bf16": 2, "fp8": 1}[cfg.kv_dtype] + (1 if cfg.kv_dtype == "fp8" else 0))    # K and V
+        tier["host_to_device_mb_per_step"] = tier["pages_fetched"] * page_bytes / n_decode / 1e6
         looked_up = tier["clusters_hit"] + tier["clusters_refreshed"] + tier["clusters_fetched"]
         tier["cluster_hit_rate"] = (tier["clusters_hit"] + tier["clusters_refreshed"]) / max(looked_up, 1)
     ctx.destroy()

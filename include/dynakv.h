@@ -93,7 +93,7 @@ typedef struct dynakv_config {
                                   pinned host memory; device memory holds a cache of cache_pages page frames per unit.
                                   Each step's selected clusters are brought into the cache whole before the attention
                                   reads them, replacing whole clusters (Section 6.2); results are those of tier = 0.
-                                  F32 / BF16 only                                                                      */
+                                  Any kv_dtype (FP8: pool and frames hold the one-byte rows and their exponents)      */
     int32_t cache_pages;       /* tier = 1: 32-token page frames per unit in device memory; must hold the clusters of
                                   any one step (about token_budget / 32 plus one per selected cluster)                */
 } dynakv_config;

@@ -147,7 +147,7 @@ extern "C" int dynakv_create(const dynakv_config* cfg, void* cuda_stream, dynakv
     if (cfg->update_mode == DYNAKV_MODE_DELAYED && cfg->buf_max < 1) return DYNAKV_ERR_ARG;
     if (cfg->update_mode == DYNAKV_MODE_LOCAL && cfg->local_max < 2) return DYNAKV_ERR_ARG;
     if (cfg->tier != 0 && cfg->tier != 1) return DYNAKV_ERR_ARG;
-    if (cfg->tier && (cfg->kv_dtype == DYNAKV_FP8 || cfg->cache_pages < 1 || cfg->n_units > 65535)) return DYNAKV_ERR_ARG;
+    if (cfg->tier && (cfg->cache_pages < 1 || cfg->n_units > 65535)) return DYNAKV_ERR_ARG;
     dynakv_ctx* c = new (std::nothrow) dynakv_ctx();
     if (!c) return DYNAKV_ERR_NOMEM;
     c->cfg = *cfg;
@@ -183,7 +183,7 @@ extern "C" int dynakv_create(const dynakv_config* cfg, void* cuda_stream, dynakv
     }
     const size_t U = t.U, P = t.P, Mx = t.max_clusters, d = t.d;
     const size_t page_elems = U * P * PAGE * d;
-    if (t.fp8) {
+    if (t.fp8 && !cfg->tier) {
         ALLOC(t.k8, page_elems, false); ALLOC(t.v8, page_elems, false);
         ALLOC(t.k8e, U * P * PAGE, true); ALLOC(t.v8e, U * P * PAGE, true);
     }
@@ -192,26 +192,32 @@ extern "C" int dynakv_create(const dynakv_config* cfg, void* cuda_stream, dynakv
         // frame cache only
         c->tier = true;
         memset(&c->ts, 0, sizeof(c->ts));
-        for (void** pp : {&t.kpages, &t.vpages}) {
+        const size_t elem = t.fp8 ? 1 : kv_bytes(*cfg);
+        void* pool[4] = {nullptr, nullptr, nullptr, nullptr};          // K rows, V rows; FP8: K and V scale exponents
+        for (int i = 0; i < (t.fp8 ? 4 : 2); i++) {
+            const size_t bytes = i < 2 ? page_elems * elem : U * P * PAGE;
             void* h = nullptr;
-            cudaError_t e = cudaHostAlloc(&h, page_elems * kv_bytes(*cfg), cudaHostAllocMapped | cudaHostAllocPortable);
-            void* dptr = nullptr;
-            if (e == cudaSuccess) { c->host_allocs.push_back(h); e = cudaHostGetDevicePointer(&dptr, h, 0); }
+            cudaError_t e = cudaHostAlloc(&h, bytes, cudaHostAllocMapped | cudaHostAllocPortable);
+            if (e == cudaSuccess) { c->host_allocs.push_back(h); e = cudaHostGetDevicePointer(&pool[i], h, 0); }
             if (e != cudaSuccess) {
-                snprintf(g_err, sizeof(g_err), "pinned host allocation of %zu bytes for the page pool failed: %s",
-                         page_elems * kv_bytes(*cfg), cudaGetErrorString(e));
+                snprintf(g_err, sizeof(g_err), "pinned host allocation of %zu bytes for the page pool failed: %s", bytes, cudaGetErrorString(e));
                 cudaGetLastError();
                 dynakv_destroy(c);
                 return DYNAKV_ERR_NOMEM;
             }
-            *pp = dptr;
+            if (i >= 2) memset(h, 0, bytes);
         }
+        if (t.fp8) {
+            t.k8 = (unsigned char*)pool[0]; t.v8 = (unsigned char*)pool[1]; t.k8e = (signed char*)pool[2]; t.v8e = (signed char*)pool[3];
+            t.kpages = nullptr; t.vpages = nullptr;
+        } else { t.kpages = pool[0]; t.vpages = pool[1]; }
         TierState& ts = c->ts;
         ts.Fc = cfg->cache_pages;
         const size_t Fc = ts.Fc;
         char *ka, *va;
-        ALLOC(ka, U * Fc * PAGE * d * kv_bytes(*cfg), true); ALLOC(va, U * Fc * PAGE * d * kv_bytes(*cfg), true);
+        ALLOC(ka, U * Fc * PAGE * d * elem, true); ALLOC(va, U * Fc * PAGE * d * elem, true);
         ts.kcache = ka; ts.vcache = va;
+        if (t.fp8) { ALLOC(ts.kecache, U * Fc * PAGE, true); ALLOC(ts.vecache, U * Fc * PAGE, true); }
         ALLOC(ts.cl_fr_head, U * Mx, false); ALLOC(ts.cl_fr_tail, U * Mx, false);
         ALLOC(ts.cl_snap, U * Mx * 4, true);
         ALLOC(ts.cl_lru, U * Mx, false);
@@ -412,7 +418,11 @@ static void enqueue_retrieve(dynakv_ctx* c, StepPtr q, int budget, StepPtrW out,
 // The tables the attention kernels read rows through: the page pool, or in the two-tier mode the frame cache.
 static Tables attn_tables(const dynakv_ctx* c) {
     Tables a = c->t;
-    if (c->tier) { a.kpages = c->ts.kcache; a.vpages = c->ts.vcache; a.P = c->ts.Fc; }
+    if (c->tier) {
+        if (a.fp8) { a.k8 = (unsigned char*)c->ts.kcache; a.v8 = (unsigned char*)c->ts.vcache; a.k8e = c->ts.kecache; a.v8e = c->ts.vecache; }
+        else { a.kpages = c->ts.kcache; a.vpages = c->ts.vcache; }
+        a.P = c->ts.Fc;
+    }
     return a;
 }
 

@@ -363,6 +363,11 @@ __global__ void __launch_bounds__(1024) k_fin_layout(Tables t, int n, int M, con
     for (int i = n + tid; i < t.max_tokens; i += blockDim.x) t.tok_cluster[(size_t)u * t.max_tokens + i] = -1;
 }
 
+template <int BYTES> struct VecOf;
+template <> struct VecOf<4> { using type = unsigned int; };
+template <> struct VecOf<8> { using type = uint2; };
+template <> struct VecOf<16> { using type = uint4; };
+
 // One warp per token: claim the next slot of the token's cluster and copy its K, V rows.
 template <typename KV, int HD>
 __global__ void __launch_bounds__(256) k_fin_scatter(Tables t, const KV* __restrict__ K, const KV* __restrict__ V,
@@ -386,8 +391,12 @@ __global__ void __launch_bounds__(256) k_fin_scatter(Tables t, const KV* __restr
         const int pos = row_pos<Epc<KV>::v>(dslot, lane * EPL);      // EPL elements stay inside one chunk
         const KV* ks = K + (size_t)w * HD + lane * EPL;
         const KV* vs = V + (size_t)w * HD + lane * EPL;
-#pragma unroll
-        for (int e = 0; e < EPL; e++) if (!t.fp8) { kp[dst + pos + e] = ks[e]; vp[dst + pos + e] = vs[e]; }
+        if (!t.fp8) {
+            // one store per lane and row (the EPL elements are contiguous on both sides and aligned to their total size)
+            using Vec = typename VecOf<sizeof(KV) * EPL>::type;
+            *reinterpret_cast<Vec*>(kp + dst + pos) = *reinterpret_cast<const Vec*>(ks);
+            *reinterpret_cast<Vec*>(vp + dst + pos) = *reinterpret_cast<const Vec*>(vs);
+        }
         if (t.fp8) {
             // the one-byte copy of the row (the rows are on the grid already, so this conversion is exact)
             if constexpr (HD == 128 && sizeof(KV) == 2) {

@@ -256,7 +256,8 @@ enum { TIER_PAGES_FETCHED = 0, TIER_HITS = 1, TIER_FETCHED = 2, TIER_REFRESHED =
        TIER_COUNTERS = 8 };
 struct TierState {
     int Fc;                          // frames per unit
-    void* kcache; void* vcache;      // [U][Fc][PAGE][d]
+    void* kcache; void* vcache;      // [U][Fc][PAGE][d] rows in the pool's storage type (one byte per element in FP8 mode)
+    signed char* kecache; signed char* vecache;   // [U][Fc][PAGE] FP8 mode: the rows' scale exponents
     int* cl_fr_head; int* cl_fr_tail;   // [U][Mmax] first / last frame of the cluster's copy (-1: no copy)
     int* cl_snap;                    // [U][Mmax][4] the cluster when it was copied: n, version, first page, last page
     unsigned int* cl_lru;            // [U][Mmax] resolve turn that last used the copy

@@ -180,20 +180,29 @@ __global__ void __launch_bounds__(256) k_tier_resolve(Tables t, TierState ts) {
     }
 }
 
-// Copies the listed pages, K and V, from the pool (host memory) into their frames.
+// Copies the listed pages, K and V, from the pool (host memory) into their frames; in FP8 mode the one-byte rows and
+// the 32 scale exponents of each page.
 __global__ void __launch_bounds__(256) k_tier_fetch(Tables t, TierState ts, int row_bytes) {
     const int u = blockIdx.y;
     const int nj = ts.n_jobs[u];
     const size_t page_bytes = (size_t)PAGE * row_bytes;
     const int v16 = (int)(page_bytes / 16);
+    const char* kpool = t.fp8 ? (const char*)t.k8 : (const char*)t.kpages;
+    const char* vpool = t.fp8 ? (const char*)t.v8 : (const char*)t.vpages;
     for (int jb = blockIdx.x; jb < nj; jb += gridDim.x) {
         const int2 job = ts.jobs[(size_t)u * (ts.Fc + t.max_clusters) + jb];
         if (job.x < 0 || job.x >= t.P || job.y < 0 || job.y >= ts.Fc) continue;
-        const uint4* ks = reinterpret_cast<const uint4*>((const char*)t.kpages + ((size_t)u * t.P + job.x) * page_bytes);
-        const uint4* vs = reinterpret_cast<const uint4*>((const char*)t.vpages + ((size_t)u * t.P + job.x) * page_bytes);
-        uint4* kd = reinterpret_cast<uint4*>((char*)ts.kcache + ((size_t)u * ts.Fc + job.y) * page_bytes);
-        uint4* vd = reinterpret_cast<uint4*>((char*)ts.vcache + ((size_t)u * ts.Fc + job.y) * page_bytes);
+        const size_t src = (size_t)u * t.P + job.x, dst = (size_t)u * ts.Fc + job.y;
+        const uint4* ks = reinterpret_cast<const uint4*>(kpool + src * page_bytes);
+        const uint4* vs = reinterpret_cast<const uint4*>(vpool + src * page_bytes);
+        uint4* kd = reinterpret_cast<uint4*>((char*)ts.kcache + dst * page_bytes);
+        uint4* vd = reinterpret_cast<uint4*>((char*)ts.vcache + dst * page_bytes);
         for (int i = threadIdx.x; i < v16; i += 256) { kd[i] = ks[i]; vd[i] = vs[i]; }
+        if (t.fp8 && threadIdx.x < 2 * (PAGE / 16)) {
+            const int i = threadIdx.x % (PAGE / 16);
+            if (threadIdx.x < PAGE / 16) reinterpret_cast<uint4*>(ts.kecache + dst * PAGE)[i] = reinterpret_cast<const uint4*>(t.k8e + src * PAGE)[i];
+            else reinterpret_cast<uint4*>(ts.vecache + dst * PAGE)[i] = reinterpret_cast<const uint4*>(t.v8e + src * PAGE)[i];
+        }
     }
 }
 
@@ -204,7 +213,7 @@ void launch_tier_init(const Tables& t, const TierState& ts, cudaStream_t s, long
 
 void launch_tier_resolve_fetch(const Tables& t, const TierState& ts, cudaStream_t s, long long* launches) {
     k_tier_resolve<<<t.U, 256, 0, s>>>(t, ts);
-    const int row_bytes = t.d * (t.kv_dtype == DYNAKV_F32 ? 4 : 2);
+    const int row_bytes = t.fp8 ? t.d : t.d * (t.kv_dtype == DYNAKV_F32 ? 4 : 2);
     k_tier_fetch<<<dim3(16, t.U), 256, 0, s>>>(t, ts, row_bytes);
     (*launches) += 2;
 }
