@@ -236,12 +236,13 @@ __device__ __forceinline__ float tc_min3(float a, float b, float c) {
     asm("min.f32 %0, %1, %2, %3;\n" : "=f"(r) : "f"(a), "f"(b), "f"(c));
     return r;
 }
-// Fixed-point filter word: bits(v) * 256 + column (see k_tc_fixed_bias), as a positive float for min/max.  The
-// multiply-add is written in PTX so that it stays an integer multiply-add (FMA pipe) and does not become
-// shift/logic instructions on the ALU pipe, which the min/max chains keep busy.
-__device__ __forceinline__ float tc_pack(float v, int col) {
+// Fixed-point filter word: bits(v) * 256 + column tag (see k_tc_fixed_bias), as a positive float for min/max.  The
+// multiply-add is written in PTX, with the factor 256 in a register the compiler knows nothing about (a kernel
+// argument) and the tag as a compile-time constant, so that it stays ONE integer multiply-add on the FMA pipe:
+// a known power of two turns it into shift-and-add on the ALU pipe, which the min/max chains keep busy.
+__device__ __forceinline__ float tc_pack(float v, unsigned mul256, int tag) {
     unsigned r;
-    asm("mad.lo.u32 %0, %1, 256, %2;\n" : "=r"(r) : "r"(__float_as_uint(v)), "r"((unsigned)col));
+    asm("mad.lo.u32 %0, %1, %2, %3;\n" : "=r"(r) : "r"(__float_as_uint(v)), "r"(mul256), "r"((unsigned)tag));
     return __uint_as_float(r);
 }
 // (t1 <= t2 <= t3) <- the three smallest of {t1, t2, t3, x, y}.
@@ -267,6 +268,7 @@ __device__ __forceinline__ void tc_insert(float& g1, int& j1, float& g2, int& j2
 
 struct TcArgs {
     int U, n, M, Mpad, KB;               // KB = 128-key blocks per unit
+    unsigned tag_mul;                    // 256, handed over as data: see tc_pack
     const float* Bfix;                   // [U][Mpad] fixed-point bias 1.5 * 2^31 + ||c_j||^2 S_u
     const float2* scale;                 // [U] (S_u, g_u = 256 / S_u)
     const float* knorm;                  // [U * n]
@@ -393,6 +395,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) k_tc_assign(const __grid_consta
             bool dead = false;
             const float2 sc = p.scale[u];
             const float m2S = -2.f * sc.x;
+            const unsigned mul256 = p.tag_mul;
             for (int nt = 0; nt < NT; nt++, tb++) {
                 if ((int)(tb & 1) != team) continue;
                 const int st = (int)(tb % TC_NACC);
@@ -427,8 +430,9 @@ __global__ void __launch_bounds__(TC_THREADS, 1) k_tc_assign(const __grid_consta
 #pragma unroll
                         for (int x = 0; x < 4; x++) {
                             const int e0 = e + 2 * x;
-                            const float x0 = tc_pack(fmaf(__uint_as_float(acc[cc & 1][e0]), m2S, bs[cc & 1][e0]), c * 32 + e0);
-                            const float x1 = tc_pack(fmaf(__uint_as_float(acc[cc & 1][e0 + 1]), m2S, bs[cc & 1][e0 + 1]), c * 32 + e0 + 1);
+                            // the tag is the column inside this group's range: a compile-time constant per element
+                            const float x0 = tc_pack(fmaf(__uint_as_float(acc[cc & 1][e0]), m2S, bs[cc & 1][e0]), mul256, cc * 32 + e0);
+                            const float x1 = tc_pack(fmaf(__uint_as_float(acc[cc & 1][e0 + 1]), m2S, bs[cc & 1][e0 + 1]), mul256, cc * 32 + e0 + 1);
                             tc_top3_pair(ch[x][0], ch[x][1], ch[x][2], x0, x1);
                         }
                     }
@@ -441,9 +445,10 @@ __global__ void __launch_bounds__(TC_THREADS, 1) k_tc_assign(const __grid_consta
                 tc_merge3(ch[2], ch[3]);
                 tc_merge3(ch[0], ch[2]);
                 const float t1 = ch[0][0], t2 = ch[0][1], t3 = ch[0][2];
-                tc_insert(g1, j1, g2, j2, g3, t1, nt * TC_BN + (int)(__float_as_uint(t1) & 0xFFu));
-                tc_insert(g1, j1, g2, j2, g3, t2, nt * TC_BN + (int)(__float_as_uint(t2) & 0xFFu));
-                tc_insert(g1, j1, g2, j2, g3, t3, nt * TC_BN + (int)(__float_as_uint(t3) & 0xFFu));
+                const int col0 = nt * TC_BN + c_first * 32;
+                tc_insert(g1, j1, g2, j2, g3, t1, col0 + (int)(__float_as_uint(t1) & 0xFFu));
+                tc_insert(g1, j1, g2, j2, g3, t2, col0 + (int)(__float_as_uint(t2) & 0xFFu));
+                tc_insert(g1, j1, g2, j2, g3, t3, col0 + (int)(__float_as_uint(t3) & 0xFFu));
             }
             // ---- hand-over: group 1 -> group 0 (slot alternates per item; the barrier orders write, read and reuse)
             float* slots = xchg + (size_t)(item_no & 1) * 3 * TC_BM * 5 + row * 5;     // [3 groups][128 keys][5]
@@ -663,6 +668,7 @@ void launch_assign_tc(const Tables& t, const void* K, long long n, int M, const 
     }
     TcArgs a;
     a.U = t.U; a.n = (int)n; a.M = M; a.Mpad = L.Mpad; a.KB = (int)((n + TC_BM - 1) / TC_BM);
+    a.tag_mul = 256u;
     a.Bfix = Bfix; a.scale = scale; a.knorm = reinterpret_cast<const float*>(base + L.knorm); a.cmax_bits = cmax;
     a.assign = assign; a.recheck_list = list; a.recheck_count = count; a.status = t.status;
     a.pair_list = pairs; a.pair_count = pair_count;
