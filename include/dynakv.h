@@ -58,6 +58,8 @@ extern "C" {
 #define DYNAKV_ST_MAX_TOKENS 4u       /* an append was dropped: unit holds max_tokens            */
 #define DYNAKV_ST_PAGE_POOL 8u        /* a split or append was skipped: no free page             */
 #define DYNAKV_ST_INTERNAL 16u        /* an internal bound was hit (bounded wait ran out, ...)   */
+#define DYNAKV_ST_BOUNDS 64u          /* checked build only: an index taken from a table was out of range; the access
+                                         was skipped (dynakv_status.bounds_site names the first such place)       */
 #define DYNAKV_ST_TIER_CACHE 32u      /* two-tier mode: a step's clusters did not fit a unit's cache; that unit's output
                                          of the step is meaningless                              */
 
@@ -118,7 +120,7 @@ typedef struct dynakv_config {
 
 typedef struct dynakv_status {
     uint32_t error_bits;       /* OR of DYNAKV_ST_*                                              */
-    int32_t reserved;
+    int32_t bounds_site;       /* checked build: first place whose index test failed, 0 = none (else always 0) */
     int64_t n_appended;        /* appends stored, summed over units                              */
     int64_t n_splits;          /* splits performed, summed over units                            */
     int64_t tokens_selected;   /* tokens attended in the last decode step, summed over units     */
@@ -323,6 +325,13 @@ int dynakv_get_kernel_times(dynakv_ctx* ctx, double* ms_total, int64_t* launches
 
 /* Number of kernels this context has launched so far (graph replays count their nodes). */
 int64_t dynakv_launch_count(dynakv_ctx* ctx);
+
+/* Test aid (no counterpart in the paper).  1 if the library was compiled with -DDYNAKV_CHECKED, else 0.  In a checked
+ * build every index a kernel takes out of a table and turns into an address (a cluster id, a page of a chain, a row of
+ * the gather list, a token slot) is tested against the array it indexes; a failing test sets DYNAKV_ST_BOUNDS, records
+ * its place in dynakv_status.bounds_site, and the access is skipped or replaced by an in-range one.  Results are those
+ * of the ordinary build; it is slower and exists for the test suite. */
+int dynakv_checked_build(void);
 
 /* Text of the last CUDA error seen by this library on the calling thread ("" if none). */
 const char* dynakv_last_error(void);

@@ -9,19 +9,20 @@ from typing import Optional
 import numpy as np
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-_LIB_PATH = os.path.join(_HERE, "libdynakv.so")
+# DYNAKV_LIBRARY=checked selects the bounds-checked build of the same sources (libdynakv_checked.so), for test runs
+_LIB_PATH = os.path.join(_HERE, "libdynakv_checked.so" if os.environ.get("DYNAKV_LIBRARY") == "checked" else "libdynakv.so")
 
 F32, BF16, FP8 = 0, 1, 2
 INIT_KMEANSPP, INIT_RANDOM = 0, 1
 MODE_ADAPTIVE, MODE_STATIC, MODE_LOCAL, MODE_DELAYED = 0, 1, 2, 3
-ST_BUDGET_EXCEEDED, ST_MAX_CLUSTERS, ST_MAX_TOKENS, ST_PAGE_POOL, ST_INTERNAL, ST_TIER_CACHE = 1, 2, 4, 8, 16, 32
+ST_BUDGET_EXCEEDED, ST_MAX_CLUSTERS, ST_MAX_TOKENS, ST_PAGE_POOL, ST_INTERNAL, ST_TIER_CACHE, ST_BOUNDS = 1, 2, 4, 8, 16, 32, 64
 
 EXPORTED_SYMBOLS = [
     "dynakv_create", "dynakv_build_index", "dynakv_append", "dynakv_decode_step", "dynakv_split_check",
     "dynakv_decode_loop", "dynakv_step_host", "dynakv_get_status", "dynakv_export_state", "dynakv_get_selection",
     "dynakv_get_build_trace", "dynakv_set_timing", "dynakv_get_kernel_times", "dynakv_launch_count", "dynakv_last_error", "dynakv_destroy",
     "dynakv_attend_rows_noalloc", "dynakv_export_kv", "dynakv_import_state", "dynakv_decode_loop_host", "dynakv_selftest_wait_expiry", "dynakv_time_gather_attention",
-    "dynakv_build_index_placed", "dynakv_get_work_list", "dynakv_work_list_capacity", "dynakv_get_tier_stats",
+    "dynakv_build_index_placed", "dynakv_get_work_list", "dynakv_work_list_capacity", "dynakv_get_tier_stats", "dynakv_checked_build",
 ]
 ERR_TOO_LARGE = -5
 NOALLOC_SCRATCH_BYTES = 4 * 1024 * 1024
@@ -41,7 +42,7 @@ class _Config(C.Structure):
 
 
 class _Status(C.Structure):
-    _fields_ = [("error_bits", C.c_uint32), ("reserved", C.c_int32), ("n_appended", C.c_int64),
+    _fields_ = [("error_bits", C.c_uint32), ("bounds_site", C.c_int32), ("n_appended", C.c_int64),
                 ("n_splits", C.c_int64), ("tokens_selected", C.c_int64), ("clusters_selected", C.c_int64),
                 ("pages_in_use", C.c_int64), ("assign_rechecked", C.c_int64), ("tokens_attended_total", C.c_int64),
                 ("clusters_selected_total", C.c_int64)]
@@ -102,6 +103,8 @@ def load_library() -> C.CDLL:
     L.dynakv_get_work_list.argtypes = [vp, vp, vp, i64]
     L.dynakv_work_list_capacity.restype = C.c_int
     L.dynakv_work_list_capacity.argtypes = [vp]
+    L.dynakv_checked_build.restype = C.c_int
+    L.dynakv_checked_build.argtypes = []
     L.dynakv_get_tier_stats.restype = C.c_int
     L.dynakv_get_tier_stats.argtypes = [vp, C.POINTER(_TierStats)]
     L.dynakv_append.restype = C.c_int
@@ -302,7 +305,7 @@ class DynaKV:
     def get_status(self) -> dict:
         s = _Status()
         self._check(self._L.dynakv_get_status(self._h, C.byref(s)), "dynakv_get_status")
-        return {k: getattr(s, k) for k, _ in _Status._fields_ if k != "reserved"}
+        return {k: getattr(s, k) for k, _ in _Status._fields_}
 
     def export_state(self) -> dict:
         U, Mx, d, nt = self.cfg.n_units, self.cfg.max_clusters, self.cfg.head_dim, self.cfg.max_tokens

@@ -22,7 +22,15 @@ def _stale(target: str, deps) -> bool:
     return any(os.path.getmtime(d) > tt for d in deps)
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
+LIB_CHECKED = os.path.join(_HERE, "libdynakv_checked.so")
+OBJ_CHECKED = os.path.join(_HERE, "_build_checked")
+
+
+def build(force: bool = False, verbose: bool = False, checked: bool = False) -> str:
+    """Build libdynakv.so, or with checked=True libdynakv_checked.so: the same sources with -DDYNAKV_CHECKED (every
+    table-derived index tested before use), which the test suite runs a few cases against."""
+    LIB, OBJ = (LIB_CHECKED, OBJ_CHECKED) if checked else (globals()["LIB"], globals()["OBJ"])
+    flags = NVCC_FLAGS + (["-DDYNAKV_CHECKED"] if checked else [])
     os.makedirs(OBJ, exist_ok=True)
     headers = [os.path.join(CSRC, f) for f in os.listdir(CSRC) if f.endswith((".cuh", ".h"))]
     headers.append(os.path.join(os.path.dirname(_HERE), "include", "dynakv.h"))
@@ -38,7 +46,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
 
     def compile_one(job):
         src, obj = job
-        r = subprocess.run(["nvcc", *NVCC_FLAGS, "-c", src, "-o", obj], capture_output=True, text=True)
+        r = subprocess.run(["nvcc", *flags, "-c", src, "-o", obj], capture_output=True, text=True)
         log = r.stdout + r.stderr
         with open(obj + ".log", "w") as f:
             f.write(log)
@@ -58,4 +66,4 @@ def build(force: bool = False, verbose: bool = False) -> str:
 
 
 if __name__ == "__main__":
-    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv))
+    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv, checked="--checked" in sys.argv))

@@ -281,6 +281,7 @@ extern "C" int dynakv_create(const dynakv_config* cfg, void* cuda_stream, dynakv
     ALLOC(t.sp_pos, U * 2 * (size_t)t.max_tokens, false);
     ALLOC(t.status, 1, true);
     ALLOC(t.counters, 8, true);
+    ALLOC(t.check_rec, 2, true);
     ALLOC(c->step_ctr, 1, true);
     ALLOC(c->step_lim, 1, true);
     ALLOC(c->loop_args, 4, true);
@@ -726,6 +727,7 @@ extern "C" int dynakv_get_status(dynakv_ctx* c, dynakv_status* host_out) {
     if (c->built) { k_sum_status<<<1, 256, 0, c->stream>>>(c->t, (long long*)(c->t.counters + 4)); c->launches++; }
     CK(cudaMemcpyAsync(&host_out->error_bits, c->t.status, sizeof(unsigned int), cudaMemcpyDeviceToHost, c->stream));
     CK(cudaMemcpyAsync(cnt, c->t.counters, sizeof(cnt), cudaMemcpyDeviceToHost, c->stream));
+    CK(cudaMemcpyAsync(&host_out->bounds_site, c->t.check_rec, sizeof(int), cudaMemcpyDeviceToHost, c->stream));
     CK(cudaStreamSynchronize(c->stream));
     host_out->n_appended = (int64_t)cnt[CNT_APPENDED];
     host_out->n_splits = (int64_t)cnt[CNT_SPLITS];
@@ -924,3 +926,11 @@ extern "C" int dynakv_get_kernel_times(dynakv_ctx* c, double* ms_total, int64_t*
 }
 
 extern "C" int64_t dynakv_launch_count(dynakv_ctx* c) { return c ? c->launches : 0; }
+
+extern "C" int dynakv_checked_build(void) {
+#ifdef DYNAKV_CHECKED
+    return 1;
+#else
+    return 0;
+#endif
+}

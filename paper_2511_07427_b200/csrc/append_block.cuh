@@ -73,6 +73,7 @@ __device__ __forceinline__ void append_block(const Tables& t, int u, StepPtr kp_
         }
     }
     if (bj == 0x7fffffff) return;    // no live cluster
+    if (!DKV_IN(t, SITE_APPEND_CLUSTER, bj, 0, t.max_clusters)) return;
     const size_t cj = (size_t)u * t.max_clusters + bj;
     const int n_old = found ? 0 : t.cl_n[cj];
     int page = found ? -1 : t.cl_tail[cj];
@@ -83,6 +84,8 @@ __device__ __forceinline__ void append_block(const Tables& t, int u, StepPtr kp_
             int fc = t.u_free_cnt[u];
             if (fc > 0) { np = t.free_stack[(size_t)u * t.P + fc - 1]; t.u_free_cnt[u] = fc - 1; }
             else { int top = t.u_page_top[u]; if (top < t.P) { np = top; t.u_page_top[u] = top + 1; } }
+            if (np >= 0 && !DKV_IN(t, SITE_APPEND_PAGE, np, 0, t.P)) np = -1;
+            if (np >= 0 && page >= 0 && !DKV_IN(t, SITE_APPEND_PAGE, page, 0, t.P)) np = -1;
             if (np >= 0) {
                 if (page >= 0) t.page_next[(size_t)u * t.P + page] = np; else t.cl_head[cj] = np;
                 t.page_next[(size_t)u * t.P + np] = -1; t.cl_tail[cj] = np;
@@ -92,6 +95,7 @@ __device__ __forceinline__ void append_block(const Tables& t, int u, StepPtr kp_
         if (np < 0) return;
         page = np;
     }
+    if (!DKV_IN(t, SITE_APPEND_PAGE, page, 0, t.P) || !DKV_IN(t, SITE_APPEND_TOKEN, N, 0, t.max_tokens)) return;
     const float n_new = (float)(n_old + 1);
     float* r = t.cl_r + cj * HD;
     float add = 0.f;

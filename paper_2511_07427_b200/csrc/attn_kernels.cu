@@ -239,12 +239,15 @@ __global__ void __launch_bounds__(AT_THREADS, 2) k_gather_attn_tma(Tables t, Ste
         while (__any_sync(0xffffffffu, active)) {
             const bool ready = active && mbar_test_wait(empty, (((unsigned)(it / AT_STAGES)) & 1u) ^ 1u);
             if (ready) {
-                const int2 cur = ent;
+                int2 cur = ent;
                 const int cu = u;
+                // checked build: a bad entry is replaced by one row of the unit's first page, so the stage still fills
+                if (!DKV_IN(t, SITE_ATTN_ENTRY, cur.y, 1, ENTRY_ROWS + 1)) cur.y = 1;
+                if (!DKV_IN(t, SITE_ATTN_ENTRY, cur.x, 0, (long long)t.P * PAGE - cur.y + 1)) cur.x = 0;
                 const int nx = it + AT_STAGES;
                 if (nx < n_items) {          // next entry: its load is in flight until the stage comes round again
                     u = unit_of(pf, u, lo + nx);
-                    ent = work[(size_t)u * t.W + (lo + nx - pf[u])];
+                    ent = DKV_IN(t, SITE_ATTN_WORK, lo + nx - pf[u], 0, t.W) ? work[(size_t)u * t.W + (lo + nx - pf[u])] : make_int2(0, 1);
                 }
                 const unsigned bytes = (unsigned)cur.y * ROWB;
                 const size_t row0 = (size_t)cu * t.P * PAGE + cur.x;

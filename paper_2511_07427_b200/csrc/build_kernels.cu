@@ -385,6 +385,7 @@ __global__ void __launch_bounds__(256) k_fin_scatter(Tables t, const KV* __restr
         if (lane == 0) slot = atomicAdd(&cursor[(size_t)u * M + j], 1);
         slot = __shfl_sync(0xffffffffu, slot, 0);
         int page = t.cl_head[(size_t)u * t.max_clusters + j] + slot / PAGE, row = slot % PAGE;
+        if (!DKV_IN(t, SITE_LAYOUT_PAGE, page, 0, t.P) || !DKV_IN(t, SITE_LAYOUT_PAGE, i, 0, t.max_tokens)) continue;
         const size_t dslot = ((size_t)u * t.P + page) * PAGE + row;
         size_t dst = dslot * HD;
         constexpr int EPL = HD / 32;   // elements per lane
@@ -442,6 +443,7 @@ __global__ void __launch_bounds__(256) k_fin_stats(Tables t, int M, const float*
     for (int s = 0; s < c; s++) {
         int row = s % PAGE;
         if (s > 0 && row == 0) page = t.page_next[(size_t)u * t.P + page];
+        if (!DKV_IN(t, SITE_STATS_PAGE, page, 0, t.P)) break;          // uniform in the warp
         const size_t kslot = ((size_t)u * t.P + page) * PAGE + row;
         float kx[EPL];
         load_key<KV, HD, EPL>(t, kslot, lane * EPL, kx);
@@ -484,6 +486,7 @@ __global__ void __launch_bounds__(128) k_export_rows(Tables t, KV* __restrict__ 
     constexpr int V16 = HD * (int)sizeof(KV) / 16;        // 16-byte pieces per row
     for (int s0 = 0; s0 < c; s0 += PAGE) {
         const int rows = min(PAGE, c - s0);
+        if (!DKV_IN(t, SITE_EXPORT_PAGE, page, 0, t.P)) break;           // uniform in the block
         for (int idx = threadIdx.x; idx < rows * V16; idx += blockDim.x) {
             const int r = idx / V16, v = idx % V16;
             const size_t slot = ((size_t)u * t.P + page) * PAGE + r;

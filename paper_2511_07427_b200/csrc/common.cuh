@@ -82,7 +82,28 @@ struct Tables {
     // status / counters
     unsigned int* status;            // [1]
     unsigned long long* counters;    // [8]: see CNT_*; 4..6 are scratch of get_status
+    int* check_rec;                  // [2] checked build: site of the first index test that failed (0: none), spare
 };
+
+// ---- checked build ------------------------------------------------------------------------------------------------
+// Compiled with -DDYNAKV_CHECKED, every index that a kernel takes out of a table and turns into an address is tested
+// against the array it indexes.  A failing test records its site once (Tables::check_rec), sets DYNAKV_ST_BOUNDS and
+// yields false; the caller then skips the access or substitutes an in-range value, so that the kernel's protocol
+// (barrier counts, bytes of copies in flight) stays whole.  Without the flag the tests compile to nothing.
+enum { SITE_ATTN_ENTRY = 1, SITE_ATTN_WORK = 2, SITE_PLAIN_ENTRY = 3, SITE_SELECT_PAGE = 4, SITE_APPEND_CLUSTER = 5,
+       SITE_APPEND_PAGE = 6, SITE_APPEND_TOKEN = 7, SITE_SPLIT_PAGE = 8, SITE_SPLIT_ID = 9, SITE_LAYOUT_PAGE = 10,
+       SITE_SPLIT_TOKEN = 11, SITE_STATS_PAGE = 12, SITE_EXPORT_PAGE = 13 };
+#ifdef DYNAKV_CHECKED
+__device__ __noinline__ static bool dkv_bounds_fail(const Tables& t, int site) {
+    atomicOr(t.status, DYNAKV_ST_BOUNDS);
+    atomicCAS(&t.check_rec[0], 0, site);
+    return false;
+}
+#define DKV_IN(t, site, v, lo, hi) \
+    ((((long long)(v) >= (long long)(lo)) && ((long long)(v) < (long long)(hi))) || dkv::dkv_bounds_fail((t), (site)))
+#else
+#define DKV_IN(t, site, v, lo, hi) true
+#endif
 
 enum { CNT_APPENDED = 0, CNT_SPLITS = 1, CNT_RECHECKED = 2, CNT_TOKENS_ATTENDED = 3, CNT_CLUSTERS_SELECTED = 7 };
 

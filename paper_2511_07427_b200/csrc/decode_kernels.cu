@@ -41,6 +41,7 @@ __global__ void __launch_bounds__(128) k_gather_attn_v1(Tables t, StepPtr qp) {
     const KV* vp = reinterpret_cast<const KV*>(t.vpages);
     for (int w = w0 + warp; w < w1; w += 4) {
         int2 ent = work[w];
+        if (!DKV_IN(t, SITE_PLAIN_ENTRY, ent.y, 1, ENTRY_ROWS + 1) || !DKV_IN(t, SITE_PLAIN_ENTRY, ent.x, 0, (long long)t.P * PAGE - ent.y + 1)) continue;
         size_t pbase = ((size_t)u * t.P * PAGE + ent.x) * HD;
         for (int r = 0; r < ent.y; r++) {
             const int pos = row_pos<Epc<KV>::v>((size_t)(ent.x + r), lane * EPL);      // the row's stored chunk order

@@ -203,7 +203,10 @@ __device__ void select_unit_radix(const Tables& t, int u, int budget, int* __res
         for (int i = 0; i < np && wpos + i < t.W; i++) {
             constexpr int EPP = PAGE / ENTRY_ROWS;       // entries per page
             work[wpos + i] = make_int2(page * PAGE + (i % EPP) * ENTRY_ROWS, min(ENTRY_ROWS, sz - ENTRY_ROWS * i));
-            if (i % EPP == EPP - 1) page = __ldcg(&t.page_next[(size_t)u * t.P + page]);
+            if (i % EPP == EPP - 1) {
+                if (!DKV_IN(t, SITE_SELECT_PAGE, page, 0, t.P)) break;
+                page = __ldcg(&t.page_next[(size_t)u * t.P + page]);
+            }
         }
         wpos += np;
     }
@@ -418,7 +421,10 @@ __device__ void select_unit(const Tables& t, int u, int budget, int* __restrict_
         for (int e = 0; e < np && wpos + e < t.W; e++) {
             constexpr int EPP = PAGE / ENTRY_ROWS;       // entries per page
             work[wpos + e] = make_int2(page * PAGE + (e % EPP) * ENTRY_ROWS, min(ENTRY_ROWS, sz - ENTRY_ROWS * e));
-            if (e % EPP == EPP - 1 && e + 1 < np) page = (e / EPP == 0) ? nxt[i] : __ldcg(NEXT + page);
+            if (e % EPP == EPP - 1 && e + 1 < np) {
+                if (!DKV_IN(t, SITE_SELECT_PAGE, page, 0, t.P)) break;
+                page = (e / EPP == 0) ? nxt[i] : __ldcg(NEXT + page);
+            }
         }
         wpos += np;
     }

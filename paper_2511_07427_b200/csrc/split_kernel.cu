@@ -407,10 +407,19 @@ __global__ void __launch_bounds__(SP_THREADS, DKV_SP_MINBLOCKS) k_split_check(Ta
             const int npg = (c + PAGE - 1) / PAGE;
             if (tid == 0) {
                 int p = t.cl_head[cj];
-                for (int i = 0; i < npg; i++) { chain[i] = p; p = pnext[p]; }
+#ifdef DYNAKV_CHECKED
+                s_ok = 1;
+#endif
+                for (int i = 0; i < npg; i++) {
+                    if (!DKV_IN(t, SITE_SPLIT_PAGE, p, 0, t.P)) { s_ok = 0; break; }
+                    chain[i] = p; p = pnext[p];
+                }
             }
             for (int e = tid; e < HD; e += SP_THREADS) cA[e] = t.cl_r[cj * HD + e];
             __syncthreads();
+#ifdef DYNAKV_CHECKED
+            if (!s_ok) continue;          // a page of the chain was out of range: the cluster is left as it is
+#endif
             // general path (the cluster does not fit the staging area): every pass walks the pages.  The labels, ranks
             // and hole list of a cluster of up to GEN_ROWS members live in the two staging areas, which this path does
             // not use otherwise (every member's label is read and written once per 2-means round); beyond that in
@@ -552,6 +561,7 @@ __global__ void __launch_bounds__(SP_THREADS, DKV_SP_MINBLOCKS) k_split_check(Ta
                         int pg;
                         if (fc > 0) pg = t.free_stack[(size_t)u * t.P + --fc]; else pg = top++;
                         newpg[i] = pg;
+                        if (!DKV_IN(t, SITE_SPLIT_PAGE, pg, 0, t.P)) ok = 0;
                     }
                     t.u_free_cnt[u] = fc; t.u_page_top[u] = top;
                 } else atomicOr(t.status, DYNAKV_ST_PAGE_POOL);
@@ -593,7 +603,7 @@ __global__ void __launch_bounds__(SP_THREADS, DKV_SP_MINBLOCKS) k_split_check(Ta
                 if (lane == 0) {
                     int tok = ptok[src];
                     ptok[dst] = tok;
-                    t.tok_cluster[(size_t)u * t.max_tokens + tok] = new_id;
+                    if (DKV_IN(t, SITE_SPLIT_TOKEN, tok, 0, t.max_tokens)) t.tok_cluster[(size_t)u * t.max_tokens + tok] = new_id;
                 }
             }
             __syncthreads();

@@ -68,7 +68,11 @@ __device__ int split_small(const Tables& t, int u, int j, int c, int iters, KV* 
     for (int e = tid; e < HD; e += THREADS) sc.cA[e] = t.cl_r[cj * HD + e];
     // every thread walks the short chain itself: no broadcast through shared memory, no barrier
 #pragma unroll
-    for (int i = 1; i < MAXPG; i++) pg[i] = (i < npg) ? pnext[pg[i - 1]] : -1;
+    for (int i = 1; i < MAXPG; i++) pg[i] = (i < npg && DKV_IN(t, SITE_SPLIT_PAGE, pg[i - 1], 0, t.P)) ? pnext[pg[i - 1]] : -1;
+#ifdef DYNAKV_CHECKED
+    // every thread has walked the same chain, so all of them leave together
+    for (int i = 0; i < MAXPG; i++) if (i < npg && !DKV_IN(t, SITE_SPLIT_PAGE, pg[i], 0, t.P)) return -1;
+#endif
     auto page_of = [&](int i) -> int {
         int r = pg[0];
 #pragma unroll
@@ -257,7 +261,7 @@ __device__ int split_small(const Tables& t, int u, int j, int c, int iters, KV* 
 
     // ---- pages for the moving child (thread 0), ranks of every member (its own thread)
     if (tid == 0) {
-        const int ok = (fc + (t.P - top) >= need) ? 1 : 0;
+        int ok = (fc + (t.P - top) >= need) ? 1 : 0;
         if (ok) {
             int used = 0;
             for (int i = 0; i < need; i++) {
@@ -268,6 +272,7 @@ __device__ int split_small(const Tables& t, int u, int j, int c, int iters, KV* 
                     used++; fc--;
                 } else pgi = top++;
                 sc.newpg[i] = pgi;
+                if (!DKV_IN(t, SITE_SPLIT_PAGE, pgi, 0, t.P)) ok = 0;
             }
         } else atomicOr(t.status, DYNAKV_ST_PAGE_POOL);
         s_ok = ok;
@@ -324,7 +329,7 @@ __device__ int split_small(const Tables& t, int u, int j, int c, int iters, KV* 
         const int code = sc.rank[tid], tok = sc.tok[tid];
         if (code >= 0) {
             ptok[(size_t)sc.newpg[code >> 5] * PAGE + (code & 31)] = tok;
-            t.tok_cluster[(size_t)u * t.max_tokens + tok] = new_id;
+            if (DKV_IN(t, SITE_SPLIT_TOKEN, tok, 0, t.max_tokens)) t.tok_cluster[(size_t)u * t.max_tokens + tok] = new_id;
         } else if (code <= -2) {
             const int h = sc.holes[-2 - code];
             ptok[(size_t)page_of(h >> 5) * PAGE + (h & 31)] = tok;

@@ -245,6 +245,8 @@ def run_parity(cfg: WorkloadConfig, units: Sequence[int], steps: int, *, assign_
                     assert np.array_equal(st["tok_cluster"][ui, : o.n], o.assign()), f"step {done + t} unit {ui}: membership"
         done += nb
     status = ctx.get_status()
+    # (only a library built with its index tests can set this bit; see tests/test_gpu_checked.py)
+    assert status["error_bits"] & P.ST_BOUNDS == 0, f"an index test failed inside a kernel, site {status['bounds_site']}"
     rep.steps = steps
     n_checks = steps // check_every
     rep.decisions = len(watch) * (cfg.n_prefill * cfg.T + (cfg.M0 if cfg.init_mode == "kmeanspp" else 0) + 2 * steps + n_checks)

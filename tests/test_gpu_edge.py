@@ -335,7 +335,7 @@ def _loop_vs_direct(cfg, units, steps, modes=("direct", "graph", "host"), cut=No
             states[mode] = ctx.export_state()
             st = ctx.get_status()
             nsplit[mode] = st["n_splits"]
-            assert st["error_bits"] & P.ST_INTERNAL == 0
+            assert st["error_bits"] & (P.ST_INTERNAL | P.ST_BOUNDS) == 0, f"status {st['error_bits']}, site {st['bounds_site']}"
             if cache_pages:
                 assert st["error_bits"] == 0
                 tier[mode] = ctx.get_tier_stats()
