@@ -279,3 +279,39 @@ def test_two_tier_mode_reports_a_cache_that_is_too_small():
     assert st["error_bits"] & P.ST_TIER_CACHE
     assert st["n_appended"] == 2 * cfg.steps
     ctx.destroy()
+
+
+def test_two_tier_mode_pool_exports_and_resumes_in_a_single_tier_context():
+    """The host-memory pool of a two-tier context holds exactly the rows it was given, also after appends and splits
+    (export_kv reads it back through the page tables), and a single-tier context resumed from that export continues
+    with the same outputs and the same membership as the two-tier one."""
+    from gen import UnitStream, make_prefill, make_decode_chunk
+    from parity_harness import make_ctx
+    cfg = CONFIGS[3].scaled(n_prefill=500, steps=120, M0=12, max_clusters=256, budget=300, T=4, new_every=32,
+                            split_size_factor=1.3, split_var_factor=1.3)
+    U = 4
+    streams = [UnitStream(cfg, u) for u in range(U)]
+    K, V = make_prefill(streams)
+    q, k, v = make_decode_chunk(streams, cfg.steps)
+    ctx = make_ctx(cfg, U, trace=0, assign_mode=1, cache_pages=96)
+    ctx.build_index(K.cuda(), V.cuda(), cfg.M0, 7)
+    half = 70
+    qd, kd, vd = q.cuda(), k.cuda(), v.cuda()
+    for t in range(half):
+        ctx.decode_step(qd[t], cfg.budget); ctx.append(kd[t], vd[t]); ctx.split_check()
+    assert ctx.get_status()["n_splits"] > 20
+    n = cfg.n_prefill + half
+    Ke, Ve = ctx.export_kv(n)
+    K_all = torch.cat([K, k[:half].transpose(0, 1)], dim=1); V_all = torch.cat([V, v[:half].transpose(0, 1)], dim=1)
+    assert torch.equal(Ke.cpu(), K_all) and torch.equal(Ve.cpu(), V_all)
+    st = ctx.export_state()
+    ctx2 = make_ctx(cfg, U, trace=0, assign_mode=1)
+    ctx2.import_state(Ke, Ve, st["tok_cluster"][:, :n], st["n_ids"], st["tau"], cfg.M0)
+    for t in range(half, cfg.steps):
+        a = ctx.decode_step(qd[t], cfg.budget).clone(); b = ctx2.decode_step(qd[t], cfg.budget).clone()
+        assert (a - b).abs().max().item() <= 2e-3
+        for c in (ctx, ctx2):
+            c.append(kd[t], vd[t]); c.split_check()
+    assert np.array_equal(ctx.export_state()["tok_cluster"], ctx2.export_state()["tok_cluster"])
+    assert ctx.get_status()["error_bits"] == 0 and ctx.get_tier_stats()["clusters_evicted"] > 0
+    ctx.destroy(); ctx2.destroy()
