@@ -17,7 +17,7 @@
 // leaves the chip.
 //
 // Kernel shape.  Persistent CTAs, one per SM, each looping over (unit, 128-key block) items.
-// Warp 0 issues TMA tensor loads (128-byte swizzle, no multicast) of the key block (kept for
+// Warp 0 issues TMA tensor loads (128-byte swizzle, every CTA loads for itself) of the key block (kept for
 // all centre tiles of the item) and of 256-centre tiles into a two-stage ring; warp 1 issues
 // tcgen05.mma (M=128, N=256, K=16, eight per tile) into one of two 256-column TMEM accumulators
 // and commits to an mbarrier; warps 2-17 drain the accumulators with tcgen05.ld, one key per
@@ -72,7 +72,7 @@ __device__ __forceinline__ bool tc_mbar_wait(unsigned bar, unsigned parity) {
     }
     return false;
 }
-// 2-D tiled TMA load (inner coordinate x in elements, outer coordinate y in rows), no multicast.
+// 2-D tiled TMA load (inner coordinate x in elements, outer coordinate y in rows); every CTA loads for itself.
 __device__ __forceinline__ void tc_tma_load_2d(unsigned dst, const CUtensorMap* map, int x, int y, unsigned bar) {
     asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];\n"
                  ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar) : "memory");
