@@ -185,15 +185,16 @@ __global__ void __launch_bounds__(AS_THREADS) k_assign_f32(const KV* __restrict_
     float* keysT = smem;                 // [HD][KS]
     float* centT = smem + (size_t)HD * KS;  // [HD][CS]
     const int u = blockIdx.y, tid = threadIdx.x;
-    const int key0 = blockIdx.x * AS_BK;
     const KV* Ku = K + (size_t)u * n * HD;
     const float* Cu = C + (size_t)u * M * HD;
     const int ty = tid >> 4, tx = tid & 15;
     const int n_here = list ? (int)counts[u] : n;          // keys this unit has to assign
-    if (key0 >= n_here) return;
     const int* lu = list ? list + (size_t)u * n : nullptr;
-    if (list && blockIdx.x == 0 && tid == 0) atomicAdd(listed_total, (unsigned long long)n_here);
+    if (list && blockIdx.x == 0 && tid == 0 && n_here > 0) atomicAdd(listed_total, (unsigned long long)n_here);
 
+    // the grid covers every 128-key tile of a full assignment; in list mode it is a few blocks per unit, each taking
+    // the tiles of the (short, device-side) list in turn
+    for (int key0 = blockIdx.x * AS_BK; key0 < n_here; key0 += gridDim.x * AS_BK) {
     for (int idx = tid; idx < AS_BK * (HD / 4); idx += AS_THREADS) {
         int key = idx % AS_BK, t4 = idx / AS_BK;
         float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -249,6 +250,8 @@ __global__ void __launch_bounds__(AS_THREADS) k_assign_f32(const KV* __restrict_
         }
         int key = key0 + ty * 8 + i;
         if (tx == 0 && key < n_here) assign[(size_t)u * n + (lu ? lu[key] : key)] = bj[i];
+    }
+    __syncthreads();          // the next tile's keys overwrite the staging area
     }
 }
 
@@ -570,7 +573,9 @@ static void assign_f32_t(const Tables& t, const void* K, long long n, int M, con
         cudaFuncSetAttribute(k_assign_f32<KV, HD>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)AssignSmem<HD>::bytes);
         if (dev >= 0 && dev < 64) opted[dev] = true;
     }
-    dim3 grid((unsigned)((n + AS_BK - 1) / AS_BK), t.U);
+    // list mode: the lists hold well under one tile per unit on every workload seen (their length is known on the device
+    // only); two blocks per unit loop over whatever there is instead of n / 128 blocks that mostly find nothing to do
+    dim3 grid(list ? 2u : (unsigned)((n + AS_BK - 1) / AS_BK), t.U);
     k_assign_f32<KV, HD><<<grid, AS_THREADS, AssignSmem<HD>::bytes, s>>>((const KV*)K, (int)n, M, C, assign, list, counts,
                                                                        listed_total);
     (*launches)++;
