@@ -181,13 +181,14 @@ __global__ void __launch_bounds__(256) k_tc_prep_centres(const float* __restrict
                                                          __half* __restrict__ B16, float* __restrict__ bias,
                                                          unsigned* __restrict__ cmax_bits, int* __restrict__ bad) {
     const int lane = threadIdx.x & 31;
-    const long long w = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
-    if (w >= (long long)U * Mpad) return;
+    const long long nwarps = ((long long)gridDim.x * blockDim.x) >> 5;
+    // a grid that loops over the rows: a warp per row would be a quarter of a million warps of a dozen instructions
+    for (long long w = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5; w < (long long)U * Mpad; w += nwarps) {
     const int u = (int)(w / Mpad), j = (int)(w % Mpad);
     if (j >= M) {
         *reinterpret_cast<uint2*>(B16 + (size_t)w * TC_D + lane * 4) = make_uint2(0u, 0u);
         if (lane == 0) bias[w] = 0.f;
-        return;
+        continue;
     }
     const size_t row = (size_t)u * M + j;
     const float4 v = *reinterpret_cast<const float4*>(C + row * TC_D + lane * 4);
@@ -202,6 +203,7 @@ __global__ void __launch_bounds__(256) k_tc_prep_centres(const float* __restrict
     if (lane == 0) {
         bias[w] = s;
         atomicMax(&cmax_bits[u], __float_as_uint(sqrtf(s)));     // non-negative floats order like their bit patterns
+    }
     }
 }
 
@@ -655,7 +657,11 @@ void launch_assign_tc(const Tables& t, const void* K, long long n, int M, const 
     unsigned long long* pair_count = reinterpret_cast<unsigned long long*>(base + L.pair_count);
     cudaMemsetAsync(pair_count, 0, 8, s);
     const long long cw = (long long)t.U * L.Mpad;
-    k_tc_prep_centres<<<(unsigned)((cw + 7) / 8), 256, 0, s>>>(C, t.U, M, L.Mpad, B16, bias, cmax, bad);
+    {
+        long long pb = (cw + 7) / 8;
+        if (pb > 148LL * 16) pb = 148LL * 16;
+        k_tc_prep_centres<<<(unsigned)pb, 256, 0, s>>>(C, t.U, M, L.Mpad, B16, bias, cmax, bad);
+    }
     float* Bfix = reinterpret_cast<float*>(base + L.bfix);
     float2* scale = reinterpret_cast<float2*>(base + L.scale);
     k_tc_fixed_bias<<<(unsigned)((cw + 255) / 256), 256, 0, s>>>(bias, cmax, reinterpret_cast<const unsigned*>(base + L.knmax), t.U, M,

@@ -315,12 +315,18 @@ __global__ void k_centroid_div_det(float* __restrict__ C, const long long* __res
 }
 
 // c_j = sum_j / count_j; an empty cluster keeps its previous centre.
-__global__ void k_centroid_div(float* __restrict__ C, const float* __restrict__ sums, const int* __restrict__ counts,
-                               long long total, int d) {
-    long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-    if (i >= total) return;
-    int c = counts[i / d];
-    if (c > 0) C[i] = sums[i] / (float)c;
+// (four elements per thread and a grid that loops: d is a multiple of 4, so a vector never straddles two clusters)
+__global__ void __launch_bounds__(256) k_centroid_div(float* __restrict__ C, const float* __restrict__ sums,
+                                                      const int* __restrict__ counts, long long total, int d) {
+    const long long stride = (long long)gridDim.x * blockDim.x * 4;
+    for (long long i = ((long long)blockIdx.x * blockDim.x + threadIdx.x) * 4; i < total; i += stride) {
+        const int c = counts[i / d];
+        if (c > 0) {
+            const float4 v = *reinterpret_cast<const float4*>(sums + i);
+            const float fc = (float)c;
+            *reinterpret_cast<float4*>(C + i) = make_float4(v.x / fc, v.y / fc, v.z / fc, v.w / fc);
+        }
+    }
 }
 
 // ------------------------------------------------------------------ finalize: layout
@@ -610,7 +616,11 @@ static void update_t(const Tables& t, const void* K, long long n, int M, const i
         return;
     }
     k_update_sums<KV, HD><<<(unsigned)blocks, 256, 0, s>>>((const KV*)K, total, (int)n, M, assign, b.sums, b.counts);
-    k_centroid_div<<<(unsigned)((cd + 255) / 256), 256, 0, s>>>(b.C, b.sums, b.counts, cd, HD);
+    {
+        long long db = (cd / 4 + 255) / 256;
+        if (db > 148LL * 16) db = 148LL * 16;
+        k_centroid_div<<<(unsigned)db, 256, 0, s>>>(b.C, b.sums, b.counts, cd, HD);
+    }
     (*launches) += 2;
 }
 
