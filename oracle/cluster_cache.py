@@ -36,7 +36,11 @@ def pages(n: int) -> int:
 
 
 class ClusterCacheModel:
-    def __init__(self, frames: int):
+    def __init__(self, frames: int, order: str = "small-first"):
+        # order "lru" is a comparison policy only (void copies, then least recently used, whatever the size): it shows
+        # what Section 6.2's first principle buys on a given stream; the library implements "small-first"
+        assert order in ("small-first", "lru")
+        self.order = order
         self.frames = frames
         self.free = frames
         self.copies: Dict[int, dict] = {}       # id -> {"n": size at copy time, "ver": splits seen then, "last": turn}
@@ -85,7 +89,10 @@ class ClusterCacheModel:
                     cls = 1
                 else:
                     cls = 2
-                key = (cls, -pages(cp["n"]), cp["last"], j)
+                if self.order == "lru":
+                    key = (0 if cls == 0 else 1, 0, cp["last"], j)
+                else:
+                    key = (cls, -pages(cp["n"]), cp["last"], j)
                 if best is None or key < best:
                     best = key
             if best is None:

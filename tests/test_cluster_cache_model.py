@@ -98,3 +98,38 @@ def test_selected_clusters_are_never_evicted_and_too_small_a_cache_fails():
     assert sorted(m.copies) == [0, 2]
     with pytest.raises(CacheTooSmall):
         m.retrieve([0, 1, 2], size)         # 2 + 2 + 1 pages cannot fit 4 frames
+
+
+def test_small_first_keeps_more_clusters_cached_than_plain_lru_on_a_decode_stream():
+    """Section 6.2, principle 1, on a synthetic decode stream followed by the oracle (config 4's recipe at a reduced
+    size): evicting large clusters first gives more cluster hits than least-recently-used order at the same cache
+    size, for about the same number of pages copied (a large cluster costs more to bring back)."""
+    import numpy as np
+    import oracle as O
+    from gen import CONFIGS, UnitStream, make_decode_chunk, make_prefill
+    cfg = CONFIGS[4].scaled(n_prefill=2048, steps=150, M0=64, max_clusters=256, budget=256, T=3)
+    s = [UnitStream(cfg, 0)]
+    K, V = make_prefill(s)
+    q, k, v = make_decode_chunk(s, cfg.steps)
+    o = O.OracleUnit(cfg.d, cfg.G, cfg.max_tokens, cfg.max_clusters, gamma=cfg.split_size_factor, alpha=cfg.split_var_factor,
+                     split_min_size=cfg.split_min_size, split_iters=cfg.split_iters)
+    o.build(K[0].double().numpy(), V[0].double().numpy(), cfg.M0, cfg.T, 1234, unit_index=0, init_mode=O.INIT_RANDOM)
+    frames = 40
+    models = {order: ClusterCacheModel(frames, order) for order in ("small-first", "lru")}
+    for t in range(cfg.steps):
+        _, ids, _ = o.decode_step(q[t, 0].double().numpy(), cfg.budget)
+        sizes = o.counts()
+        for m in models.values():
+            m.retrieve(ids, sizes)
+        o.append(k[t, 0].double().numpy(), v[t, 0].double().numpy())
+        before = o.counts().copy()
+        o.split_check()
+        for j in np.nonzero(o.counts()[: len(before)] < before)[0]:
+            for m in models.values():
+                m.note_split(int(j))
+    hits = {name: m.c["clusters_hit"] + m.c["clusters_refreshed"] for name, m in models.items()}
+    fetched = {name: m.c["pages_fetched"] for name, m in models.items()}
+    print(f"\ncluster hits {hits}, pages copied {fetched}, {frames} frames")
+    assert min(m.c["clusters_evicted"] for m in models.values()) > 100
+    assert hits["small-first"] > 1.1 * hits["lru"]
+    assert abs(fetched["small-first"] - fetched["lru"]) < 0.1 * fetched["lru"]
