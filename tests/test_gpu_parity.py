@@ -317,3 +317,24 @@ def test_two_tier_mode_pool_exports_and_resumes_in_a_single_tier_context():
     assert np.array_equal(ctx.export_state()["tok_cluster"], ctx2.export_state()["tok_cluster"])
     assert ctx.get_status()["error_bits"] == 0 and ctx.get_tier_stats()["clusters_evicted"] > 0
     ctx.destroy(); ctx2.destroy()
+
+
+@pytest.mark.parametrize("budget,cache_pages", [(1, 8), (100000, 200)])
+def test_two_tier_mode_at_the_ends_of_the_budget_range(budget, cache_pages):
+    """Budget 1: every step retrieves its best cluster whole although it alone exceeds the budget, so the cache holds
+    one or two clusters at a time.  A budget above the context: every step retrieves every cluster, the cache is as
+    large as the pool, nothing is ever evicted, and after the first step only appended pages and the pages of split
+    clusters travel.  Outputs, state and cache counters against the oracle and its cache model as in the other runs."""
+    cfg = CONFIGS[3].scaled(n_prefill=400, steps=60, M0=10, max_clusters=128, budget=budget, T=3, new_every=32,
+                            split_size_factor=1.3, split_var_factor=1.3)
+    rep = _run(cfg, [0, 1], cfg.steps, assign_mode=1, cache_pages=cache_pages)
+    ts = rep.tier_stats
+    print(f"[two tiers, budget {budget}] {ts}")
+    assert rep.splits > 0
+    if budget == 1:
+        assert rep.status_bits & P_ST_BUDGET_EXCEEDED and rep.status_bits & (16 | 32 | 64) == 0 and ts["clusters_evicted"] > 0
+    else:
+        assert rep.status_bits == 0 and ts["clusters_evicted"] == 0 and ts["clusters_refreshed"] > 0 and ts["copies_dropped_stale"] > 0
+
+
+P_ST_BUDGET_EXCEEDED = 1
