@@ -329,6 +329,9 @@ static int build_index_impl(dynakv_ctx* c, const void* K, const void* V, int64_t
     ALLOC_B(b.counts, U * M, false);
     ALLOC_B(b.cursor, U * M, false);
     ALLOC_B(b.picks, U * M, false);
+    if (!t.det_sums) {
+        ALLOC_B(b.upd_offset, U * M, false); ALLOC_B(b.upd_cursor, U * M, false); ALLOC_B(b.upd_order, U * (size_t)n, false);
+    }
     if (c->cfg.init_mode == DYNAKV_INIT_KMEANSPP) ALLOC_B(b.D2, U * (size_t)n, false);
     int* assign_buf = nullptr;
     if (c->cfg.trace) { ALLOC_B(c->trace_assign, (size_t)T * U * n, false); }

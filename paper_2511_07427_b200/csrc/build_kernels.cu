@@ -278,6 +278,78 @@ __global__ void __launch_bounds__(256) k_update_sums(const KV* __restrict__ K, l
     }
 }
 
+// Eq. 4 by member lists instead of atomic sums: count the members of every cluster, lay the key indices out cluster by
+// cluster (a counting sort of the assignment), and let one warp per cluster add its members' rows in registers and
+// write the new centre.  The keys are read once, as whole rows; the only atomics are the two integer ones per key.
+__global__ void __launch_bounds__(256) k_upd_hist(const int* __restrict__ assign, long long n_total, int n, int M,
+                                                   int* __restrict__ counts) {
+    const long long stride = (long long)gridDim.x * blockDim.x;
+    for (long long w = (long long)blockIdx.x * blockDim.x + threadIdx.x; w < n_total; w += stride) {
+        const int j = assign[w];
+        if (j >= 0 && j < M) atomicAdd(&counts[(w / n) * M + j], 1);
+    }
+}
+// One block per unit: exclusive prefix of the counts.
+__global__ void __launch_bounds__(1024) k_upd_scan(const int* __restrict__ counts, int M, int* __restrict__ offset,
+                                                    int* __restrict__ cursor) {
+    __shared__ int sh[33];
+    const int u = blockIdx.x;
+    int run = 0;
+    for (int base = 0; base < M; base += 1024) {
+        const int j = base + threadIdx.x;
+        const int c = j < M ? counts[(size_t)u * M + j] : 0;
+        int tot;
+        const int at = run + block_scan_excl(c, sh, &tot);
+        if (j < M) { offset[(size_t)u * M + j] = at; cursor[(size_t)u * M + j] = at; }
+        run += tot;
+        __syncthreads();
+    }
+}
+__global__ void __launch_bounds__(256) k_upd_scatter(const int* __restrict__ assign, long long n_total, int n, int M,
+                                                      int* __restrict__ cursor, int* __restrict__ order) {
+    const long long stride = (long long)gridDim.x * blockDim.x;
+    for (long long w = (long long)blockIdx.x * blockDim.x + threadIdx.x; w < n_total; w += stride) {
+        const int j = assign[w];
+        if (j < 0 || j >= M) continue;
+        const long long u = w / n;
+        const int pos = atomicAdd(&cursor[u * M + j], 1);
+        if (pos >= 0 && pos < n) order[u * n + pos] = (int)(w - u * n);
+    }
+}
+// One warp per (unit, cluster), the grid looping: the members' rows are added in list order, 4 elements per lane; an
+// empty cluster keeps its centre.
+template <typename KV, int HD>
+__global__ void __launch_bounds__(256) k_upd_reduce(const KV* __restrict__ K, int U, int n, int M,
+                                                     const int* __restrict__ counts, const int* __restrict__ offset,
+                                                     const int* __restrict__ order, float* __restrict__ C) {
+    const int lane = threadIdx.x & 31;
+    const long long nwarps = ((long long)gridDim.x * blockDim.x) >> 5;
+    for (long long w = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5; w < (long long)U * M; w += nwarps) {
+        const int u = (int)(w / M);
+        const int c = counts[w];
+        if (c <= 0) continue;
+        const int* ord = order + (size_t)u * n + offset[w];
+        const KV* Ku = K + (size_t)u * n * HD;
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int m0 = 0; m0 < c; m0 += 32) {
+            const int mine = (m0 + lane < c) ? ord[m0 + lane] : 0;         // 32 member indices with one load
+            const int rows = min(32, c - m0);
+#pragma unroll 8
+            for (int r = 0; r < rows; r++) {
+                const int i = __shfl_sync(0xffffffffu, mine, r);
+                if (lane * 4 < HD) {
+                    const float4 v = ld4(Ku + (size_t)i * HD, lane * 4);
+                    acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+                }
+            }
+        }
+        if (lane * 4 < HD) {
+            const float fc = (float)c;
+            *reinterpret_cast<float4*>(C + (size_t)w * HD + lane * 4) = make_float4(acc.x / fc, acc.y / fc, acc.z / fc, acc.w / fc);
+        }
+    }
+}
+
 // The same with sums that do not depend on the order of arrival: every element is rounded to a multiple of 2^-24 and
 // added as a 64-bit integer.  Elements of 2^18 or more are clamped and reported.
 constexpr float DET_SCALE = 16777216.f;     // 2^24
@@ -603,6 +675,18 @@ template <typename KV, int HD>
 static void update_t(const Tables& t, const void* K, long long n, int M, const int* assign, const BuildScratch& b,
                      cudaStream_t s, long long* launches) {
     long long total = (long long)t.U * n;
+    if (!t.det_sums && b.upd_order && b.upd_offset && b.upd_cursor) {
+        cudaMemsetAsync(b.counts, 0, sizeof(int) * (size_t)t.U * M, s);
+        const unsigned gb = (unsigned)((total + 255) / 256 < 148LL * 16 ? (total + 255) / 256 : 148LL * 16);
+        k_upd_hist<<<gb, 256, 0, s>>>(assign, total, (int)n, M, b.counts);
+        k_upd_scan<<<t.U, 1024, 0, s>>>(b.counts, M, b.upd_offset, b.upd_cursor);
+        k_upd_scatter<<<gb, 256, 0, s>>>(assign, total, (int)n, M, b.upd_cursor, b.upd_order);
+        const long long cw = (long long)t.U * M;
+        const unsigned rb = (unsigned)((cw + 7) / 8 < 148LL * 16 ? (cw + 7) / 8 : 148LL * 16);
+        k_upd_reduce<KV, HD><<<rb, 256, 0, s>>>((const KV*)K, t.U, (int)n, M, b.counts, b.upd_offset, b.upd_order, b.C);
+        (*launches) += 4;
+        return;
+    }
     cudaMemsetAsync(b.sums, 0, sizeof(float) * (size_t)t.U * M * HD * (t.det_sums ? 2 : 1), s);
     cudaMemsetAsync(b.counts, 0, sizeof(int) * (size_t)t.U * M, s);
     long long blocks = (total + 7) / 8;

@@ -223,6 +223,10 @@ struct BuildScratch {
     float* D2;           // [U][n] k-means++ distances
     int* picks;          // [U][M]
     int* cursor;         // [U][M]
+    // centroid update by member lists (optional: all three or none)
+    int* upd_offset;     // [U][M] first position of the cluster's members in upd_order
+    int* upd_cursor;     // [U][M] next free position while the lists are filled
+    int* upd_order;      // [U][n] key indices (inside the unit), cluster by cluster
 };
 
 void launch_init_centres(const Tables& t, const void* K, long long n, int M, unsigned long long seed,
