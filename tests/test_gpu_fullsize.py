@@ -20,8 +20,12 @@ DIRECT_STEPS = 3
 # config 3 (1K prefill, drifting keys, 64 clusters to start with) runs 200 loop iterations: its clusters split all the time
 # (the last case is config 4 with its rows in FP8 storage: the oracle is handed the rows as the library keeps them)
 @pytest.mark.parametrize("cid,SAMPLED,GRAPH_STEPS,kv", [(4, [0, 101, 255], 13, ""), (2, [0, 77, 255], 13, ""), (3, [0, 130, 255], 200, ""),
-                                                       (5, [0, 900, 1791], 13, ""), (4, [3, 128, 250], 13, "fp8")])
+                                                       (5, [0, 900, 1791], 13, ""), (4, [3, 128, 250], 13, "fp8"),
+                                                       (4, [5, 99, 254], 13, "tier")])
 def test_full_size_sampled_units(cid, SAMPLED, GRAPH_STEPS, kv):
+    # ("tier": config 4 in the two-tier mode -- the 14 GB page pool in pinned host memory, 256 frames per unit in HBM)
+    tier = kv == "tier"
+    kv = "" if tier else kv
     cfg = CONFIGS[cid] if not kv else CONFIGS[cid].scaled(kv_dtype=kv)
     rows = lambda x: stored(x.cpu(), cfg)
     U, n = cfg.U, cfg.n_prefill
@@ -30,7 +34,7 @@ def test_full_size_sampled_units(cid, SAMPLED, GRAPH_STEPS, kv):
         streams = [UnitStream(cfg, u, device="cuda") for u in range(U)]
         K, V = make_prefill(streams)
         q, k, v = make_decode_chunk(streams, DIRECT_STEPS + GRAPH_STEPS)
-        ctx = make_ctx(cfg, U, trace=0, assign_mode=0)
+        ctx = make_ctx(cfg, U, trace=0, assign_mode=0, cache_pages=256 if tier else 0)
         ctx.build_index(K, V, cfg.M0, 1234)
         st = ctx.export_state()
         rep = ParityReport()
@@ -84,8 +88,11 @@ def test_full_size_sampled_units(cid, SAMPLED, GRAPH_STEPS, kv):
                 o.split_check()
         for u in SAMPLED:
             check_state(oracles[u], st, u, rep, f"after the graph loop, unit {u}")
-        assert status["error_bits"] & (P.ST_INTERNAL | P.ST_PAGE_POOL | P.ST_MAX_TOKENS) == 0
+        assert status["error_bits"] & (P.ST_INTERNAL | P.ST_PAGE_POOL | P.ST_MAX_TOKENS | P.ST_TIER_CACHE | P.ST_BOUNDS) == 0
         assert status["n_splits"] > 0
+        if tier:
+            ts = ctx.get_tier_stats()
+            assert ts["clusters_evicted"] > 0 and ts["clusters_hit"] > 0 and ts["frames_total"] == 256 * U
         # ---- properties that must hold for EVERY unit, sampled or not (Eq. 3 and Eq. 4 on the final state): every token
         # in exactly one live cluster, sizes equal to the membership counts, representatives equal to the member means,
         # M2 equal to the members' squared distances to them
