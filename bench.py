@@ -488,8 +488,12 @@ def run_ours(args, cfg):
         tier["pool_pages_per_unit_in_use"] = status["pages_in_use"] / U
         n_decode = max(pos, 1)
         tier["pages_fetched_per_step"] = tier["pages_fetched"] / n_decode
-        page_bytes = 2 * 32 * (cfg.d * {"f32": 4, "bf16": 2, "fp8": 1}[cfg.kv_dtype] + (1 if cfg.kv_dtype == "fp8" else 0))    # K and V
-        tier["host_to_device_mb_per_step"] = tier["pages_fetched"] * page_bytes / n_decode / 1e6
+        # K and V rows that travelled (of a page only the rows that hold entries; in FP8 storage also the 64 scale
+        # exponents of every page touched)
+        row_bytes = 2 * cfg.d * {"f32": 4, "bf16": 2, "fp8": 1}[cfg.kv_dtype]
+        moved = tier["rows_fetched"] * row_bytes + (tier["pages_fetched"] * 64 if cfg.kv_dtype == "fp8" else 0)
+        tier["host_to_device_mb_per_step"] = moved / n_decode / 1e6
+        tier["rows_fetched_per_step"] = tier["rows_fetched"] / n_decode
         looked_up = tier["clusters_hit"] + tier["clusters_refreshed"] + tier["clusters_fetched"]
         tier["cluster_hit_rate"] = (tier["clusters_hit"] + tier["clusters_refreshed"]) / max(looked_up, 1)
     ctx.destroy()

@@ -96,7 +96,7 @@ typedef struct dynakv_config {
                                   Each step's selected clusters are brought into the cache whole before the attention
                                   reads them, replacing whole clusters (Section 6.2); results are those of tier = 0.
                                   Any kv_dtype (FP8: pool and frames hold the one-byte rows and their exponents)      */
-    int32_t cache_pages;       /* tier = 1: 32-token page frames per unit in device memory; must hold the clusters of
+    int32_t cache_pages;       /* tier = 1: 32-token page frames per unit in device memory (< 2^20); must hold the clusters of
                                   any one step (about token_budget / 32 plus one per selected cluster)                */
 } dynakv_config;
 
@@ -136,7 +136,7 @@ typedef struct dynakv_status {
  * the pages from its former last page on are copied) or fetched (all its pages are copied); evicted counts clusters
  * that made room, dropped_stale copies made void by a split. */
 typedef struct dynakv_tier_stats {
-    int64_t pages_fetched;
+    int64_t pages_fetched;     /* pages touched by a copy (whole or in part) */
     int64_t clusters_hit;
     int64_t clusters_fetched;
     int64_t clusters_refreshed;
@@ -144,6 +144,8 @@ typedef struct dynakv_tier_stats {
     int64_t copies_dropped_stale;
     int64_t frames_in_use;     /* now, summed over units */
     int64_t frames_total;      /* n_units * cache_pages  */
+    int64_t rows_fetched;      /* K/V rows copied: of a page only the rows that hold entries, of a refreshed cluster's
+                                  former last page only the rows appended since the copy */
 } dynakv_tier_stats;
 
 /* Create a context on the current CUDA device; all later work runs on `cuda_stream`

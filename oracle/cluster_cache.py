@@ -9,7 +9,8 @@ so that the counters of an implementation can be compared with it exactly:
   * `retrieve(selected, size)` is one decode step: every selected cluster is
       - a HIT when a copy exists that was made after the cluster's last split and at its present size;
       - GROWN when such a copy exists but entries were appended since: the page that was the last one at copy time is
-        copied again if it was not full, and one frame is taken per page the cluster has gained;
+        copied again if it was not full (only the rows added since), and one frame is taken per page the cluster has
+        gained;
       - MISSING otherwise: a copy from before a split is dropped first, then every page is copied into new frames;
   * when the free frames do not cover what the step needs, whole clusters NOT selected in this step are evicted until
     they do, in this order: copies made void by a split; then clusters unchanged since they were copied -- more pages
@@ -47,7 +48,7 @@ class ClusterCacheModel:
         self.ver: Dict[int, int] = {}
         self.clock = 0
         self.c = {"pages_fetched": 0, "clusters_hit": 0, "clusters_fetched": 0, "clusters_refreshed": 0,
-                  "clusters_evicted": 0, "copies_dropped_stale": 0}
+                  "clusters_evicted": 0, "copies_dropped_stale": 0, "rows_fetched": 0}
 
     def note_split(self, j: int) -> None:
         self.ver[j] = self.ver.get(j, 0) + 1
@@ -105,12 +106,14 @@ class ClusterCacheModel:
             extra = pages(n) - pages(cp["n"])
             self.c["pages_fetched"] += extra + (1 if cp["n"] % PAGE != 0 else 0)
             self.c["clusters_refreshed"] += 1
+            self.c["rows_fetched"] += n - cp["n"]         # only the entries appended since the copy travel
             self.free -= extra
             cp["n"] = n
         for j in missing:
             n = int(size[j])
             self.c["pages_fetched"] += pages(n)
             self.c["clusters_fetched"] += 1
+            self.c["rows_fetched"] += n
             self.free -= pages(n)
             self.copies[j] = {"n": n, "ver": self.ver.get(j, 0), "last": self.clock}
 

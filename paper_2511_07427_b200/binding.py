@@ -49,7 +49,8 @@ class _Status(C.Structure):
 
 class _TierStats(C.Structure):
     _fields_ = [(k, C.c_int64) for k in ("pages_fetched", "clusters_hit", "clusters_fetched", "clusters_refreshed",
-                                         "clusters_evicted", "copies_dropped_stale", "frames_in_use", "frames_total")]
+                                         "clusters_evicted", "copies_dropped_stale", "frames_in_use", "frames_total",
+                                         "rows_fetched")]
 
 
 KERNEL_CLASSES = ["init", "assign", "update", "finalize", "select", "attn", "combine", "append", "split", "front", "tier"]

@@ -147,7 +147,7 @@ extern "C" int dynakv_create(const dynakv_config* cfg, void* cuda_stream, dynakv
     if (cfg->update_mode == DYNAKV_MODE_DELAYED && cfg->buf_max < 1) return DYNAKV_ERR_ARG;
     if (cfg->update_mode == DYNAKV_MODE_LOCAL && cfg->local_max < 2) return DYNAKV_ERR_ARG;
     if (cfg->tier != 0 && cfg->tier != 1) return DYNAKV_ERR_ARG;
-    if (cfg->tier && (cfg->cache_pages < 1 || cfg->n_units > 65535)) return DYNAKV_ERR_ARG;
+    if (cfg->tier && (cfg->cache_pages < 1 || cfg->cache_pages >= (1 << 20) || cfg->n_units > 65535)) return DYNAKV_ERR_ARG;
     dynakv_ctx* c = new (std::nothrow) dynakv_ctx();
     if (!c) return DYNAKV_ERR_NOMEM;
     c->cfg = *cfg;
@@ -854,6 +854,7 @@ extern "C" int dynakv_get_tier_stats(dynakv_ctx* c, dynakv_tier_stats* out) {
     out->clusters_refreshed = (int64_t)cnt[TIER_REFRESHED];
     out->clusters_evicted = (int64_t)cnt[TIER_EVICTED];
     out->copies_dropped_stale = (int64_t)cnt[TIER_STALE];
+    out->rows_fetched = (int64_t)cnt[TIER_ROWS];
     out->frames_total = (int64_t)c->t.U * c->ts.Fc;
     out->frames_in_use = out->frames_total;
     for (int f : free_cnt) out->frames_in_use -= f;

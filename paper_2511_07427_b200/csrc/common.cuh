@@ -277,7 +277,7 @@ void launch_append_split(const Tables& t, float gamma, int var_enabled, int min_
 
 // Two-tier mode: the page pool (Tables::kpages / vpages) is pinned host memory and this is the HBM cache of page
 // frames over it, per unit, filled and replaced in whole clusters.
-enum { TIER_PAGES_FETCHED = 0, TIER_HITS = 1, TIER_FETCHED = 2, TIER_REFRESHED = 3, TIER_EVICTED = 4, TIER_STALE = 5,
+enum { TIER_PAGES_FETCHED = 0, TIER_HITS = 1, TIER_FETCHED = 2, TIER_REFRESHED = 3, TIER_EVICTED = 4, TIER_STALE = 5, TIER_ROWS = 6,
        TIER_COUNTERS = 8 };
 struct TierState {
     int Fc;                          // frames per unit
@@ -290,7 +290,7 @@ struct TierState {
     int* frame_page; int* frame_next;   // [U][Fc] page the frame copies; next frame of the same cluster's copy
     int* fr_free; int* fr_free_cnt;  // [U][Fc] stack of free frames, [U] its height
     int* miss_list;                  // [U][Mmax] selected clusters that need frames this turn
-    int2* jobs; int* n_jobs;         // [U][Fc + Mmax] (page, frame) copies of this turn, [U] how many
+    int2* jobs; int* n_jobs;         // [U][Fc + Mmax] copies of this turn: (page, frame | first row << 20 | rows - 1 << 25), [U] how many
     unsigned int* clock;             // [U] resolve turns so far
     unsigned long long* counters;    // [TIER_COUNTERS]
 };

@@ -129,14 +129,22 @@ __global__ void __launch_bounds__(256) k_tier_resolve(Tables t, TierState ts) {
             if (lane != 0) continue;
             const int e = miss[m], j = e & ~TIER_GROWN;
             const int n = cl_n[j];
-            int page, prev, todo;
+            // a job copies rows [row0, row0 + rows) of a page into the same rows of a frame: only rows that hold entries,
+            // and of a grown cluster's former last page only the ones added since
+            auto job = [&](int pg, int f, int row0, int rows) {
+                jobs[atomicAdd(&s_njobs, 1)] = make_int2(pg, f | (row0 << 20) | ((rows - 1) << 25));
+                atomicAdd(&s_cnt[TIER_PAGES_FETCHED], 1);
+                atomicAdd(&s_cnt[TIER_ROWS], rows);
+            };
+            int page, prev, todo, pk;          // pk: number of the next page inside the cluster
             if (e & TIER_GROWN) {
                 const int sn = snap[4 * j], old_tail = snap[4 * j + 3];
-                if (sn % PAGE != 0 && old_tail >= 0 && old_tail < P) { jobs[atomicAdd(&s_njobs, 1)] = make_int2(old_tail, page_frame[old_tail]); atomicAdd(&s_cnt[TIER_PAGES_FETCHED], 1); }
-                page = (old_tail >= 0 && old_tail < P) ? pnext[old_tail] : -1; prev = fr_tail[j]; todo = pages_of(n) - pages_of(sn);
+                pk = pages_of(sn);
+                if (sn % PAGE != 0 && old_tail >= 0 && old_tail < P) job(old_tail, page_frame[old_tail], sn % PAGE, min(n, pk * PAGE) - sn);
+                page = (old_tail >= 0 && old_tail < P) ? pnext[old_tail] : -1; prev = fr_tail[j]; todo = pages_of(n) - pk;
                 atomicAdd(&s_cnt[TIER_REFRESHED], 1);
             } else {
-                page = cl_head[j]; prev = -1; todo = pages_of(n);
+                page = cl_head[j]; prev = -1; todo = pages_of(n); pk = 0;
                 atomicAdd(&s_cnt[TIER_FETCHED], 1);
             }
             for (int k = 0; k < todo && page >= 0 && page < P; k++) {
@@ -149,8 +157,7 @@ __global__ void __launch_bounds__(256) k_tier_resolve(Tables t, TierState ts) {
                 prev = f;
                 frame_page[f] = page;
                 page_frame[page] = f;
-                jobs[atomicAdd(&s_njobs, 1)] = make_int2(page, f);
-                atomicAdd(&s_cnt[TIER_PAGES_FETCHED], 1);
+                job(page, f, 0, min(PAGE, n - (pk + k) * PAGE));
                 page = pnext[page];
             }
             fr_tail[j] = prev;
@@ -180,23 +187,25 @@ __global__ void __launch_bounds__(256) k_tier_resolve(Tables t, TierState ts) {
     }
 }
 
-// Copies the listed pages, K and V, from the pool (host memory) into their frames; in FP8 mode the one-byte rows and
-// the 32 scale exponents of each page.
+// Copies the listed rows, K and V, from the pool (host memory) into the same rows of their frames; in FP8 mode the
+// one-byte rows and the page's 32 scale exponents.
 __global__ void __launch_bounds__(256) k_tier_fetch(Tables t, TierState ts, int row_bytes) {
     const int u = blockIdx.y;
     const int nj = ts.n_jobs[u];
     const size_t page_bytes = (size_t)PAGE * row_bytes;
-    const int v16 = (int)(page_bytes / 16);
     const char* kpool = t.fp8 ? (const char*)t.k8 : (const char*)t.kpages;
     const char* vpool = t.fp8 ? (const char*)t.v8 : (const char*)t.vpages;
     for (int jb = blockIdx.x; jb < nj; jb += gridDim.x) {
         const int2 job = ts.jobs[(size_t)u * (ts.Fc + t.max_clusters) + jb];
-        if (job.x < 0 || job.x >= t.P || job.y < 0 || job.y >= ts.Fc) continue;
-        const size_t src = (size_t)u * t.P + job.x, dst = (size_t)u * ts.Fc + job.y;
-        const uint4* ks = reinterpret_cast<const uint4*>(kpool + src * page_bytes);
-        const uint4* vs = reinterpret_cast<const uint4*>(vpool + src * page_bytes);
-        uint4* kd = reinterpret_cast<uint4*>((char*)ts.kcache + dst * page_bytes);
-        uint4* vd = reinterpret_cast<uint4*>((char*)ts.vcache + dst * page_bytes);
+        const int f = job.y & 0xFFFFF, row0 = (job.y >> 20) & 31, rows = ((job.y >> 25) & 31) + 1;
+        if (job.x < 0 || job.x >= t.P || f >= ts.Fc || row0 + rows > PAGE) continue;
+        const size_t src = (size_t)u * t.P + job.x, dst = (size_t)u * ts.Fc + f;
+        const size_t off = (size_t)row0 * row_bytes;
+        const int v16 = rows * row_bytes / 16;
+        const uint4* ks = reinterpret_cast<const uint4*>(kpool + src * page_bytes + off);
+        const uint4* vs = reinterpret_cast<const uint4*>(vpool + src * page_bytes + off);
+        uint4* kd = reinterpret_cast<uint4*>((char*)ts.kcache + dst * page_bytes + off);
+        uint4* vd = reinterpret_cast<uint4*>((char*)ts.vcache + dst * page_bytes + off);
         for (int i = threadIdx.x; i < v16; i += 256) { kd[i] = ks[i]; vd[i] = vs[i]; }
         if (t.fp8 && threadIdx.x < 2 * (PAGE / 16)) {
             const int i = threadIdx.x % (PAGE / 16);

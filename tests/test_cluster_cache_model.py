@@ -15,8 +15,9 @@ def test_first_use_fetches_whole_clusters_and_a_repeat_hits():
     size = {0: 40, 1: 10, 2: 64}            # 2 + 1 + 2 pages
     m.retrieve([0, 1, 2], size)
     assert m.c["pages_fetched"] == 5 and m.c["clusters_fetched"] == 3 and m.frames_in_use == 5
+    assert m.c["rows_fetched"] == 40 + 10 + 64          # only rows that hold entries travel
     m.retrieve([2, 0], size)
-    assert m.c["clusters_hit"] == 2 and m.c["pages_fetched"] == 5 and m.c["clusters_evicted"] == 0
+    assert m.c["clusters_hit"] == 2 and m.c["pages_fetched"] == 5 and m.c["clusters_evicted"] == 0 and m.c["rows_fetched"] == 114
 
 
 def test_an_appended_cluster_is_refreshed_from_its_former_last_page_on():
@@ -35,6 +36,7 @@ def test_an_appended_cluster_is_refreshed_from_its_former_last_page_on():
     size[0] = 130                           # 70 -> 130: page 3 again (6 of 32 rows then) and pages 4, 5
     m.retrieve([0], size)
     assert m.c["pages_fetched"] == 8 and m.frames_in_use == 5 and m.c["clusters_fetched"] == 1
+    assert m.c["rows_fetched"] == 40 + 1 + 23 + 6 + 60        # every entry travelled exactly once
 
 
 def test_a_split_voids_the_copy_even_when_the_size_comes_back():
