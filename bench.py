@@ -542,7 +542,8 @@ def main():
                     help="build with correlation-aware placement from this many reference queries (0: clusters in id order)")
     ap.add_argument("--tier", type=int, default=0,
                     help="two-tier mode: the page pool in pinned host memory and this many 32-token page frames per unit in HBM")
-    ap.add_argument("--e2e-steps", type=int, default=160)
+    ap.add_argument("--e2e-steps", type=int, default=272,
+                    help="steps of the end-to-end legs: half one step per call, half one host-array loop call (as long as a default timed region)")
     ap.add_argument("--profile-steps", type=int, default=64)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--budget", type=int, default=0, help="override the config's token budget (tuning aid)")
