@@ -226,7 +226,8 @@ def test_correlation_aware_placement_lengthens_contiguous_access():
 
 @pytest.mark.parametrize("cid,cache_pages,attn_mode,variant", [(3, 20, 0, ""), (2, 24, 0, ""), (2, 48, 1, ""), (1, 24, 0, ""),
                                                                (30, 96, 0, ""), (30, 96, 0, "fp8"), (2, 24, 1, "fp8"),
-                                                               (30, 96, 0, "delayed"), (2, 24, 0, "placed")])
+                                                               (30, 96, 0, "delayed"), (2, 24, 0, "placed"),
+                                                               (3, 20, 0, "static"), (30, 24, 0, "local")])
 def test_two_tier_mode(cid, cache_pages, attn_mode, variant):
     """The two-tier mode (Section 6; Section 7 on CPU-GPU platforms): the page pool in pinned host memory, a cache of
     cache_pages frames per unit in device memory, whole clusters brought in and replaced (Section 6.2).  The cache is
@@ -237,7 +238,8 @@ def test_two_tier_mode(cid, cache_pages, attn_mode, variant):
     config 1 stores fp32 rows; attn_mode 1 reads the frames with the plain kernel; variant "fp8" keeps pool and frames in
     the one-byte storage (rows and scale exponents travel together); "delayed" adds Algorithm 1's delayed split, whose
     splits then fall on clusters the step has just brought into the cache; "placed" builds the pool with the
-    correlation-aware placement first."""
+    correlation-aware placement first; "static" and "local" are the two baseline update modes (no splits; new
+    entries clustered among themselves)."""
     if cid == 30:
         cfg = CONFIGS[3].scaled(n_prefill=500, steps=160, M0=12, max_clusters=256, budget=300, T=4, new_every=32,
                                 split_size_factor=1.3, split_var_factor=1.3)
@@ -251,13 +253,15 @@ def test_two_tier_mode(cid, cache_pages, attn_mode, variant):
         cfg = cfg.scaled(kv_dtype="fp8")
     elif variant == "delayed":
         cfg = cfg.scaled(update_mode="delayed", buf_max=6)
+    elif variant in ("static", "local"):
+        cfg = cfg.scaled(update_mode=variant, local_max=24)
     rep = _run(cfg, [0] if cid == 1 else [0, 1, 2], cfg.steps, assign_mode=1, attn_mode=attn_mode, cache_pages=cache_pages,
                placement_queries=16 if variant == "placed" else 0)
     ts = rep.tier_stats
     print(f"[two tiers, {cache_pages} frames] {ts}")
     assert rep.status_bits == 0
     assert ts["clusters_hit"] > 0 and ts["clusters_refreshed"] > 0 and ts["clusters_evicted"] > 0
-    if cid in (3, 30):
+    if cid in (3, 30) and variant != "static":
         assert rep.splits > 0 and ts["copies_dropped_stale"] > 0
 
 
