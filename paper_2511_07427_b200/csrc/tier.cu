@@ -221,6 +221,10 @@ void launch_tier_init(const Tables& t, const TierState& ts, cudaStream_t s, long
 }
 
 void launch_tier_resolve_fetch(const Tables& t, const TierState& ts, cudaStream_t s, long long* launches) {
+    // Ordinary launches on purpose.  The kernels of a step are otherwise chained by programmatic dependent launch, and
+    // the attention kernel lets its successor -- the kernel that appends -- move in as soon as it has started itself.
+    // If these two did the same, the append of the step could run beside k_tier_resolve, which reads the very sizes and
+    // page chains the append changes.  As full launches they finish before the attention kernel can start.
     k_tier_resolve<<<t.U, 256, 0, s>>>(t, ts);
     const int row_bytes = t.fp8 ? t.d : t.d * (t.kv_dtype == DYNAKV_F32 ? 4 : 2);
     k_tier_fetch<<<dim3(16, t.U), 256, 0, s>>>(t, ts, row_bytes);
