@@ -380,7 +380,7 @@ def run_ours(args, cfg):
     attn_bytes = tokens_per_launch * row_bytes + 2 * U * cfg.G * cfg.d * 4
     achieved = attn_bytes / (attn_ms * 1e-3) / 1e9 if attn_ms > 0 else 0.0
     kernels = {k: (v["ms"] / v["launches"] * 1e3 if v["launches"] else None) for k, v in kt.items()
-               if k in ("front", "select", "attn", "combine", "append", "split")}
+               if k in ("front", "select", "attn", "combine", "append", "split", "tier")}
     roofline = {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                 "frac": achieved / peaks["hbm_gbs"],
                 "traffic": (args.attn_traffic_bytes if args.attn_traffic_bytes is not None else
