@@ -133,8 +133,8 @@ typedef struct dynakv_status {
 
 /* Counters of the two-tier mode since dynakv_create, summed over units (dynakv_get_tier_stats):
  * a selected cluster is a hit (its copy in the cache is current), refreshed (it only took appends since it was copied:
- * the pages from its former last page on are copied) or fetched (all its pages are copied); evicted counts clusters
- * that made room, dropped_stale copies made void by a split. */
+ * the rows added since are copied) or fetched (all its rows are copied); evicted counts clusters that made room,
+ * dropped_stale copies made void by a split. */
 typedef struct dynakv_tier_stats {
     int64_t pages_fetched;     /* pages touched by a copy (whole or in part) */
     int64_t clusters_hit;
