@@ -52,7 +52,7 @@ __global__ void __launch_bounds__(256) k_tier_resolve(Tables t, TierState ts) {
     int* fr_free = ts.fr_free + (size_t)u * Fc;
     int* miss = ts.miss_list + (size_t)u * Mx;
     int2* jobs = ts.jobs + (size_t)u * (Fc + Mx);
-    __shared__ int s_nmiss, s_free, s_need, s_fail, s_njobs, s_cnt[TIER_COUNTERS];
+    __shared__ int s_nmiss, s_free, s_need, s_fail, s_njobs, s_victim, s_cnt[TIER_COUNTERS];
     __shared__ unsigned long long s_best[8];
     const unsigned int clock = ts.clock[u] + 1u;
     if (tid == 0) { s_nmiss = 0; s_free = ts.fr_free_cnt[u]; s_need = 0; s_fail = 0; s_njobs = 0; }
@@ -96,17 +96,27 @@ __global__ void __launch_bounds__(256) k_tier_resolve(Tables t, TierState ts) {
         if (lane == 0 && !(e & TIER_GROWN) && fr_head[e] >= 0) { drop(e); atomicAdd(&s_cnt[TIER_STALE], 1); }
     }
     __syncthreads();
-    // ---- cluster-aligned replacement
-    while (s_free < s_need && !s_fail) {
-        unsigned long long best = ~0ull;
-        for (int j = tid; j < Mx; j += 256)
-            if (fr_head[j] >= 0 && lru[j] != clock) {
-                const int sn = snap[4 * j];
-                const unsigned long long cls = (snap[4 * j + 1] != cl_ver[j] || snap[4 * j + 2] != cl_head[j]) ? 0ull : (cl_n[j] == sn ? 1ull : 2ull);
-                const unsigned long long k = (cls << 60) | ((unsigned long long)(0xFFFFF - pages_of(sn)) << 40) |
-                                             ((unsigned long long)(lru[j] & 0xFFFFFFFu) << 12) | (unsigned long long)j;
-                if (k < best) best = k;
-            }
+    // ---- cluster-aligned replacement.  A cluster's eviction key does not change while victims are taken (only the
+    // victim's own copy goes), so every thread keeps the smallest key of the ids it owns (tid, tid + 256, ...) in a
+    // register; an eviction is then one block-wide minimum, the return of the victim's frames by thread 0, and a
+    // rescan by the one thread that owned the victim.
+    auto key_of = [&](int j) -> unsigned long long {
+        if (fr_head[j] < 0 || lru[j] == clock) return ~0ull;           // no copy, or in use by this step
+        const int sn = snap[4 * j];
+        const unsigned long long cls = (snap[4 * j + 1] != cl_ver[j] || snap[4 * j + 2] != cl_head[j]) ? 0ull : (cl_n[j] == sn ? 1ull : 2ull);
+        return (cls << 60) | ((unsigned long long)(0xFFFFF - pages_of(sn)) << 40) |
+               ((unsigned long long)(lru[j] & 0xFFFFFFFu) << 12) | (unsigned long long)j;
+    };
+    unsigned long long mine = ~0ull;
+    // Whether another victim is needed is read by every thread at the same point -- right behind a barrier, before
+    // anything may change the free count again -- and kept in a register: a thread that is late (the one that rescans)
+    // must not find the count already lowered by the hand-out of frames below and go round once more on its own.
+    bool more = s_free < s_need;
+    if (more) {
+        for (int j = tid; j < Mx; j += 256) { const unsigned long long k = key_of(j); if (k < mine) mine = k; }
+    }
+    while (more) {
+        unsigned long long best = mine;
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) { const unsigned long long y = __shfl_xor_sync(0xffffffffu, best, o); if (y < best) best = y; }
         if (lane == 0) s_best[warp] = best;
@@ -117,12 +127,19 @@ __global__ void __launch_bounds__(256) k_tier_resolve(Tables t, TierState ts) {
             if (b == ~0ull) s_fail = 1;                 // nothing left to evict: the cache cannot hold this step's clusters
             else {
                 const int v = (int)(b & 0xFFFull);
+                s_victim = v;
                 s_cnt[(b >> 60) == 0ull ? TIER_STALE : TIER_EVICTED] += 1;
                 drop(v);
             }
         }
         __syncthreads();
+        more = s_free < s_need && !s_fail;
+        if (more && (s_victim & 255) == tid) {          // the victim was one of this thread's ids
+            mine = ~0ull;
+            for (int j = tid; j < Mx; j += 256) { const unsigned long long k = key_of(j); if (k < mine) mine = k; }
+        }
     }
+    __syncthreads();          // nobody hands out frames before every thread has left the loop
     if (!s_fail) {
         // ---- frames and copy jobs (pops only from here on)
         for (int m = warp; m < nmiss; m += 8) {
