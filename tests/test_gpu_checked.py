@@ -20,7 +20,7 @@ def test_parity_and_edge_suites_on_the_bounds_checked_build():
     env = dict(os.environ, DYNAKV_LIBRARY="checked")
     cmd = [sys.executable, "-m", "pytest", "-x", "-q", "-m", "gpu", "-p", "no:cacheprovider",
            os.path.join(ROOT, "tests", "test_gpu_parity.py"), os.path.join(ROOT, "tests", "test_gpu_edge.py")]
-    r = subprocess.run(cmd, cwd=ROOT, env=env, capture_output=True, text=True, timeout=3000)
+    r = subprocess.run(cmd, cwd=ROOT, env=env, capture_output=True, text=True, timeout=800)
     tail = (r.stdout + r.stderr)[-4000:]
     assert r.returncode == 0, tail
     assert " passed" in tail and "failed" not in tail, tail
